@@ -1,0 +1,252 @@
+/*
+ * sgs.h - C interface of the SubGraph-Stationary SubNet inference library for NVIDIA B200.
+ *
+ * The library executes a stream of inference queries, each activating a different SubNet of one
+ * weight-shared SuperNet (paper: "SubGraph Stationary Hardware-Software Inference Co-design",
+ * Sections 2.1, 2.2 and 3.1).  A SubNet is never copied out of the SuperNet: elastic width and
+ * expand ratio select the first K' filters / first C' channels of a stored layer, elastic kernel
+ * selects the centre k x k window of the stored kernel, elastic depth keeps the first d blocks of
+ * a stage.  The weights shared by recent queries (their common SubGraph) are kept on chip instead
+ * of being fetched again from HBM (Section 2.2, Section 4.2 "Persistent Buffer", Section 4.3.1).
+ *
+ * Conventions
+ *   - Every function returns an sgs_status_t (SGS_OK == 0); none throws or aborts.  A text for the
+ *     last failure of a handle is available from sgs_last_error().
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA device memory on the
+ *     device the SuperNet was loaded on (for example torch.Tensor.data_ptr()).
+ *   - Activations are NHWC.  In SGS_BF16 mode inputs are bfloat16 and arithmetic is bf16 x bf16
+ *     with fp32 accumulation; every layer output is rounded to bf16 when it is stored.  In
+ *     SGS_F32 mode everything is fp32.  Logits are always fp32, [batch][n_classes].
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - A handle is not re-entrant: use it from one host thread / one stream at a time.
+ *   - The library needs a CUDA device of compute capability 10.0 and fails with SGS_EUNSUPPORTED
+ *     or SGS_ECUDA otherwise; there is no CPU fallback.
+ */
+#ifndef SGS_H_
+#define SGS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SGS_MAX_STAGES 8
+#define SGS_MAX_BLOCKS 8
+
+typedef struct sgs_supernet sgs_supernet_t; /* opaque; owns all device weight memory */
+
+typedef enum {
+    SGS_OK = 0,
+    SGS_EINVAL = 1,      /* NULL pointer, bad size, bad enum */
+    SGS_ECONFIG = 2,     /* SubNet config outside the SuperNet's elastic sets */
+    SGS_ENOMEM = 3,      /* host or device allocation failed */
+    SGS_ECUDA = 4,       /* a CUDA call failed */
+    SGS_ETIMEOUT = 5,    /* a bounded device-side wait ran out (kernel returned cleanly) */
+    SGS_EUNSUPPORTED = 6 /* shape / device not supported */
+} sgs_status_t;
+
+typedef enum { SGS_F32 = 0, SGS_BF16 = 1 } sgs_dtype_t;
+typedef enum { SGS_TINY = 0, SGS_RESNET = 1, SGS_MBV3 = 2 } sgs_family_t;
+
+/* SuperNet family and maxima.  Only `family` selects behaviour; the other fields are checked
+ * against the family's built-in definition (0 = do not check). */
+typedef struct {
+    int family; /* sgs_family_t */
+    int n_stages;
+    int max_depth[SGS_MAX_STAGES];
+    int base_width[SGS_MAX_STAGES];
+    int stem_width;
+    int n_classes;
+    int max_kernel;
+} sgs_arch_desc_t;
+
+/* Elastic choices of one SubNet (paper Section 2.1).
+ *   depth[s]      blocks kept in stage s: the first depth[s] blocks
+ *   width[0]      stem width multiplier; width[1+s] width multiplier of stage s
+ *   expand[s][b]  expand ratio of block b of stage s
+ *   kernel[s][b]  depthwise kernel size of block b of stage s (MobileNetV3-shaped family)
+ * Fields a family does not use are ignored. */
+typedef struct {
+    int depth[SGS_MAX_STAGES];
+    float width[SGS_MAX_STAGES + 1];
+    float expand[SGS_MAX_STAGES][SGS_MAX_BLOCKS];
+    int kernel[SGS_MAX_STAGES][SGS_MAX_BLOCKS];
+} sgs_subnet_cfg_t;
+
+/* Options of sgs_stream_run. */
+typedef struct {
+    int cache_enabled;  /* 1: keep the SubGraph shared by recent queries resident in L2 */
+    int window_q;       /* the cached SubGraph is re-chosen every window_q queries from the last
+                           window_q SubNets (paper Section 3.3 and Appendix A.1); >= 1 */
+    size_t cache_budget_bytes; /* 0 = the device's persisting-L2 maximum */
+    int use_graphs;     /* 1: replay one captured CUDA graph per distinct (config, batch, res);
+                           ignored on the legacy default stream, which cannot be captured */
+    int record_latency; /* 1: bracket every query with events and fill the latency statistics */
+    int weights_evict_first; /* with the cache off: 1 marks weight loads evict-first, which removes
+                                the reuse the hardware L2 replacement gives for free */
+} sgs_stream_opts_t;
+
+/* Results of sgs_stream_run (all host-side; filled after the stream has been synchronised). */
+typedef struct {
+    int n_queries;
+    double total_ms;        /* device time of the whole stream (events on the given stream) */
+    double queries_per_s;   /* n_queries / total time */
+    double images_per_s;    /* queries_per_s * batch_per_query */
+    double p50_ms, p99_ms, mean_ms; /* per query; 0 unless record_latency */
+    double useful_flops;    /* 2*M*K'*C'*k*k summed over the sliced layers of all queries */
+    double weight_bytes;    /* stored-weight bytes the SubNets touch, summed over queries */
+    double hbm_weight_bytes;/* analytic: bytes of SN_t not inside the cached SubGraph G_t */
+    double hit_ratio;       /* mean over t of ||SN_t ∩ G_t||_2 / ||SN_t||_2 (paper Appendix A.4) */
+    double byte_hit_ratio;  /* 1 - hbm_weight_bytes / weight_bytes */
+    long long kernel_launches;
+    int plan_hits, plan_misses;
+    int cache_updates;      /* how many times the cached SubGraph changed */
+} sgs_stream_stats_t;
+
+/* State of the SubGraph cache. */
+typedef struct {
+    int enabled;
+    int window_q;
+    size_t budget_bytes;           /* after clamping to what the device offers */
+    size_t l2_bytes;               /* cudaDevAttrL2CacheSize */
+    size_t persisting_l2_max;      /* cudaDevAttrMaxPersistingL2CacheSize */
+    size_t access_window_max;      /* cudaDevAttrMaxAccessPolicyWindowSize */
+    size_t cached_subgraph_bytes;  /* weight bytes of the SubGraph currently marked resident */
+    size_t supernet_bytes;         /* device bytes of all stored weights */
+    size_t device_bytes_allocated; /* every device byte the handle owns (weights + workspaces) */
+} sgs_cache_stats_t;
+
+/*
+ * sgs_supernet_load - build a SuperNet on `device` from a host blob (Section 2.1: one stored set of
+ * weights contains every SubNet).
+ *   arch       family (and optional maxima to cross-check)
+ *   host_blob  host pointer, `nbytes` bytes, in the self-describing record format written by the
+ *              workload generator: header of 8 uint32 (magic 'SGSB', version 1, family, n_records,
+ *              seed, 0, 0, 0); per stored layer a record header of 8 uint32 (kind 0 conv / 1 depthwise
+ *              / 2 linear, K_max, C_max, R, S, has_bn, has_bias, 0) followed by fp32
+ *              weight[K_max][C_max][R][S], then gamma, beta, mean, var [K_max] if has_bn, then
+ *              bias[K_max] if has_bias.  The blob is copied; the caller keeps ownership.
+ *   compute_dtype  SGS_BF16 (weights re-laid out as bf16 [K][R][S][C]) or SGS_F32
+ *   out        receives the handle; free with sgs_supernet_free
+ * Batch norm is folded into a per-filter scale and shift at load.
+ * Errors: SGS_EINVAL (NULL, bad header, blob does not match the family), SGS_ENOMEM, SGS_ECUDA,
+ * SGS_EUNSUPPORTED (no sm_100 device).
+ */
+sgs_status_t sgs_supernet_load(const sgs_arch_desc_t *arch, const void *host_blob, size_t nbytes,
+                               sgs_dtype_t compute_dtype, int device, sgs_supernet_t **out);
+
+/* Check a config against the SuperNet's elastic sets (Section 2.1).  SGS_OK or SGS_ECONFIG. */
+sgs_status_t sgs_subnet_validate(const sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg);
+
+/*
+ * sgs_subnet_run - one query: inference of the SubNet `cfg` on `batch` images (Section 3.1: the
+ * accelerator performs inference of the query using the selected SubNet).
+ *   d_input   device pointer, [batch][res][res][3] NHWC, compute dtype, caller-owned, read only
+ *   d_logits  device pointer, [batch][n_classes] fp32, caller-owned, written
+ * Asynchronous on `cuda_stream`.  Invalid config -> SGS_ECONFIG before anything is launched.
+ * No sliced copy of any weight is made; the only device memory that may grow is the activation
+ * workspace (and the split-reduction scratch) on the first use of a larger (batch, res).
+ */
+sgs_status_t sgs_subnet_run(sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, const void *d_input, int batch,
+                            int res, void *d_logits, void *cuda_stream);
+
+/*
+ * sgs_stream_run - a stream of queries (Sections 2.1 and 3.1), query t using cfgs[t] on
+ * inputs[t] = d_inputs + t*batch_per_query*res*res*3 elements, writing logits[t] =
+ * d_logits + t*batch_per_query*n_classes floats.  With the cache enabled the SubGraph shared by the
+ * last window_q queries (element-wise minimum of their layer encodings = their exact intersection,
+ * Section 2.2, Appendix A.4) is marked resident for the following queries.
+ * Synchronises the stream before filling `stats` (may be NULL).  `opts` NULL = cache on, window 4,
+ * graphs on, latency recorded.
+ */
+sgs_status_t sgs_stream_run(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs,
+                            const void *d_inputs, int batch_per_query, int res, void *d_logits,
+                            const sgs_stream_opts_t *opts, sgs_stream_stats_t *stats, void *cuda_stream);
+
+/*
+ * sgs_stream_run_host - the same stream with HOST buffers: each query's input is copied host->device
+ * and its logits device->host inside the call (inputs in the compute dtype, logits fp32).  Host
+ * memory may be pageable or pinned; pinned memory overlaps better.
+ */
+sgs_status_t sgs_stream_run_host(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs,
+                                 const void *h_inputs, int batch_per_query, int res, void *h_logits,
+                                 const sgs_stream_opts_t *opts, sgs_stream_stats_t *stats, void *cuda_stream);
+
+/* Configure the SubGraph cache used by sgs_subnet_run (sgs_stream_run takes its own options).
+ * budget_bytes 0 = device maximum.  window_q >= 1. */
+sgs_status_t sgs_cache_configure(sgs_supernet_t *net, int enabled, size_t budget_bytes, int window_q);
+sgs_status_t sgs_cache_stats(const sgs_supernet_t *net, sgs_cache_stats_t *out);
+
+/*
+ * Vector encoding of a SubNet (Section 3.3): for every stored layer i, out[3i] = K_i (filters),
+ * out[3i+1] = C_i (channels), out[3i+2] = k_i (kernel size); zeros for layers the SubNet does not
+ * use.  `out` is a host array of 3*sgs_num_layers() ints.
+ */
+int sgs_num_layers(const sgs_supernet_t *net);
+sgs_status_t sgs_subnet_encode(const sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, int *out);
+
+/* Useful FLOPs (2*M*K'*C'*k*k over sliced layers) and touched weight bytes of one query. */
+sgs_status_t sgs_subnet_cost(const sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, int batch, int res,
+                             double *flops, double *weight_bytes, double *activation_bytes);
+
+/*
+ * sgs_conv2d_sliced - one sliced convolution layer with its fused epilogue, on caller-owned device
+ * tensors (paper Section 2.1: the layer uses the first K filters and first C channels of the stored
+ * tensor and the centre k x k window of its stored R x R kernel; Section 4.2 "Output Buffer": only
+ * final outputs leave the chip):
+ *   y[n][ho][wo][f] = act( scale[f] * sum_{r,s<k} sum_{c<C} x[n][ho*stride+r-p][wo*stride+s-p][c]
+ *                          * w[f][o+r][o+s][c] + shift[f] + res[n][ho][wo][f] ),   p = (k-1)/2, o = (R-k)/2
+ *   d_x     [N][H][W][C] NHWC, dtype elements            d_y, d_res  [N][Ho][Wo][K] (d_res may be NULL)
+ *   d_w     stored weights, [Kmax][R][R][Cmax] (depthwise: [R][R][Kmax]), dtype elements
+ *   d_scale, d_shift  [>= K] fp32
+ * impl 0 = automatic (tensor cores when dtype is bf16, C, K, Cmax are multiples of 8, pointers are
+ * 16-byte aligned and stride-2 inputs have even sizes), 1 = CUDA-core kernel, 2 = tensor cores or
+ * SGS_EUNSUPPORTED.  weight_policy 0 = no L2 hint, 1 = evict-last for weight tiles with filter <
+ * cache_k and channel < cache_c and evict-first for the rest, 2 = all weights evict-first.
+ * Asynchronous on `cuda_stream`.  The tensor-core path may split the reduction over several CTAs
+ * using a per-device scratch buffer that this function allocates on demand (cudaMalloc) and keeps;
+ * calls that overlap on the same device must therefore not run concurrently.
+ */
+typedef struct {
+    int N, H, W, C, K;      /* input dims, sliced channels C, sliced filters K */
+    int Kmax, Cmax, R;      /* stored tensor dims */
+    int k, stride, act;     /* kernel size, stride (1 or 2), activation 0 none / 1 ReLU / 2 h-swish */
+    int dtype;              /* sgs_dtype_t */
+    int impl;
+    int depthwise;
+    int cache_k, cache_c, weight_policy;
+    int split_k_off;        /* 1: never split the reduction */
+} sgs_conv_desc_t;
+sgs_status_t sgs_conv2d_sliced(const sgs_conv_desc_t *desc, const void *d_x, const void *d_w, const float *d_scale,
+                               const float *d_shift, const void *d_res, void *d_y, void *cuda_stream);
+
+/* Nonzero once a kernel of this process has reported that one of its bounded waits ran out. */
+int sgs_device_status(void);
+
+/* Library options by name (debug and measurement aids): "conv_impl" 0 = automatic, 1 = force the
+ * CUDA-core kernels; "profile" see sgs_profile_read.  Unknown name -> SGS_EINVAL. */
+sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long value);
+
+/*
+ * Per-kernel-class timing.  After sgs_set_option(net, "profile", 2) (2 = on and reset, 1 = on, 0 = off)
+ * every kernel the handle launches is bracketed by CUDA events on the launching stream (graphs are
+ * bypassed meanwhile).  kernel_class: 0 tensor-core convolution, 1 CUDA-core convolution,
+ * 2 depthwise convolution, 3 everything else.  Returns the launches, their summed device time, their
+ * summed algorithmic bytes (sliced weights + input + output + residual of each launch) and useful
+ * FLOPs since the last reset.  Synchronises the device.
+ */
+sgs_status_t sgs_profile_read(sgs_supernet_t *net, int kernel_class, long long *launches, double *total_ms,
+                              double *alg_bytes, double *flops);
+
+/* Counters by name ("kernel_launches", "plan_hits", "plan_misses", "device_bytes", "tc_convs"). */
+long long sgs_get_counter(const sgs_supernet_t *net, const char *name);
+
+const char *sgs_last_error(const sgs_supernet_t *net);
+void sgs_supernet_free(sgs_supernet_t *net);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SGS_H_ */

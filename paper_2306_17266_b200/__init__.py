@@ -1,0 +1,5 @@
+"""SubGraph-Stationary SubNet inference on B200: ctypes binding of the CUDA library plus the
+seeded workload generators.  The CUDA library is loaded on first use, never at import."""
+from . import workload  # noqa: F401
+from .binding import (SGS_BF16, SGS_F32, CacheStats, ConvDesc, SgsError, StreamOpts, StreamStats, SuperNet,  # noqa: F401
+                      conv2d_sliced, device_status, lib)

@@ -1,0 +1,199 @@
+"""Thin ctypes binding of libsgs.so: argument marshalling only, same names as include/sgs.h.
+
+Device buffers are passed as integer addresses (for example ``tensor.data_ptr()``), streams as the
+integer ``cudaStream_t`` (``torch.cuda.current_stream().cuda_stream``).  There is no CPU fallback:
+importing works without the library, every call raises if it cannot be loaded.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+from .workload import ArchDesc, SubnetCfg, arch_desc, cfg_array
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsgs.so")
+
+SGS_OK, SGS_EINVAL, SGS_ECONFIG, SGS_ENOMEM, SGS_ECUDA, SGS_ETIMEOUT, SGS_EUNSUPPORTED = range(7)
+SGS_F32, SGS_BF16 = 0, 1
+STATUS_NAMES = ["SGS_OK", "SGS_EINVAL", "SGS_ECONFIG", "SGS_ENOMEM", "SGS_ECUDA", "SGS_ETIMEOUT", "SGS_EUNSUPPORTED"]
+
+EXPORTS = [
+    "sgs_supernet_load", "sgs_subnet_validate", "sgs_subnet_run", "sgs_stream_run", "sgs_stream_run_host",
+    "sgs_cache_configure", "sgs_cache_stats", "sgs_num_layers", "sgs_subnet_encode", "sgs_subnet_cost",
+    "sgs_set_option", "sgs_get_counter", "sgs_last_error", "sgs_supernet_free", "sgs_conv2d_sliced", "sgs_device_status",
+    "sgs_profile_read",
+]
+
+
+class ConvDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("N", "H", "W", "C", "K", "Kmax", "Cmax", "R", "k", "stride", "act", "dtype",
+                                             "impl", "depthwise", "cache_k", "cache_c", "weight_policy", "split_k_off")]
+
+
+class StreamOpts(ctypes.Structure):
+    _fields_ = [("cache_enabled", ctypes.c_int), ("window_q", ctypes.c_int), ("cache_budget_bytes", ctypes.c_size_t),
+                ("use_graphs", ctypes.c_int), ("record_latency", ctypes.c_int), ("weights_evict_first", ctypes.c_int)]
+
+
+class StreamStats(ctypes.Structure):
+    _fields_ = [("n_queries", ctypes.c_int), ("total_ms", ctypes.c_double), ("queries_per_s", ctypes.c_double),
+                ("images_per_s", ctypes.c_double), ("p50_ms", ctypes.c_double), ("p99_ms", ctypes.c_double),
+                ("mean_ms", ctypes.c_double), ("useful_flops", ctypes.c_double), ("weight_bytes", ctypes.c_double),
+                ("hbm_weight_bytes", ctypes.c_double), ("hit_ratio", ctypes.c_double), ("byte_hit_ratio", ctypes.c_double),
+                ("kernel_launches", ctypes.c_longlong), ("plan_hits", ctypes.c_int), ("plan_misses", ctypes.c_int),
+                ("cache_updates", ctypes.c_int)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class CacheStats(ctypes.Structure):
+    _fields_ = [("enabled", ctypes.c_int), ("window_q", ctypes.c_int), ("budget_bytes", ctypes.c_size_t),
+                ("l2_bytes", ctypes.c_size_t), ("persisting_l2_max", ctypes.c_size_t), ("access_window_max", ctypes.c_size_t),
+                ("cached_subgraph_bytes", ctypes.c_size_t), ("supernet_bytes", ctypes.c_size_t),
+                ("device_bytes_allocated", ctypes.c_size_t)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class SgsError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__(f"{STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else status}: {text}")
+        self.status = status
+
+
+_lib = None
+
+
+def lib():
+    """Load libsgs.so (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2306_17266_b200.build` first")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci, cs = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.sgs_supernet_load.argtypes = [vp, vp, cs, ci, ci, ctypes.POINTER(vp)]
+        L.sgs_subnet_validate.argtypes = [vp, vp]
+        L.sgs_subnet_run.argtypes = [vp, vp, vp, ci, ci, vp, vp]
+        L.sgs_stream_run.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, vp, vp]
+        L.sgs_stream_run_host.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, vp, vp]
+        L.sgs_cache_configure.argtypes = [vp, ci, cs, ci]
+        L.sgs_cache_stats.argtypes = [vp, vp]
+        L.sgs_num_layers.argtypes = [vp]
+        L.sgs_subnet_encode.argtypes = [vp, vp, vp]
+        L.sgs_subnet_cost.argtypes = [vp, vp, ci, ci, vp, vp, vp]
+        L.sgs_set_option.argtypes = [vp, ctypes.c_char_p, ctypes.c_longlong]
+        L.sgs_get_counter.argtypes = [vp, ctypes.c_char_p]
+        L.sgs_get_counter.restype = ctypes.c_longlong
+        L.sgs_last_error.argtypes = [vp]
+        L.sgs_last_error.restype = ctypes.c_char_p
+        L.sgs_supernet_free.argtypes = [vp]
+        L.sgs_supernet_free.restype = None
+        L.sgs_conv2d_sliced.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+        L.sgs_device_status.argtypes = []
+        L.sgs_profile_read.argtypes = [vp, ci, vp, vp, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _addr(buf) -> int:
+    """Integer address of a host buffer (numpy array / ctypes object) or pass an int through."""
+    if buf is None:
+        return 0
+    if isinstance(buf, int):
+        return buf
+    if hasattr(buf, "ctypes"):
+        return buf.ctypes.data
+    return ctypes.addressof(buf)
+
+
+def conv2d_sliced(desc: ConvDesc, d_x: int, d_w: int, d_scale: int, d_shift: int, d_res: int, d_y: int, stream: int = 0):
+    st = lib().sgs_conv2d_sliced(ctypes.byref(desc), d_x, d_w, d_scale, d_shift, d_res or None, d_y, stream)
+    if st != SGS_OK:
+        raise SgsError(st, "sgs_conv2d_sliced")
+
+
+def device_status() -> int:
+    return int(lib().sgs_device_status())
+
+
+class SuperNet:
+    """Owner of one loaded SuperNet handle."""
+
+    def __init__(self, family: int, host_blob, dtype: int = SGS_BF16, device: int = 0, arch: Optional[ArchDesc] = None):
+        self._h = ctypes.c_void_p()
+        self.family, self.dtype, self.device = family, dtype, device
+        a = arch if arch is not None else arch_desc(family)
+        nbytes = host_blob.nbytes if hasattr(host_blob, "nbytes") else len(host_blob)
+        st = lib().sgs_supernet_load(ctypes.byref(a), _addr(host_blob), nbytes, dtype, device, ctypes.byref(self._h))
+        if st != SGS_OK:
+            self._h = ctypes.c_void_p()
+            raise SgsError(st, "sgs_supernet_load failed")
+        self.n_classes = a.n_classes
+        self.n_layers = lib().sgs_num_layers(self._h)
+
+    def _check(self, st: int):
+        if st != SGS_OK:
+            raise SgsError(st, lib().sgs_last_error(self._h).decode())
+
+    def close(self):
+        if self._h:
+            lib().sgs_supernet_free(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def subnet_validate(self, cfg: SubnetCfg) -> int:
+        return lib().sgs_subnet_validate(self._h, ctypes.byref(cfg))
+
+    def subnet_run(self, cfg: SubnetCfg, d_input: int, batch: int, res: int, d_logits: int, stream: int = 0):
+        self._check(lib().sgs_subnet_run(self._h, ctypes.byref(cfg), d_input, batch, res, d_logits, stream))
+
+    def stream_run(self, cfgs: Sequence[SubnetCfg], d_inputs, batch: int, res: int, d_logits,
+                   opts: Optional[StreamOpts] = None, stream: int = 0, host: bool = False) -> StreamStats:
+        arr = cfgs if isinstance(cfgs, ctypes.Array) else cfg_array(cfgs)
+        stats = StreamStats()
+        fn = lib().sgs_stream_run_host if host else lib().sgs_stream_run
+        self._check(fn(self._h, len(arr), ctypes.addressof(arr), _addr(d_inputs), batch, res, _addr(d_logits),
+                       ctypes.addressof(opts) if opts is not None else None, ctypes.addressof(stats), stream))
+        return stats
+
+    def cache_configure(self, enabled: bool, budget_bytes: int = 0, window_q: int = 4):
+        self._check(lib().sgs_cache_configure(self._h, int(enabled), budget_bytes, window_q))
+
+    def cache_stats(self) -> CacheStats:
+        s = CacheStats()
+        self._check(lib().sgs_cache_stats(self._h, ctypes.addressof(s)))
+        return s
+
+    def subnet_encode(self, cfg: SubnetCfg):
+        import numpy as np
+        out = np.zeros((self.n_layers, 3), dtype=np.int32)
+        self._check(lib().sgs_subnet_encode(self._h, ctypes.byref(cfg), out.ctypes.data))
+        return out
+
+    def subnet_cost(self, cfg: SubnetCfg, batch: int, res: int):
+        f, w, a = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+        self._check(lib().sgs_subnet_cost(self._h, ctypes.byref(cfg), batch, res, ctypes.addressof(f), ctypes.addressof(w),
+                                          ctypes.addressof(a)))
+        return f.value, w.value, a.value
+
+    def profile_read(self, kernel_class: int):
+        n, ms, b, f = ctypes.c_longlong(), ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+        self._check(lib().sgs_profile_read(self._h, kernel_class, ctypes.addressof(n), ctypes.addressof(ms),
+                                           ctypes.addressof(b), ctypes.addressof(f)))
+        return {"launches": n.value, "total_ms": ms.value, "alg_bytes": b.value, "flops": f.value}
+
+    def set_option(self, name: str, value: int):
+        self._check(lib().sgs_set_option(self._h, name.encode(), value))
+
+    def get_counter(self, name: str) -> int:
+        return int(lib().sgs_get_counter(self._h, name.encode()))

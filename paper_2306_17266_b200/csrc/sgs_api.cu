@@ -1,0 +1,1225 @@
+// Host side of libsgs: the C interface, SuperNet loading, SubNet slice plans, plan execution,
+// query streams and the SubGraph cache policy.
+#include "sgs_internal.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <map>
+
+using namespace sgs;
+
+namespace {
+
+constexpr uint32_t BLOB_MAGIC = 0x42534753u;  // 'SGSB'
+
+struct LayerSpec {
+    std::string name;
+    int kind, K, C, R;
+    bool bn, bias;
+};
+
+// nearest multiple of 8 to num/den (ties up), at least 8
+int round8(long long num, long long den) {
+    long long q = (2 * num + 8 * den) / (16 * den);
+    return (int)std::max<long long>(8, 8 * q);
+}
+int per_mille(float f) { return (int)std::floor((double)f * 1000.0 + 0.5); }
+
+struct FamilyDef {
+    int n_stages = 0;
+    std::vector<int> width, max_depth, base_depth, stride, act, se;
+    int stem = 0, classes = 0, max_kernel = 0;
+};
+
+FamilyDef family_def(int family) {
+    FamilyDef d;
+    if (family == SGS_TINY) {
+        d.n_stages = 3; d.width = {16, 32, 64}; d.max_depth = {3, 3, 3}; d.base_depth = {1, 1, 1};
+        d.stride = {1, 2, 2}; d.stem = 16; d.classes = 10; d.max_kernel = 3;
+    } else if (family == SGS_RESNET) {
+        d.n_stages = 4; d.width = {256, 512, 1024, 2048}; d.base_depth = {2, 2, 4, 2}; d.max_depth = {4, 4, 6, 4};
+        d.stride = {1, 2, 2, 2}; d.stem = 64; d.classes = 1000; d.max_kernel = 7;
+    } else if (family == SGS_MBV3) {
+        d.n_stages = 5; d.width = {24, 40, 80, 112, 160}; d.max_depth = {4, 4, 4, 4, 4}; d.base_depth = {2, 2, 2, 2, 2};
+        d.stride = {2, 2, 2, 1, 2}; d.act = {ACT_RELU, ACT_RELU, ACT_HSWISH, ACT_HSWISH, ACT_HSWISH};
+        d.se = {0, 1, 0, 1, 1}; d.stem = 16; d.classes = 1000; d.max_kernel = 7;
+    }
+    return d;
+}
+
+std::string bname(int s, int b, const char *leaf) {
+    char buf[64];
+    snprintf(buf, sizeof buf, "s%db%d.%s", s, b, leaf);
+    return buf;
+}
+
+// Stored layers in blob order.
+std::vector<LayerSpec> stored_layers(int family) {
+    FamilyDef d = family_def(family);
+    std::vector<LayerSpec> v;
+    auto conv = [&](std::string n, int K, int C, int R) { v.push_back({std::move(n), KIND_CONV, K, C, R, true, false}); };
+    auto lin = [&](std::string n, int K, int C) { v.push_back({std::move(n), KIND_LINEAR, K, C, 1, false, true}); };
+    auto dw = [&](std::string n, int K, int R) { v.push_back({std::move(n), KIND_DW, K, 1, R, true, false}); };
+    if (family == SGS_TINY) {
+        conv("stem", d.stem, 3, 3);
+        int in = d.stem;
+        for (int s = 0; s < d.n_stages; s++) {
+            for (int b = 0; b < d.max_depth[s]; b++) {
+                int cin = b ? d.width[s] : in;
+                conv(bname(s, b, "conv1"), d.width[s], cin, 3);
+                conv(bname(s, b, "conv2"), d.width[s], d.width[s], 3);
+                if (b == 0 && s > 0) conv(bname(s, b, "proj"), d.width[s], cin, 1);
+            }
+            in = d.width[s];
+        }
+        lin("fc", d.classes, in);
+    } else if (family == SGS_RESNET) {
+        conv("stem", d.stem, 3, 7);
+        int in = d.stem;
+        for (int s = 0; s < d.n_stages; s++) {
+            int mid = round8((long long)d.width[s] * 350, 1000);
+            for (int b = 0; b < d.max_depth[s]; b++) {
+                int cin = b ? d.width[s] : in;
+                conv(bname(s, b, "conv1"), mid, cin, 1);
+                conv(bname(s, b, "conv2"), mid, mid, 3);
+                conv(bname(s, b, "conv3"), d.width[s], mid, 1);
+                if (b == 0) conv(bname(s, b, "proj"), d.width[s], cin, 1);
+            }
+            in = d.width[s];
+        }
+        lin("fc", d.classes, in);
+    } else if (family == SGS_MBV3) {
+        conv("stem", d.stem, 3, 3);
+        dw("first.dw", d.stem, 3);
+        conv("first.pw", d.stem, d.stem, 1);
+        int in = d.stem;
+        for (int s = 0; s < d.n_stages; s++) {
+            for (int b = 0; b < d.max_depth[s]; b++) {
+                int cin = b ? d.width[s] : in, mid = 6 * cin;
+                conv(bname(s, b, "expand"), mid, cin, 1);
+                dw(bname(s, b, "dw"), mid, 7);
+                if (d.se[s]) {
+                    int sq = round8(mid, 4);
+                    lin(bname(s, b, "se1"), sq, mid);
+                    lin(bname(s, b, "se2"), mid, sq);
+                }
+                conv(bname(s, b, "project"), d.width[s], mid, 1);
+            }
+            in = d.width[s];
+        }
+        conv("head.conv", 960, in, 1);
+        lin("head.mix", 1280, 960);
+        lin("fc", d.classes, 1280);
+    }
+    return v;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+struct CacheState {
+    bool enabled = false;
+    int window_q = 4;
+    size_t budget = 0;
+    std::deque<std::vector<int>> window;  // last encodings (3 ints per layer)
+    std::vector<int> G;                   // cached SubGraph encoding, clipped to the budget
+    size_t G_bytes = 0;
+    int epoch = 0;                        // bumped whenever G changes
+    int since_update = 0;
+    int evict_first_when_off = 0;
+};
+
+struct ProfRec { int cls; cudaEvent_t a, b; double bytes, flops; };
+
+}  // namespace
+
+struct sgs_supernet {
+    int family = 0, device = 0;
+    sgs_dtype_t dtype = SGS_BF16;
+    FamilyDef def;
+    std::vector<StoredLayer> layers;
+    std::map<std::string, int> by_name;
+    char *weight_arena = nullptr;
+    size_t weight_arena_bytes = 0;
+    float *param_arena = nullptr;  // folded scale / shift
+    size_t param_arena_bytes = 0;
+    // activation workspaces
+    void *act[4] = {nullptr, nullptr, nullptr, nullptr};
+    size_t act_elems = 0;
+    float *vec[3] = {nullptr, nullptr, nullptr};
+    size_t vec_elems = 0;
+    int *cache_tbl = nullptr;       // device: [policy, K_0, C_0, K_1, C_1, ...] read by the conv kernels
+    int cache_tbl_epoch = -1;       // cache epoch the device table reflects
+    float *splitk_ws = nullptr;     // split-K scratch of the tensor-core kernel
+    unsigned *splitk_counters = nullptr;
+    size_t splitk_ws_elems = 0;
+    unsigned splitk_n_counters = 0;
+    void *host_stage_in = nullptr;  // device staging for the host-buffer stream
+    float *host_stage_out = nullptr;
+    size_t stage_in_bytes = 0, stage_out_bytes = 0;
+    size_t device_bytes = 0;
+    std::unordered_map<std::string, std::unique_ptr<Plan>> plans;
+    CacheState cache;
+    size_t l2_bytes = 0, persist_max = 0, window_max = 0;
+    long long kernel_launches = 0;
+    int plan_hits = 0, plan_misses = 0;
+    int force_plain = 0;
+    // per-kernel-class timing (option "profile"): 0 tensor-core conv, 1 CUDA-core conv, 2 depthwise, 3 other
+    int profile = 0;
+    std::vector<ProfRec> prof_pending;
+    std::vector<cudaEvent_t> prof_pool;
+    double prof_ms[4] = {0, 0, 0, 0}, prof_bytes[4] = {0, 0, 0, 0}, prof_flops[4] = {0, 0, 0, 0};
+    long long prof_launches[4] = {0, 0, 0, 0};
+    mutable std::string err;
+    size_t elem() const { return dtype == SGS_BF16 ? 2 : 4; }
+    int idx(const std::string &n) const {
+        auto it = by_name.find(n);
+        return it == by_name.end() ? -1 : it->second;
+    }
+};
+
+namespace {
+
+sgs_status_t fail(const sgs_supernet *n, sgs_status_t st, const std::string &msg) {
+    if (n) n->err = msg;
+    return st;
+}
+#define CU(call)                                                                                        \
+    do {                                                                                                \
+        cudaError_t e_ = (call);                                                                        \
+        if (e_ != cudaSuccess)                                                                          \
+            return fail(net, e_ == cudaErrorMemoryAllocation ? SGS_ENOMEM : SGS_ECUDA,                  \
+                        std::string(#call) + ": " + cudaGetErrorString(e_));                            \
+    } while (0)
+
+sgs_status_t dev_alloc(sgs_supernet *net, void **p, size_t bytes) {
+    CU(cudaMalloc(p, bytes));
+    net->device_bytes += bytes;
+    return SGS_OK;
+}
+void dev_free(sgs_supernet *net, void *p, size_t bytes) {
+    if (!p) return;
+    cudaFree(p);
+    net->device_bytes -= bytes;
+}
+void drop_graphs(sgs_supernet *net) {
+    for (auto &kv : net->plans)
+        if (kv.second->graph) { cudaGraphExecDestroy(kv.second->graph); kv.second->graph = nullptr; }
+}
+
+// ------------------------------------------------------------------------------------------
+// Config -> per-layer slices (paper Section 2.1: elastic depth, width / expand ratio, kernel)
+// ------------------------------------------------------------------------------------------
+bool in_set(int v, std::initializer_list<int> s) { return std::find(s.begin(), s.end(), v) != s.end(); }
+
+bool cfg_valid(const sgs_supernet *net, const sgs_subnet_cfg_t *c) {
+    const FamilyDef &d = net->def;
+    for (int s = 0; s < d.n_stages; s++) {
+        int dep = c->depth[s];
+        if (net->family == SGS_TINY) {
+            if (!in_set(dep, {1, 2, 3}) || !in_set(per_mille(c->width[s + 1]), {500, 750, 1000})) return false;
+        } else if (net->family == SGS_RESNET) {
+            if (dep < d.base_depth[s] || dep > d.max_depth[s]) return false;
+            if (!in_set(per_mille(c->width[s + 1]), {650, 800, 1000})) return false;
+            for (int b = 0; b < dep; b++)
+                if (!in_set(per_mille(c->expand[s][b]), {200, 250, 350})) return false;
+        } else {
+            if (!in_set(dep, {2, 3, 4})) return false;
+            for (int b = 0; b < dep; b++) {
+                if (!in_set(per_mille(c->expand[s][b]), {3000, 4000, 6000})) return false;
+                if (!in_set(c->kernel[s][b], {3, 5, 7})) return false;
+            }
+        }
+    }
+    if (net->family == SGS_RESNET && !in_set(per_mille(c->width[0]), {650, 800, 1000})) return false;
+    return true;
+}
+
+std::vector<Slice> slices_for(const sgs_supernet *net, const sgs_subnet_cfg_t *c) {
+    const FamilyDef &d = net->def;
+    std::vector<Slice> sl(net->layers.size());
+    auto use = [&](const std::string &name, int K, int C, int k) {
+        int i = net->idx(name);
+        sl[i].active = 1; sl[i].K = K; sl[i].C = C; sl[i].k = k;
+    };
+    if (net->family == SGS_TINY) {
+        std::vector<int> w(3);
+        for (int s = 0; s < 3; s++) w[s] = d.width[s] * per_mille(c->width[s + 1]) / 1000;
+        use("stem", w[0], 3, 3);
+        int in = w[0];
+        for (int s = 0; s < 3; s++) {
+            for (int b = 0; b < c->depth[s]; b++) {
+                int cin = b ? w[s] : in;
+                use(bname(s, b, "conv1"), w[s], cin, 3);
+                use(bname(s, b, "conv2"), w[s], w[s], 3);
+                if (b == 0 && s > 0) use(bname(s, b, "proj"), w[s], cin, 1);
+            }
+            in = w[s];
+        }
+        use("fc", d.classes, in, 1);
+    } else if (net->family == SGS_RESNET) {
+        int in = round8((long long)d.stem * per_mille(c->width[0]), 1000);
+        use("stem", in, 3, 7);
+        for (int s = 0; s < 4; s++) {
+            int out = round8((long long)d.width[s] * per_mille(c->width[s + 1]), 1000);
+            for (int b = 0; b < c->depth[s]; b++) {
+                int cin = b ? out : in;
+                int mid = round8((long long)out * per_mille(c->expand[s][b]), 1000);
+                use(bname(s, b, "conv1"), mid, cin, 1);
+                use(bname(s, b, "conv2"), mid, mid, 3);
+                use(bname(s, b, "conv3"), out, mid, 1);
+                if (b == 0) use(bname(s, b, "proj"), out, cin, 1);
+            }
+            in = out;
+        }
+        use("fc", d.classes, in, 1);
+    } else {
+        use("stem", d.stem, 3, 3);
+        use("first.dw", d.stem, 1, 3);
+        use("first.pw", d.stem, d.stem, 1);
+        int in = d.stem;
+        for (int s = 0; s < 5; s++) {
+            for (int b = 0; b < c->depth[s]; b++) {
+                int cin = b ? d.width[s] : in;
+                int mid = round8((long long)cin * per_mille(c->expand[s][b]), 1000);
+                use(bname(s, b, "expand"), mid, cin, 1);
+                use(bname(s, b, "dw"), mid, 1, c->kernel[s][b]);
+                if (d.se[s]) {
+                    int sq = round8(mid, 4);
+                    use(bname(s, b, "se1"), sq, mid, 1);
+                    use(bname(s, b, "se2"), mid, sq, 1);
+                }
+                use(bname(s, b, "project"), d.width[s], mid, 1);
+            }
+            in = d.width[s];
+        }
+        use("head.conv", 960, in, 1);
+        use("head.mix", 1280, 960, 1);
+        use("fc", d.classes, 1280, 1);
+    }
+    return sl;
+}
+
+std::vector<int> encoding_of(const std::vector<Slice> &sl) {
+    std::vector<int> e(3 * sl.size());
+    for (size_t i = 0; i < sl.size(); i++) { e[3 * i] = sl[i].K; e[3 * i + 1] = sl[i].C; e[3 * i + 2] = sl[i].k; }
+    return e;
+}
+
+// ------------------------------------------------------------------------------------------
+// Plan construction
+// ------------------------------------------------------------------------------------------
+struct Builder {
+    sgs_supernet *net;
+    Plan *plan;
+    int N;
+    size_t max_elems = 0;
+
+    void note(size_t elems) { max_elems = std::max(max_elems, elems); }
+
+    // convolution (regular or depthwise) of stored layer `name`
+    void conv(const std::string &name, int in, int out, int res, int &H, int &W, int stride, int act) {
+        int li = net->idx(name);
+        const StoredLayer &L = net->layers[li];
+        const Slice &s = plan->slices[li];
+        Op op;
+        op.type = L.kind == KIND_DW ? OP_DW : OP_CONV;
+        op.layer = li; op.in = in; op.out = out; op.res = res;
+        ConvArgs &a = op.conv;
+        a.w = L.w; a.scale = L.scale; a.shift = L.shift;
+        a.N = N; a.H = H; a.W = W; a.C = L.kind == KIND_DW ? s.K : s.C; a.K = s.K;
+        a.k = s.k; a.stride = stride; a.act = act;
+        int p = (s.k - 1) / 2;
+        a.Ho = (H + 2 * p - s.k) / stride + 1;
+        a.Wo = (W + 2 * p - s.k) / stride + 1;
+        a.Kmax = L.K; a.Cmax = L.C; a.R = L.R;
+        double M = (double)N * a.Ho * a.Wo;
+        double per_out = L.kind == KIND_DW ? (double)s.k * s.k : (double)s.C * s.k * s.k;
+        op.flops = 2.0 * M * s.K * per_out;
+        op.alg_bytes = ((double)s.K * per_out + (double)N * H * W * a.C + M * s.K * (res >= 0 ? 2 : 1)) * net->elem();
+        plan->flops += op.flops;
+        plan->weight_bytes += (double)s.K * per_out * net->elem();
+        plan->act_bytes += ((double)N * H * W * a.C + M * s.K * (res >= 0 ? 2 : 1)) * net->elem();
+        note((size_t)M * s.K);
+        H = a.Ho; W = a.Wo;
+        plan->ops.push_back(op);
+    }
+    void linear(const std::string &name, int vin, int vout, int act) {
+        int li = net->idx(name);
+        const Slice &s = plan->slices[li];
+        Op op;
+        op.type = OP_LINEAR; op.layer = li; op.vin = vin; op.vout = vout; op.N = N; op.C = s.C; op.K = s.K; op.act = act;
+        op.flops = 2.0 * N * s.K * s.C;
+        op.alg_bytes = (double)s.K * s.C * net->elem() + 4.0 * N * (s.K + s.C);
+        plan->flops += op.flops;
+        plan->weight_bytes += (double)s.K * s.C * net->elem();
+        plan->ops.push_back(op);
+    }
+    void gap(int in, int vout, int H, int W, int C) {
+        Op op;
+        op.type = OP_GAP; op.in = in; op.vout = vout; op.N = N; op.H = H; op.W = W; op.C = C;
+        op.alg_bytes = (double)N * H * W * C * net->elem() + 4.0 * N * C;
+        plan->ops.push_back(op);
+    }
+};
+
+sgs_status_t build_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch, int res, Plan *plan) {
+    const FamilyDef &d = net->def;
+    plan->batch = batch; plan->res = res;
+    plan->slices = slices_for(net, cfg);
+    Builder B{net, plan, batch};
+    int H = res, W = res;
+    // activation buffers: X current tensor, T1/T2 temporaries, SC shortcut
+    int X = 0, T1 = 1, T2 = 2, SC = 3;
+    if (net->family == SGS_TINY) {
+        B.conv("stem", -1, X, -1, H, W, 1, ACT_RELU);
+        for (int s = 0; s < 3; s++)
+            for (int b = 0; b < cfg->depth[s]; b++) {
+                int st = b == 0 ? d.stride[s] : 1, shortcut = X;
+                int h1 = H, w1 = W;
+                if (b == 0 && s > 0) { int h = H, w = W; B.conv(bname(s, b, "proj"), X, SC, -1, h, w, st, ACT_NONE); shortcut = SC; }
+                B.conv(bname(s, b, "conv1"), X, T1, -1, h1, w1, st, ACT_RELU);
+                B.conv(bname(s, b, "conv2"), T1, T2, shortcut, h1, w1, 1, ACT_RELU);
+                std::swap(X, T2); H = h1; W = w1;
+            }
+        int C = plan->slices[net->idx("fc")].C;
+        B.gap(X, 0, H, W, C);
+        B.linear("fc", 0, -1, ACT_NONE);
+    } else if (net->family == SGS_RESNET) {
+        B.conv("stem", -1, T1, -1, H, W, 2, ACT_RELU);
+        {
+            Op op;
+            op.type = OP_MAXPOOL; op.in = T1; op.out = X; op.N = batch; op.H = H; op.W = W; op.C = plan->slices[net->idx("stem")].K;
+            int Hp = (H - 1) / 2 + 1, Wp = (W - 1) / 2 + 1;
+            op.alg_bytes = ((double)batch * H * W + (double)batch * Hp * Wp) * op.C * net->elem();
+            plan->ops.push_back(op);
+            H = Hp; W = Wp;
+            B.note((size_t)batch * H * W * op.C);
+        }
+        for (int s = 0; s < 4; s++)
+            for (int b = 0; b < cfg->depth[s]; b++) {
+                int st = b == 0 ? d.stride[s] : 1, shortcut = X;
+                int h = H, w = W;
+                if (b == 0) { int h0 = H, w0 = W; B.conv(bname(s, b, "proj"), X, SC, -1, h0, w0, st, ACT_NONE); shortcut = SC; }
+                B.conv(bname(s, b, "conv1"), X, T1, -1, h, w, 1, ACT_RELU);
+                B.conv(bname(s, b, "conv2"), T1, T2, -1, h, w, st, ACT_RELU);
+                B.conv(bname(s, b, "conv3"), T2, T1, shortcut, h, w, 1, ACT_RELU);
+                std::swap(X, T1); H = h; W = w;
+            }
+        int C = plan->slices[net->idx("fc")].C;
+        B.gap(X, 0, H, W, C);
+        B.linear("fc", 0, -1, ACT_NONE);
+    } else {
+        B.conv("stem", -1, X, -1, H, W, 2, ACT_HSWISH);
+        { int h = H, w = W; B.conv("first.dw", X, T1, -1, h, w, 1, ACT_RELU); }
+        { int h = H, w = W; B.conv("first.pw", T1, T2, X, h, w, 1, ACT_NONE); }
+        std::swap(X, T2);
+        int C = d.stem;
+        for (int s = 0; s < 5; s++)
+            for (int b = 0; b < cfg->depth[s]; b++) {
+                int st = b == 0 ? d.stride[s] : 1, out = d.width[s];
+                int mid = plan->slices[net->idx(bname(s, b, "expand"))].K;
+                int h = H, w = W;
+                B.conv(bname(s, b, "expand"), X, T1, -1, h, w, 1, d.act[s]);
+                B.conv(bname(s, b, "dw"), T1, T2, -1, h, w, st, d.act[s]);
+                if (d.se[s]) {
+                    B.gap(T2, 0, h, w, mid);
+                    Op g;
+                    g.type = OP_SE_GATE; g.layer = net->idx(bname(s, b, "se1")); g.layer2 = net->idx(bname(s, b, "se2"));
+                    g.vin = 0; g.vout = 1; g.N = batch; g.C = mid; g.K = plan->slices[g.layer].K;
+                    g.flops = 4.0 * batch * mid * g.K;
+                    g.alg_bytes = 2.0 * mid * g.K * net->elem();
+                    plan->flops += g.flops;
+                    plan->weight_bytes += 2.0 * mid * g.K * net->elem();
+                    plan->ops.push_back(g);
+                    Op sc;
+                    sc.type = OP_SCALE; sc.in = T2; sc.out = T2; sc.vin = 1; sc.N = batch; sc.H = h; sc.W = w; sc.C = mid;
+                    sc.alg_bytes = 2.0 * batch * h * w * mid * net->elem();
+                    plan->ops.push_back(sc);
+                }
+                int resid = (st == 1 && C == out) ? X : -1;
+                B.conv(bname(s, b, "project"), T2, T1, resid, h, w, 1, ACT_NONE);
+                std::swap(X, T1); H = h; W = w; C = out;
+            }
+        { int h = H, w = W; B.conv("head.conv", X, T1, -1, h, w, 1, ACT_HSWISH); }
+        B.gap(T1, 0, H, W, 960);
+        B.linear("head.mix", 0, 1, ACT_HSWISH);
+        B.linear("fc", 1, -1, ACT_NONE);
+    }
+    plan->act_elems = B.max_elems;
+    return SGS_OK;
+}
+
+sgs_status_t ensure_workspace(sgs_supernet *net, size_t act_elems, int batch) {
+    if (act_elems > net->act_elems) {
+        for (int i = 0; i < 4; i++) { dev_free(net, net->act[i], net->act_elems * net->elem() + 256); net->act[i] = nullptr; }
+        net->act_elems = 0;
+        drop_graphs(net);
+        for (auto &kv : net->plans) kv.second->prepared = false;
+        for (int i = 0; i < 4; i++) {
+            sgs_status_t st = dev_alloc(net, &net->act[i], act_elems * net->elem() + 256);
+            if (st != SGS_OK) return st;
+        }
+        net->act_elems = act_elems;
+    }
+    size_t vneed = (size_t)batch * 2048;
+    if (vneed > net->vec_elems) {
+        for (int i = 0; i < 3; i++) { dev_free(net, net->vec[i], net->vec_elems * 4); net->vec[i] = nullptr; }
+        net->vec_elems = 0;
+        drop_graphs(net);
+        for (int i = 0; i < 3; i++) {
+            sgs_status_t st = dev_alloc(net, (void **)&net->vec[i], vneed * 4);
+            if (st != SGS_OK) return st;
+        }
+        net->vec_elems = vneed;
+    }
+    return SGS_OK;
+}
+
+// Chooses the implementation of every convolution of a plan and fixes its buffer addresses (the
+// tensor maps of the tensor-core kernel hold absolute addresses of the activation workspaces).
+sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
+    size_t ws_need = 0;
+    unsigned ctr_need = 0;
+    for (Op &op : plan->ops) {
+        if (op.type != OP_CONV && op.type != OP_DW) continue;
+        op.conv.x = op.in >= 0 ? net->act[op.in] : nullptr;
+        op.conv.y = net->act[op.out];
+        op.conv.res = op.res >= 0 ? net->act[op.res] : nullptr;
+        op.impl = 0;
+        op.tc.reset();
+        if (op.type != OP_CONV || op.in < 0) continue;
+        if (net->dtype != SGS_BF16 || net->force_plain || !tc_available()) continue;
+        std::string why;
+        op.tc = tc_conv_prepare(op.conv, net->device, &why);
+        if (op.tc) {
+            op.impl = 1;
+            ws_need = std::max(ws_need, tc_conv_ws_elems(*op.tc));
+            if (tc_conv_ws_elems(*op.tc)) ctr_need = std::max(ctr_need, tc_conv_tiles(*op.tc));
+        }
+    }
+    if (ws_need > net->splitk_ws_elems || ctr_need > net->splitk_n_counters) {
+        drop_graphs(net);
+        const size_t we = std::max(ws_need, net->splitk_ws_elems);
+        const unsigned ce = std::max(ctr_need, std::max(net->splitk_n_counters, 1024u));
+        dev_free(net, net->splitk_ws, net->splitk_ws_elems * 4);  // cudaFree waits for work in flight
+        dev_free(net, net->splitk_counters, (size_t)net->splitk_n_counters * 4);
+        net->splitk_ws = nullptr; net->splitk_counters = nullptr;
+        net->splitk_ws_elems = 0; net->splitk_n_counters = 0;
+        sgs_status_t st = dev_alloc(net, (void **)&net->splitk_ws, std::max<size_t>(we, 1) * 4);
+        if (st != SGS_OK) return st;
+        st = dev_alloc(net, (void **)&net->splitk_counters, (size_t)ce * 4);
+        if (st != SGS_OK) return st;
+        CU(cudaMemset(net->splitk_counters, 0, (size_t)ce * 4));
+        net->splitk_ws_elems = std::max<size_t>(we, 1); net->splitk_n_counters = ce;
+    }
+    plan->prepared = true;
+    return SGS_OK;
+}
+
+sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch, int res, Plan **out) {
+    std::string key(reinterpret_cast<const char *>(cfg), sizeof(*cfg));
+    key.append(reinterpret_cast<const char *>(&batch), sizeof batch);
+    key.append(reinterpret_cast<const char *>(&res), sizeof res);
+    auto it = net->plans.find(key);
+    if (it != net->plans.end()) { net->plan_hits++; *out = it->second.get(); return SGS_OK; }
+    if (!cfg_valid(net, cfg)) return fail(net, SGS_ECONFIG, "SubNet config outside the elastic sets of this SuperNet");
+    net->plan_misses++;
+    std::unique_ptr<Plan> p(new Plan);
+    sgs_status_t st = build_plan(net, cfg, batch, res, p.get());
+    if (st != SGS_OK) return st;
+    *out = p.get();
+    net->plans.emplace(std::move(key), std::move(p));
+    return SGS_OK;
+}
+
+template <typename T>
+sgs_status_t run_ops(sgs_supernet *net, Plan *plan, const void *d_input, void *d_logits, cudaStream_t st, size_t first,
+                     size_t last) {
+    auto abuf = [&](int id) -> void * { return id < 0 ? const_cast<void *>(d_input) : net->act[id]; };
+    for (size_t oi = first; oi < last; oi++) {
+        Op &op = plan->ops[oi];
+        ProfRec rec{};
+        if (net->profile) {
+            rec.cls = op.type == OP_CONV ? (op.impl == 1 ? 0 : 1) : op.type == OP_DW ? 2 : 3;
+            rec.bytes = op.alg_bytes; rec.flops = op.flops;
+            for (cudaEvent_t *e : {&rec.a, &rec.b}) {
+                if (net->prof_pool.empty()) { CU(cudaEventCreate(e)); }
+                else { *e = net->prof_pool.back(); net->prof_pool.pop_back(); }
+            }
+            CU(cudaEventRecord(rec.a, st));
+        }
+        switch (op.type) {
+        case OP_CONV:
+        case OP_DW: {
+            ConvArgs a = op.conv;
+            if (op.in < 0) a.x = d_input;
+            a.cache_tbl = net->cache_tbl; a.layer = op.layer;
+            a.ws = net->splitk_ws; a.counters = net->splitk_counters;
+            a.ws_elems = net->splitk_ws_elems; a.n_counters = net->splitk_n_counters;
+            if (op.type == OP_DW) { CU(launch_dw<T>(a, st)); net->kernel_launches++; }
+            else if (op.impl == 1) { int n = 0; CU(tc_conv_launch(*op.tc, a, st, &n)); net->kernel_launches += n; }
+            else { CU(launch_conv_plain<T>(a, st)); net->kernel_launches++; }
+            break;
+        }
+        case OP_MAXPOOL:
+            CU(launch_maxpool3s2<T>((const T *)abuf(op.in), (T *)net->act[op.out], op.N, op.H, op.W, op.C, st));
+            net->kernel_launches++;
+            break;
+        case OP_GAP:
+            CU(launch_gap<T>((const T *)abuf(op.in), net->vec[op.vout], op.N, op.H * op.W, op.C, st));
+            net->kernel_launches++;
+            break;
+        case OP_SE_GATE: {
+            const StoredLayer &L1 = net->layers[op.layer], &L2 = net->layers[op.layer2];
+            CU(launch_se_gate<T>(net->vec[op.vin], (const T *)L1.w, L1.shift, (const T *)L2.w, L2.shift, net->vec[op.vout],
+                                 op.N, op.C, op.K, L1.C, L2.C, st));
+            net->kernel_launches++;
+            break;
+        }
+        case OP_SCALE:
+            CU(launch_scale<T>((const T *)net->act[op.in], net->vec[op.vin], (T *)net->act[op.out], op.N, op.H * op.W, op.C, st));
+            net->kernel_launches++;
+            break;
+        case OP_LINEAR: {
+            const StoredLayer &L = net->layers[op.layer];
+            float *y = op.vout < 0 ? static_cast<float *>(d_logits) : net->vec[op.vout];
+            CU(launch_linear<T>(net->vec[op.vin], (const T *)L.w, L.shift, y, op.N, op.C, op.K, L.C, op.act, st));
+            net->kernel_launches++;
+            break;
+        }
+        }
+        if (net->profile) {
+            CU(cudaEventRecord(rec.b, st));
+            net->prof_pending.push_back(rec);
+        }
+    }
+    return SGS_OK;
+}
+
+void fold_profile(sgs_supernet *net) {
+    if (net->prof_pending.empty()) return;
+    cudaDeviceSynchronize();
+    for (auto &r : net->prof_pending) {
+        float ms = 0;
+        if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) {
+            net->prof_ms[r.cls] += ms; net->prof_bytes[r.cls] += r.bytes; net->prof_flops[r.cls] += r.flops;
+            net->prof_launches[r.cls]++;
+        }
+        net->prof_pool.push_back(r.a);
+        net->prof_pool.push_back(r.b);
+    }
+    net->prof_pending.clear();
+}
+
+sgs_status_t run_plan(sgs_supernet *net, Plan *plan, const void *d_input, void *d_logits, cudaStream_t st, size_t first,
+                      size_t last) {
+    return net->dtype == SGS_BF16 ? run_ops<__nv_bfloat16>(net, plan, d_input, d_logits, st, first, last)
+                                  : run_ops<float>(net, plan, d_input, d_logits, st, first, last);
+}
+
+// Brings the device copy of the cache table up to date with the host policy state.
+sgs_status_t push_cache_table(sgs_supernet *net, cudaStream_t st) {
+    const CacheState &cs = net->cache;
+    if (net->cache_tbl_epoch == cs.epoch) return SGS_OK;
+    std::vector<int> tbl(1 + 2 * net->layers.size(), 0);
+    if (cs.enabled && !cs.G.empty()) {
+        tbl[0] = 1;
+        for (size_t li = 0; li < net->layers.size(); li++) { tbl[1 + 2 * li] = cs.G[3 * li]; tbl[2 + 2 * li] = cs.G[3 * li + 1]; }
+    } else if (!cs.enabled && cs.evict_first_when_off) {
+        tbl[0] = 2;
+    }
+    // pageable source: the runtime stages the bytes before the call returns, so tbl may go out of scope
+    CU(cudaMemcpyAsync(net->cache_tbl, tbl.data(), tbl.size() * sizeof(int), cudaMemcpyHostToDevice, st));
+    net->cache_tbl_epoch = cs.epoch;
+    return SGS_OK;
+}
+
+// Run one query.  With graphs, the first op (reads the caller's input) and the last op (writes the
+// caller's logits) are launched directly; everything between touches only buffers the handle owns and
+// is replayed as one captured graph per plan, independent of the caller's pointers and of the cache
+// state (kernels read the cache box from device memory).
+sgs_status_t run_query(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, const void *d_input, int batch, int res,
+                       void *d_logits, cudaStream_t st, bool use_graph, Plan **plan_out) {
+    Plan *plan = nullptr;
+    sgs_status_t rc = get_plan(net, cfg, batch, res, &plan);
+    if (rc != SGS_OK) return rc;
+    rc = ensure_workspace(net, plan->act_elems, batch);
+    if (rc != SGS_OK) return rc;
+    if (!plan->prepared) {
+        rc = choose_impls(net, plan);
+        if (rc != SGS_OK) return rc;
+    }
+    if (plan_out) *plan_out = plan;
+    rc = push_cache_table(net, st);
+    if (rc != SGS_OK) return rc;
+    const size_t n_ops = plan->ops.size();
+    if (!use_graph || net->profile || n_ops < 3) {
+        long long before = net->kernel_launches;
+        rc = run_plan(net, plan, d_input, d_logits, st, 0, n_ops);
+        plan->launches = (int)(net->kernel_launches - before);
+        return rc;
+    }
+    if (!plan->graph) {
+        cudaGraph_t g = nullptr;
+        CU(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+        long long before = net->kernel_launches;
+        rc = run_plan(net, plan, d_input, d_logits, st, 1, n_ops - 1);
+        plan->launches = (int)(net->kernel_launches - before) + 2;
+        net->kernel_launches = before;
+        cudaError_t e = cudaStreamEndCapture(st, &g);
+        if (rc != SGS_OK) { if (g) cudaGraphDestroy(g); return rc; }
+        if (e != cudaSuccess) return fail(net, SGS_ECUDA, std::string("graph capture: ") + cudaGetErrorString(e));
+        e = cudaGraphInstantiate(&plan->graph, g, 0);
+        cudaGraphDestroy(g);
+        if (e != cudaSuccess) return fail(net, SGS_ECUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
+    }
+    long long before = net->kernel_launches;
+    rc = run_plan(net, plan, d_input, d_logits, st, 0, 1);
+    if (rc != SGS_OK) return rc;
+    CU(cudaGraphLaunch(plan->graph, st));
+    rc = run_plan(net, plan, d_input, d_logits, st, n_ops - 1, n_ops);
+    net->kernel_launches = before + plan->launches;
+    return rc;
+}
+
+// ------------------------------------------------------------------------------------------
+// SubGraph cache policy (paper Section 2.2, 3.3, Appendix A.1 and A.4)
+// ------------------------------------------------------------------------------------------
+size_t layer_box_bytes(const sgs_supernet *net, int li, int K, int C, int k) {
+    const StoredLayer &L = net->layers[li];
+    size_t per = L.kind == KIND_DW ? (size_t)k * k : (size_t)C * k * k;
+    return (size_t)K * per * net->elem();
+}
+
+// G = element-wise minimum of the encodings in the window (the exact intersection of those SubNets,
+// because every slice is a prefix / centred window), kept layer by layer in network order while it
+// fits the byte budget.
+void recompute_cached_subgraph(sgs_supernet *net) {
+    CacheState &cs = net->cache;
+    if (cs.window.empty()) return;
+    std::vector<int> g = cs.window.front();
+    for (const auto &e : cs.window)
+        for (size_t i = 0; i < g.size(); i++) g[i] = std::min(g[i], e[i]);
+    size_t used = 0;
+    for (size_t li = 0; li < net->layers.size(); li++) {
+        size_t b = layer_box_bytes(net, (int)li, g[3 * li], g[3 * li + 1], g[3 * li + 2]);
+        if (used + b > cs.budget) { g[3 * li] = g[3 * li + 1] = g[3 * li + 2] = 0; continue; }
+        used += b;
+    }
+    if (g != cs.G) { cs.G = std::move(g); cs.epoch++; }
+    cs.G_bytes = used;
+}
+
+struct QueryAccount { double weight_bytes = 0, miss_bytes = 0, hit_ratio = 0; };
+
+QueryAccount account_query(const sgs_supernet *net, const std::vector<int> &sn) {
+    const CacheState &cs = net->cache;
+    QueryAccount a;
+    double num = 0, den = 0;
+    for (size_t li = 0; li < net->layers.size(); li++) {
+        int K = sn[3 * li], C = sn[3 * li + 1], k = sn[3 * li + 2];
+        if (!K) continue;
+        size_t all = layer_box_bytes(net, (int)li, K, C, k), common = 0;
+        int gK = 0, gC = 0;
+        if (cs.enabled && !cs.G.empty()) {
+            gK = std::min(K, cs.G[3 * li]); gC = std::min(C, cs.G[3 * li + 1]);
+            int gk = std::min(k, cs.G[3 * li + 2]);
+            common = layer_box_bytes(net, (int)li, gK, gC, gk);
+        }
+        a.weight_bytes += (double)all;
+        a.miss_bytes += (double)(all - common);
+        num += (double)gK * gK + (double)gC * gC;
+        den += (double)K * K + (double)C * C;
+    }
+    a.hit_ratio = den > 0 ? std::sqrt(num) / std::sqrt(den) : 0;
+    return a;
+}
+
+void cache_observe(sgs_supernet *net, const std::vector<int> &enc) {
+    CacheState &cs = net->cache;
+    cs.window.push_back(enc);
+    while ((int)cs.window.size() > cs.window_q) cs.window.pop_front();
+    if (++cs.since_update >= cs.window_q) {
+        cs.since_update = 0;
+        recompute_cached_subgraph(net);
+    }
+}
+
+void cache_reset(sgs_supernet *net, bool enabled, size_t budget, int window_q) {
+    CacheState &cs = net->cache;
+    cs.enabled = enabled;
+    cs.window_q = std::max(1, window_q);
+    size_t cap = net->persist_max ? net->persist_max : net->l2_bytes;
+    cs.budget = budget ? std::min(budget, net->l2_bytes ? net->l2_bytes : budget) : cap;
+    cs.window.clear();
+    cs.G.clear();
+    cs.G_bytes = 0;
+    cs.since_update = 0;
+    cs.epoch++;
+}
+
+}  // namespace
+
+// =============================================================================================
+// C interface
+// =============================================================================================
+extern "C" {
+
+sgs_status_t sgs_supernet_load(const sgs_arch_desc_t *arch, const void *host_blob, size_t nbytes,
+                               sgs_dtype_t compute_dtype, int device, sgs_supernet_t **out) {
+    if (!arch || !host_blob || !out || nbytes < 32 || nbytes % 4) return SGS_EINVAL;
+    if (compute_dtype != SGS_F32 && compute_dtype != SGS_BF16) return SGS_EINVAL;
+    if (arch->family < SGS_TINY || arch->family > SGS_MBV3) return SGS_EINVAL;
+    *out = nullptr;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return SGS_ECUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SGS_ECUDA;
+    if (prop.major != 10) return SGS_EUNSUPPORTED;
+    const uint32_t *words = static_cast<const uint32_t *>(host_blob);
+    if (words[0] != BLOB_MAGIC || words[1] != 1u || (int)words[2] != arch->family) return SGS_EINVAL;
+
+    std::unique_ptr<sgs_supernet> holder(new (std::nothrow) sgs_supernet);
+    if (!holder) return SGS_ENOMEM;
+    sgs_supernet *net = holder.get();
+    net->family = arch->family; net->device = device; net->dtype = compute_dtype;
+    net->def = family_def(arch->family);
+    // optional cross-checks of the descriptor
+    if (arch->n_stages && arch->n_stages != net->def.n_stages) return SGS_EINVAL;
+    if (arch->n_classes && arch->n_classes != net->def.classes) return SGS_EINVAL;
+    if (arch->stem_width && arch->stem_width != net->def.stem) return SGS_EINVAL;
+    for (int s = 0; s < net->def.n_stages; s++) {
+        if (arch->max_depth[s] && arch->max_depth[s] != net->def.max_depth[s]) return SGS_EINVAL;
+        if (arch->base_width[s] && arch->base_width[s] != net->def.width[s]) return SGS_EINVAL;
+    }
+    DeviceGuard guard(device);
+    if (!guard.ok) return SGS_ECUDA;
+
+    // walk the records against the family definition
+    std::vector<LayerSpec> specs = stored_layers(arch->family);
+    if ((size_t)words[3] != specs.size()) return SGS_EINVAL;
+    size_t pos = 8, total_words = nbytes / 4;
+    struct Rec { size_t w_off, bn_off, bias_off; };
+    std::vector<Rec> recs;
+    size_t arena = 0, params = 0;
+    for (const LayerSpec &sp : specs) {
+        if (pos + 8 > total_words) return SGS_EINVAL;
+        const uint32_t *h = words + pos;
+        if ((int)h[0] != sp.kind || (int)h[1] != sp.K || (int)h[2] != sp.C || (int)h[3] != sp.R || (int)h[4] != sp.R ||
+            (h[5] != 0) != sp.bn || (h[6] != 0) != sp.bias)
+            return SGS_EINVAL;
+        size_t nw = (size_t)sp.K * sp.C * sp.R * sp.R;
+        Rec r{pos + 8, 0, 0};
+        size_t q = pos + 8 + nw;
+        if (sp.bn) { r.bn_off = q; q += 4 * (size_t)sp.K; }
+        if (sp.bias) { r.bias_off = q; q += sp.K; }
+        if (q > total_words) return SGS_EINVAL;
+        pos = q;
+        recs.push_back(r);
+        arena += (nw * (compute_dtype == SGS_BF16 ? 2 : 4) + 255) / 256 * 256;
+        params += ((size_t)sp.K + 63) / 64 * 64 * 2;
+    }
+    if (pos != total_words) return SGS_EINVAL;
+
+    sgs_status_t st;
+    float *stage = nullptr;
+    if ((st = dev_alloc(net, (void **)&stage, nbytes)) != SGS_OK) return st;
+    auto cleanup_stage = [&]() { dev_free(net, stage, nbytes); };
+    if ((st = dev_alloc(net, (void **)&net->weight_arena, arena)) != SGS_OK) { cleanup_stage(); sgs_supernet_free(holder.release()); return st; }
+    net->weight_arena_bytes = arena;
+    if ((st = dev_alloc(net, (void **)&net->param_arena, params * 4)) != SGS_OK) { cleanup_stage(); sgs_supernet_free(holder.release()); return st; }
+    net->param_arena_bytes = params * 4;
+    cudaError_t e = cudaMemcpy(stage, host_blob, nbytes, cudaMemcpyHostToDevice);
+    size_t aoff = 0, poff = 0;
+    const int bf = compute_dtype == SGS_BF16;
+    for (size_t i = 0; i < specs.size() && e == cudaSuccess; i++) {
+        const LayerSpec &sp = specs[i];
+        StoredLayer L;
+        L.kind = sp.kind; L.K = sp.K; L.C = sp.C; L.R = sp.R; L.S = sp.R; L.has_bn = sp.bn; L.has_bias = sp.bias; L.name = sp.name;
+        size_t nw = (size_t)sp.K * sp.C * sp.R * sp.R;
+        L.w = net->weight_arena + aoff;
+        L.w_bytes = nw * net->elem();
+        aoff += (L.w_bytes + 255) / 256 * 256;
+        L.scale = net->param_arena + poff;
+        L.shift = L.scale + ((size_t)sp.K + 63) / 64 * 64;
+        poff += ((size_t)sp.K + 63) / 64 * 64 * 2;
+        const float *src = stage + recs[i].w_off;
+        if (sp.kind == KIND_CONV) e = launch_relayout_conv(src, L.w, sp.K, sp.C, sp.R, sp.R, bf, 0);
+        else if (sp.kind == KIND_DW) e = launch_relayout_dw(src, L.w, sp.K, sp.R, sp.R, bf, 0);
+        else e = launch_convert(src, L.w, nw, bf, 0);
+        if (e != cudaSuccess) break;
+        const float *bn = sp.bn ? stage + recs[i].bn_off : nullptr;
+        const float *bias = sp.bias ? stage + recs[i].bias_off : nullptr;
+        e = launch_fold_bn(bn, bn ? bn + sp.K : nullptr, bn ? bn + 2 * sp.K : nullptr, bn ? bn + 3 * sp.K : nullptr, bias,
+                           L.scale, L.shift, sp.K, 0);
+        net->by_name[sp.name] = (int)net->layers.size();
+        net->layers.push_back(L);
+    }
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    cleanup_stage();
+    if (e != cudaSuccess) { sgs_supernet_free(holder.release()); return e == cudaErrorMemoryAllocation ? SGS_ENOMEM : SGS_ECUDA; }
+
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrL2CacheSize, device) == cudaSuccess) net->l2_bytes = (size_t)v;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxPersistingL2CacheSize, device) == cudaSuccess) net->persist_max = (size_t)v;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxAccessPolicyWindowSize, device) == cudaSuccess) net->window_max = (size_t)v;
+    {
+        size_t n = 1 + 2 * net->layers.size();
+        if (dev_alloc(net, (void **)&net->cache_tbl, n * sizeof(int)) != SGS_OK ||
+            cudaMemset(net->cache_tbl, 0, n * sizeof(int)) != cudaSuccess) {
+            sgs_supernet_free(holder.release());
+            return SGS_ENOMEM;
+        }
+    }
+    if (compute_dtype == SGS_BF16 && tc_available() && tc_conv_init(device) != cudaSuccess) {
+        sgs_supernet_free(holder.release());
+        return SGS_ECUDA;
+    }
+    cache_reset(net, false, 0, 4);
+    *out = holder.release();
+    return SGS_OK;
+}
+
+void sgs_supernet_free(sgs_supernet_t *net) {
+    if (!net) return;
+    DeviceGuard guard(net->device);
+    cudaDeviceSynchronize();
+    for (auto &kv : net->plans)
+        if (kv.second->graph) cudaGraphExecDestroy(kv.second->graph);
+    net->plans.clear();
+    for (auto &r : net->prof_pending) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (auto &e : net->prof_pool) cudaEventDestroy(e);
+    cudaFree(net->weight_arena);
+    cudaFree(net->param_arena);
+    for (int i = 0; i < 4; i++) cudaFree(net->act[i]);
+    for (int i = 0; i < 3; i++) cudaFree(net->vec[i]);
+    cudaFree(net->cache_tbl);
+    cudaFree(net->splitk_ws);
+    cudaFree(net->splitk_counters);
+    cudaFree(net->host_stage_in);
+    cudaFree(net->host_stage_out);
+    delete net;
+}
+
+sgs_status_t sgs_subnet_validate(const sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg) {
+    if (!net || !cfg) return SGS_EINVAL;
+    return cfg_valid(net, cfg) ? SGS_OK : fail(net, SGS_ECONFIG, "SubNet config outside the elastic sets of this SuperNet");
+}
+
+int sgs_num_layers(const sgs_supernet_t *net) { return net ? (int)net->layers.size() : 0; }
+
+sgs_status_t sgs_subnet_encode(const sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, int *out) {
+    if (!net || !cfg || !out) return SGS_EINVAL;
+    if (!cfg_valid(net, cfg)) return fail(net, SGS_ECONFIG, "SubNet config outside the elastic sets of this SuperNet");
+    std::vector<int> e = encoding_of(slices_for(net, cfg));
+    std::memcpy(out, e.data(), e.size() * sizeof(int));
+    return SGS_OK;
+}
+
+sgs_status_t sgs_subnet_cost(const sgs_supernet_t *cnet, const sgs_subnet_cfg_t *cfg, int batch, int res, double *flops,
+                             double *weight_bytes, double *activation_bytes) {
+    sgs_supernet *net = const_cast<sgs_supernet *>(cnet);
+    if (!net || !cfg || batch <= 0 || res <= 0) return SGS_EINVAL;
+    if (!cfg_valid(net, cfg)) return fail(net, SGS_ECONFIG, "SubNet config outside the elastic sets of this SuperNet");
+    Plan p;
+    sgs_status_t st = build_plan(net, cfg, batch, res, &p);
+    if (st != SGS_OK) return st;
+    if (flops) *flops = p.flops;
+    if (weight_bytes) *weight_bytes = p.weight_bytes;
+    if (activation_bytes) *activation_bytes = p.act_bytes;
+    return SGS_OK;
+}
+
+sgs_status_t sgs_subnet_run(sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, const void *d_input, int batch, int res,
+                            void *d_logits, void *cuda_stream) {
+    if (!net) return SGS_EINVAL;
+    if (!cfg || !d_input || !d_logits || batch <= 0 || res < 8 || res > 1024) return fail(net, SGS_EINVAL, "bad argument");
+    DeviceGuard guard(net->device);
+    if (!guard.ok) return fail(net, SGS_ECUDA, "cudaSetDevice failed");
+    Plan *plan = nullptr;
+    sgs_status_t rc = run_query(net, cfg, d_input, batch, res, d_logits, (cudaStream_t)cuda_stream, false, &plan);
+    if (rc != SGS_OK) return rc;
+    if (net->cache.enabled) cache_observe(net, encoding_of(plan->slices));
+    return SGS_OK;
+}
+
+static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs, const void *inputs,
+                                int batch, int res, void *logits, const sgs_stream_opts_t *opts,
+                                sgs_stream_stats_t *stats, cudaStream_t st, bool host_buffers) {
+    if (!net) return SGS_EINVAL;
+    if (n_queries < 0 || (n_queries && (!cfgs || !inputs || !logits)) || batch <= 0 || res < 8 || res > 1024)
+        return fail(net, SGS_EINVAL, "bad argument");
+    DeviceGuard guard(net->device);
+    if (!guard.ok) return fail(net, SGS_ECUDA, "cudaSetDevice failed");
+    sgs_stream_opts_t o;
+    if (opts) o = *opts;
+    else { o.cache_enabled = 1; o.window_q = 4; o.cache_budget_bytes = 0; o.use_graphs = 1; o.record_latency = 1; o.weights_evict_first = 0; }
+    if (o.window_q < 1) return fail(net, SGS_EINVAL, "window_q must be >= 1");
+    for (int t = 0; t < n_queries; t++)
+        if (!cfg_valid(net, &cfgs[t])) return fail(net, SGS_ECONFIG, "query " + std::to_string(t) + ": config outside the elastic sets");
+    cache_reset(net, o.cache_enabled != 0, o.cache_budget_bytes, o.window_q);
+    net->cache.evict_first_when_off = (!o.cache_enabled && o.weights_evict_first) ? 1 : 0;
+
+    const size_t in_elems = (size_t)batch * res * res * 3, in_bytes = in_elems * net->elem();
+    const size_t out_bytes = (size_t)batch * net->def.classes * sizeof(float);
+    if (host_buffers) {
+        // two staging slots so that the copy of query t+1 can overlap query t
+        if (net->stage_in_bytes < 2 * in_bytes) {
+            dev_free(net, net->host_stage_in, net->stage_in_bytes);
+            net->host_stage_in = nullptr; net->stage_in_bytes = 0;
+            sgs_status_t rc = dev_alloc(net, &net->host_stage_in, 2 * in_bytes);
+            if (rc != SGS_OK) return rc;
+            net->stage_in_bytes = 2 * in_bytes;
+        }
+        if (net->stage_out_bytes < 2 * out_bytes) {
+            dev_free(net, net->host_stage_out, net->stage_out_bytes);
+            net->host_stage_out = nullptr; net->stage_out_bytes = 0;
+            sgs_status_t rc = dev_alloc(net, (void **)&net->host_stage_out, 2 * out_bytes);
+            if (rc != SGS_OK) return rc;
+            net->stage_out_bytes = 2 * out_bytes;
+        }
+    }
+    std::vector<cudaEvent_t> ev;
+    if (o.record_latency) {
+        ev.resize((size_t)n_queries + 1);
+        for (auto &e : ev) CU(cudaEventCreate(&e));
+    }
+    cudaEvent_t e0, e1;
+    CU(cudaEventCreate(&e0));
+    CU(cudaEventCreate(&e1));
+    const long long launches0 = net->kernel_launches;
+    const int hits0 = net->plan_hits, miss0 = net->plan_misses;
+    double flops = 0, wbytes = 0, miss_bytes = 0, hit = 0;
+    int updates = 0;
+    sgs_status_t rc = SGS_OK;
+    CU(cudaEventRecord(e0, st));
+    if (o.record_latency && n_queries) CU(cudaEventRecord(ev[0], st));
+    for (int t = 0; t < n_queries && rc == SGS_OK; t++) {
+        const void *din;
+        void *dout;
+        if (host_buffers) {
+            din = static_cast<char *>(net->host_stage_in) + (size_t)(t & 1) * in_bytes;
+            dout = reinterpret_cast<char *>(net->host_stage_out) + (size_t)(t & 1) * out_bytes;
+            cudaError_t ce = cudaMemcpyAsync(const_cast<void *>(din), static_cast<const char *>(inputs) + (size_t)t * in_bytes,
+                                             in_bytes, cudaMemcpyHostToDevice, st);
+            if (ce != cudaSuccess) { rc = fail(net, SGS_ECUDA, cudaGetErrorString(ce)); break; }
+        } else {
+            din = static_cast<const char *>(inputs) + (size_t)t * in_bytes;
+            dout = static_cast<char *>(logits) + (size_t)t * out_bytes;
+        }
+        Plan *plan = nullptr;
+        const int epoch_before = net->cache.epoch;
+        // the legacy default stream cannot be captured: run it without graphs
+        rc = run_query(net, &cfgs[t], din, batch, res, dout, st, o.use_graphs != 0 && st != nullptr, &plan);
+        if (rc != SGS_OK) break;
+        if (host_buffers) {
+            cudaError_t ce = cudaMemcpyAsync(static_cast<char *>(logits) + (size_t)t * out_bytes, dout, out_bytes,
+                                             cudaMemcpyDeviceToHost, st);
+            if (ce != cudaSuccess) { rc = fail(net, SGS_ECUDA, cudaGetErrorString(ce)); break; }
+        }
+        if (o.record_latency) {
+            cudaError_t ce = cudaEventRecord(ev[(size_t)t + 1], st);
+            if (ce != cudaSuccess) { rc = fail(net, SGS_ECUDA, cudaGetErrorString(ce)); break; }
+        }
+        std::vector<int> enc = encoding_of(plan->slices);
+        QueryAccount qa = account_query(net, enc);
+        flops += plan->flops; wbytes += qa.weight_bytes; miss_bytes += qa.miss_bytes; hit += qa.hit_ratio;
+        if (net->cache.enabled) {
+            cache_observe(net, enc);
+            if (net->cache.epoch != epoch_before) updates++;
+        }
+    }
+    cudaError_t ce = cudaEventRecord(e1, st);
+    cudaError_t se = cudaStreamSynchronize(st);
+    if (rc == SGS_OK && (ce != cudaSuccess || se != cudaSuccess))
+        rc = fail(net, SGS_ECUDA, std::string("stream: ") + cudaGetErrorString(se != cudaSuccess ? se : ce));
+    if (rc == SGS_OK && tc_conv_status()) rc = fail(net, SGS_ETIMEOUT, "a bounded device-side wait ran out in the tensor-core kernel");
+    if (rc == SGS_OK && stats) {
+        std::memset(stats, 0, sizeof(*stats));
+        float ms = 0;
+        cudaEventElapsedTime(&ms, e0, e1);
+        stats->n_queries = n_queries;
+        stats->total_ms = ms;
+        stats->queries_per_s = ms > 0 ? n_queries / (ms * 1e-3) : 0;
+        stats->images_per_s = stats->queries_per_s * batch;
+        if (o.record_latency && n_queries) {
+            std::vector<float> lat((size_t)n_queries);
+            double sum = 0;
+            for (int t = 0; t < n_queries; t++) { cudaEventElapsedTime(&lat[t], ev[t], ev[(size_t)t + 1]); sum += lat[t]; }
+            std::sort(lat.begin(), lat.end());
+            stats->p50_ms = lat[(size_t)(n_queries - 1) / 2];
+            stats->p99_ms = lat[(size_t)std::min<long long>(n_queries - 1, (long long)std::ceil(0.99 * n_queries) - 1)];
+            stats->mean_ms = sum / n_queries;
+        }
+        stats->useful_flops = flops;
+        stats->weight_bytes = wbytes;
+        stats->hbm_weight_bytes = miss_bytes;
+        stats->hit_ratio = n_queries ? hit / n_queries : 0;
+        stats->byte_hit_ratio = wbytes > 0 ? 1.0 - miss_bytes / wbytes : 0;
+        stats->kernel_launches = net->kernel_launches - launches0;
+        stats->plan_hits = net->plan_hits - hits0;
+        stats->plan_misses = net->plan_misses - miss0;
+        stats->cache_updates = updates;
+    }
+    for (auto &e : ev) cudaEventDestroy(e);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    return rc;
+}
+
+sgs_status_t sgs_stream_run(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs, const void *d_inputs,
+                            int batch_per_query, int res, void *d_logits, const sgs_stream_opts_t *opts,
+                            sgs_stream_stats_t *stats, void *cuda_stream) {
+    return stream_impl(net, n_queries, cfgs, d_inputs, batch_per_query, res, d_logits, opts, stats, (cudaStream_t)cuda_stream, false);
+}
+
+sgs_status_t sgs_stream_run_host(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs, const void *h_inputs,
+                                 int batch_per_query, int res, void *h_logits, const sgs_stream_opts_t *opts,
+                                 sgs_stream_stats_t *stats, void *cuda_stream) {
+    return stream_impl(net, n_queries, cfgs, h_inputs, batch_per_query, res, h_logits, opts, stats, (cudaStream_t)cuda_stream, true);
+}
+
+sgs_status_t sgs_cache_configure(sgs_supernet_t *net, int enabled, size_t budget_bytes, int window_q) {
+    if (!net) return SGS_EINVAL;
+    if (window_q < 1) return fail(net, SGS_EINVAL, "window_q must be >= 1");
+    cache_reset(net, enabled != 0, budget_bytes, window_q);
+    return SGS_OK;
+}
+
+sgs_status_t sgs_cache_stats(const sgs_supernet_t *net, sgs_cache_stats_t *out) {
+    if (!net || !out) return SGS_EINVAL;
+    std::memset(out, 0, sizeof(*out));
+    out->enabled = net->cache.enabled;
+    out->window_q = net->cache.window_q;
+    out->budget_bytes = net->cache.budget;
+    out->l2_bytes = net->l2_bytes;
+    out->persisting_l2_max = net->persist_max;
+    out->access_window_max = net->window_max;
+    out->cached_subgraph_bytes = net->cache.G_bytes;
+    out->supernet_bytes = net->weight_arena_bytes;
+    out->device_bytes_allocated = net->device_bytes;
+    return SGS_OK;
+}
+
+sgs_status_t sgs_profile_read(sgs_supernet_t *net, int kernel_class, long long *launches, double *total_ms,
+                              double *alg_bytes, double *flops) {
+    if (!net || kernel_class < 0 || kernel_class > 3) return SGS_EINVAL;
+    DeviceGuard guard(net->device);
+    fold_profile(net);
+    if (launches) *launches = net->prof_launches[kernel_class];
+    if (total_ms) *total_ms = net->prof_ms[kernel_class];
+    if (alg_bytes) *alg_bytes = net->prof_bytes[kernel_class];
+    if (flops) *flops = net->prof_flops[kernel_class];
+    return SGS_OK;
+}
+
+sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long value) {
+    if (!net || !name) return SGS_EINVAL;
+    std::string n(name);
+    if (n == "conv_impl") {
+        net->force_plain = value == 1;
+        DeviceGuard guard(net->device);
+        cudaDeviceSynchronize();
+        drop_graphs(net);
+        net->plans.clear();
+        return SGS_OK;
+    }
+    if (n == "profile") {
+        DeviceGuard guard(net->device);
+        fold_profile(net);
+        net->profile = value != 0;
+        if (value == 2 || value == 0)
+            for (int i = 0; i < 4; i++) { net->prof_ms[i] = net->prof_bytes[i] = net->prof_flops[i] = 0; net->prof_launches[i] = 0; }
+        return SGS_OK;
+    }
+    return fail(net, SGS_EINVAL, "unknown option " + n);
+}
+
+long long sgs_get_counter(const sgs_supernet_t *net, const char *name) {
+    if (!net || !name) return -1;
+    std::string n(name);
+    if (n == "kernel_launches") return net->kernel_launches;
+    if (n == "plan_hits") return net->plan_hits;
+    if (n == "plan_misses") return net->plan_misses;
+    if (n == "device_bytes") return (long long)net->device_bytes;
+    if (n == "tc_convs") {
+        long long c = 0;
+        for (auto &kv : net->plans)
+            for (const Op &op : kv.second->ops) c += op.impl == 1;
+        return c;
+    }
+    return -1;
+}
+
+const char *sgs_last_error(const sgs_supernet_t *net) { return net ? net->err.c_str() : "null handle"; }
+
+// Stand-alone sliced convolution.  The split-K scratch of the tensor-core kernel is one buffer per
+// device, grown on demand and shared by all calls of this function.
+sgs_status_t sgs_conv2d_sliced(const sgs_conv_desc_t *d, const void *d_x, const void *d_w, const float *d_scale,
+                               const float *d_shift, const void *d_res, void *d_y, void *cuda_stream) {
+    if (!d || !d_x || !d_w || !d_scale || !d_shift || !d_y) return SGS_EINVAL;
+    if (d->N <= 0 || d->H <= 0 || d->W <= 0 || d->C <= 0 || d->K <= 0 || d->k <= 0 || (d->k & 1) == 0 || d->k > d->R ||
+        ((d->R - d->k) & 1) || d->K > d->Kmax || (!d->depthwise && d->C > d->Cmax) || (d->stride != 1 && d->stride != 2) ||
+        (d->dtype != SGS_F32 && d->dtype != SGS_BF16) || d->act < 0 || d->act > 2 || d->impl < 0 || d->impl > 2)
+        return SGS_EINVAL;
+    ConvArgs a;
+    a.x = d_x; a.w = d_w; a.scale = d_scale; a.shift = d_shift; a.res = d_res; a.y = d_y;
+    a.N = d->N; a.H = d->H; a.W = d->W; a.C = d->depthwise ? d->K : d->C; a.K = d->K;
+    a.Kmax = d->Kmax; a.Cmax = d->depthwise ? 1 : d->Cmax; a.R = d->R; a.k = d->k; a.stride = d->stride; a.act = d->act;
+    const int p = (d->k - 1) / 2;
+    a.Ho = (d->H + 2 * p - d->k) / d->stride + 1;
+    a.Wo = (d->W + 2 * p - d->k) / d->stride + 1;
+    a.cacheK = d->cache_k; a.cacheC = d->cache_c; a.weight_policy = d->weight_policy;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    if (d->depthwise) {
+        if (d->impl == 2) return SGS_EUNSUPPORTED;
+        e = d->dtype == SGS_BF16 ? launch_dw<__nv_bfloat16>(a, st) : launch_dw<float>(a, st);
+        return e == cudaSuccess ? SGS_OK : SGS_ECUDA;
+    }
+    if (d->impl != 1 && d->dtype == SGS_BF16 && tc_available()) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SGS_ECUDA;
+        std::string why;
+        std::shared_ptr<TcConvPlan> plan = tc_conv_prepare(a, dev, &why);
+        if (plan) {
+            static float *ws[64] = {};
+            static unsigned *ctr[64] = {};
+            static size_t ws_elems[64] = {};
+            static unsigned n_ctr[64] = {};
+            const size_t need = d->split_k_off ? 0 : tc_conv_ws_elems(*plan);
+            const unsigned tiles = tc_conv_tiles(*plan);
+            if (need > ws_elems[dev] || (need && tiles > n_ctr[dev])) {
+                cudaFree(ws[dev]); cudaFree(ctr[dev]);
+                ws[dev] = nullptr; ctr[dev] = nullptr; ws_elems[dev] = 0; n_ctr[dev] = 0;
+                const unsigned nc = std::max(tiles, 4096u);
+                if (cudaMalloc((void **)&ws[dev], need * 4) != cudaSuccess) return SGS_ENOMEM;
+                if (cudaMalloc((void **)&ctr[dev], (size_t)nc * 4) != cudaSuccess) return SGS_ENOMEM;
+                if (cudaMemset(ctr[dev], 0, (size_t)nc * 4) != cudaSuccess) return SGS_ECUDA;
+                ws_elems[dev] = need; n_ctr[dev] = nc;
+            }
+            if (!d->split_k_off) { a.ws = ws[dev]; a.counters = ctr[dev]; a.ws_elems = ws_elems[dev]; a.n_counters = n_ctr[dev]; }
+            int n = 0;
+            e = tc_conv_launch(*plan, a, st, &n);
+            return e == cudaSuccess ? SGS_OK : SGS_ECUDA;
+        }
+    }
+    if (d->impl == 2) return SGS_EUNSUPPORTED;
+    e = d->dtype == SGS_BF16 ? launch_conv_plain<__nv_bfloat16>(a, st) : launch_conv_plain<float>(a, st);
+    return e == cudaSuccess ? SGS_OK : SGS_ECUDA;
+}
+
+int sgs_device_status(void) { return tc_conv_status(); }
+
+}  // extern "C"

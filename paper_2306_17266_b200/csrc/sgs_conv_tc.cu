@@ -1,0 +1,614 @@
+// Sliced convolution as an implicit GEMM on the 5th-generation tensor cores (tcgen05) of sm_100a.
+//
+//   D[m][f] = sum_{r,s} sum_{c<C'} x[n][ho*st + r - p][wo*st + s - p][c] * w[f][o+r][o+s][c],  f < K'
+//
+// GEMM view: M = output pixels (128 TMEM lanes per CTA), N = output filters (BN columns), K = taps x
+// channels.  Operands are staged in shared memory by TMA with the 128-byte swizzle; the accumulator
+// lives in tensor memory; an epilogue applies the folded batch norm, residual and activation and
+// stores bf16 NHWC.
+//
+// Slicing is folded into the TMA descriptors (paper Section 2.1: a SubNet only *selects* weights of
+// the SuperNet; Section 1: no SubNet is extracted): the weight map has the extents (C', R*R, K') of
+// the slice and the strides of the stored [Kmax][R][R][Cmax] tensor, so a tile that overhangs the
+// slice is zero-filled by the hardware and no sliced copy of a weight exists anywhere.
+//
+// Activation tiles are rectangular boxes (bw x bh x bn output pixels, <= 128) fetched per filter tap
+// with shifted box coordinates; image borders are the hardware's out-of-bounds zero fill.  Stride 2
+// reads one of four "parity" views of the input (even/odd rows x even/odd columns), each a plain
+// tensor map with doubled strides.
+//
+// SubGraph-Stationary reuse (paper Section 2.2, Section 4.2 Persistent / Dynamic Buffer): weight tiles
+// inside the cached SubGraph's prefix box (filter < cacheK and channel < cacheC) are loaded with an
+// L2 evict-last policy, all other weight tiles evict-first, so the shared weights stay on chip across
+// queries while the distinct weights of each SubNet stream through.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 =
+// epilogue (one TMEM lane quadrant each).  Every wait is bounded; when one runs out the kernel sets
+// a status word, lets its in-flight copies land, frees its tensor memory and returns.
+#include "sgs_internal.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+namespace sgs {
+
+namespace {
+
+constexpr int TILE_M = 128;   // output pixels per CTA (TMEM lanes)
+constexpr int CHUNK_C = 64;   // channels per pipeline stage (64 bf16 = one 128-byte swizzle row)
+constexpr int A_STAGE_BYTES = TILE_M * CHUNK_C * 2;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s per wait
+
+struct TcParams {
+    CUtensorMap tmA[4];  // activation views: [0] stride 1, or [ph*2+pw] parity views for stride 2
+    CUtensorMap tmW;     // sliced weight view (C', R*R, K')
+    const float *scale, *shift;
+    const __nv_bfloat16 *res;
+    __nv_bfloat16 *y;
+    float *ws;               // split-K workspace: [splits][M][K] fp32 partial tiles
+    unsigned *counters;      // one arrival counter per output tile (zero between launches)
+    int *status;             // device status word: nonzero after a bounded wait ran out
+    int N, Ho, Wo, K, C;     // output dims, sliced filters, sliced channels
+    int k, stride, R, o, p;  // kernel size, stride, stored kernel size, crop offset, padding
+    int bw, bh, bn;          // tile box in output pixels
+    int tiles_w, tiles_h;    // tiles along w and h (tiles along n = gridDim.x / (tiles_w*tiles_h))
+    int cchunks, iters;      // channel chunks per tap, total pipeline iterations (k*k*cchunks)
+    int splits, act;
+    int cacheK, cacheC, weight_policy;
+    const int *cache_tbl;    // optional device table overriding the three values above (see ConvArgs)
+    int layer;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false if the phase did not complete within WAIT_LIMIT_NS or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 64; i++)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ uint64_t make_policy(int kind) {  // 0 normal, 1 evict-last, 2 evict-first
+    uint64_t pol;
+    if (kind == 1) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    else if (kind == 2) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2,
+                                            int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_hint(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], "
+        "[%2], %6;"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t *v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes with the 128-byte
+// swizzle: start address >> 4, leading offset 1 (unused for swizzled K-major), stride offset
+// 1024 B (8 rows) >> 4, descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ float act_fn(float v, int act) {
+    if (act == ACT_RELU) return fmaxf(v, 0.f);
+    if (act == ACT_HSWISH) return v * fminf(fmaxf(v + 3.f, 0.f), 6.f) / 6.f;
+    return v;
+}
+
+// Folded batch norm, residual, activation and bf16 store of 8 consecutive filters of one pixel.
+template <int BN>
+__device__ __forceinline__ void finish8(float *o, const float *scale_s, const float *shift_s, int j0,
+                                        const __nv_bfloat16 *res, __nv_bfloat16 *y, size_t oi, int act) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) o[j] = o[j] * scale_s[j0 + j] + shift_s[j0 + j];
+    if (res) {
+        uint4 rv = *reinterpret_cast<const uint4 *>(res + oi);
+        const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+#pragma unroll
+        for (int j = 0; j < 4; j++) { float2 t = __bfloat1622float2(rb[j]); o[2 * j] += t.x; o[2 * j + 1] += t.y; }
+    }
+    uint4 ov;
+    __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+    for (int j = 0; j < 4; j++) ob[j] = __floats2bfloat162_rn(act_fn(o[2 * j], act), act_fn(o[2 * j + 1], act));
+    *reinterpret_cast<uint4 *>(y + oi) = ov;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The kernel.  grid = (m tiles, n tiles, K splits), block = 192.
+// Dynamic shared memory (1024-byte aligned): STAGES x [A tile 16 KB | B tile BN*128 B].
+// ---------------------------------------------------------------------------------------------
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__ TcParams p) {
+    constexpr int B_STAGE_BYTES = BN * CHUNK_C * 2;
+    constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+    constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s, last_s;
+    __shared__ float scale_s[BN], shift_s[BN];
+
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    volatile int *abort_flag = &abort_s;
+
+    // tile coordinates
+    const int tiles_hw = p.tiles_w * p.tiles_h;
+    const int tn = blockIdx.x / tiles_hw, th = (blockIdx.x % tiles_hw) / p.tiles_w, tw = blockIdx.x % p.tiles_w;
+    const int n0 = tn * p.bn, h0 = th * p.bh, w0 = tw * p.bw;
+    const int f0 = blockIdx.y * BN;
+    // K range of this split
+    const int per = (p.iters + p.splits - 1) / p.splits;
+    const int it_begin = blockIdx.z * per, it_end = min(p.iters, it_begin + per);
+    const int n_it = max(0, it_end - it_begin);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&accum_bar, 1);
+        abort_s = 0;
+        last_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(&tmem_base_s, BN);
+    if (warp >= 2) {
+        for (int j = threadIdx.x - 64; j < BN; j += 128) {
+            int f = f0 + j;
+            scale_s[j] = f < p.K ? p.scale[f] : 0.f;
+            shift_s[j] = f < p.K ? p.shift[f] : 0.f;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint64_t pol_keep = make_policy(1), pol_stream = make_policy(2), pol_norm = make_policy(0);
+            const uint32_t tx = (uint32_t)(p.bw * p.bh * p.bn * CHUNK_C * 2 + B_STAGE_BYTES);
+            int weight_policy = p.weight_policy, cacheK = p.cacheK, cacheC = p.cacheC;
+            if (p.cache_tbl) {
+                weight_policy = __ldg(p.cache_tbl);
+                cacheK = __ldg(p.cache_tbl + 1 + 2 * p.layer);
+                cacheC = __ldg(p.cache_tbl + 2 + 2 * p.layer);
+            }
+            for (int i = 0; i < n_it; i++) {
+                const int s = i % STAGES, round = i / STAGES;
+                if (round > 0 && !mbar_wait(&empty_bar[s], (round - 1) & 1, abort_flag)) break;
+                const int it = it_begin + i;
+                const int tap = it / p.cchunks, c0 = (it % p.cchunks) * CHUNK_C;
+                const int r = tap / p.k, sx = tap % p.k;
+                uint8_t *sa = smem + s * STAGE_BYTES, *sb = sa + A_STAGE_BYTES;
+                mbar_expect_tx(&full_bar[s], tx);
+                int dh = r - p.p, dw = sx - p.p;
+                if (p.stride == 1) {
+                    tma_load_4d(sa, &p.tmA[0], &full_bar[s], c0, w0 + dw, h0 + dh, n0);
+                } else {
+                    const int ph = dh & 1, pw = dw & 1;
+                    tma_load_4d(sa, &p.tmA[ph * 2 + pw], &full_bar[s], c0, w0 + ((dw - pw) >> 1), h0 + ((dh - ph) >> 1), n0);
+                }
+                uint64_t pol = pol_norm;
+                if (weight_policy == 1) pol = (f0 < cacheK && c0 < cacheC) ? pol_keep : pol_stream;
+                else if (weight_policy == 2) pol = pol_stream;
+                tma_load_3d_hint(sb, &p.tmW, &full_bar[s], c0, (p.o + r) * p.R + (p.o + sx), f0, pol);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            for (int i = 0; i < n_it && ok; i++) {
+                const int s = i % STAGES, round = i / STAGES;
+                ok = mbar_wait(&full_bar[s], round & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const int it = it_begin + i;
+                const int c0 = (it % p.cchunks) * CHUNK_C;
+                const int ksteps = (min(CHUNK_C, p.C - c0) + 15) / 16;
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_STAGE_BYTES;
+                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+                for (int q = 0; q < ksteps; q++)
+                    umma_bf16(tmem_base, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), IDESC, (i > 0 || q > 0) ? 1u : 0u);
+                umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+            }
+            if (ok) umma_commit(&accum_bar);  // accumulator complete
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quad = warp & 3;            // TMEM lane quadrant this warp may read
+        const int row = quad * 32 + lane;     // tile row = output pixel within the box
+        const int rows = p.bw * p.bh * p.bn;
+        const int dn = row / (p.bh * p.bw), dhh = (row / p.bw) % p.bh, dww = row % p.bw;
+        const int n = n0 + dn, h = h0 + dhh, w = w0 + dww;
+        const bool valid = row < rows && n < p.N && h < p.Ho && w < p.Wo;
+        const size_t m = valid ? ((size_t)n * p.Ho + h) * p.Wo + w : 0;
+        bool ok = n_it > 0 ? mbar_wait(&accum_bar, 0, abort_flag) : true;
+        ok = __all_sync(0xffffffffu, ok);
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        if (p.splits == 1) {
+            if (ok) {
+#pragma unroll 1
+                for (int j0 = 0; j0 < BN; j0 += 16) {
+                    if (f0 + j0 >= p.K) break;  // uniform across the CTA
+                    uint32_t v[16];
+                    tmem_ld16(taddr + j0, v);
+                    tmem_ld_wait();
+                    if (valid) {
+#pragma unroll
+                        for (int g = 0; g < 2; g++) {
+                            const int f = f0 + j0 + g * 8;
+                            if (f < p.K) {
+                                float o[8];
+#pragma unroll
+                                for (int j = 0; j < 8; j++) o[j] = __uint_as_float(v[g * 8 + j]);
+                                finish8<BN>(o, scale_s, shift_s, j0 + g * 8, p.res, p.y, m * p.K + f, p.act);
+                            }
+                        }
+                    }
+                }
+            }
+        } else {
+            // split K: every split stores its partial tile into its own slice of the fp32 workspace;
+            // the split that arrives last at the tile's counter sums the slices in split order (so the
+            // result does not depend on arrival order), applies the epilogue and resets the counter.
+            const size_t slice = (size_t)p.N * p.Ho * p.Wo * p.K;
+            if (ok && n_it > 0) {
+                float *part = p.ws + (size_t)blockIdx.z * slice;
+#pragma unroll 1
+                for (int j0 = 0; j0 < BN; j0 += 16) {
+                    if (f0 + j0 >= p.K) break;
+                    uint32_t v[16];
+                    tmem_ld16(taddr + j0, v);
+                    tmem_ld_wait();
+                    if (valid) {
+#pragma unroll
+                        for (int g = 0; g < 4; g++) {
+                            const int f = f0 + j0 + g * 4;
+                            if (f < p.K)
+                                __stcg(reinterpret_cast<float4 *>(part + m * p.K + f),
+                                       make_float4(__uint_as_float(v[g * 4]), __uint_as_float(v[g * 4 + 1]),
+                                                   __uint_as_float(v[g * 4 + 2]), __uint_as_float(v[g * 4 + 3])));
+                        }
+                    }
+                }
+            }
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 64) {
+                const unsigned tile = blockIdx.y * gridDim.x + blockIdx.x;
+                const unsigned prev = atomicAdd(&p.counters[tile], 1u);
+                last_s = (prev == (unsigned)p.splits - 1) ? 1 : 0;
+                if (last_s) p.counters[tile] = 0u;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (last_s) {
+                __threadfence();
+                const int live = (p.iters + per - 1) / per;  // splits that own at least one iteration
+                if (valid) {
+                    for (int j0 = 0; j0 < BN; j0 += 8) {
+                        const int f = f0 + j0;
+                        if (f >= p.K) break;
+                        const size_t oi = m * p.K + f;
+                        float o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                        for (int z = 0; z < live; z++) {
+                            const float *src = p.ws + (size_t)z * slice + oi;
+                            float4 a0 = __ldcg(reinterpret_cast<const float4 *>(src));
+                            float4 a1 = __ldcg(reinterpret_cast<const float4 *>(src + 4));
+                            o[0] += a0.x; o[1] += a0.y; o[2] += a0.z; o[3] += a0.w;
+                            o[4] += a1.x; o[5] += a1.y; o[6] += a1.z; o[7] += a1.w;
+                        }
+                        finish8<BN>(o, scale_s, shift_s, j0, p.res, p.y, oi, p.act);
+                    }
+                }
+            }
+        }
+    }
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (abort_s) {
+        // a wait ran out: report, give copies that may still be in flight time to land in this
+        // CTA's shared memory, then release the tensor memory
+        if (threadIdx.x == 0) atomicExch(p.status, 1);
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 2000000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, BN); }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+bool encode_map(CUtensorMap *m, const void *base, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
+                const uint32_t *box) {
+    cuuint64_t gd[5], gs[4];
+    cuuint32_t bx[5], es[5];
+    for (int i = 0; i < rank; i++) { gd[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i + 1 < rank; i++) gs[i] = strides_bytes[i];
+    CUresult r = encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), gd, gs, bx, es,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+struct DeviceScratch {
+    int *status = nullptr;
+    int sms = 0;
+    bool attrs_set = false;
+};
+DeviceScratch g_dev[64];
+std::mutex g_mu;
+int g_status_seen = 0;
+
+template <int BN, int STAGES> constexpr int smem_bytes() { return STAGES * (A_STAGE_BYTES + BN * CHUNK_C * 2) + 1024; }
+
+}  // namespace
+
+struct TcConvPlan {
+    TcParams prm;
+    dim3 grid;
+    int bn_tile = 128;
+    size_t ws_elems = 0;
+    unsigned n_tiles = 0;
+};
+
+bool tc_available() { return encode_fn() != nullptr; }
+size_t tc_conv_ws_elems(const TcConvPlan &p) { return p.ws_elems; }
+unsigned tc_conv_tiles(const TcConvPlan &p) { return p.n_tiles; }
+
+int tc_conv_status() {
+    std::lock_guard<std::mutex> lk(g_mu);
+    for (int d = 0; d < 64; d++) {
+        if (!g_dev[d].status) continue;
+        int v = 0;
+        int cur = -1;
+        cudaGetDevice(&cur);
+        if (cur != d) continue;  // only the current device's word is readable without switching
+        if (cudaMemcpy(&v, g_dev[d].status, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess && v) g_status_seen = 1;
+    }
+    return g_status_seen;
+}
+
+// Picks the output-pixel box (bw, bh, bn), bw*bh*bn <= 128, that wastes the fewest tile rows.
+static void choose_box(int N, int Ho, int Wo, int *bw_, int *bh_, int *bn_) {
+    double best = -1;
+    int bbw = 1, bbh = 1, bbn = 1;
+    for (int bw = 1; bw <= std::min(Wo, TILE_M); bw++) {
+        for (int bh = 1; bh <= std::min(Ho, TILE_M / bw); bh++) {
+            int bn = std::min(N, TILE_M / (bw * bh));
+            if (bn < 1) continue;
+            long long tiles = (long long)((Wo + bw - 1) / bw) * ((Ho + bh - 1) / bh) * ((N + bn - 1) / bn);
+            double util = (double)N * Ho * Wo / (double)(tiles * TILE_M);
+            double score = util + 1e-6 * bw;  // prefer long contiguous runs
+            if (score > best) { best = score; bbw = bw; bbh = bh; bbn = bn; }
+        }
+    }
+    *bw_ = bbw; *bh_ = bbh; *bn_ = bbn;
+}
+
+std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::string *why) {
+    auto no = [&](const char *msg) { if (why) *why = msg; return std::shared_ptr<TcConvPlan>(); };
+    if (!encode_fn()) return no("cuTensorMapEncodeTiled unavailable");
+    if (a.C % 8 || a.K % 8 || a.Cmax % 8) return no("channel counts must be multiples of 8");
+    if (a.C < 8 || a.K < 8) return no("too few channels");
+    if (a.k % 2 == 0 || a.k > a.R) return no("kernel size");
+    if (a.stride != 1 && a.stride != 2) return no("stride");
+    if (a.stride == 2 && ((a.H | a.W) & 1)) return no("stride 2 needs even input sizes");
+    if ((reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.w) | reinterpret_cast<uintptr_t>(a.y) |
+         reinterpret_cast<uintptr_t>(a.res)) & 15)
+        return no("pointers must be 16-byte aligned");
+    if (device < 0 || device >= 64) return no("device index");
+
+    auto plan = std::make_shared<TcConvPlan>();
+    TcParams &p = plan->prm;
+    std::memset(&p, 0, sizeof(p));
+    p.N = a.N; p.Ho = a.Ho; p.Wo = a.Wo; p.K = a.K; p.C = a.C;
+    p.k = a.k; p.stride = a.stride; p.R = a.R; p.o = (a.R - a.k) / 2; p.p = (a.k - 1) / 2;
+    p.act = a.act;
+    const bool flat = a.k == 1 && a.stride == 1;
+    const uint64_t C = (uint64_t)a.C, eb = 2;
+    if (flat) {
+        // 1x1 stride 1: the activation tensor is a plain [M][C] matrix, tiles are 128 consecutive pixels
+        const uint64_t M = (uint64_t)a.N * a.H * a.W;
+        p.bw = TILE_M; p.bh = 1; p.bn = 1;
+        p.N = 1; p.Ho = 1; p.Wo = (int)M;
+        uint64_t dims[4] = {C, M, 1, 1}, str[3] = {C * eb, M * C * eb, M * C * eb};
+        uint32_t box[4] = {CHUNK_C, TILE_M, 1, 1};
+        if (!encode_map(&p.tmA[0], a.x, 4, dims, str, box)) return no("activation tensor map");
+    } else {
+        choose_box(a.N, a.Ho, a.Wo, &p.bw, &p.bh, &p.bn);
+        uint32_t box[4] = {CHUNK_C, (uint32_t)p.bw, (uint32_t)p.bh, (uint32_t)p.bn};
+        if (a.stride == 1) {
+            uint64_t dims[4] = {C, (uint64_t)a.W, (uint64_t)a.H, (uint64_t)a.N};
+            uint64_t str[3] = {C * eb, (uint64_t)a.W * C * eb, (uint64_t)a.H * a.W * C * eb};
+            if (!encode_map(&p.tmA[0], a.x, 4, dims, str, box)) return no("activation tensor map");
+        } else {
+            for (int ph = 0; ph < 2; ph++)
+                for (int pw = 0; pw < 2; pw++) {
+                    const char *base = static_cast<const char *>(a.x) + ((size_t)ph * a.W + pw) * C * eb;
+                    uint64_t dims[4] = {C, (uint64_t)a.W / 2, (uint64_t)a.H / 2, (uint64_t)a.N};
+                    uint64_t str[3] = {2 * C * eb, 2 * (uint64_t)a.W * C * eb, (uint64_t)a.H * a.W * C * eb};
+                    if (!encode_map(&p.tmA[ph * 2 + pw], base, 4, dims, str, box)) return no("activation tensor map");
+                }
+        }
+    }
+    p.tiles_w = (p.Wo + p.bw - 1) / p.bw;
+    p.tiles_h = (p.Ho + p.bh - 1) / p.bh;
+    const int tiles_n = (p.N + p.bn - 1) / p.bn;
+    const int mtiles = p.tiles_w * p.tiles_h * tiles_n;
+
+    // filter tile: 128 wide unless the layer is narrow or too few CTAs would stream the weights
+    int sms = 148;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        DeviceScratch &ds = g_dev[device];
+        if (!ds.sms) cudaDeviceGetAttribute(&ds.sms, cudaDevAttrMultiProcessorCount, device);
+        if (ds.sms > 0) sms = ds.sms;
+    }
+    int BN = a.K <= 64 ? 64 : 128;
+    if (BN == 128 && mtiles * ((a.K + 127) / 128) < sms) BN = 64;
+    plan->bn_tile = BN;
+    {
+        uint64_t dims[3] = {C, (uint64_t)a.R * a.R, (uint64_t)a.K};
+        uint64_t str[2] = {(uint64_t)a.Cmax * eb, (uint64_t)a.R * a.R * a.Cmax * eb};
+        uint32_t box[3] = {CHUNK_C, 1, (uint32_t)BN};
+        if (!encode_map(&p.tmW, a.w, 3, dims, str, box)) return no("weight tensor map");
+    }
+    p.cchunks = (a.C + CHUNK_C - 1) / CHUNK_C;
+    p.iters = a.k * a.k * p.cchunks;
+    const int ntiles = (a.K + BN - 1) / BN;
+    // split the K loop when the tiles alone cannot fill the machine
+    int splits = 1;
+    const int ctas = mtiles * ntiles;
+    if (ctas < sms && p.iters >= 4) {
+        splits = std::min(std::min((sms + ctas - 1) / ctas, p.iters / 2), 8);
+        if (splits < 1) splits = 1;
+        // every split must own at least one iteration
+        while (splits > 1 && (p.iters + splits - 1) / splits * (splits - 1) >= p.iters) splits--;
+    }
+    p.splits = splits;
+    plan->grid = dim3((unsigned)mtiles, (unsigned)ntiles, (unsigned)splits);
+    plan->n_tiles = (unsigned)(mtiles * ntiles);
+    plan->ws_elems = splits > 1 ? (size_t)splits * a.N * a.Ho * a.Wo * a.K : 0;
+    return plan;
+}
+
+template <int BN, int STAGES> static cudaError_t launch_variant(const TcConvPlan &pl, const TcParams &prm, cudaStream_t st) {
+    conv_tc_kernel<BN, STAGES><<<pl.grid, 192, smem_bytes<BN, STAGES>(), st>>>(prm);
+    return cudaGetLastError();
+}
+
+// One-time set-up of the current device: status word and the kernels' shared-memory limits.  Must
+// run outside stream capture (it allocates).
+cudaError_t tc_conv_init(int dev) {
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceScratch &ds = g_dev[dev];
+    if (ds.attrs_set && ds.status) return cudaSuccess;
+    cudaError_t e;
+    if (!ds.status) {
+        if ((e = cudaMalloc(&ds.status, sizeof(int))) != cudaSuccess) return e;
+        if ((e = cudaMemset(ds.status, 0, sizeof(int))) != cudaSuccess) return e;
+    }
+    if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 4>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
+    ds.attrs_set = true;
+    return cudaSuccess;
+}
+
+cudaError_t tc_conv_launch(const TcConvPlan &pl, const ConvArgs &a, cudaStream_t st, int *launches) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if ((e = tc_conv_init(dev)) != cudaSuccess) return e;
+    TcParams prm = pl.prm;
+    prm.scale = a.scale; prm.shift = a.shift;
+    prm.res = static_cast<const __nv_bfloat16 *>(a.res);
+    prm.y = static_cast<__nv_bfloat16 *>(a.y);
+    prm.status = g_dev[dev].status;
+    prm.cacheK = a.cacheK; prm.cacheC = a.cacheC; prm.weight_policy = a.weight_policy;
+    prm.cache_tbl = a.cache_tbl; prm.layer = a.layer;
+    prm.ws = a.ws; prm.counters = a.counters;
+    if (prm.splits > 1 && (!a.ws || !a.counters || a.ws_elems < pl.ws_elems || a.n_counters < pl.n_tiles)) {
+        // no workspace: run unsplit
+        prm.splits = 1;
+    }
+    TcConvPlan run = pl;
+    run.grid.z = (unsigned)prm.splits;
+    if (pl.bn_tile == 64) e = launch_variant<64, 4>(run, prm, st);
+    else e = launch_variant<128, 3>(run, prm, st);
+    if (launches) *launches = 1;
+    return e;
+}
+
+}  // namespace sgs

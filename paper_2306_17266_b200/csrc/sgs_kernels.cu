@@ -1,0 +1,402 @@
+// Plain CUDA-core kernels: sliced convolution (shared-memory implicit GEMM in fp32), depthwise
+// convolution with centre-cropped kernels, pooling, squeeze-excite, linear layers, and the
+// load-time re-layout / batch-norm folding kernels.
+//
+// These are the complete path in fp32 mode and, in bf16 mode, serve the layers the tensor-core
+// kernel does not take (3-channel stems, channel counts that are not multiples of 8).
+#include "sgs_internal.h"
+
+#include <algorithm>
+
+namespace sgs {
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float apply_act(float v, int act) {
+    if (act == ACT_RELU) return fmaxf(v, 0.f);
+    if (act == ACT_HSWISH) return v * fminf(fmaxf(v + 3.f, 0.f), 6.f) / 6.f;
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sliced convolution as an implicit GEMM on CUDA cores.
+//   D[m][f] = sum_kk A[m][kk] * B[f][kk],  m = output pixel, f < K', kk = (r*k + s)*C' + c
+//   A[m][kk] = x[n][ho*st + r - p][wo*st + s - p][c]   (zero outside the image)
+//   B[f][kk] = w[f][o + r][o + s][c]                   (stored [Kmax][R][R][Cmax], o = (R-k)/2)
+// 64 x 64 output tile per block, 16-wide k chunks, 4 x 4 outputs per thread.
+// ---------------------------------------------------------------------------------------------
+constexpr int PT_M = 64, PT_N = 64, PT_K = 16;
+
+template <typename T>
+__global__ void __launch_bounds__(256) conv_plain_kernel(ConvArgs a) {
+    __shared__ float As[PT_K][PT_M + 4];
+    __shared__ float Bs[PT_K][PT_N + 4];
+    const T *__restrict__ x = static_cast<const T *>(a.x);
+    const T *__restrict__ w = static_cast<const T *>(a.w);
+    const int M = a.N * a.Ho * a.Wo;
+    const int KK = a.k * a.k * a.C;
+    const int p = (a.k - 1) / 2, o = (a.R - a.k) / 2;
+    const int m0 = blockIdx.x * PT_M, f0 = blockIdx.y * PT_N;
+    const int t = threadIdx.x;
+    const int lk = t % PT_K, lrow = t / PT_K;  // loader coordinates
+    const int tx = t % 16, ty = t / 16;        // compute coordinates
+
+    // decode the four pixels this thread loads
+    int pn[4], ph[4], pw[4];
+    bool pv[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        int m = m0 + lrow + 16 * j;
+        pv[j] = m < M;
+        int mm = pv[j] ? m : 0;
+        pw[j] = mm % a.Wo;
+        ph[j] = (mm / a.Wo) % a.Ho;
+        pn[j] = mm / (a.Wo * a.Ho);
+    }
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; i++)
+#pragma unroll
+        for (int j = 0; j < 4; j++) acc[i][j] = 0.f;
+
+    for (int kk0 = 0; kk0 < KK; kk0 += PT_K) {
+        const int kk = kk0 + lk;
+        const bool kv = kk < KK;
+        int c = 0, r = 0, s = 0;
+        if (kv) {
+            c = kk % a.C;
+            int rs = kk / a.C;
+            s = rs % a.k;
+            r = rs / a.k;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            float v = 0.f;
+            if (kv && pv[j]) {
+                int hi = ph[j] * a.stride + r - p, wi = pw[j] * a.stride + s - p;
+                if (hi >= 0 && hi < a.H && wi >= 0 && wi < a.W)
+                    v = to_f<T>(x[(((size_t)pn[j] * a.H + hi) * a.W + wi) * a.C + c]);
+            }
+            As[lk][lrow + 16 * j] = v;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            int f = f0 + lrow + 16 * j;
+            float v = 0.f;
+            if (kv && f < a.K) v = to_f<T>(w[(((size_t)f * a.R + (o + r)) * a.R + (o + s)) * a.Cmax + c]);
+            Bs[lk][lrow + 16 * j] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < PT_K; q++) {
+            float av[4], bv[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++) av[i] = As[q][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; j++) bv[j] = Bs[q][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; i++)
+#pragma unroll
+                for (int j = 0; j < 4; j++) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    const T *__restrict__ res = static_cast<const T *>(a.res);
+    T *__restrict__ y = static_cast<T *>(a.y);
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        int m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            int f = f0 + tx * 4 + j;
+            if (f >= a.K) continue;
+            float v = acc[i][j] * a.scale[f] + a.shift[f];
+            size_t oi = (size_t)m * a.K + f;
+            if (res) v += to_f<T>(res[oi]);
+            y[oi] = from_f<T>(apply_act(v, a.act));
+        }
+    }
+}
+
+template <typename T> cudaError_t launch_conv_plain(const ConvArgs &a, cudaStream_t st) {
+    int M = a.N * a.Ho * a.Wo;
+    if (M <= 0 || a.K <= 0) return cudaSuccess;
+    dim3 grid((M + PT_M - 1) / PT_M, (a.K + PT_N - 1) / PT_N);
+    conv_plain_kernel<T><<<grid, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+template cudaError_t launch_conv_plain<float>(const ConvArgs &, cudaStream_t);
+template cudaError_t launch_conv_plain<__nv_bfloat16>(const ConvArgs &, cudaStream_t);
+
+// ---------------------------------------------------------------------------------------------
+// Depthwise k x k convolution, kernel = centre window of the stored R x R kernel, weights
+// [R][R][Kmax].  One thread per (pixel, channel), channels fastest (coalesced NHWC).
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) dw_plain_kernel(ConvArgs a) {
+    const T *__restrict__ x = static_cast<const T *>(a.x);
+    const T *__restrict__ w = static_cast<const T *>(a.w);
+    T *__restrict__ y = static_cast<T *>(a.y);
+    const size_t total = (size_t)a.N * a.Ho * a.Wo * a.K;
+    const int p = (a.k - 1) / 2, o = (a.R - a.k) / 2;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        int c = (int)(i % a.K);
+        size_t m = i / a.K;
+        int wo = (int)(m % a.Wo), ho = (int)((m / a.Wo) % a.Ho), n = (int)(m / ((size_t)a.Wo * a.Ho));
+        float acc = 0.f;
+        for (int r = 0; r < a.k; r++) {
+            int hi = ho * a.stride + r - p;
+            if (hi < 0 || hi >= a.H) continue;
+            for (int s = 0; s < a.k; s++) {
+                int wi = wo * a.stride + s - p;
+                if (wi < 0 || wi >= a.W) continue;
+                acc = fmaf(to_f<T>(x[(((size_t)n * a.H + hi) * a.W + wi) * a.K + c]),
+                           to_f<T>(w[((size_t)(o + r) * a.R + (o + s)) * a.Kmax + c]), acc);
+            }
+        }
+        float v = acc * a.scale[c] + a.shift[c];
+        y[i] = from_f<T>(apply_act(v, a.act));
+    }
+}
+
+template <typename T> cudaError_t launch_dw(const ConvArgs &a, cudaStream_t st) {
+    size_t total = (size_t)a.N * a.Ho * a.Wo * a.K;
+    if (!total) return cudaSuccess;
+    int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
+    dw_plain_kernel<T><<<blocks, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+template cudaError_t launch_dw<float>(const ConvArgs &, cudaStream_t);
+template cudaError_t launch_dw<__nv_bfloat16>(const ConvArgs &, cudaStream_t);
+
+// ---------------------------------------------------------------------------------------------
+// 3x3 stride-2 max pool, padding 1 (only in-image taps compared)
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void maxpool_kernel(const T *__restrict__ x, T *__restrict__ y, int N, int H, int W, int C, int Ho, int Wo) {
+    size_t total = (size_t)N * Ho * Wo * C;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        int c = (int)(i % C);
+        size_t m = i / C;
+        int wo = (int)(m % Wo), ho = (int)((m / Wo) % Ho), n = (int)(m / ((size_t)Wo * Ho));
+        float best = -INFINITY;
+        for (int r = 0; r < 3; r++) {
+            int hi = 2 * ho + r - 1;
+            if (hi < 0 || hi >= H) continue;
+            for (int s = 0; s < 3; s++) {
+                int wi = 2 * wo + s - 1;
+                if (wi < 0 || wi >= W) continue;
+                best = fmaxf(best, to_f<T>(x[(((size_t)n * H + hi) * W + wi) * C + c]));
+            }
+        }
+        y[i] = from_f<T>(best);
+    }
+}
+template <typename T> cudaError_t launch_maxpool3s2(const T *x, T *y, int N, int H, int W, int C, cudaStream_t st) {
+    int Ho = (H - 1) / 2 + 1, Wo = (W - 1) / 2 + 1;
+    size_t total = (size_t)N * Ho * Wo * C;
+    if (!total) return cudaSuccess;
+    int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
+    maxpool_kernel<T><<<blocks, 256, 0, st>>>(x, y, N, H, W, C, Ho, Wo);
+    return cudaGetLastError();
+}
+template cudaError_t launch_maxpool3s2<float>(const float *, float *, int, int, int, int, cudaStream_t);
+template cudaError_t launch_maxpool3s2<__nv_bfloat16>(const __nv_bfloat16 *, __nv_bfloat16 *, int, int, int, int, cudaStream_t);
+
+// ---------------------------------------------------------------------------------------------
+// Global average pool: g[n][c] = mean_{hw} x[n][hw][c], fp32 result.
+// grid (ceil(C/32), N), block (32, 8): 8 pixel lanes per channel, reduced through shared memory.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void gap_kernel(const T *__restrict__ x, float *__restrict__ g, int HW, int C) {
+    __shared__ float part[8][33];
+    int c = blockIdx.x * 32 + threadIdx.x, n = blockIdx.y;
+    float s = 0.f;
+    if (c < C)
+        for (int i = threadIdx.y; i < HW; i += 8) s += to_f<T>(x[((size_t)n * HW + i) * C + c]);
+    part[threadIdx.y][threadIdx.x] = s;
+    __syncthreads();
+    if (threadIdx.y == 0 && c < C) {
+        float tot = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; j++) tot += part[j][threadIdx.x];
+        g[(size_t)n * C + c] = tot / (float)HW;
+    }
+}
+template <typename T> cudaError_t launch_gap(const T *x, float *g, int N, int HW, int C, cudaStream_t st) {
+    if (N <= 0 || C <= 0) return cudaSuccess;
+    dim3 grid((C + 31) / 32, N), block(32, 8);
+    gap_kernel<T><<<grid, block, 0, st>>>(x, g, HW, C);
+    return cudaGetLastError();
+}
+template cudaError_t launch_gap<float>(const float *, float *, int, int, int, cudaStream_t);
+template cudaError_t launch_gap<__nv_bfloat16>(const __nv_bfloat16 *, float *, int, int, int, cudaStream_t);
+
+// ---------------------------------------------------------------------------------------------
+// Squeeze-excite gate: z = relu(W1[:sq,:mid] g + b1), gate = hsigmoid(W2[:mid,:sq] z + b2).
+// One block per image; warps stride over outputs and reduce with shuffles.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) se_gate_kernel(const float *__restrict__ g, const T *__restrict__ w1,
+                                                      const float *__restrict__ b1, const T *__restrict__ w2,
+                                                      const float *__restrict__ b2, float *__restrict__ gate, int mid,
+                                                      int sq, int w1_ld, int w2_ld) {
+    extern __shared__ float sm[];
+    float *gs = sm, *zs = sm + mid;
+    int n = blockIdx.x, lane = threadIdx.x % 32, warp = threadIdx.x / 32, nw = blockDim.x / 32;
+    for (int c = threadIdx.x; c < mid; c += blockDim.x) gs[c] = g[(size_t)n * mid + c];
+    __syncthreads();
+    for (int j = warp; j < sq; j += nw) {
+        float s = 0.f;
+        for (int c = lane; c < mid; c += 32) s = fmaf(to_f<T>(w1[(size_t)j * w1_ld + c]), gs[c], s);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) zs[j] = fmaxf(s + b1[j], 0.f);
+    }
+    __syncthreads();
+    for (int c = warp; c < mid; c += nw) {
+        float s = 0.f;
+        for (int j = lane; j < sq; j += 32) s = fmaf(to_f<T>(w2[(size_t)c * w2_ld + j]), zs[j], s);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) gate[(size_t)n * mid + c] = fminf(fmaxf(s + b2[c] + 3.f, 0.f), 6.f) / 6.f;
+    }
+}
+template <typename T>
+cudaError_t launch_se_gate(const float *g, const T *w1, const float *b1, const T *w2, const float *b2, float *gate,
+                           int N, int mid, int sq, int w1_ld, int w2_ld, cudaStream_t st) {
+    if (N <= 0) return cudaSuccess;
+    se_gate_kernel<T><<<N, 256, (size_t)(mid + sq) * sizeof(float), st>>>(g, w1, b1, w2, b2, gate, mid, sq, w1_ld, w2_ld);
+    return cudaGetLastError();
+}
+template cudaError_t launch_se_gate<float>(const float *, const float *, const float *, const float *, const float *, float *, int, int, int, int, int, cudaStream_t);
+template cudaError_t launch_se_gate<__nv_bfloat16>(const float *, const __nv_bfloat16 *, const float *, const __nv_bfloat16 *, const float *, float *, int, int, int, int, int, cudaStream_t);
+
+// y[n][hw][c] = x[n][hw][c] * gate[n][c]
+template <typename T>
+__global__ void scale_kernel(const T *__restrict__ x, const float *__restrict__ gate, T *__restrict__ y, size_t total,
+                             int HW, int C) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        int c = (int)(i % C);
+        size_t n = i / ((size_t)HW * C);
+        y[i] = from_f<T>(to_f<T>(x[i]) * gate[n * C + c]);
+    }
+}
+template <typename T> cudaError_t launch_scale(const T *x, const float *gate, T *y, int N, int HW, int C, cudaStream_t st) {
+    size_t total = (size_t)N * HW * C;
+    if (!total) return cudaSuccess;
+    int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
+    scale_kernel<T><<<blocks, 256, 0, st>>>(x, gate, y, total, HW, C);
+    return cudaGetLastError();
+}
+template cudaError_t launch_scale<float>(const float *, const float *, float *, int, int, int, cudaStream_t);
+template cudaError_t launch_scale<__nv_bfloat16>(const __nv_bfloat16 *, const float *, __nv_bfloat16 *, int, int, int, cudaStream_t);
+
+// ---------------------------------------------------------------------------------------------
+// Sliced linear layer on fp32 vectors: y[n][j] = act(sum_{c<C} w[j][c] v[n][c] + bias[j]), j < K.
+// One warp per (n, j).
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) linear_kernel(const float *__restrict__ v, const T *__restrict__ w,
+                                                     const float *__restrict__ bias, float *__restrict__ y, int N,
+                                                     int C, int K, int ld, int act) {
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x % 32;
+    if (warp >= N * K) return;
+    int n = warp / K, j = warp % K;
+    float s = 0.f;
+    for (int c = lane; c < C; c += 32) s = fmaf(to_f<T>(w[(size_t)j * ld + c]), v[(size_t)n * C + c], s);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) y[(size_t)n * K + j] = apply_act(s + bias[j], act);
+}
+template <typename T>
+cudaError_t launch_linear(const float *v, const T *w, const float *bias, float *y, int N, int C, int K, int ld, int act,
+                          cudaStream_t st) {
+    long long warps = (long long)N * K;
+    if (warps <= 0) return cudaSuccess;
+    int blocks = (int)((warps * 32 + 255) / 256);
+    linear_kernel<T><<<blocks, 256, 0, st>>>(v, w, bias, y, N, C, K, ld, act);
+    return cudaGetLastError();
+}
+template cudaError_t launch_linear<float>(const float *, const float *, const float *, float *, int, int, int, int, int, cudaStream_t);
+template cudaError_t launch_linear<__nv_bfloat16>(const float *, const __nv_bfloat16 *, const float *, float *, int, int, int, int, int, cudaStream_t);
+
+// ---------------------------------------------------------------------------------------------
+// Load-time kernels
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void relayout_conv_kernel(const float *__restrict__ src, T *__restrict__ dst, int K, int C, int R, int S) {
+    size_t total = (size_t)K * C * R * S;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        // i indexes dst [K][R][S][C]
+        int c = (int)(i % C);
+        size_t q = i / C;
+        int s = (int)(q % S), r = (int)((q / S) % R), f = (int)(q / ((size_t)S * R));
+        dst[i] = from_f<T>(src[(((size_t)f * C + c) * R + r) * S + s]);
+    }
+}
+cudaError_t launch_relayout_conv(const float *src, void *dst, int K, int C, int R, int S, int bf16, cudaStream_t st) {
+    size_t total = (size_t)K * C * R * S;
+    int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 32);
+    if (bf16) relayout_conv_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(src, static_cast<__nv_bfloat16 *>(dst), K, C, R, S);
+    else relayout_conv_kernel<float><<<blocks, 256, 0, st>>>(src, static_cast<float *>(dst), K, C, R, S);
+    return cudaGetLastError();
+}
+
+template <typename T>
+__global__ void relayout_dw_kernel(const float *__restrict__ src, T *__restrict__ dst, int K, int R, int S) {
+    size_t total = (size_t)K * R * S;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        // dst [R][S][K], src [K][1][R][S]
+        int f = (int)(i % K);
+        size_t q = i / K;
+        dst[i] = from_f<T>(src[(size_t)f * R * S + q]);
+    }
+}
+cudaError_t launch_relayout_dw(const float *src, void *dst, int K, int R, int S, int bf16, cudaStream_t st) {
+    size_t total = (size_t)K * R * S;
+    int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 32);
+    if (bf16) relayout_dw_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(src, static_cast<__nv_bfloat16 *>(dst), K, R, S);
+    else relayout_dw_kernel<float><<<blocks, 256, 0, st>>>(src, static_cast<float *>(dst), K, R, S);
+    return cudaGetLastError();
+}
+
+template <typename T> __global__ void convert_kernel(const float *__restrict__ src, T *__restrict__ dst, size_t n) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = from_f<T>(src[i]);
+}
+cudaError_t launch_convert(const float *src, void *dst, size_t n, int bf16, cudaStream_t st) {
+    if (!n) return cudaSuccess;
+    int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 32);
+    if (bf16) convert_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(src, static_cast<__nv_bfloat16 *>(dst), n);
+    else convert_kernel<float><<<blocks, 256, 0, st>>>(src, static_cast<float *>(dst), n);
+    return cudaGetLastError();
+}
+
+// Batch-norm folding: scale = gamma / sqrt(var + 1e-5), shift = beta - mean * scale (+ bias).
+__global__ void fold_bn_kernel(const float *gamma, const float *beta, const float *mean, const float *var,
+                               const float *bias, float *scale, float *shift, int K) {
+    int f = blockIdx.x * blockDim.x + threadIdx.x;
+    if (f >= K) return;
+    float sc = 1.f, sh = 0.f;
+    if (gamma) {
+        sc = gamma[f] / sqrtf(var[f] + 1e-5f);
+        sh = beta[f] - mean[f] * sc;
+    }
+    if (bias) sh += bias[f];
+    scale[f] = sc;
+    shift[f] = sh;
+}
+cudaError_t launch_fold_bn(const float *gamma, const float *beta, const float *mean, const float *var,
+                           const float *bias, float *scale, float *shift, int K, cudaStream_t st) {
+    fold_bn_kernel<<<(K + 127) / 128, 128, 0, st>>>(gamma, beta, mean, var, bias, scale, shift, K);
+    return cudaGetLastError();
+}
+
+}  // namespace sgs
