@@ -1,0 +1,170 @@
+"""GPU parity: libsgs (through the C interface) against the CPU checker on the same seeded inputs.
+
+Tolerances: fp32 mode max|err| <= 1e-4 * max|ref| per output row; bf16 mode (fp32 accumulation, every
+stored tensor rounded to bf16) max|err| <= 2e-2 * max|ref| against the checker run with the same
+storage rounding points.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2306_17266_b200 as sgs
+from paper_2306_17266_b200 import workload as wl
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16 = 2e-2
+
+
+def test_library_reports_bad_arguments():
+    blob = wl.make_blob(wl.TINY, 0)
+    _, _, g = gu.nets(wl.TINY, False)
+    bad = wl.extreme_cfg(wl.TINY, True)
+    bad.width[2] = 0.6
+    assert g.subnet_validate(bad) == sgs.binding.SGS_ECONFIG
+    x = torch.zeros((1, 32, 32, 3), device="cuda")
+    out = torch.zeros((1, 10), device="cuda")
+    before = g.get_counter("kernel_launches")
+    with pytest.raises(sgs.SgsError) as e:
+        g.subnet_run(bad, x.data_ptr(), 1, 32, out.data_ptr())
+    assert e.value.status == sgs.binding.SGS_ECONFIG
+    assert g.get_counter("kernel_launches") == before  # nothing launched
+    with pytest.raises(sgs.SgsError):
+        sgs.SuperNet(wl.RESNET, blob)  # blob of another family
+    with pytest.raises(sgs.SgsError):
+        sgs.SuperNet(wl.TINY, blob[:-4])
+
+
+def test_tiny_fp32_all_queries():
+    _, onet, gnet = gu.nets(wl.TINY, False)
+    xs = wl.make_inputs(8, 1, 32, seed=1)
+    cfgs = wl.uniform_stream(wl.TINY, 8, seed=2)
+    for x, c in zip(xs, cfgs):
+        ref = onet.forward(c, x, oracle.FP32)
+        got = gu.gpu_forward(gnet, c, x, False)
+        assert gu.rel_err(got, ref) <= TOL_F32
+        np.testing.assert_array_equal(got.argmax(-1), ref.argmax(-1))
+
+
+def test_tiny_bf16_all_queries():
+    _, onet, gnet = gu.nets(wl.TINY, True)
+    xs = wl.make_inputs(8, 1, 32, seed=1, bf16=True)
+    cfgs = wl.uniform_stream(wl.TINY, 8, seed=2)
+    for x, c in zip(xs, cfgs):
+        ref = onet.forward(c, x, oracle.BF16_STORE)
+        got = gu.gpu_forward(gnet, c, x, True)
+        assert gu.rel_err(got, ref) <= TOL_BF16
+
+
+@pytest.mark.parametrize("fam", [wl.RESNET, wl.MBV3])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_small_resolution_configs(fam, bf16):
+    # 64x64 inputs keep the checker fast while every layer type, stride and elastic choice runs;
+    # batch 3 and an odd feature-map size (res 72 -> 9, 5, 3 in the last stages) give ragged tiles
+    _, onet, gnet = gu.nets(fam, bf16)
+    cfgs = wl.uniform_stream(fam, 4, seed=7) + [wl.extreme_cfg(fam, False), wl.extreme_cfg(fam, True)]
+    for i, c in enumerate(cfgs):
+        res, batch = (64, 3) if i % 2 == 0 else (72, 2)
+        x = wl.make_inputs(1, batch, res, seed=20 + i, bf16=bf16)[0]
+        ref = onet.forward(c, x, oracle.BF16_STORE if bf16 else oracle.FP32)
+        got = gu.gpu_forward(gnet, c, x, bf16)
+        assert np.all(np.isfinite(got))
+        assert gu.rel_err(got, ref) <= (TOL_BF16 if bf16 else TOL_F32), (fam, bf16, i)
+    if bf16 and fam == wl.RESNET:
+        assert gnet.get_counter("tc_convs") > 0  # the tensor-core kernel is the path that ran
+
+
+@pytest.mark.parametrize("fam", [wl.RESNET, wl.MBV3])
+def test_full_resolution_bf16(fam):
+    _, onet, gnet = gu.nets(fam, True)
+    cfgs = wl.uniform_stream(fam, 3, seed=2 if fam == wl.RESNET else 3)
+    xs = wl.make_inputs(3, 1, 224, seed=1, bf16=True)
+    for x, c in zip(xs, cfgs):
+        ref = onet.forward(c, x, oracle.BF16_STORE)
+        got = gu.gpu_forward(gnet, c, x, True)
+        assert gu.rel_err(got, ref) <= TOL_BF16
+
+
+def test_no_sliced_weight_copy_is_made():
+    # device memory owned by the handle does not change across configs once the workspace for the
+    # largest shape exists
+    _, _, gnet = gu.nets(wl.RESNET, True)
+    x = wl.make_inputs(1, 1, 64, seed=1, bf16=True)[0]
+    gu.gpu_forward(gnet, wl.extreme_cfg(wl.RESNET, True), x, True)
+    for c in wl.uniform_stream(wl.RESNET, 5, seed=31):
+        gu.gpu_forward(gnet, c, x, True)
+    base = gnet.get_counter("device_bytes")
+    for c in wl.uniform_stream(wl.RESNET, 8, seed=32):
+        gu.gpu_forward(gnet, c, x, True)
+    # only the split-reduction scratch may have grown, never by as much as the smallest sliced layer set
+    assert gnet.get_counter("device_bytes") - base < 4 << 20
+
+
+def test_stream_run_matches_single_queries_and_counts_bytes():
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    n, res = 12, 64
+    cfgs = wl.markov_stream(n, seed=4)
+    xs = wl.make_inputs(n, 1, res, seed=1, bf16=True)
+    singles = np.stack([gu.gpu_forward(gnet, c, x, True)[0] for c, x in zip(cfgs, xs)])
+    d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
+    d_out = torch.zeros((n, 1000), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()  # graphs cannot be captured on the legacy default stream
+    torch.cuda.synchronize()
+    for graphs in (0, 1):
+        for cache in (0, 1):
+            d_out.zero_()
+            torch.cuda.synchronize()
+            opts = sgs.StreamOpts(cache_enabled=cache, window_q=4, cache_budget_bytes=0, use_graphs=graphs, record_latency=1)
+            st = gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+            np.testing.assert_array_equal(d_out.cpu().numpy(), singles)  # deterministic, bit for bit
+            assert st.n_queries == n and st.kernel_launches > 0 and st.p50_ms > 0
+            encs = [onet.encode(c) for c in cfgs]
+            wbytes = sum(oracle.encoding_weights(e) for e in encs) * 2
+            assert abs(st.weight_bytes - wbytes) < 1
+            if cache:
+                assert 0 < st.hbm_weight_bytes < st.weight_bytes and 0 < st.hit_ratio <= 1
+            else:
+                assert st.hbm_weight_bytes == st.weight_bytes and st.hit_ratio == 0
+    # host-buffer variant
+    h_out = np.zeros((n, 1000), dtype=np.float32)
+    h_in = d_in.cpu().view(torch.int16).numpy()
+    gnet.stream_run(cfgs, h_in, 1, res, h_out, None, stream.cuda_stream, host=True)
+    np.testing.assert_array_equal(h_out, singles)
+
+
+def test_cache_accounting_matches_checker_formulas():
+    # hit ratio and missed bytes of a stream, recomputed from the checker's encodings and formulas
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    n, res, q = 16, 64, 4
+    cfgs = wl.markov_stream(n, seed=9)
+    d_in = gu.to_device(wl.make_inputs(n, 1, res, seed=2, bf16=True).reshape(n, res, res, 3), True)
+    d_out = torch.zeros((n, 1000), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    opts = sgs.StreamOpts(cache_enabled=1, window_q=q, cache_budget_bytes=0, use_graphs=0, record_latency=0)
+    st = gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+    encs = [onet.encode(c) for c in cfgs]
+    G, hits, missed = None, [], 0
+    for t, e in enumerate(encs):
+        if G is None:
+            hits.append(0.0)
+            missed += oracle.encoding_weights(e) * 2
+        else:
+            hits.append(oracle.hit_ratio(e, G))
+            missed += (oracle.encoding_weights(e) - oracle.encoding_weights(oracle.intersect(e, G))) * 2
+        if (t + 1) % q == 0:  # every q queries: G = intersection of the last q SubNets
+            G = encs[t - q + 1]
+            for f in encs[t - q + 2:t + 1]:
+                G = oracle.intersect(G, f)
+    assert abs(st.hit_ratio - np.mean(hits)) < 1e-9
+    assert abs(st.hbm_weight_bytes - missed) < 1
+
+
+def test_encoding_matches_checker():
+    for fam in (wl.TINY, wl.RESNET, wl.MBV3):
+        _, onet, gnet = gu.nets(fam, True)
+        for c in wl.uniform_stream(fam, 5, seed=3) + [wl.extreme_cfg(fam, False), wl.extreme_cfg(fam, True)]:
+            np.testing.assert_array_equal(gnet.subnet_encode(c), onet.encode(c))
