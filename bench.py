@@ -1,0 +1,283 @@
+#!/usr/bin/env python
+"""Benchmark of the SubNet query stream (ResNet-50-shaped SuperNet, batch 1, 224x224, bf16).
+
+    python bench.py --gpus N --steps K --warmup W            # this library
+    python bench.py --impl reference --steps K --warmup W    # the CPU checker on the host cores
+
+A step is one pass of the whole hot path over the query stream: `--queries` SubNet queries, each a
+different uniformly sampled SubNet config, through sgs_stream_run with inputs resident in HBM.
+Prints one JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2306_17266_b200 import workload as wl  # noqa: E402
+
+RES, BATCH = 224, 1
+METRIC, UNIT = "subnet_queries_per_s", "queries/s"
+WORKLOAD = "ResNet-50-shaped SuperNet, 1000-query stream at batch 1, 224x224x3, SubNets sampled uniformly (seed 2)"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_oracle_qps(n_queries: int):
+    """Times the CPU checker, as it stands, on the first queries of the same workload."""
+    import oracle
+    blob = wl.make_blob(wl.RESNET, seed=0, bf16_weights=True)
+    net = oracle.Net(wl.RESNET, blob)
+    cfgs = wl.uniform_stream(wl.RESNET, 1000, seed=2)[:n_queries]
+    xs = wl.make_inputs(n_queries, BATCH, RES, seed=1, bf16=True)
+    t0 = time.perf_counter()
+    for c, x in zip(cfgs, xs):
+        net.forward(c, x, oracle.BF16_STORE)
+    dt = time.perf_counter() - t0
+    return n_queries / dt, dt, oracle.num_threads()
+
+
+def run_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    per_step = max(1, args.ref_queries)
+    import oracle
+    blob = wl.make_blob(wl.RESNET, seed=0, bf16_weights=True)
+    net = oracle.Net(wl.RESNET, blob)
+    cfgs = wl.uniform_stream(wl.RESNET, 1000, seed=2)
+    xs = wl.make_inputs(per_step, BATCH, RES, seed=1, bf16=True)
+    k = 0
+    for _ in range(args.warmup):
+        net.forward(cfgs[k % 1000], xs[0], oracle.BF16_STORE)
+        k += 1
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        for i in range(per_step):
+            net.forward(cfgs[k % 1000], xs[i], oracle.BF16_STORE)
+            k += 1
+    dt = time.perf_counter() - t0
+    qps = args.steps * per_step / dt
+    sample = f"{per_step} queries per step of the same stream (a whole step is 1000 queries)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="sgs", choices=["sgs", "reference"])
+    ap.add_argument("--queries", type=int, default=1000, help="queries per step")
+    ap.add_argument("--cpu-queries", type=int, default=24, help="queries the CPU baseline is timed on (0 = skip)")
+    ap.add_argument("--ref-queries", type=int, default=8, help="queries per step of --impl reference")
+    ap.add_argument("--cache", type=int, default=1)
+    ap.add_argument("--window", type=int, default=4)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2306_17266_b200 as sgs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    peaks = measured_peaks()
+    nq = args.queries
+    warmup = max(3, args.warmup)
+    # replicas: every rank holds the SuperNet and serves its own query stream (no data-path collective)
+    blob = wl.make_blob(wl.RESNET, seed=0, bf16_weights=True)
+    net = sgs.SuperNet(wl.RESNET, blob, sgs.SGS_BF16, device=local)
+    base = wl.uniform_stream(wl.RESNET, 1000, seed=2)
+    cfgs = [base[(i + 131 * rank) % 1000] for i in range(nq)]
+    arr = wl.cfg_array(cfgs)
+    x_host = torch.from_numpy(wl.make_inputs(nq, BATCH, RES, seed=1 + rank, bf16=True).reshape(nq * BATCH, RES, RES, 3))
+    x_host = x_host.to(torch.bfloat16).contiguous().pin_memory()
+    x_dev = x_host.cuda()
+    logits = torch.zeros((nq * BATCH, 1000), dtype=torch.float32, device="cuda")
+    logits_host = torch.zeros((nq * BATCH, 1000), dtype=torch.float32).pin_memory()
+    stream = torch.cuda.Stream()
+
+    def mk_opts(graphs=1, latency=0):
+        return sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=graphs,
+                              record_latency=latency, weights_evict_first=0)
+
+    def step(host=False, o=None):
+        o = o or mk_opts()
+        if host:
+            return net.stream_run(arr, x_host.data_ptr(), BATCH, RES, logits_host.data_ptr(), o, stream.cuda_stream, host=True)
+        return net.stream_run(arr, x_dev.data_ptr(), BATCH, RES, logits.data_ptr(), o, stream.cuda_stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches = 0
+        e0.record(stream)
+        for _ in range(steps):
+            launches += fn().kernel_launches
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, launches
+
+    for _ in range(warmup):
+        step()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, launches = timed(step, args.steps)
+    clocks = sampler.stop()
+    value = world * nq * args.steps / (ms * 1e-3)
+
+    # latency distribution (one extra pass with per-query events)
+    st_lat = step(o=mk_opts(latency=1))
+
+    # end to end: host buffers in, host logits out, copies inside the timed region
+    step(host=True)
+    ms_e2e, _ = timed(lambda: step(host=True), args.steps)
+    e2e_value = world * nq * args.steps / (ms_e2e * 1e-3)
+    in_bytes = nq * BATCH * RES * RES * 3 * 2
+    out_bytes = nq * BATCH * 1000 * 4
+
+    out = None
+    if rank == 0:
+        # dominant kernel: CUDA events around every launch of one more pass, per kernel class
+        net.set_option("profile", 2)
+        step(o=mk_opts(graphs=0))
+        prof = [net.profile_read(c) for c in range(4)]
+        net.set_option("profile", 0)
+        tc = prof[0]
+        total_ms = sum(p["total_ms"] for p in prof)
+        sec = tc["total_ms"] * 1e-3
+        achieved_gbs = tc["alg_bytes"] / sec / 1e9 if sec > 0 else 0.0
+        achieved_tf = tc["flops"] / sec / 1e12 if sec > 0 else 0.0
+        roofline = {
+            "kernel": "conv_tc_kernel (sliced implicit-GEMM convolution, tcgen05 + TMA)", "bound": "hbm",
+            "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+            "launches": tc["launches"], "avg_launch_us": tc["total_ms"] * 1e3 / max(1, tc["launches"]),
+            "alg_bytes_per_launch": tc["alg_bytes"] / max(1, tc["launches"]),
+            "share_of_kernel_time": tc["total_ms"] / total_ms if total_ms > 0 else None,
+            "tensor_tflops": achieved_tf, "tensor_frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"],
+            "kernel_time_ms_by_class": {"conv_tc": prof[0]["total_ms"], "conv_cuda_core": prof[1]["total_ms"],
+                                        "depthwise": prof[2]["total_ms"], "other": prof[3]["total_ms"]},
+        }
+        cpu = None
+        if args.cpu_queries > 0 and world == 1:
+            qps, dt, cores = cpu_oracle_qps(args.cpu_queries)
+            cpu = {"value": qps, "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": f"first {args.cpu_queries} queries of the same stream, {dt:.1f} s"}
+        cs = net.cache_stats()
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "queries_per_step": nq, "batch": BATCH, "res": RES,
+                       "l2": "inputs (301 MB per step) and the SuperNet (96 MB) exceed L2; no flush",
+                       "cache": bool(args.cache), "window_q": args.window, "parallelism": f"replicas x{world}"},
+            "p50_ms": st_lat.p50_ms, "p99_ms": st_lat.p99_ms, "mean_ms": st_lat.mean_ms,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_bytes},
+            "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu,
+            "useful_tflops": st_lat.useful_flops / (st_lat.total_ms * 1e-3) / 1e12,
+            "sgs": {"weight_bytes_per_query": st_lat.weight_bytes / nq, "hbm_weight_bytes_per_query": st_lat.hbm_weight_bytes / nq,
+                    "hit_ratio": st_lat.hit_ratio, "byte_hit_ratio": st_lat.byte_hit_ratio, "cache_updates": st_lat.cache_updates,
+                    "budget_bytes": cs.budget_bytes, "l2_bytes": cs.l2_bytes},
+        }
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if out is not None:
+        print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()
