@@ -222,6 +222,36 @@ typedef struct {
 sgs_status_t sgs_conv2d_sliced(const sgs_conv_desc_t *desc, const void *d_x, const void *d_w, const float *d_scale,
                                const float *d_shift, const void *d_res, void *d_y, void *cuda_stream);
 
+/*
+ * sgs_conv2d_sliced_static - sgs_conv2d_sliced for callers that may not allocate device memory.
+ * (The paper has no counterpart to this call; it exists for the way the library is deployed.)
+ *
+ * Who needs it: code that runs while a stream is being captured into a CUDA graph, services that gave
+ * all device memory to their own pool at start-up, and latency-critical loops that cannot afford the
+ * device-wide synchronisation cudaMalloc and cudaFree imply.  sgs_conv2d_sliced may call cudaMalloc to
+ * grow its split-reduction scratch; this variant never does.  Its scratch is a fixed array of
+ * SGS_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the library
+ * holds that much memory until the process exits.
+ *
+ * Same arguments, layouts and result as sgs_conv2d_sliced, with these limits:
+ *   - tensor-core path only: dtype SGS_BF16, not depthwise, impl 0 or 2; otherwise SGS_EUNSUPPORTED
+ *     (also for shapes the tensor-core kernel does not take).
+ *   - a layer whose split reduction needs more than SGS_STATIC_SCRATCH_BYTES of partial tiles, or more
+ *     than 4096 output tiles, is rejected with SGS_ENOMEM and nothing is launched.  (Partial tiles take
+ *     splits * N*Ho*Wo*K * 4 bytes with splits <= 8; layers large enough to fill the GPU are not split
+ *     and need no scratch at all.  Set split_k_off = 1 to run any shape without scratch.)
+ *   - no cudaMalloc, cudaFree or other allocating device call is made, on any call.
+ * The first call on each device looks up the device address of the array and sets the kernels'
+ * shared-memory limit; make that first call outside any stream capture.  Later calls only enqueue a
+ * small memset (the arrival counters must start at zero) and the kernel on `cuda_stream`.
+ * All calls on a device share the one array and it keeps whatever the last call left in it: two calls
+ * whose kernels may overlap on the GPU (different streams, or concurrent host threads) race on it and
+ * give wrong results.  Issue them on one stream, or order them with events.
+ */
+#define SGS_STATIC_SCRATCH_BYTES (8u << 20)
+sgs_status_t sgs_conv2d_sliced_static(const sgs_conv_desc_t *desc, const void *d_x, const void *d_w, const float *d_scale,
+                                      const float *d_shift, const void *d_res, void *d_y, void *cuda_stream);
+
 /* Nonzero once a kernel of this process has reported that one of its bounded waits ran out. */
 int sgs_device_status(void);
 

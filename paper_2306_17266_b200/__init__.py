@@ -2,4 +2,4 @@
 seeded workload generators.  The CUDA library is loaded on first use, never at import."""
 from . import workload  # noqa: F401
 from .binding import (SGS_BF16, SGS_F32, CacheStats, ConvDesc, SgsError, StreamOpts, StreamStats, SuperNet,  # noqa: F401
-                      conv2d_sliced, device_status, lib)
+                      conv2d_sliced, conv2d_sliced_static, device_status, lib)

@@ -23,7 +23,7 @@ EXPORTS = [
     "sgs_supernet_load", "sgs_subnet_validate", "sgs_subnet_run", "sgs_stream_run", "sgs_stream_run_host",
     "sgs_cache_configure", "sgs_cache_stats", "sgs_num_layers", "sgs_subnet_encode", "sgs_subnet_cost",
     "sgs_set_option", "sgs_get_counter", "sgs_last_error", "sgs_supernet_free", "sgs_conv2d_sliced", "sgs_device_status",
-    "sgs_profile_read",
+    "sgs_profile_read", "sgs_conv2d_sliced_static",
 ]
 
 
@@ -94,6 +94,7 @@ def lib():
         L.sgs_supernet_free.argtypes = [vp]
         L.sgs_supernet_free.restype = None
         L.sgs_conv2d_sliced.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+        L.sgs_conv2d_sliced_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
         L.sgs_device_status.argtypes = []
         L.sgs_profile_read.argtypes = [vp, ci, vp, vp, vp, vp]
         _lib = L
@@ -115,6 +116,14 @@ def conv2d_sliced(desc: ConvDesc, d_x: int, d_w: int, d_scale: int, d_shift: int
     st = lib().sgs_conv2d_sliced(ctypes.byref(desc), d_x, d_w, d_scale, d_shift, d_res or None, d_y, stream)
     if st != SGS_OK:
         raise SgsError(st, "sgs_conv2d_sliced")
+
+
+def conv2d_sliced_static(desc: ConvDesc, d_x: int, d_w: int, d_scale: int, d_shift: int, d_res: int, d_y: int,
+                         stream: int = 0):
+    """The sliced convolution without any device allocation (fixed scratch inside the library)."""
+    st = lib().sgs_conv2d_sliced_static(ctypes.byref(desc), d_x, d_w, d_scale, d_shift, d_res or None, d_y, stream)
+    if st != SGS_OK:
+        raise SgsError(st, "sgs_conv2d_sliced_static")
 
 
 def device_status() -> int:

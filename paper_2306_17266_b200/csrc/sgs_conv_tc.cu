@@ -612,3 +612,95 @@ cudaError_t tc_conv_launch(const TcConvPlan &pl, const ConvArgs &a, cudaStream_t
 }
 
 }  // namespace sgs
+
+// =============================================================================================
+// Sliced convolution for callers that must not allocate device memory.
+//
+// Some users of this library run where cudaMalloc is off limits: inside a region that is being
+// captured into a CUDA graph, inside a serving process whose whole device memory was handed to a
+// pool at start-up, or in a latency-critical loop where an implicit device synchronisation (which
+// cudaMalloc / cudaFree cause) is not acceptable.  For them the split-reduction scratch of the
+// tensor-core kernel lives in a fixed array that is part of the loaded library image.
+// =============================================================================================
+namespace sgs {
+namespace {
+
+constexpr size_t STATIC_WS_FLOATS = SGS_STATIC_SCRATCH_BYTES / sizeof(float);
+constexpr unsigned STATIC_COUNTERS = 4096;
+
+struct StaticScratch {
+    float ws[STATIC_WS_FLOATS];          // partial tiles of the split reduction
+    unsigned counters[STATIC_COUNTERS];  // one arrival counter per output tile
+    int status;                          // set by a kernel whose bounded wait ran out
+};
+// Every GPU that loads the library holds this array until the process exits.
+static __device__ __align__(256) StaticScratch g_static_scratch;
+
+// Device address of the array per device.  In host code the symbol's name is only a handle; the
+// address a kernel can use has to be asked for with cudaGetSymbolAddress while that device is current.
+StaticScratch *g_static_ptr[64] = {};
+std::mutex g_static_mu;
+
+cudaError_t static_scratch_setup(int dev, StaticScratch **out) {
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        StaticScratch *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress((void **)&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 4>())) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
+        if ((e = cudaMemset(&ptr->status, 0, sizeof(int))) != cudaSuccess) return e;
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace sgs
+
+extern "C" sgs_status_t sgs_conv2d_sliced_static(const sgs_conv_desc_t *d, const void *d_x, const void *d_w,
+                                                 const float *d_scale, const float *d_shift, const void *d_res, void *d_y,
+                                                 void *cuda_stream) {
+    using namespace sgs;
+    if (!d || !d_x || !d_w || !d_scale || !d_shift || !d_y) return SGS_EINVAL;
+    if (d->N <= 0 || d->H <= 0 || d->W <= 0 || d->C <= 0 || d->K <= 0 || d->k <= 0 || (d->k & 1) == 0 || d->k > d->R ||
+        ((d->R - d->k) & 1) || d->K > d->Kmax || d->C > d->Cmax || (d->stride != 1 && d->stride != 2) || d->act < 0 || d->act > 2)
+        return SGS_EINVAL;
+    if (d->dtype != SGS_BF16 || d->depthwise || d->impl == 1 || !tc_available()) return SGS_EUNSUPPORTED;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SGS_ECUDA;
+    StaticScratch *sc = nullptr;
+    if (static_scratch_setup(dev, &sc) != cudaSuccess) return SGS_ECUDA;
+
+    ConvArgs a;
+    a.x = d_x; a.w = d_w; a.scale = d_scale; a.shift = d_shift; a.res = d_res; a.y = d_y;
+    a.N = d->N; a.H = d->H; a.W = d->W; a.C = d->C; a.K = d->K;
+    a.Kmax = d->Kmax; a.Cmax = d->Cmax; a.R = d->R; a.k = d->k; a.stride = d->stride; a.act = d->act;
+    const int p = (d->k - 1) / 2;
+    a.Ho = (d->H + 2 * p - d->k) / d->stride + 1;
+    a.Wo = (d->W + 2 * p - d->k) / d->stride + 1;
+    a.cacheK = d->cache_k; a.cacheC = d->cache_c; a.weight_policy = d->weight_policy;
+    std::shared_ptr<TcConvPlan> plan = tc_conv_prepare(a, dev, nullptr);  // host memory only
+    if (!plan) return SGS_EUNSUPPORTED;
+    TcParams prm = plan->prm;
+    if (d->split_k_off) prm.splits = 1;
+    if (prm.splits > 1 && (plan->ws_elems > STATIC_WS_FLOATS || plan->n_tiles > STATIC_COUNTERS))
+        return SGS_ENOMEM;  // the layer's split reduction does not fit SGS_STATIC_SCRATCH_BYTES
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (prm.splits > 1) {
+        // the counters must start at zero; an earlier call that was cut short could have left them dirty
+        if (cudaMemsetAsync(sc->counters, 0, (size_t)plan->n_tiles * sizeof(unsigned), st) != cudaSuccess) return SGS_ECUDA;
+    }
+    prm.scale = a.scale; prm.shift = a.shift;
+    prm.res = static_cast<const __nv_bfloat16 *>(a.res);
+    prm.y = static_cast<__nv_bfloat16 *>(a.y);
+    prm.status = &sc->status;
+    prm.cacheK = a.cacheK; prm.cacheC = a.cacheC; prm.weight_policy = a.weight_policy;
+    prm.cache_tbl = nullptr; prm.layer = 0;
+    prm.ws = sc->ws; prm.counters = sc->counters;
+    TcConvPlan run = *plan;
+    run.grid.z = (unsigned)prm.splits;
+    cudaError_t e = plan->bn_tile == 64 ? launch_variant<64, 4>(run, prm, st) : launch_variant<128, 3>(run, prm, st);
+    return e == cudaSuccess ? SGS_OK : SGS_ECUDA;
+}
