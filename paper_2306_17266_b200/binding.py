@@ -13,7 +13,7 @@ from typing import Optional, Sequence
 from .workload import ArchDesc, SubnetCfg, arch_desc, cfg_array
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsgs.so")
+LIB_PATH = os.environ.get("SGS_LIB") or os.path.join(_HERE, "libsgs.so")  # SGS_LIB: use another build of the library
 
 SGS_OK, SGS_EINVAL, SGS_ECONFIG, SGS_ENOMEM, SGS_ECUDA, SGS_ETIMEOUT, SGS_EUNSUPPORTED = range(7)
 SGS_F32, SGS_BF16 = 0, 1

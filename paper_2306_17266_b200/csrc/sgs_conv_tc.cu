@@ -121,6 +121,22 @@ __device__ __forceinline__ void tma_load_3d_hint(void *dst, const CUtensorMap *m
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+// True in exactly one lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -234,55 +250,63 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            const uint64_t pol_keep = make_policy(1), pol_stream = make_policy(2), pol_norm = make_policy(0);
-            const uint32_t tx = (uint32_t)(p.bw * p.bh * p.bn * CHUNK_C * 2 + B_STAGE_BYTES);
-            int weight_policy = p.weight_policy, cacheK = p.cacheK, cacheC = p.cacheC;
-            if (p.cache_tbl) {
-                weight_policy = __ldg(p.cache_tbl);
-                cacheK = __ldg(p.cache_tbl + 1 + 2 * p.layer);
-                cacheC = __ldg(p.cache_tbl + 2 + 2 * p.layer);
-            }
-            for (int i = 0; i < n_it; i++) {
-                const int s = i % STAGES, round = i / STAGES;
-                if (round > 0 && !mbar_wait(&empty_bar[s], (round - 1) & 1, abort_flag)) break;
-                const int it = it_begin + i;
-                const int tap = it / p.cchunks, c0 = (it % p.cchunks) * CHUNK_C;
-                const int r = tap / p.k, sx = tap % p.k;
-                uint8_t *sa = smem + s * STAGE_BYTES, *sb = sa + A_STAGE_BYTES;
+        // The whole warp runs the loop converged, so every operand of the copy instructions is a
+        // warp-uniform value; only the copy instructions themselves are issued by one elected lane.
+        const uint64_t pol_keep = make_policy(1), pol_stream = make_policy(2);
+        const uint32_t tx = (uint32_t)(p.bw * p.bh * p.bn * CHUNK_C * 2 + B_STAGE_BYTES);
+        int weight_policy = p.weight_policy, cacheK = p.cacheK, cacheC = p.cacheC;
+        if (p.cache_tbl) {
+            weight_policy = __ldg(p.cache_tbl);
+            cacheK = __ldg(p.cache_tbl + 1 + 2 * p.layer);
+            cacheC = __ldg(p.cache_tbl + 2 + 2 * p.layer);
+        }
+        // (tap row r, tap column sx, channel chunk cc) of iteration it_begin, then stepped
+        int cc = it_begin % p.cchunks, tap = it_begin / p.cchunks;
+        int r = tap / p.k, sx = tap % p.k;
+        for (int i = 0; i < n_it; i++) {
+            const int s = i % STAGES, round = i / STAGES;
+            bool ok = round == 0 || mbar_wait(&empty_bar[s], (round - 1) & 1, abort_flag);
+            if (!__all_sync(0xffffffffu, ok)) break;
+            const int c0 = cc * CHUNK_C;
+            uint8_t *sa = smem + s * STAGE_BYTES, *sb = sa + A_STAGE_BYTES;
+            const int dh = r - p.p, dw = sx - p.p;
+            const int tapw = (p.o + r) * p.R + (p.o + sx);
+            if (elect_one()) {
                 mbar_expect_tx(&full_bar[s], tx);
-                int dh = r - p.p, dw = sx - p.p;
                 if (p.stride == 1) {
                     tma_load_4d(sa, &p.tmA[0], &full_bar[s], c0, w0 + dw, h0 + dh, n0);
                 } else {
                     const int ph = dh & 1, pw = dw & 1;
                     tma_load_4d(sa, &p.tmA[ph * 2 + pw], &full_bar[s], c0, w0 + ((dw - pw) >> 1), h0 + ((dh - ph) >> 1), n0);
                 }
-                uint64_t pol = pol_norm;
-                if (weight_policy == 1) pol = (f0 < cacheK && c0 < cacheC) ? pol_keep : pol_stream;
-                else if (weight_policy == 2) pol = pol_stream;
-                tma_load_3d_hint(sb, &p.tmW, &full_bar[s], c0, (p.o + r) * p.R + (p.o + sx), f0, pol);
+                if (weight_policy == 0) tma_load_3d(sb, &p.tmW, &full_bar[s], c0, tapw, f0);
+                else tma_load_3d_hint(sb, &p.tmW, &full_bar[s], c0, tapw, f0,
+                                      (weight_policy == 1 && f0 < cacheK && c0 < cacheC) ? pol_keep : pol_stream);
             }
+            __syncwarp();
+            if (++cc == p.cchunks) { cc = 0; if (++sx == p.k) { sx = 0; ++r; } }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            bool ok = true;
-            for (int i = 0; i < n_it && ok; i++) {
-                const int s = i % STAGES, round = i / STAGES;
-                ok = mbar_wait(&full_bar[s], round & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                const int it = it_begin + i;
-                const int c0 = (it % p.cchunks) * CHUNK_C;
-                const int ksteps = (min(CHUNK_C, p.C - c0) + 15) / 16;
-                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_STAGE_BYTES;
-                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+        // Same structure: converged warp, one elected lane issues the MMAs and their commits.
+        bool ok = true;
+        int cc = it_begin % p.cchunks;
+        for (int i = 0; i < n_it; i++) {
+            const int s = i % STAGES, round = i / STAGES;
+            ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], round & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const int ksteps = (min(CHUNK_C, p.C - cc * CHUNK_C) + 15) / 16;
+            const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_STAGE_BYTES;
+            const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+            if (elect_one()) {
                 for (int q = 0; q < ksteps; q++)
                     umma_bf16(tmem_base, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), IDESC, (i > 0 || q > 0) ? 1u : 0u);
                 umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+                if (i == n_it - 1) umma_commit(&accum_bar);  // accumulator complete
             }
-            if (ok) umma_commit(&accum_bar);  // accumulator complete
+            __syncwarp();
+            if (++cc == p.cchunks) cc = 0;
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
