@@ -236,14 +236,15 @@ sgs_status_t sgs_conv2d_sliced(const sgs_conv_desc_t *desc, const void *d_x, con
  * Same arguments, layouts and result as sgs_conv2d_sliced, with these limits:
  *   - tensor-core path only: dtype SGS_BF16, not depthwise, impl 0 or 2; otherwise SGS_EUNSUPPORTED
  *     (also for shapes the tensor-core kernel does not take).
- *   - a layer whose split reduction needs more than SGS_STATIC_SCRATCH_BYTES of partial tiles, or more
- *     than 4096 output tiles, is rejected with SGS_ENOMEM and nothing is launched.  (Partial tiles take
+ *   - a layer whose split reduction needs more than SGS_STATIC_SCRATCH_BYTES of partial tiles is
+ *     rejected with SGS_ENOMEM and nothing is launched.  (Partial tiles take
  *     splits * N*Ho*Wo*K * 4 bytes with splits <= 8; layers large enough to fill the GPU are not split
  *     and need no scratch at all.  Set split_k_off = 1 to run any shape without scratch.)
  *   - no cudaMalloc, cudaFree or other allocating device call is made, on any call.
  * The first call on each device looks up the device address of the array and sets the kernels'
- * shared-memory limit; make that first call outside any stream capture.  Later calls only enqueue a
- * small memset (the arrival counters must start at zero) and the kernel on `cuda_stream`.
+ * shared-memory limit; make that first call outside any stream capture.  Later calls only enqueue
+ * kernels on `cuda_stream` (nothing in the array has to start at zero: what the second step of a
+ * split reduction reads was written by the first step of the same call).
  * All calls on a device share the one array and it keeps whatever the last call left in it: two calls
  * whose kernels may overlap on the GPU (different streams, or concurrent host threads) race on it and
  * give wrong results.  Issue them on one stream, or order them with events.

@@ -161,9 +161,7 @@ struct sgs_supernet {
     int *cache_tbl = nullptr;       // device: [policy, K_0, C_0, K_1, C_1, ...] read by the conv kernels
     int cache_tbl_epoch = -1;       // cache epoch the device table reflects
     float *splitk_ws = nullptr;     // split-K scratch of the tensor-core kernel
-    unsigned *splitk_counters = nullptr;
     size_t splitk_ws_elems = 0;
-    unsigned splitk_n_counters = 0;
     void *host_stage_in = nullptr;  // device staging for the host-buffer stream
     float *host_stage_out = nullptr;
     size_t stage_in_bytes = 0, stage_out_bytes = 0;
@@ -490,7 +488,6 @@ sgs_status_t ensure_workspace(sgs_supernet *net, size_t act_elems, int batch) {
 // tensor maps of the tensor-core kernel hold absolute addresses of the activation workspaces).
 sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
     size_t ws_need = 0;
-    unsigned ctr_need = 0;
     for (Op &op : plan->ops) {
         if (op.type != OP_CONV && op.type != OP_DW) continue;
         op.conv.x = op.in >= 0 ? net->act[op.in] : nullptr;
@@ -505,23 +502,16 @@ sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
         if (op.tc) {
             op.impl = 1;
             ws_need = std::max(ws_need, tc_conv_ws_elems(*op.tc));
-            if (tc_conv_ws_elems(*op.tc)) ctr_need = std::max(ctr_need, tc_conv_tiles(*op.tc));
         }
     }
-    if (ws_need > net->splitk_ws_elems || ctr_need > net->splitk_n_counters) {
+    if (ws_need > net->splitk_ws_elems) {
         drop_graphs(net);
-        const size_t we = std::max(ws_need, net->splitk_ws_elems);
-        const unsigned ce = std::max(ctr_need, std::max(net->splitk_n_counters, 1024u));
         dev_free(net, net->splitk_ws, net->splitk_ws_elems * 4);  // cudaFree waits for work in flight
-        dev_free(net, net->splitk_counters, (size_t)net->splitk_n_counters * 4);
-        net->splitk_ws = nullptr; net->splitk_counters = nullptr;
-        net->splitk_ws_elems = 0; net->splitk_n_counters = 0;
-        sgs_status_t st = dev_alloc(net, (void **)&net->splitk_ws, std::max<size_t>(we, 1) * 4);
+        net->splitk_ws = nullptr;
+        net->splitk_ws_elems = 0;
+        sgs_status_t st = dev_alloc(net, (void **)&net->splitk_ws, ws_need * 4);
         if (st != SGS_OK) return st;
-        st = dev_alloc(net, (void **)&net->splitk_counters, (size_t)ce * 4);
-        if (st != SGS_OK) return st;
-        CU(cudaMemset(net->splitk_counters, 0, (size_t)ce * 4));
-        net->splitk_ws_elems = std::max<size_t>(we, 1); net->splitk_n_counters = ce;
+        net->splitk_ws_elems = ws_need;
     }
     plan->prepared = true;
     return SGS_OK;
@@ -565,8 +555,7 @@ sgs_status_t run_ops(sgs_supernet *net, Plan *plan, const void *d_input, void *d
             ConvArgs a = op.conv;
             if (op.in < 0) a.x = d_input;
             a.cache_tbl = net->cache_tbl; a.layer = op.layer;
-            a.ws = net->splitk_ws; a.counters = net->splitk_counters;
-            a.ws_elems = net->splitk_ws_elems; a.n_counters = net->splitk_n_counters;
+            a.ws = net->splitk_ws; a.ws_elems = net->splitk_ws_elems;
             if (op.type == OP_DW) { CU(launch_dw<T>(a, st)); net->kernel_launches++; }
             else if (op.impl == 1) { int n = 0; CU(tc_conv_launch(*op.tc, a, st, &n)); net->kernel_launches += n; }
             else { CU(launch_conv_plain<T>(a, st)); net->kernel_launches++; }
@@ -906,7 +895,6 @@ void sgs_supernet_free(sgs_supernet_t *net) {
     for (int i = 0; i < 3; i++) cudaFree(net->vec[i]);
     cudaFree(net->cache_tbl);
     cudaFree(net->splitk_ws);
-    cudaFree(net->splitk_counters);
     cudaFree(net->host_stage_in);
     cudaFree(net->host_stage_out);
     delete net;
@@ -1195,21 +1183,15 @@ sgs_status_t sgs_conv2d_sliced(const sgs_conv_desc_t *d, const void *d_x, const 
         std::shared_ptr<TcConvPlan> plan = tc_conv_prepare(a, dev, &why);
         if (plan) {
             static float *ws[64] = {};
-            static unsigned *ctr[64] = {};
             static size_t ws_elems[64] = {};
-            static unsigned n_ctr[64] = {};
             const size_t need = d->split_k_off ? 0 : tc_conv_ws_elems(*plan);
-            const unsigned tiles = tc_conv_tiles(*plan);
-            if (need > ws_elems[dev] || (need && tiles > n_ctr[dev])) {
-                cudaFree(ws[dev]); cudaFree(ctr[dev]);
-                ws[dev] = nullptr; ctr[dev] = nullptr; ws_elems[dev] = 0; n_ctr[dev] = 0;
-                const unsigned nc = std::max(tiles, 4096u);
+            if (need > ws_elems[dev]) {
+                cudaFree(ws[dev]);
+                ws[dev] = nullptr; ws_elems[dev] = 0;
                 if (cudaMalloc((void **)&ws[dev], need * 4) != cudaSuccess) return SGS_ENOMEM;
-                if (cudaMalloc((void **)&ctr[dev], (size_t)nc * 4) != cudaSuccess) return SGS_ENOMEM;
-                if (cudaMemset(ctr[dev], 0, (size_t)nc * 4) != cudaSuccess) return SGS_ECUDA;
-                ws_elems[dev] = need; n_ctr[dev] = nc;
+                ws_elems[dev] = need;
             }
-            if (!d->split_k_off) { a.ws = ws[dev]; a.counters = ctr[dev]; a.ws_elems = ws_elems[dev]; a.n_counters = n_ctr[dev]; }
+            if (!d->split_k_off) { a.ws = ws[dev]; a.ws_elems = ws_elems[dev]; }
             int n = 0;
             e = tc_conv_launch(*plan, a, st, &n);
             return e == cudaSuccess ? SGS_OK : SGS_ECUDA;

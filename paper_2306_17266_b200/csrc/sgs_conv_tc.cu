@@ -48,7 +48,7 @@ struct TcParams {
     const __nv_bfloat16 *res;
     __nv_bfloat16 *y;
     float *ws;               // split-K workspace: [splits][M][K] fp32 partial tiles
-    unsigned *counters;      // one arrival counter per output tile (zero between launches)
+    size_t slice;            // M*K, elements of one workspace slice
     int *status;             // device status word: nonzero after a bounded wait ran out
     int N, Ho, Wo, K, C;     // output dims, sliced filters, sliced channels
     int k, stride, R, o, p;  // kernel size, stride, stored kernel size, crop offset, padding
@@ -163,6 +163,17 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t *v) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -180,12 +191,9 @@ __device__ __forceinline__ float act_fn(float v, int act) {
     return v;
 }
 
-// Folded batch norm, residual, activation and bf16 store of 8 consecutive filters of one pixel.
-template <int BN>
-__device__ __forceinline__ void finish8(float *o, const float *scale_s, const float *shift_s, int j0,
-                                        const __nv_bfloat16 *res, __nv_bfloat16 *y, size_t oi, int act) {
-#pragma unroll
-    for (int j = 0; j < 8; j++) o[j] = o[j] * scale_s[j0 + j] + shift_s[j0 + j];
+// Residual, activation and bf16 store of 8 consecutive filters of one pixel (o already holds
+// accumulator * scale + shift).
+__device__ __forceinline__ void finish_store(float *o, const __nv_bfloat16 *res, __nv_bfloat16 *y, size_t oi, int act) {
     if (res) {
         uint4 rv = *reinterpret_cast<const uint4 *>(res + oi);
         const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
@@ -207,11 +215,11 @@ template <int BN, int STAGES>
 __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__ TcParams p) {
     constexpr int B_STAGE_BYTES = BN * CHUNK_C * 2;
     constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
     extern __shared__ uint8_t smem_raw[];
+    __shared__ int row_m[TILE_M];  // output pixel index of each tile row, -1 outside the tensor
     __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s, last_s;
+    __shared__ int abort_s;
     __shared__ float scale_s[BN], shift_s[BN];
 
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -223,6 +231,9 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
     const int tn = blockIdx.x / tiles_hw, th = (blockIdx.x % tiles_hw) / p.tiles_w, tw = blockIdx.x % p.tiles_w;
     const int n0 = tn * p.bn, h0 = th * p.bh, w0 = tw * p.bw;
     const int f0 = blockIdx.y * BN;
+    // MMA shape: M = 128, N = this tile's filters rounded up to 16, bf16 x bf16 -> fp32, both K-major
+    const int n_mma = min(BN, (p.K - f0 + 15) & ~15);
+    const uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
     // K range of this split
     const int per = (p.iters + p.splits - 1) / p.splits;
     const int it_begin = blockIdx.z * per, it_end = min(p.iters, it_begin + per);
@@ -232,7 +243,6 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
         for (int s = 0; s < STAGES; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         mbar_init(&accum_bar, 1);
         abort_s = 0;
-        last_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(&tmem_base_s, BN);
@@ -310,90 +320,65 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // Each thread owns one tile row (= TMEM lane = output pixel).
         const int quad = warp & 3;            // TMEM lane quadrant this warp may read
         const int row = quad * 32 + lane;     // tile row = output pixel within the box
-        const int rows = p.bw * p.bh * p.bn;
-        const int dn = row / (p.bh * p.bw), dhh = (row / p.bw) % p.bh, dww = row % p.bw;
-        const int n = n0 + dn, h = h0 + dhh, w = w0 + dww;
-        const bool valid = row < rows && n < p.N && h < p.Ho && w < p.Wo;
-        const size_t m = valid ? ((size_t)n * p.Ho + h) * p.Wo + w : 0;
+        {
+            const int rows = p.bw * p.bh * p.bn;
+            const int dn = row / (p.bh * p.bw), dhh = (row / p.bw) % p.bh, dww = row % p.bw;
+            const int n = n0 + dn, h = h0 + dhh, w = w0 + dww;
+            const bool valid = row < rows && n < p.N && h < p.Ho && w < p.Wo;
+            row_m[row] = valid ? (int)(((size_t)n * p.Ho + h) * p.Wo + w) : -1;
+        }
         bool ok = n_it > 0 ? mbar_wait(&accum_bar, 0, abort_flag) : true;
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const int ncols = min(BN, p.K - f0);  // filters of this tile, a multiple of 8
         if (p.splits == 1) {
+            // straight from tensor memory to global memory: each thread finishes its own pixel row,
+            // 8 filters (16 bytes) per store
             if (ok) {
+                const int m = row_m[row];
 #pragma unroll 1
-                for (int j0 = 0; j0 < BN; j0 += 16) {
-                    if (f0 + j0 >= p.K) break;  // uniform across the CTA
-                    uint32_t v[16];
-                    tmem_ld16(taddr + j0, v);
+                for (int j0 = 0; j0 < ncols; j0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + j0, v);
                     tmem_ld_wait();
-                    if (valid) {
+                    if (m >= 0) {
 #pragma unroll
-                        for (int g = 0; g < 2; g++) {
-                            const int f = f0 + j0 + g * 8;
-                            if (f < p.K) {
+                        for (int g = 0; g < 4; g++) {
+                            const int c = j0 + 8 * g;
+                            if (c < ncols) {
                                 float o[8];
 #pragma unroll
-                                for (int j = 0; j < 8; j++) o[j] = __uint_as_float(v[g * 8 + j]);
-                                finish8<BN>(o, scale_s, shift_s, j0 + g * 8, p.res, p.y, m * p.K + f, p.act);
+                                for (int j = 0; j < 8; j++) o[j] = __uint_as_float(v[8 * g + j]) * scale_s[c + j] + shift_s[c + j];
+                                finish_store(o, p.res, p.y, (size_t)m * p.K + f0 + c, p.act);
                             }
                         }
                     }
                 }
             }
         } else {
-            // split K: every split stores its partial tile into its own slice of the fp32 workspace;
-            // the split that arrives last at the tile's counter sums the slices in split order (so the
-            // result does not depend on arrival order), applies the epilogue and resets the counter.
-            const size_t slice = (size_t)p.N * p.Ho * p.Wo * p.K;
+            // split K: this CTA covers only part of the reduction; it stores its fp32 partial tile into
+            // its own slice of the workspace and splitk_finish_kernel adds the slices in split order.
             if (ok && n_it > 0) {
-                float *part = p.ws + (size_t)blockIdx.z * slice;
+                const int m = row_m[row];
+                float *part = p.ws + (size_t)blockIdx.z * p.slice + (size_t)(m < 0 ? 0 : m) * p.K + f0;
 #pragma unroll 1
-                for (int j0 = 0; j0 < BN; j0 += 16) {
-                    if (f0 + j0 >= p.K) break;
-                    uint32_t v[16];
-                    tmem_ld16(taddr + j0, v);
+                for (int j0 = 0; j0 < ncols; j0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + j0, v);
                     tmem_ld_wait();
-                    if (valid) {
+                    if (m >= 0) {
 #pragma unroll
-                        for (int g = 0; g < 4; g++) {
-                            const int f = f0 + j0 + g * 4;
-                            if (f < p.K)
-                                __stcg(reinterpret_cast<float4 *>(part + m * p.K + f),
-                                       make_float4(__uint_as_float(v[g * 4]), __uint_as_float(v[g * 4 + 1]),
-                                                   __uint_as_float(v[g * 4 + 2]), __uint_as_float(v[g * 4 + 3])));
+                        for (int g = 0; g < 8; g++) {
+                            const int c = j0 + 4 * g;
+                            if (c < ncols)
+                                __stcg(reinterpret_cast<float4 *>(part + c),
+                                       make_float4(__uint_as_float(v[4 * g]), __uint_as_float(v[4 * g + 1]),
+                                                   __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3])));
                         }
-                    }
-                }
-            }
-            __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (threadIdx.x == 64) {
-                const unsigned tile = blockIdx.y * gridDim.x + blockIdx.x;
-                const unsigned prev = atomicAdd(&p.counters[tile], 1u);
-                last_s = (prev == (unsigned)p.splits - 1) ? 1 : 0;
-                if (last_s) p.counters[tile] = 0u;
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (last_s) {
-                __threadfence();
-                const int live = (p.iters + per - 1) / per;  // splits that own at least one iteration
-                if (valid) {
-                    for (int j0 = 0; j0 < BN; j0 += 8) {
-                        const int f = f0 + j0;
-                        if (f >= p.K) break;
-                        const size_t oi = m * p.K + f;
-                        float o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                        for (int z = 0; z < live; z++) {
-                            const float *src = p.ws + (size_t)z * slice + oi;
-                            float4 a0 = __ldcg(reinterpret_cast<const float4 *>(src));
-                            float4 a1 = __ldcg(reinterpret_cast<const float4 *>(src + 4));
-                            o[0] += a0.x; o[1] += a0.y; o[2] += a0.z; o[3] += a0.w;
-                            o[4] += a1.x; o[5] += a1.y; o[6] += a1.z; o[7] += a1.w;
-                        }
-                        finish8<BN>(o, scale_s, shift_s, j0, p.res, p.y, oi, p.act);
                     }
                 }
             }
@@ -411,6 +396,39 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
         __syncthreads();
     }
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, BN); }
+}
+
+// Second step of a split reduction: out = act(scale * (slice_0 + slice_1 + ...) + shift + res), the
+// slices added in split order so that the result is the same on every run.  One thread per 8 filters
+// of one pixel; all of a thread's loads are issued before the first add.
+__global__ void __launch_bounds__(256) splitk_finish_kernel(const float *__restrict__ ws, size_t slice, int live,
+                                                            const float *__restrict__ scale, const float *__restrict__ shift,
+                                                            const __nv_bfloat16 *res, __nv_bfloat16 *y, size_t groups, int K,
+                                                            int act) {
+    const size_t g = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
+    if (g >= groups) return;
+    const size_t oi = g * 8;
+    const int f = (int)(oi % (size_t)K);
+    float4 q[8][2];
+#pragma unroll
+    for (int z = 0; z < 8; z++) {
+        if (z < live) {
+            const float *src = ws + (size_t)z * slice + oi;
+            q[z][0] = __ldcg(reinterpret_cast<const float4 *>(src));
+            q[z][1] = __ldcg(reinterpret_cast<const float4 *>(src + 4));
+        }
+    }
+    float o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int z = 0; z < 8; z++) {
+        if (z < live) {
+            o[0] += q[z][0].x; o[1] += q[z][0].y; o[2] += q[z][0].z; o[3] += q[z][0].w;
+            o[4] += q[z][1].x; o[5] += q[z][1].y; o[6] += q[z][1].z; o[7] += q[z][1].w;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; j++) o[j] = o[j] * scale[f + j] + shift[f + j];
+    finish_store(o, res, y, oi, act);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -463,12 +481,10 @@ struct TcConvPlan {
     dim3 grid;
     int bn_tile = 128;
     size_t ws_elems = 0;
-    unsigned n_tiles = 0;
 };
 
 bool tc_available() { return encode_fn() != nullptr; }
 size_t tc_conv_ws_elems(const TcConvPlan &p) { return p.ws_elems; }
-unsigned tc_conv_tiles(const TcConvPlan &p) { return p.n_tiles; }
 
 int tc_conv_status() {
     std::lock_guard<std::mutex> lk(g_mu);
@@ -559,8 +575,17 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
         if (!ds.sms) cudaDeviceGetAttribute(&ds.sms, cudaDevAttrMultiProcessorCount, device);
         if (ds.sms > 0) sms = ds.sms;
     }
-    int BN = a.K <= 64 ? 64 : 128;
-    if (BN == 128 && mtiles * ((a.K + 127) / 128) < sms) BN = 64;
+    p.cchunks = (a.C + CHUNK_C - 1) / CHUNK_C;
+    p.iters = a.k * a.k * p.cchunks;
+    // Filter tile.  Issuing one MMA costs the issuing thread about the same whatever its width, so wide
+    // tiles are preferred as long as tiles x K splits can still occupy every SM.
+    // a split costs a second (small) kernel, so it has to save at least a dozen pipeline iterations
+    const int max_splits = p.iters >= 16 ? std::min(8, p.iters / 4) : 1;
+    int BN = 64;
+    for (int cand : {128}) {  // 256-wide tiles leave one CTA per SM, which this non-persistent kernel cannot afford
+        if (a.K <= cand / 2) continue;  // would be mostly padding
+        if ((long long)mtiles * ((a.K + cand - 1) / cand) * max_splits >= sms) { BN = cand; break; }
+    }
     plan->bn_tile = BN;
     {
         uint64_t dims[3] = {C, (uint64_t)a.R * a.R, (uint64_t)a.K};
@@ -568,23 +593,31 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
         uint32_t box[3] = {CHUNK_C, 1, (uint32_t)BN};
         if (!encode_map(&p.tmW, a.w, 3, dims, str, box)) return no("weight tensor map");
     }
-    p.cchunks = (a.C + CHUNK_C - 1) / CHUNK_C;
-    p.iters = a.k * a.k * p.cchunks;
     const int ntiles = (a.K + BN - 1) / BN;
     // split the K loop when the tiles alone cannot fill the machine
     int splits = 1;
     const int ctas = mtiles * ntiles;
-    if (ctas < sms && p.iters >= 4) {
-        splits = std::min(std::min((sms + ctas - 1) / ctas, p.iters / 2), 8);
+    if (ctas < sms && max_splits > 1) {
+        splits = std::min((sms + ctas - 1) / ctas, max_splits);
         if (splits < 1) splits = 1;
         // every split must own at least one iteration
         while (splits > 1 && (p.iters + splits - 1) / splits * (splits - 1) >= p.iters) splits--;
     }
     p.splits = splits;
+    p.slice = (size_t)a.N * a.Ho * a.Wo * a.K;
     plan->grid = dim3((unsigned)mtiles, (unsigned)ntiles, (unsigned)splits);
-    plan->n_tiles = (unsigned)(mtiles * ntiles);
     plan->ws_elems = splits > 1 ? (size_t)splits * a.N * a.Ho * a.Wo * a.K : 0;
     return plan;
+}
+
+// Launches the second step of a split reduction for the layer described by prm.
+static cudaError_t launch_finish(const TcParams &prm, cudaStream_t st) {
+    const int per = (prm.iters + prm.splits - 1) / prm.splits;
+    const int live = (prm.iters + per - 1) / per;  // splits that own at least one iteration
+    const size_t groups = prm.slice / 8;
+    splitk_finish_kernel<<<(unsigned)((groups + 255) / 256), 256, 0, st>>>(prm.ws, prm.slice, live, prm.scale, prm.shift, prm.res,
+                                                                         prm.y, groups, prm.K, prm.act);
+    return cudaGetLastError();
 }
 
 template <int BN, int STAGES> static cudaError_t launch_variant(const TcConvPlan &pl, const TcParams &prm, cudaStream_t st) {
@@ -606,6 +639,7 @@ cudaError_t tc_conv_init(int dev) {
     }
     if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 4>())) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(conv_tc_kernel<256, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<256, 4>())) != cudaSuccess) return e;
     ds.attrs_set = true;
     return cudaSuccess;
 }
@@ -622,16 +656,17 @@ cudaError_t tc_conv_launch(const TcConvPlan &pl, const ConvArgs &a, cudaStream_t
     prm.status = g_dev[dev].status;
     prm.cacheK = a.cacheK; prm.cacheC = a.cacheC; prm.weight_policy = a.weight_policy;
     prm.cache_tbl = a.cache_tbl; prm.layer = a.layer;
-    prm.ws = a.ws; prm.counters = a.counters;
-    if (prm.splits > 1 && (!a.ws || !a.counters || a.ws_elems < pl.ws_elems || a.n_counters < pl.n_tiles)) {
-        // no workspace: run unsplit
-        prm.splits = 1;
-    }
+    prm.ws = a.ws;
+    if (prm.splits > 1 && (!a.ws || a.ws_elems < pl.ws_elems)) prm.splits = 1;  // no workspace: run unsplit
     TcConvPlan run = pl;
     run.grid.z = (unsigned)prm.splits;
     if (pl.bn_tile == 64) e = launch_variant<64, 4>(run, prm, st);
-    else e = launch_variant<128, 3>(run, prm, st);
+    else if (pl.bn_tile == 128) e = launch_variant<128, 3>(run, prm, st);
+    else e = launch_variant<256, 4>(run, prm, st);
     if (launches) *launches = 1;
+    if (e != cudaSuccess || prm.splits == 1) return e;
+    e = launch_finish(prm, st);
+    if (launches) *launches = 2;
     return e;
 }
 
@@ -650,12 +685,10 @@ namespace sgs {
 namespace {
 
 constexpr size_t STATIC_WS_FLOATS = SGS_STATIC_SCRATCH_BYTES / sizeof(float);
-constexpr unsigned STATIC_COUNTERS = 4096;
 
 struct StaticScratch {
-    float ws[STATIC_WS_FLOATS];          // partial tiles of the split reduction
-    unsigned counters[STATIC_COUNTERS];  // one arrival counter per output tile
-    int status;                          // set by a kernel whose bounded wait ran out
+    float ws[STATIC_WS_FLOATS];  // partial tiles of the split reduction
+    int status;                  // set by a kernel whose bounded wait ran out
 };
 // Every GPU that loads the library holds this array until the process exits.
 static __device__ __align__(256) StaticScratch g_static_scratch;
@@ -673,6 +706,7 @@ cudaError_t static_scratch_setup(int dev, StaticScratch **out) {
         if (e != cudaSuccess) return e;
         if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 4>())) != cudaSuccess) return e;
         if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(conv_tc_kernel<256, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<256, 4>())) != cudaSuccess) return e;
         if ((e = cudaMemset(&ptr->status, 0, sizeof(int))) != cudaSuccess) return e;
         g_static_ptr[dev] = ptr;
     }
@@ -709,22 +743,23 @@ extern "C" sgs_status_t sgs_conv2d_sliced_static(const sgs_conv_desc_t *d, const
     if (!plan) return SGS_EUNSUPPORTED;
     TcParams prm = plan->prm;
     if (d->split_k_off) prm.splits = 1;
-    if (prm.splits > 1 && (plan->ws_elems > STATIC_WS_FLOATS || plan->n_tiles > STATIC_COUNTERS))
+    if (prm.splits > 1 && plan->ws_elems > STATIC_WS_FLOATS)
         return SGS_ENOMEM;  // the layer's split reduction does not fit SGS_STATIC_SCRATCH_BYTES
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (prm.splits > 1) {
-        // the counters must start at zero; an earlier call that was cut short could have left them dirty
-        if (cudaMemsetAsync(sc->counters, 0, (size_t)plan->n_tiles * sizeof(unsigned), st) != cudaSuccess) return SGS_ECUDA;
-    }
+    // Nothing in the array has to start at zero: every partial-tile element that is read back by the
+    // second step is written by the first step of the same call.
     prm.scale = a.scale; prm.shift = a.shift;
     prm.res = static_cast<const __nv_bfloat16 *>(a.res);
     prm.y = static_cast<__nv_bfloat16 *>(a.y);
     prm.status = &sc->status;
     prm.cacheK = a.cacheK; prm.cacheC = a.cacheC; prm.weight_policy = a.weight_policy;
     prm.cache_tbl = nullptr; prm.layer = 0;
-    prm.ws = sc->ws; prm.counters = sc->counters;
+    prm.ws = sc->ws;
     TcConvPlan run = *plan;
     run.grid.z = (unsigned)prm.splits;
-    cudaError_t e = plan->bn_tile == 64 ? launch_variant<64, 4>(run, prm, st) : launch_variant<128, 3>(run, prm, st);
+    cudaError_t e = plan->bn_tile == 64    ? launch_variant<64, 4>(run, prm, st)
+                    : plan->bn_tile == 128 ? launch_variant<128, 3>(run, prm, st)
+                                           : launch_variant<256, 4>(run, prm, st);
+    if (e == cudaSuccess && prm.splits > 1) e = launch_finish(prm, st);
     return e == cudaSuccess ? SGS_OK : SGS_ECUDA;
 }

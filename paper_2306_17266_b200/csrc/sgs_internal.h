@@ -56,12 +56,9 @@ struct ConvArgs {
     // (lets a captured graph follow cache updates without being re-captured)
     const int *cache_tbl = nullptr;
     int layer = 0;
-    // split-K scratch of the tensor-core kernel: fp32 partial tiles [splits][M][K] and per-tile
-    // arrival counters (zero between launches; the kernel resets them itself)
+    // split-K scratch of the tensor-core kernel: fp32 partial tiles [splits][M][K]
     float *ws = nullptr;
-    unsigned *counters = nullptr;
     size_t ws_elems = 0;
-    unsigned n_counters = 0;
 };
 
 enum OpType { OP_CONV, OP_DW, OP_MAXPOOL, OP_GAP, OP_SE_GATE, OP_SCALE, OP_LINEAR };
@@ -113,7 +110,6 @@ cudaError_t launch_fold_bn(const float *gamma, const float *beta, const float *m
 // Returns nullptr when the shape is not handled by the tensor-core kernel (caller falls back).
 std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::string *why);
 size_t tc_conv_ws_elems(const TcConvPlan &p);      // fp32 elements of split-K scratch the plan wants (0 = none)
-unsigned tc_conv_tiles(const TcConvPlan &p);       // arrival counters the plan wants
 cudaError_t tc_conv_launch(const TcConvPlan &p, const ConvArgs &a, cudaStream_t st, int *launches);
 cudaError_t tc_conv_init(int device);  // one-time device set-up; call outside stream capture
 bool tc_available();

@@ -55,9 +55,9 @@ def test_static_variant_matches_the_allocating_entry_point_twice(case):
 
 
 def test_static_variant_rejects_what_it_cannot_hold():
-    # 128 pixels x 9216 filters split in two: 9 MiB of fp32 partial sums, more than the fixed 8 MiB:
-    # refused, nothing launched
-    big = (2, 8, 8, 64, 64, 9216, 9216, 3, 3, 1, 0, False)
+    # 128 pixels x 9216 filters split three ways: 13.5 MiB of fp32 partial sums, more than the fixed
+    # 8 MiB: refused, nothing launched
+    big = (2, 8, 8, 128, 128, 9216, 9216, 3, 3, 1, 0, False)
     N, H, W, Cmax, C, Kmax, K, R, k, stride, act, _ = big
     x = torch.zeros((N, H, W, C), dtype=torch.bfloat16, device="cuda")
     w = torch.zeros((Kmax, R, R, Cmax), dtype=torch.bfloat16, device="cuda")
