@@ -168,8 +168,8 @@ def main():
     # replicas: every rank holds the SuperNet and serves its own query stream (no data-path collective)
     blob = wl.make_blob(wl.RESNET, seed=0, bf16_weights=True)
     net = sgs.SuperNet(wl.RESNET, blob, sgs.SGS_BF16, device=local)
-    base = wl.uniform_stream(wl.RESNET, 1000, seed=2)
-    cfgs = [base[(i + 131 * rank) % 1000] for i in range(nq)]
+    from paper_2306_17266_b200 import replicas
+    cfgs = replicas.rotated_stream(wl.uniform_stream(wl.RESNET, 1000, seed=2), rank, nq)
     arr = wl.cfg_array(cfgs)
     x_host = torch.from_numpy(wl.make_inputs(nq, BATCH, RES, seed=1 + rank, bf16=True).reshape(nq * BATCH, RES, RES, 3))
     x_host = x_host.to(torch.bfloat16).contiguous().pin_memory()
