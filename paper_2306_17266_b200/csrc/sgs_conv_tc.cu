@@ -137,6 +137,11 @@ __device__ __forceinline__ bool elect_one() {
         : "=r"(pred));
     return pred != 0;
 }
+// Programmatic dependent launch: wait() returns once the grids this one depends on have completed and
+// their writes are visible; launch_dependents() lets the next grid in the stream start its own prologue
+// early.  Both are no-ops for a grid that was launched without the attribute.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -257,6 +262,7 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
+    pdl_launch_dependents();  // the next layer may start its prologue and its weight loads now
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -273,25 +279,40 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
         // (tap row r, tap column sx, channel chunk cc) of iteration it_begin, then stepped
         int cc = it_begin % p.cchunks, tap = it_begin / p.cchunks;
         int r = tap / p.k, sx = tap % p.k;
+        auto load_weights = [&](int s, int c0, int tapw) {
+            uint8_t *sb = smem + s * STAGE_BYTES + A_STAGE_BYTES;
+            mbar_expect_tx(&full_bar[s], tx);
+            if (weight_policy == 0) tma_load_3d(sb, &p.tmW, &full_bar[s], c0, tapw, f0);
+            else tma_load_3d_hint(sb, &p.tmW, &full_bar[s], c0, tapw, f0,
+                                  (weight_policy == 1 && f0 < cacheK && c0 < cacheC) ? pol_keep : pol_stream);
+        };
+        // Weights do not depend on the previous layer: fill the first stages' weight halves before
+        // waiting for it, so that their latency overlaps the previous layer's tail.
+        {
+            int cc2 = cc, r2 = r, sx2 = sx;
+            const int pre = min(n_it, STAGES);
+            for (int i = 0; i < pre; i++) {
+                if (elect_one()) load_weights(i, cc2 * CHUNK_C, (p.o + r2) * p.R + (p.o + sx2));
+                __syncwarp();
+                if (++cc2 == p.cchunks) { cc2 = 0; if (++sx2 == p.k) { sx2 = 0; ++r2; } }
+            }
+        }
+        pdl_wait();  // activations (and the buffers this layer overwrites) belong to the previous layers until here
         for (int i = 0; i < n_it; i++) {
             const int s = i % STAGES, round = i / STAGES;
             bool ok = round == 0 || mbar_wait(&empty_bar[s], (round - 1) & 1, abort_flag);
             if (!__all_sync(0xffffffffu, ok)) break;
             const int c0 = cc * CHUNK_C;
-            uint8_t *sa = smem + s * STAGE_BYTES, *sb = sa + A_STAGE_BYTES;
+            uint8_t *sa = smem + s * STAGE_BYTES;
             const int dh = r - p.p, dw = sx - p.p;
-            const int tapw = (p.o + r) * p.R + (p.o + sx);
             if (elect_one()) {
-                mbar_expect_tx(&full_bar[s], tx);
+                if (round > 0) load_weights(s, c0, (p.o + r) * p.R + (p.o + sx));
                 if (p.stride == 1) {
                     tma_load_4d(sa, &p.tmA[0], &full_bar[s], c0, w0 + dw, h0 + dh, n0);
                 } else {
                     const int ph = dh & 1, pw = dw & 1;
                     tma_load_4d(sa, &p.tmA[ph * 2 + pw], &full_bar[s], c0, w0 + ((dw - pw) >> 1), h0 + ((dh - ph) >> 1), n0);
                 }
-                if (weight_policy == 0) tma_load_3d(sb, &p.tmW, &full_bar[s], c0, tapw, f0);
-                else tma_load_3d_hint(sb, &p.tmW, &full_bar[s], c0, tapw, f0,
-                                      (weight_policy == 1 && f0 < cacheK && c0 < cacheC) ? pol_keep : pol_stream);
             }
             __syncwarp();
             if (++cc == p.cchunks) { cc = 0; if (++sx == p.k) { sx = 0; ++r; } }
@@ -330,6 +351,7 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
             const bool valid = row < rows && n < p.N && h < p.Ho && w < p.Wo;
             row_m[row] = valid ? (int)(((size_t)n * p.Ho + h) * p.Wo + w) : -1;
         }
+        pdl_wait();  // residual reads and output writes must not pass the previous layers
         bool ok = n_it > 0 ? mbar_wait(&accum_bar, 0, abort_flag) : true;
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after();
@@ -621,8 +643,17 @@ static cudaError_t launch_finish(const TcParams &prm, cudaStream_t st) {
 }
 
 template <int BN, int STAGES> static cudaError_t launch_variant(const TcConvPlan &pl, const TcParams &prm, cudaStream_t st) {
-    conv_tc_kernel<BN, STAGES><<<pl.grid, 192, smem_bytes<BN, STAGES>(), st>>>(prm);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = pl.grid;
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = smem_bytes<BN, STAGES>();
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, conv_tc_kernel<BN, STAGES>, prm);
 }
 
 // One-time set-up of the current device: status word and the kernels' shared-memory limits.  Must
