@@ -192,7 +192,7 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
 
 __device__ __forceinline__ float act_fn(float v, int act) {
     if (act == ACT_RELU) return fmaxf(v, 0.f);
-    if (act == ACT_HSWISH) return v * fminf(fmaxf(v + 3.f, 0.f), 6.f) / 6.f;
+    if (act == ACT_HSWISH) return v * fminf(fmaxf(v + 3.f, 0.f), 6.f) * (1.f / 6.f);
     return v;
 }
 

@@ -19,7 +19,7 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float
 
 __device__ __forceinline__ float apply_act(float v, int act) {
     if (act == ACT_RELU) return fmaxf(v, 0.f);
-    if (act == ACT_HSWISH) return v * fminf(fmaxf(v + 3.f, 0.f), 6.f) / 6.f;
+    if (act == ACT_HSWISH) return v * fminf(fmaxf(v + 3.f, 0.f), 6.f) * (1.f / 6.f);
     return v;
 }
 
@@ -165,9 +165,104 @@ __global__ void __launch_bounds__(256) dw_plain_kernel(ConvArgs a) {
     }
 }
 
+// Vectorised bf16 depthwise convolution.  A thread owns 8 channels (one 16-byte vector) of TW = 4
+// neighbouring output pixels of one output row: per filter row it loads the (TW-1)*ST + K input
+// columns once and uses each for every tap it belongs to, so global loads per output drop from K*K
+// to about K*(1 + (K-1)/(TW*ST)); neighbouring threads cover neighbouring channel vectors, so every
+// load and store of a warp is one contiguous run.  fp32 accumulation with packed 2-wide FMAs.
+// HBM traffic per output element: 2 B read + 2 B written (rows are re-read from L1/L2, not DRAM).
+__device__ __forceinline__ float2 bf2_lo(uint32_t u) { return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)); }
+
+template <int K, int ST>
+__global__ void __launch_bounds__(256) dw_vec_kernel(ConvArgs a) {
+    constexpr int TW = 4, NCOL = (TW - 1) * ST + K, P = (K - 1) / 2;
+    // grid: x covers (channel vector, pixel block) of one output row, y = output row, z = image;
+    // all index arithmetic stays in 32 bits
+    const int groups = a.K / 8, wblocks = (a.Wo + TW - 1) / TW;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= groups * wblocks) return;
+    const int cg = idx % groups, wb = idx / groups;
+    const int ho = blockIdx.y, n = blockIdx.z;
+    const int c0 = cg * 8, wo0 = wb * TW, o = (a.R - K) / 2;
+    const __nv_bfloat16 *__restrict__ x = static_cast<const __nv_bfloat16 *>(a.x);
+    const __nv_bfloat16 *__restrict__ w = static_cast<const __nv_bfloat16 *>(a.w);
+
+    float2 acc[TW][4];
+#pragma unroll
+    for (int t = 0; t < TW; t++)
+#pragma unroll
+        for (int j = 0; j < 4; j++) acc[t][j] = make_float2(0.f, 0.f);
+
+    const __nv_bfloat16 *ximg = x + ((size_t)n * a.H) * a.W * a.K + c0;
+#pragma unroll
+    for (int r = 0; r < K; r++) {
+        const int hi = ho * ST + r - P;
+        if (hi < 0 || hi >= a.H) continue;
+        const __nv_bfloat16 *xrow = ximg + (size_t)hi * a.W * a.K;
+        uint4 col[NCOL];
+#pragma unroll
+        for (int j = 0; j < NCOL; j++) {
+            const int wi = wo0 * ST + j - P;
+            col[j] = (wi >= 0 && wi < a.W) ? __ldg(reinterpret_cast<const uint4 *>(xrow + wi * a.K)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        const __nv_bfloat16 *wrow = w + ((o + r) * a.R + o) * a.Kmax + c0;
+#pragma unroll
+        for (int s = 0; s < K; s++) {
+            const uint4 wv = __ldg(reinterpret_cast<const uint4 *>(wrow + s * a.Kmax));
+            const float2 w0 = bf2_lo(wv.x), w1 = bf2_lo(wv.y), w2 = bf2_lo(wv.z), w3 = bf2_lo(wv.w);
+#pragma unroll
+            for (int t = 0; t < TW; t++) {
+                const uint4 xv = col[t * ST + s];
+                acc[t][0] = __ffma2_rn(bf2_lo(xv.x), w0, acc[t][0]);
+                acc[t][1] = __ffma2_rn(bf2_lo(xv.y), w1, acc[t][1]);
+                acc[t][2] = __ffma2_rn(bf2_lo(xv.z), w2, acc[t][2]);
+                acc[t][3] = __ffma2_rn(bf2_lo(xv.w), w3, acc[t][3]);
+            }
+        }
+    }
+    const float4 s0 = __ldg(reinterpret_cast<const float4 *>(a.scale + c0)), s1 = __ldg(reinterpret_cast<const float4 *>(a.scale + c0 + 4));
+    const float4 h0 = __ldg(reinterpret_cast<const float4 *>(a.shift + c0)), h1 = __ldg(reinterpret_cast<const float4 *>(a.shift + c0 + 4));
+    __nv_bfloat16 *yrow = static_cast<__nv_bfloat16 *>(a.y) + (((size_t)n * a.Ho + ho) * a.Wo) * a.K + c0;
+#pragma unroll
+    for (int t = 0; t < TW; t++) {
+        const int wo = wo0 + t;
+        if (wo >= a.Wo) break;
+        float v[8] = {acc[t][0].x * s0.x + h0.x, acc[t][0].y * s0.y + h0.y, acc[t][1].x * s0.z + h0.z, acc[t][1].y * s0.w + h0.w,
+                      acc[t][2].x * s1.x + h1.x, acc[t][2].y * s1.y + h1.y, acc[t][3].x * s1.z + h1.z, acc[t][3].y * s1.w + h1.w};
+        uint4 ov;
+        __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+        for (int j = 0; j < 4; j++) ob[j] = __floats2bfloat162_rn(apply_act(v[2 * j], a.act), apply_act(v[2 * j + 1], a.act));
+        *reinterpret_cast<uint4 *>(yrow + wo * a.K) = ov;
+    }
+}
+
+template <int K, int ST> static cudaError_t launch_dw_vec(const ConvArgs &a, cudaStream_t st) {
+    const int per_row = ((a.Wo + 3) / 4) * (a.K / 8);
+    const int block = per_row >= 256 ? 256 : per_row >= 128 ? 128 : 64;
+    dim3 grid((per_row + block - 1) / block, a.Ho, a.N);
+    dw_vec_kernel<K, ST><<<grid, block, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
 template <typename T> cudaError_t launch_dw(const ConvArgs &a, cudaStream_t st) {
     size_t total = (size_t)a.N * a.Ho * a.Wo * a.K;
     if (!total) return cudaSuccess;
+    if (sizeof(T) == 2 && a.K % 8 == 0 && a.Kmax % 8 == 0 && (a.stride == 1 || a.stride == 2) && a.Ho <= 65535 && a.N <= 65535 &&
+        (size_t)a.W * a.K < (1u << 30) &&
+        ((reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.w) | reinterpret_cast<uintptr_t>(a.y)) & 15) == 0 &&
+        ((reinterpret_cast<uintptr_t>(a.scale) | reinterpret_cast<uintptr_t>(a.shift)) & 15) == 0) {
+        const int key = a.k * 10 + a.stride;
+        switch (key) {
+        case 31: return launch_dw_vec<3, 1>(a, st);
+        case 32: return launch_dw_vec<3, 2>(a, st);
+        case 51: return launch_dw_vec<5, 1>(a, st);
+        case 52: return launch_dw_vec<5, 2>(a, st);
+        case 71: return launch_dw_vec<7, 1>(a, st);
+        case 72: return launch_dw_vec<7, 2>(a, st);
+        default: break;
+        }
+    }
     int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
     dw_plain_kernel<T><<<blocks, 256, 0, st>>>(a);
     return cudaGetLastError();
