@@ -132,6 +132,89 @@ def run_reference(args):
     }))
 
 
+# ----------------------------------------------------------------------------------------------
+# Other configurations (not part of the default line): each prints one JSON line of its own.
+# ----------------------------------------------------------------------------------------------
+def _stream_pool(net, sgs, torch, cfgs, batch, res, opts, stream, pool_groups, family):
+    """Runs `cfgs` as consecutive sgs_stream_run calls over a pool of `pool_groups` resident inputs."""
+    n_cls = 1000
+    x = torch.from_numpy(wl.make_inputs(pool_groups, batch, res, seed=1, bf16=True).reshape(pool_groups * batch, res, res, 3))
+    x = x.cuda().to(torch.bfloat16).contiguous()
+    logits = torch.zeros((pool_groups * batch, n_cls), dtype=torch.float32, device="cuda")
+    tot = {"ms": 0.0, "q": 0, "flops": 0.0, "wbytes": 0.0, "miss": 0.0, "hit": 0.0, "launches": 0, "p50": []}
+    for i in range(0, len(cfgs), pool_groups):
+        part = cfgs[i:i + pool_groups]
+        st = net.stream_run(wl.cfg_array(part), x.data_ptr(), batch, res, logits.data_ptr(), opts, stream.cuda_stream)
+        tot["ms"] += st.total_ms; tot["q"] += len(part); tot["flops"] += st.useful_flops; tot["wbytes"] += st.weight_bytes
+        tot["miss"] += st.hbm_weight_bytes; tot["hit"] += st.hit_ratio * len(part); tot["launches"] += st.kernel_launches
+        tot["p50"].append(st.p50_ms)
+    return tot
+
+
+def run_suite(args):
+    import torch
+    import paper_2306_17266_b200 as sgs
+    peaks = measured_peaks()
+    stream = torch.cuda.Stream()
+    out = {"suite": args.suite, "data": "synthetic", "dtype": "bf16", "n_gpus": 1}
+    if args.suite == "sweep":
+        # throughput sweep: 20k images as groups of 16 images sharing a config (4 groups = one batch of 64)
+        net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
+        n_groups = args.queries // 16 if args.queries != 1000 else 1250
+        cfgs = wl.uniform_stream(wl.RESNET, n_groups, seed=5)
+        rows = []
+        for res in (160, 192, 224):
+            opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=0)
+            _stream_pool(net, sgs, torch, cfgs[:64], 16, res, opts, stream, 64, wl.RESNET)  # warm-up: plans, graphs
+            t = _stream_pool(net, sgs, torch, cfgs, 16, res, opts, stream, 64, wl.RESNET)
+            tf = t["flops"] / (t["ms"] * 1e-3) / 1e12
+            rows.append({"res": res, "images_per_s": t["q"] * 16 / (t["ms"] * 1e-3), "useful_tflops": tf,
+                         "frac_of_bf16_sustained_peak": tf / peaks["bf16_tflops_sustained"], "frac_of_bf16_burst_peak": tf / peaks["bf16_tflops"],
+                         "gflop_per_image": t["flops"] / (t["q"] * 16) / 1e9, "ms": t["ms"]})
+        out.update({"metric": "subnet_images_per_s", "unit": "images/s", "value": rows[-1]["images_per_s"], "rows": rows,
+                    "config": {"workload": "ResNet-50-shaped SuperNet throughput sweep, 16 images per SubNet config, 20k images per resolution, configs uniform (seed 5)",
+                               "peaks": peaks}})
+    elif args.suite == "sgs":
+        # locality stream: Markov chain of configs; cache on / off, window Q in {1, 4, 8}, batch 1 and 16
+        net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
+        n = args.queries if args.queries != 1000 else 5000
+        cfgs = wl.markov_stream(n, seed=4)
+        rows = []
+        for batch, nq in ((1, n), (16, max(64, n // 8))):
+            pool = 500 if batch == 1 else 32
+            warm = sgs.StreamOpts(cache_enabled=0, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=0, weights_evict_first=0)
+            _stream_pool(net, sgs, torch, cfgs[:nq], batch, 224, warm, stream, pool, wl.RESNET)  # builds every plan and graph
+            for cache, q, ef in ((0, 4, 0), (0, 4, 1), (1, 1, 0), (1, 4, 0), (1, 8, 0)):
+                opts = sgs.StreamOpts(cache_enabled=cache, window_q=q, cache_budget_bytes=0, use_graphs=1, record_latency=1, weights_evict_first=ef)
+                _stream_pool(net, sgs, torch, cfgs[:pool], batch, 224, opts, stream, pool, wl.RESNET)
+                t = _stream_pool(net, sgs, torch, cfgs[:nq], batch, 224, opts, stream, pool, wl.RESNET)
+                rows.append({"batch": batch, "cache": cache, "window_q": q, "weights_evict_first": ef, "queries": t["q"],
+                             "queries_per_s": t["q"] / (t["ms"] * 1e-3), "p50_ms": float(np.median(t["p50"])),
+                             "weight_mb_per_query": t["wbytes"] / t["q"] / 1e6, "hbm_weight_mb_per_query": t["miss"] / t["q"] / 1e6,
+                             "hit_ratio": t["hit"] / t["q"]})
+        out.update({"metric": "hbm_weight_bytes_per_query", "unit": "MB/query (analytic)", "value": rows[3]["hbm_weight_mb_per_query"], "rows": rows,
+                    "config": {"workload": "SGS locality stream on the ResNet-50-shaped SuperNet: Markov chain of configs (p=0.9 one stage's depth or width changes), seed 4, 224x224",
+                               "note": "the cached SubGraph restarts at every pool boundary (500 queries at batch 1, 32 at batch 16)"}})
+    elif args.suite == "mbv3":
+        net = sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16)
+        cfgs = wl.uniform_stream(wl.MBV3, args.queries, seed=3)
+        opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=1)
+        _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
+        t = _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
+        net.set_option("profile", 2)
+        popts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=0, record_latency=0)
+        _stream_pool(net, sgs, torch, cfgs, 1, 224, popts, stream, len(cfgs), wl.MBV3)
+        prof = [net.profile_read(c) for c in range(4)]
+        net.set_option("profile", 0)
+        out.update({"metric": METRIC, "unit": UNIT, "value": t["q"] / (t["ms"] * 1e-3), "p50_ms": float(np.median(t["p50"])),
+                    "gflop_per_query": t["flops"] / t["q"] / 1e9, "kernel_launches_per_query": t["launches"] / t["q"],
+                    "kernel_time_ms_by_class": {"conv_tc": prof[0]["total_ms"], "conv_cuda_core": prof[1]["total_ms"],
+                                                "depthwise": prof[2]["total_ms"], "other": prof[3]["total_ms"]},
+                    "depthwise_gbs_at_batch1": prof[2]["alg_bytes"] / (prof[2]["total_ms"] * 1e-3) / 1e9 if prof[2]["total_ms"] else None,
+                    "config": {"workload": "MobileNetV3-shaped SuperNet, 1000-query stream at batch 1, 224x224, configs uniform (seed 3)"}})
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -143,9 +226,14 @@ def main():
     ap.add_argument("--ref-queries", type=int, default=8, help="queries per step of --impl reference")
     ap.add_argument("--cache", type=int, default=1)
     ap.add_argument("--window", type=int, default=4)
+    ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "mbv3"],
+                    help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.suite != "stream":
+        run_suite(args)
         return
 
     import torch
