@@ -164,7 +164,7 @@ def run_suite(args):
         cfgs = wl.uniform_stream(wl.RESNET, n_groups, seed=5)
         rows = []
         for res in (160, 192, 224):
-            opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=0)
+            opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=0, concurrency=args.concurrency)
             _stream_pool(net, sgs, torch, cfgs[:64], 16, res, opts, stream, 64, wl.RESNET)  # warm-up: plans, graphs
             t = _stream_pool(net, sgs, torch, cfgs, 16, res, opts, stream, 64, wl.RESNET)
             tf = t["flops"] / (t["ms"] * 1e-3) / 1e12
@@ -185,7 +185,7 @@ def run_suite(args):
             warm = sgs.StreamOpts(cache_enabled=0, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=0, weights_evict_first=0)
             _stream_pool(net, sgs, torch, cfgs[:nq], batch, 224, warm, stream, pool, wl.RESNET)  # builds every plan and graph
             for cache, q, ef in ((0, 4, 0), (0, 4, 1), (1, 1, 0), (1, 4, 0), (1, 8, 0)):
-                opts = sgs.StreamOpts(cache_enabled=cache, window_q=q, cache_budget_bytes=0, use_graphs=1, record_latency=1, weights_evict_first=ef)
+                opts = sgs.StreamOpts(cache_enabled=cache, window_q=q, cache_budget_bytes=0, use_graphs=1, record_latency=1, weights_evict_first=ef, concurrency=args.concurrency)
                 _stream_pool(net, sgs, torch, cfgs[:pool], batch, 224, opts, stream, pool, wl.RESNET)
                 t = _stream_pool(net, sgs, torch, cfgs[:nq], batch, 224, opts, stream, pool, wl.RESNET)
                 rows.append({"batch": batch, "cache": cache, "window_q": q, "weights_evict_first": ef, "queries": t["q"],
@@ -198,7 +198,8 @@ def run_suite(args):
     elif args.suite == "mbv3":
         net = sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16)
         cfgs = wl.uniform_stream(wl.MBV3, args.queries, seed=3)
-        opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=1)
+        opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=1,
+                              concurrency=args.concurrency)
         _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
         t = _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
         net.set_option("profile", 2)
@@ -226,6 +227,7 @@ def main():
     ap.add_argument("--ref-queries", type=int, default=8, help="queries per step of --impl reference")
     ap.add_argument("--cache", type=int, default=1)
     ap.add_argument("--window", type=int, default=4)
+    ap.add_argument("--concurrency", type=int, default=4, help="independent queries in flight at once")
     ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "mbv3"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()
@@ -268,7 +270,7 @@ def main():
 
     def mk_opts(graphs=1, latency=0):
         return sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=graphs,
-                              record_latency=latency, weights_evict_first=0)
+                              record_latency=latency, weights_evict_first=0, concurrency=args.concurrency)
 
     def step(host=False, o=None):
         o = o or mk_opts()
@@ -351,7 +353,8 @@ def main():
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "queries_per_step": nq, "batch": BATCH, "res": RES,
                        "l2": "inputs (301 MB per step) and the SuperNet (96 MB) exceed L2; no flush",
-                       "cache": bool(args.cache), "window_q": args.window, "parallelism": f"replicas x{world}"},
+                       "cache": bool(args.cache), "window_q": args.window, "queries_in_flight": args.concurrency,
+                       "parallelism": f"replicas x{world}"},
             "p50_ms": st_lat.p50_ms, "p99_ms": st_lat.p99_ms, "mean_ms": st_lat.mean_ms,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_bytes},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu,

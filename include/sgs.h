@@ -86,6 +86,10 @@ typedef struct {
     int record_latency; /* 1: bracket every query with events and fill the latency statistics */
     int weights_evict_first; /* with the cache off: 1 marks weight loads evict-first, which removes
                                 the reuse the hardware L2 replacement gives for free */
+    int concurrency;    /* queries of the stream in flight at once (they are independent; each gets its
+                           own workspaces and CUDA stream, query t uses slot t % concurrency; the
+                           caching decisions still follow the stream order).  0 or 1 = one at a time;
+                           at most 16.  Results do not depend on it. */
 } sgs_stream_opts_t;
 
 /* Results of sgs_stream_run (all host-side; filled after the stream has been synchronised). */
@@ -159,7 +163,8 @@ sgs_status_t sgs_subnet_run(sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, co
  * last window_q queries (element-wise minimum of their layer encodings = their exact intersection,
  * Section 2.2, Appendix A.4) is marked resident for the following queries.
  * Synchronises the stream before filling `stats` (may be NULL).  `opts` NULL = cache on, window 4,
- * graphs on, latency recorded.
+ * graphs on, latency recorded, one query at a time.  Per-query latency is measured from the moment
+ * the query's first operation starts on its slot's stream to its last operation's end.
  */
 sgs_status_t sgs_stream_run(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs,
                             const void *d_inputs, int batch_per_query, int res, void *d_logits,

@@ -153,17 +153,24 @@ struct sgs_supernet {
     size_t weight_arena_bytes = 0;
     float *param_arena = nullptr;  // folded scale / shift
     size_t param_arena_bytes = 0;
-    // activation workspaces
-    void *act[4] = {nullptr, nullptr, nullptr, nullptr};
+    // Workspaces of the queries in flight.  Queries of a stream are independent, so up to
+    // `concurrency` of them run at the same time, each in its own slot (own activation buffers, own
+    // scratch, own CUDA stream); slot 0 runs on the caller's stream.
+    struct Slot {
+        void *act[4] = {nullptr, nullptr, nullptr, nullptr};
+        float *vec[3] = {nullptr, nullptr, nullptr};
+        float *ws = nullptr;        // split-K scratch of the tensor-core kernel
+        void *stage_in = nullptr;   // device staging for host-buffer streams
+        float *stage_out = nullptr;
+        cudaStream_t st = nullptr;  // internal stream (slots >= 1)
+        cudaEvent_t ev = nullptr;
+    };
+    std::vector<Slot> slots;
     size_t act_elems = 0;
-    float *vec[3] = {nullptr, nullptr, nullptr};
     size_t vec_elems = 0;
     int *cache_tbl = nullptr;       // device: [policy, K_0, C_0, K_1, C_1, ...] read by the conv kernels
     int cache_tbl_epoch = -1;       // cache epoch the device table reflects
-    float *splitk_ws = nullptr;     // split-K scratch of the tensor-core kernel
     size_t splitk_ws_elems = 0;
-    void *host_stage_in = nullptr;  // device staging for the host-buffer stream
-    float *host_stage_out = nullptr;
     size_t stage_in_bytes = 0, stage_out_bytes = 0;
     size_t device_bytes = 0;
     std::unordered_map<std::string, std::unique_ptr<Plan>> plans;
@@ -458,26 +465,56 @@ sgs_status_t build_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batc
     return SGS_OK;
 }
 
+// Makes sure `n_slots` slots exist, each with buffers for the sizes in use.
+sgs_status_t ensure_slots(sgs_supernet *net, int n_slots) {
+    while ((int)net->slots.size() < n_slots) {
+        sgs_supernet::Slot sl;
+        if (!net->slots.empty()) {
+            CU(cudaStreamCreateWithFlags(&sl.st, cudaStreamNonBlocking));
+            CU(cudaEventCreateWithFlags(&sl.ev, cudaEventDisableTiming));
+        }
+        for (int i = 0; i < 4 && net->act_elems; i++) {
+            sgs_status_t st = dev_alloc(net, &sl.act[i], net->act_elems * net->elem() + 256);
+            if (st != SGS_OK) return st;
+        }
+        for (int i = 0; i < 3 && net->vec_elems; i++) {
+            sgs_status_t st = dev_alloc(net, (void **)&sl.vec[i], net->vec_elems * 4);
+            if (st != SGS_OK) return st;
+        }
+        if (net->splitk_ws_elems) {
+            sgs_status_t st = dev_alloc(net, (void **)&sl.ws, net->splitk_ws_elems * 4);
+            if (st != SGS_OK) return st;
+        }
+        net->slots.push_back(sl);
+    }
+    return SGS_OK;
+}
+
 sgs_status_t ensure_workspace(sgs_supernet *net, size_t act_elems, int batch) {
+    if (net->slots.empty()) { sgs_status_t st = ensure_slots(net, 1); if (st != SGS_OK) return st; }
     if (act_elems > net->act_elems) {
-        for (int i = 0; i < 4; i++) { dev_free(net, net->act[i], net->act_elems * net->elem() + 256); net->act[i] = nullptr; }
-        net->act_elems = 0;
         drop_graphs(net);
         for (auto &kv : net->plans) kv.second->prepared = false;
-        for (int i = 0; i < 4; i++) {
-            sgs_status_t st = dev_alloc(net, &net->act[i], act_elems * net->elem() + 256);
-            if (st != SGS_OK) return st;
+        for (auto &sl : net->slots) {
+            for (int i = 0; i < 4; i++) {
+                dev_free(net, sl.act[i], net->act_elems * net->elem() + 256);
+                sl.act[i] = nullptr;
+                sgs_status_t st = dev_alloc(net, &sl.act[i], act_elems * net->elem() + 256);
+                if (st != SGS_OK) return st;
+            }
         }
         net->act_elems = act_elems;
     }
     size_t vneed = (size_t)batch * 2048;
     if (vneed > net->vec_elems) {
-        for (int i = 0; i < 3; i++) { dev_free(net, net->vec[i], net->vec_elems * 4); net->vec[i] = nullptr; }
-        net->vec_elems = 0;
         drop_graphs(net);
-        for (int i = 0; i < 3; i++) {
-            sgs_status_t st = dev_alloc(net, (void **)&net->vec[i], vneed * 4);
-            if (st != SGS_OK) return st;
+        for (auto &sl : net->slots) {
+            for (int i = 0; i < 3; i++) {
+                dev_free(net, sl.vec[i], net->vec_elems * 4);
+                sl.vec[i] = nullptr;
+                sgs_status_t st = dev_alloc(net, (void **)&sl.vec[i], vneed * 4);
+                if (st != SGS_OK) return st;
+            }
         }
         net->vec_elems = vneed;
     }
@@ -490,9 +527,10 @@ sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
     size_t ws_need = 0;
     for (Op &op : plan->ops) {
         if (op.type != OP_CONV && op.type != OP_DW) continue;
-        op.conv.x = op.in >= 0 ? net->act[op.in] : nullptr;
-        op.conv.y = net->act[op.out];
-        op.conv.res = op.res >= 0 ? net->act[op.res] : nullptr;
+        const sgs_supernet::Slot &sl = net->slots[plan->slot];
+        op.conv.x = op.in >= 0 ? sl.act[op.in] : nullptr;
+        op.conv.y = sl.act[op.out];
+        op.conv.res = op.res >= 0 ? sl.act[op.res] : nullptr;
         op.impl = 0;
         op.tc.reset();
         if (op.type != OP_CONV || op.in < 0) continue;
@@ -506,21 +544,23 @@ sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
     }
     if (ws_need > net->splitk_ws_elems) {
         drop_graphs(net);
-        dev_free(net, net->splitk_ws, net->splitk_ws_elems * 4);  // cudaFree waits for work in flight
-        net->splitk_ws = nullptr;
-        net->splitk_ws_elems = 0;
-        sgs_status_t st = dev_alloc(net, (void **)&net->splitk_ws, ws_need * 4);
-        if (st != SGS_OK) return st;
+        for (auto &sl : net->slots) {
+            dev_free(net, sl.ws, net->splitk_ws_elems * 4);  // cudaFree waits for work in flight
+            sl.ws = nullptr;
+            sgs_status_t st = dev_alloc(net, (void **)&sl.ws, ws_need * 4);
+            if (st != SGS_OK) return st;
+        }
         net->splitk_ws_elems = ws_need;
     }
     plan->prepared = true;
     return SGS_OK;
 }
 
-sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch, int res, Plan **out) {
+sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch, int res, int slot, Plan **out) {
     std::string key(reinterpret_cast<const char *>(cfg), sizeof(*cfg));
     key.append(reinterpret_cast<const char *>(&batch), sizeof batch);
     key.append(reinterpret_cast<const char *>(&res), sizeof res);
+    key.append(reinterpret_cast<const char *>(&slot), sizeof slot);
     auto it = net->plans.find(key);
     if (it != net->plans.end()) { net->plan_hits++; *out = it->second.get(); return SGS_OK; }
     if (!cfg_valid(net, cfg)) return fail(net, SGS_ECONFIG, "SubNet config outside the elastic sets of this SuperNet");
@@ -528,6 +568,7 @@ sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch,
     std::unique_ptr<Plan> p(new Plan);
     sgs_status_t st = build_plan(net, cfg, batch, res, p.get());
     if (st != SGS_OK) return st;
+    p->slot = slot;
     *out = p.get();
     net->plans.emplace(std::move(key), std::move(p));
     return SGS_OK;
@@ -536,7 +577,8 @@ sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch,
 template <typename T>
 sgs_status_t run_ops(sgs_supernet *net, Plan *plan, const void *d_input, void *d_logits, cudaStream_t st, size_t first,
                      size_t last) {
-    auto abuf = [&](int id) -> void * { return id < 0 ? const_cast<void *>(d_input) : net->act[id]; };
+    const sgs_supernet::Slot &sl = net->slots[plan->slot];
+    auto abuf = [&](int id) -> void * { return id < 0 ? const_cast<void *>(d_input) : sl.act[id]; };
     for (size_t oi = first; oi < last; oi++) {
         Op &op = plan->ops[oi];
         ProfRec rec{};
@@ -555,35 +597,35 @@ sgs_status_t run_ops(sgs_supernet *net, Plan *plan, const void *d_input, void *d
             ConvArgs a = op.conv;
             if (op.in < 0) a.x = d_input;
             a.cache_tbl = net->cache_tbl; a.layer = op.layer;
-            a.ws = net->splitk_ws; a.ws_elems = net->splitk_ws_elems;
+            a.ws = sl.ws; a.ws_elems = net->splitk_ws_elems;
             if (op.type == OP_DW) { CU(launch_dw<T>(a, st)); net->kernel_launches++; }
             else if (op.impl == 1) { int n = 0; CU(tc_conv_launch(*op.tc, a, st, &n)); net->kernel_launches += n; }
             else { CU(launch_conv_plain<T>(a, st)); net->kernel_launches++; }
             break;
         }
         case OP_MAXPOOL:
-            CU(launch_maxpool3s2<T>((const T *)abuf(op.in), (T *)net->act[op.out], op.N, op.H, op.W, op.C, st));
+            CU(launch_maxpool3s2<T>((const T *)abuf(op.in), (T *)sl.act[op.out], op.N, op.H, op.W, op.C, st));
             net->kernel_launches++;
             break;
         case OP_GAP:
-            CU(launch_gap<T>((const T *)abuf(op.in), net->vec[op.vout], op.N, op.H * op.W, op.C, st));
+            CU(launch_gap<T>((const T *)abuf(op.in), sl.vec[op.vout], op.N, op.H * op.W, op.C, st));
             net->kernel_launches++;
             break;
         case OP_SE_GATE: {
             const StoredLayer &L1 = net->layers[op.layer], &L2 = net->layers[op.layer2];
-            CU(launch_se_gate<T>(net->vec[op.vin], (const T *)L1.w, L1.shift, (const T *)L2.w, L2.shift, net->vec[op.vout],
+            CU(launch_se_gate<T>(sl.vec[op.vin], (const T *)L1.w, L1.shift, (const T *)L2.w, L2.shift, sl.vec[op.vout],
                                  op.N, op.C, op.K, L1.C, L2.C, st));
             net->kernel_launches++;
             break;
         }
         case OP_SCALE:
-            CU(launch_scale<T>((const T *)net->act[op.in], net->vec[op.vin], (T *)net->act[op.out], op.N, op.H * op.W, op.C, st));
+            CU(launch_scale<T>((const T *)sl.act[op.in], sl.vec[op.vin], (T *)sl.act[op.out], op.N, op.H * op.W, op.C, st));
             net->kernel_launches++;
             break;
         case OP_LINEAR: {
             const StoredLayer &L = net->layers[op.layer];
-            float *y = op.vout < 0 ? static_cast<float *>(d_logits) : net->vec[op.vout];
-            CU(launch_linear<T>(net->vec[op.vin], (const T *)L.w, L.shift, y, op.N, op.C, op.K, L.C, op.act, st));
+            float *y = op.vout < 0 ? static_cast<float *>(d_logits) : sl.vec[op.vout];
+            CU(launch_linear<T>(sl.vec[op.vin], (const T *)L.w, L.shift, y, op.N, op.C, op.K, L.C, op.act, st));
             net->kernel_launches++;
             break;
         }
@@ -639,9 +681,9 @@ sgs_status_t push_cache_table(sgs_supernet *net, cudaStream_t st) {
 // is replayed as one captured graph per plan, independent of the caller's pointers and of the cache
 // state (kernels read the cache box from device memory).
 sgs_status_t run_query(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, const void *d_input, int batch, int res,
-                       void *d_logits, cudaStream_t st, bool use_graph, Plan **plan_out) {
+                       void *d_logits, cudaStream_t st, bool use_graph, int slot, Plan **plan_out) {
     Plan *plan = nullptr;
-    sgs_status_t rc = get_plan(net, cfg, batch, res, &plan);
+    sgs_status_t rc = get_plan(net, cfg, batch, res, slot, &plan);
     if (rc != SGS_OK) return rc;
     rc = ensure_workspace(net, plan->act_elems, batch);
     if (rc != SGS_OK) return rc;
@@ -891,12 +933,16 @@ void sgs_supernet_free(sgs_supernet_t *net) {
     for (auto &e : net->prof_pool) cudaEventDestroy(e);
     cudaFree(net->weight_arena);
     cudaFree(net->param_arena);
-    for (int i = 0; i < 4; i++) cudaFree(net->act[i]);
-    for (int i = 0; i < 3; i++) cudaFree(net->vec[i]);
+    for (auto &sl : net->slots) {
+        for (int i = 0; i < 4; i++) cudaFree(sl.act[i]);
+        for (int i = 0; i < 3; i++) cudaFree(sl.vec[i]);
+        cudaFree(sl.ws);
+        cudaFree(sl.stage_in);
+        cudaFree(sl.stage_out);
+        if (sl.ev) cudaEventDestroy(sl.ev);
+        if (sl.st) cudaStreamDestroy(sl.st);
+    }
     cudaFree(net->cache_tbl);
-    cudaFree(net->splitk_ws);
-    cudaFree(net->host_stage_in);
-    cudaFree(net->host_stage_out);
     delete net;
 }
 
@@ -936,7 +982,7 @@ sgs_status_t sgs_subnet_run(sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, co
     DeviceGuard guard(net->device);
     if (!guard.ok) return fail(net, SGS_ECUDA, "cudaSetDevice failed");
     Plan *plan = nullptr;
-    sgs_status_t rc = run_query(net, cfg, d_input, batch, res, d_logits, (cudaStream_t)cuda_stream, false, &plan);
+    sgs_status_t rc = run_query(net, cfg, d_input, batch, res, d_logits, (cudaStream_t)cuda_stream, false, 0, &plan);
     if (rc != SGS_OK) return rc;
     if (net->cache.enabled) cache_observe(net, encoding_of(plan->slices));
     return SGS_OK;
@@ -952,35 +998,40 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
     if (!guard.ok) return fail(net, SGS_ECUDA, "cudaSetDevice failed");
     sgs_stream_opts_t o;
     if (opts) o = *opts;
-    else { o.cache_enabled = 1; o.window_q = 4; o.cache_budget_bytes = 0; o.use_graphs = 1; o.record_latency = 1; o.weights_evict_first = 0; }
+    else { o.cache_enabled = 1; o.window_q = 4; o.cache_budget_bytes = 0; o.use_graphs = 1; o.record_latency = 1; o.weights_evict_first = 0; o.concurrency = 1; }
     if (o.window_q < 1) return fail(net, SGS_EINVAL, "window_q must be >= 1");
+    if (o.concurrency < 0 || o.concurrency > 16) return fail(net, SGS_EINVAL, "concurrency must be in [0, 16]");
     for (int t = 0; t < n_queries; t++)
         if (!cfg_valid(net, &cfgs[t])) return fail(net, SGS_ECONFIG, "query " + std::to_string(t) + ": config outside the elastic sets");
     cache_reset(net, o.cache_enabled != 0, o.cache_budget_bytes, o.window_q);
     net->cache.evict_first_when_off = (!o.cache_enabled && o.weights_evict_first) ? 1 : 0;
+    // queries in flight at once: each runs in its own slot; per-kernel profiling wants them one by one
+    const int S = net->profile ? 1 : std::max(1, std::min(o.concurrency ? o.concurrency : 1, std::max(1, n_queries)));
+    {
+        sgs_status_t rc = ensure_slots(net, S);
+        if (rc != SGS_OK) return rc;
+    }
 
     const size_t in_elems = (size_t)batch * res * res * 3, in_bytes = in_elems * net->elem();
     const size_t out_bytes = (size_t)batch * net->def.classes * sizeof(float);
     if (host_buffers) {
-        // two staging slots so that the copy of query t+1 can overlap query t
-        if (net->stage_in_bytes < 2 * in_bytes) {
-            dev_free(net, net->host_stage_in, net->stage_in_bytes);
-            net->host_stage_in = nullptr; net->stage_in_bytes = 0;
-            sgs_status_t rc = dev_alloc(net, &net->host_stage_in, 2 * in_bytes);
-            if (rc != SGS_OK) return rc;
-            net->stage_in_bytes = 2 * in_bytes;
+        // one staging pair per slot: consecutive queries of a slot are ordered by the slot's stream
+        if (net->stage_in_bytes < in_bytes || net->stage_out_bytes < out_bytes) {
+            for (auto &sl : net->slots) {
+                dev_free(net, sl.stage_in, net->stage_in_bytes); sl.stage_in = nullptr;
+                dev_free(net, sl.stage_out, net->stage_out_bytes); sl.stage_out = nullptr;
+            }
+            net->stage_in_bytes = std::max(net->stage_in_bytes, in_bytes);
+            net->stage_out_bytes = std::max(net->stage_out_bytes, out_bytes);
         }
-        if (net->stage_out_bytes < 2 * out_bytes) {
-            dev_free(net, net->host_stage_out, net->stage_out_bytes);
-            net->host_stage_out = nullptr; net->stage_out_bytes = 0;
-            sgs_status_t rc = dev_alloc(net, (void **)&net->host_stage_out, 2 * out_bytes);
-            if (rc != SGS_OK) return rc;
-            net->stage_out_bytes = 2 * out_bytes;
+        for (auto &sl : net->slots) {
+            if (!sl.stage_in) { sgs_status_t rc = dev_alloc(net, &sl.stage_in, net->stage_in_bytes); if (rc != SGS_OK) return rc; }
+            if (!sl.stage_out) { sgs_status_t rc = dev_alloc(net, (void **)&sl.stage_out, net->stage_out_bytes); if (rc != SGS_OK) return rc; }
         }
     }
-    std::vector<cudaEvent_t> ev;
+    std::vector<cudaEvent_t> ev;  // per query: start and end on the query's stream
     if (o.record_latency) {
-        ev.resize((size_t)n_queries + 1);
+        ev.resize(2 * (size_t)n_queries);
         for (auto &e : ev) CU(cudaEventCreate(&e));
     }
     cudaEvent_t e0, e1;
@@ -992,15 +1043,22 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
     int updates = 0;
     sgs_status_t rc = SGS_OK;
     CU(cudaEventRecord(e0, st));
-    if (o.record_latency && n_queries) CU(cudaEventRecord(ev[0], st));
+    for (int sidx = 1; sidx < S; sidx++) CU(cudaStreamWaitEvent(net->slots[sidx].st, e0, 0));  // fork
     for (int t = 0; t < n_queries && rc == SGS_OK; t++) {
+        const int slot = t % S;
+        sgs_supernet::Slot &sl = net->slots[slot];
+        cudaStream_t qs = slot == 0 ? st : sl.st;
         const void *din;
         void *dout;
+        if (o.record_latency) {
+            cudaError_t ce = cudaEventRecord(ev[2 * (size_t)t], qs);
+            if (ce != cudaSuccess) { rc = fail(net, SGS_ECUDA, cudaGetErrorString(ce)); break; }
+        }
         if (host_buffers) {
-            din = static_cast<char *>(net->host_stage_in) + (size_t)(t & 1) * in_bytes;
-            dout = reinterpret_cast<char *>(net->host_stage_out) + (size_t)(t & 1) * out_bytes;
-            cudaError_t ce = cudaMemcpyAsync(const_cast<void *>(din), static_cast<const char *>(inputs) + (size_t)t * in_bytes,
-                                             in_bytes, cudaMemcpyHostToDevice, st);
+            din = sl.stage_in;
+            dout = sl.stage_out;
+            cudaError_t ce = cudaMemcpyAsync(sl.stage_in, static_cast<const char *>(inputs) + (size_t)t * in_bytes, in_bytes,
+                                             cudaMemcpyHostToDevice, qs);
             if (ce != cudaSuccess) { rc = fail(net, SGS_ECUDA, cudaGetErrorString(ce)); break; }
         } else {
             din = static_cast<const char *>(inputs) + (size_t)t * in_bytes;
@@ -1009,15 +1067,15 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
         Plan *plan = nullptr;
         const int epoch_before = net->cache.epoch;
         // the legacy default stream cannot be captured: run it without graphs
-        rc = run_query(net, &cfgs[t], din, batch, res, dout, st, o.use_graphs != 0 && st != nullptr, &plan);
+        rc = run_query(net, &cfgs[t], din, batch, res, dout, qs, o.use_graphs != 0 && qs != nullptr, slot, &plan);
         if (rc != SGS_OK) break;
         if (host_buffers) {
             cudaError_t ce = cudaMemcpyAsync(static_cast<char *>(logits) + (size_t)t * out_bytes, dout, out_bytes,
-                                             cudaMemcpyDeviceToHost, st);
+                                             cudaMemcpyDeviceToHost, qs);
             if (ce != cudaSuccess) { rc = fail(net, SGS_ECUDA, cudaGetErrorString(ce)); break; }
         }
         if (o.record_latency) {
-            cudaError_t ce = cudaEventRecord(ev[(size_t)t + 1], st);
+            cudaError_t ce = cudaEventRecord(ev[2 * (size_t)t + 1], qs);
             if (ce != cudaSuccess) { rc = fail(net, SGS_ECUDA, cudaGetErrorString(ce)); break; }
         }
         std::vector<int> enc = encoding_of(plan->slices);
@@ -1028,10 +1086,15 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
             if (net->cache.epoch != epoch_before) updates++;
         }
     }
+    for (int sidx = 1; sidx < S; sidx++) {  // join
+        cudaEventRecord(net->slots[sidx].ev, net->slots[sidx].st);
+        cudaStreamWaitEvent(st, net->slots[sidx].ev, 0);
+    }
     cudaError_t ce = cudaEventRecord(e1, st);
     cudaError_t se = cudaStreamSynchronize(st);
     if (rc == SGS_OK && (ce != cudaSuccess || se != cudaSuccess))
         rc = fail(net, SGS_ECUDA, std::string("stream: ") + cudaGetErrorString(se != cudaSuccess ? se : ce));
+    if (rc != SGS_OK) cudaDeviceSynchronize();  // leave no work of the other slots behind
     if (rc == SGS_OK && tc_conv_status()) rc = fail(net, SGS_ETIMEOUT, "a bounded device-side wait ran out in the tensor-core kernel");
     if (rc == SGS_OK && stats) {
         std::memset(stats, 0, sizeof(*stats));
@@ -1044,7 +1107,7 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
         if (o.record_latency && n_queries) {
             std::vector<float> lat((size_t)n_queries);
             double sum = 0;
-            for (int t = 0; t < n_queries; t++) { cudaEventElapsedTime(&lat[t], ev[t], ev[(size_t)t + 1]); sum += lat[t]; }
+            for (int t = 0; t < n_queries; t++) { cudaEventElapsedTime(&lat[t], ev[2 * (size_t)t], ev[2 * (size_t)t + 1]); sum += lat[t]; }
             std::sort(lat.begin(), lat.end());
             stats->p50_ms = lat[(size_t)(n_queries - 1) / 2];
             stats->p99_ms = lat[(size_t)std::min<long long>(n_queries - 1, (long long)std::ceil(0.99 * n_queries) - 1)];

@@ -86,6 +86,7 @@ struct Plan {
     cudaGraphExec_t graph = nullptr;  // ops [1, n-1): everything that touches only internal buffers
     int launches = 0;
     bool prepared = false;  // implementations chosen and buffer addresses fixed
+    int slot = 0;           // which set of workspaces the plan's buffer addresses refer to
 };
 
 // ---- launchers implemented in sgs_kernels.cu (T = float or __nv_bfloat16) -------------------

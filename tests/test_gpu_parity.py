@@ -128,10 +128,22 @@ def test_stream_run_matches_single_queries_and_counts_bytes():
                 assert 0 < st.hbm_weight_bytes < st.weight_bytes and 0 < st.hit_ratio <= 1
             else:
                 assert st.hbm_weight_bytes == st.weight_bytes and st.hit_ratio == 0
+    # several queries in flight: same bits
+    for conc in (2, 3):
+        d_out.zero_()
+        torch.cuda.synchronize()
+        opts = sgs.StreamOpts(cache_enabled=1, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=1, concurrency=conc)
+        st = gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+        np.testing.assert_array_equal(d_out.cpu().numpy(), singles)
+        assert st.p50_ms > 0
     # host-buffer variant
     h_out = np.zeros((n, 1000), dtype=np.float32)
     h_in = d_in.cpu().view(torch.int16).numpy()
     gnet.stream_run(cfgs, h_in, 1, res, h_out, None, stream.cuda_stream, host=True)
+    np.testing.assert_array_equal(h_out, singles)
+    h_out[:] = 0
+    opts = sgs.StreamOpts(cache_enabled=1, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=0, concurrency=4)
+    gnet.stream_run(cfgs, h_in, 1, res, h_out, opts, stream.cuda_stream, host=True)
     np.testing.assert_array_equal(h_out, singles)
 
 
