@@ -227,7 +227,7 @@ def main():
     ap.add_argument("--ref-queries", type=int, default=8, help="queries per step of --impl reference")
     ap.add_argument("--cache", type=int, default=1)
     ap.add_argument("--window", type=int, default=4)
-    ap.add_argument("--concurrency", type=int, default=4, help="independent queries in flight at once")
+    ap.add_argument("--concurrency", type=int, default=8, help="independent queries in flight at once")
     ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "mbv3"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()

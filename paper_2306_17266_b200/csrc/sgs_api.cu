@@ -170,6 +170,9 @@ struct sgs_supernet {
     size_t vec_elems = 0;
     int *cache_tbl = nullptr;       // device: [policy, K_0, C_0, K_1, C_1, ...] read by the conv kernels
     int cache_tbl_epoch = -1;       // cache epoch the device table reflects
+    int *tbl_ring = nullptr;        // pinned host ring of table images (async uploads need stable sources)
+    cudaEvent_t tbl_ring_ev[16] = {};  // upload of ring entry i has completed
+    int tbl_ring_pos = 0;
     size_t splitk_ws_elems = 0;
     size_t stage_in_bytes = 0, stage_out_bytes = 0;
     size_t device_bytes = 0;
@@ -569,6 +572,7 @@ sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch,
     sgs_status_t st = build_plan(net, cfg, batch, res, p.get());
     if (st != SGS_OK) return st;
     p->slot = slot;
+    p->enc = encoding_of(p->slices);
     *out = p.get();
     net->plans.emplace(std::move(key), std::move(p));
     return SGS_OK;
@@ -659,19 +663,25 @@ sgs_status_t run_plan(sgs_supernet *net, Plan *plan, const void *d_input, void *
                                   : run_ops<float>(net, plan, d_input, d_logits, st, first, last);
 }
 
-// Brings the device copy of the cache table up to date with the host policy state.
+// Brings the device copy of the cache table up to date with the host policy state.  The image is
+// built in a pinned ring entry so that the copy is truly asynchronous.
 sgs_status_t push_cache_table(sgs_supernet *net, cudaStream_t st) {
     const CacheState &cs = net->cache;
     if (net->cache_tbl_epoch == cs.epoch) return SGS_OK;
-    std::vector<int> tbl(1 + 2 * net->layers.size(), 0);
+    const size_t n = 1 + 2 * net->layers.size();
+    const int slot = net->tbl_ring_pos;
+    net->tbl_ring_pos = (slot + 1) % 16;
+    CU(cudaEventSynchronize(net->tbl_ring_ev[slot]));  // the upload that last used this entry (16 updates ago)
+    int *tbl = net->tbl_ring + (size_t)slot * n;
+    std::memset(tbl, 0, n * sizeof(int));
     if (cs.enabled && !cs.G.empty()) {
         tbl[0] = 1;
         for (size_t li = 0; li < net->layers.size(); li++) { tbl[1 + 2 * li] = cs.G[3 * li]; tbl[2 + 2 * li] = cs.G[3 * li + 1]; }
     } else if (!cs.enabled && cs.evict_first_when_off) {
         tbl[0] = 2;
     }
-    // pageable source: the runtime stages the bytes before the call returns, so tbl may go out of scope
-    CU(cudaMemcpyAsync(net->cache_tbl, tbl.data(), tbl.size() * sizeof(int), cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(net->cache_tbl, tbl, n * sizeof(int), cudaMemcpyHostToDevice, st));
+    CU(cudaEventRecord(net->tbl_ring_ev[slot], st));
     net->cache_tbl_epoch = cs.epoch;
     return SGS_OK;
 }
@@ -907,8 +917,11 @@ sgs_status_t sgs_supernet_load(const sgs_arch_desc_t *arch, const void *host_blo
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxAccessPolicyWindowSize, device) == cudaSuccess) net->window_max = (size_t)v;
     {
         size_t n = 1 + 2 * net->layers.size();
-        if (dev_alloc(net, (void **)&net->cache_tbl, n * sizeof(int)) != SGS_OK ||
-            cudaMemset(net->cache_tbl, 0, n * sizeof(int)) != cudaSuccess) {
+        bool ok = dev_alloc(net, (void **)&net->cache_tbl, n * sizeof(int)) == SGS_OK &&
+                  cudaMemset(net->cache_tbl, 0, n * sizeof(int)) == cudaSuccess &&
+                  cudaMallocHost((void **)&net->tbl_ring, 16 * n * sizeof(int)) == cudaSuccess;
+        for (int i = 0; i < 16 && ok; i++) ok = cudaEventCreateWithFlags(&net->tbl_ring_ev[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
             sgs_supernet_free(holder.release());
             return SGS_ENOMEM;
         }
@@ -943,6 +956,9 @@ void sgs_supernet_free(sgs_supernet_t *net) {
         if (sl.st) cudaStreamDestroy(sl.st);
     }
     cudaFree(net->cache_tbl);
+    cudaFreeHost(net->tbl_ring);
+    for (int i = 0; i < 16; i++)
+        if (net->tbl_ring_ev[i]) cudaEventDestroy(net->tbl_ring_ev[i]);
     delete net;
 }
 
@@ -984,7 +1000,7 @@ sgs_status_t sgs_subnet_run(sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, co
     Plan *plan = nullptr;
     sgs_status_t rc = run_query(net, cfg, d_input, batch, res, d_logits, (cudaStream_t)cuda_stream, false, 0, &plan);
     if (rc != SGS_OK) return rc;
-    if (net->cache.enabled) cache_observe(net, encoding_of(plan->slices));
+    if (net->cache.enabled) cache_observe(net, plan->enc);
     return SGS_OK;
 }
 
@@ -1078,7 +1094,7 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
             cudaError_t ce = cudaEventRecord(ev[2 * (size_t)t + 1], qs);
             if (ce != cudaSuccess) { rc = fail(net, SGS_ECUDA, cudaGetErrorString(ce)); break; }
         }
-        std::vector<int> enc = encoding_of(plan->slices);
+        const std::vector<int> &enc = plan->enc;
         QueryAccount qa = account_query(net, enc);
         flops += plan->flops; wbytes += qa.weight_bytes; miss_bytes += qa.miss_bytes; hit += qa.hit_ratio;
         if (net->cache.enabled) {

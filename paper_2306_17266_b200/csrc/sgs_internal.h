@@ -82,6 +82,7 @@ struct Plan {
     int batch = 0, res = 0;
     double flops = 0, weight_bytes = 0, act_bytes = 0;
     std::vector<Slice> slices;
+    std::vector<int> enc;  // (K, C, k) per stored layer: the SubNet's vector encoding
     size_t act_elems = 0;  // elements each activation buffer must hold
     cudaGraphExec_t graph = nullptr;  // ops [1, n-1): everything that touches only internal buffers
     int launches = 0;
