@@ -182,7 +182,8 @@ def run_suite(args):
         rows = []
         for batch, nq in ((1, n), (16, max(64, n // 8))):
             pool = 500 if batch == 1 else 32
-            warm = sgs.StreamOpts(cache_enabled=0, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=0, weights_evict_first=0)
+            warm = sgs.StreamOpts(cache_enabled=0, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=0, weights_evict_first=0,
+                                  concurrency=args.concurrency)
             _stream_pool(net, sgs, torch, cfgs[:nq], batch, 224, warm, stream, pool, wl.RESNET)  # builds every plan and graph
             for cache, q, ef in ((0, 4, 0), (0, 4, 1), (1, 1, 0), (1, 4, 0), (1, 8, 0)):
                 opts = sgs.StreamOpts(cache_enabled=cache, window_q=q, cache_budget_bytes=0, use_graphs=1, record_latency=1, weights_evict_first=ef, concurrency=args.concurrency)
@@ -195,6 +196,23 @@ def run_suite(args):
         out.update({"metric": "hbm_weight_bytes_per_query", "unit": "MB/query (analytic)", "value": rows[3]["hbm_weight_mb_per_query"], "rows": rows,
                     "config": {"workload": "SGS locality stream on the ResNet-50-shaped SuperNet: Markov chain of configs (p=0.9 one stage's depth or width changes), seed 4, 224x224",
                                "note": "the cached SubGraph restarts at every pool boundary (500 queries at batch 1, 32 at batch 16)"}})
+    elif args.suite == "sgs-probe":
+        # one short locality stream, one variant, one query at a time, no graphs: meant to be run under a
+        # profiler that sums DRAM bytes over the kernels of the measured part (its launch range is printed)
+        net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
+        n = args.queries if args.queries != 1000 else 48
+        cfgs = wl.markov_stream(16 + n, seed=4)
+        opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=0, record_latency=0,
+                              weights_evict_first=args.evict_first, concurrency=1)
+        before = net.get_counter("kernel_launches")
+        _stream_pool(net, sgs, torch, cfgs[:16], args.batch, 224, opts, stream, 16, wl.RESNET)
+        skip = net.get_counter("kernel_launches") - before
+        t = _stream_pool(net, sgs, torch, cfgs[16:], args.batch, 224, opts, stream, n, wl.RESNET)
+        out.update({"metric": "hbm_weight_bytes_per_query", "unit": "MB/query (analytic)", "value": t["miss"] / t["q"] / 1e6,
+                    "weight_mb_per_query": t["wbytes"] / t["q"] / 1e6, "hit_ratio": t["hit"] / t["q"], "queries": t["q"],
+                    "launches_before_measured_part": skip, "launches_in_measured_part": t["launches"],
+                    "config": {"batch": args.batch, "cache": args.cache, "window_q": args.window, "weights_evict_first": args.evict_first,
+                               "note": "load-time kernels precede the warm-up launches; count them with the profiler's launch list"}})
     elif args.suite == "mbv3":
         net = sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16)
         cfgs = wl.uniform_stream(wl.MBV3, args.queries, seed=3)
@@ -228,7 +246,9 @@ def main():
     ap.add_argument("--cache", type=int, default=1)
     ap.add_argument("--window", type=int, default=4)
     ap.add_argument("--concurrency", type=int, default=8, help="independent queries in flight at once")
-    ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "mbv3"],
+    ap.add_argument("--batch", type=int, default=1, help="images per query (sgs-probe)")
+    ap.add_argument("--evict-first", type=int, default=0, help="with --cache 0: mark weight loads evict-first (sgs-probe)")
+    ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()
     if args.impl == "reference":

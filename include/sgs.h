@@ -209,7 +209,7 @@ sgs_status_t sgs_subnet_cost(const sgs_supernet_t *net, const sgs_subnet_cfg_t *
  * impl 0 = automatic (tensor cores when dtype is bf16, C, K, Cmax are multiples of 8, pointers are
  * 16-byte aligned and stride-2 inputs have even sizes), 1 = CUDA-core kernel, 2 = tensor cores or
  * SGS_EUNSUPPORTED.  weight_policy 0 = no L2 hint, 1 = evict-last for weight tiles with filter <
- * cache_k and channel < cache_c and evict-first for the rest, 2 = all weights evict-first.
+ * cache_k and channel < cache_c (default replacement for the rest), 2 = all weights evict-first.
  * Asynchronous on `cuda_stream`.  The tensor-core path may split the reduction over several CTAs
  * using a per-device scratch buffer that this function allocates on demand (cudaMalloc) and keeps;
  * calls that overlap on the same device must therefore not run concurrently.

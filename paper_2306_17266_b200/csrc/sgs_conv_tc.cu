@@ -19,8 +19,8 @@
 //
 // SubGraph-Stationary reuse (paper Section 2.2, Section 4.2 Persistent / Dynamic Buffer): weight tiles
 // inside the cached SubGraph's prefix box (filter < cacheK and channel < cacheC) are loaded with an
-// L2 evict-last policy, all other weight tiles evict-first, so the shared weights stay on chip across
-// queries while the distinct weights of each SubNet stream through.
+// L2 evict-last policy so that the shared weights stay on chip across queries; the distinct weights
+// of each SubNet take the default replacement.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 =
 // epilogue (one TMEM lane quadrant each).  Every wait is bounded; when one runs out the kernel sets
@@ -282,9 +282,13 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
         auto load_weights = [&](int s, int c0, int tapw) {
             uint8_t *sb = smem + s * STAGE_BYTES + A_STAGE_BYTES;
             mbar_expect_tx(&full_bar[s], tx);
-            if (weight_policy == 0) tma_load_3d(sb, &p.tmW, &full_bar[s], c0, tapw, f0);
-            else tma_load_3d_hint(sb, &p.tmW, &full_bar[s], c0, tapw, f0,
-                                  (weight_policy == 1 && f0 < cacheK && c0 < cacheC) ? pol_keep : pol_stream);
+            // policy 1: tiles of the cached SubGraph are kept (evict-last), the rest take the default
+            // replacement (measured: marking them evict-first loses to plain LRU whenever the SuperNet
+            // fits in L2); policy 2: everything evict-first (the "no reuse at all" reference point)
+            const bool in_box = weight_policy == 1 && f0 < cacheK && c0 < cacheC;
+            if (weight_policy == 2) tma_load_3d_hint(sb, &p.tmW, &full_bar[s], c0, tapw, f0, pol_stream);
+            else if (in_box) tma_load_3d_hint(sb, &p.tmW, &full_bar[s], c0, tapw, f0, pol_keep);
+            else tma_load_3d(sb, &p.tmW, &full_bar[s], c0, tapw, f0);
         };
         // Weights do not depend on the previous layer: fill the first stages' weight halves before
         // waiting for it, so that their latency overlaps the previous layer's tail.
