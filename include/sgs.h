@@ -268,7 +268,8 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
 /*
  * Per-kernel-class timing.  After sgs_set_option(net, "profile", 2) (2 = on and reset, 1 = on, 0 = off)
  * every kernel the handle launches is bracketed by CUDA events on the launching stream (graphs are
- * bypassed meanwhile).  kernel_class: 0 tensor-core convolution, 1 CUDA-core convolution,
+ * bypassed and queries run one at a time meanwhile; a short sleeping kernel ahead of every 8 queries
+ * lets the host queue their launches first, so the intervals hold device time, not launch latency).  kernel_class: 0 tensor-core convolution, 1 CUDA-core convolution,
  * 2 depthwise convolution, 3 everything else.  Returns the launches, their summed device time, their
  * summed algorithmic bytes (sliced weights + input + output + residual of each launch) and useful
  * FLOPs since the last reset.  Synchronises the device.
@@ -276,7 +277,10 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
 sgs_status_t sgs_profile_read(sgs_supernet_t *net, int kernel_class, long long *launches, double *total_ms,
                               double *alg_bytes, double *flops);
 
-/* Counters by name ("kernel_launches", "plan_hits", "plan_misses", "device_bytes", "tc_convs"). */
+/* Counters by name ("kernel_launches", "plan_hits", "plan_misses", "device_bytes", "tc_convs";
+ * diagnostics: "host_us_stream", "host_us_query", "host_us_table", "host_us_graph", "host_us_direct" =
+ * accumulated host microseconds spent issuing streams / queries / cache-table updates / graph
+ * launches / direct launches). */
 long long sgs_get_counter(const sgs_supernet_t *net, const char *name);
 
 const char *sgs_last_error(const sgs_supernet_t *net);

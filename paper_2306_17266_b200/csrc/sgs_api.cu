@@ -8,6 +8,7 @@
 #include <cstring>
 #include <deque>
 #include <map>
+#include <chrono>
 
 using namespace sgs;
 
@@ -139,8 +140,6 @@ struct CacheState {
     int evict_first_when_off = 0;
 };
 
-struct ProfRec { int cls; cudaEvent_t a, b; double bytes, flops; };
-
 }  // namespace
 
 struct sgs_supernet {
@@ -182,10 +181,10 @@ struct sgs_supernet {
     long long kernel_launches = 0;
     int plan_hits = 0, plan_misses = 0;
     int force_plain = 0;
+    double host_us_graph = 0, host_us_direct = 0, host_us_stream = 0, host_us_query = 0, host_us_table = 0;  // host time spent issuing work (diagnostic counters)
     // per-kernel-class timing (option "profile"): 0 tensor-core conv, 1 CUDA-core conv, 2 depthwise, 3 other
     int profile = 0;
-    std::vector<ProfRec> prof_pending;
-    std::vector<cudaEvent_t> prof_pool;
+    std::vector<Plan *> prof_used;  // plans run since the last fold, in order
     double prof_ms[4] = {0, 0, 0, 0}, prof_bytes[4] = {0, 0, 0, 0}, prof_flops[4] = {0, 0, 0, 0};
     long long prof_launches[4] = {0, 0, 0, 0};
     mutable std::string err;
@@ -221,8 +220,9 @@ void dev_free(sgs_supernet *net, void *p, size_t bytes) {
     net->device_bytes -= bytes;
 }
 void drop_graphs(sgs_supernet *net) {
-    for (auto &kv : net->plans)
+    for (auto &kv : net->plans) {
         if (kv.second->graph) { cudaGraphExecDestroy(kv.second->graph); kv.second->graph = nullptr; }
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -585,15 +585,14 @@ sgs_status_t run_ops(sgs_supernet *net, Plan *plan, const void *d_input, void *d
     auto abuf = [&](int id) -> void * { return id < 0 ? const_cast<void *>(d_input) : sl.act[id]; };
     for (size_t oi = first; oi < last; oi++) {
         Op &op = plan->ops[oi];
-        ProfRec rec{};
         if (net->profile) {
-            rec.cls = op.type == OP_CONV ? (op.impl == 1 ? 0 : 1) : op.type == OP_DW ? 2 : 3;
-            rec.bytes = op.alg_bytes; rec.flops = op.flops;
-            for (cudaEvent_t *e : {&rec.a, &rec.b}) {
-                if (net->prof_pool.empty()) { CU(cudaEventCreate(e)); }
-                else { *e = net->prof_pool.back(); net->prof_pool.pop_back(); }
+            // one event pair per op of the plan
+            if (plan->prof_ev.size() != 2 * plan->ops.size()) {
+                for (cudaEvent_t e : plan->prof_ev) cudaEventDestroy(e);
+                plan->prof_ev.assign(2 * plan->ops.size(), nullptr);
+                for (auto &e : plan->prof_ev) CU(cudaEventCreate(&e));
             }
-            CU(cudaEventRecord(rec.a, st));
+            CU(cudaEventRecord(plan->prof_ev[2 * oi], st));
         }
         switch (op.type) {
         case OP_CONV:
@@ -634,27 +633,36 @@ sgs_status_t run_ops(sgs_supernet *net, Plan *plan, const void *d_input, void *d
             break;
         }
         }
-        if (net->profile) {
-            CU(cudaEventRecord(rec.b, st));
-            net->prof_pending.push_back(rec);
-        }
+        if (net->profile) CU(cudaEventRecord(plan->prof_ev[2 * oi + 1], st));
     }
     return SGS_OK;
 }
 
+// Adds the per-op durations of every plan run since the last fold to the per-class totals.  A plan
+// that ran several times contributes its latest timestamps once per run.
 void fold_profile(sgs_supernet *net) {
-    if (net->prof_pending.empty()) return;
+    if (net->prof_used.empty()) return;
     cudaDeviceSynchronize();
-    for (auto &r : net->prof_pending) {
-        float ms = 0;
-        if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) {
-            net->prof_ms[r.cls] += ms; net->prof_bytes[r.cls] += r.bytes; net->prof_flops[r.cls] += r.flops;
-            net->prof_launches[r.cls]++;
+    for (Plan *plan : net->prof_used) {
+        if (plan->prof_ev.size() != 2 * plan->ops.size()) continue;
+        for (size_t oi = 0; oi < plan->ops.size(); oi++) {
+            const Op &op = plan->ops[oi];
+            const int cls = op.type == OP_CONV ? (op.impl == 1 ? 0 : 1) : op.type == OP_DW ? 2 : 3;
+            float ms = 0;
+            if (cudaEventElapsedTime(&ms, plan->prof_ev[2 * oi], plan->prof_ev[2 * oi + 1]) == cudaSuccess) {
+                net->prof_ms[cls] += ms; net->prof_bytes[cls] += op.alg_bytes; net->prof_flops[cls] += op.flops;
+                net->prof_launches[cls]++;
+            }
         }
-        net->prof_pool.push_back(r.a);
-        net->prof_pool.push_back(r.b);
     }
-    net->prof_pending.clear();
+    net->prof_used.clear();
+}
+
+void destroy_plan_resources(Plan *plan) {
+    if (plan->graph) cudaGraphExecDestroy(plan->graph);
+    plan->graph = nullptr;
+    for (cudaEvent_t e : plan->prof_ev) cudaEventDestroy(e);
+    plan->prof_ev.clear();
 }
 
 sgs_status_t run_plan(sgs_supernet *net, Plan *plan, const void *d_input, void *d_logits, cudaStream_t st, size_t first,
@@ -702,16 +710,22 @@ sgs_status_t run_query(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, const voi
         if (rc != SGS_OK) return rc;
     }
     if (plan_out) *plan_out = plan;
-    rc = push_cache_table(net, st);
+    {
+        const auto p0 = std::chrono::steady_clock::now();
+        rc = push_cache_table(net, st);
+        net->host_us_table += std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - p0).count();
+    }
     if (rc != SGS_OK) return rc;
     const size_t n_ops = plan->ops.size();
+    if (net->profile) net->prof_used.push_back(plan);
     if (!use_graph || net->profile || n_ops < 3) {
         long long before = net->kernel_launches;
         rc = run_plan(net, plan, d_input, d_logits, st, 0, n_ops);
         plan->launches = (int)(net->kernel_launches - before);
         return rc;
     }
-    if (!plan->graph) {
+    cudaGraphExec_t &graph = plan->graph;
+    if (!graph) {
         cudaGraph_t g = nullptr;
         CU(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
         long long before = net->kernel_launches;
@@ -721,15 +735,21 @@ sgs_status_t run_query(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, const voi
         cudaError_t e = cudaStreamEndCapture(st, &g);
         if (rc != SGS_OK) { if (g) cudaGraphDestroy(g); return rc; }
         if (e != cudaSuccess) return fail(net, SGS_ECUDA, std::string("graph capture: ") + cudaGetErrorString(e));
-        e = cudaGraphInstantiate(&plan->graph, g, 0);
+        e = cudaGraphInstantiate(&graph, g, 0);
         cudaGraphDestroy(g);
         if (e != cudaSuccess) return fail(net, SGS_ECUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
     }
     long long before = net->kernel_launches;
+    auto t0 = std::chrono::steady_clock::now();
     rc = run_plan(net, plan, d_input, d_logits, st, 0, 1);
     if (rc != SGS_OK) return rc;
-    CU(cudaGraphLaunch(plan->graph, st));
+    auto t1 = std::chrono::steady_clock::now();
+    CU(cudaGraphLaunch(graph, st));
+    auto t2 = std::chrono::steady_clock::now();
     rc = run_plan(net, plan, d_input, d_logits, st, n_ops - 1, n_ops);
+    auto t3 = std::chrono::steady_clock::now();
+    net->host_us_graph += std::chrono::duration<double, std::micro>(t2 - t1).count();
+    net->host_us_direct += std::chrono::duration<double, std::micro>(t1 - t0).count() + std::chrono::duration<double, std::micro>(t3 - t2).count();
     net->kernel_launches = before + plan->launches;
     return rc;
 }
@@ -939,11 +959,9 @@ void sgs_supernet_free(sgs_supernet_t *net) {
     if (!net) return;
     DeviceGuard guard(net->device);
     cudaDeviceSynchronize();
-    for (auto &kv : net->plans)
-        if (kv.second->graph) cudaGraphExecDestroy(kv.second->graph);
+    for (auto &kv : net->plans) destroy_plan_resources(kv.second.get());
     net->plans.clear();
-    for (auto &r : net->prof_pending) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
-    for (auto &e : net->prof_pool) cudaEventDestroy(e);
+    net->prof_used.clear();
     cudaFree(net->weight_arena);
     cudaFree(net->param_arena);
     for (auto &sl : net->slots) {
@@ -1059,6 +1077,7 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
     int updates = 0;
     sgs_status_t rc = SGS_OK;
     CU(cudaEventRecord(e0, st));
+    const auto host_t0 = std::chrono::steady_clock::now();
     for (int sidx = 1; sidx < S; sidx++) CU(cudaStreamWaitEvent(net->slots[sidx].st, e0, 0));  // fork
     for (int t = 0; t < n_queries && rc == SGS_OK; t++) {
         const int slot = t % S;
@@ -1080,10 +1099,19 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
             din = static_cast<const char *>(inputs) + (size_t)t * in_bytes;
             dout = static_cast<char *>(logits) + (size_t)t * out_bytes;
         }
+        // Profiling brackets every launch with events.  To keep the host's launch latency out of those
+        // intervals the stream is first held for a few milliseconds by a sleeping kernel, so that the
+        // launches of the next 8 queries are already queued when the GPU reaches them.
+        if (net->profile && t % 8 == 0) {
+            cudaError_t ce = launch_delay(6000, qs);
+            if (ce != cudaSuccess) { rc = fail(net, SGS_ECUDA, cudaGetErrorString(ce)); break; }
+        }
         Plan *plan = nullptr;
         const int epoch_before = net->cache.epoch;
         // the legacy default stream cannot be captured: run it without graphs
+        const auto q0 = std::chrono::steady_clock::now();
         rc = run_query(net, &cfgs[t], din, batch, res, dout, qs, o.use_graphs != 0 && qs != nullptr, slot, &plan);
+        net->host_us_query += std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - q0).count();
         if (rc != SGS_OK) break;
         if (host_buffers) {
             cudaError_t ce = cudaMemcpyAsync(static_cast<char *>(logits) + (size_t)t * out_bytes, dout, out_bytes,
@@ -1102,6 +1130,7 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
             if (net->cache.epoch != epoch_before) updates++;
         }
     }
+    net->host_us_stream += std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - host_t0).count();
     for (int sidx = 1; sidx < S; sidx++) {  // join
         cudaEventRecord(net->slots[sidx].ev, net->slots[sidx].st);
         cudaStreamWaitEvent(st, net->slots[sidx].ev, 0);
@@ -1198,7 +1227,8 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
         net->force_plain = value == 1;
         DeviceGuard guard(net->device);
         cudaDeviceSynchronize();
-        drop_graphs(net);
+        fold_profile(net);
+        for (auto &kv : net->plans) destroy_plan_resources(kv.second.get());
         net->plans.clear();
         return SGS_OK;
     }
@@ -1220,6 +1250,11 @@ long long sgs_get_counter(const sgs_supernet_t *net, const char *name) {
     if (n == "plan_hits") return net->plan_hits;
     if (n == "plan_misses") return net->plan_misses;
     if (n == "device_bytes") return (long long)net->device_bytes;
+    if (n == "host_us_graph") return (long long)net->host_us_graph;
+    if (n == "host_us_direct") return (long long)net->host_us_direct;
+    if (n == "host_us_stream") return (long long)net->host_us_stream;
+    if (n == "host_us_query") return (long long)net->host_us_query;
+    if (n == "host_us_table") return (long long)net->host_us_table;
     if (n == "tc_convs") {
         long long c = 0;
         for (auto &kv : net->plans)

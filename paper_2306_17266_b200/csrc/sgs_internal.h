@@ -85,6 +85,7 @@ struct Plan {
     std::vector<int> enc;  // (K, C, k) per stored layer: the SubNet's vector encoding
     size_t act_elems = 0;  // elements each activation buffer must hold
     cudaGraphExec_t graph = nullptr;  // ops [1, n-1): everything that touches only internal buffers
+    std::vector<cudaEvent_t> prof_ev;      // start / end event of every op (profiling)
     int launches = 0;
     bool prepared = false;  // implementations chosen and buffer addresses fixed
     int slot = 0;           // which set of workspaces the plan's buffer addresses refer to
@@ -105,6 +106,7 @@ cudaError_t launch_linear(const float *v, const T *w, const float *bias, float *
 cudaError_t launch_relayout_conv(const float *src, void *dst, int K, int C, int R, int S, int bf16, cudaStream_t st);
 cudaError_t launch_relayout_dw(const float *src, void *dst, int K, int R, int S, int bf16, cudaStream_t st);
 cudaError_t launch_convert(const float *src, void *dst, size_t n, int bf16, cudaStream_t st);
+cudaError_t launch_delay(unsigned microseconds, cudaStream_t st);  // one thread sleeping for a bounded time
 cudaError_t launch_fold_bn(const float *gamma, const float *beta, const float *mean, const float *var,
                            const float *bias, float *scale, float *shift, int K, cudaStream_t st);
 

@@ -474,6 +474,20 @@ cudaError_t launch_convert(const float *src, void *dst, size_t n, int bf16, cuda
     return cudaGetLastError();
 }
 
+// Holds a stream for about `us` microseconds (bounded: the loop ends on its own).
+__global__ void delay_kernel(unsigned us) {
+    unsigned long long t0, t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+    do {
+        __nanosleep(2000);
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    } while (t - t0 < (unsigned long long)us * 1000ull);
+}
+cudaError_t launch_delay(unsigned microseconds, cudaStream_t st) {
+    delay_kernel<<<1, 1, 0, st>>>(microseconds > 50000u ? 50000u : microseconds);
+    return cudaGetLastError();
+}
+
 // Batch-norm folding: scale = gamma / sqrt(var + 1e-5), shift = beta - mean * scale (+ bias).
 __global__ void fold_bn_kernel(const float *gamma, const float *beta, const float *mean, const float *var,
                                const float *bias, float *scale, float *shift, int K) {
