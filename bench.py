@@ -22,6 +22,8 @@ import numpy as np
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
+# 16 queries in flight need more than the default 8 hardware work queues; must be set before CUDA starts
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
 
 from paper_2306_17266_b200 import workload as wl  # noqa: E402
 
@@ -52,7 +54,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -245,7 +247,7 @@ def main():
     ap.add_argument("--ref-queries", type=int, default=8, help="queries per step of --impl reference")
     ap.add_argument("--cache", type=int, default=1)
     ap.add_argument("--window", type=int, default=4)
-    ap.add_argument("--concurrency", type=int, default=8, help="independent queries in flight at once")
+    ap.add_argument("--concurrency", type=int, default=16, help="independent queries in flight at once")
     ap.add_argument("--batch", type=int, default=1, help="images per query (sgs-probe)")
     ap.add_argument("--evict-first", type=int, default=0, help="with --cache 0: mark weight loads evict-first (sgs-probe)")
     ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3"],
@@ -348,6 +350,7 @@ def main():
         # launch configuration is taken as share x (1).
         step(o=mk_opts(conc=1))
         seq = step(o=mk_opts(conc=1))
+        seq_lat = step(o=mk_opts(conc=1, latency=1))
         net.set_option("profile", 2)
         step(o=mk_opts(graphs=0))
         prof = [net.profile_read(c) for c in range(4)]
@@ -387,6 +390,7 @@ def main():
                        "cache": bool(args.cache), "window_q": args.window, "queries_in_flight": args.concurrency,
                        "parallelism": f"replicas x{world}"},
             "p50_ms": st_lat.p50_ms, "p99_ms": st_lat.p99_ms, "mean_ms": st_lat.mean_ms,
+            "one_query_at_a_time": {"queries_per_s": seq_lat.queries_per_s, "p50_ms": seq_lat.p50_ms, "p99_ms": seq_lat.p99_ms},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_bytes},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu,
             "useful_tflops": st_lat.useful_flops / (st_lat.total_ms * 1e-3) / 1e12,

@@ -89,7 +89,10 @@ typedef struct {
     int concurrency;    /* queries of the stream in flight at once (they are independent; each gets its
                            own workspaces and CUDA stream, query t uses slot t % concurrency; the
                            caching decisions still follow the stream order).  0 or 1 = one at a time;
-                           at most 16.  Results do not depend on it. */
+                           at most 16.  From 12 up the convolutions pick tiles for aggregate throughput
+                           instead of single-launch latency.  More than 8 only overlap if the process
+                           raised CUDA_DEVICE_MAX_CONNECTIONS before its CUDA context was created.
+                           Results are bit-identical for a given tile choice (i.e. for <12 and for >=12). */
 } sgs_stream_opts_t;
 
 /* Results of sgs_stream_run (all host-side; filled after the stream has been synchronised). */

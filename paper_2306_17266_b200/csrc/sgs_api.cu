@@ -181,6 +181,7 @@ struct sgs_supernet {
     long long kernel_launches = 0;
     int plan_hits = 0, plan_misses = 0;
     int force_plain = 0;
+    int throughput_mode = 0;  // set by streams that keep many queries in flight; part of the plan key
     double host_us_graph = 0, host_us_direct = 0, host_us_stream = 0, host_us_query = 0, host_us_table = 0;  // host time spent issuing work (diagnostic counters)
     // per-kernel-class timing (option "profile"): 0 tensor-core conv, 1 CUDA-core conv, 2 depthwise, 3 other
     int profile = 0;
@@ -536,6 +537,7 @@ sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
         op.conv.res = op.res >= 0 ? sl.act[op.res] : nullptr;
         op.impl = 0;
         op.tc.reset();
+        op.conv.throughput = plan->throughput;
         if (op.type != OP_CONV || op.in < 0) continue;
         if (net->dtype != SGS_BF16 || net->force_plain || !tc_available()) continue;
         std::string why;
@@ -564,6 +566,7 @@ sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch,
     key.append(reinterpret_cast<const char *>(&batch), sizeof batch);
     key.append(reinterpret_cast<const char *>(&res), sizeof res);
     key.append(reinterpret_cast<const char *>(&slot), sizeof slot);
+    key.append(reinterpret_cast<const char *>(&net->throughput_mode), sizeof net->throughput_mode);
     auto it = net->plans.find(key);
     if (it != net->plans.end()) { net->plan_hits++; *out = it->second.get(); return SGS_OK; }
     if (!cfg_valid(net, cfg)) return fail(net, SGS_ECONFIG, "SubNet config outside the elastic sets of this SuperNet");
@@ -572,6 +575,7 @@ sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch,
     sgs_status_t st = build_plan(net, cfg, batch, res, p.get());
     if (st != SGS_OK) return st;
     p->slot = slot;
+    p->throughput = net->throughput_mode;
     p->enc = encoding_of(p->slices);
     *out = p.get();
     net->plans.emplace(std::move(key), std::move(p));
@@ -1045,6 +1049,7 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
         sgs_status_t rc = ensure_slots(net, S);
         if (rc != SGS_OK) return rc;
     }
+    net->throughput_mode = S >= 12 ? 1 : 0;
 
     const size_t in_elems = (size_t)batch * res * res * 3, in_bytes = in_elems * net->elem();
     const size_t out_bytes = (size_t)batch * net->def.classes * sizeof(float);
@@ -1171,6 +1176,7 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
     for (auto &e : ev) cudaEventDestroy(e);
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
+    net->throughput_mode = 0;
     return rc;
 }
 

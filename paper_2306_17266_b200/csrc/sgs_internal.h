@@ -56,6 +56,7 @@ struct ConvArgs {
     // (lets a captured graph follow cache updates without being re-captured)
     const int *cache_tbl = nullptr;
     int layer = 0;
+    int throughput = 0;  // 1: pick tiles for aggregate throughput (many launches in flight), 0: for the latency of this launch
     // split-K scratch of the tensor-core kernel: fp32 partial tiles [splits][M][K]
     float *ws = nullptr;
     size_t ws_elems = 0;
@@ -89,6 +90,7 @@ struct Plan {
     int launches = 0;
     bool prepared = false;  // implementations chosen and buffer addresses fixed
     int slot = 0;           // which set of workspaces the plan's buffer addresses refer to
+    int throughput = 0;     // tile choice of the plan's convolutions (see ConvArgs::throughput)
 };
 
 // ---- launchers implemented in sgs_kernels.cu (T = float or __nv_bfloat16) -------------------
