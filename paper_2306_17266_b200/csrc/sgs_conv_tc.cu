@@ -679,7 +679,7 @@ cudaError_t tc_conv_init(int dev) {
         if ((e = cudaMalloc(&ds.status, sizeof(int))) != cudaSuccess) return e;
         if ((e = cudaMemset(ds.status, 0, sizeof(int))) != cudaSuccess) return e;
     }
-    if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 4>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 3>())) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(conv_tc_kernel<256, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<256, 4>())) != cudaSuccess) return e;
     ds.attrs_set = true;
@@ -702,7 +702,7 @@ cudaError_t tc_conv_launch(const TcConvPlan &pl, const ConvArgs &a, cudaStream_t
     if (prm.splits > 1 && (!a.ws || a.ws_elems < pl.ws_elems)) prm.splits = 1;  // no workspace: run unsplit
     TcConvPlan run = pl;
     run.grid.z = (unsigned)prm.splits;
-    if (pl.bn_tile == 64) e = launch_variant<64, 4>(run, prm, st);
+    if (pl.bn_tile == 64) e = launch_variant<64, 3>(run, prm, st);
     else if (pl.bn_tile == 128) e = launch_variant<128, 3>(run, prm, st);
     else e = launch_variant<256, 4>(run, prm, st);
     if (launches) *launches = 1;
@@ -746,7 +746,7 @@ cudaError_t static_scratch_setup(int dev, StaticScratch **out) {
         StaticScratch *ptr = nullptr;
         cudaError_t e = cudaGetSymbolAddress((void **)&ptr, g_static_scratch);
         if (e != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 4>())) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 3>())) != cudaSuccess) return e;
         if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
         if ((e = cudaFuncSetAttribute(conv_tc_kernel<256, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<256, 4>())) != cudaSuccess) return e;
         if ((e = cudaMemset(&ptr->status, 0, sizeof(int))) != cudaSuccess) return e;
@@ -799,7 +799,7 @@ extern "C" sgs_status_t sgs_conv2d_sliced_static(const sgs_conv_desc_t *d, const
     prm.ws = sc->ws;
     TcConvPlan run = *plan;
     run.grid.z = (unsigned)prm.splits;
-    cudaError_t e = plan->bn_tile == 64    ? launch_variant<64, 4>(run, prm, st)
+    cudaError_t e = plan->bn_tile == 64    ? launch_variant<64, 3>(run, prm, st)
                     : plan->bn_tile == 128 ? launch_variant<128, 3>(run, prm, st)
                                            : launch_variant<256, 4>(run, prm, st);
     if (e == cudaSuccess && prm.splits > 1) e = launch_finish(prm, st);
