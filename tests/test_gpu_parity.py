@@ -180,3 +180,31 @@ def test_encoding_matches_checker():
         _, onet, gnet = gu.nets(fam, True)
         for c in wl.uniform_stream(fam, 5, seed=3) + [wl.extreme_cfg(fam, False), wl.extreme_cfg(fam, True)]:
             np.testing.assert_array_equal(gnet.subnet_encode(c), onet.encode(c))
+
+
+def test_bench_launch_configuration_sampled_against_checker():
+    # the benchmark's configuration (224x224, batch 1, graphs, cache on, 16 queries in flight) on the
+    # first 48 queries of its stream; four sampled queries are recomputed by the checker, all logits
+    # must be finite, and the stream must reproduce itself bit for bit
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    n, res = 48, 224
+    cfgs = wl.uniform_stream(wl.RESNET, 1000, seed=2)[:n]
+    xs = wl.make_inputs(n, 1, res, seed=1, bf16=True)
+    d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
+    d_out = torch.zeros((n, 1000), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    opts = sgs.StreamOpts(cache_enabled=1, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=0, concurrency=16)
+    gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+    first = d_out.cpu().numpy().copy()
+    d_out.zero_()
+    torch.cuda.synchronize()
+    gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+    np.testing.assert_array_equal(d_out.cpu().numpy(), first)
+    assert np.all(np.isfinite(first))
+    agree = []
+    for t in (0, 13, 30, 47):
+        ref = onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)
+        assert gu.rel_err(first[t:t + 1], ref) <= TOL_BF16, t
+        agree.append(int(first[t].argmax() == ref[0].argmax()))
+    assert sum(agree) >= 3
