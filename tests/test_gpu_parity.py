@@ -208,3 +208,33 @@ def test_bench_launch_configuration_sampled_against_checker():
         assert gu.rel_err(first[t:t + 1], ref) <= TOL_BF16, t
         agree.append(int(first[t].argmax() == ref[0].argmax()))
     assert sum(agree) >= 3
+
+
+def test_argmax_agreement_on_the_resnet_stream():
+    # 200 queries of the benchmark stream: top-1 class against the checker run with the same storage
+    # rounding points.  Bar: >= 99.5 % agreement.  A disagreement only counts as one if the checker's
+    # own logit at the GPU's class is further from its maximum than the error bound (2e-2 * max|ref|):
+    # with random weights a few top-2 margins are smaller than one bf16 rounding step.
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    n, res = 200, 224
+    cfgs = wl.uniform_stream(wl.RESNET, 1000, seed=2)[:n]
+    xs = wl.make_inputs(n, 1, res, seed=1, bf16=True)
+    d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
+    d_out = torch.zeros((n, 1000), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    opts = sgs.StreamOpts(cache_enabled=1, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=0, concurrency=8)
+    gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+    got = d_out.cpu().numpy()
+    strict = tie_aware = 0
+    worst = 0.0
+    for t in range(n):
+        ref = onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)[0]
+        worst = max(worst, float(np.abs(got[t] - ref).max() / np.abs(ref).max()))
+        g = int(got[t].argmax())
+        strict += g == int(ref.argmax())
+        tie_aware += (ref.max() - ref[g]) <= 2e-2 * np.abs(ref).max()
+    print(f"argmax agreement: strict {strict}/{n}, tie-aware {tie_aware}/{n}, worst rel err {worst:.2e}")
+    assert worst <= TOL_BF16
+    assert tie_aware / n >= 0.995
+    assert strict / n >= 0.995
