@@ -324,8 +324,41 @@ __global__ void gap_kernel(const T *__restrict__ x, float *__restrict__ g, int H
         g[(size_t)n * C + c] = tot / (float)HW;
     }
 }
+// bf16, C % 8 == 0: one warp per (image, 8-channel vector); lanes stride over the pixels with 16-byte
+// loads and the lane sums are combined by a fixed shuffle tree (same result every run).
+__device__ __forceinline__ float2 bf2f(uint32_t u) { return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)); }
+
+__global__ void __launch_bounds__(256) gap_vec_kernel(const __nv_bfloat16 *__restrict__ x, float *__restrict__ g, int N, int HW, int C) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const int cvecs = C >> 3;
+    if (warp >= N * cvecs) return;
+    const int n = warp / cvecs, cv = warp % cvecs;
+    const __nv_bfloat16 *base = x + (size_t)n * HW * C + cv * 8;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int i = lane; i < HW; i += 32) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(base + (size_t)i * C));
+        const float2 a = bf2f(v.x), b = bf2f(v.y), c = bf2f(v.z), d = bf2f(v.w);
+        acc[0] += a.x; acc[1] += a.y; acc[2] += b.x; acc[3] += b.y; acc[4] += c.x; acc[5] += c.y; acc[6] += d.x; acc[7] += d.y;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; j++)
+#pragma unroll
+        for (int o = 16; o; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+    if (lane == 0) {
+        const float inv = 1.f / (float)HW;
+        float4 *dst = reinterpret_cast<float4 *>(g + (size_t)n * C + cv * 8);
+        dst[0] = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+        dst[1] = make_float4(acc[4] * inv, acc[5] * inv, acc[6] * inv, acc[7] * inv);
+    }
+}
+
 template <typename T> cudaError_t launch_gap(const T *x, float *g, int N, int HW, int C, cudaStream_t st) {
     if (N <= 0 || C <= 0) return cudaSuccess;
+    if (sizeof(T) == 2 && C % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0 && (reinterpret_cast<uintptr_t>(g) & 15) == 0) {
+        const int warps = N * (C / 8);
+        gap_vec_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16 *>(x), g, N, HW, C);
+        return cudaGetLastError();
+    }
     dim3 grid((C + 31) / 32, N), block(32, 8);
     gap_kernel<T><<<grid, block, 0, st>>>(x, g, HW, C);
     return cudaGetLastError();
@@ -338,7 +371,7 @@ template cudaError_t launch_gap<__nv_bfloat16>(const __nv_bfloat16 *, float *, i
 // One block per image; warps stride over outputs and reduce with shuffles.
 // ---------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256) se_gate_kernel(const float *__restrict__ g, const T *__restrict__ w1,
+__global__ void __launch_bounds__(1024) se_gate_kernel(const float *__restrict__ g, const T *__restrict__ w1,
                                                       const float *__restrict__ b1, const T *__restrict__ w2,
                                                       const float *__restrict__ b2, float *__restrict__ gate, int mid,
                                                       int sq, int w1_ld, int w2_ld) {
@@ -367,7 +400,7 @@ template <typename T>
 cudaError_t launch_se_gate(const float *g, const T *w1, const float *b1, const T *w2, const float *b2, float *gate,
                            int N, int mid, int sq, int w1_ld, int w2_ld, cudaStream_t st) {
     if (N <= 0) return cudaSuccess;
-    se_gate_kernel<T><<<N, 256, (size_t)(mid + sq) * sizeof(float), st>>>(g, w1, b1, w2, b2, gate, mid, sq, w1_ld, w2_ld);
+    se_gate_kernel<T><<<N, 1024, (size_t)(mid + sq) * sizeof(float), st>>>(g, w1, b1, w2, b2, gate, mid, sq, w1_ld, w2_ld);
     return cudaGetLastError();
 }
 template cudaError_t launch_se_gate<float>(const float *, const float *, const float *, const float *, const float *, float *, int, int, int, int, int, cudaStream_t);
@@ -383,9 +416,34 @@ __global__ void scale_kernel(const T *__restrict__ x, const float *__restrict__ 
         y[i] = from_f<T>(to_f<T>(x[i]) * gate[n * C + c]);
     }
 }
+__global__ void __launch_bounds__(256) scale_vec_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ gate,
+                                                        __nv_bfloat16 *__restrict__ y, int vecs_per_image, int cvecs, int C, int total) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;  // one 8-channel vector
+    if (i >= total) return;
+    const int n = i / vecs_per_image, cv = i % cvecs;
+    const uint4 v = *reinterpret_cast<const uint4 *>(x + (size_t)i * 8);
+    const float4 g0 = __ldg(reinterpret_cast<const float4 *>(gate + (size_t)n * C + cv * 8));
+    const float4 g1 = __ldg(reinterpret_cast<const float4 *>(gate + (size_t)n * C + cv * 8 + 4));
+    const float2 a = bf2f(v.x), b = bf2f(v.y), c = bf2f(v.z), d = bf2f(v.w);
+    uint4 o;
+    __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&o);
+    ob[0] = __floats2bfloat162_rn(a.x * g0.x, a.y * g0.y);
+    ob[1] = __floats2bfloat162_rn(b.x * g0.z, b.y * g0.w);
+    ob[2] = __floats2bfloat162_rn(c.x * g1.x, c.y * g1.y);
+    ob[3] = __floats2bfloat162_rn(d.x * g1.z, d.y * g1.w);
+    *reinterpret_cast<uint4 *>(y + (size_t)i * 8) = o;
+}
+
 template <typename T> cudaError_t launch_scale(const T *x, const float *gate, T *y, int N, int HW, int C, cudaStream_t st) {
     size_t total = (size_t)N * HW * C;
     if (!total) return cudaSuccess;
+    if (sizeof(T) == 2 && C % 8 == 0 && total / 8 < (1u << 30) &&
+        ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(gate)) & 15) == 0) {
+        const int tv = (int)(total / 8);
+        scale_vec_kernel<<<(tv + 255) / 256, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16 *>(x), gate,
+                                                          reinterpret_cast<__nv_bfloat16 *>(y), HW * (C / 8), C / 8, C, tv);
+        return cudaGetLastError();
+    }
     int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
     scale_kernel<T><<<blocks, 256, 0, st>>>(x, gate, y, total, HW, C);
     return cudaGetLastError();
@@ -410,11 +468,38 @@ __global__ void __launch_bounds__(256) linear_kernel(const float *__restrict__ v
     for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if (lane == 0) y[(size_t)n * K + j] = apply_act(s + bias[j], act);
 }
+// bf16 weights, C % 8 == 0, ld % 8 == 0: each lane takes 8 weights (16 bytes) and 8 inputs per step
+__global__ void __launch_bounds__(256) linear_vec_kernel(const float *__restrict__ v, const __nv_bfloat16 *__restrict__ w,
+                                                         const float *__restrict__ bias, float *__restrict__ y, int N, int C,
+                                                         int K, int ld, int act) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= N * K) return;
+    const int n = warp / K, j = warp % K;
+    const __nv_bfloat16 *wr = w + (size_t)j * ld;
+    const float *vr = v + (size_t)n * C;
+    float s = 0.f;
+    for (int c = lane * 8; c < C; c += 256) {
+        const uint4 wv = __ldg(reinterpret_cast<const uint4 *>(wr + c));
+        const float4 x0 = *reinterpret_cast<const float4 *>(vr + c), x1 = *reinterpret_cast<const float4 *>(vr + c + 4);
+        const float2 a = bf2f(wv.x), b = bf2f(wv.y), cc = bf2f(wv.z), d = bf2f(wv.w);
+        s = fmaf(a.x, x0.x, s); s = fmaf(a.y, x0.y, s); s = fmaf(b.x, x0.z, s); s = fmaf(b.y, x0.w, s);
+        s = fmaf(cc.x, x1.x, s); s = fmaf(cc.y, x1.y, s); s = fmaf(d.x, x1.z, s); s = fmaf(d.y, x1.w, s);
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) y[(size_t)n * K + j] = apply_act(s + bias[j], act);
+}
+
 template <typename T>
 cudaError_t launch_linear(const float *v, const T *w, const float *bias, float *y, int N, int C, int K, int ld, int act,
                           cudaStream_t st) {
     long long warps = (long long)N * K;
     if (warps <= 0) return cudaSuccess;
+    if (sizeof(T) == 2 && C % 8 == 0 && ld % 8 == 0 && ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(v)) & 15) == 0) {
+        linear_vec_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(v, reinterpret_cast<const __nv_bfloat16 *>(w), bias, y, N,
+                                                                               C, K, ld, act);
+        return cudaGetLastError();
+    }
     int blocks = (int)((warps * 32 + 255) / 256);
     linear_kernel<T><<<blocks, 256, 0, st>>>(v, w, bias, y, N, C, K, ld, act);
     return cudaGetLastError();
