@@ -93,6 +93,15 @@ typedef struct {
                            instead of single-launch latency.  More than 8 only overlap if the process
                            raised CUDA_DEVICE_MAX_CONNECTIONS before its CUDA context was created.
                            Results are bit-identical for a given tile choice (i.e. for <12 and for >=12). */
+    int wave;           /* 0 = off.  G > 0 (at most 64, bf16 handles only): G consecutive queries form a
+                           wave that advances through the layers together; at every layer the tensor-core
+                           convolutions of all members whose SubNet has that layer are ONE grouped launch
+                           (each member with its own slice of the shared weights), so a launch fills the
+                           GPU although a single batch-1 SubNet cannot.  `concurrency` then counts waves
+                           in flight (0 = 2, at most 4) and use_graphs is ignored.  Every query of a wave
+                           starts and ends with its wave (that is its recorded latency).  The cached
+                           SubGraph is still re-chosen in stream order; the L2 hints of a wave use the
+                           choice in force when the wave was issued. */
 } sgs_stream_opts_t;
 
 /* Results of sgs_stream_run (all host-side; filled after the stream has been synchronised). */

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <cstdlib>
 #include <deque>
 #include <map>
 #include <chrono>
@@ -152,6 +153,10 @@ struct sgs_supernet {
     size_t weight_arena_bytes = 0;
     float *param_arena = nullptr;  // folded scale / shift
     size_t param_arena_bytes = 0;
+    // bf16 handles: the stem's weights once more as a GEMM operand [K][stem_kkp] (rows = the stored
+    // (r, s, c) order, zero padded to a multiple of 8), used with the patch matrix of the input
+    void *stem_gemm_w = nullptr;
+    int stem_kkp = 0;
     // Workspaces of the queries in flight.  Queries of a stream are independent, so up to
     // `concurrency` of them run at the same time, each in its own slot (own activation buffers, own
     // scratch, own CUDA stream); slot 0 runs on the caller's stream.
@@ -165,6 +170,22 @@ struct sgs_supernet {
         cudaEvent_t ev = nullptr;
     };
     std::vector<Slot> slots;
+    // Wave execution (many queries advance through the layers together, one grouped launch per layer):
+    // each wave in flight has its own stream, launch-table buffers and staging buffers.
+    struct WaveCtx {
+        cudaStream_t st = nullptr;
+        cudaEvent_t done = nullptr;  // everything issued for the last wave of this context has finished
+        char *h_tbl = nullptr, *d_tbl = nullptr;  // launch tables of one wave: pinned host image and device copy
+        size_t tbl_bytes = 0;
+        void *stage_in = nullptr;    // host-buffer streams: the wave's inputs / logits on the device
+        float *stage_out = nullptr;
+        size_t stage_in_bytes = 0, stage_out_bytes = 0;
+        bool busy = false;
+    };
+    std::vector<WaveCtx> waves;
+    std::vector<std::unique_ptr<GroupLaunch>> group_pool;  // parameter blocks of a wave's grouped launches (reused)
+    std::unordered_map<long long, int> op_rank;        // (op type, anchor layer) -> position in the largest SubNet
+    int sms = 148;
     size_t act_elems = 0;
     size_t vec_elems = 0;
     int *cache_tbl = nullptr;       // device: [policy, K_0, C_0, K_1, C_1, ...] read by the conv kernels
@@ -363,6 +384,31 @@ struct Builder {
         H = a.Ho; W = a.Wo;
         plan->ops.push_back(op);
     }
+    // Stem (3 input channels): on bf16 handles with a filter count that is a multiple of 8 it runs on the
+    // tensor cores as patch matrix (tmp) x GEMM weights; otherwise as a direct convolution.
+    void stem(const std::string &name, int out, int tmp, int &H, int &W, int stride, int act) {
+        const int li = net->idx(name);
+        const StoredLayer &L = net->layers[li];
+        const Slice &s = plan->slices[li];
+        const size_t first = plan->ops.size();
+        const int Hin = H, Win = W;
+        conv(name, -1, out, -1, H, W, stride, act);
+        if (!net->stem_gemm_w || net->force_plain || s.K % 8 || (s.k != 3 && s.k != 7)) return;
+        Op &cv = plan->ops[first];
+        const int KKp = net->stem_kkp;
+        Op im;
+        im.type = OP_IM2COL; im.layer = li; im.in = -1; im.out = tmp;
+        im.N = N; im.H = Hin; im.W = Win; im.C = 3; im.K = KKp;
+        im.conv = cv.conv;  // geometry (k, stride, output dims)
+        im.alg_bytes = ((double)N * Hin * Win * 3 + (double)N * H * W * KKp) * net->elem();
+        cv.in = tmp;
+        ConvArgs &a = cv.conv;
+        a.w = net->stem_gemm_w;
+        a.H = H; a.W = W; a.C = KKp; a.Cmax = KKp; a.R = 1; a.k = 1; a.stride = 1;
+        note((size_t)N * H * W * KKp);
+        plan->ops.insert(plan->ops.begin() + (long)first, im);
+        (void)L;
+    }
     void linear(const std::string &name, int vin, int vout, int act) {
         int li = net->idx(name);
         const Slice &s = plan->slices[li];
@@ -391,7 +437,7 @@ sgs_status_t build_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batc
     // activation buffers: X current tensor, T1/T2 temporaries, SC shortcut
     int X = 0, T1 = 1, T2 = 2, SC = 3;
     if (net->family == SGS_TINY) {
-        B.conv("stem", -1, X, -1, H, W, 1, ACT_RELU);
+        B.stem("stem", X, T1, H, W, 1, ACT_RELU);
         for (int s = 0; s < 3; s++)
             for (int b = 0; b < cfg->depth[s]; b++) {
                 int st = b == 0 ? d.stride[s] : 1, shortcut = X;
@@ -405,7 +451,7 @@ sgs_status_t build_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batc
         B.gap(X, 0, H, W, C);
         B.linear("fc", 0, -1, ACT_NONE);
     } else if (net->family == SGS_RESNET) {
-        B.conv("stem", -1, T1, -1, H, W, 2, ACT_RELU);
+        B.stem("stem", T1, T2, H, W, 2, ACT_RELU);
         {
             Op op;
             op.type = OP_MAXPOOL; op.in = T1; op.out = X; op.N = batch; op.H = H; op.W = W; op.C = plan->slices[net->idx("stem")].K;
@@ -429,7 +475,7 @@ sgs_status_t build_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batc
         B.gap(X, 0, H, W, C);
         B.linear("fc", 0, -1, ACT_NONE);
     } else {
-        B.conv("stem", -1, X, -1, H, W, 2, ACT_HSWISH);
+        B.stem("stem", X, T1, H, W, 2, ACT_HSWISH);
         { int h = H, w = W; B.conv("first.dw", X, T1, -1, h, w, 1, ACT_RELU); }
         { int h = H, w = W; B.conv("first.pw", T1, T2, X, h, w, 1, ACT_NONE); }
         std::swap(X, T2);
@@ -561,6 +607,34 @@ sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
     return SGS_OK;
 }
 
+// Key of an op that is the same for every SubNet: its type and the stored layer it uses; ops without
+// a layer (pools, the SE scale) are anchored to the next op that has one.
+long long op_key(const Plan &p, size_t oi) {
+    int anchor = p.ops[oi].layer;
+    for (size_t j = oi + 1; anchor < 0 && j < p.ops.size(); j++) anchor = p.ops[j].layer;
+    return ((long long)p.ops[oi].type << 32) | (unsigned)anchor;
+}
+
+// The largest SubNet runs every op any SubNet runs, in the same relative order (depth keeps the first
+// blocks of a stage), so the position of an op in its op list orders the ops of all SubNets.
+sgs_status_t ensure_ranks(sgs_supernet *net) {
+    if (!net->op_rank.empty()) return SGS_OK;
+    sgs_subnet_cfg_t c;
+    std::memset(&c, 0, sizeof c);
+    const FamilyDef &d = net->def;
+    for (int s = 0; s < d.n_stages; s++) {
+        c.depth[s] = d.max_depth[s];
+        c.width[s + 1] = 1.0f;
+        for (int b = 0; b < SGS_MAX_BLOCKS; b++) { c.expand[s][b] = net->family == SGS_MBV3 ? 6.0f : 0.35f; c.kernel[s][b] = 7; }
+    }
+    c.width[0] = 1.0f;
+    Plan p;
+    sgs_status_t st = build_plan(net, &c, 1, 64, &p);
+    if (st != SGS_OK) return st;
+    for (size_t i = 0; i < p.ops.size(); i++) net->op_rank[op_key(p, i)] = (int)i;
+    return SGS_OK;
+}
+
 sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch, int res, int slot, Plan **out) {
     std::string key(reinterpret_cast<const char *>(cfg), sizeof(*cfg));
     key.append(reinterpret_cast<const char *>(&batch), sizeof batch);
@@ -577,16 +651,104 @@ sgs_status_t get_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batch,
     p->slot = slot;
     p->throughput = net->throughput_mode;
     p->enc = encoding_of(p->slices);
+    if ((st = ensure_ranks(net)) != SGS_OK) return st;
+    for (size_t i = 0; i < p->ops.size(); i++) {
+        auto it = net->op_rank.find(op_key(*p, i));
+        if (it == net->op_rank.end()) return fail(net, SGS_ECONFIG, "op outside the largest SubNet");
+        p->ops[i].rank = it->second;
+    }
     *out = p.get();
     net->plans.emplace(std::move(key), std::move(p));
+    return SGS_OK;
+}
+
+// Argument record of a max pool, global average pool, linear or patch-matrix op (bf16 handles).
+SmallEntry small_entry(const sgs_supernet *net, const Plan *plan, const Op &op, const void *d_input, void *d_logits) {
+    const sgs_supernet::Slot &sl = net->slots[plan->slot];
+    SmallEntry e;
+    std::memset(&e, 0, sizeof e);
+    switch (op.type) {
+    case OP_MAXPOOL:
+        e.x = op.in < 0 ? d_input : sl.act[op.in]; e.y = sl.act[op.out];
+        e.N = op.N; e.H = op.H; e.W = op.W; e.C = op.C; e.Ho = (op.H - 1) / 2 + 1; e.Wo = (op.W - 1) / 2 + 1;
+        break;
+    case OP_GAP:
+        e.x = op.in < 0 ? d_input : sl.act[op.in]; e.y = sl.vec[op.vout];
+        e.N = op.N; e.H = op.H; e.W = op.W; e.C = op.C;
+        break;
+    case OP_LINEAR: {
+        const StoredLayer &L = net->layers[op.layer];
+        e.x = sl.vec[op.vin]; e.y = op.vout < 0 ? d_logits : (void *)sl.vec[op.vout];
+        e.w = L.w; e.bias = L.shift;
+        e.N = op.N; e.C = op.C; e.K = op.K; e.ld = L.C; e.act = op.act;
+        break;
+    }
+    case OP_IM2COL:
+        e.x = d_input; e.y = sl.act[op.out];
+        e.N = op.N; e.H = op.H; e.W = op.W; e.C = 3;
+        e.Ho = op.conv.Ho; e.Wo = op.conv.Wo; e.k = op.conv.k; e.stride = op.conv.stride; e.KKp = op.K;
+        break;
+    default: break;
+    }
+    return e;
+}
+
+// Launches one op of a plan on `st`.
+template <typename T>
+sgs_status_t launch_op(sgs_supernet *net, Plan *plan, Op &op, const void *d_input, void *d_logits, cudaStream_t st) {
+    const sgs_supernet::Slot &sl = net->slots[plan->slot];
+    auto abuf = [&](int id) -> void * { return id < 0 ? const_cast<void *>(d_input) : sl.act[id]; };
+    switch (op.type) {
+    case OP_CONV:
+    case OP_DW: {
+        ConvArgs a = op.conv;
+        if (op.in < 0) a.x = d_input;
+        a.cache_tbl = net->cache_tbl; a.layer = op.layer;
+        a.ws = sl.ws; a.ws_elems = net->splitk_ws_elems;
+        if (op.type == OP_DW) { CU(launch_dw<T>(a, st)); net->kernel_launches++; }
+        else if (op.impl == 1) { int n = 0; CU(tc_conv_launch(*op.tc, a, st, &n)); net->kernel_launches += n; }
+        else { CU(launch_conv_plain<T>(a, st)); net->kernel_launches++; }
+        break;
+    }
+    case OP_IM2COL: {
+        SmallEntry e = small_entry(net, plan, op, d_input, d_logits);
+        CU(launch_small(OP_IM2COL, &e, nullptr, 1, st));
+        net->kernel_launches++;
+        break;
+    }
+    case OP_MAXPOOL:
+        CU(launch_maxpool3s2<T>((const T *)abuf(op.in), (T *)sl.act[op.out], op.N, op.H, op.W, op.C, st));
+        net->kernel_launches++;
+        break;
+    case OP_GAP:
+        CU(launch_gap<T>((const T *)abuf(op.in), sl.vec[op.vout], op.N, op.H * op.W, op.C, st));
+        net->kernel_launches++;
+        break;
+    case OP_SE_GATE: {
+        const StoredLayer &L1 = net->layers[op.layer], &L2 = net->layers[op.layer2];
+        CU(launch_se_gate<T>(sl.vec[op.vin], (const T *)L1.w, L1.shift, (const T *)L2.w, L2.shift, sl.vec[op.vout],
+                             op.N, op.C, op.K, L1.C, L2.C, st));
+        net->kernel_launches++;
+        break;
+    }
+    case OP_SCALE:
+        CU(launch_scale<T>((const T *)sl.act[op.in], sl.vec[op.vin], (T *)sl.act[op.out], op.N, op.H * op.W, op.C, st));
+        net->kernel_launches++;
+        break;
+    case OP_LINEAR: {
+        const StoredLayer &L = net->layers[op.layer];
+        float *y = op.vout < 0 ? static_cast<float *>(d_logits) : sl.vec[op.vout];
+        CU(launch_linear<T>(sl.vec[op.vin], (const T *)L.w, L.shift, y, op.N, op.C, op.K, L.C, op.act, st));
+        net->kernel_launches++;
+        break;
+    }
+    }
     return SGS_OK;
 }
 
 template <typename T>
 sgs_status_t run_ops(sgs_supernet *net, Plan *plan, const void *d_input, void *d_logits, cudaStream_t st, size_t first,
                      size_t last) {
-    const sgs_supernet::Slot &sl = net->slots[plan->slot];
-    auto abuf = [&](int id) -> void * { return id < 0 ? const_cast<void *>(d_input) : sl.act[id]; };
     for (size_t oi = first; oi < last; oi++) {
         Op &op = plan->ops[oi];
         if (net->profile) {
@@ -598,45 +760,8 @@ sgs_status_t run_ops(sgs_supernet *net, Plan *plan, const void *d_input, void *d
             }
             CU(cudaEventRecord(plan->prof_ev[2 * oi], st));
         }
-        switch (op.type) {
-        case OP_CONV:
-        case OP_DW: {
-            ConvArgs a = op.conv;
-            if (op.in < 0) a.x = d_input;
-            a.cache_tbl = net->cache_tbl; a.layer = op.layer;
-            a.ws = sl.ws; a.ws_elems = net->splitk_ws_elems;
-            if (op.type == OP_DW) { CU(launch_dw<T>(a, st)); net->kernel_launches++; }
-            else if (op.impl == 1) { int n = 0; CU(tc_conv_launch(*op.tc, a, st, &n)); net->kernel_launches += n; }
-            else { CU(launch_conv_plain<T>(a, st)); net->kernel_launches++; }
-            break;
-        }
-        case OP_MAXPOOL:
-            CU(launch_maxpool3s2<T>((const T *)abuf(op.in), (T *)sl.act[op.out], op.N, op.H, op.W, op.C, st));
-            net->kernel_launches++;
-            break;
-        case OP_GAP:
-            CU(launch_gap<T>((const T *)abuf(op.in), sl.vec[op.vout], op.N, op.H * op.W, op.C, st));
-            net->kernel_launches++;
-            break;
-        case OP_SE_GATE: {
-            const StoredLayer &L1 = net->layers[op.layer], &L2 = net->layers[op.layer2];
-            CU(launch_se_gate<T>(sl.vec[op.vin], (const T *)L1.w, L1.shift, (const T *)L2.w, L2.shift, sl.vec[op.vout],
-                                 op.N, op.C, op.K, L1.C, L2.C, st));
-            net->kernel_launches++;
-            break;
-        }
-        case OP_SCALE:
-            CU(launch_scale<T>((const T *)sl.act[op.in], sl.vec[op.vin], (T *)sl.act[op.out], op.N, op.H * op.W, op.C, st));
-            net->kernel_launches++;
-            break;
-        case OP_LINEAR: {
-            const StoredLayer &L = net->layers[op.layer];
-            float *y = op.vout < 0 ? static_cast<float *>(d_logits) : sl.vec[op.vout];
-            CU(launch_linear<T>(sl.vec[op.vin], (const T *)L.w, L.shift, y, op.N, op.C, op.K, L.C, op.act, st));
-            net->kernel_launches++;
-            break;
-        }
-        }
+        sgs_status_t rc = launch_op<T>(net, plan, op, d_input, d_logits, st);
+        if (rc != SGS_OK) return rc;
         if (net->profile) CU(cudaEventRecord(plan->prof_ev[2 * oi + 1], st));
     }
     return SGS_OK;
@@ -931,11 +1056,19 @@ sgs_status_t sgs_supernet_load(const sgs_arch_desc_t *arch, const void *host_blo
         net->by_name[sp.name] = (int)net->layers.size();
         net->layers.push_back(L);
     }
+    if (e == cudaSuccess && bf && !net->layers.empty() && net->layers[0].kind == KIND_CONV && net->layers[0].C == 3) {
+        const StoredLayer &L = net->layers[0];
+        const int KK = L.R * L.R * 3;
+        net->stem_kkp = (KK + 7) / 8 * 8;
+        if (dev_alloc(net, &net->stem_gemm_w, (size_t)L.K * net->stem_kkp * 2) != SGS_OK) e = cudaErrorMemoryAllocation;
+        else e = launch_stem_gemm_weights(L.w, net->stem_gemm_w, L.K, KK, net->stem_kkp, 0);
+    }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     cleanup_stage();
     if (e != cudaSuccess) { sgs_supernet_free(holder.release()); return e == cudaErrorMemoryAllocation ? SGS_ENOMEM : SGS_ECUDA; }
 
     int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && v > 0) net->sms = v;
     if (cudaDeviceGetAttribute(&v, cudaDevAttrL2CacheSize, device) == cudaSuccess) net->l2_bytes = (size_t)v;
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxPersistingL2CacheSize, device) == cudaSuccess) net->persist_max = (size_t)v;
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxAccessPolicyWindowSize, device) == cudaSuccess) net->window_max = (size_t)v;
@@ -968,6 +1101,7 @@ void sgs_supernet_free(sgs_supernet_t *net) {
     net->prof_used.clear();
     cudaFree(net->weight_arena);
     cudaFree(net->param_arena);
+    cudaFree(net->stem_gemm_w);
     for (auto &sl : net->slots) {
         for (int i = 0; i < 4; i++) cudaFree(sl.act[i]);
         for (int i = 0; i < 3; i++) cudaFree(sl.vec[i]);
@@ -976,6 +1110,14 @@ void sgs_supernet_free(sgs_supernet_t *net) {
         cudaFree(sl.stage_out);
         if (sl.ev) cudaEventDestroy(sl.ev);
         if (sl.st) cudaStreamDestroy(sl.st);
+    }
+    for (auto &w : net->waves) {
+        cudaFree(w.d_tbl);
+        cudaFreeHost(w.h_tbl);
+        cudaFree(w.stage_in);
+        cudaFree(w.stage_out);
+        if (w.done) cudaEventDestroy(w.done);
+        if (w.st) cudaStreamDestroy(w.st);
     }
     cudaFree(net->cache_tbl);
     cudaFreeHost(net->tbl_ring);
@@ -1026,6 +1168,246 @@ sgs_status_t sgs_subnet_run(sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, co
     return SGS_OK;
 }
 
+// ------------------------------------------------------------------------------------------
+// Wave execution of a stream.  `G` consecutive queries form a wave; the wave walks the op list of the
+// largest SubNet, and at every position the members whose SubNet has that op run it together: the
+// tensor-core convolutions of all members are ONE grouped launch (sgs_conv_group.cu), the remaining op
+// types are launched per member.  Up to `W` waves are in flight on their own streams.
+// ------------------------------------------------------------------------------------------
+static sgs_status_t ensure_waves(sgs_supernet *net, int W) {
+    while ((int)net->waves.size() < W) {
+        sgs_supernet::WaveCtx w;
+        CU(cudaStreamCreateWithFlags(&w.st, cudaStreamNonBlocking));
+        CU(cudaEventCreateWithFlags(&w.done, cudaEventDisableTiming));
+        net->waves.push_back(w);
+    }
+    return SGS_OK;
+}
+
+static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs, const void *inputs, int batch,
+                              int res, void *logits, const sgs_stream_opts_t &o, sgs_stream_stats_t *stats, cudaStream_t st,
+                              bool host_buffers) {
+    const int G = std::min(o.wave, TC_GROUP_MAX_ENTRIES);
+    const int W = std::max(1, std::min(o.concurrency ? o.concurrency : 2, 4));
+    sgs_status_t rc = ensure_slots(net, G * W);
+    if (rc != SGS_OK) return rc;
+    if ((rc = ensure_waves(net, W)) != SGS_OK) return rc;
+    if ((rc = ensure_ranks(net)) != SGS_OK) return rc;
+    net->throughput_mode = 2;
+    const size_t in_bytes = (size_t)batch * res * res * 3 * net->elem();
+    const size_t out_bytes = (size_t)batch * net->def.classes * sizeof(float);
+    const int n_ranks = (int)net->op_rank.size();
+    const int n_waves = (n_queries + G - 1) / G;
+    std::vector<cudaEvent_t> ev;  // per wave: start and end on the wave's stream
+    if (o.record_latency) {
+        ev.resize(2 * (size_t)n_waves);
+        for (auto &e : ev) CU(cudaEventCreate(&e));
+    }
+    cudaEvent_t e0, e1;
+    CU(cudaEventCreate(&e0));
+    CU(cudaEventCreate(&e1));
+    const long long launches0 = net->kernel_launches;
+    const int hits0 = net->plan_hits, miss0 = net->plan_misses;
+    double flops = 0, wbytes = 0, miss_bytes = 0, hit = 0;
+    int updates = 0;
+    CU(cudaEventRecord(e0, st));
+    for (int w = 0; w < W; w++) { CU(cudaStreamWaitEvent(net->waves[w].st, e0, 0)); net->waves[w].busy = false; }
+    const auto host_t0 = std::chrono::steady_clock::now();
+    std::vector<Plan *> plans((size_t)G);
+    std::vector<std::vector<std::pair<int, int>>> buckets((size_t)n_ranks);  // per rank: (member, op index)
+    struct Launch { int rank; GroupLaunch *group; int small_kind; size_t off; int count; };  // group == nullptr && small_kind < 0: the bucket's ungrouped ops, per member
+    std::vector<Launch> launches;
+    for (int wv = 0; wv < n_waves && rc == SGS_OK; wv++) {
+        const int ci = wv % W, q0 = wv * G, members = std::min(G, n_queries - q0);
+        // plans of the members (each member owns slot ci * G + m)
+        for (int m = 0; m < members && rc == SGS_OK; m++) {
+            rc = get_plan(net, &cfgs[q0 + m], batch, res, ci * G + m, &plans[m]);
+            if (rc == SGS_OK) rc = ensure_workspace(net, plans[m]->act_elems, batch);
+        }
+        for (int m = 0; m < members && rc == SGS_OK; m++)
+            if (!plans[m]->prepared) rc = choose_impls(net, plans[m]);
+        if (rc != SGS_OK) break;
+        sgs_supernet::WaveCtx &cx = net->waves[ci];  // (taken after ensure_*: the vector does not move later)
+        if (cx.busy) CU(cudaEventSynchronize(cx.done));  // its table image and staging buffers are free again
+        if (host_buffers) {
+            const size_t need_in = (size_t)G * in_bytes, need_out = (size_t)G * out_bytes;
+            if (cx.stage_in_bytes < need_in) {
+                dev_free(net, cx.stage_in, cx.stage_in_bytes); cx.stage_in = nullptr; cx.stage_in_bytes = 0;
+                if ((rc = dev_alloc(net, &cx.stage_in, need_in)) != SGS_OK) break;
+                cx.stage_in_bytes = need_in;
+            }
+            if (cx.stage_out_bytes < need_out) {
+                dev_free(net, cx.stage_out, cx.stage_out_bytes); cx.stage_out = nullptr; cx.stage_out_bytes = 0;
+                if ((rc = dev_alloc(net, (void **)&cx.stage_out, need_out)) != SGS_OK) break;
+                cx.stage_out_bytes = need_out;
+            }
+        }
+        // merge the members' op lists by rank
+        for (auto &b : buckets) b.clear();
+        size_t n_tc = 0;
+        for (int m = 0; m < members; m++)
+            for (size_t oi = 0; oi < plans[m]->ops.size(); oi++) {
+                buckets[(size_t)plans[m]->ops[oi].rank].emplace_back(m, (int)oi);
+                n_tc += plans[m]->ops[oi].impl == 1 && plans[m]->ops[oi].type == OP_CONV;
+            }
+        size_t n_small = 0;
+        for (int m = 0; m < members; m++) n_small += plans[m]->ops.size();
+        const size_t need_tbl = (n_tc + n_small) * TC_GROUP_ENTRY_BYTES + 256;
+        if (cx.tbl_bytes < need_tbl) {
+            cudaFreeHost(cx.h_tbl); cx.h_tbl = nullptr;
+            dev_free(net, cx.d_tbl, cx.tbl_bytes); cx.d_tbl = nullptr; cx.tbl_bytes = 0;
+            const size_t bytes = need_tbl * 2;
+            if (cudaMallocHost((void **)&cx.h_tbl, bytes) != cudaSuccess) { rc = fail(net, SGS_ENOMEM, "pinned launch table"); break; }
+            if ((rc = dev_alloc(net, (void **)&cx.d_tbl, bytes)) != SGS_OK) break;
+            cx.tbl_bytes = bytes;
+        }
+        const void *din0 = static_cast<const char *>(inputs) + (size_t)q0 * in_bytes;
+        void *dout0 = static_cast<char *>(logits) + (size_t)q0 * out_bytes;
+        // tables and parameter blocks of the grouped launches
+        launches.clear();
+        size_t off = 0, used = 0;
+        auto next_group = [&]() -> GroupLaunch * {
+            if (used == net->group_pool.size()) net->group_pool.emplace_back(new GroupLaunch);
+            GroupLaunch *g = net->group_pool[used++].get();
+            g->reset(cx.d_tbl + off);
+            return g;
+        };
+        for (int r = 0; r < n_ranks; r++) {
+            const auto &b = buckets[(size_t)r];
+            if (b.empty()) continue;
+            GroupLaunch *g = nullptr;
+            for (const auto &mo : b) {
+                Plan *pl = plans[mo.first];
+                const Op &op = pl->ops[(size_t)mo.second];
+                if (op.type != OP_CONV || op.impl != 1) continue;  // launched per member below
+                if (!g || !g->fits(*op.tc)) { g = next_group(); launches.push_back({r, g, -1, 0, 0}); }
+                ConvArgs a = op.conv;
+                a.layer = op.layer;
+                g->add(cx.h_tbl + off, *op.tc, a);
+                off += TC_GROUP_ENTRY_BYTES;
+            }
+            // max pool / average pool / linear / patch matrix: one launch over the members when every
+            // member's op has the vectorised form; the remaining ops run member by member
+            const Op &op0 = plans[b[0].first]->ops[(size_t)b[0].second];
+            const int kind = op0.type;
+            bool grouped = kind == OP_MAXPOOL || kind == OP_GAP || kind == OP_LINEAR || kind == OP_IM2COL;
+            if (grouped) {
+                const size_t off0 = off;
+                for (const auto &mo : b) {
+                    const void *xin = static_cast<const char *>(host_buffers ? cx.stage_in : din0) + (size_t)mo.first * in_bytes;
+                    void *yout = static_cast<char *>(host_buffers ? (void *)cx.stage_out : dout0) + (size_t)mo.first * out_bytes;
+                    SmallEntry se = small_entry(net, plans[mo.first], plans[mo.first]->ops[(size_t)mo.second], xin, yout);
+                    grouped = grouped && small_supported(kind, se);
+                    std::memcpy(cx.h_tbl + off, &se, sizeof se);
+                    off += sizeof se;
+                }
+                if (grouped) { launches.push_back({r, nullptr, kind, off0, (int)b.size()}); continue; }
+                off = off0;
+            }
+            launches.push_back({r, nullptr, -1, 0, 0});  // the bucket's remaining ops, member by member
+        }
+        cudaStream_t ws = cx.st;
+        const void *din = din0;
+        void *dout = dout0;
+        if (off) CU(cudaMemcpyAsync(cx.d_tbl, cx.h_tbl, off, cudaMemcpyHostToDevice, ws));
+        if ((rc = push_cache_table(net, ws)) != SGS_OK) break;
+        if (o.record_latency) CU(cudaEventRecord(ev[2 * (size_t)wv], ws));
+        if (host_buffers) {
+            CU(cudaMemcpyAsync(cx.stage_in, din, (size_t)members * in_bytes, cudaMemcpyHostToDevice, ws));
+            din = cx.stage_in;
+        }
+        void *dlog = host_buffers ? (void *)cx.stage_out : dout;
+        for (const Launch &L : launches) {
+            if (L.group) {
+                CU(L.group->launch(net->cache_tbl, net->sms, ws));
+                net->kernel_launches++;
+                continue;
+            }
+            if (L.small_kind >= 0) {
+                CU(launch_small(L.small_kind, reinterpret_cast<const SmallEntry *>(cx.h_tbl + L.off),
+                                reinterpret_cast<const SmallEntry *>(cx.d_tbl + L.off), L.count, ws));
+                net->kernel_launches++;
+                continue;
+            }
+            for (const auto &mo : buckets[(size_t)L.rank]) {
+                Plan *pl = plans[mo.first];
+                Op &op = pl->ops[(size_t)mo.second];
+                if (op.type == OP_CONV && op.impl == 1) continue;
+                const void *xin = static_cast<const char *>(din) + (size_t)mo.first * in_bytes;
+                void *yout = static_cast<char *>(dlog) + (size_t)mo.first * out_bytes;
+                rc = net->dtype == SGS_BF16 ? launch_op<__nv_bfloat16>(net, pl, op, xin, yout, ws) : launch_op<float>(net, pl, op, xin, yout, ws);
+                if (rc != SGS_OK) break;
+            }
+            if (rc != SGS_OK) break;
+        }
+        if (rc != SGS_OK) break;
+        if (host_buffers) CU(cudaMemcpyAsync(dout, cx.stage_out, (size_t)members * out_bytes, cudaMemcpyDeviceToHost, ws));
+        if (o.record_latency) CU(cudaEventRecord(ev[2 * (size_t)wv + 1], ws));
+        CU(cudaEventRecord(cx.done, ws));
+        cx.busy = true;
+        // accounting and cache policy follow the stream order; the device-side hints of a wave use the
+        // cached SubGraph as it stood when the wave was issued
+        for (int m = 0; m < members; m++) {
+            const int epoch_before = net->cache.epoch;
+            QueryAccount qa = account_query(net, plans[m]->enc);
+            flops += plans[m]->flops; wbytes += qa.weight_bytes; miss_bytes += qa.miss_bytes; hit += qa.hit_ratio;
+            if (net->cache.enabled) {
+                cache_observe(net, plans[m]->enc);
+                if (net->cache.epoch != epoch_before) updates++;
+            }
+        }
+    }
+    net->host_us_stream += std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - host_t0).count();
+    for (int w = 0; w < W; w++) {  // join
+        cudaEventRecord(net->waves[w].done, net->waves[w].st);
+        cudaStreamWaitEvent(st, net->waves[w].done, 0);
+    }
+    cudaError_t ce = cudaEventRecord(e1, st);
+    cudaError_t se = cudaStreamSynchronize(st);
+    if (rc == SGS_OK && (ce != cudaSuccess || se != cudaSuccess))
+        rc = fail(net, SGS_ECUDA, std::string("stream: ") + cudaGetErrorString(se != cudaSuccess ? se : ce));
+    if (rc != SGS_OK) cudaDeviceSynchronize();
+    if (rc == SGS_OK && tc_conv_status()) rc = fail(net, SGS_ETIMEOUT, "a bounded device-side wait ran out in the tensor-core kernel");
+    if (rc == SGS_OK && stats) {
+        std::memset(stats, 0, sizeof(*stats));
+        float ms = 0;
+        cudaEventElapsedTime(&ms, e0, e1);
+        stats->n_queries = n_queries;
+        stats->total_ms = ms;
+        stats->queries_per_s = ms > 0 ? n_queries / (ms * 1e-3) : 0;
+        stats->images_per_s = stats->queries_per_s * batch;
+        if (o.record_latency && n_queries) {
+            // every query of a wave starts and ends with its wave
+            std::vector<float> lat;
+            double sum = 0;
+            for (int wv = 0; wv < n_waves; wv++) {
+                float l = 0;
+                cudaEventElapsedTime(&l, ev[2 * (size_t)wv], ev[2 * (size_t)wv + 1]);
+                const int members = std::min(G, n_queries - wv * G);
+                for (int m = 0; m < members; m++) { lat.push_back(l); sum += l; }
+            }
+            std::sort(lat.begin(), lat.end());
+            stats->p50_ms = lat[(size_t)(n_queries - 1) / 2];
+            stats->p99_ms = lat[(size_t)std::min<long long>(n_queries - 1, (long long)std::ceil(0.99 * n_queries) - 1)];
+            stats->mean_ms = sum / n_queries;
+        }
+        stats->useful_flops = flops;
+        stats->weight_bytes = wbytes;
+        stats->hbm_weight_bytes = miss_bytes;
+        stats->hit_ratio = n_queries ? hit / n_queries : 0;
+        stats->byte_hit_ratio = wbytes > 0 ? 1.0 - miss_bytes / wbytes : 0;
+        stats->kernel_launches = net->kernel_launches - launches0;
+        stats->plan_hits = net->plan_hits - hits0;
+        stats->plan_misses = net->plan_misses - miss0;
+        stats->cache_updates = updates;
+    }
+    for (auto &e : ev) cudaEventDestroy(e);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    net->throughput_mode = 0;
+    return rc;
+}
+
 static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs, const void *inputs,
                                 int batch, int res, void *logits, const sgs_stream_opts_t *opts,
                                 sgs_stream_stats_t *stats, cudaStream_t st, bool host_buffers) {
@@ -1036,13 +1418,16 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
     if (!guard.ok) return fail(net, SGS_ECUDA, "cudaSetDevice failed");
     sgs_stream_opts_t o;
     if (opts) o = *opts;
-    else { o.cache_enabled = 1; o.window_q = 4; o.cache_budget_bytes = 0; o.use_graphs = 1; o.record_latency = 1; o.weights_evict_first = 0; o.concurrency = 1; }
+    else { o.cache_enabled = 1; o.window_q = 4; o.cache_budget_bytes = 0; o.use_graphs = 1; o.record_latency = 1; o.weights_evict_first = 0; o.concurrency = 1; o.wave = 0; }
     if (o.window_q < 1) return fail(net, SGS_EINVAL, "window_q must be >= 1");
     if (o.concurrency < 0 || o.concurrency > 16) return fail(net, SGS_EINVAL, "concurrency must be in [0, 16]");
     for (int t = 0; t < n_queries; t++)
         if (!cfg_valid(net, &cfgs[t])) return fail(net, SGS_ECONFIG, "query " + std::to_string(t) + ": config outside the elastic sets");
+    if (o.wave < 0) return fail(net, SGS_EINVAL, "wave must be >= 0");
     cache_reset(net, o.cache_enabled != 0, o.cache_budget_bytes, o.window_q);
     net->cache.evict_first_when_off = (!o.cache_enabled && o.weights_evict_first) ? 1 : 0;
+    if (o.wave > 0 && n_queries > 0 && !net->profile && net->dtype == SGS_BF16 && tc_available() && !net->force_plain)
+        return wave_impl(net, n_queries, cfgs, inputs, batch, res, logits, o, stats, st, host_buffers);
     // queries in flight at once: each runs in its own slot; per-kernel profiling wants them one by one
     const int S = net->profile ? 1 : std::max(1, std::min(o.concurrency ? o.concurrency : 1, std::max(1, n_queries)));
     {

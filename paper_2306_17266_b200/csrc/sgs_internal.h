@@ -56,13 +56,14 @@ struct ConvArgs {
     // (lets a captured graph follow cache updates without being re-captured)
     const int *cache_tbl = nullptr;
     int layer = 0;
-    int throughput = 0;  // 1: pick tiles for aggregate throughput (many launches in flight), 0: for the latency of this launch
+    int throughput = 0;  // 0: tiles for the latency of this launch; 1: for aggregate throughput (many launches in flight);
+                         // 2: member of a grouped launch (128-filter tiles, reduction never split)
     // split-K scratch of the tensor-core kernel: fp32 partial tiles [splits][M][K]
     float *ws = nullptr;
     size_t ws_elems = 0;
 };
 
-enum OpType { OP_CONV, OP_DW, OP_MAXPOOL, OP_GAP, OP_SE_GATE, OP_SCALE, OP_LINEAR };
+enum OpType { OP_CONV, OP_DW, OP_MAXPOOL, OP_GAP, OP_SE_GATE, OP_SCALE, OP_LINEAR, OP_IM2COL };
 
 struct TcConvPlan;  // tensor-core launch description (sgs_conv_tc.cu)
 
@@ -76,6 +77,7 @@ struct Op {
     int impl = 0;                     // 0 plain CUDA-core kernel, 1 tensor-core kernel
     double alg_bytes = 0, flops = 0;  // algorithmic traffic (weights + input + output + residual) and useful FLOPs
     std::shared_ptr<TcConvPlan> tc;
+    int rank = -1;                    // position of this op in the largest SubNet's op list (wave merging)
 };
 
 struct Plan {
@@ -112,6 +114,28 @@ cudaError_t launch_delay(unsigned microseconds, cudaStream_t st);  // one thread
 cudaError_t launch_fold_bn(const float *gamma, const float *beta, const float *mean, const float *var,
                            const float *bias, float *scale, float *shift, int K, cudaStream_t st);
 
+// ---- bf16 kernels that take their arguments as a record, alone or as one member of a grouped launch
+// (one launch serves many queries in flight: blockIdx.y selects the member's record in a device table)
+struct alignas(16) SmallEntry {
+    const void *x;       // input tensor / vector
+    void *y;             // output tensor / vector
+    const void *w;       // linear: weights [K][ld] bf16
+    const float *bias;   // linear: bias [K]
+    int N, H, W, C;      // input dims (linear: C inputs; gap: H*W pixels)
+    int K, ld, act;      // linear: outputs, row pitch of w, activation
+    int Ho, Wo;          // output dims (max pool, patch matrix)
+    int k, stride, KKp;  // patch matrix: kernel size, stride, padded row length
+    int pad_[12];
+};
+static_assert(sizeof(SmallEntry) == 128, "record size");
+// kind: OP_MAXPOOL (3x3 stride 2, C % 8 == 0), OP_GAP (C % 8 == 0), OP_LINEAR (C % 8 == 0, ld % 8 == 0),
+// OP_IM2COL (3 input channels; k in {3, 7}; stride in {1, 2}).  `h` is the host image of the `n` records
+// at device address `d` (it sizes the grid); with d == nullptr, n must be 1 and the record is passed by value.
+bool small_supported(int kind, const SmallEntry &e);
+cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int n, cudaStream_t st);
+// Stem weights as a GEMM operand: dst[f][kk] = src[f][kk] for kk < KK (the stored [K][R][R][3] row), 0 up to KKp.
+cudaError_t launch_stem_gemm_weights(const void *src, void *dst, int K, int KK, int KKp, cudaStream_t st);
+
 // ---- tensor-core convolution (sgs_conv_tc.cu) -----------------------------------------------
 // Returns nullptr when the shape is not handled by the tensor-core kernel (caller falls back).
 std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::string *why);
@@ -120,5 +144,33 @@ cudaError_t tc_conv_launch(const TcConvPlan &p, const ConvArgs &a, cudaStream_t 
 cudaError_t tc_conv_init(int device);  // one-time device set-up; call outside stream capture
 bool tc_available();
 int tc_conv_status();  // nonzero once any tensor-core kernel reported a bounded wait running out
+int *tc_status_word(int device);  // device address of that status word (after tc_conv_init), else nullptr
+
+// ---- grouped tensor-core convolution (sgs_conv_group.cu) -------------------------------------
+// One launch runs the same stored layer for up to TC_GROUP_MAX_ENTRIES members (queries in flight).
+// A member is described by a TC_GROUP_ENTRY_BYTES record in a device table and by its tensor maps,
+// which travel in the kernel's parameter block.  Plans for it are prepared with
+// ConvArgs::throughput == 2 (128-filter tiles, reduction never split).
+constexpr int TC_GROUP_ENTRY_BYTES = 128;
+constexpr int TC_GROUP_MAX_ENTRIES = 64;
+constexpr int TC_GROUP_MAPS_SMALL = 64, TC_GROUP_MAPS_LARGE = 248;  // tensor maps per launch (two kernel variants)
+class GroupLaunch {
+public:
+    GroupLaunch();
+    ~GroupLaunch();
+    GroupLaunch(const GroupLaunch &) = delete;
+    GroupLaunch &operator=(const GroupLaunch &) = delete;
+    void reset(const void *d_entries);       // start a launch whose member records will live at d_entries
+    bool fits(const TcConvPlan &p) const;   // room for one more member (records and tensor maps)?
+    // Adds a member: writes its record to host_entry (the host image of the next device record).
+    void add(void *host_entry, const TcConvPlan &p, const ConvArgs &a);
+    int members() const;
+    int tiles() const;
+    cudaError_t launch(const int *cache_tbl, int sms, cudaStream_t st);
+private:
+    struct Impl;
+    Impl *impl;
+};
+cudaError_t tc_group_init(int device);
 
 }  // namespace sgs

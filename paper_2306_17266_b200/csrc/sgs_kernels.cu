@@ -508,6 +508,197 @@ template cudaError_t launch_linear<float>(const float *, const float *, const fl
 template cudaError_t launch_linear<__nv_bfloat16>(const float *, const __nv_bfloat16 *, const float *, float *, int, int, int, int, int, cudaStream_t);
 
 // ---------------------------------------------------------------------------------------------
+// Record-driven bf16 kernels (see SmallEntry): each body works on one member; the `single` kernels get
+// the record by value, the `group` kernels pick it from a device table with blockIdx.y.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t bf2_max(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&a), *reinterpret_cast<const __nv_bfloat162 *>(&b));
+    return *reinterpret_cast<uint32_t *>(&r);
+}
+
+// 3x3 stride-2 max pool, padding 1: a thread owns 8 channels of one output pixel.
+__device__ __forceinline__ void maxpool_body(const SmallEntry &e, int bx, int nbx) {
+    const int cv = e.C >> 3;
+    const int total = e.N * e.Ho * e.Wo * cv;
+    const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(e.x);
+    __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(e.y);
+    for (int i = bx * blockDim.x + threadIdx.x; i < total; i += nbx * blockDim.x) {
+        const int c = i % cv, m = i / cv;
+        const int wo = m % e.Wo, ho = (m / e.Wo) % e.Ho, n = m / (e.Wo * e.Ho);
+        uint4 best = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);  // -inf pairs
+#pragma unroll
+        for (int r = 0; r < 3; r++) {
+            const int hi = 2 * ho + r - 1;
+            if (hi < 0 || hi >= e.H) continue;
+#pragma unroll
+            for (int s = 0; s < 3; s++) {
+                const int wi = 2 * wo + s - 1;
+                if (wi < 0 || wi >= e.W) continue;
+                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x + (((size_t)n * e.H + hi) * e.W + wi) * e.C) + c);
+                best.x = bf2_max(best.x, v.x); best.y = bf2_max(best.y, v.y); best.z = bf2_max(best.z, v.z); best.w = bf2_max(best.w, v.w);
+            }
+        }
+        reinterpret_cast<uint4 *>(y + (size_t)m * e.C)[c] = best;
+    }
+}
+
+// Global average pool: one warp per 8-channel vector of one image (fixed shuffle tree).
+__device__ __forceinline__ void gap_body(const SmallEntry &e, int bx) {
+    const int warp = (bx * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const int cvecs = e.C >> 3, HW = e.H * e.W;
+    if (warp >= e.N * cvecs) return;
+    const int n = warp / cvecs, cv = warp % cvecs;
+    const __nv_bfloat16 *base = static_cast<const __nv_bfloat16 *>(e.x) + (size_t)n * HW * e.C + cv * 8;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int i = lane; i < HW; i += 32) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(base + (size_t)i * e.C));
+        const float2 a = bf2f(v.x), b = bf2f(v.y), c = bf2f(v.z), d = bf2f(v.w);
+        acc[0] += a.x; acc[1] += a.y; acc[2] += b.x; acc[3] += b.y; acc[4] += c.x; acc[5] += c.y; acc[6] += d.x; acc[7] += d.y;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; j++)
+#pragma unroll
+        for (int o = 16; o; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+    if (lane == 0) {
+        const float inv = 1.f / (float)HW;
+        float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(e.y) + (size_t)n * e.C + cv * 8);
+        dst[0] = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+        dst[1] = make_float4(acc[4] * inv, acc[5] * inv, acc[6] * inv, acc[7] * inv);
+    }
+}
+
+// Sliced linear layer on fp32 vectors: one warp per (image, output), 16-byte weight loads.
+__device__ __forceinline__ void linear_body(const SmallEntry &e, int bx) {
+    const int warp = (bx * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= e.N * e.K) return;
+    const int n = warp / e.K, j = warp % e.K;
+    const __nv_bfloat16 *wr = static_cast<const __nv_bfloat16 *>(e.w) + (size_t)j * e.ld;
+    const float *vr = static_cast<const float *>(e.x) + (size_t)n * e.C;
+    float s = 0.f;
+    for (int c = lane * 8; c < e.C; c += 256) {
+        const uint4 wv = __ldg(reinterpret_cast<const uint4 *>(wr + c));
+        const float4 x0 = *reinterpret_cast<const float4 *>(vr + c), x1 = *reinterpret_cast<const float4 *>(vr + c + 4);
+        const float2 a = bf2f(wv.x), b = bf2f(wv.y), cc = bf2f(wv.z), d = bf2f(wv.w);
+        s = fmaf(a.x, x0.x, s); s = fmaf(a.y, x0.y, s); s = fmaf(b.x, x0.z, s); s = fmaf(b.y, x0.w, s);
+        s = fmaf(cc.x, x1.x, s); s = fmaf(cc.y, x1.y, s); s = fmaf(d.x, x1.z, s); s = fmaf(d.y, x1.w, s);
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) static_cast<float *>(e.y)[(size_t)n * e.K + j] = apply_act(s + e.bias[j], e.act);
+}
+
+// Patch matrix of a convolution with 3 input channels (the stems): row m = output pixel, column
+// kk = (r * k + s) * 3 + c holds x[n][ho*st + r - p][wo*st + s - p][c] (0 outside the image and for the
+// padding columns kk >= k*k*3).  With it the stem is a GEMM on the tensor cores like every other layer.
+// A thread writes 8 consecutive columns of one row (one 16-byte store).
+template <int K, int ST>
+__device__ __forceinline__ void im2col_body(const SmallEntry &e, int bx, int nbx) {
+    constexpr int P = (K - 1) / 2, KK = K * K * 3;
+    const int gv = e.KKp >> 3;
+    const int total = e.N * e.Ho * e.Wo * gv;
+    const unsigned short *x = static_cast<const unsigned short *>(e.x);
+    uint4 *y = static_cast<uint4 *>(e.y);
+    for (int i = bx * blockDim.x + threadIdx.x; i < total; i += nbx * blockDim.x) {
+        const int g = i % gv, m = i / gv;
+        const int wo = m % e.Wo, ho = (m / e.Wo) % e.Ho, n = m / (e.Wo * e.Ho);
+        const unsigned short *ximg = x + (size_t)n * e.H * e.W * 3;
+        unsigned short v[8];
+#pragma unroll
+        for (int q = 0; q < 8; q++) {
+            const int kk = g * 8 + q;
+            const int c = kk % 3, rs = kk / 3, s = rs % K, r = rs / K;
+            const int hi = ho * ST + r - P, wi = wo * ST + s - P;
+            v[q] = (kk < KK && hi >= 0 && hi < e.H && wi >= 0 && wi < e.W) ? __ldg(ximg + ((size_t)hi * e.W + wi) * 3 + c) : (unsigned short)0;
+        }
+        y[i] = make_uint4(v[0] | ((uint32_t)v[1] << 16), v[2] | ((uint32_t)v[3] << 16), v[4] | ((uint32_t)v[5] << 16), v[6] | ((uint32_t)v[7] << 16));
+    }
+}
+
+template <int KIND, int K, int ST> __device__ __forceinline__ void small_body(const SmallEntry &e, int bx, int nbx) {
+    if (KIND == OP_MAXPOOL) maxpool_body(e, bx, nbx);
+    else if (KIND == OP_GAP) gap_body(e, bx);
+    else if (KIND == OP_LINEAR) linear_body(e, bx);
+    else im2col_body<K, ST>(e, bx, nbx);
+}
+template <int KIND, int K, int ST> __global__ void __launch_bounds__(256) small_single_kernel(const SmallEntry e) {
+    small_body<KIND, K, ST>(e, blockIdx.x, gridDim.x);
+}
+template <int KIND, int K, int ST> __global__ void __launch_bounds__(256) small_group_kernel(const SmallEntry *__restrict__ tbl) {
+    __shared__ SmallEntry e;
+    if (threadIdx.x < 8) reinterpret_cast<uint4 *>(&e)[threadIdx.x] = __ldg(reinterpret_cast<const uint4 *>(tbl + blockIdx.y) + threadIdx.x);
+    __syncthreads();
+    small_body<KIND, K, ST>(e, blockIdx.x, gridDim.x);
+}
+
+bool small_supported(int kind, const SmallEntry &e) {
+    auto al = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
+    if (!al(e.x) || !al(e.y)) return false;
+    switch (kind) {
+    case OP_MAXPOOL: return e.C % 8 == 0 && (long long)e.N * e.Ho * e.Wo * (e.C / 8) < (1ll << 31);
+    case OP_GAP: return e.C % 8 == 0;
+    case OP_LINEAR: return e.C % 8 == 0 && e.ld % 8 == 0 && al(e.w);
+    case OP_IM2COL: return (e.k == 3 || e.k == 7) && (e.stride == 1 || e.stride == 2) && e.KKp % 8 == 0 && e.KKp >= e.k * e.k * 3 &&
+                           (long long)e.N * e.Ho * e.Wo * (e.KKp / 8) < (1ll << 31);
+    default: return false;
+    }
+}
+
+// blocks along x that one member needs
+static long long small_blocks(int kind, const SmallEntry &e) {
+    switch (kind) {
+    case OP_MAXPOOL: return ((long long)e.N * e.Ho * e.Wo * (e.C / 8) + 255) / 256;
+    case OP_GAP: return ((long long)e.N * (e.C / 8) * 32 + 255) / 256;
+    case OP_LINEAR: return ((long long)e.N * e.K * 32 + 255) / 256;
+    default: return ((long long)e.N * e.Ho * e.Wo * (e.KKp / 8) + 255) / 256;
+    }
+}
+
+template <int KIND, int K, int ST>
+static cudaError_t launch_small_t(const SmallEntry *h, const SmallEntry *d, int n, unsigned bx, cudaStream_t st) {
+    if (d) small_group_kernel<KIND, K, ST><<<dim3(bx, (unsigned)n), 256, 0, st>>>(d);
+    else small_single_kernel<KIND, K, ST><<<bx, 256, 0, st>>>(*h);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int n, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    if ((!d && n != 1) || n > 65535) return cudaErrorInvalidValue;
+    long long blocks = 1;
+    for (int i = 0; i < n; i++) blocks = std::max(blocks, small_blocks(kind, h[i]));
+    // grid-stride kernels (max pool, patch matrix) need not cover every element with a block of their own
+    if (kind == OP_MAXPOOL || kind == OP_IM2COL) blocks = std::min<long long>(blocks, 148 * 16);
+    const unsigned bx = (unsigned)blocks;
+    switch (kind) {
+    case OP_MAXPOOL: return launch_small_t<OP_MAXPOOL, 0, 0>(h, d, n, bx, st);
+    case OP_GAP: return launch_small_t<OP_GAP, 0, 0>(h, d, n, bx, st);
+    case OP_LINEAR: return launch_small_t<OP_LINEAR, 0, 0>(h, d, n, bx, st);
+    case OP_IM2COL: {
+        const int key = h[0].k * 10 + h[0].stride;
+        for (int i = 1; i < n; i++)
+            if (h[i].k * 10 + h[i].stride != key) return cudaErrorInvalidValue;
+        if (key == 72) return launch_small_t<OP_IM2COL, 7, 2>(h, d, n, bx, st);
+        if (key == 71) return launch_small_t<OP_IM2COL, 7, 1>(h, d, n, bx, st);
+        if (key == 32) return launch_small_t<OP_IM2COL, 3, 2>(h, d, n, bx, st);
+        if (key == 31) return launch_small_t<OP_IM2COL, 3, 1>(h, d, n, bx, st);
+        return cudaErrorInvalidValue;
+    }
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+__global__ void stem_gemm_weights_kernel(const __nv_bfloat16 *__restrict__ src, __nv_bfloat16 *__restrict__ dst, int K, int KK, int KKp) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= K * KKp) return;
+    const int f = i / KKp, kk = i % KKp;
+    dst[i] = kk < KK ? src[(size_t)f * KK + kk] : __float2bfloat16_rn(0.f);
+}
+cudaError_t launch_stem_gemm_weights(const void *src, void *dst, int K, int KK, int KKp, cudaStream_t st) {
+    const int total = K * KKp;
+    stem_gemm_weights_kernel<<<(total + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(src), static_cast<__nv_bfloat16 *>(dst), K, KK, KKp);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Load-time kernels
 // ---------------------------------------------------------------------------------------------
 template <typename T>

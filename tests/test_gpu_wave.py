@@ -1,0 +1,96 @@
+"""GPU parity of the wave execution (grouped launches over many queries in flight) against the CPU checker.
+
+Same tolerance as the other bf16 parity tests: max|err| <= 2e-2 * max|ref| per output row against the
+checker run with the same storage rounding points.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2306_17266_b200 as sgs
+from paper_2306_17266_b200 import workload as wl
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+
+
+def _run(gnet, cfgs, d_in, batch, res, n_classes, wave, conc, host=False, latency=0):
+    n = len(cfgs)
+    stream = torch.cuda.Stream()
+    opts = sgs.StreamOpts(cache_enabled=1, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=latency,
+                          concurrency=conc, wave=wave)
+    if host:
+        h_out = np.zeros((n * batch, n_classes), dtype=np.float32)
+        h_in = d_in.cpu().view(torch.int16).numpy()
+        st = gnet.stream_run(cfgs, h_in, batch, res, h_out, opts, stream.cuda_stream, host=True)
+        return h_out, st
+    d_out = torch.zeros((n * batch, n_classes), dtype=torch.float32, device="cuda")
+    torch.cuda.synchronize()
+    st = gnet.stream_run(cfgs, d_in.data_ptr(), batch, res, d_out.data_ptr(), opts, stream.cuda_stream)
+    return d_out.cpu().numpy(), st
+
+
+def test_resnet_wave_matches_checker_and_is_deterministic():
+    # 21 queries in waves of 8 (a ragged last wave of 5), two waves in flight, 64x64 inputs
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    n, res = 21, 64
+    cfgs = wl.uniform_stream(wl.RESNET, n - 2, seed=11) + [wl.extreme_cfg(wl.RESNET, False), wl.extreme_cfg(wl.RESNET, True)]
+    xs = wl.make_inputs(n, 1, res, seed=5, bf16=True)
+    d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
+    got, st = _run(gnet, cfgs, d_in, 1, res, 1000, wave=8, conc=2, latency=1)
+    assert st.p50_ms > 0 and st.kernel_launches > 0
+    for t in range(n):
+        ref = onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)
+        assert gu.rel_err(got[t:t + 1], ref) <= TOL_BF16, t
+    again, _ = _run(gnet, cfgs, d_in, 1, res, 1000, wave=8, conc=2)
+    np.testing.assert_array_equal(again, got)
+    # other wave sizes and the host-buffer variant give the same bits (a tile never depends on its neighbours)
+    for wave, conc in ((1, 1), (5, 3), (64, 1)):
+        other, _ = _run(gnet, cfgs, d_in, 1, res, 1000, wave=wave, conc=conc)
+        np.testing.assert_array_equal(other, got)
+    hosted, _ = _run(gnet, cfgs, d_in, 1, res, 1000, wave=8, conc=2, host=True)
+    np.testing.assert_array_equal(hosted, got)
+
+
+def test_resnet_wave_accounting_equals_the_sequential_stream():
+    # the cache policy and its byte accounting follow the stream order whatever the execution mode
+    _, _, gnet = gu.nets(wl.RESNET, True)
+    n, res = 16, 64
+    cfgs = wl.markov_stream(n, seed=9)
+    d_in = gu.to_device(wl.make_inputs(n, 1, res, seed=2, bf16=True).reshape(n, res, res, 3), True)
+    _, seq = _run(gnet, cfgs, d_in, 1, res, 1000, wave=0, conc=1)
+    _, wav = _run(gnet, cfgs, d_in, 1, res, 1000, wave=8, conc=2)
+    assert wav.hit_ratio == seq.hit_ratio and wav.hbm_weight_bytes == seq.hbm_weight_bytes
+    assert wav.weight_bytes == seq.weight_bytes and wav.useful_flops == seq.useful_flops
+    assert wav.kernel_launches < seq.kernel_launches
+
+
+def test_resnet_wave_batched_members_224():
+    # members with several images each (4 configs x 4 images), full resolution: sampled against the checker
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    groups, batch, res = 4, 4, 224
+    cfgs = wl.uniform_stream(wl.RESNET, groups, seed=5)
+    xs = wl.make_inputs(groups, batch, res, seed=3, bf16=True)
+    d_in = gu.to_device(xs.reshape(groups * batch, res, res, 3), True)
+    got, _ = _run(gnet, cfgs, d_in, batch, res, 1000, wave=4, conc=1)
+    assert np.all(np.isfinite(got))
+    for g in (0, 3):
+        ref = onet.forward(cfgs[g], xs[g], oracle.BF16_STORE)
+        assert gu.rel_err(got[g * batch:(g + 1) * batch], ref) <= TOL_BF16, g
+
+
+def test_wave_mode_on_the_other_families():
+    # MobileNetV3-shaped (depthwise, SE) and Tiny SuperNets: ops without a grouped kernel run per member
+    for fam, res, ncls in ((wl.MBV3, 64, 1000), (wl.TINY, 32, 10)):
+        _, onet, gnet = gu.nets(fam, True)
+        n = 6
+        cfgs = wl.uniform_stream(fam, n, seed=7)
+        xs = wl.make_inputs(n, 1, res, seed=8, bf16=True)
+        d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
+        got, _ = _run(gnet, cfgs, d_in, 1, res, ncls, wave=4, conc=2)
+        for t in range(n):
+            ref = onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)
+            assert gu.rel_err(got[t:t + 1], ref) <= TOL_BF16, (fam, t)
