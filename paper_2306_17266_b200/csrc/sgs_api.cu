@@ -1219,6 +1219,13 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
     std::vector<Launch> launches;
     for (int wv = 0; wv < n_waves && rc == SGS_OK; wv++) {
         const int ci = wv % W, q0 = wv * G, members = std::min(G, n_queries - q0);
+        auto tick = [](std::chrono::steady_clock::time_point &t0) {
+            const auto now = std::chrono::steady_clock::now();
+            const double us = std::chrono::duration<double, std::micro>(now - t0).count();
+            t0 = now;
+            return us;
+        };
+        auto tp = std::chrono::steady_clock::now();
         // plans of the members (each member owns slot ci * G + m)
         for (int m = 0; m < members && rc == SGS_OK; m++) {
             rc = get_plan(net, &cfgs[q0 + m], batch, res, ci * G + m, &plans[m]);
@@ -1227,8 +1234,10 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
         for (int m = 0; m < members && rc == SGS_OK; m++)
             if (!plans[m]->prepared) rc = choose_impls(net, plans[m]);
         if (rc != SGS_OK) break;
+        net->host_us_query += tick(tp);
         sgs_supernet::WaveCtx &cx = net->waves[ci];  // (taken after ensure_*: the vector does not move later)
         if (cx.busy) CU(cudaEventSynchronize(cx.done));  // its table image and staging buffers are free again
+        net->host_us_direct += tick(tp);
         if (host_buffers) {
             const size_t need_in = (size_t)G * in_bytes, need_out = (size_t)G * out_bytes;
             if (cx.stage_in_bytes < need_in) {
@@ -1306,6 +1315,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             }
             launches.push_back({r, nullptr, -1, 0, 0});  // the bucket's remaining ops, member by member
         }
+        net->host_us_table += tick(tp);
         cudaStream_t ws = cx.st;
         const void *din = din0;
         void *dout = dout0;
@@ -1345,6 +1355,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
         if (o.record_latency) CU(cudaEventRecord(ev[2 * (size_t)wv + 1], ws));
         CU(cudaEventRecord(cx.done, ws));
         cx.busy = true;
+        net->host_us_graph += tick(tp);
         // accounting and cache policy follow the stream order; the device-side hints of a wave use the
         // cached SubGraph as it stood when the wave was issued
         for (int m = 0; m < members; m++) {

@@ -2,9 +2,9 @@
 // with its own SubNet slice (paper Section 2.1: every query selects its own filters / channels of the
 // shared layer; Section 3.1: a stream of such queries).  A launch gets a table with one entry per
 // member (query): its tensor maps, slice extents, tile geometry and buffers.  All members' output tiles
-// form one list of tiles; persistent CTAs (two per SM) walk that list with a fixed stride.
+// form one list of tiles; persistent CTAs (one per SM) walk that list with a fixed stride.
 //
-// Per CTA: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = epilogue.  The shared-memory ring
+// Per CTA: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = epilogue.  The shared-memory ring
 // of operand stages runs on across tiles, and the fp32 accumulator in tensor memory is double
 // buffered (2 x 128 columns), so the epilogue of tile j (tensor memory -> folded batch norm ->
 // residual -> activation -> bf16 NHWC) overlaps the loads and MMAs of tile j + 1.
@@ -19,25 +19,41 @@
 
 namespace sgs {
 
+#ifdef SGS_ROLE_TIMING
+__device__ unsigned long long g_role_cycles[16];
+#endif
+
 namespace {
 
-constexpr int G_BN = 128;
-constexpr int G_STAGES = 3;
-constexpr int G_STAGE_BYTES = A_STAGE_BYTES + G_BN * CHUNK_C * 2;
-constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + 1024;
+constexpr int G_MAX_STAGES = 6;
+constexpr int G_X_BYTES = 128 * CHUNK_C * 2;  // operand on the MMA's row side: 128 rows
+constexpr int G_RING_BYTES = 192 * 1024;      // operand ring: 6 stages of 16 + 16 KB, or 4 stages of 16 + 32 KB (256-column tiles)
+constexpr int G_SMEM_BYTES = G_RING_BYTES + 1024;
+constexpr int G_ACC_COLS = 256;                   // tensor-memory columns of one accumulator buffer
+constexpr int G_EPI_WARPS = 8;                    // two per tensor-memory lane quadrant: each takes part of the columns
+constexpr int G_THREADS = 64 + 32 * G_EPI_WARPS + 32;  // weight producer, MMA warp, epilogue warps, pixel producer
+constexpr int G_PIX_WARP = 2 + G_EPI_WARPS;
 
+// One member (query) of a grouped launch.
+//   normal  : MMA rows = a box of <= 128 output pixels, MMA columns = bn_tile (64 / 128 / 256) filters
+//   swapped : MMA rows = 128 filters, MMA columns = ALL output pixels of the member (<= 256, padded to 16)
 struct __align__(16) GroupEntry {
-    int map_a, map_w;        // indices into the launch's tensor maps: activation view(s) (4 for stride-2 kernels
-                             // larger than 1x1: the parity views; else 1) and the sliced weight view
     const float *scale, *shift;
     const __nv_bfloat16 *res;
     __nv_bfloat16 *y;
+    int map_a, map_w;        // indices into the launch's tensor maps: activation view(s) (4 for stride-2 kernels
+                             // larger than 1x1: the parity views; else 1) and the sliced weight view
     int tile_begin;          // index of this member's first tile in the launch's tile list
-    int mtiles, ntiles;      // pixel tiles and filter tiles of this member
+    int mtiles;              // pixel tiles of this member (tile = filter tile * mtiles + pixel tile)
     int N, Ho, Wo, K, C;
-    int k, stride, R, o, p;
-    int bw, bh, bn, tiles_w, tiles_h;
-    int cchunks, iters, act, layer;
+    int R, tap0;             // stored kernel size; tap index of the cropped kernel's first tap
+    int tiles_w, tiles_hw, cchunks, iters, layer;
+    short bw, bh, bn;        // pixel box
+    short bn_tile;           // MMA columns of a full tile
+    short pix_rows;          // rows of the pixel box (bw * bh * bn)
+    short pad0_;
+    unsigned char k, stride, p, act, swap, pad1_[3];
+    int pad2_[3];
 };
 static_assert(sizeof(GroupEntry) == TC_GROUP_ENTRY_BYTES, "entry size");
 
@@ -47,8 +63,32 @@ __device__ __forceinline__ int find_entry(const GroupEntry *es, int n, int t, in
     const unsigned b1 = __ballot_sync(0xffffffffu, lane + 32 < n && es[lane + 32].tile_begin <= t);
     return __popc(b0) + __popc(b1) - 1;
 }
+// Same for one thread.
+__device__ __forceinline__ int find_entry_serial(const GroupEntry *es, int n, int t) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (es[mid].tile_begin <= t) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
 
-__device__ __forceinline__ void epilogue_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void epilogue_bar() { asm volatile("bar.sync 1, %0;" ::"n"(32 * G_EPI_WARPS) : "memory"); }
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *m) { asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory"); }
+
+// Where the epilogue splits a tile's columns between the two warps of a lane quadrant (a multiple of 32).
+__device__ __forceinline__ int split_cols(int ncols) { return ((ncols + 63) >> 6) << 5; }
+
+#ifdef SGS_ROLE_TIMING
+// Development aid (not compiled into the library): cycles each warp role spends waiting, summed over CTAs and launches.
+#define ROLE_T0() const long long rt0_ = clock64()
+#define ROLE_ADD(var) var += clock64() - rt0_
+#define ROLE_FLUSH(idx, var) do { if (lane == 0) atomicAdd(&g_role_cycles[idx], (unsigned long long)(var)); } while (0)
+#else
+#define ROLE_T0()
+#define ROLE_ADD(var)
+#define ROLE_FLUSH(idx, var)
+#endif
 
 // Kernel parameters.  The tensor maps travel in the parameter block (the TMA unit reads them from
 // there); the per-member records travel in a device table.
@@ -57,22 +97,22 @@ template <int NMAPS> struct GroupParams {
     const int *cache_tbl;
     int *status;
     int n_entries, total_tiles;
-    int pad_[8];
+    int n_stages, stage_bytes;  // operand ring of this launch
+    int pad_[6];
     CUtensorMap maps[NMAPS];
 };
 static_assert(sizeof(GroupParams<TC_GROUP_MAPS_LARGE>) <= 32764, "kernel parameter block");
 
 template <int NMAPS>
-__global__ void __launch_bounds__(192, 1) conv_group_kernel(const __grid_constant__ GroupParams<NMAPS> P) {
+__global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_constant__ GroupParams<NMAPS> P) {
     const GroupEntry *__restrict__ entries = P.entries;
     const int n_entries = P.n_entries, total_tiles = P.total_tiles;
     const int *__restrict__ cache_tbl = P.cache_tbl;
     int *status = P.status;
     extern __shared__ uint8_t smem_raw[];
     __shared__ GroupEntry es[TC_GROUP_MAX_ENTRIES];
-    __shared__ int row_m[TILE_M];  // output pixel index of each tile row, -1 outside the tensor
-    __shared__ float scale_s[G_BN], shift_s[G_BN];
-    __shared__ __align__(8) uint64_t full_bar[G_STAGES], empty_bar[G_STAGES], acc_full[2], acc_empty[2];
+    __shared__ float scale_s[2][G_ACC_COLS], shift_s[2][G_ACC_COLS];  // folded batch norm of the current / next tile's filters (normal tiles)
+    __shared__ __align__(8) uint64_t full_bar[G_MAX_STAGES], empty_bar[G_MAX_STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
@@ -85,183 +125,307 @@ __global__ void __launch_bounds__(192, 1) conv_group_kernel(const __grid_constan
     for (int i = threadIdx.x; i < n_entries * (int)(sizeof(GroupEntry) / 16); i += blockDim.x)
         reinterpret_cast<uint4 *>(es)[i] = __ldg(reinterpret_cast<const uint4 *>(entries) + i);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < G_STAGES; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        // a stage is full once both producers' copies have landed; it is empty once its MMAs have read it
+        for (int s = 0; s < G_MAX_STAGES; s++) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], G_EPI_WARPS); }
         abort_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(&tmem_base_s, 2 * G_BN);
+    if (warp == 1) tmem_alloc(&tmem_base_s, 2 * G_ACC_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
+    const int n_stages = P.n_stages, stage_bytes = P.stage_bytes;
     pdl_launch_dependents();
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ weight producer
+        // Weights do not depend on the previous layer, so this warp never waits for it: it runs ahead
+        // as far as the ring allows.  The warp runs its loop converged; one elected lane issues.
         const uint64_t pol_keep = make_policy(1), pol_stream = make_policy(2);
         const int weight_policy = cache_tbl ? __ldg(cache_tbl) : 0;
-        uint32_t it = 0;
-        bool first = true;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-            const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
-            const int local = t - e.tile_begin, nt = local / e.mtiles, mt = local % e.mtiles;
-            const int tiles_hw = e.tiles_w * e.tiles_h;
-            const int n0 = (mt / tiles_hw) * e.bn, h0 = ((mt % tiles_hw) / e.tiles_w) * e.bh, w0 = (mt % e.tiles_w) * e.bw;
-            const int f0 = nt * G_BN;
-            const uint32_t tx = (uint32_t)(e.bw * e.bh * e.bn * CHUNK_C * 2 + G_BN * CHUNK_C * 2);
-            const CUtensorMap *map_a = &P.maps[e.map_a], *map_w = &P.maps[e.map_w];
-            const int k = e.k, cchunks = e.cchunks, iters = e.iters, R = e.R, o = e.o, pad = e.p, stride = e.stride;
-            int cacheK = 0, cacheC = 0;
-            if (weight_policy == 1) { cacheK = __ldg(cache_tbl + 1 + 2 * e.layer); cacheC = __ldg(cache_tbl + 2 + 2 * e.layer); }
-            auto load_weights = [&](int s, int c0, int tapw) {
-                uint8_t *sb = smem + s * G_STAGE_BYTES + A_STAGE_BYTES;
-                mbar_expect_tx(&full_bar[s], tx);
-                // weight tiles inside the cached SubGraph's box are kept in L2 (evict-last); policy 2
-                // marks every weight load evict-first (the "no reuse" reference point)
-                if (weight_policy == 2) tma_load_3d_hint(sb, map_w, &full_bar[s], c0, tapw, f0, pol_stream);
-                else if (weight_policy == 1 && f0 < cacheK && c0 < cacheC) tma_load_3d_hint(sb, map_w, &full_bar[s], c0, tapw, f0, pol_keep);
-                else tma_load_3d(sb, map_w, &full_bar[s], c0, tapw, f0);
-            };
-            int pre = 0;
-            if (first) {
-                // Weights do not depend on the previous layer: the first stages' weight halves are
-                // requested before waiting for it.
-                first = false;
-                pre = min(iters, G_STAGES);
-                int cc2 = 0, r2 = 0, sx2 = 0;
-                for (int i = 0; i < pre; i++) {
-                    if (elect_one()) load_weights(i, cc2 * CHUNK_C, (o + r2) * R + (o + sx2));
-                    __syncwarp();
-                    if (++cc2 == cchunks) { cc2 = 0; if (++sx2 == k) { sx2 = 0; ++r2; } }
-                }
-                pdl_wait();
-            }
-            int cc = 0, r = 0, sx = 0;
-            bool ok = true;
-            for (int i = 0; i < iters; i++, it++) {
-                const int s = it % G_STAGES;
-                const uint32_t round = it / G_STAGES;
-                ok = round == 0 || mbar_wait(&empty_bar[s], (round - 1) & 1, abort_flag);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const int c0 = cc * CHUNK_C;
-                uint8_t *sa = smem + s * G_STAGE_BYTES;
-                const int dh = r - pad, dw = sx - pad;
-                if (elect_one()) {
-                    if (i >= pre) load_weights(s, c0, (o + r) * R + (o + sx));
-                    if (stride == 1) {
-                        tma_load_4d(sa, map_a, &full_bar[s], c0, w0 + dw, h0 + dh, n0);
-                    } else {
-                        const int ph = dh & 1, pw = dw & 1;
-                        tma_load_4d(sa, map_a + ph * 2 + pw, &full_bar[s], c0, w0 + ((dw - pw) >> 1), h0 + ((dh - ph) >> 1), n0);
-                    }
-                }
-                __syncwarp();
-                if (++cc == cchunks) { cc = 0; if (++sx == k) { sx = 0; ++r; } }
-            }
-            if (!ok) break;
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        uint32_t it = 0;
-        int j = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, j++) {
+        int s = 0;
+        uint32_t phase = 0;
+        bool wrapped = false, ok = true;
+        long long tw_ = 0; (void)tw_;
+        const long long tk0_ = clock64(); (void)tk0_;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
             const int nt = (t - e.tile_begin) / e.mtiles;
-            const int f0 = nt * G_BN;
-            const int n_mma = min(G_BN, (e.K - f0 + 15) & ~15);
+            const int wrows = e.swap ? 128 : e.bn_tile;  // rows of the weight box
+            const int f0 = nt * wrows;
+            const uint32_t w_bytes = (uint32_t)(wrows * CHUNK_C * 2);
+            uint8_t *dst0 = smem + (e.swap ? 0 : G_X_BYTES);
+            const CUtensorMap *map_w = &P.maps[e.map_w];
+            const int k = e.k, cchunks = e.cchunks, R = e.R;
+            int kind = 0;  // 0 default replacement, 1 keep (inside the cached SubGraph's box, up to channel cacheC), 2 stream
+            int cacheC = 0;
+            if (weight_policy == 2) kind = 2;
+            else if (weight_policy == 1 && f0 < __ldg(cache_tbl + 1 + 2 * e.layer)) { kind = 1; cacheC = __ldg(cache_tbl + 2 + 2 * e.layer); }
+            int tap_row = e.tap0;
+            for (int r = 0; r < k && ok; r++, tap_row += R) {
+                for (int sx = 0; sx < k && ok; sx++) {
+                    for (int cc = 0, c0 = 0; cc < cchunks; cc++, c0 += CHUNK_C) {
+                        { ROLE_T0(); if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag)); ROLE_ADD(tw_); }
+                        if (!ok) break;
+                        if (elect_one()) {
+                            uint8_t *sb = dst0 + s * stage_bytes;
+                            mbar_expect_tx(&full_bar[s], w_bytes);
+                            if (kind == 2) tma_load_3d_hint(sb, map_w, &full_bar[s], c0, tap_row + sx, f0, pol_stream);
+                            else if (kind == 1 && c0 < cacheC) tma_load_3d_hint(sb, map_w, &full_bar[s], c0, tap_row + sx, f0, pol_keep);
+                            else tma_load_3d(sb, map_w, &full_bar[s], c0, tap_row + sx, f0);
+                        }
+                        __syncwarp();
+                        if (++s == n_stages) { s = 0; phase ^= 1; wrapped = true; }
+                    }
+                }
+            }
+            const int tn = t + (int)gridDim.x;
+            if (ok && tn < total_tiles && elect_one()) prefetch_tensormap(&P.maps[es[find_entry_serial(es, n_entries, tn)].map_w]);
+            __syncwarp();
+        }
+        ROLE_FLUSH(0, tw_); ROLE_FLUSH(1, clock64() - tk0_);
+    } else if (warp == G_PIX_WARP) {
+        // ------------------------------------------------------------------ activation producer
+        int s = 0;
+        uint32_t phase = 0;
+        bool wrapped = false, ok = true;
+        long long tw_ = 0, tpdl_ = 0; (void)tw_; (void)tpdl_;
+        const long long tk0_ = clock64(); (void)tk0_;
+        { ROLE_T0(); pdl_wait(); ROLE_ADD(tpdl_); }  // activations (and the buffers this layer overwrites) belong to the previous layers until here
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
+            const int mt = (t - e.tile_begin) % e.mtiles;
+            const int n0 = (mt / e.tiles_hw) * e.bn, h0 = ((mt % e.tiles_hw) / e.tiles_w) * e.bh, w0 = (mt % e.tiles_w) * e.bw;
+            const uint32_t pix_bytes = (uint32_t)(e.pix_rows * CHUNK_C * 2);
+            uint8_t *dst0 = smem + (e.swap ? G_X_BYTES : 0);
+            const CUtensorMap *map_a = &P.maps[e.map_a];
+            const int k = e.k, cchunks = e.cchunks, pad = e.p, stride = e.stride;
+            for (int r = 0; r < k && ok; r++) {
+                for (int sx = 0; sx < k && ok; sx++) {
+                    const int dh = r - pad, dw = sx - pad;
+                    // stride 2: one of the four parity views, at half the offset
+                    const int ph = stride == 2 ? (dh & 1) : 0, pw = stride == 2 ? (dw & 1) : 0;
+                    const CUtensorMap *m = map_a + ph * 2 + pw;
+                    const int cw = stride == 2 ? w0 + ((dw - pw) >> 1) : w0 + dw, ch = stride == 2 ? h0 + ((dh - ph) >> 1) : h0 + dh;
+                    for (int cc = 0, c0 = 0; cc < cchunks; cc++, c0 += CHUNK_C) {
+                        { ROLE_T0(); if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag)); ROLE_ADD(tw_); }
+                        if (!ok) break;
+                        if (elect_one()) {
+                            mbar_expect_tx(&full_bar[s], pix_bytes);
+                            tma_load_4d(dst0 + s * stage_bytes, m, &full_bar[s], c0, cw, ch, n0);
+                        }
+                        __syncwarp();
+                        if (++s == n_stages) { s = 0; phase ^= 1; wrapped = true; }
+                    }
+                }
+            }
+            const int tn = t + (int)gridDim.x;
+            if (ok && tn < total_tiles && elect_one()) prefetch_tensormap(&P.maps[es[find_entry_serial(es, n_entries, tn)].map_a]);
+            __syncwarp();
+        }
+        ROLE_FLUSH(2, tw_); ROLE_FLUSH(3, tpdl_); ROLE_FLUSH(4, clock64() - tk0_);
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        int s = 0;
+        uint32_t phase = 0;
+        int j = 0;
+        const uint32_t ring = smem_u32(smem);
+        bool ok = true;
+        long long tfull_ = 0, tacc_ = 0; (void)tfull_; (void)tacc_;
+        const long long tk0_ = clock64(); (void)tk0_;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, j++) {
+            const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
+            const int nt = (t - e.tile_begin) / e.mtiles;
+            // MMA shape: 128 rows; columns = this tile's filters (normal) or the member's pixels (swapped),
+            // rounded up to 16; bf16 x bf16 -> fp32, both operands K-major
+            const int n_mma = e.swap ? e.bn_tile : min((int)e.bn_tile, (e.K - nt * e.bn_tile + 15) & ~15);
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
             const int buf = j & 1;
-            const int C = e.C, cchunks = e.cchunks, iters = e.iters;
-            bool ok = j < 2 || mbar_wait(&acc_empty[buf], ((j >> 1) - 1) & 1, abort_flag);  // epilogue drained this buffer
-            ok = __all_sync(0xffffffffu, ok);
+            const int cchunks = e.cchunks, taps = e.k * e.k;
+            const int last_ksteps = (e.C - (cchunks - 1) * CHUNK_C + 15) / 16;  // 16-channel steps of a tap's last chunk
+            { ROLE_T0(); ok = j < 2 || mbar_wait(&acc_empty[buf], ((j >> 1) - 1) & 1, abort_flag);  // epilogue drained this buffer
+            ok = __all_sync(0xffffffffu, ok); ROLE_ADD(tacc_); }
             if (!ok) break;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * G_BN);
-            int cc = 0;
-            for (int i = 0; i < iters; i++, it++) {
-                const int s = it % G_STAGES;
-                const uint32_t round = it / G_STAGES;
-                ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], round & 1, abort_flag));
-                if (!ok) break;
-                tc_fence_after();
-                const int ksteps = (min(CHUNK_C, C - cc * CHUNK_C) + 15) / 16;
-                const uint32_t sa = smem_u32(smem + s * G_STAGE_BYTES), sb = sa + A_STAGE_BYTES;
-                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
-                if (elect_one()) {
-                    for (int q = 0; q < ksteps; q++)
-                        umma_bf16(d_tmem, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), idesc, (i > 0 || q > 0) ? 1u : 0u);
-                    umma_commit(&empty_bar[s]);
-                    if (i == iters - 1) umma_commit(&acc_full[buf]);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * G_ACC_COLS);
+            uint32_t accumulate = 0;
+            for (int tap = 0; tap < taps && ok; tap++) {
+                for (int cc = 0; cc < cchunks; cc++) {
+                    { ROLE_T0(); ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], phase, abort_flag)); ROLE_ADD(tfull_); }
+                    if (!ok) break;
+                    tc_fence_after();
+                    const int ksteps = cc == cchunks - 1 ? last_ksteps : CHUNK_C / 16;
+                    const uint32_t sx_ = ring + (uint32_t)(s * stage_bytes);
+                    const uint64_t da = smem_desc_sw128(sx_), db = smem_desc_sw128(sx_ + G_X_BYTES);
+                    if (elect_one()) {
+                        for (int q = 0; q < ksteps; q++) { umma_bf16(d_tmem, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), idesc, accumulate); accumulate = 1; }
+                        umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+                        if (tap == taps - 1 && cc == cchunks - 1) umma_commit(&acc_full[buf]);  // accumulator complete
+                    }
+                    __syncwarp();
+                    accumulate = 1;
+                    if (++s == n_stages) { s = 0; phase ^= 1; }
                 }
-                __syncwarp();
-                if (++cc == cchunks) cc = 0;
             }
-            if (!ok) break;
         }
+        ROLE_FLUSH(5, tfull_); ROLE_FLUSH(6, tacc_); ROLE_FLUSH(7, clock64() - tk0_);
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
-        const int quad = warp & 3;         // TMEM lane quadrant this warp may read
-        const int row = quad * 32 + lane;  // tile row = output pixel within the box
-        const int et = threadIdx.x - 64;   // 0..127
-        pdl_wait();  // residual reads and output writes must not pass the previous layers
-        bool alive = true;  // after a failed wait the warp only keeps the named barriers in step
+        // ------------------------------------------------------------------ epilogue (warps 2..9)
+        // Two warps share a tensor-memory lane quadrant; each takes part of the tile's columns.
+        const int quad = warp & 3;                // tensor-memory lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;         // which part of the columns
+        const int row = quad * 32 + lane;         // accumulator row: output pixel (normal) or filter (swapped)
+        const int et = threadIdx.x - 64;          // 0..255
+        long long tpdl_ = 0, tbar_ = 0, tacc_ = 0, twork_ = 0; (void)tpdl_; (void)tbar_; (void)tacc_; (void)twork_;
+        const long long tk0_ = clock64(); (void)tk0_;
+        { ROLE_T0(); pdl_wait(); ROLE_ADD(tpdl_); }  // residual reads and output writes must not pass the previous layers
+        bool alive = true;  // after a failed wait the warp only keeps the named barrier in step
+        // folded batch norm of a normal tile: thread et fetches filter et's scale and shift
+        auto fetch_bn = [&](int tile, float *sc, float *sh) {
+            *sc = 0.f; *sh = 0.f;
+            if (tile >= total_tiles) return;
+            const GroupEntry &e = es[find_entry(es, n_entries, tile, lane)];
+            if (e.swap) return;
+            const int f = ((tile - e.tile_begin) / e.mtiles) * e.bn_tile + et;
+            if (et < e.bn_tile && f < e.K) { *sc = __ldg(e.scale + f); *sh = __ldg(e.shift + f); }
+        };
+        {
+            float sc, sh;
+            fetch_bn(blockIdx.x, &sc, &sh);
+            scale_s[0][et] = sc; shift_s[0][et] = sh;
+        }
         int j = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, j++) {
             const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
             const int local = t - e.tile_begin, nt = local / e.mtiles, mt = local % e.mtiles;
-            const int tiles_hw = e.tiles_w * e.tiles_h;
-            const int n0 = (mt / tiles_hw) * e.bn, h0 = ((mt % tiles_hw) / e.tiles_w) * e.bh, w0 = (mt % e.tiles_w) * e.bw;
-            const int f0 = nt * G_BN;
             const int K = e.K, act = e.act;
             const __nv_bfloat16 *res = e.res;
             __nv_bfloat16 *y = e.y;
-            epilogue_bar();  // every epilogue thread is done with the previous tile's tables
-            {
-                const int rows = e.bw * e.bh * e.bn;
-                const int dn = row / (e.bh * e.bw), dhh = (row / e.bw) % e.bh, dww = row % e.bw;
-                const int n = n0 + dn, h = h0 + dhh, w = w0 + dww;
-                const bool valid = row < rows && n < e.N && h < e.Ho && w < e.Wo;
-                row_m[row] = valid ? (int)(((size_t)n * e.Ho + h) * e.Wo + w) : -1;
-                const int f = f0 + et;
-                scale_s[et] = f < K ? __ldg(e.scale + f) : 0.f;
-                shift_s[et] = f < K ? __ldg(e.shift + f) : 0.f;
-            }
-            epilogue_bar();
             const int buf = j & 1;
-            if (alive) {
-                bool ok = mbar_wait(&acc_full[buf], (j >> 1) & 1, abort_flag);
-                alive = __all_sync(0xffffffffu, ok);
-            }
-            if (!alive) continue;
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * G_BN);
-            const int ncols = min(G_BN, K - f0);  // filters of this tile, a multiple of 8
-            const int m = row_m[row];
-#pragma unroll 1
-            for (int j0 = 0; j0 < ncols; j0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(taddr + j0, v);
-                tmem_ld_wait();
-                if (m >= 0) {
+            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * G_ACC_COLS);
+            float nsc, nsh;
+            fetch_bn(t + (int)gridDim.x, &nsc, &nsh);  // requested now, stored after this tile's work
+            if (!e.swap) {
+                // ---- normal tile: this thread owns output pixel `m`, columns are filters
+                const int n0 = (mt / e.tiles_hw) * e.bn, h0 = ((mt % e.tiles_hw) / e.tiles_w) * e.bh, w0 = (mt % e.tiles_w) * e.bw;
+                const int f0 = nt * e.bn_tile;
+                int m;
+                {
+                    const int dn = row / (e.bh * e.bw), dhh = (row / e.bw) % e.bh, dww = row % e.bw;
+                    const int n = n0 + dn, h = h0 + dhh, w = w0 + dww;
+                    const bool valid = row < e.pix_rows && n < e.N && h < e.Ho && w < e.Wo;
+                    m = valid ? (int)(((size_t)n * e.Ho + h) * e.Wo + w) : -1;
+                }
+                const int ncols = min((int)e.bn_tile, K - f0);  // filters of this tile, a multiple of 8
+                const int split = split_cols(ncols);
+                const int cbeg = half ? split : 0, cend = half ? ncols : min(ncols, split);
+                const size_t obase = (size_t)(m < 0 ? 0 : m) * K + f0;
+                // the residual does not depend on the accumulator: the first 32 columns' part is requested
+                // before waiting, every further part one step ahead of its use
+                auto load_res = [&](int c0, uint4 *rv) {
 #pragma unroll
                     for (int g = 0; g < 4; g++) {
-                        const int c = j0 + 8 * g;
-                        if (c < ncols) {
-                            float ov[8];
+                        const int c = c0 + 8 * g;
+                        rv[g] = (res && m >= 0 && c < cend) ? __ldg(reinterpret_cast<const uint4 *>(res + obase + c)) : make_uint4(0u, 0u, 0u, 0u);
+                    }
+                };
+                uint4 rv[4];
+                load_res(cbeg, rv);
+                { ROLE_T0(); epilogue_bar(); ROLE_ADD(tbar_); }  // this tile's scale / shift (written during the previous tile) are visible
+                const float *sc = scale_s[buf], *sh = shift_s[buf];
+                { ROLE_T0(); if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (j >> 1) & 1, abort_flag)); ROLE_ADD(tacc_); }
+                ROLE_T0();
+                if (alive) {
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c0 = cbeg; c0 < cend; c0 += 32) {  // warp-uniform bounds
+                        uint32_t v[32];
+                        tmem_ld32(tacc + c0, v);
+                        uint4 rn[4];
+                        load_res(c0 + 32, rn);
+                        tmem_ld_wait();
+                        if (m >= 0) {
 #pragma unroll
-                            for (int q = 0; q < 8; q++) ov[q] = __uint_as_float(v[8 * g + q]) * scale_s[c + q] + shift_s[c + q];
-                            finish_store(ov, res, y, (size_t)m * K + f0 + c, act);
+                            for (int g = 0; g < 4; g++) {
+                                const int c = c0 + 8 * g;
+                                if (c < cend) {
+                                    float ov[8];
+#pragma unroll
+                                    for (int q = 0; q < 8; q++) ov[q] = __uint_as_float(v[8 * g + q]) * sc[c + q] + sh[c + q];
+                                    const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv[g]);
+#pragma unroll
+                                    for (int q = 0; q < 4; q++) { const float2 f2 = __bfloat1622float2(rb[q]); ov[2 * q] += f2.x; ov[2 * q + 1] += f2.y; }
+                                    finish_store(ov, nullptr, y, obase + c, act);
+                                }
+                            }
                         }
+#pragma unroll
+                        for (int g = 0; g < 4; g++) rv[g] = rn[g];
+                    }
+                }
+                ROLE_ADD(twork_);
+            } else {
+                // ---- swapped tile: this thread owns filter `f`, columns are the member's output pixels
+                const int f = nt * 128 + row;
+                const bool fvalid = f < K;
+                const int npix = e.pix_rows;  // == N * Ho * Wo: the pixel tile is the whole member
+                const int split = split_cols(npix);
+                const int cbeg = half ? split : 0, cend = half ? npix : min(npix, split);
+                float sc = 0.f, sh = 0.f;
+                if (fvalid) { sc = __ldg(e.scale + f); sh = __ldg(e.shift + f); }
+                const unsigned short *resu = reinterpret_cast<const unsigned short *>(res);
+                auto load_res = [&](int c0, uint32_t *rv) {  // 32 pixels, two per register
+#pragma unroll
+                    for (int q = 0; q < 16; q++) {
+                        const int p0 = c0 + 2 * q;
+                        uint32_t lo = 0, hi = 0;
+                        if (res && fvalid && p0 < cend) lo = __ldg(resu + (size_t)p0 * K + f);
+                        if (res && fvalid && p0 + 1 < cend) hi = __ldg(resu + (size_t)(p0 + 1) * K + f);
+                        rv[q] = lo | (hi << 16);
+                    }
+                };
+                uint32_t rv[16];
+                load_res(cbeg, rv);
+                epilogue_bar();
+                if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (j >> 1) & 1, abort_flag));
+                if (alive) {
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c0 = cbeg; c0 < cend; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(tacc + c0, v);
+                        uint32_t rn[16];
+                        load_res(c0 + 32, rn);
+                        tmem_ld_wait();
+                        if (fvalid) {
+#pragma unroll
+                            for (int q = 0; q < 32; q++) {
+                                const int px = c0 + q;
+                                if (px < cend) {
+                                    const uint32_t rbits = (q & 1) ? (rv[q >> 1] & 0xffff0000u) : (rv[q >> 1] << 16);
+                                    const float o = act_fn(__uint_as_float(v[q]) * sc + sh + __uint_as_float(rbits), act);
+                                    y[(size_t)px * K + f] = __float2bfloat16_rn(o);
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < 16; q++) rv[q] = rn[q];
                     }
                 }
             }
-            // hand the accumulator buffer back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            if (alive) {
+                // hand the accumulator buffer back to the MMA warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            }
+            // all epilogue threads read buffer buf ^ 1 for the last time during tile j - 1, which they have
+            // all left (barrier above)
+            scale_s[buf ^ 1][et] = nsc; shift_s[buf ^ 1][et] = nsh;
         }
+        if (warp == 2) { ROLE_FLUSH(8, tpdl_); ROLE_FLUSH(9, tbar_); ROLE_FLUSH(10, tacc_); ROLE_FLUSH(11, twork_); ROLE_FLUSH(12, clock64() - tk0_); }
     }
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
@@ -272,7 +436,7 @@ __global__ void __launch_bounds__(192, 1) conv_group_kernel(const __grid_constan
         while (global_ns() - t0 < 2000000ull) __nanosleep(1000);
         __syncthreads();
     }
-    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 2 * G_BN); }
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 2 * G_ACC_COLS); }
 }
 
 }  // namespace
@@ -284,6 +448,7 @@ static int views_of(const TcParams &p) { return (p.stride == 2 && p.k > 1) ? 4 :
 struct GroupLaunch::Impl {
     GroupParams<TC_GROUP_MAPS_LARGE> prm;  // host image of the parameter block (the small variant is a prefix)
     int n_maps = 0;
+    bool wide = false;  // some member's column-side operand has more than 128 rows
 };
 
 GroupLaunch::GroupLaunch() : impl(new Impl) { reset(nullptr); }
@@ -291,6 +456,7 @@ GroupLaunch::~GroupLaunch() { delete impl; }
 
 void GroupLaunch::reset(const void *d_entries) {
     impl->n_maps = 0;
+    impl->wide = false;
     impl->prm.entries = static_cast<const GroupEntry *>(d_entries);
     impl->prm.n_entries = 0;
     impl->prm.total_tiles = 0;
@@ -318,14 +484,19 @@ void GroupLaunch::add(void *host_entry, const TcConvPlan &pl, const ConvArgs &a)
     e.y = static_cast<__nv_bfloat16 *>(a.y);
     e.tile_begin = impl->prm.total_tiles;
     e.mtiles = (int)pl.grid.x;
-    e.ntiles = (a.K + G_BN - 1) / G_BN;
     e.N = p.N; e.Ho = p.Ho; e.Wo = p.Wo; e.K = p.K; e.C = p.C;
-    e.k = p.k; e.stride = p.stride; e.R = p.R; e.o = p.o; e.p = p.p;
-    e.bw = p.bw; e.bh = p.bh; e.bn = p.bn; e.tiles_w = p.tiles_w; e.tiles_h = p.tiles_h;
-    e.cchunks = p.cchunks; e.iters = p.iters; e.act = p.act; e.layer = a.layer;
+    e.R = p.R; e.tap0 = p.o * p.R + p.o;
+    e.tiles_w = p.tiles_w; e.tiles_hw = p.tiles_w * p.tiles_h;
+    e.cchunks = p.cchunks; e.iters = p.iters; e.layer = a.layer;
+    e.bw = (short)p.bw; e.bh = (short)p.bh; e.bn = (short)p.bn;
+    e.pix_rows = (short)(p.bw * p.bh * p.bn);
+    e.swap = (unsigned char)pl.swap;
+    e.bn_tile = (short)(pl.swap ? (e.pix_rows + 15) / 16 * 16 : pl.bn_tile);
+    e.k = (unsigned char)p.k; e.stride = (unsigned char)p.stride; e.p = (unsigned char)p.p; e.act = (unsigned char)p.act;
+    if ((pl.swap ? e.pix_rows : e.bn_tile) > 128) impl->wide = true;
     std::memcpy(host_entry, &e, sizeof e);
     impl->prm.n_entries++;
-    impl->prm.total_tiles += e.mtiles * e.ntiles;
+    impl->prm.total_tiles += e.mtiles * (int)pl.grid.y;
 }
 
 cudaError_t tc_group_init(int) {
@@ -342,9 +513,12 @@ cudaError_t GroupLaunch::launch(const int *cache_tbl, int sms, cudaStream_t st) 
     impl->prm.status = tc_status_word(dev);
     if (!impl->prm.status) return cudaErrorInitializationError;
     impl->prm.cache_tbl = cache_tbl;
+    // 256-column tiles need 16 + 32 KB per stage (4 stages); everything narrower gets 6 stages of 16 + 16 KB
+    impl->prm.stage_bytes = G_X_BYTES + (impl->wide ? 256 : 128) * CHUNK_C * 2;
+    impl->prm.n_stages = G_RING_BYTES / impl->prm.stage_bytes;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)std::min(impl->prm.total_tiles, 2 * std::max(1, sms)));
-    cfg.blockDim = dim3(192);
+    cfg.gridDim = dim3((unsigned)std::min(impl->prm.total_tiles, std::max(1, sms)));
+    cfg.blockDim = dim3(G_THREADS);
     cfg.dynamicSmemBytes = G_SMEM_BYTES;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -362,3 +536,14 @@ cudaError_t GroupLaunch::launch(const int *cache_tbl, int sms, cudaStream_t st) 
 }
 
 }  // namespace sgs
+
+#ifdef SGS_ROLE_TIMING
+extern "C" int sgs_debug_role_cycles(unsigned long long *out16, int reset) {
+    cudaError_t e = cudaMemcpyFromSymbol(out16, sgs::g_role_cycles, sizeof(unsigned long long) * 16);
+    if (e == cudaSuccess && reset) {
+        unsigned long long z[16] = {};
+        e = cudaMemcpyToSymbol(sgs::g_role_cycles, z, sizeof z);
+    }
+    return e == cudaSuccess ? 0 : 1;
+}
+#endif

@@ -386,16 +386,24 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
     p.act = a.act;
     const bool flat = a.k == 1 && a.stride == 1;
     const uint64_t C = (uint64_t)a.C, eb = 2;
+    // Grouped launches (throughput == 2) run a layer with very few output pixels "swapped": the filters
+    // take the 128-row side of the MMA and ALL pixels of the member form the other operand (one pixel
+    // tile), so that no MMA rows are wasted on a 2x2 or 4x4 map.  (The kernel takes up to 256 pixels
+    // this way; measured on 7x7 and 14x14 maps it was no faster than pixel rows, so the limit is 32.)
+    const long long m_total = (long long)a.N * a.Ho * a.Wo;
+    const bool swap = a.throughput == 2 && m_total <= 32;
+    plan->swap = swap ? 1 : 0;
     if (flat) {
         // 1x1 stride 1: the activation tensor is a plain [M][C] matrix, tiles are 128 consecutive pixels
         const uint64_t M = (uint64_t)a.N * a.H * a.W;
-        p.bw = TILE_M; p.bh = 1; p.bn = 1;
+        p.bw = swap ? (int)M : TILE_M; p.bh = 1; p.bn = 1;
         p.N = 1; p.Ho = 1; p.Wo = (int)M;
         uint64_t dims[4] = {C, M, 1, 1}, str[3] = {C * eb, M * C * eb, M * C * eb};
-        uint32_t box[4] = {CHUNK_C, TILE_M, 1, 1};
+        uint32_t box[4] = {CHUNK_C, (uint32_t)p.bw, 1, 1};
         if (!encode_map(&p.tmA[0], a.x, 4, dims, str, box)) return no("activation tensor map");
     } else {
-        choose_box(a.N, a.Ho, a.Wo, &p.bw, &p.bh, &p.bn);
+        if (swap) { p.bw = a.Wo; p.bh = a.Ho; p.bn = a.N; }
+        else choose_box(a.N, a.Ho, a.Wo, &p.bw, &p.bh, &p.bn);
         uint32_t box[4] = {CHUNK_C, (uint32_t)p.bw, (uint32_t)p.bh, (uint32_t)p.bn};
         if (a.stride == 1) {
             uint64_t dims[4] = {C, (uint64_t)a.W, (uint64_t)a.H, (uint64_t)a.N};
@@ -442,7 +450,12 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
         BN = a.K > 64 ? 128 : 64;
         max_splits = p.iters >= 32 ? std::min(4, p.iters / 8) : 1;
     }
-    if (a.throughput == 2) { BN = 128; max_splits = 1; }  // grouped launch: one tile shape, no split
+    if (a.throughput == 2) {
+        // grouped launch: no split; filter tile = the narrowest of 64 / 128 / 256 that holds the layer
+        // (256 at most), or 128 filters on the MMA's row side when swapped
+        max_splits = 1;
+        BN = swap ? 128 : a.K <= 64 ? 64 : a.K <= 128 ? 128 : 256;
+    }
     plan->bn_tile = BN;
     {
         uint64_t dims[3] = {C, (uint64_t)a.R * a.R, (uint64_t)a.K};

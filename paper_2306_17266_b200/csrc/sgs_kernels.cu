@@ -590,35 +590,47 @@ __device__ __forceinline__ void linear_body(const SmallEntry &e, int bx) {
 // Patch matrix of a convolution with 3 input channels (the stems): row m = output pixel, column
 // kk = (r * k + s) * 3 + c holds x[n][ho*st + r - p][wo*st + s - p][c] (0 outside the image and for the
 // padding columns kk >= k*k*3).  With it the stem is a GEMM on the tensor cores like every other layer.
-// A thread writes 8 consecutive columns of one row (one 16-byte store).
+// A block owns one output row of one image: it stages the k input rows in shared memory (16-byte
+// loads), then every thread assembles 8 consecutive columns of a patch row and writes them with one
+// 16-byte store, consecutive threads to consecutive addresses.
+constexpr int IM2COL_MAX_W = 1024;  // widest input row the shared-memory staging holds (7 rows x 3 channels)
 template <int K, int ST>
-__device__ __forceinline__ void im2col_body(const SmallEntry &e, int bx, int nbx) {
+__device__ __forceinline__ void im2col_body(const SmallEntry &e, int bx) {
     constexpr int P = (K - 1) / 2, KK = K * K * 3;
+    __shared__ __align__(16) unsigned short rows[K][IM2COL_MAX_W * 3];
+    if (bx >= e.N * e.Ho) return;
+    const int n = bx / e.Ho, ho = bx % e.Ho;
+    const int rowlen = e.W * 3;  // elements; a multiple of 8 (checked by the host)
+    const unsigned short *ximg = static_cast<const unsigned short *>(e.x) + (size_t)n * e.H * rowlen;
+#pragma unroll
+    for (int r = 0; r < K; r++) {
+        const int hi = ho * ST + r - P;
+        if (hi < 0 || hi >= e.H) continue;  // never read below
+        const uint4 *src = reinterpret_cast<const uint4 *>(ximg + (size_t)hi * rowlen);
+        for (int i = threadIdx.x; i < rowlen / 8; i += blockDim.x) reinterpret_cast<uint4 *>(rows[r])[i] = __ldg(src + i);
+    }
+    __syncthreads();
     const int gv = e.KKp >> 3;
-    const int total = e.N * e.Ho * e.Wo * gv;
-    const unsigned short *x = static_cast<const unsigned short *>(e.x);
-    uint4 *y = static_cast<uint4 *>(e.y);
-    for (int i = bx * blockDim.x + threadIdx.x; i < total; i += nbx * blockDim.x) {
-        const int g = i % gv, m = i / gv;
-        const int wo = m % e.Wo, ho = (m / e.Wo) % e.Ho, n = m / (e.Wo * e.Ho);
-        const unsigned short *ximg = x + (size_t)n * e.H * e.W * 3;
+    uint4 *y = static_cast<uint4 *>(e.y) + ((size_t)n * e.Ho + ho) * e.Wo * gv;
+    for (int i = threadIdx.x; i < e.Wo * gv; i += blockDim.x) {
+        const int g = i % gv, wo = i / gv;
         unsigned short v[8];
 #pragma unroll
         for (int q = 0; q < 8; q++) {
             const int kk = g * 8 + q;
             const int c = kk % 3, rs = kk / 3, s = rs % K, r = rs / K;
             const int hi = ho * ST + r - P, wi = wo * ST + s - P;
-            v[q] = (kk < KK && hi >= 0 && hi < e.H && wi >= 0 && wi < e.W) ? __ldg(ximg + ((size_t)hi * e.W + wi) * 3 + c) : (unsigned short)0;
+            v[q] = (kk < KK && hi >= 0 && hi < e.H && wi >= 0 && wi < e.W) ? rows[r][wi * 3 + c] : (unsigned short)0;
         }
         y[i] = make_uint4(v[0] | ((uint32_t)v[1] << 16), v[2] | ((uint32_t)v[3] << 16), v[4] | ((uint32_t)v[5] << 16), v[6] | ((uint32_t)v[7] << 16));
     }
 }
 
 template <int KIND, int K, int ST> __device__ __forceinline__ void small_body(const SmallEntry &e, int bx, int nbx) {
-    if (KIND == OP_MAXPOOL) maxpool_body(e, bx, nbx);
-    else if (KIND == OP_GAP) gap_body(e, bx);
-    else if (KIND == OP_LINEAR) linear_body(e, bx);
-    else im2col_body<K, ST>(e, bx, nbx);
+    if constexpr (KIND == OP_MAXPOOL) maxpool_body(e, bx, nbx);
+    else if constexpr (KIND == OP_GAP) gap_body(e, bx);
+    else if constexpr (KIND == OP_LINEAR) linear_body(e, bx);
+    else im2col_body<K, ST>(e, bx);
 }
 template <int KIND, int K, int ST> __global__ void __launch_bounds__(256) small_single_kernel(const SmallEntry e) {
     small_body<KIND, K, ST>(e, blockIdx.x, gridDim.x);
@@ -638,7 +650,7 @@ bool small_supported(int kind, const SmallEntry &e) {
     case OP_GAP: return e.C % 8 == 0;
     case OP_LINEAR: return e.C % 8 == 0 && e.ld % 8 == 0 && al(e.w);
     case OP_IM2COL: return (e.k == 3 || e.k == 7) && (e.stride == 1 || e.stride == 2) && e.KKp % 8 == 0 && e.KKp >= e.k * e.k * 3 &&
-                           (long long)e.N * e.Ho * e.Wo * (e.KKp / 8) < (1ll << 31);
+                           e.W % 8 == 0 && e.W <= IM2COL_MAX_W && (long long)e.N * e.Ho < (1ll << 31) && (long long)e.Wo * (e.KKp / 8) < (1ll << 31);
     default: return false;
     }
 }
@@ -649,7 +661,7 @@ static long long small_blocks(int kind, const SmallEntry &e) {
     case OP_MAXPOOL: return ((long long)e.N * e.Ho * e.Wo * (e.C / 8) + 255) / 256;
     case OP_GAP: return ((long long)e.N * (e.C / 8) * 32 + 255) / 256;
     case OP_LINEAR: return ((long long)e.N * e.K * 32 + 255) / 256;
-    default: return ((long long)e.N * e.Ho * e.Wo * (e.KKp / 8) + 255) / 256;
+    default: return (long long)e.N * e.Ho;  // patch matrix: one block per output row
     }
 }
 
@@ -665,8 +677,8 @@ cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int
     if ((!d && n != 1) || n > 65535) return cudaErrorInvalidValue;
     long long blocks = 1;
     for (int i = 0; i < n; i++) blocks = std::max(blocks, small_blocks(kind, h[i]));
-    // grid-stride kernels (max pool, patch matrix) need not cover every element with a block of their own
-    if (kind == OP_MAXPOOL || kind == OP_IM2COL) blocks = std::min<long long>(blocks, 148 * 16);
+    // the grid-stride kernel (max pool) need not cover every element with a block of its own
+    if (kind == OP_MAXPOOL) blocks = std::min<long long>(blocks, 148 * 16);
     const unsigned bx = (unsigned)blocks;
     switch (kind) {
     case OP_MAXPOOL: return launch_small_t<OP_MAXPOOL, 0, 0>(h, d, n, bx, st);

@@ -198,7 +198,8 @@ __device__ __forceinline__ void finish_store(float *o, const __nv_bfloat16 *res,
 struct TcConvPlan {
     TcParams prm;
     dim3 grid;
-    int bn_tile = 128;
+    int bn_tile = 128;   // filters per tile
+    int swap = 0;        // grouped launches only: filters on the MMA's row side, all pixels on the column side
     size_t ws_elems = 0;
 };
 
