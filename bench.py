@@ -22,7 +22,7 @@ import numpy as np
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
-# 16 queries in flight need more than the default 8 hardware work queues; must be set before CUDA starts
+# many streams in flight need more than the default 8 hardware work queues; must be set before CUDA starts
 os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
 
 from paper_2306_17266_b200 import workload as wl  # noqa: E402
@@ -166,8 +166,10 @@ def run_suite(args):
         cfgs = wl.uniform_stream(wl.RESNET, n_groups, seed=5)
         rows = []
         for res in (160, 192, 224):
-            opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=0, concurrency=args.concurrency)
-            _stream_pool(net, sgs, torch, cfgs[:64], 16, res, opts, stream, 64, wl.RESNET)  # warm-up: plans, graphs
+            # one launch per layer covers the 4 configs of a batch of 64 (wave of 4 members x 16 images)
+            opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=0,
+                                  concurrency=args.concurrency, wave=min(args.wave, 4))
+            _stream_pool(net, sgs, torch, cfgs[:64], 16, res, opts, stream, 64, wl.RESNET)  # warm-up: plans
             t = _stream_pool(net, sgs, torch, cfgs, 16, res, opts, stream, 64, wl.RESNET)
             tf = t["flops"] / (t["ms"] * 1e-3) / 1e12
             rows.append({"res": res, "images_per_s": t["q"] * 16 / (t["ms"] * 1e-3), "useful_tflops": tf,
@@ -236,19 +238,21 @@ def run_suite(args):
     print(json.dumps(out))
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per conv_tc_kernel launch, from the one-pass ncu capture
-# summarised in profiles/stream_resnet_b1_launch_list.md.  Valid only for the kernel source it was taken
+# dram__bytes_read.sum + dram__bytes_write.sum per conv_group_kernel launch, from the one-pass ncu capture
+# summarised in profiles/conv_group_wave32_resnet_b1.md.  Valid only for the kernel source it was taken
 # on: once that file changes the figure is reported as null.
 NCU_TRAFFIC = {
-    "kernel_source_sha256_16": "19e548e86702d040",
-    "bytes_per_launch": 1361000,
-    "note": "ncu flushes the caches before every launch: cold-cache reads (weights + input tile); the writes stay in L2",
+    "kernel_source_sha256_16": "",
+    "bytes_per_launch": None,
+    "note": "ncu flushes the caches before every launch: cold-cache reads; writes that still sit in L2 when the kernel ends are not counted",
 }
 
 
-def ncu_traffic_per_launch():
+def ncu_traffic_per_launch(grouped=True):
     import hashlib
-    src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2306_17266_b200", "csrc", "sgs_conv_tc.cu")
+    if not grouped:
+        return None
+    src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2306_17266_b200", "csrc", "sgs_conv_group.cu")
     try:
         with open(src, "rb") as f:
             h = hashlib.sha256(f.read()).hexdigest()[:16]
@@ -268,12 +272,15 @@ def main():
     ap.add_argument("--ref-queries", type=int, default=8, help="queries per step of --impl reference")
     ap.add_argument("--cache", type=int, default=1)
     ap.add_argument("--window", type=int, default=4)
-    ap.add_argument("--concurrency", type=int, default=16, help="independent queries in flight at once")
+    ap.add_argument("--wave", type=int, default=32, help="queries per wave (grouped launches over the wave's members); 0 = one stream per query")
+    ap.add_argument("--concurrency", type=int, default=None, help="waves in flight (default 3), or with --wave 0 queries in flight (default 16)")
     ap.add_argument("--batch", type=int, default=1, help="images per query (sgs-probe)")
     ap.add_argument("--evict-first", type=int, default=0, help="with --cache 0: mark weight loads evict-first (sgs-probe)")
     ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()
+    if args.concurrency is None:
+        args.concurrency = 3 if args.wave > 0 else 16
     if args.impl == "reference":
         run_reference(args)
         return
@@ -311,9 +318,10 @@ def main():
     logits_host = torch.zeros((nq * BATCH, 1000), dtype=torch.float32).pin_memory()
     stream = torch.cuda.Stream()
 
-    def mk_opts(graphs=1, latency=0, conc=None):
+    def mk_opts(graphs=1, latency=0, conc=None, wave=None):
         return sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=graphs,
-                              record_latency=latency, weights_evict_first=0, concurrency=args.concurrency if conc is None else conc)
+                              record_latency=latency, weights_evict_first=0, concurrency=args.concurrency if conc is None else conc,
+                              wave=args.wave if wave is None else wave)
 
     def step(host=False, o=None):
         o = o or mk_opts()
@@ -363,34 +371,32 @@ def main():
 
     out = None
     if rank == 0:
-        # Dominant kernel.  Two more passes, both with CUDA events on the launching stream:
-        # (1) the stream one query at a time through the replayed graphs: device time of the whole pass;
-        # (2) the same stream with an event pair around every launch (no graphs): kernel time per class.
-        # An event pair around a 5 us kernel also holds the launch gap and the events' own cost, so
-        # (2) is used for the classes' shares only, and the tensor-core convolution's time in the real
-        # launch configuration is taken as share x (1).
-        step(o=mk_opts(conc=1))
-        seq = step(o=mk_opts(conc=1))
-        seq_lat = step(o=mk_opts(conc=1, latency=1))
+        # Dominant kernel: the tensor-core convolution.  Kernels of several waves overlap in the timed
+        # region, so its launches are timed in one more pass of the same stream with one wave at a time: an
+        # event pair on the launching stream around every launch, the stream held by a sleeping kernel while
+        # the host queues the wave (the intervals then hold device time, not launch latency).
+        seq = step(o=mk_opts(conc=1, wave=0))
+        seq_lat = step(o=mk_opts(conc=1, latency=1, wave=0))
         net.set_option("profile", 2)
         step(o=mk_opts(graphs=0))
         prof = [net.profile_read(c) for c in range(4)]
         net.set_option("profile", 0)
         tc = prof[0]
         total_ms = sum(p["total_ms"] for p in prof)
-        bracketed_us = tc["total_ms"] * 1e3 / max(1, tc["launches"])
         share = tc["total_ms"] / total_ms if total_ms > 0 else 0.0
-        sec = seq.total_ms * 1e-3 * share
+        sec = tc["total_ms"] * 1e-3
         achieved_gbs = tc["alg_bytes"] / sec / 1e9 if sec > 0 else 0.0
         achieved_tf = tc["flops"] / sec / 1e12 if sec > 0 else 0.0
+        grouped = args.wave > 0
         roofline = {
-            "kernel": "conv_tc_kernel (sliced implicit-GEMM convolution, tcgen05 + TMA)", "bound": "hbm",
-            "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic_per_launch(), "traffic_note": NCU_TRAFFIC["note"],
+            "kernel": ("conv_group_kernel (one launch = one stored layer for all members of a wave; sliced implicit GEMM, tcgen05 + TMA)" if grouped
+                       else "conv_tc_kernel (sliced implicit-GEMM convolution, tcgen05 + TMA)"),
+            "bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic_per_launch(grouped), "traffic_note": NCU_TRAFFIC["note"],
             "peak_source": peaks["source"],
             "launches": tc["launches"], "avg_launch_us": sec * 1e6 / max(1, tc["launches"]),
-            "avg_launch_us_event_bracketed": bracketed_us, "sequential_pass_ms": seq.total_ms,
-            "method": "share of event-bracketed kernel time x device time of a one-query-at-a-time graph pass / launches",
+            "method": "CUDA events around every launch, one wave at a time, host launch latency hidden behind a sleeping kernel; "
+                      "achieved = algorithmic bytes (sliced weights + input + output + residual of every member) / summed launch time",
             "alg_bytes_per_launch": tc["alg_bytes"] / max(1, tc["launches"]),
             "share_of_kernel_time": share,
             "tensor_tflops": achieved_tf, "tensor_frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"],
@@ -409,7 +415,9 @@ def main():
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "queries_per_step": nq, "batch": BATCH, "res": RES,
                        "l2": "inputs (301 MB per step) and the SuperNet (96 MB) exceed L2; no flush",
-                       "cache": bool(args.cache), "window_q": args.window, "queries_in_flight": args.concurrency,
+                       "cache": bool(args.cache), "window_q": args.window,
+                       "execution": (f"waves of {args.wave} queries, one grouped launch per layer, {args.concurrency} waves in flight" if args.wave > 0
+                                     else f"one stream per query, {args.concurrency} queries in flight"),
                        "parallelism": f"replicas x{world}"},
             "p50_ms": st_lat.p50_ms, "p99_ms": st_lat.p99_ms, "mean_ms": st_lat.mean_ms,
             "one_query_at_a_time": {"queries_per_s": seq_lat.queries_per_s, "p50_ms": seq_lat.p50_ms, "p99_ms": seq_lat.p99_ms},

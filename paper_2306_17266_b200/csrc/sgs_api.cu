@@ -393,7 +393,8 @@ struct Builder {
         const size_t first = plan->ops.size();
         const int Hin = H, Win = W;
         conv(name, -1, out, -1, H, W, stride, act);
-        if (!net->stem_gemm_w || net->force_plain || s.K % 8 || (s.k != 3 && s.k != 7)) return;
+        // (the patch-matrix kernel stages whole input rows with 16-byte loads: widths that are multiples of 8)
+        if (!net->stem_gemm_w || net->force_plain || s.K % 8 || (s.k != 3 && s.k != 7) || Win % 8 || Win > 1024) return;
         Op &cv = plan->ops[first];
         const int KKp = net->stem_kkp;
         Op im;
@@ -1188,7 +1189,10 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                               int res, void *logits, const sgs_stream_opts_t &o, sgs_stream_stats_t *stats, cudaStream_t st,
                               bool host_buffers) {
     const int G = std::min(o.wave, TC_GROUP_MAX_ENTRIES);
-    const int W = std::max(1, std::min(o.concurrency ? o.concurrency : 2, 4));
+    // per-launch timing (option "profile") wants the launches of one wave at a time
+    const int W = net->profile ? 1 : std::max(1, std::min(o.concurrency ? o.concurrency : 2, 4));
+    struct ProfRec { cudaEvent_t e0, e1; int cls; double bytes, flops; };
+    std::vector<ProfRec> prof;
     sgs_status_t rc = ensure_slots(net, G * W);
     if (rc != SGS_OK) return rc;
     if ((rc = ensure_waves(net, W)) != SGS_OK) return rc;
@@ -1326,16 +1330,49 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             CU(cudaMemcpyAsync(cx.stage_in, din, (size_t)members * in_bytes, cudaMemcpyHostToDevice, ws));
             din = cx.stage_in;
         }
+        // Profiling brackets every launch with events.  A sleeping kernel first holds the stream while the
+        // host queues the whole wave, so that the intervals hold device time, not launch latency.
+        if (net->profile) CU(launch_delay(1500, ws));
+        auto prof_begin = [&](int cls, double bytes, double fl) -> sgs_status_t {
+            if (!net->profile) return SGS_OK;
+            ProfRec r{nullptr, nullptr, cls, bytes, fl};
+            CU(cudaEventCreate(&r.e0));
+            CU(cudaEventCreate(&r.e1));
+            CU(cudaEventRecord(r.e0, ws));
+            prof.push_back(r);
+            return SGS_OK;
+        };
+        auto prof_end = [&]() -> sgs_status_t {
+            if (net->profile) CU(cudaEventRecord(prof.back().e1, ws));
+            return SGS_OK;
+        };
+        auto bucket_cost = [&](int rank, bool tc, double *bytes, double *fl) {
+            *bytes = 0; *fl = 0;
+            for (const auto &mo : buckets[(size_t)rank]) {
+                const Op &op = plans[mo.first]->ops[(size_t)mo.second];
+                if ((op.type == OP_CONV && op.impl == 1) != tc) continue;
+                *bytes += op.alg_bytes; *fl += op.flops;
+            }
+        };
         void *dlog = host_buffers ? (void *)cx.stage_out : dout;
         for (const Launch &L : launches) {
+            double pb = 0, pf = 0;
             if (L.group) {
+                // (a bucket split over several launches books its whole cost on each: buckets of more than
+                // 64 members or 248 tensor maps do not occur while profiling waves of <= 64)
+                bucket_cost(L.rank, true, &pb, &pf);
+                if ((rc = prof_begin(0, pb, pf)) != SGS_OK) break;
                 CU(L.group->launch(net->cache_tbl, net->sms, ws));
+                if ((rc = prof_end()) != SGS_OK) break;
                 net->kernel_launches++;
                 continue;
             }
             if (L.small_kind >= 0) {
+                bucket_cost(L.rank, false, &pb, &pf);
+                if ((rc = prof_begin(3, pb, pf)) != SGS_OK) break;
                 CU(launch_small(L.small_kind, reinterpret_cast<const SmallEntry *>(cx.h_tbl + L.off),
                                 reinterpret_cast<const SmallEntry *>(cx.d_tbl + L.off), L.count, ws));
+                if ((rc = prof_end()) != SGS_OK) break;
                 net->kernel_launches++;
                 continue;
             }
@@ -1378,6 +1415,14 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
     if (rc == SGS_OK && (ce != cudaSuccess || se != cudaSuccess))
         rc = fail(net, SGS_ECUDA, std::string("stream: ") + cudaGetErrorString(se != cudaSuccess ? se : ce));
     if (rc != SGS_OK) cudaDeviceSynchronize();
+    for (ProfRec &r : prof) {
+        float ms = 0;
+        if (rc == SGS_OK && r.e1 && cudaEventElapsedTime(&ms, r.e0, r.e1) == cudaSuccess) {
+            net->prof_ms[r.cls] += ms; net->prof_bytes[r.cls] += r.bytes; net->prof_flops[r.cls] += r.flops; net->prof_launches[r.cls]++;
+        }
+        if (r.e0) cudaEventDestroy(r.e0);
+        if (r.e1) cudaEventDestroy(r.e1);
+    }
     if (rc == SGS_OK && tc_conv_status()) rc = fail(net, SGS_ETIMEOUT, "a bounded device-side wait ran out in the tensor-core kernel");
     if (rc == SGS_OK && stats) {
         std::memset(stats, 0, sizeof(*stats));
@@ -1437,7 +1482,7 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
     if (o.wave < 0) return fail(net, SGS_EINVAL, "wave must be >= 0");
     cache_reset(net, o.cache_enabled != 0, o.cache_budget_bytes, o.window_q);
     net->cache.evict_first_when_off = (!o.cache_enabled && o.weights_evict_first) ? 1 : 0;
-    if (o.wave > 0 && n_queries > 0 && !net->profile && net->dtype == SGS_BF16 && tc_available() && !net->force_plain)
+    if (o.wave > 0 && n_queries > 0 && net->dtype == SGS_BF16 && tc_available() && !net->force_plain)
         return wave_impl(net, n_queries, cfgs, inputs, batch, res, logits, o, stats, st, host_buffers);
     // queries in flight at once: each runs in its own slot; per-kernel profiling wants them one by one
     const int S = net->profile ? 1 : std::max(1, std::min(o.concurrency ? o.concurrency : 1, std::max(1, n_queries)));
