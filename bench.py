@@ -279,6 +279,8 @@ def main():
     ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()
+    if args.suite in ("sgs", "sgs-probe", "mbv3"):
+        args.wave = 0  # these suites run one stream per query (depthwise / SE layers and the DRAM probe have no grouped launch)
     if args.concurrency is None:
         args.concurrency = 3 if args.wave > 0 else 16
     if args.impl == "reference":
