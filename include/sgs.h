@@ -98,7 +98,7 @@ typedef struct {
                            convolutions of all members whose SubNet has that layer are ONE grouped launch
                            (each member with its own slice of the shared weights), so a launch fills the
                            GPU although a single batch-1 SubNet cannot.  `concurrency` then counts waves
-                           in flight (0 = 2, at most 4) and use_graphs is ignored.  Every query of a wave
+                           in flight (0 = 2, at most 8) and use_graphs is ignored.  Every query of a wave
                            starts and ends with its wave (that is its recorded latency).  The cached
                            SubGraph is still re-chosen in stream order; the L2 hints of a wave use the
                            choice in force when the wave was issued. */

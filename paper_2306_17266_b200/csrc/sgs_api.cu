@@ -1190,7 +1190,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                               bool host_buffers) {
     const int G = std::min(o.wave, TC_GROUP_MAX_ENTRIES);
     // per-launch timing (option "profile") wants the launches of one wave at a time
-    const int W = net->profile ? 1 : std::max(1, std::min(o.concurrency ? o.concurrency : 2, 4));
+    const int W = net->profile ? 1 : std::max(1, std::min(o.concurrency ? o.concurrency : 2, 8));
     struct ProfRec { cudaEvent_t e0, e1; int cls; double bytes, flops; };
     std::vector<ProfRec> prof;
     sgs_status_t rc = ensure_slots(net, G * W);

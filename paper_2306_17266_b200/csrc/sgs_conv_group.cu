@@ -4,13 +4,14 @@
 // member (query): its tensor maps, slice extents, tile geometry and buffers.  All members' output tiles
 // form one list of tiles; persistent CTAs (one per SM) walk that list with a fixed stride.
 //
-// Per CTA: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = epilogue.  The shared-memory ring
-// of operand stages runs on across tiles, and the fp32 accumulator in tensor memory is double
-// buffered (2 x 128 columns), so the epilogue of tile j (tensor memory -> folded batch norm ->
-// residual -> activation -> bf16 NHWC) overlaps the loads and MMAs of tile j + 1.
+// Per CTA: warp 0 = weight producer, warp 10 = activation producer, warp 1 = MMA issuer, warps 2..9 =
+// two epilogue groups.  The shared-memory ring of operand stages runs on across tiles, and the fp32
+// accumulator in tensor memory is double buffered (2 x 256 columns, one buffer per epilogue group), so the
+// epilogues of tiles j and j + 1 (tensor memory -> folded batch norm -> residual -> activation -> bf16
+// NHWC) overlap each other and the loads and MMAs of the tiles that follow.
 //
 // The arithmetic of one tile is that of conv_tc_kernel (sgs_conv_tc.cu): implicit GEMM with
-// 128 output pixels x up to 128 filters, 64 channels per stage, slicing through the tensor maps'
+// 128 output pixels x up to 256 filters, 64 channels per stage, slicing through the tensor maps'
 // extents.  The reduction is never split here: with many members in flight the tiles alone fill the GPU.
 #include "sgs_tc.cuh"
 
@@ -30,7 +31,7 @@ constexpr int G_X_BYTES = 128 * CHUNK_C * 2;  // operand on the MMA's row side: 
 constexpr int G_RING_BYTES = 192 * 1024;      // operand ring: 6 stages of 16 + 16 KB, or 4 stages of 16 + 32 KB (256-column tiles)
 constexpr int G_SMEM_BYTES = G_RING_BYTES + 1024;
 constexpr int G_ACC_COLS = 256;                   // tensor-memory columns of one accumulator buffer
-constexpr int G_EPI_WARPS = 8;                    // two per tensor-memory lane quadrant: each takes part of the columns
+constexpr int G_EPI_WARPS = 8;                    // two groups of four (one warp per tensor-memory lane quadrant)
 constexpr int G_THREADS = 64 + 32 * G_EPI_WARPS + 32;  // weight producer, MMA warp, epilogue warps, pixel producer
 constexpr int G_PIX_WARP = 2 + G_EPI_WARPS;
 
@@ -73,11 +74,9 @@ __device__ __forceinline__ int find_entry_serial(const GroupEntry *es, int n, in
     return lo;
 }
 
-__device__ __forceinline__ void epilogue_bar() { asm volatile("bar.sync 1, %0;" ::"n"(32 * G_EPI_WARPS) : "memory"); }
+// Named barrier of one epilogue group (4 warps): id 1 or 2.
+__device__ __forceinline__ void group_bar(int grp) { asm volatile("bar.sync %0, 128;" ::"r"(grp + 1) : "memory"); }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *m) { asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory"); }
-
-// Where the epilogue splits a tile's columns between the two warps of a lane quadrant (a multiple of 32).
-__device__ __forceinline__ int split_cols(int ncols) { return ((ncols + 63) >> 6) << 5; }
 
 #ifdef SGS_ROLE_TIMING
 // Development aid (not compiled into the library): cycles each warp role spends waiting, summed over CTAs and launches.
@@ -111,7 +110,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
     int *status = P.status;
     extern __shared__ uint8_t smem_raw[];
     __shared__ GroupEntry es[TC_GROUP_MAX_ENTRIES];
-    __shared__ float scale_s[2][G_ACC_COLS], shift_s[2][G_ACC_COLS];  // folded batch norm of the current / next tile's filters (normal tiles)
+    __shared__ float scale_s[2][2][G_ACC_COLS], shift_s[2][2][G_ACC_COLS];  // per epilogue group: folded batch norm of its current / next tile's filters
     __shared__ __align__(8) uint64_t full_bar[G_MAX_STAGES], empty_bar[G_MAX_STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
@@ -127,7 +126,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
     if (threadIdx.x == 0) {
         // a stage is full once both producers' copies have landed; it is empty once its MMAs have read it
         for (int s = 0; s < G_MAX_STAGES; s++) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], G_EPI_WARPS); }
+        for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], G_EPI_WARPS / 2); }
         abort_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -273,40 +272,49 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         ROLE_FLUSH(5, tfull_); ROLE_FLUSH(6, tacc_); ROLE_FLUSH(7, clock64() - tk0_);
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9)
-        // Two warps share a tensor-memory lane quadrant; each takes part of the tile's columns.
+        // Two groups of four warps (one per tensor-memory lane quadrant).  Group g owns accumulator buffer g
+        // and takes the CTA's tiles j with j % 2 == g, so the epilogues of two consecutive tiles run side by
+        // side; a thread handles one accumulator row and all of the tile's columns, 32 at a time.
         const int quad = warp & 3;                // tensor-memory lane quadrant this warp may read
-        const int half = (warp - 2) >> 2;         // which part of the columns
+        const int grp = (warp - 2) >> 2;          // epilogue group = accumulator buffer
         const int row = quad * 32 + lane;         // accumulator row: output pixel (normal) or filter (swapped)
-        const int et = threadIdx.x - 64;          // 0..255
+        const int et = (threadIdx.x - 64) & 127;  // thread within the group
+        float(*scale_g)[G_ACC_COLS] = scale_s[grp];
+        float(*shift_g)[G_ACC_COLS] = shift_s[grp];
+        const int stride2 = 2 * (int)gridDim.x;
         long long tpdl_ = 0, tbar_ = 0, tacc_ = 0, twork_ = 0; (void)tpdl_; (void)tbar_; (void)tacc_; (void)twork_;
         const long long tk0_ = clock64(); (void)tk0_;
         { ROLE_T0(); pdl_wait(); ROLE_ADD(tpdl_); }  // residual reads and output writes must not pass the previous layers
         bool alive = true;  // after a failed wait the warp only keeps the named barrier in step
-        // folded batch norm of a normal tile: thread et fetches filter et's scale and shift
-        auto fetch_bn = [&](int tile, float *sc, float *sh) {
-            *sc = 0.f; *sh = 0.f;
+        // folded batch norm of a normal tile: thread et fetches the scale and shift of filters et and et + 128
+        auto fetch_bn = [&](int tile, float *v) {
+            v[0] = v[1] = v[2] = v[3] = 0.f;
             if (tile >= total_tiles) return;
             const GroupEntry &e = es[find_entry(es, n_entries, tile, lane)];
             if (e.swap) return;
             const int f = ((tile - e.tile_begin) / e.mtiles) * e.bn_tile + et;
-            if (et < e.bn_tile && f < e.K) { *sc = __ldg(e.scale + f); *sh = __ldg(e.shift + f); }
+            if (et < e.bn_tile && f < e.K) { v[0] = __ldg(e.scale + f); v[1] = __ldg(e.shift + f); }
+            if (et + 128 < e.bn_tile && f + 128 < e.K) { v[2] = __ldg(e.scale + f + 128); v[3] = __ldg(e.shift + f + 128); }
+        };
+        auto store_bn = [&](int b, const float *v) {
+            scale_g[b][et] = v[0]; shift_g[b][et] = v[1]; scale_g[b][et + 128] = v[2]; shift_g[b][et + 128] = v[3];
         };
         {
-            float sc, sh;
-            fetch_bn(blockIdx.x, &sc, &sh);
-            scale_s[0][et] = sc; shift_s[0][et] = sh;
+            float v[4];
+            fetch_bn((int)blockIdx.x + grp * (int)gridDim.x, v);
+            store_bn(0, v);
         }
-        int j = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, j++) {
+        int jj = 0;  // tiles this group has taken
+        for (int t = (int)blockIdx.x + grp * (int)gridDim.x; t < total_tiles; t += stride2, jj++) {
             const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
             const int local = t - e.tile_begin, nt = local / e.mtiles, mt = local % e.mtiles;
             const int K = e.K, act = e.act;
             const __nv_bfloat16 *res = e.res;
             __nv_bfloat16 *y = e.y;
-            const int buf = j & 1;
-            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * G_ACC_COLS);
-            float nsc, nsh;
-            fetch_bn(t + (int)gridDim.x, &nsc, &nsh);  // requested now, stored after this tile's work
+            const int sb = jj & 1;  // which of the group's two scale / shift tables
+            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(grp * G_ACC_COLS);
+            float nbn[4];
+            fetch_bn(t + stride2, nbn);  // requested now, stored after this tile's work
             if (!e.swap) {
                 // ---- normal tile: this thread owns output pixel `m`, columns are filters
                 const int n0 = (mt / e.tiles_hw) * e.bn, h0 = ((mt % e.tiles_hw) / e.tiles_w) * e.bh, w0 = (mt % e.tiles_w) * e.bw;
@@ -318,9 +326,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                     const bool valid = row < e.pix_rows && n < e.N && h < e.Ho && w < e.Wo;
                     m = valid ? (int)(((size_t)n * e.Ho + h) * e.Wo + w) : -1;
                 }
-                const int ncols = min((int)e.bn_tile, K - f0);  // filters of this tile, a multiple of 8
-                const int split = split_cols(ncols);
-                const int cbeg = half ? split : 0, cend = half ? ncols : min(ncols, split);
+                const int cend = min((int)e.bn_tile, K - f0);  // filters of this tile, a multiple of 8
                 const size_t obase = (size_t)(m < 0 ? 0 : m) * K + f0;
                 // the residual does not depend on the accumulator: the first 32 columns' part is requested
                 // before waiting, every further part one step ahead of its use
@@ -332,15 +338,15 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                     }
                 };
                 uint4 rv[4];
-                load_res(cbeg, rv);
-                { ROLE_T0(); epilogue_bar(); ROLE_ADD(tbar_); }  // this tile's scale / shift (written during the previous tile) are visible
-                const float *sc = scale_s[buf], *sh = shift_s[buf];
-                { ROLE_T0(); if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (j >> 1) & 1, abort_flag)); ROLE_ADD(tacc_); }
+                load_res(0, rv);
+                { ROLE_T0(); group_bar(grp); ROLE_ADD(tbar_); }  // this tile's scale / shift (written during the group's previous tile) are visible
+                const float *sc = scale_g[sb], *sh = shift_g[sb];
+                { ROLE_T0(); if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&acc_full[grp], jj & 1, abort_flag)); ROLE_ADD(tacc_); }
                 ROLE_T0();
                 if (alive) {
                     tc_fence_after();
 #pragma unroll 1
-                    for (int c0 = cbeg; c0 < cend; c0 += 32) {  // warp-uniform bounds
+                    for (int c0 = 0; c0 < cend; c0 += 32) {  // warp-uniform bounds
                         uint32_t v[32];
                         tmem_ld32(tacc + c0, v);
                         uint4 rn[4];
@@ -370,9 +376,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                 // ---- swapped tile: this thread owns filter `f`, columns are the member's output pixels
                 const int f = nt * 128 + row;
                 const bool fvalid = f < K;
-                const int npix = e.pix_rows;  // == N * Ho * Wo: the pixel tile is the whole member
-                const int split = split_cols(npix);
-                const int cbeg = half ? split : 0, cend = half ? npix : min(npix, split);
+                const int cend = e.pix_rows;  // == N * Ho * Wo: the pixel tile is the whole member
                 float sc = 0.f, sh = 0.f;
                 if (fvalid) { sc = __ldg(e.scale + f); sh = __ldg(e.shift + f); }
                 const unsigned short *resu = reinterpret_cast<const unsigned short *>(res);
@@ -387,13 +391,13 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                     }
                 };
                 uint32_t rv[16];
-                load_res(cbeg, rv);
-                epilogue_bar();
-                if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (j >> 1) & 1, abort_flag));
+                load_res(0, rv);
+                group_bar(grp);
+                if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&acc_full[grp], jj & 1, abort_flag));
                 if (alive) {
                     tc_fence_after();
 #pragma unroll 1
-                    for (int c0 = cbeg; c0 < cend; c0 += 32) {
+                    for (int c0 = 0; c0 < cend; c0 += 32) {
                         uint32_t v[32];
                         tmem_ld32(tacc + c0, v);
                         uint32_t rn[16];
@@ -419,11 +423,11 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                 // hand the accumulator buffer back to the MMA warp
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                if (lane == 0) mbar_arrive(&acc_empty[grp]);
             }
-            // all epilogue threads read buffer buf ^ 1 for the last time during tile j - 1, which they have
-            // all left (barrier above)
-            scale_s[buf ^ 1][et] = nsc; shift_s[buf ^ 1][et] = nsh;
+            // the group read table sb ^ 1 for the last time during its previous tile, which all of its
+            // threads have left (barrier above)
+            store_bn(sb ^ 1, nbn);
         }
         if (warp == 2) { ROLE_FLUSH(8, tpdl_); ROLE_FLUSH(9, tbar_); ROLE_FLUSH(10, tacc_); ROLE_FLUSH(11, twork_); ROLE_FLUSH(12, clock64() - tk0_); }
     }
