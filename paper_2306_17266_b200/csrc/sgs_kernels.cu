@@ -741,32 +741,47 @@ constexpr int IM2COL_MAX_W = 1024;  // widest input row the shared-memory stagin
 template <int K, int ST>
 __device__ __forceinline__ void im2col_body(const SmallEntry &e, int bx) {
     constexpr int P = (K - 1) / 2, KK = K * K * 3;
-    __shared__ __align__(16) unsigned short rows[K][IM2COL_MAX_W * 3];
+    constexpr int ROWLEN = (IM2COL_MAX_W + 2 * P) * 3;  // a staged row with P zero pixels on either side
+    // rows[r] = input row ho*ST + r - P, shifted right by P pixels and zero outside the image, so that the
+    // patch element (r, s, c) of output column wo is rows[r][(wo*ST + s) * 3 + c] without any bounds test
+    __shared__ __align__(16) unsigned short rows[K][ROWLEN];
     if (bx >= e.N * e.Ho) return;
     const int n = bx / e.Ho, ho = bx % e.Ho;
     const int rowlen = e.W * 3;  // elements; a multiple of 8 (checked by the host)
     const unsigned short *ximg = static_cast<const unsigned short *>(e.x) + (size_t)n * e.H * rowlen;
+    const int padded = rowlen + 2 * P * 3;
 #pragma unroll
     for (int r = 0; r < K; r++) {
         const int hi = ho * ST + r - P;
-        if (hi < 0 || hi >= e.H) continue;  // never read below
-        const uint4 *src = reinterpret_cast<const uint4 *>(ximg + (size_t)hi * rowlen);
-        for (int i = threadIdx.x; i < rowlen / 8; i += blockDim.x) reinterpret_cast<uint4 *>(rows[r])[i] = __ldg(src + i);
+        const bool rok = hi >= 0 && hi < e.H;
+        const unsigned short *src = ximg + (size_t)(rok ? hi : 0) * rowlen;
+        for (int i = threadIdx.x; i < padded; i += blockDim.x) {
+            const int j = i - P * 3;
+            rows[r][i] = (rok && j >= 0 && j < rowlen) ? __ldg(src + j) : (unsigned short)0;
+        }
     }
     __syncthreads();
+    // a thread keeps one group of 8 patch columns (their 8 offsets into `rows` stay in registers) and walks
+    // the output columns; neighbouring threads write neighbouring 16-byte pieces
     const int gv = e.KKp >> 3;
+    const int lanes_w = blockDim.x / gv;  // output columns in flight per block
+    const int g = threadIdx.x % gv, wl = threadIdx.x / gv;
+    if (wl >= lanes_w) return;
+    int off[8];
+#pragma unroll
+    for (int q = 0; q < 8; q++) {
+        const int kk = g * 8 + q;
+        const int c = kk % 3, rs = kk / 3, s = rs % K, r = rs / K;
+        off[q] = kk < KK ? r * ROWLEN + s * 3 + c : -1;  // -1: padding column, always zero
+    }
     uint4 *y = static_cast<uint4 *>(e.y) + ((size_t)n * e.Ho + ho) * e.Wo * gv;
-    for (int i = threadIdx.x; i < e.Wo * gv; i += blockDim.x) {
-        const int g = i % gv, wo = i / gv;
+    const unsigned short *base = &rows[0][0];
+    for (int wo = wl; wo < e.Wo; wo += lanes_w) {
+        const unsigned short *p = base + wo * ST * 3;
         unsigned short v[8];
 #pragma unroll
-        for (int q = 0; q < 8; q++) {
-            const int kk = g * 8 + q;
-            const int c = kk % 3, rs = kk / 3, s = rs % K, r = rs / K;
-            const int hi = ho * ST + r - P, wi = wo * ST + s - P;
-            v[q] = (kk < KK && hi >= 0 && hi < e.H && wi >= 0 && wi < e.W) ? rows[r][wi * 3 + c] : (unsigned short)0;
-        }
-        y[i] = make_uint4(v[0] | ((uint32_t)v[1] << 16), v[2] | ((uint32_t)v[3] << 16), v[4] | ((uint32_t)v[5] << 16), v[6] | ((uint32_t)v[7] << 16));
+        for (int q = 0; q < 8; q++) v[q] = off[q] >= 0 ? p[off[q]] : (unsigned short)0;
+        y[wo * gv + g] = make_uint4(v[0] | ((uint32_t)v[1] << 16), v[2] | ((uint32_t)v[3] << 16), v[4] | ((uint32_t)v[5] << 16), v[6] | ((uint32_t)v[7] << 16));
     }
 }
 
