@@ -273,7 +273,7 @@ def main():
     ap.add_argument("--cache", type=int, default=1)
     ap.add_argument("--window", type=int, default=4)
     ap.add_argument("--wave", type=int, default=32, help="queries per wave (grouped launches over the wave's members); 0 = one stream per query")
-    ap.add_argument("--concurrency", type=int, default=None, help="waves in flight (default 3), or with --wave 0 queries in flight (default 16)")
+    ap.add_argument("--concurrency", type=int, default=None, help="waves in flight (default 4), or with --wave 0 queries in flight (default 16)")
     ap.add_argument("--batch", type=int, default=1, help="images per query (sgs-probe)")
     ap.add_argument("--evict-first", type=int, default=0, help="with --cache 0: mark weight loads evict-first (sgs-probe)")
     ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3"],
@@ -282,7 +282,7 @@ def main():
     if args.suite in ("sgs", "sgs-probe", "mbv3"):
         args.wave = 0  # these suites run one stream per query (depthwise / SE layers and the DRAM probe have no grouped launch)
     if args.concurrency is None:
-        args.concurrency = 3 if args.wave > 0 else 16
+        args.concurrency = 4 if args.wave > 0 else 16
     if args.impl == "reference":
         run_reference(args)
         return

@@ -801,6 +801,51 @@ template <int KIND, int K, int ST> __global__ void __launch_bounds__(256) small_
     small_body<KIND, K, ST>(e, blockIdx.x, gridDim.x);
 }
 
+// Linear layer for several members that use the SAME stored layer (same weights, outputs, batch): a warp
+// owns one (image, output) pair for up to LIN_CHUNK members, loads every 16-byte piece of the weight row
+// once and uses it for each member whose (sliced) input is that long.  Per member the arithmetic and its
+// order are those of linear_body.
+constexpr int LIN_CHUNK = 8;
+__global__ void __launch_bounds__(256) linear_multi_kernel(const SmallEntry *__restrict__ tbl, int n_members) {
+    __shared__ SmallEntry es[LIN_CHUNK];
+    const int m0 = blockIdx.y * LIN_CHUNK, nm = min(LIN_CHUNK, n_members - m0);
+    if ((int)threadIdx.x < nm * 8) reinterpret_cast<uint4 *>(es)[threadIdx.x] = __ldg(reinterpret_cast<const uint4 *>(tbl + m0) + threadIdx.x);
+    __syncthreads();
+    const SmallEntry &e0 = es[0];
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= e0.N * e0.K) return;
+    const int n = warp / e0.K, j = warp % e0.K;
+    const __nv_bfloat16 *wr = static_cast<const __nv_bfloat16 *>(e0.w) + (size_t)j * e0.ld;
+    int Cmax = 0;
+    for (int m = 0; m < nm; m++) Cmax = max(Cmax, es[m].C);
+    float s[LIN_CHUNK];
+#pragma unroll
+    for (int m = 0; m < LIN_CHUNK; m++) s[m] = 0.f;
+    for (int c = lane * 8; c < Cmax; c += 256) {
+        const uint4 wv = __ldg(reinterpret_cast<const uint4 *>(wr + c));
+        const float2 a = bf2f(wv.x), b = bf2f(wv.y), cc = bf2f(wv.z), d = bf2f(wv.w);
+#pragma unroll
+        for (int m = 0; m < LIN_CHUNK; m++) {
+            if (m < nm && c < es[m].C) {
+                const float *vr = static_cast<const float *>(es[m].x) + (size_t)n * es[m].C + c;
+                const float4 x0 = *reinterpret_cast<const float4 *>(vr), x1 = *reinterpret_cast<const float4 *>(vr + 4);
+                float t = s[m];
+                t = fmaf(a.x, x0.x, t); t = fmaf(a.y, x0.y, t); t = fmaf(b.x, x0.z, t); t = fmaf(b.y, x0.w, t);
+                t = fmaf(cc.x, x1.x, t); t = fmaf(cc.y, x1.y, t); t = fmaf(d.x, x1.z, t); t = fmaf(d.y, x1.w, t);
+                s[m] = t;
+            }
+        }
+    }
+    const float bias = e0.bias[j];
+#pragma unroll
+    for (int m = 0; m < LIN_CHUNK; m++) {
+        float t = s[m];
+#pragma unroll
+        for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (lane == 0 && m < nm) static_cast<float *>(es[m].y)[(size_t)n * e0.K + j] = apply_act(t + bias, e0.act);
+    }
+}
+
 bool small_supported(int kind, const SmallEntry &e) {
     auto al = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
     if (!al(e.x) || !al(e.y)) return false;
@@ -842,7 +887,16 @@ cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int
     switch (kind) {
     case OP_MAXPOOL: return launch_small_t<OP_MAXPOOL, 0, 0>(h, d, n, bx, st);
     case OP_GAP: return launch_small_t<OP_GAP, 0, 0>(h, d, n, bx, st);
-    case OP_LINEAR: return launch_small_t<OP_LINEAR, 0, 0>(h, d, n, bx, st);
+    case OP_LINEAR: {
+        bool same = d != nullptr && n > 1;
+        for (int i = 1; i < n && same; i++)
+            same = h[i].w == h[0].w && h[i].K == h[0].K && h[i].ld == h[0].ld && h[i].N == h[0].N && h[i].act == h[0].act && h[i].bias == h[0].bias;
+        if (same) {  // one stored layer for all members: share its weight rows
+            linear_multi_kernel<<<dim3(bx, (unsigned)((n + LIN_CHUNK - 1) / LIN_CHUNK)), 256, 0, st>>>(d, n);
+            return cudaGetLastError();
+        }
+        return launch_small_t<OP_LINEAR, 0, 0>(h, d, n, bx, st);
+    }
     case OP_IM2COL: {
         const int key = h[0].k * 10 + h[0].stride;
         for (int i = 1; i < n; i++)
