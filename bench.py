@@ -221,11 +221,11 @@ def run_suite(args):
         net = sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16)
         cfgs = wl.uniform_stream(wl.MBV3, args.queries, seed=3)
         opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=1,
-                              concurrency=args.concurrency)
+                              concurrency=args.concurrency, wave=args.wave)
         _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
         t = _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
         net.set_option("profile", 2)
-        popts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=0, record_latency=0)
+        popts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=0, record_latency=0, wave=args.wave)
         _stream_pool(net, sgs, torch, cfgs, 1, 224, popts, stream, len(cfgs), wl.MBV3)
         prof = [net.profile_read(c) for c in range(4)]
         net.set_option("profile", 0)
@@ -234,7 +234,8 @@ def run_suite(args):
                     "kernel_time_ms_by_class": {"conv_tc": prof[0]["total_ms"], "conv_cuda_core": prof[1]["total_ms"],
                                                 "depthwise": prof[2]["total_ms"], "other": prof[3]["total_ms"]},
                     "depthwise_gbs_at_batch1": prof[2]["alg_bytes"] / (prof[2]["total_ms"] * 1e-3) / 1e9 if prof[2]["total_ms"] else None,
-                    "config": {"workload": "MobileNetV3-shaped SuperNet, 1000-query stream at batch 1, 224x224, configs uniform (seed 3)"}})
+                    "config": {"workload": "MobileNetV3-shaped SuperNet, 1000-query stream at batch 1, 224x224, configs uniform (seed 3)",
+                               "execution": f"waves of {args.wave}, {args.concurrency} in flight" if args.wave > 0 else f"one stream per query, {args.concurrency} in flight"}})
     print(json.dumps(out))
 
 
@@ -279,8 +280,8 @@ def main():
     ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()
-    if args.suite in ("sgs", "sgs-probe", "mbv3"):
-        args.wave = 0  # these suites run one stream per query (depthwise / SE layers and the DRAM probe have no grouped launch)
+    if args.suite in ("sgs", "sgs-probe"):
+        args.wave = 0  # these suites run one stream per query (cache on / off comparisons and the DRAM probe)
     if args.concurrency is None:
         args.concurrency = 4 if args.wave > 0 else 16
     if args.impl == "reference":

@@ -684,6 +684,17 @@ SmallEntry small_entry(const sgs_supernet *net, const Plan *plan, const Op &op, 
         e.N = op.N; e.C = op.C; e.K = op.K; e.ld = L.C; e.act = op.act;
         break;
     }
+    case OP_SCALE:
+        e.x = sl.act[op.in]; e.y = sl.act[op.out]; e.w = sl.vec[op.vin];
+        e.N = op.N; e.H = op.H; e.W = op.W; e.C = op.C;
+        break;
+    case OP_SE_GATE: {
+        const StoredLayer &L1 = net->layers[op.layer], &L2 = net->layers[op.layer2];
+        e.x = sl.vec[op.vin]; e.y = sl.vec[op.vout];
+        e.w = L1.w; e.bias = L1.shift; e.ld = L1.C; e.w2 = L2.w; e.bias2 = L2.shift; e.ld2 = L2.C;
+        e.N = op.N; e.C = op.C; e.K = op.K;
+        break;
+    }
     case OP_IM2COL:
         e.x = d_input; e.y = sl.act[op.out];
         e.N = op.N; e.H = op.H; e.W = op.W; e.C = 3;
@@ -1265,7 +1276,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             }
         size_t n_small = 0;
         for (int m = 0; m < members; m++) n_small += plans[m]->ops.size();
-        const size_t need_tbl = (n_tc + n_small) * TC_GROUP_ENTRY_BYTES + 256;
+        const size_t need_tbl = (n_tc + 2 * n_small) * TC_GROUP_ENTRY_BYTES + 256;  // (depthwise records take two slots)
         if (cx.tbl_bytes < need_tbl) {
             cudaFreeHost(cx.h_tbl); cx.h_tbl = nullptr;
             dev_free(net, cx.d_tbl, cx.tbl_bytes); cx.d_tbl = nullptr; cx.tbl_bytes = 0;
@@ -1303,7 +1314,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             // member's op has the vectorised form; the remaining ops run member by member
             const Op &op0 = plans[b[0].first]->ops[(size_t)b[0].second];
             const int kind = op0.type;
-            bool grouped = kind == OP_MAXPOOL || kind == OP_GAP || kind == OP_LINEAR || kind == OP_IM2COL;
+            bool grouped = kind == OP_MAXPOOL || kind == OP_GAP || kind == OP_LINEAR || kind == OP_IM2COL || kind == OP_SCALE || kind == OP_SE_GATE;
             if (grouped) {
                 const size_t off0 = off;
                 for (const auto &mo : b) {
@@ -1315,6 +1326,39 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                     off += sizeof se;
                 }
                 if (grouped) { launches.push_back({r, nullptr, kind, off0, (int)b.size()}); continue; }
+                off = off0;
+            }
+            if (kind == OP_DW) {
+                // depthwise: members with the same kernel size share a launch (stride, activation and image
+                // size are the layer's); a member the vectorised kernels do not take sends the bucket back
+                // to member-by-member launches
+                const size_t off0 = off;
+                const size_t l0 = launches.size();
+                bool ok = true;
+                for (int kk : {3, 5, 7}) {
+                    const size_t offk = off;
+                    int cnt = 0;
+                    for (const auto &mo : b) {
+                        const Op &op = plans[mo.first]->ops[(size_t)mo.second];
+                        if (op.conv.k != kk) continue;
+                        ConvArgs a = op.conv;
+                        a.layer = op.layer;
+                        std::memcpy(cx.h_tbl + off, &a, sizeof a);
+                        off += DW_ENTRY_BYTES;
+                        cnt++;
+                    }
+                    if (cnt) launches.push_back({r, nullptr, OP_DW, offk, cnt});
+                }
+                size_t total = 0;
+                for (size_t i = l0; i < launches.size(); i++) total += (size_t)launches[i].count;
+                ok = total == b.size() && net->dtype == SGS_BF16;
+                for (size_t i = l0; i < launches.size() && ok; i++) {
+                    // dry check with the launcher's own rules (it launches nothing when it refuses)
+                    const ConvArgs &a0 = *reinterpret_cast<const ConvArgs *>(cx.h_tbl + launches[i].off);
+                    ok = a0.K % 8 == 0 && (long long)a0.N * launches[i].count <= 65535;
+                }
+                if (ok) continue;
+                launches.resize(l0);
                 off = off0;
             }
             launches.push_back({r, nullptr, -1, 0, 0});  // the bucket's remaining ops, member by member
@@ -1365,6 +1409,24 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                 CU(L.group->launch(net->cache_tbl, net->sms, ws));
                 if ((rc = prof_end()) != SGS_OK) break;
                 net->kernel_launches++;
+                continue;
+            }
+            if (L.small_kind == OP_DW) {
+                bucket_cost(L.rank, false, &pb, &pf);
+                if ((rc = prof_begin(2, pb, pf)) != SGS_OK) break;
+                cudaError_t de = launch_dw_group(cx.h_tbl + L.off, cx.d_tbl + L.off, L.count, ws);
+                if (de == cudaErrorNotSupported) {
+                    // (not expected after the checks above) run these members one by one
+                    for (int i = 0; i < L.count && rc == SGS_OK; i++) {
+                        const ConvArgs &a = *reinterpret_cast<const ConvArgs *>(cx.h_tbl + L.off + (size_t)i * DW_ENTRY_BYTES);
+                        CU(launch_dw<__nv_bfloat16>(a, ws));
+                        net->kernel_launches++;
+                    }
+                } else {
+                    CU(de);
+                    net->kernel_launches++;
+                }
+                if ((rc = prof_end()) != SGS_OK) break;
                 continue;
             }
             if (L.small_kind >= 0) {

@@ -125,14 +125,23 @@ struct alignas(16) SmallEntry {
     int K, ld, act;      // linear: outputs, row pitch of w, activation
     int Ho, Wo;          // output dims (max pool, patch matrix)
     int k, stride, KKp;  // patch matrix: kernel size, stride, padded row length
-    int pad_[12];
+    const void *w2;      // SE gate: second FC weights [C][ld2] bf16 (first FC: w [K][ld], K = squeeze width)
+    const float *bias2;  // SE gate: second FC bias [C]
+    int ld2;
+    int pad_[7];
 };
 static_assert(sizeof(SmallEntry) == 128, "record size");
 // kind: OP_MAXPOOL (3x3 stride 2, C % 8 == 0), OP_GAP (C % 8 == 0), OP_LINEAR (C % 8 == 0, ld % 8 == 0),
+// OP_SCALE (SE scale, gate vector in w; C % 8 == 0), OP_SE_GATE (grouped launches only),
 // OP_IM2COL (3 input channels; k in {3, 7}; stride in {1, 2}).  `h` is the host image of the `n` records
 // at device address `d` (it sizes the grid); with d == nullptr, n must be 1 and the record is passed by value.
 bool small_supported(int kind, const SmallEntry &e);
 cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int n, cudaStream_t st);
+// Depthwise convolution of several members in one launch: h_tbl / d_tbl = host image and device copy of
+// `members` ConvArgs records, DW_ENTRY_BYTES apart.  All members must share kernel size, stride, activation and
+// image dims and take the vectorised bf16 kernels; otherwise cudaErrorNotSupported and nothing is launched.
+constexpr int DW_ENTRY_BYTES = 256;
+cudaError_t launch_dw_group(const char *h_tbl, const char *d_tbl, int members, cudaStream_t st);
 // Stem weights as a GEMM operand: dst[f][kk] = src[f][kk] for kk < KK (the stored [K][R][R][3] row), 0 up to KKp.
 cudaError_t launch_stem_gemm_weights(const void *src, void *dst, int K, int KK, int KKp, cudaStream_t st);
 

@@ -173,8 +173,22 @@ __global__ void __launch_bounds__(256) dw_plain_kernel(ConvArgs a) {
 // HBM traffic per output element: 2 B read + 2 B written (rows are re-read from L1/L2, not DRAM).
 __device__ __forceinline__ float2 bf2_lo(uint32_t u) { return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u)); }
 
-template <int K, int ST>
-__global__ void __launch_bounds__(256) dw_vec_kernel(ConvArgs a) {
+// Argument record of a depthwise kernel: by value, or (GROUP: one launch for many queries in flight) from a
+// device table with DW_ENTRY_BYTES per member, blockIdx.z = member * images + image.
+#define SGS_DW_ARGS()                                                                                          \
+    __shared__ __align__(16) unsigned char a_raw_[sizeof(ConvArgs)];                                           \
+    if (GROUP) {                                                                                               \
+        const uint32_t *src_ = reinterpret_cast<const uint32_t *>(tbl + (size_t)(blockIdx.z / n_img) * DW_ENTRY_BYTES); \
+        for (int i_ = threadIdx.x; i_ < (int)(sizeof(ConvArgs) / 4); i_ += blockDim.x) reinterpret_cast<uint32_t *>(a_raw_)[i_] = __ldg(src_ + i_); \
+        __syncthreads();                                                                                       \
+    }                                                                                                          \
+    const ConvArgs &a = GROUP ? *reinterpret_cast<const ConvArgs *>(a_raw_) : a1;                              \
+    const int n = GROUP ? (int)(blockIdx.z % n_img) : (int)blockIdx.z;
+static_assert(sizeof(ConvArgs) % 4 == 0 && sizeof(ConvArgs) <= DW_ENTRY_BYTES, "depthwise table record");
+
+template <int K, int ST, bool GROUP>
+__global__ void __launch_bounds__(256) dw_vec_kernel(const ConvArgs a1, const char *__restrict__ tbl, int n_img) {
+    SGS_DW_ARGS()
     constexpr int TW = 4, NCOL = (TW - 1) * ST + K, P = (K - 1) / 2;
     // grid: x covers (channel vector, pixel block) of one output row, y = output row, z = image;
     // all index arithmetic stays in 32 bits
@@ -182,7 +196,7 @@ __global__ void __launch_bounds__(256) dw_vec_kernel(ConvArgs a) {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= groups * wblocks) return;
     const int cg = idx % groups, wb = idx / groups;
-    const int ho = blockIdx.y, n = blockIdx.z;
+    const int ho = blockIdx.y;
     const int c0 = cg * 8, wo0 = wb * TW, o = (a.R - K) / 2;
     const __nv_bfloat16 *__restrict__ x = static_cast<const __nv_bfloat16 *>(a.x);
     const __nv_bfloat16 *__restrict__ w = static_cast<const __nv_bfloat16 *>(a.w);
@@ -245,14 +259,15 @@ __global__ void __launch_bounds__(256) dw_vec_kernel(ConvArgs a) {
 // in flight, not by occupancy).  Patches whose halo lies inside the image take a path without bounds
 // tests.  The epilogue is packed: one FMA for the folded batch norm per channel pair, and h-swish as
 // x * clamp(x / 6 + 0.5, 0, 1) (= x * relu6(x + 3) / 6): one saturating FMA and one packed multiply.
-template <int K, int ST, int TH, int TW, bool PRELOAD, int ACT>
-__global__ void __launch_bounds__(128) dw_tile_kernel(ConvArgs a) {
+template <int K, int ST, int TH, int TW, bool PRELOAD, int ACT, bool GROUP>
+__global__ void __launch_bounds__(128) dw_tile_kernel(const ConvArgs a1, const char *__restrict__ tbl, int n_img) {
+    SGS_DW_ARGS()
     constexpr int P = (K - 1) / 2, NCOL = (TW - 1) * ST + K, NROW = (TH - 1) * ST + K;
     const int groups = a.K / 8, wblocks = (a.Wo + TW - 1) / TW;
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= groups * wblocks) return;
     const int cg = idx % groups, wb = idx / groups;
-    const int ho0 = blockIdx.y * TH, n = blockIdx.z;
+    const int ho0 = blockIdx.y * TH;
     const int c0 = cg * 8, wo0 = wb * TW, o = (a.R - K) / 2;
     const __nv_bfloat16 *__restrict__ x = static_cast<const __nv_bfloat16 *>(a.x);
     const __nv_bfloat16 *__restrict__ w = static_cast<const __nv_bfloat16 *>(a.w);
@@ -368,44 +383,69 @@ __global__ void __launch_bounds__(128) dw_tile_kernel(ConvArgs a) {
     }
 }
 
-template <int K, int ST, int TH, int TW, bool PRELOAD> static cudaError_t launch_dw_tile(const ConvArgs &a, cudaStream_t st) {
-    const int per_row = ((a.Wo + TW - 1) / TW) * (a.K / 8);
-    dim3 grid((per_row + 127) / 128, (a.Ho + TH - 1) / TH, a.N);
-    if (a.act == ACT_RELU) dw_tile_kernel<K, ST, TH, TW, PRELOAD, ACT_RELU><<<grid, 128, 0, st>>>(a);
-    else if (a.act == ACT_HSWISH) dw_tile_kernel<K, ST, TH, TW, PRELOAD, ACT_HSWISH><<<grid, 128, 0, st>>>(a);
-    else dw_tile_kernel<K, ST, TH, TW, PRELOAD, ACT_NONE><<<grid, 128, 0, st>>>(a);
+// `a` = the (first) member; grouped: kmax = the widest member's channel count, tbl = device table, members > 0
+template <int K, int ST, int TH, int TW, bool PRELOAD, bool GROUP>
+static cudaError_t launch_dw_tile(const ConvArgs &a, int kmax, const char *tbl, int members, cudaStream_t st) {
+    const int per_row = ((a.Wo + TW - 1) / TW) * (kmax / 8);
+    dim3 grid((per_row + 127) / 128, (a.Ho + TH - 1) / TH, a.N * (GROUP ? members : 1));
+    if (a.act == ACT_RELU) dw_tile_kernel<K, ST, TH, TW, PRELOAD, ACT_RELU, GROUP><<<grid, 128, 0, st>>>(a, tbl, a.N);
+    else if (a.act == ACT_HSWISH) dw_tile_kernel<K, ST, TH, TW, PRELOAD, ACT_HSWISH, GROUP><<<grid, 128, 0, st>>>(a, tbl, a.N);
+    else dw_tile_kernel<K, ST, TH, TW, PRELOAD, ACT_NONE, GROUP><<<grid, 128, 0, st>>>(a, tbl, a.N);
     return cudaGetLastError();
 }
 
-template <int K, int ST> static cudaError_t launch_dw_vec(const ConvArgs &a, cudaStream_t st) {
-    const int per_row = ((a.Wo + 3) / 4) * (a.K / 8);
+template <int K, int ST, bool GROUP>
+static cudaError_t launch_dw_vec(const ConvArgs &a, int kmax, const char *tbl, int members, cudaStream_t st) {
+    const int per_row = ((a.Wo + 3) / 4) * (kmax / 8);
     const int block = per_row >= 256 ? 256 : per_row >= 128 ? 128 : 64;
-    dim3 grid((per_row + block - 1) / block, a.Ho, a.N);
-    dw_vec_kernel<K, ST><<<grid, block, 0, st>>>(a);
+    dim3 grid((per_row + block - 1) / block, a.Ho, a.N * (GROUP ? members : 1));
+    dw_vec_kernel<K, ST, GROUP><<<grid, block, 0, st>>>(a, tbl, a.N);
     return cudaGetLastError();
+}
+
+static bool dw_vec_eligible(const ConvArgs &a) {
+    return a.K % 8 == 0 && a.Kmax % 8 == 0 && (a.stride == 1 || a.stride == 2) && a.Ho <= 65535 && a.N <= 65535 &&
+           (size_t)a.W * a.K < (1u << 30) &&
+           ((reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.w) | reinterpret_cast<uintptr_t>(a.y)) & 15) == 0 &&
+           ((reinterpret_cast<uintptr_t>(a.scale) | reinterpret_cast<uintptr_t>(a.shift)) & 15) == 0;
+}
+
+// The vectorised bf16 kernel of a (kernel size, stride) pair; measured on working sets beyond L2
+// (N64 56x56 C480) the tiled kernel wins for k3 and for k5 stride 1.
+template <bool GROUP>
+static cudaError_t launch_dw_bf16(const ConvArgs &a, int kmax, const char *tbl, int members, cudaStream_t st) {
+    switch (a.k * 10 + a.stride) {
+    case 31: return launch_dw_tile<3, 1, 2, 4, true, GROUP>(a, kmax, tbl, members, st);
+    case 32: return launch_dw_tile<3, 2, 1, 4, false, GROUP>(a, kmax, tbl, members, st);
+    case 51: return launch_dw_tile<5, 1, 1, 4, true, GROUP>(a, kmax, tbl, members, st);
+    case 52: return launch_dw_vec<5, 2, GROUP>(a, kmax, tbl, members, st);
+    case 71: return launch_dw_vec<7, 1, GROUP>(a, kmax, tbl, members, st);
+    case 72: return launch_dw_vec<7, 2, GROUP>(a, kmax, tbl, members, st);
+    default: return cudaErrorNotSupported;
+    }
+}
+
+cudaError_t launch_dw_group(const char *h_tbl, const char *d_tbl, int members, cudaStream_t st) {
+    if (members <= 0) return cudaSuccess;
+    const ConvArgs &a0 = *reinterpret_cast<const ConvArgs *>(h_tbl);
+    int kmax = 0;
+    for (int i = 0; i < members; i++) {
+        const ConvArgs &a = *reinterpret_cast<const ConvArgs *>(h_tbl + (size_t)i * DW_ENTRY_BYTES);
+        if (!dw_vec_eligible(a) || a.k != a0.k || a.stride != a0.stride || a.act != a0.act || a.N != a0.N || a.H != a0.H || a.W != a0.W ||
+            a.Ho != a0.Ho || a.Wo != a0.Wo)
+            return cudaErrorNotSupported;
+        kmax = std::max(kmax, a.K);
+    }
+    if ((long long)a0.N * members > 65535) return cudaErrorNotSupported;
+    return launch_dw_bf16<true>(a0, kmax, d_tbl, members, st);
 }
 
 template <typename T> cudaError_t launch_dw(const ConvArgs &a, cudaStream_t st) {
     size_t total = (size_t)a.N * a.Ho * a.Wo * a.K;
     if (!total) return cudaSuccess;
-    if (sizeof(T) == 2 && a.K % 8 == 0 && a.Kmax % 8 == 0 && (a.stride == 1 || a.stride == 2) && a.Ho <= 65535 && a.N <= 65535 &&
-        (size_t)a.W * a.K < (1u << 30) &&
-        ((reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.w) | reinterpret_cast<uintptr_t>(a.y)) & 15) == 0 &&
-        ((reinterpret_cast<uintptr_t>(a.scale) | reinterpret_cast<uintptr_t>(a.shift)) & 15) == 0) {
-        const int key = a.k * 10 + a.stride;
-        // measured on working sets beyond L2 (N64 56x56 C480): the tiled kernel wins for these three shapes
-        if (key == 31) return launch_dw_tile<3, 1, 2, 4, true>(a, st);
-        if (key == 32) return launch_dw_tile<3, 2, 1, 4, false>(a, st);
-        if (key == 51) return launch_dw_tile<5, 1, 1, 4, true>(a, st);
-        switch (key) {
-        case 31: return launch_dw_vec<3, 1>(a, st);
-        case 32: return launch_dw_vec<3, 2>(a, st);
-        case 51: return launch_dw_vec<5, 1>(a, st);
-        case 52: return launch_dw_vec<5, 2>(a, st);
-        case 71: return launch_dw_vec<7, 1>(a, st);
-        case 72: return launch_dw_vec<7, 2>(a, st);
-        default: break;
-        }
+    if (sizeof(T) == 2 && dw_vec_eligible(a)) {
+        cudaError_t e = launch_dw_bf16<false>(a, a.K, nullptr, 1, st);
+        if (e != cudaErrorNotSupported) return e;
     }
     int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
     dw_plain_kernel<T><<<blocks, 256, 0, st>>>(a);
@@ -711,6 +751,61 @@ __device__ __forceinline__ void gap_body(const SmallEntry &e, int bx) {
     }
 }
 
+// y[n][hw][c] = x[n][hw][c] * gate[n][c] (gate = e.w, fp32): a thread scales one 8-channel vector.
+__device__ __forceinline__ void scale_body(const SmallEntry &e, int bx, int nbx) {
+    const int cvecs = e.C >> 3, per_image = e.H * e.W * cvecs, total = e.N * per_image;
+    const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(e.x);
+    const float *gate = static_cast<const float *>(e.w);
+    __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(e.y);
+    for (int i = bx * blockDim.x + threadIdx.x; i < total; i += nbx * blockDim.x) {
+        const int n = i / per_image, cv = i % cvecs;
+        const uint4 v = *reinterpret_cast<const uint4 *>(x + (size_t)i * 8);
+        const float4 g0 = __ldg(reinterpret_cast<const float4 *>(gate + (size_t)n * e.C + cv * 8));
+        const float4 g1 = __ldg(reinterpret_cast<const float4 *>(gate + (size_t)n * e.C + cv * 8 + 4));
+        const float2 a = bf2f(v.x), b = bf2f(v.y), c = bf2f(v.z), d = bf2f(v.w);
+        uint4 o;
+        __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&o);
+        ob[0] = __floats2bfloat162_rn(a.x * g0.x, a.y * g0.y);
+        ob[1] = __floats2bfloat162_rn(b.x * g0.z, b.y * g0.w);
+        ob[2] = __floats2bfloat162_rn(c.x * g1.x, c.y * g1.y);
+        ob[3] = __floats2bfloat162_rn(d.x * g1.z, d.y * g1.w);
+        *reinterpret_cast<uint4 *>(y + (size_t)i * 8) = o;
+    }
+}
+
+// Squeeze-excite gate of one image of one member (se_gate_kernel's arithmetic): x = pooled vector,
+// w / bias = first FC (K = squeeze width, ld), w2 / bias2 = second FC (ld2), y = gate; C = mid channels.
+__global__ void __launch_bounds__(1024) se_gate_group_kernel(const SmallEntry *__restrict__ tbl) {
+    extern __shared__ float sm[];
+    __shared__ SmallEntry e;
+    if (threadIdx.x < 8) reinterpret_cast<uint4 *>(&e)[threadIdx.x] = __ldg(reinterpret_cast<const uint4 *>(tbl + blockIdx.y) + threadIdx.x);
+    __syncthreads();
+    const int mid = e.C, sq = e.K;
+    float *gs = sm, *zs = sm + mid;
+    const int n = blockIdx.x, lane = threadIdx.x % 32, warp = threadIdx.x / 32, nw = blockDim.x / 32;
+    if (n >= e.N) return;
+    const float *g = static_cast<const float *>(e.x);
+    const __nv_bfloat16 *w1 = static_cast<const __nv_bfloat16 *>(e.w), *w2 = static_cast<const __nv_bfloat16 *>(e.w2);
+    float *gate = static_cast<float *>(e.y);
+    for (int c = threadIdx.x; c < mid; c += blockDim.x) gs[c] = g[(size_t)n * mid + c];
+    __syncthreads();
+    for (int j = warp; j < sq; j += nw) {
+        float s = 0.f;
+        for (int c = lane; c < mid; c += 32) s = fmaf(__bfloat162float(w1[(size_t)j * e.ld + c]), gs[c], s);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) zs[j] = fmaxf(s + e.bias[j], 0.f);
+    }
+    __syncthreads();
+    for (int c = warp; c < mid; c += nw) {
+        float s = 0.f;
+        for (int j = lane; j < sq; j += 32) s = fmaf(__bfloat162float(w2[(size_t)c * e.ld2 + j]), zs[j], s);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) gate[(size_t)n * mid + c] = fminf(fmaxf(s + e.bias2[c] + 3.f, 0.f), 6.f) / 6.f;
+    }
+}
+
 // Sliced linear layer on fp32 vectors: one warp per (image, output), 16-byte weight loads.
 __device__ __forceinline__ void linear_body(const SmallEntry &e, int bx) {
     const int warp = (bx * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
@@ -789,6 +884,7 @@ template <int KIND, int K, int ST> __device__ __forceinline__ void small_body(co
     if constexpr (KIND == OP_MAXPOOL) maxpool_body(e, bx, nbx);
     else if constexpr (KIND == OP_GAP) gap_body(e, bx);
     else if constexpr (KIND == OP_LINEAR) linear_body(e, bx);
+    else if constexpr (KIND == OP_SCALE) scale_body(e, bx, nbx);
     else im2col_body<K, ST>(e, bx);
 }
 template <int KIND, int K, int ST> __global__ void __launch_bounds__(256) small_single_kernel(const SmallEntry e) {
@@ -852,6 +948,8 @@ bool small_supported(int kind, const SmallEntry &e) {
     switch (kind) {
     case OP_MAXPOOL: return e.C % 8 == 0 && (long long)e.N * e.Ho * e.Wo * (e.C / 8) < (1ll << 31);
     case OP_GAP: return e.C % 8 == 0;
+    case OP_SCALE: return e.C % 8 == 0 && al(e.w) && (long long)e.N * e.H * e.W * (e.C / 8) < (1ll << 31);
+    case OP_SE_GATE: return e.w2 != nullptr;
     case OP_LINEAR: return e.C % 8 == 0 && e.ld % 8 == 0 && al(e.w);
     case OP_IM2COL: return (e.k == 3 || e.k == 7) && (e.stride == 1 || e.stride == 2) && e.KKp % 8 == 0 && e.KKp >= e.k * e.k * 3 &&
                            e.W % 8 == 0 && e.W <= IM2COL_MAX_W && (long long)e.N * e.Ho < (1ll << 31) && (long long)e.Wo * (e.KKp / 8) < (1ll << 31);
@@ -864,6 +962,7 @@ static long long small_blocks(int kind, const SmallEntry &e) {
     switch (kind) {
     case OP_MAXPOOL: return ((long long)e.N * e.Ho * e.Wo * (e.C / 8) + 255) / 256;
     case OP_GAP: return ((long long)e.N * (e.C / 8) * 32 + 255) / 256;
+    case OP_SCALE: return ((long long)e.N * e.H * e.W * (e.C / 8) + 255) / 256;
     case OP_LINEAR: return ((long long)e.N * e.K * 32 + 255) / 256;
     default: return (long long)e.N * e.Ho;  // patch matrix: one block per output row
     }
@@ -881,12 +980,20 @@ cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int
     if ((!d && n != 1) || n > 65535) return cudaErrorInvalidValue;
     long long blocks = 1;
     for (int i = 0; i < n; i++) blocks = std::max(blocks, small_blocks(kind, h[i]));
-    // the grid-stride kernel (max pool) need not cover every element with a block of its own
-    if (kind == OP_MAXPOOL) blocks = std::min<long long>(blocks, 148 * 16);
+    // the grid-stride kernels (max pool, SE scale) need not cover every element with a block of their own
+    if (kind == OP_MAXPOOL || kind == OP_SCALE) blocks = std::min<long long>(blocks, 148 * 16);
     const unsigned bx = (unsigned)blocks;
     switch (kind) {
     case OP_MAXPOOL: return launch_small_t<OP_MAXPOOL, 0, 0>(h, d, n, bx, st);
     case OP_GAP: return launch_small_t<OP_GAP, 0, 0>(h, d, n, bx, st);
+    case OP_SCALE: return launch_small_t<OP_SCALE, 0, 0>(h, d, n, bx, st);
+    case OP_SE_GATE: {
+        if (!d) return cudaErrorInvalidValue;
+        int nimg = 0, fl = 0;
+        for (int i = 0; i < n; i++) { nimg = std::max(nimg, h[i].N); fl = std::max(fl, h[i].C + h[i].K); }
+        se_gate_group_kernel<<<dim3((unsigned)nimg, (unsigned)n), 1024, (size_t)fl * sizeof(float), st>>>(d);
+        return cudaGetLastError();
+    }
     case OP_LINEAR: {
         bool same = d != nullptr && n > 1;
         for (int i = 1; i < n && same; i++)

@@ -83,10 +83,10 @@ def test_resnet_wave_batched_members_224():
 
 
 def test_wave_mode_on_the_other_families():
-    # MobileNetV3-shaped (depthwise, SE) and Tiny SuperNets: ops without a grouped kernel run per member
-    for fam, res, ncls in ((wl.MBV3, 64, 1000), (wl.TINY, 32, 10)):
+    # MobileNetV3-shaped (depthwise and SE layers grouped by kernel size) and Tiny SuperNets (CUDA-core
+    # convolutions run per member)
+    for fam, res, ncls, n in ((wl.MBV3, 64, 1000, 6), (wl.MBV3, 96, 1000, 11), (wl.TINY, 32, 10, 6)):
         _, onet, gnet = gu.nets(fam, True)
-        n = 6
         cfgs = wl.uniform_stream(fam, n, seed=7)
         xs = wl.make_inputs(n, 1, res, seed=8, bf16=True)
         d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
