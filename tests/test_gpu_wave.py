@@ -94,3 +94,28 @@ def test_wave_mode_on_the_other_families():
         for t in range(n):
             ref = onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)
             assert gu.rel_err(got[t:t + 1], ref) <= TOL_BF16, (fam, t)
+
+
+def test_bench_wave_configuration_sampled_against_checker():
+    # the benchmark's launch configuration (224x224, batch 1, waves of 32, 4 waves in flight, cache on) on the
+    # first 160 queries of its stream: sampled queries recomputed by the checker, every logit finite, the
+    # stream reproduces itself bit for bit, and the top-1 class of the sampled queries agrees
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    n, res = 160, 224
+    cfgs = wl.uniform_stream(wl.RESNET, 1000, seed=2)[:n]
+    xs = wl.make_inputs(n, 1, res, seed=1, bf16=True)
+    d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
+    first, st = _run(gnet, cfgs, d_in, 1, res, 1000, wave=32, conc=4, latency=1)
+    again, _ = _run(gnet, cfgs, d_in, 1, res, 1000, wave=32, conc=4)
+    np.testing.assert_array_equal(again, first)
+    assert np.all(np.isfinite(first)) and st.p50_ms > 0
+    sample = list(range(0, n, 7))
+    strict = 0
+    worst = 0.0
+    for t in sample:
+        ref = onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)
+        worst = max(worst, gu.rel_err(first[t:t + 1], ref))
+        strict += int(first[t].argmax() == ref[0].argmax())
+    print(f"wave configuration: worst rel err {worst:.2e}, top-1 agreement {strict}/{len(sample)}")
+    assert worst <= TOL_BF16
+    assert strict >= len(sample) - 1
