@@ -157,6 +157,8 @@ struct sgs_supernet {
     // (r, s, c) order, zero padded to a multiple of 8), used with the patch matrix of the input
     void *stem_gemm_w = nullptr;
     int stem_kkp = 0;
+    // ... and as [K][k][64] for the window view used by waves: per filter row an 8-pixel x 8-channel window
+    void *stem_win_w = nullptr;
     // Workspaces of the queries in flight.  Queries of a stream are independent, so up to
     // `concurrency` of them run at the same time, each in its own slot (own activation buffers, own
     // scratch, own CUDA stream); slot 0 runs on the caller's stream.
@@ -394,6 +396,28 @@ struct Builder {
         const int Hin = H, Win = W;
         conv(name, -1, out, -1, H, W, stride, act);
         // (the patch-matrix kernel stages whole input rows with 16-byte loads: widths that are multiples of 8)
+        if (net->throughput_mode == 2 && net->stem_win_w && !net->force_plain && s.K % 8 == 0 && (s.k == 3 || s.k == 7)) {
+            // Waves: no patch matrix.  The image is copied once into an 8-channel buffer with a zero margin
+            // (16 bytes per pixel, so that pixels can be TMA rows); the 64 contiguous elements that start at
+            // padded pixel wo * stride are the 8-pixel window of output column wo, and the stem becomes a
+            // convolution over the k filter ROWS with 64 "channels" per row.
+            Op &cv = plan->ops[first];
+            const int P = (s.k - 1) / 2;
+            int Hp = std::max((H - 1) * stride + s.k, Hin + P), Wp = std::max((W - 1) * stride + 8, Win + P);
+            Hp += Hp & 1; Wp += Wp & 1;
+            Op pd;
+            pd.type = OP_PAD8; pd.layer = li; pd.in = -1; pd.out = tmp;
+            pd.N = N; pd.H = Hin; pd.W = Win; pd.C = 3; pd.K = P;
+            pd.conv.Ho = Hp; pd.conv.Wo = Wp;
+            pd.alg_bytes = ((double)N * Hin * Win * 3 + (double)N * Hp * Wp * 8) * net->elem();
+            cv.in = tmp;
+            ConvArgs &a = cv.conv;
+            a.w = net->stem_win_w;
+            a.H = Hp; a.W = Wp; a.C = 64; a.Cmax = 64; a.win = 1;
+            note((size_t)N * Hp * Wp * 8);
+            plan->ops.insert(plan->ops.begin() + (long)first, pd);
+            return;
+        }
         if (!net->stem_gemm_w || net->force_plain || s.K % 8 || (s.k != 3 && s.k != 7) || Win % 8 || Win > 1024) return;
         Op &cv = plan->ops[first];
         const int KKp = net->stem_kkp;
@@ -589,6 +613,7 @@ sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
         if (net->dtype != SGS_BF16 || net->force_plain || !tc_available()) continue;
         std::string why;
         op.tc = tc_conv_prepare(op.conv, net->device, &why);
+        if (!op.tc && op.conv.win) return fail(net, SGS_EUNSUPPORTED, "window view of the stem: " + why);
         if (op.tc) {
             op.impl = 1;
             ws_need = std::max(ws_need, tc_conv_ws_elems(*op.tc));
@@ -629,10 +654,16 @@ sgs_status_t ensure_ranks(sgs_supernet *net) {
         for (int b = 0; b < SGS_MAX_BLOCKS; b++) { c.expand[s][b] = net->family == SGS_MBV3 ? 6.0f : 0.35f; c.kernel[s][b] = 7; }
     }
     c.width[0] = 1.0f;
-    Plan p;
-    sgs_status_t st = build_plan(net, &c, 1, 64, &p);
-    if (st != SGS_OK) return st;
-    for (size_t i = 0; i < p.ops.size(); i++) net->op_rank[op_key(p, i)] = (int)i;
+    // (the stem has two forms, patch matrix + GEMM and padded copy + window view: both are ranked)
+    const int mode = net->throughput_mode;
+    for (int m : {0, 2}) {
+        net->throughput_mode = m;
+        Plan p;
+        sgs_status_t st = build_plan(net, &c, 1, 64, &p);
+        if (st != SGS_OK) { net->throughput_mode = mode; return st; }
+        for (size_t i = 0; i < p.ops.size(); i++) net->op_rank.emplace(op_key(p, i), (int)i);
+    }
+    net->throughput_mode = mode;
     return SGS_OK;
 }
 
@@ -695,6 +726,10 @@ SmallEntry small_entry(const sgs_supernet *net, const Plan *plan, const Op &op, 
         e.N = op.N; e.C = op.C; e.K = op.K;
         break;
     }
+    case OP_PAD8:
+        e.x = d_input; e.y = sl.act[op.out];
+        e.N = op.N; e.H = op.H; e.W = op.W; e.C = 3; e.k = op.K; e.Ho = op.conv.Ho; e.Wo = op.conv.Wo;
+        break;
     case OP_IM2COL:
         e.x = d_input; e.y = sl.act[op.out];
         e.N = op.N; e.H = op.H; e.W = op.W; e.C = 3;
@@ -722,9 +757,10 @@ sgs_status_t launch_op(sgs_supernet *net, Plan *plan, Op &op, const void *d_inpu
         else { CU(launch_conv_plain<T>(a, st)); net->kernel_launches++; }
         break;
     }
+    case OP_PAD8:
     case OP_IM2COL: {
         SmallEntry e = small_entry(net, plan, op, d_input, d_logits);
-        CU(launch_small(OP_IM2COL, &e, nullptr, 1, st));
+        CU(launch_small(op.type, &e, nullptr, 1, st));
         net->kernel_launches++;
         break;
     }
@@ -1074,6 +1110,10 @@ sgs_status_t sgs_supernet_load(const sgs_arch_desc_t *arch, const void *host_blo
         net->stem_kkp = (KK + 7) / 8 * 8;
         if (dev_alloc(net, &net->stem_gemm_w, (size_t)L.K * net->stem_kkp * 2) != SGS_OK) e = cudaErrorMemoryAllocation;
         else e = launch_stem_gemm_weights(L.w, net->stem_gemm_w, L.K, KK, net->stem_kkp, 0);
+        if (e == cudaSuccess && L.R <= 8) {
+            if (dev_alloc(net, &net->stem_win_w, (size_t)L.K * L.R * 64 * 2) != SGS_OK) e = cudaErrorMemoryAllocation;
+            else e = launch_stem_window_weights(L.w, net->stem_win_w, L.K, L.R, 0);
+        }
     }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     cleanup_stage();
@@ -1114,6 +1154,7 @@ void sgs_supernet_free(sgs_supernet_t *net) {
     cudaFree(net->weight_arena);
     cudaFree(net->param_arena);
     cudaFree(net->stem_gemm_w);
+    cudaFree(net->stem_win_w);
     for (auto &sl : net->slots) {
         for (int i = 0; i < 4; i++) cudaFree(sl.act[i]);
         for (int i = 0; i < 3; i++) cudaFree(sl.vec[i]);
@@ -1314,7 +1355,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             // member's op has the vectorised form; the remaining ops run member by member
             const Op &op0 = plans[b[0].first]->ops[(size_t)b[0].second];
             const int kind = op0.type;
-            bool grouped = kind == OP_MAXPOOL || kind == OP_GAP || kind == OP_LINEAR || kind == OP_IM2COL || kind == OP_SCALE || kind == OP_SE_GATE;
+            bool grouped = kind == OP_MAXPOOL || kind == OP_GAP || kind == OP_LINEAR || kind == OP_IM2COL || kind == OP_SCALE || kind == OP_SE_GATE || kind == OP_PAD8;
             if (grouped) {
                 const size_t off0 = off;
                 for (const auto &mo : b) {

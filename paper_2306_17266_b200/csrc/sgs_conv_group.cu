@@ -53,7 +53,7 @@ struct __align__(16) GroupEntry {
     short bn_tile;           // MMA columns of a full tile
     short pix_rows;          // rows of the pixel box (bw * bh * bn)
     short pad0_;
-    unsigned char k, stride, p, act, swap, pad1_[3];
+    unsigned char k, stride, p, act, swap, kw, pad1_[2];  // k x kw taps
     int pad2_[3];
 };
 static_assert(sizeof(GroupEntry) == TC_GROUP_ENTRY_BYTES, "entry size");
@@ -157,14 +157,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             const uint32_t w_bytes = (uint32_t)(wrows * CHUNK_C * 2);
             uint8_t *dst0 = smem + (e.swap ? 0 : G_X_BYTES);
             const CUtensorMap *map_w = &P.maps[e.map_w];
-            const int k = e.k, cchunks = e.cchunks, R = e.R;
+            const int k = e.k, kw = e.kw, cchunks = e.cchunks, R = e.R;
             int kind = 0;  // 0 default replacement, 1 keep (inside the cached SubGraph's box, up to channel cacheC), 2 stream
             int cacheC = 0;
             if (weight_policy == 2) kind = 2;
             else if (weight_policy == 1 && f0 < __ldg(cache_tbl + 1 + 2 * e.layer)) { kind = 1; cacheC = __ldg(cache_tbl + 2 + 2 * e.layer); }
             int tap_row = e.tap0;
             for (int r = 0; r < k && ok; r++, tap_row += R) {
-                for (int sx = 0; sx < k && ok; sx++) {
+                for (int sx = 0; sx < kw && ok; sx++) {
                     for (int cc = 0, c0 = 0; cc < cchunks; cc++, c0 += CHUNK_C) {
                         { ROLE_T0(); if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag)); ROLE_ADD(tw_); }
                         if (!ok) break;
@@ -200,9 +200,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             const uint32_t pix_bytes = (uint32_t)(e.pix_rows * CHUNK_C * 2);
             uint8_t *dst0 = smem + (e.swap ? G_X_BYTES : 0);
             const CUtensorMap *map_a = &P.maps[e.map_a];
-            const int k = e.k, cchunks = e.cchunks, pad = e.p, stride = e.stride;
+            const int k = e.k, kw = e.kw, cchunks = e.cchunks, pad = e.p, stride = e.stride;
             for (int r = 0; r < k && ok; r++) {
-                for (int sx = 0; sx < k && ok; sx++) {
+                for (int sx = 0; sx < kw && ok; sx++) {
                     const int dh = r - pad, dw = sx - pad;
                     // stride 2: one of the four parity views, at half the offset
                     const int ph = stride == 2 ? (dh & 1) : 0, pw = stride == 2 ? (dw & 1) : 0;
@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             const int n_mma = e.swap ? e.bn_tile : min((int)e.bn_tile, (e.K - nt * e.bn_tile + 15) & ~15);
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
             const int buf = j & 1;
-            const int cchunks = e.cchunks, taps = e.k * e.k;
+            const int cchunks = e.cchunks, taps = e.k * e.kw;
             const int last_ksteps = (e.C - (cchunks - 1) * CHUNK_C + 15) / 16;  // 16-channel steps of a tap's last chunk
             { ROLE_T0(); ok = j < 2 || mbar_wait(&acc_empty[buf], ((j >> 1) - 1) & 1, abort_flag);  // epilogue drained this buffer
             ok = __all_sync(0xffffffffu, ok); ROLE_ADD(tacc_); }
@@ -447,7 +447,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
 
 // Number of activation views a member needs: the four parity views only when a stride-2 kernel
 // reaches odd offsets, i.e. for kernels larger than 1x1.
-static int views_of(const TcParams &p) { return (p.stride == 2 && p.k > 1) ? 4 : 1; }
+static int views_of(const TcParams &p) { return (p.stride == 2 && p.k > 1) ? 4 : 1; }  // (a stride-2 window view uses views 0 and 2 of 4)
 
 struct GroupLaunch::Impl {
     GroupParams<TC_GROUP_MAPS_LARGE> prm;  // host image of the parameter block (the small variant is a prefix)
@@ -496,7 +496,7 @@ void GroupLaunch::add(void *host_entry, const TcConvPlan &pl, const ConvArgs &a)
     e.pix_rows = (short)(p.bw * p.bh * p.bn);
     e.swap = (unsigned char)pl.swap;
     e.bn_tile = (short)(pl.swap ? (e.pix_rows + 15) / 16 * 16 : pl.bn_tile);
-    e.k = (unsigned char)p.k; e.stride = (unsigned char)p.stride; e.p = (unsigned char)p.p; e.act = (unsigned char)p.act;
+    e.k = (unsigned char)p.k; e.kw = (unsigned char)pl.kw; e.stride = (unsigned char)p.stride; e.p = (unsigned char)p.p; e.act = (unsigned char)p.act;
     if ((pl.swap ? e.pix_rows : e.bn_tile) > 128) impl->wide = true;
     std::memcpy(host_entry, &e, sizeof e);
     impl->prm.n_entries++;

@@ -383,6 +383,12 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
     std::memset(&p, 0, sizeof(p));
     p.N = a.N; p.Ho = a.Ho; p.Wo = a.Wo; p.K = a.K; p.C = a.C;
     p.k = a.k; p.stride = a.stride; p.R = a.R; p.o = (a.R - a.k) / 2; p.p = (a.k - 1) / 2;
+    plan->kw = a.k;
+    if (a.win) {
+        // window view of a stem: taps = the k filter rows, no arithmetic padding (the margin is in the buffer)
+        if (a.throughput != 2 || a.C != CHUNK_C || a.Cmax != CHUNK_C) return no("window view");
+        plan->kw = 1; p.R = 1; p.o = 0; p.p = 0;
+    }
     p.act = a.act;
     const bool flat = a.k == 1 && a.stride == 1;
     const uint64_t C = (uint64_t)a.C, eb = 2;
@@ -404,8 +410,22 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
     } else {
         if (swap) { p.bw = a.Wo; p.bh = a.Ho; p.bn = a.N; }
         else choose_box(a.N, a.Ho, a.Wo, &p.bw, &p.bh, &p.bn);
+        if (a.win) {
+            // dim 0 = the 64-element window of output column wo (starts at padded pixel wo * stride), dim 1 = wo,
+            // dim 2 = input row (stride 2: rows of one parity), dim 3 = image
+            uint32_t wbox[4] = {CHUNK_C, (uint32_t)p.bw, (uint32_t)p.bh, (uint32_t)p.bn};
+            const uint64_t px = 8 * eb, st = (uint64_t)a.stride;
+            for (int ph = 0; ph < a.stride; ph++) {
+                const char *base = static_cast<const char *>(a.x) + (size_t)ph * a.W * px;
+                uint64_t dims[4] = {CHUNK_C, (uint64_t)a.Wo, (uint64_t)(a.H - ph + a.stride - 1) / st, (uint64_t)a.N};
+                uint64_t str[3] = {st * px, st * (uint64_t)a.W * px, (uint64_t)a.H * a.W * px};
+                if (!encode_map(&p.tmA[ph * 2], base, 4, dims, str, wbox)) return no("window tensor map");
+            }
+        }
         uint32_t box[4] = {CHUNK_C, (uint32_t)p.bw, (uint32_t)p.bh, (uint32_t)p.bn};
-        if (a.stride == 1) {
+        if (a.win) {
+            // (encoded above)
+        } else if (a.stride == 1) {
             uint64_t dims[4] = {C, (uint64_t)a.W, (uint64_t)a.H, (uint64_t)a.N};
             uint64_t str[3] = {C * eb, (uint64_t)a.W * C * eb, (uint64_t)a.H * a.W * C * eb};
             if (!encode_map(&p.tmA[0], a.x, 4, dims, str, box)) return no("activation tensor map");
@@ -433,7 +453,7 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
         if (ds.sms > 0) sms = ds.sms;
     }
     p.cchunks = (a.C + CHUNK_C - 1) / CHUNK_C;
-    p.iters = a.k * a.k * p.cchunks;
+    p.iters = a.k * plan->kw * p.cchunks;
     // Filter tile.  Issuing one MMA costs the issuing thread about the same whatever its width, so wide
     // tiles are preferred as long as tiles x K splits can still occupy every SM.
     // a split costs a second (small) kernel, so it has to save at least a dozen pipeline iterations
@@ -458,8 +478,9 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
     }
     plan->bn_tile = BN;
     {
-        uint64_t dims[3] = {C, (uint64_t)a.R * a.R, (uint64_t)a.K};
-        uint64_t str[2] = {(uint64_t)a.Cmax * eb, (uint64_t)a.R * a.R * a.Cmax * eb};
+        const uint64_t taps = a.win ? (uint64_t)a.k : (uint64_t)a.R * a.R;  // stored taps per filter
+        uint64_t dims[3] = {C, taps, (uint64_t)a.K};
+        uint64_t str[2] = {(uint64_t)a.Cmax * eb, taps * a.Cmax * eb};
         uint32_t box[3] = {CHUNK_C, 1, (uint32_t)BN};
         if (!encode_map(&p.tmW, a.w, 3, dims, str, box)) return no("weight tensor map");
     }

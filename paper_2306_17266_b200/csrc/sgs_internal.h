@@ -48,6 +48,11 @@ struct ConvArgs {
     int N = 0, H = 0, W = 0, C = 0, Ho = 0, Wo = 0, K = 0;
     int Kmax = 0, Cmax = 0, R = 0;  // stored dims (square kernels)
     int k = 1, stride = 1, act = 0;
+    // Window view of a 3-channel stem (grouped launches): x is the input padded to 8 channels with a zero
+    // margin, [N][H][W][8] with H, W the PADDED sizes; an "input channel" chunk is the 8-pixel x 8-channel
+    // window that starts at output column wo * stride (64 contiguous elements), the taps are the k filter ROWS
+    // only (C = Cmax = 64, R = 1), and the weights are [Kmax][k][64] with zeros where the window has no tap.
+    int win = 0;
     // SubGraph cache box of this layer: weight tiles with filter < cacheK and channel < cacheC are
     // loaded with an evict-last L2 policy; weight_policy 0 = none, 1 = use the box, 2 = all evict-first
     int cacheK = 0, cacheC = 0, weight_policy = 0;
@@ -63,7 +68,7 @@ struct ConvArgs {
     size_t ws_elems = 0;
 };
 
-enum OpType { OP_CONV, OP_DW, OP_MAXPOOL, OP_GAP, OP_SE_GATE, OP_SCALE, OP_LINEAR, OP_IM2COL };
+enum OpType { OP_CONV, OP_DW, OP_MAXPOOL, OP_GAP, OP_SE_GATE, OP_SCALE, OP_LINEAR, OP_IM2COL, OP_PAD8 };
 
 struct TcConvPlan;  // tensor-core launch description (sgs_conv_tc.cu)
 
@@ -133,7 +138,8 @@ struct alignas(16) SmallEntry {
 static_assert(sizeof(SmallEntry) == 128, "record size");
 // kind: OP_MAXPOOL (3x3 stride 2, C % 8 == 0), OP_GAP (C % 8 == 0), OP_LINEAR (C % 8 == 0, ld % 8 == 0),
 // OP_SCALE (SE scale, gate vector in w; C % 8 == 0), OP_SE_GATE (grouped launches only),
-// OP_IM2COL (3 input channels; k in {3, 7}; stride in {1, 2}).  `h` is the host image of the `n` records
+// OP_IM2COL (3 input channels; k in {3, 7}; stride in {1, 2}), OP_PAD8 (3-channel image -> 8 channels with a
+// zero margin: k = margin left / top, Ho x Wo = padded size).  `h` is the host image of the `n` records
 // at device address `d` (it sizes the grid); with d == nullptr, n must be 1 and the record is passed by value.
 bool small_supported(int kind, const SmallEntry &e);
 cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int n, cudaStream_t st);
@@ -142,6 +148,8 @@ cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int
 // image dims and take the vectorised bf16 kernels; otherwise cudaErrorNotSupported and nothing is launched.
 constexpr int DW_ENTRY_BYTES = 256;
 cudaError_t launch_dw_group(const char *h_tbl, const char *d_tbl, int members, cudaStream_t st);
+// Stem weights for the window view: dst[f][r][px * 8 + c] = src[f][r][px][c] (px < k, c < 3), else 0; dst [K][k][64].
+cudaError_t launch_stem_window_weights(const void *src, void *dst, int K, int k, cudaStream_t st);
 // Stem weights as a GEMM operand: dst[f][kk] = src[f][kk] for kk < KK (the stored [K][R][R][3] row), 0 up to KKp.
 cudaError_t launch_stem_gemm_weights(const void *src, void *dst, int K, int KK, int KKp, cudaStream_t st);
 

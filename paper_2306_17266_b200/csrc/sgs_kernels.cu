@@ -880,11 +880,31 @@ __device__ __forceinline__ void im2col_body(const SmallEntry &e, int bx) {
     }
 }
 
+// 3-channel image -> [N][Ho][Wo][8] with the image at (k, k) and zeros elsewhere (margins and channels 3..7):
+// the input of the window-view stem.  A thread writes one padded pixel (16 bytes).
+__device__ __forceinline__ void pad8_body(const SmallEntry &e, int bx, int nbx) {
+    const int total = e.N * e.Ho * e.Wo;
+    const unsigned short *x = static_cast<const unsigned short *>(e.x);
+    uint4 *y = static_cast<uint4 *>(e.y);
+    for (int i = bx * blockDim.x + threadIdx.x; i < total; i += nbx * blockDim.x) {
+        const int wp = i % e.Wo, hp = (i / e.Wo) % e.Ho, n = i / (e.Wo * e.Ho);
+        const int h = hp - e.k, w = wp - e.k;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (h >= 0 && h < e.H && w >= 0 && w < e.W) {
+            const unsigned short *p = x + (((size_t)n * e.H + h) * e.W + w) * 3;
+            v.x = __ldg(p) | ((uint32_t)__ldg(p + 1) << 16);
+            v.y = __ldg(p + 2);
+        }
+        y[i] = v;
+    }
+}
+
 template <int KIND, int K, int ST> __device__ __forceinline__ void small_body(const SmallEntry &e, int bx, int nbx) {
     if constexpr (KIND == OP_MAXPOOL) maxpool_body(e, bx, nbx);
     else if constexpr (KIND == OP_GAP) gap_body(e, bx);
     else if constexpr (KIND == OP_LINEAR) linear_body(e, bx);
     else if constexpr (KIND == OP_SCALE) scale_body(e, bx, nbx);
+    else if constexpr (KIND == OP_PAD8) pad8_body(e, bx, nbx);
     else im2col_body<K, ST>(e, bx);
 }
 template <int KIND, int K, int ST> __global__ void __launch_bounds__(256) small_single_kernel(const SmallEntry e) {
@@ -950,6 +970,7 @@ bool small_supported(int kind, const SmallEntry &e) {
     case OP_GAP: return e.C % 8 == 0;
     case OP_SCALE: return e.C % 8 == 0 && al(e.w) && (long long)e.N * e.H * e.W * (e.C / 8) < (1ll << 31);
     case OP_SE_GATE: return e.w2 != nullptr;
+    case OP_PAD8: return (long long)e.N * e.Ho * e.Wo < (1ll << 31);
     case OP_LINEAR: return e.C % 8 == 0 && e.ld % 8 == 0 && al(e.w);
     case OP_IM2COL: return (e.k == 3 || e.k == 7) && (e.stride == 1 || e.stride == 2) && e.KKp % 8 == 0 && e.KKp >= e.k * e.k * 3 &&
                            e.W % 8 == 0 && e.W <= IM2COL_MAX_W && (long long)e.N * e.Ho < (1ll << 31) && (long long)e.Wo * (e.KKp / 8) < (1ll << 31);
@@ -963,6 +984,7 @@ static long long small_blocks(int kind, const SmallEntry &e) {
     case OP_MAXPOOL: return ((long long)e.N * e.Ho * e.Wo * (e.C / 8) + 255) / 256;
     case OP_GAP: return ((long long)e.N * (e.C / 8) * 32 + 255) / 256;
     case OP_SCALE: return ((long long)e.N * e.H * e.W * (e.C / 8) + 255) / 256;
+    case OP_PAD8: return ((long long)e.N * e.Ho * e.Wo + 255) / 256;
     case OP_LINEAR: return ((long long)e.N * e.K * 32 + 255) / 256;
     default: return (long long)e.N * e.Ho;  // patch matrix: one block per output row
     }
@@ -981,12 +1003,13 @@ cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int
     long long blocks = 1;
     for (int i = 0; i < n; i++) blocks = std::max(blocks, small_blocks(kind, h[i]));
     // the grid-stride kernels (max pool, SE scale) need not cover every element with a block of their own
-    if (kind == OP_MAXPOOL || kind == OP_SCALE) blocks = std::min<long long>(blocks, 148 * 16);
+    if (kind == OP_MAXPOOL || kind == OP_SCALE || kind == OP_PAD8) blocks = std::min<long long>(blocks, 148 * 16);
     const unsigned bx = (unsigned)blocks;
     switch (kind) {
     case OP_MAXPOOL: return launch_small_t<OP_MAXPOOL, 0, 0>(h, d, n, bx, st);
     case OP_GAP: return launch_small_t<OP_GAP, 0, 0>(h, d, n, bx, st);
     case OP_SCALE: return launch_small_t<OP_SCALE, 0, 0>(h, d, n, bx, st);
+    case OP_PAD8: return launch_small_t<OP_PAD8, 0, 0>(h, d, n, bx, st);
     case OP_SE_GATE: {
         if (!d) return cudaErrorInvalidValue;
         int nimg = 0, fl = 0;
@@ -1023,6 +1046,17 @@ __global__ void stem_gemm_weights_kernel(const __nv_bfloat16 *__restrict__ src, 
     if (i >= K * KKp) return;
     const int f = i / KKp, kk = i % KKp;
     dst[i] = kk < KK ? src[(size_t)f * KK + kk] : __float2bfloat16_rn(0.f);
+}
+__global__ void stem_window_weights_kernel(const __nv_bfloat16 *__restrict__ src, __nv_bfloat16 *__restrict__ dst, int K, int k) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;  // dst index [f][r][px][c8]
+    if (i >= K * k * 64) return;
+    const int c = i % 8, px = (i / 8) % 8, r = (i / 64) % k, f = i / (64 * k);
+    dst[i] = (px < k && c < 3) ? src[(((size_t)f * k + r) * k + px) * 3 + c] : __float2bfloat16_rn(0.f);
+}
+cudaError_t launch_stem_window_weights(const void *src, void *dst, int K, int k, cudaStream_t st) {
+    const int total = K * k * 64;
+    stem_window_weights_kernel<<<(total + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(src), static_cast<__nv_bfloat16 *>(dst), K, k);
+    return cudaGetLastError();
 }
 cudaError_t launch_stem_gemm_weights(const void *src, void *dst, int K, int KK, int KKp, cudaStream_t st) {
     const int total = K * KKp;

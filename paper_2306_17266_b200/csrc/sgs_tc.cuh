@@ -200,6 +200,7 @@ struct TcConvPlan {
     dim3 grid;
     int bn_tile = 128;   // filters per tile
     int swap = 0;        // grouped launches only: filters on the MMA's row side, all pixels on the column side
+    int kw = 1;          // taps along x (k for square kernels, 1 for the window view of a stem)
     size_t ws_elems = 0;
 };
 
