@@ -1271,8 +1271,9 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
     const auto host_t0 = std::chrono::steady_clock::now();
     std::vector<Plan *> plans((size_t)G);
     std::vector<std::vector<std::pair<int, int>>> buckets((size_t)n_ranks);  // per rank: (member, op index)
-    struct Launch { int rank; GroupLaunch *group; int small_kind; size_t off; int count; };  // group == nullptr && small_kind < 0: the bucket's ungrouped ops, per member
+    struct Launch { int rank; GroupLaunch *group; int small_kind; size_t off; int count; int rank2 = -1; };  // rank2: a second bucket merged into this launch;  // group == nullptr && small_kind < 0: the bucket's ungrouped ops, per member
     std::vector<Launch> launches;
+    std::vector<char> merged;  // per rank: its bucket went into the previous bucket's launch
     for (int wv = 0; wv < n_waves && rc == SGS_OK; wv++) {
         const int ci = wv % W, q0 = wv * G, members = std::min(G, n_queries - q0);
         auto tick = [](std::chrono::steady_clock::time_point &t0) {
@@ -1337,10 +1338,12 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             g->reset(cx.d_tbl + off);
             return g;
         };
+        merged.assign((size_t)n_ranks, 0);
         for (int r = 0; r < n_ranks; r++) {
             const auto &b = buckets[(size_t)r];
-            if (b.empty()) continue;
+            if (b.empty() || merged[(size_t)r]) continue;
             GroupLaunch *g = nullptr;
+            const size_t first_launch = launches.size();
             for (const auto &mo : b) {
                 Plan *pl = plans[mo.first];
                 const Op &op = pl->ops[(size_t)mo.second];
@@ -1350,6 +1353,49 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                 a.layer = op.layer;
                 g->add(cx.h_tbl + off, *op.tc, a);
                 off += TC_GROUP_ENTRY_BYTES;
+            }
+            // Two consecutive convolution layers that do not depend on each other (a block's projection
+            // shortcut and its first convolution both read the block input) share one launch when they fit.
+            if (g && launches.size() == first_launch + 1) {
+                int r2 = r + 1;
+                while (r2 < n_ranks && buckets[(size_t)r2].empty()) r2++;
+                if (r2 < n_ranks) {
+                    auto all_tc = [&](const std::vector<std::pair<int, int>> &bb) {
+                        for (const auto &mo : bb) {
+                            const Op &op = plans[mo.first]->ops[(size_t)mo.second];
+                            if (op.type != OP_CONV || op.impl != 1) return false;
+                        }
+                        return true;
+                    };
+                    const auto &b2 = buckets[(size_t)r2];
+                    bool ok = all_tc(b) && all_tc(b2) && g->members() + (int)b2.size() <= TC_GROUP_MAX_ENTRIES;
+                    for (const auto &m2 : b2) {
+                        if (!ok) break;
+                        const Op &o2 = plans[m2.first]->ops[(size_t)m2.second];
+                        for (const auto &m1 : b) {
+                            if (m1.first != m2.first) continue;
+                            const Op &o1 = plans[m1.first]->ops[(size_t)m1.second];
+                            // same member: no read-after-write, write-after-read or write-after-write between them
+                            if (o2.in == o1.out || o2.res == o1.out || o2.out == o1.out || o2.out == o1.in || (o1.res >= 0 && o2.out == o1.res)) ok = false;
+                        }
+                    }
+                    if (ok) {
+                        // (fits() also bounds the tensor maps; checked entry by entry, undone as a whole is not
+                        // possible, so test the worst case first: 5 maps per member)
+                        ok = g->members() + (int)b2.size() <= TC_GROUP_MAX_ENTRIES && g->maps() + 5 * (int)b2.size() <= TC_GROUP_MAPS_LARGE;
+                    }
+                    if (ok) {
+                        for (const auto &mo : b2) {
+                            const Op &op = plans[mo.first]->ops[(size_t)mo.second];
+                            ConvArgs a = op.conv;
+                            a.layer = op.layer;
+                            g->add(cx.h_tbl + off, *op.tc, a);
+                            off += TC_GROUP_ENTRY_BYTES;
+                        }
+                        launches.back().rank2 = r2;
+                        merged[(size_t)r2] = 1;
+                    }
+                }
             }
             // max pool / average pool / linear / patch matrix: one launch over the members when every
             // member's op has the vectorised form; the remaining ops run member by member
@@ -1446,6 +1492,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                 // (a bucket split over several launches books its whole cost on each: buckets of more than
                 // 64 members or 248 tensor maps do not occur while profiling waves of <= 64)
                 bucket_cost(L.rank, true, &pb, &pf);
+                if (L.rank2 >= 0) { double b2 = 0, f2 = 0; bucket_cost(L.rank2, true, &b2, &f2); pb += b2; pf += f2; }
                 if ((rc = prof_begin(0, pb, pf)) != SGS_OK) break;
                 CU(L.group->launch(net->cache_tbl, net->sms, ws));
                 if ((rc = prof_end()) != SGS_OK) break;

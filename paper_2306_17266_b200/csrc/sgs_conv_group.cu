@@ -466,6 +466,7 @@ void GroupLaunch::reset(const void *d_entries) {
     impl->prm.total_tiles = 0;
 }
 int GroupLaunch::members() const { return impl->prm.n_entries; }
+int GroupLaunch::maps() const { return impl->n_maps; }
 int GroupLaunch::tiles() const { return impl->prm.total_tiles; }
 
 bool GroupLaunch::fits(const TcConvPlan &pl) const {

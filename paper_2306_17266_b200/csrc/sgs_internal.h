@@ -182,6 +182,7 @@ public:
     // Adds a member: writes its record to host_entry (the host image of the next device record).
     void add(void *host_entry, const TcConvPlan &p, const ConvArgs &a);
     int members() const;
+    int maps() const;                       // tensor maps used so far
     int tiles() const;
     cudaError_t launch(const int *cache_tbl, int sms, cudaStream_t st);
 private:
