@@ -218,3 +218,78 @@ def layer_gap(x) -> np.ndarray:
 
 def bf16_round(v: float) -> float:
     return float(lib().orc_bf16_round(v))
+
+
+# ------------------------------------------------------------------------------------------------
+# Scheduler's caching decision (paper Section 3.3 "Amortizing Caching Choices", "Predicting the Next
+# SubGraph", Algorithm 1's cache branch, Section 3.2 for the candidate set S).  Plain loops on the
+# (K, C, k) encodings; test infrastructure only.
+# ------------------------------------------------------------------------------------------------
+def layer_weights(enc: np.ndarray) -> np.ndarray:
+    """Weights of every layer of an encoding: K * C * k * k."""
+    e = np.asarray(enc, dtype=np.int64).reshape(-1, 3)
+    return e[:, 0] * e[:, 1] * e[:, 2] * e[:, 2]
+
+
+def clip_to_budget(enc: np.ndarray, budget_weights: int) -> np.ndarray:
+    """A cacheable SubGraph of at most `budget_weights` weights (Section 3.2: SubGraphs in S have about the
+    cache's size): walking the layers in network order, a layer's box is kept if it still fits beside the
+    boxes kept so far, else the layer is left out."""
+    e = np.array(enc, dtype=np.int32).reshape(-1, 3).copy()
+    used = 0
+    for i, w in enumerate(layer_weights(e)):
+        if used + int(w) > budget_weights:
+            e[i, :] = 0
+        else:
+            used += int(w)
+    return e.reshape(np.asarray(enc).shape)
+
+
+def nearest_candidate(window, candidates) -> int:
+    """Index j of the candidate SubGraph closest to the running average of the SubNets in `window`
+    (Algorithm 1: CacheState = argmin_j Dist(G_j, AvgNet); Dist = Euclidean distance on the (K_i, C_i)
+    vector encoding of Section 3.3).  With Q = len(window) and S = the element-wise sum over the window,
+    Dist^2 * Q^2 = sum_i (Q * G_ji - S_i)^2: compared exactly in integers.  Ties go to the lowest index."""
+    q = len(window)
+    s = np.zeros_like(np.asarray(window[0], dtype=np.int64).reshape(-1, 3))
+    for e in window:
+        s = s + np.asarray(e, dtype=np.int64).reshape(-1, 3)
+    best, best_d = -1, None
+    for j, g in enumerate(candidates):
+        g3 = np.asarray(g, dtype=np.int64).reshape(-1, 3)
+        d = 0
+        for i in range(g3.shape[0]):
+            for c in range(2):  # K and C entries
+                t = q * int(g3[i, c]) - int(s[i, c])
+                d += t * t
+        if best_d is None or d < best_d:
+            best, best_d = j, d
+    return best
+
+
+def sched_stream(encs, candidates, q: int):
+    """Serve the SubNets `encs` in order; after every q-th query the cached SubGraph becomes the candidate
+    nearest to the average of the last q served SubNets (Algorithm 1).  Query t is accounted against the
+    SubGraph cached before it is served (none before the first decision).  Returns per-query hit ratios
+    (Appendix A.4), missed weights, and the list of choices (one per decision)."""
+    hits, missed, choices = [], [], []
+    window, g, since = [], None, 0
+    candidates = [np.ascontiguousarray(c, dtype=np.int32).reshape(-1, 3) for c in candidates]
+    for e in encs:
+        e = np.ascontiguousarray(e, dtype=np.int32).reshape(-1, 3)
+        if g is None:
+            hits.append(0.0)
+            missed.append(encoding_weights(e))
+        else:
+            hits.append(hit_ratio(e, g))
+            missed.append(encoding_weights(e) - encoding_weights(intersect(e, g)))
+        window.append(e)
+        if len(window) > q:
+            window.pop(0)
+        since += 1
+        if since >= q:
+            since = 0
+            j = nearest_candidate(window, candidates)
+            choices.append(j)
+            g = candidates[j]
+    return hits, missed, choices

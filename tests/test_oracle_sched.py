@@ -1,0 +1,77 @@
+"""CPU pins of the checker's scheduler functions (Algorithm 1's caching decision, Section 3.3): hand-computed
+vectors, closed forms and special cases that fix the running average, the distance, tie handling, the
+budget clipping and the timing of the decisions."""
+import numpy as np
+
+import oracle
+
+
+def enc(*kc):
+    """Encoding from (K, C) pairs with 1x1 kernels."""
+    return np.array([v for k, c in kc for v in (k, c, 1)], dtype=np.int32).reshape(-1, 3)
+
+
+def test_nearest_candidate_on_hand_computed_vectors():
+    # window mean = ((4+8)/2, 2) = (6, 2); distances^2: (8,2) -> 4, (6,2) -> 0, (5,4) -> 1 + 4 = 5
+    window = [enc((4, 2)), enc((8, 2))]
+    cands = [enc((8, 2)), enc((6, 2)), enc((5, 4))]
+    assert oracle.nearest_candidate(window, cands) == 1
+    # a single-query window: the nearest candidate to the SubNet itself
+    assert oracle.nearest_candidate([enc((5, 3))], cands) == 2  # (5,4): 1; (6,2): 1+1 = 2; (8,2): 9+1 = 10
+    # ties go to the lowest index; the kernel-size entry takes no part in the distance
+    a, b = enc((7, 2)), enc((5, 2))
+    assert oracle.nearest_candidate([enc((6, 2))], [a, b]) == 0
+    assert oracle.nearest_candidate([enc((6, 2))], [b, a]) == 0
+    g3 = np.array([[6, 2, 3]], dtype=np.int32)  # same (K, C), other kernel size
+    assert oracle.nearest_candidate([enc((6, 2))], [a, g3]) == 1
+
+
+def test_average_keeps_what_intersection_loses():
+    # Section 3.3: a filter count used by most (not all) SubNets of the window still pulls the choice.
+    # Window: three SubNets with K = 8 and one with K = 2: intersection has K = 2, the mean K = 6.5
+    window = [enc((8, 4))] * 3 + [enc((2, 4))]
+    cands = [enc((2, 4)), enc((6, 4)), enc((8, 4))]
+    assert oracle.nearest_candidate(window, cands) == 1  # |6-6.5| < |8-6.5| < |2-6.5|
+    inter = window[0]
+    for e in window[1:]:
+        inter = oracle.intersect(inter, e)
+    assert list(inter[0, :2]) == [2, 4]
+
+
+def test_identical_subnets_choose_themselves():
+    e = enc((16, 8), (32, 16), (10, 32))
+    others = [enc((8, 8), (16, 8), (10, 16)), enc((16, 16), (32, 32), (10, 64))]
+    for pos in range(3):
+        cands = others[:pos] + [e] + others[pos:]
+        hits, missed, choices = oracle.sched_stream([e] * 6, cands, 2)
+        assert choices == [pos] * 3
+        assert hits[:2] == [0.0, 0.0] and missed[:2] == [oracle.encoding_weights(e)] * 2  # nothing cached before the first decision
+        assert hits[2:] == [1.0] * 4 and missed[2:] == [0] * 4
+
+
+def test_clip_to_budget_rule():
+    e = np.array([5, 2, 1, 5, 4, 1, 5, 1, 1], dtype=np.int32)  # layer weights 10, 20, 5
+    assert list(oracle.layer_weights(e)) == [10, 20, 5]
+    assert list(oracle.clip_to_budget(e, 100)) == list(e)
+    assert list(oracle.clip_to_budget(e, 16)) == [5, 2, 1, 0, 0, 0, 5, 1, 1]   # 10 kept, 20 does not fit, 5 fits
+    assert list(oracle.clip_to_budget(e, 9)) == [0, 0, 0, 0, 0, 0, 5, 1, 1]
+    assert list(oracle.clip_to_budget(e, 30)) == [5, 2, 1, 5, 4, 1, 0, 0, 0]
+    k3 = np.array([2, 2, 3], dtype=np.int32)  # 3x3 kernel: 2*2*9 = 36 weights
+    assert list(oracle.layer_weights(k3)) == [36] and list(oracle.clip_to_budget(k3, 35)) == [0, 0, 0]
+
+
+def test_decisions_every_q_queries_use_the_last_q_subnets():
+    small, big = enc((4, 4)), enc((16, 4))
+    cands = [small, big]
+    stream = [small, small, big, big, big, small]
+    hits, missed, choices = oracle.sched_stream(stream, cands, 2)
+    # decisions after queries 1, 3, 5 from windows (s,s), (b,b), (b,s): means K = 4, 16, 10 -> small, big, tie -> lowest index
+    assert choices == [0, 1, 0]
+    # query 2 (big) is served with `small` cached: shared K = 4 of 16, C = 4 of 4
+    assert abs(hits[2] - np.sqrt(4 * 4 + 4 * 4) / np.sqrt(16 * 16 + 4 * 4)) < 1e-12
+    assert missed[2] == 16 * 4 - 4 * 4
+    # queries 4 (big) and 5 (small) with `big` cached: everything shared
+    assert hits[4] == 1.0 and hits[5] == 1.0 and missed[4] == 0 and missed[5] == 0
+    # q = 1: the cache follows the previous query
+    _, _, ch1 = oracle.sched_stream(stream, cands, 1)
+    assert ch1 == [0, 0, 1, 1, 1, 0]
