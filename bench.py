@@ -217,6 +217,33 @@ def run_suite(args):
                     "launches_before_measured_part": skip, "launches_in_measured_part": t["launches"],
                     "config": {"batch": args.batch, "cache": args.cache, "window_q": args.window, "weights_evict_first": args.evict_first,
                                "note": "load-time kernels precede the warm-up launches; count them with the profiler's launch list"}})
+    elif args.suite == "sched":
+        # caching decision of Algorithm 1 (nearest candidate SubGraph to the running average) beside the
+        # intersection of the window, over the window length Q, the size of the candidate set and the budget
+        net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
+        n = args.queries
+        cfgs = wl.markov_stream(n, seed=4)
+        rows = []
+        warm = sgs.StreamOpts(cache_enabled=0, window_q=4, record_latency=0, concurrency=args.concurrency, wave=args.wave)
+        _stream_pool(net, sgs, torch, cfgs, 1, 224, warm, stream, n, wl.RESNET)
+        for budget_mb in (0, 24):
+            for n_cand in (0, 16, 64, 256):
+                net.cache_set_candidates(wl.candidate_cfgs(wl.RESNET, n_cand, seed=6) if n_cand else [])
+                for q in (1, 2, 4, 8, 16):
+                    opts = sgs.StreamOpts(cache_enabled=1, window_q=q, cache_budget_bytes=budget_mb << 20, record_latency=0,
+                                          concurrency=args.concurrency, wave=args.wave,
+                                          policy=sgs.SGS_POLICY_AVGNET if n_cand else sgs.SGS_POLICY_INTERSECTION)
+                    t = _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, n, wl.RESNET)
+                    rows.append({"policy": "avgnet" if n_cand else "intersection", "candidates": n_cand, "window_q": q,
+                                 "budget_mb": net.cache_stats().budget_bytes / 2**20, "hit_ratio": t["hit"] / t["q"],
+                                 "weight_mb_per_query": t["wbytes"] / t["q"] / 1e6, "hbm_weight_mb_per_query": t["miss"] / t["q"] / 1e6,
+                                 "queries_per_s": t["q"] / (t["ms"] * 1e-3)})
+        net.cache_set_candidates([])
+        best = max(rows, key=lambda r: r["hit_ratio"])
+        out.update({"metric": "cache_hit_ratio", "unit": "mean ||SN ∩ G|| / ||SN|| (analytic)", "value": best["hit_ratio"], "best": best, "rows": rows,
+                    "config": {"workload": f"SGS locality stream on the ResNet-50-shaped SuperNet: {n} queries, Markov chain of configs (p=0.9 one stage's depth or width changes), seed 4, 224x224, batch 1",
+                               "candidates": "smallest and largest SubNet plus uniform draws (seed 6), each clipped to the budget",
+                               "execution": f"waves of {args.wave}, {args.concurrency} in flight" if args.wave > 0 else f"one stream per query, {args.concurrency} in flight"}})
     elif args.suite == "mbv3":
         net = sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16)
         cfgs = wl.uniform_stream(wl.MBV3, args.queries, seed=3)
@@ -243,8 +270,8 @@ def run_suite(args):
 # summarised in profiles/conv_group_wave32_resnet_b1.md.  Valid only for the kernel source it was taken
 # on: once that file changes the figure is reported as null.
 NCU_TRAFFIC = {
-    "kernel_source_sha256_16": "a80d10f62284941f",
-    "bytes_per_launch": 14650000,
+    "kernel_source_sha256_16": "ed0fba9bebd59063",
+    "bytes_per_launch": 15260000,
     "note": "ncu flushes the caches before every launch: cold-cache reads; writes that still sit in L2 when the kernel ends are not counted",
 }
 
@@ -277,7 +304,7 @@ def main():
     ap.add_argument("--concurrency", type=int, default=None, help="waves in flight (default 4), or with --wave 0 queries in flight (default 16)")
     ap.add_argument("--batch", type=int, default=1, help="images per query (sgs-probe)")
     ap.add_argument("--evict-first", type=int, default=0, help="with --cache 0: mark weight loads evict-first (sgs-probe)")
-    ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3"],
+    ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3", "sched"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()
     if args.suite in ("sgs", "sgs-probe"):

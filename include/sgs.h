@@ -75,6 +75,8 @@ typedef struct {
     int kernel[SGS_MAX_STAGES][SGS_MAX_BLOCKS];
 } sgs_subnet_cfg_t;
 
+enum { SGS_POLICY_INTERSECTION = 0, SGS_POLICY_AVGNET = 1 };
+
 /* Options of sgs_stream_run. */
 typedef struct {
     int cache_enabled;  /* 1: keep the SubGraph shared by recent queries resident in L2 */
@@ -102,6 +104,10 @@ typedef struct {
                            starts and ends with its wave (that is its recorded latency).  The cached
                            SubGraph is still re-chosen in stream order; the L2 hints of a wave use the
                            choice in force when the wave was issued. */
+    int policy;         /* how the cached SubGraph is chosen every window_q queries:
+                           SGS_POLICY_INTERSECTION (0): the SubGraph common to the last window_q SubNets;
+                           SGS_POLICY_AVGNET (1): Algorithm 1 - the candidate SubGraph (sgs_cache_set_candidates)
+                           nearest to the running average of the last window_q SubNets' encodings */
 } sgs_stream_opts_t;
 
 /* Results of sgs_stream_run (all host-side; filled after the stream has been synchronised). */
@@ -132,6 +138,10 @@ typedef struct {
     size_t cached_subgraph_bytes;  /* weight bytes of the SubGraph currently marked resident */
     size_t supernet_bytes;         /* device bytes of all stored weights */
     size_t device_bytes_allocated; /* every device byte the handle owns (weights + workspaces) */
+    int policy;                    /* SGS_POLICY_* in force */
+    int n_candidates;              /* size of the candidate set S */
+    int decisions;                 /* caching decisions taken since the cache was last reset */
+    int last_choice;               /* index into S of the last AvgNet decision; -1 = none yet */
 } sgs_cache_stats_t;
 
 /*
@@ -195,6 +205,23 @@ sgs_status_t sgs_stream_run_host(sgs_supernet_t *net, int n_queries, const sgs_s
  * budget_bytes 0 = device maximum.  window_q >= 1. */
 sgs_status_t sgs_cache_configure(sgs_supernet_t *net, int enabled, size_t budget_bytes, int window_q);
 sgs_status_t sgs_cache_stats(const sgs_supernet_t *net, sgs_cache_stats_t *out);
+
+/*
+ * sgs_cache_set_candidates - the set S of cacheable SubGraphs the scheduler chooses from (Section 3.2;
+ * Algorithm 1's G_j).  cfgs: host array of n SubNet configs; candidate j is the vector encoding
+ * (Section 3.3) of cfgs[j], with layers dropped, in network order, once the byte budget of the cache
+ * is used up (re-applied whenever the budget changes).  The configs are copied.  n = 0 removes the set
+ * and returns to SGS_POLICY_INTERSECTION.  Host-only; takes effect at the next caching decision.
+ * Errors: SGS_EINVAL, SGS_ECONFIG (a config outside the elastic sets; the old set is kept).
+ *
+ * sgs_cache_set_policy - policy of the cache used by sgs_subnet_run (sgs_stream_run takes it from its
+ * options).  SGS_POLICY_AVGNET: after every window_q queries, AvgNet = element-wise mean of the last
+ * window_q encodings and the cached SubGraph becomes argmin_j Dist(G_j, AvgNet), Dist = Euclidean
+ * distance over the (K_i, C_i) entries, compared exactly, ties to the lowest j.  SGS_EINVAL without a
+ * candidate set.
+ */
+sgs_status_t sgs_cache_set_candidates(sgs_supernet_t *net, const sgs_subnet_cfg_t *cfgs, int n);
+sgs_status_t sgs_cache_set_policy(sgs_supernet_t *net, int policy);
 
 /*
  * Vector encoding of a SubNet (Section 3.3): for every stored layer i, out[3i] = K_i (filters),

@@ -16,6 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("SGS_LIB") or os.path.join(_HERE, "libsgs.so")  # SGS_LIB: use another build of the library
 
 SGS_OK, SGS_EINVAL, SGS_ECONFIG, SGS_ENOMEM, SGS_ECUDA, SGS_ETIMEOUT, SGS_EUNSUPPORTED = range(7)
+SGS_POLICY_INTERSECTION, SGS_POLICY_AVGNET = 0, 1
 SGS_F32, SGS_BF16 = 0, 1
 STATUS_NAMES = ["SGS_OK", "SGS_EINVAL", "SGS_ECONFIG", "SGS_ENOMEM", "SGS_ECUDA", "SGS_ETIMEOUT", "SGS_EUNSUPPORTED"]
 
@@ -23,7 +24,7 @@ EXPORTS = [
     "sgs_supernet_load", "sgs_subnet_validate", "sgs_subnet_run", "sgs_stream_run", "sgs_stream_run_host",
     "sgs_cache_configure", "sgs_cache_stats", "sgs_num_layers", "sgs_subnet_encode", "sgs_subnet_cost",
     "sgs_set_option", "sgs_get_counter", "sgs_last_error", "sgs_supernet_free", "sgs_conv2d_sliced", "sgs_device_status",
-    "sgs_profile_read", "sgs_conv2d_sliced_static",
+    "sgs_profile_read", "sgs_conv2d_sliced_static", "sgs_cache_set_candidates", "sgs_cache_set_policy",
 ]
 
 
@@ -35,7 +36,7 @@ class ConvDesc(ctypes.Structure):
 class StreamOpts(ctypes.Structure):
     _fields_ = [("cache_enabled", ctypes.c_int), ("window_q", ctypes.c_int), ("cache_budget_bytes", ctypes.c_size_t),
                 ("use_graphs", ctypes.c_int), ("record_latency", ctypes.c_int), ("weights_evict_first", ctypes.c_int),
-                ("concurrency", ctypes.c_int), ("wave", ctypes.c_int)]
+                ("concurrency", ctypes.c_int), ("wave", ctypes.c_int), ("policy", ctypes.c_int)]
 
 
 class StreamStats(ctypes.Structure):
@@ -54,7 +55,8 @@ class CacheStats(ctypes.Structure):
     _fields_ = [("enabled", ctypes.c_int), ("window_q", ctypes.c_int), ("budget_bytes", ctypes.c_size_t),
                 ("l2_bytes", ctypes.c_size_t), ("persisting_l2_max", ctypes.c_size_t), ("access_window_max", ctypes.c_size_t),
                 ("cached_subgraph_bytes", ctypes.c_size_t), ("supernet_bytes", ctypes.c_size_t),
-                ("device_bytes_allocated", ctypes.c_size_t)]
+                ("device_bytes_allocated", ctypes.c_size_t), ("policy", ctypes.c_int), ("n_candidates", ctypes.c_int),
+                ("decisions", ctypes.c_int), ("last_choice", ctypes.c_int)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -84,6 +86,8 @@ def lib():
         L.sgs_stream_run_host.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, vp, vp]
         L.sgs_cache_configure.argtypes = [vp, ci, cs, ci]
         L.sgs_cache_stats.argtypes = [vp, vp]
+        L.sgs_cache_set_candidates.argtypes = [vp, vp, ci]
+        L.sgs_cache_set_policy.argtypes = [vp, ci]
         L.sgs_num_layers.argtypes = [vp]
         L.sgs_subnet_encode.argtypes = [vp, vp, vp]
         L.sgs_subnet_cost.argtypes = [vp, vp, ci, ci, vp, vp, vp]
@@ -178,6 +182,14 @@ class SuperNet:
 
     def cache_configure(self, enabled: bool, budget_bytes: int = 0, window_q: int = 4):
         self._check(lib().sgs_cache_configure(self._h, int(enabled), budget_bytes, window_q))
+
+    def cache_set_candidates(self, cfgs: Sequence[SubnetCfg]):
+        arr = cfgs if isinstance(cfgs, ctypes.Array) else (cfg_array(cfgs) if len(cfgs) else None)
+        self._check(lib().sgs_cache_set_candidates(self._h, ctypes.addressof(arr) if arr is not None else None,
+                                                   len(arr) if arr is not None else 0))
+
+    def cache_set_policy(self, policy: int):
+        self._check(lib().sgs_cache_set_policy(self._h, policy))
 
     def cache_stats(self) -> CacheStats:
         s = CacheStats()

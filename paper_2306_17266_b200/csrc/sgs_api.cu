@@ -139,6 +139,10 @@ struct CacheState {
     int epoch = 0;                        // bumped whenever G changes
     int since_update = 0;
     int evict_first_when_off = 0;
+    int policy = 0;                       // 0: intersection of the window; 1: candidate nearest to the window's average
+    std::vector<std::vector<int>> cand_raw, cand;  // candidate SubGraph encodings as given / clipped to the budget
+    std::vector<size_t> cand_bytes;
+    int decisions = 0, last_choice = -1;
 };
 
 }  // namespace
@@ -943,18 +947,61 @@ size_t layer_box_bytes(const sgs_supernet *net, int li, int K, int C, int k) {
 // G = element-wise minimum of the encodings in the window (the exact intersection of those SubNets,
 // because every slice is a prefix / centred window), kept layer by layer in network order while it
 // fits the byte budget.
-void recompute_cached_subgraph(sgs_supernet *net) {
-    CacheState &cs = net->cache;
-    if (cs.window.empty()) return;
-    std::vector<int> g = cs.window.front();
-    for (const auto &e : cs.window)
-        for (size_t i = 0; i < g.size(); i++) g[i] = std::min(g[i], e[i]);
+// Keeps the layers of `g` in network order while they fit the byte budget; returns the bytes kept.
+size_t clip_to_budget(const sgs_supernet *net, std::vector<int> &g, size_t budget) {
     size_t used = 0;
     for (size_t li = 0; li < net->layers.size(); li++) {
         size_t b = layer_box_bytes(net, (int)li, g[3 * li], g[3 * li + 1], g[3 * li + 2]);
-        if (used + b > cs.budget) { g[3 * li] = g[3 * li + 1] = g[3 * li + 2] = 0; continue; }
+        if (used + b > budget) { g[3 * li] = g[3 * li + 1] = g[3 * li + 2] = 0; continue; }
         used += b;
     }
+    return used;
+}
+
+void clip_candidates(sgs_supernet *net) {
+    CacheState &cs = net->cache;
+    cs.cand = cs.cand_raw;
+    cs.cand_bytes.assign(cs.cand.size(), 0);
+    for (size_t j = 0; j < cs.cand.size(); j++) cs.cand_bytes[j] = clip_to_budget(net, cs.cand[j], cs.budget);
+}
+
+// Algorithm 1's caching decision: AvgNet = mean of the window's encodings; the cached SubGraph becomes
+// the candidate G_j with the smallest Euclidean distance to it on the (K_i, C_i) entries (Section 3.3).
+// With Q = window length and S = element-wise sum, Q^2 * Dist^2 = sum_i (Q * G_ji - S_i)^2 is compared
+// exactly in 64-bit integers; ties go to the lowest index.
+void choose_nearest_candidate(sgs_supernet *net) {
+    CacheState &cs = net->cache;
+    const long long Q = (long long)cs.window.size();
+    const size_t n = cs.window.front().size();
+    std::vector<long long> S(n, 0);
+    for (const auto &e : cs.window)
+        for (size_t i = 0; i < n; i++) S[i] += e[i];
+    int best = -1;
+    unsigned long long best_d = 0;
+    for (size_t j = 0; j < cs.cand.size(); j++) {
+        unsigned long long d = 0;
+        for (size_t i = 0; i < n; i++) {
+            if (i % 3 == 2) continue;  // the kernel-size entry takes no part in the distance
+            long long t = Q * cs.cand[j][i] - S[i];
+            d += (unsigned long long)(t * t);
+        }
+        if (best < 0 || d < best_d) { best = (int)j; best_d = d; }
+    }
+    cs.decisions++;
+    cs.last_choice = best;
+    if (cs.cand[best] != cs.G) { cs.G = cs.cand[best]; cs.epoch++; }
+    cs.G_bytes = cs.cand_bytes[best];
+}
+
+void recompute_cached_subgraph(sgs_supernet *net) {
+    CacheState &cs = net->cache;
+    if (cs.window.empty()) return;
+    if (cs.policy == 1 && !cs.cand.empty()) { choose_nearest_candidate(net); return; }
+    std::vector<int> g = cs.window.front();
+    for (const auto &e : cs.window)
+        for (size_t i = 0; i < g.size(); i++) g[i] = std::min(g[i], e[i]);
+    size_t used = clip_to_budget(net, g, cs.budget);
+    cs.decisions++;
     if (g != cs.G) { cs.G = std::move(g); cs.epoch++; }
     cs.G_bytes = used;
 }
@@ -1004,7 +1051,10 @@ void cache_reset(sgs_supernet *net, bool enabled, size_t budget, int window_q) {
     cs.G.clear();
     cs.G_bytes = 0;
     cs.since_update = 0;
+    cs.decisions = 0;
+    cs.last_choice = -1;
     cs.epoch++;
+    clip_candidates(net);
 }
 
 }  // namespace
@@ -1624,12 +1674,16 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
     if (!guard.ok) return fail(net, SGS_ECUDA, "cudaSetDevice failed");
     sgs_stream_opts_t o;
     if (opts) o = *opts;
-    else { o.cache_enabled = 1; o.window_q = 4; o.cache_budget_bytes = 0; o.use_graphs = 1; o.record_latency = 1; o.weights_evict_first = 0; o.concurrency = 1; o.wave = 0; }
+    else { o.cache_enabled = 1; o.window_q = 4; o.cache_budget_bytes = 0; o.use_graphs = 1; o.record_latency = 1; o.weights_evict_first = 0; o.concurrency = 1; o.wave = 0; o.policy = 0; }
     if (o.window_q < 1) return fail(net, SGS_EINVAL, "window_q must be >= 1");
     if (o.concurrency < 0 || o.concurrency > 16) return fail(net, SGS_EINVAL, "concurrency must be in [0, 16]");
     for (int t = 0; t < n_queries; t++)
         if (!cfg_valid(net, &cfgs[t])) return fail(net, SGS_ECONFIG, "query " + std::to_string(t) + ": config outside the elastic sets");
     if (o.wave < 0) return fail(net, SGS_EINVAL, "wave must be >= 0");
+    if (o.policy != SGS_POLICY_INTERSECTION && o.policy != SGS_POLICY_AVGNET) return fail(net, SGS_EINVAL, "unknown cache policy");
+    if (o.policy == SGS_POLICY_AVGNET && o.cache_enabled && net->cache.cand_raw.empty())
+        return fail(net, SGS_EINVAL, "the AvgNet policy needs a candidate set (sgs_cache_set_candidates)");
+    net->cache.policy = o.policy;
     cache_reset(net, o.cache_enabled != 0, o.cache_budget_bytes, o.window_q);
     net->cache.evict_first_when_off = (!o.cache_enabled && o.weights_evict_first) ? 1 : 0;
     if (o.wave > 0 && n_queries > 0 && net->dtype == SGS_BF16 && tc_available() && !net->force_plain)
@@ -1790,6 +1844,28 @@ sgs_status_t sgs_cache_configure(sgs_supernet_t *net, int enabled, size_t budget
     return SGS_OK;
 }
 
+sgs_status_t sgs_cache_set_candidates(sgs_supernet_t *net, const sgs_subnet_cfg_t *cfgs, int n) {
+    if (!net || n < 0 || (n && !cfgs)) return SGS_EINVAL;
+    std::vector<std::vector<int>> raw;
+    for (int j = 0; j < n; j++) {
+        if (!cfg_valid(net, &cfgs[j])) return fail(net, SGS_ECONFIG, "candidate " + std::to_string(j) + ": config outside the elastic sets");
+        raw.push_back(encoding_of(slices_for(net, &cfgs[j])));
+    }
+    net->cache.cand_raw = std::move(raw);
+    clip_candidates(net);
+    if (n == 0) net->cache.policy = 0;
+    return SGS_OK;
+}
+
+sgs_status_t sgs_cache_set_policy(sgs_supernet_t *net, int policy) {
+    if (!net) return SGS_EINVAL;
+    if (policy != SGS_POLICY_INTERSECTION && policy != SGS_POLICY_AVGNET) return fail(net, SGS_EINVAL, "unknown cache policy");
+    if (policy == SGS_POLICY_AVGNET && net->cache.cand_raw.empty())
+        return fail(net, SGS_EINVAL, "the AvgNet policy needs a candidate set (sgs_cache_set_candidates)");
+    net->cache.policy = policy;
+    return SGS_OK;
+}
+
 sgs_status_t sgs_cache_stats(const sgs_supernet_t *net, sgs_cache_stats_t *out) {
     if (!net || !out) return SGS_EINVAL;
     std::memset(out, 0, sizeof(*out));
@@ -1802,6 +1878,10 @@ sgs_status_t sgs_cache_stats(const sgs_supernet_t *net, sgs_cache_stats_t *out) 
     out->cached_subgraph_bytes = net->cache.G_bytes;
     out->supernet_bytes = net->weight_arena_bytes;
     out->device_bytes_allocated = net->device_bytes;
+    out->policy = net->cache.policy;
+    out->n_candidates = (int)net->cache.cand_raw.size();
+    out->decisions = net->cache.decisions;
+    out->last_choice = net->cache.last_choice;
     return SGS_OK;
 }
 

@@ -339,6 +339,16 @@ def uniform_stream(family: int, n: int, seed: int) -> List[SubnetCfg]:
     return [sample_cfg(family, rng) for _ in range(n)]
 
 
+def candidate_cfgs(family: int, n: int, seed: int) -> List[SubnetCfg]:
+    """A set of n SubNet configs whose encodings serve as the scheduler's cacheable SubGraphs (Section 3.2):
+    the smallest and the largest SubNet, then seeded uniform draws."""
+    rng = np.random.default_rng(seed)
+    out = [extreme_cfg(family, False), extreme_cfg(family, True)][:n]
+    while len(out) < n:
+        out.append(sample_cfg(family, rng))
+    return out
+
+
 def copy_cfg(c: SubnetCfg) -> SubnetCfg:
     d = SubnetCfg()
     ctypes.memmove(ctypes.byref(d), ctypes.byref(c), ctypes.sizeof(SubnetCfg))
