@@ -293,3 +293,46 @@ def sched_stream(encs, candidates, q: int):
             choices.append(j)
             g = candidates[j]
     return hits, missed, choices
+
+
+STRICT_ACCURACY, STRICT_LATENCY = 0, 1
+
+
+def select_subnet(policy: int, a_t: float, l_t: float, accuracy, latency_col) -> int:
+    """Per-query SubNet selection of Algorithm 1 (Section 3.3) for the cache state whose latency column is
+    `latency_col`.  STRICT_ACCURACY: the fastest SubNet among those with accuracy >= A_t.  STRICT_LATENCY: the
+    most accurate SubNet among those with latency <= L_t.  Where the paper is silent: an empty feasible set
+    falls back to the most accurate SubNet (STRICT_ACCURACY) or the fastest one (STRICT_LATENCY); ties are
+    broken by the other quantity (higher accuracy / lower latency), then by the lowest index."""
+    n = len(accuracy)
+    by_latency = lambda i: (latency_col[i], -accuracy[i], i)
+    by_accuracy = lambda i: (-accuracy[i], latency_col[i], i)
+    if policy == STRICT_ACCURACY:
+        feasible = [i for i in range(n) if accuracy[i] >= a_t]
+        return min(feasible, key=by_latency) if feasible else min(range(n), key=by_accuracy)
+    feasible = [i for i in range(n) if latency_col[i] <= l_t]
+    return min(feasible, key=by_accuracy) if feasible else min(range(n), key=by_latency)
+
+
+def sushi_sched(queries, accuracy, table, subnet_encs, cand_encs, q: int):
+    """Algorithm 1 as a whole.  queries: (policy, A_t, L_t) per query; table[i][j]: latency of SubNet i with
+    candidate SubGraph j cached, column M = len(cand_encs) for an empty cache (the state before the first
+    caching decision).  Every query is served with the SubNet selected for the current cache state; after
+    every q-th query the cache state becomes the candidate nearest to the average of the last q served
+    SubNets.  Returns (served SubNet index per query, cache state each query was served under)."""
+    m = len(cand_encs)
+    state, window, since = m, [], 0
+    served, states = [], []
+    for policy, a_t, l_t in queries:
+        col = [row[state] for row in table]
+        i = select_subnet(policy, a_t, l_t, accuracy, col)
+        served.append(i)
+        states.append(state)
+        window.append(subnet_encs[i])
+        if len(window) > q:
+            window.pop(0)
+        since += 1
+        if since >= q:
+            since = 0
+            state = nearest_candidate(window, cand_encs)
+    return served, states

@@ -75,3 +75,61 @@ def test_decisions_every_q_queries_use_the_last_q_subnets():
     # q = 1: the cache follows the previous query
     _, _, ch1 = oracle.sched_stream(stream, cands, 1)
     assert ch1 == [0, 0, 1, 1, 1, 0]
+
+
+# ---- per-query SubNet selection and Algorithm 1 as a whole ------------------------------------------------
+ACC = [0.70, 0.74, 0.78, 0.80]
+LAT = [1.0, 1.5, 2.5, 2.0]  # SubNet 3 is both faster and more accurate than SubNet 2
+
+
+def test_select_subnet_strict_accuracy():
+    A, L = oracle.STRICT_ACCURACY, oracle.STRICT_LATENCY
+    assert oracle.select_subnet(A, 0.60, 0.0, ACC, LAT) == 0      # everything feasible: the fastest
+    assert oracle.select_subnet(A, 0.74, 0.0, ACC, LAT) == 1      # accuracy bound is inclusive
+    assert oracle.select_subnet(A, 0.75, 0.0, ACC, LAT) == 3      # {2, 3} feasible: 3 is faster
+    assert oracle.select_subnet(A, 0.90, 0.0, ACC, LAT) == 3      # nothing feasible: the most accurate
+    # the latency bound plays no part under STRICT_ACCURACY (the served latency may exceed it)
+    assert oracle.select_subnet(A, 0.75, 0.1, ACC, LAT) == 3
+    # ties on latency: the more accurate one, then the lowest index
+    assert oracle.select_subnet(A, 0.0, 0.0, [0.7, 0.8, 0.8], [1.0, 1.0, 1.0]) == 1
+    assert oracle.select_subnet(L, 0.0, 5.0, [0.8, 0.8], [2.0, 1.0]) == 1   # ties on accuracy: the faster one
+
+
+def test_select_subnet_strict_latency():
+    L = oracle.STRICT_LATENCY
+    assert oracle.select_subnet(L, 0.0, 3.0, ACC, LAT) == 3       # everything feasible: the most accurate
+    assert oracle.select_subnet(L, 0.0, 1.5, ACC, LAT) == 1       # latency bound is inclusive
+    assert oracle.select_subnet(L, 0.0, 1.9, ACC, LAT) == 1
+    assert oracle.select_subnet(L, 0.0, 2.0, ACC, LAT) == 3
+    assert oracle.select_subnet(L, 0.0, 0.5, ACC, LAT) == 0       # nothing feasible: the fastest
+    assert oracle.select_subnet(L, 0.99, 1.2, ACC, LAT) == 0      # the accuracy bound plays no part
+
+
+def test_selection_depends_on_the_cache_state_column():
+    # the same query picks another SubNet once the cached SubGraph makes that SubNet fast enough
+    table = [[1.0, 1.0, 1.2], [1.4, 2.0, 2.2]]          # columns: G_0, G_1, empty cache
+    acc = [0.70, 0.80]
+    L = oracle.STRICT_LATENCY
+    assert oracle.select_subnet(L, 0.0, 1.5, acc, [r[0] for r in table]) == 1
+    assert oracle.select_subnet(L, 0.0, 1.5, acc, [r[1] for r in table]) == 0
+    assert oracle.select_subnet(L, 0.0, 1.5, acc, [r[2] for r in table]) == 0
+
+
+def test_algorithm_1_hand_run():
+    # two SubNets (small, big), two candidates equal to them; q = 2
+    small, big = enc((4, 4)), enc((16, 4))
+    table = [[1.0, 1.1, 1.2],      # small: G_0 = small cached, G_1 = big cached, nothing cached
+             [2.0, 1.4, 2.4]]      # big is fast only while the big SubGraph is cached
+    acc = [0.70, 0.80]
+    A, L = oracle.STRICT_ACCURACY, oracle.STRICT_LATENCY
+    queries = [(L, 0.0, 2.0),      # empty cache: big takes 2.4 > 2.0 -> small
+               (A, 0.75, 0.0),     # accuracy forces big; window (small, big): mean K = 10, tie -> G_0
+               (L, 0.0, 2.0),      # G_0 cached: big takes 2.0 <= 2.0 -> big
+               (L, 0.0, 1.5),      # G_0: big 2.0 > 1.5 -> small; window (big, small): tie -> G_0 again
+               (A, 0.75, 0.0),     # big
+               (A, 0.75, 0.0),     # big; window (big, big) -> G_1
+               (L, 0.0, 1.5),      # G_1: big takes 1.4 -> big
+               (L, 0.0, 1.05)]     # G_1: small 1.1, big 1.4, none feasible -> the fastest = small
+    served, states = oracle.sushi_sched(queries, acc, table, [small, big], [small, big], 2)
+    assert served == [0, 1, 1, 0, 1, 1, 1, 0]
+    assert states == [2, 2, 0, 0, 0, 0, 1, 1]
