@@ -244,6 +244,44 @@ def run_suite(args):
                     "config": {"workload": f"SGS locality stream on the ResNet-50-shaped SuperNet: {n} queries, Markov chain of configs (p=0.9 one stage's depth or width changes), seed 4, 224x224, batch 1",
                                "candidates": "smallest and largest SubNet plus uniform draws (seed 6), each clipped to the budget",
                                "execution": f"waves of {args.wave}, {args.concurrency} in flight" if args.wave > 0 else f"one stream per query, {args.concurrency} in flight"}})
+    elif args.suite == "table":
+        # the latency table of Section 3.2 measured on this device (rows SubNets, columns cached SubGraphs, last
+        # column = nothing cached) and Algorithm 1 driven by it; accuracies are a FLOPs-monotone stand-in
+        import time
+        net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
+        batch, res, n_sub, n_cand = args.batch, 224, 8, 8
+        subnets = wl.candidate_cfgs(wl.RESNET, n_sub, seed=11)
+        acc = wl.proxy_accuracy([net.subnet_cost(c, batch, res)[0] for c in subnets])
+        x = torch.from_numpy(wl.make_inputs(1, batch, res, seed=1, bf16=True).reshape(batch, res, res, 3)).cuda().to(torch.bfloat16).contiguous()
+        logits = torch.zeros((batch, 1000), dtype=torch.float32, device="cuda")
+        rows = []
+        for budget_mb in (0, 24):
+            net.cache_set_candidates(wl.candidate_cfgs(wl.RESNET, n_cand, seed=6))
+            net.cache_configure(True, budget_mb << 20, args.window)
+            sched = sgs.Scheduler(net, subnets, acc, args.window)
+            sched.measure(x.data_ptr(), batch, res, logits.data_ptr(), reps=9, flush_bytes=256 << 20, stream=stream.cuda_stream)
+            table = sched.get_table()
+            none = table[:, -1]
+            gain = (none[:, None] - table[:, :-1]) / none[:, None]
+            n = 100000
+            policy, a_t, l_t = wl.sched_queries(n, seed=8, accuracy=acc, latency=table.reshape(-1))
+            t0 = time.perf_counter()
+            served, state = sched.step(policy, a_t, l_t)
+            lookup_ns = (time.perf_counter() - t0) / n * 1e9
+            lat = table[served, state]
+            met = np.where(policy == 0, acc[served] >= a_t, lat <= l_t)
+            rows.append({"budget_mb": net.cache_stats().budget_bytes / 2**20, "table_ms": np.round(table, 4).tolist(),
+                         "best_column_gain_mean": float(gain.max(axis=1).mean()), "best_column_gain_max": float(gain.max()),
+                         "column_spread_mean": float(((table[:, :-1].max(axis=1) - table[:, :-1].min(axis=1)) / none).mean()),
+                         "step_ns": lookup_ns, "hard_constraint_met": float(met.mean()),
+                         "served_histogram": np.bincount(served, minlength=n_sub).tolist(),
+                         "cache_state_histogram": np.bincount(state, minlength=n_cand + 1).tolist()})
+            sched.close()
+        net.cache_set_candidates([])
+        out.update({"metric": "latency_table_best_column_gain", "unit": "mean over SubNets of (L[i][none] - min_j L[i][j]) / L[i][none]",
+                    "value": rows[0]["best_column_gain_mean"], "rows": rows, "accuracy_proxy": np.round(acc, 4).tolist(),
+                    "config": {"workload": f"ResNet-50-shaped SuperNet, {n_sub} SubNets x ({n_cand} candidate SubGraphs + empty cache), batch {batch}, 224x224; one query at a time, 256 MB overwritten before every timed run, median of 9",
+                               "scheduler": f"Algorithm 1 with Q = {args.window} on 100000 synthetic (policy, A_t, L_t) queries (seed 8); step_ns includes the caching decision every Q queries"}})
     elif args.suite == "mbv3":
         net = sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16)
         cfgs = wl.uniform_stream(wl.MBV3, args.queries, seed=3)
@@ -304,7 +342,7 @@ def main():
     ap.add_argument("--concurrency", type=int, default=None, help="waves in flight (default 4), or with --wave 0 queries in flight (default 16)")
     ap.add_argument("--batch", type=int, default=1, help="images per query (sgs-probe)")
     ap.add_argument("--evict-first", type=int, default=0, help="with --cache 0: mark weight loads evict-first (sgs-probe)")
-    ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3", "sched"],
+    ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3", "sched", "table"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()
     if args.suite in ("sgs", "sgs-probe"):

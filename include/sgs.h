@@ -138,7 +138,7 @@ typedef struct {
     size_t cached_subgraph_bytes;  /* weight bytes of the SubGraph currently marked resident */
     size_t supernet_bytes;         /* device bytes of all stored weights */
     size_t device_bytes_allocated; /* every device byte the handle owns (weights + workspaces) */
-    int policy;                    /* SGS_POLICY_* in force */
+    int policy;                    /* SGS_POLICY_* in force; 2 while a scheduler object pins the cache */
     int n_candidates;              /* size of the candidate set S */
     int decisions;                 /* caching decisions taken since the cache was last reset */
     int last_choice;               /* index into S of the last AvgNet decision; -1 = none yet */
@@ -222,6 +222,51 @@ sgs_status_t sgs_cache_stats(const sgs_supernet_t *net, sgs_cache_stats_t *out);
  */
 sgs_status_t sgs_cache_set_candidates(sgs_supernet_t *net, const sgs_subnet_cfg_t *cfgs, int n);
 sgs_status_t sgs_cache_set_policy(sgs_supernet_t *net, int policy);
+
+/*
+ * Scheduler object: Algorithm 1 (Section 3.3) over a latency table with SubNets as rows and cacheable
+ * SubGraphs as columns (Section 3.2).  Host-side state only, apart from sgs_sched_measure.
+ *
+ * sgs_sched_create - rows = `subnets` (host array of n_subnets configs, copied) with their `accuracy`
+ *   (host array of n_subnets doubles, copied; any monotone proxy will do), columns = the candidate set
+ *   installed with sgs_cache_set_candidates at this moment (M of them) plus column M = nothing cached.
+ *   window_q >= 1 = Algorithm 1's Q.  The table starts as zeros; the cache of `net` is emptied and from
+ *   now on moves only when the scheduler decides (sgs_subnet_run no longer re-chooses it; a later
+ *   sgs_stream_run takes the cache back).  `net` must outlive the scheduler; do not change the candidate
+ *   set or the cache budget while it lives.  Errors: SGS_EINVAL (no candidate set, bad argument),
+ *   SGS_ECONFIG, SGS_ENOMEM.
+ * sgs_sched_dims - n_subnets and n_columns (= M + 1); either pointer may be NULL.
+ * sgs_sched_set_table / sgs_sched_get_table - latency[i * n_columns + j], host doubles, any unit.
+ * sgs_sched_measure - fills the table on the device: for every column j the cache is pinned to SubGraph j
+ *   and every SubNet i runs once untimed and then `reps` (1..1000) times on `cuda_stream` between two
+ *   events; entry = median in milliseconds.  Before each timed run `flush_bytes` bytes of scratch owned by
+ *   the scheduler are overwritten (0 = no flush): this stands for the other traffic of a serving system
+ *   that pushes unprotected weights out of L2 between two queries.  d_input [batch][res][res][3] in the
+ *   compute dtype and d_logits [batch][n_classes] fp32 are caller-owned device buffers.  Synchronises
+ *   the stream.  Afterwards the cache is pinned to the scheduler's current state again.
+ * sgs_sched_step - n queries in order.  Query t = (policy[t], a_t[t], l_t[t]) with policy
+ *   SGS_STRICT_ACCURACY (serve the fastest SubNet among those with accuracy >= a_t) or SGS_STRICT_LATENCY
+ *   (serve the most accurate SubNet among those with latency <= l_t), latency taken from the column of the
+ *   current cache state.  An empty feasible set falls back to the most accurate / the fastest SubNet; ties
+ *   are broken by the other quantity, then by the lowest row.  subnet[t] receives the row served,
+ *   cache_state[t] (may be NULL) the column it was served under.  After every window_q-th query the cache
+ *   state becomes the candidate nearest to the mean encoding of the last window_q served SubNets (as
+ *   SGS_POLICY_AVGNET) and is enacted on `net` when the call returns.  All arrays are host arrays.
+ * sgs_sched_subnet - copies row i's config to *out (to pass to sgs_subnet_run).
+ */
+typedef struct sgs_sched sgs_sched_t;
+enum { SGS_STRICT_ACCURACY = 0, SGS_STRICT_LATENCY = 1 };
+sgs_status_t sgs_sched_create(sgs_supernet_t *net, const sgs_subnet_cfg_t *subnets, const double *accuracy, int n_subnets,
+                              int window_q, sgs_sched_t **out);
+void sgs_sched_free(sgs_sched_t *sched);
+sgs_status_t sgs_sched_dims(const sgs_sched_t *sched, int *n_subnets, int *n_columns);
+sgs_status_t sgs_sched_set_table(sgs_sched_t *sched, const double *latency);
+sgs_status_t sgs_sched_get_table(const sgs_sched_t *sched, double *latency);
+sgs_status_t sgs_sched_measure(sgs_sched_t *sched, const void *d_input, int batch, int res, void *d_logits, int reps,
+                               size_t flush_bytes, void *cuda_stream);
+sgs_status_t sgs_sched_step(sgs_sched_t *sched, int n, const int *policy, const double *a_t, const double *l_t,
+                            int *subnet, int *cache_state);
+sgs_status_t sgs_sched_subnet(const sgs_sched_t *sched, int i, sgs_subnet_cfg_t *out);
 
 /*
  * Vector encoding of a SubNet (Section 3.3): for every stored layer i, out[3i] = K_i (filters),

@@ -17,6 +17,7 @@ LIB_PATH = os.environ.get("SGS_LIB") or os.path.join(_HERE, "libsgs.so")  # SGS_
 
 SGS_OK, SGS_EINVAL, SGS_ECONFIG, SGS_ENOMEM, SGS_ECUDA, SGS_ETIMEOUT, SGS_EUNSUPPORTED = range(7)
 SGS_POLICY_INTERSECTION, SGS_POLICY_AVGNET = 0, 1
+SGS_STRICT_ACCURACY, SGS_STRICT_LATENCY = 0, 1
 SGS_F32, SGS_BF16 = 0, 1
 STATUS_NAMES = ["SGS_OK", "SGS_EINVAL", "SGS_ECONFIG", "SGS_ENOMEM", "SGS_ECUDA", "SGS_ETIMEOUT", "SGS_EUNSUPPORTED"]
 
@@ -25,6 +26,8 @@ EXPORTS = [
     "sgs_cache_configure", "sgs_cache_stats", "sgs_num_layers", "sgs_subnet_encode", "sgs_subnet_cost",
     "sgs_set_option", "sgs_get_counter", "sgs_last_error", "sgs_supernet_free", "sgs_conv2d_sliced", "sgs_device_status",
     "sgs_profile_read", "sgs_conv2d_sliced_static", "sgs_cache_set_candidates", "sgs_cache_set_policy",
+    "sgs_sched_create", "sgs_sched_free", "sgs_sched_dims", "sgs_sched_set_table", "sgs_sched_get_table", "sgs_sched_measure",
+    "sgs_sched_step", "sgs_sched_subnet",
 ]
 
 
@@ -62,6 +65,69 @@ class CacheStats(ctypes.Structure):
         return {n: getattr(self, n) for n, _ in self._fields_}
 
 
+class Scheduler:
+    """sgs_sched_*: Algorithm 1 over a latency table (rows = SubNets, columns = the SuperNet's candidate SubGraphs
+    plus one for an empty cache).  Argument marshalling only."""
+
+    def __init__(self, net: "SuperNet", subnets: Sequence, accuracy: Sequence[float], window_q: int):
+        import numpy as np
+        self.net = net
+        arr = subnets if isinstance(subnets, ctypes.Array) else cfg_array(subnets)
+        acc = np.ascontiguousarray(accuracy, dtype=np.float64)
+        if acc.shape != (len(arr),):
+            raise ValueError("one accuracy per SubNet")
+        self._h = ctypes.c_void_p()
+        net._check(lib().sgs_sched_create(net._h, ctypes.addressof(arr), acc.ctypes.data, len(arr), window_q, ctypes.byref(self._h)))
+        n, m = ctypes.c_int(), ctypes.c_int()
+        net._check(lib().sgs_sched_dims(self._h, ctypes.addressof(n), ctypes.addressof(m)))
+        self.n_subnets, self.n_columns = n.value, m.value
+
+    def close(self):
+        if self._h:
+            lib().sgs_sched_free(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_table(self, table):
+        import numpy as np
+        tb = np.ascontiguousarray(table, dtype=np.float64)
+        if tb.shape != (self.n_subnets, self.n_columns):
+            raise ValueError("table must be [n_subnets][n_columns]")
+        self.net._check(lib().sgs_sched_set_table(self._h, tb.ctypes.data))
+
+    def get_table(self):
+        import numpy as np
+        tb = np.zeros((self.n_subnets, self.n_columns), dtype=np.float64)
+        self.net._check(lib().sgs_sched_get_table(self._h, tb.ctypes.data))
+        return tb
+
+    def measure(self, d_input: int, batch: int, res: int, d_logits: int, reps: int = 5, flush_bytes: int = 0, stream: int = 0):
+        self.net._check(lib().sgs_sched_measure(self._h, d_input, batch, res, d_logits, reps, flush_bytes, stream))
+
+    def step(self, policy, a_t, l_t):
+        """Arrays (or scalars) of query policies, accuracy and latency targets -> (served rows, cache-state columns)."""
+        import numpy as np
+        pol = np.ascontiguousarray(np.atleast_1d(policy), dtype=np.int32)
+        a = np.ascontiguousarray(np.atleast_1d(a_t), dtype=np.float64)
+        l = np.ascontiguousarray(np.atleast_1d(l_t), dtype=np.float64)
+        if not (pol.shape == a.shape == l.shape) or pol.ndim != 1:
+            raise ValueError("policy, a_t and l_t must be 1-d and of one length")
+        sub = np.zeros(len(pol), dtype=np.int32)
+        state = np.zeros(len(pol), dtype=np.int32)
+        self.net._check(lib().sgs_sched_step(self._h, len(pol), pol.ctypes.data, a.ctypes.data, l.ctypes.data, sub.ctypes.data, state.ctypes.data))
+        return sub, state
+
+    def subnet(self, i: int) -> SubnetCfg:
+        c = SubnetCfg()
+        self.net._check(lib().sgs_sched_subnet(self._h, i, ctypes.byref(c)))
+        return c
+
+
 class SgsError(RuntimeError):
     def __init__(self, status: int, text: str):
         super().__init__(f"{STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else status}: {text}")
@@ -88,6 +154,15 @@ def lib():
         L.sgs_cache_stats.argtypes = [vp, vp]
         L.sgs_cache_set_candidates.argtypes = [vp, vp, ci]
         L.sgs_cache_set_policy.argtypes = [vp, ci]
+        L.sgs_sched_create.argtypes = [vp, vp, vp, ci, ci, ctypes.POINTER(vp)]
+        L.sgs_sched_free.argtypes = [vp]
+        L.sgs_sched_free.restype = None
+        L.sgs_sched_dims.argtypes = [vp, vp, vp]
+        L.sgs_sched_set_table.argtypes = [vp, vp]
+        L.sgs_sched_get_table.argtypes = [vp, vp]
+        L.sgs_sched_measure.argtypes = [vp, vp, ci, ci, vp, ci, cs, vp]
+        L.sgs_sched_step.argtypes = [vp, ci, vp, vp, vp, vp, vp]
+        L.sgs_sched_subnet.argtypes = [vp, ci, vp]
         L.sgs_num_layers.argtypes = [vp]
         L.sgs_subnet_encode.argtypes = [vp, vp, vp]
         L.sgs_subnet_cost.argtypes = [vp, vp, ci, ci, vp, vp, vp]

@@ -139,7 +139,8 @@ struct CacheState {
     int epoch = 0;                        // bumped whenever G changes
     int since_update = 0;
     int evict_first_when_off = 0;
-    int policy = 0;                       // 0: intersection of the window; 1: candidate nearest to the window's average
+    int policy = 0;                       // 0: intersection of the window; 1: candidate nearest to the window's average;
+                                          // 2: pinned by a scheduler object (observations change nothing)
     std::vector<std::vector<int>> cand_raw, cand;  // candidate SubGraph encodings as given / clipped to the budget
     std::vector<size_t> cand_bytes;
     int decisions = 0, last_choice = -1;
@@ -969,24 +970,29 @@ void clip_candidates(sgs_supernet *net) {
 // the candidate G_j with the smallest Euclidean distance to it on the (K_i, C_i) entries (Section 3.3).
 // With Q = window length and S = element-wise sum, Q^2 * Dist^2 = sum_i (Q * G_ji - S_i)^2 is compared
 // exactly in 64-bit integers; ties go to the lowest index.
-void choose_nearest_candidate(sgs_supernet *net) {
-    CacheState &cs = net->cache;
-    const long long Q = (long long)cs.window.size();
-    const size_t n = cs.window.front().size();
+int nearest_candidate(const std::deque<std::vector<int>> &window, const std::vector<std::vector<int>> &cand) {
+    const long long Q = (long long)window.size();
+    const size_t n = window.front().size();
     std::vector<long long> S(n, 0);
-    for (const auto &e : cs.window)
+    for (const auto &e : window)
         for (size_t i = 0; i < n; i++) S[i] += e[i];
     int best = -1;
     unsigned long long best_d = 0;
-    for (size_t j = 0; j < cs.cand.size(); j++) {
+    for (size_t j = 0; j < cand.size(); j++) {
         unsigned long long d = 0;
         for (size_t i = 0; i < n; i++) {
             if (i % 3 == 2) continue;  // the kernel-size entry takes no part in the distance
-            long long t = Q * cs.cand[j][i] - S[i];
+            long long t = Q * cand[j][i] - S[i];
             d += (unsigned long long)(t * t);
         }
         if (best < 0 || d < best_d) { best = (int)j; best_d = d; }
     }
+    return best;
+}
+
+void choose_nearest_candidate(sgs_supernet *net) {
+    CacheState &cs = net->cache;
+    const int best = nearest_candidate(cs.window, cs.cand);
     cs.decisions++;
     cs.last_choice = best;
     if (cs.cand[best] != cs.G) { cs.G = cs.cand[best]; cs.epoch++; }
@@ -1031,8 +1037,24 @@ QueryAccount account_query(const sgs_supernet *net, const std::vector<int> &sn) 
     return a;
 }
 
+// The cached SubGraph becomes candidate j (anything outside [0, |S|) empties the cache) and stays until the
+// next pin: observations no longer move it.
+void cache_pin(sgs_supernet *net, int j) {
+    CacheState &cs = net->cache;
+    cs.enabled = true;
+    cs.policy = 2;
+    std::vector<int> g;
+    size_t bytes = 0;
+    if (j >= 0 && j < (int)cs.cand.size()) { g = cs.cand[j]; bytes = cs.cand_bytes[j]; }
+    else j = -1;
+    if (g != cs.G) { cs.G = std::move(g); cs.epoch++; }
+    cs.G_bytes = bytes;
+    cs.last_choice = j;
+}
+
 void cache_observe(sgs_supernet *net, const std::vector<int> &enc) {
     CacheState &cs = net->cache;
+    if (cs.policy == 2) return;
     cs.window.push_back(enc);
     while ((int)cs.window.size() > cs.window_q) cs.window.pop_front();
     if (++cs.since_update >= cs.window_q) {
@@ -1863,6 +1885,171 @@ sgs_status_t sgs_cache_set_policy(sgs_supernet_t *net, int policy) {
     if (policy == SGS_POLICY_AVGNET && net->cache.cand_raw.empty())
         return fail(net, SGS_EINVAL, "the AvgNet policy needs a candidate set (sgs_cache_set_candidates)");
     net->cache.policy = policy;
+    return SGS_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Scheduler object: Algorithm 1 (Section 3.3) over a latency table (Section 3.2)
+// ------------------------------------------------------------------------------------------
+}  // extern "C"
+
+struct sgs_sched {
+    sgs_supernet *net = nullptr;
+    int N = 0, M = 0, q = 1;
+    std::vector<sgs_subnet_cfg_t> subnets;
+    std::vector<std::vector<int>> encs;
+    std::vector<double> acc, table;  // table[i * (M + 1) + j]; column M = nothing cached
+    std::deque<std::vector<int>> window;
+    int since = 0, state = 0;
+    void *flush = nullptr;
+    size_t flush_bytes = 0;
+};
+
+namespace {
+int sched_select(const sgs_sched *s, int policy, double a_t, double l_t) {
+    const int W = s->M + 1;
+    int best = -1;
+    bool best_feasible = false;
+    for (int i = 0; i < s->N; i++) {
+        const double lat = s->table[(size_t)i * W + s->state], acc = s->acc[i];
+        const bool feasible = policy == SGS_STRICT_ACCURACY ? acc >= a_t : lat <= l_t;
+        if (best < 0) { best = i; best_feasible = feasible; continue; }
+        if (feasible != best_feasible) { if (feasible) { best = i; best_feasible = true; } continue; }
+        const double blat = s->table[(size_t)best * W + s->state], bacc = s->acc[best];
+        // among feasible SubNets: the fastest (STRICT_ACCURACY) / the most accurate (STRICT_LATENCY); with no
+        // feasible SubNet the roles swap (the most accurate / the fastest); ties by the other quantity
+        const bool by_latency = (policy == SGS_STRICT_ACCURACY) == feasible;
+        const bool better = by_latency ? (lat < blat || (lat == blat && acc > bacc)) : (acc > bacc || (acc == bacc && lat < blat));
+        if (better) best = i;
+    }
+    return best;
+}
+}  // namespace
+
+extern "C" {
+
+sgs_status_t sgs_sched_create(sgs_supernet_t *net, const sgs_subnet_cfg_t *subnets, const double *accuracy, int n_subnets,
+                              int window_q, sgs_sched_t **out) {
+    if (!net || !out) return SGS_EINVAL;
+    if (!subnets || !accuracy || n_subnets < 1 || window_q < 1) return fail(net, SGS_EINVAL, "bad argument");
+    if (net->cache.cand_raw.empty()) return fail(net, SGS_EINVAL, "a scheduler needs a candidate set (sgs_cache_set_candidates)");
+    std::unique_ptr<sgs_sched> s(new (std::nothrow) sgs_sched);
+    if (!s) return SGS_ENOMEM;
+    s->net = net; s->N = n_subnets; s->M = (int)net->cache.cand_raw.size(); s->q = window_q;
+    for (int i = 0; i < n_subnets; i++) {
+        if (!cfg_valid(net, &subnets[i])) return fail(net, SGS_ECONFIG, "SubNet " + std::to_string(i) + ": config outside the elastic sets");
+        s->subnets.push_back(subnets[i]);
+        s->encs.push_back(encoding_of(slices_for(net, &subnets[i])));
+        s->acc.push_back(accuracy[i]);
+    }
+    s->table.assign((size_t)s->N * (s->M + 1), 0.0);
+    s->state = s->M;
+    cache_pin(net, -1);
+    *out = s.release();
+    return SGS_OK;
+}
+
+void sgs_sched_free(sgs_sched_t *s) {
+    if (!s) return;
+    if (s->flush) {
+        DeviceGuard guard(s->net->device);
+        cudaDeviceSynchronize();
+        dev_free(s->net, s->flush, s->flush_bytes);
+    }
+    if (s->net->cache.policy == 2) { s->net->cache.policy = 0; cache_reset(s->net, false, s->net->cache.budget, s->net->cache.window_q); }
+    delete s;
+}
+
+sgs_status_t sgs_sched_dims(const sgs_sched_t *s, int *n_subnets, int *n_columns) {
+    if (!s) return SGS_EINVAL;
+    if (n_subnets) *n_subnets = s->N;
+    if (n_columns) *n_columns = s->M + 1;
+    return SGS_OK;
+}
+
+sgs_status_t sgs_sched_set_table(sgs_sched_t *s, const double *latency) {
+    if (!s || !latency) return SGS_EINVAL;
+    std::copy(latency, latency + s->table.size(), s->table.begin());
+    return SGS_OK;
+}
+
+sgs_status_t sgs_sched_get_table(const sgs_sched_t *s, double *latency) {
+    if (!s || !latency) return SGS_EINVAL;
+    std::copy(s->table.begin(), s->table.end(), latency);
+    return SGS_OK;
+}
+
+sgs_status_t sgs_sched_measure(sgs_sched_t *s, const void *d_input, int batch, int res, void *d_logits, int reps,
+                               size_t flush_bytes, void *cuda_stream) {
+    if (!s) return SGS_EINVAL;
+    sgs_supernet *net = s->net;
+    if (!d_input || !d_logits || batch <= 0 || res < 8 || res > 1024 || reps < 1 || reps > 1000) return fail(net, SGS_EINVAL, "bad argument");
+    DeviceGuard guard(net->device);
+    if (!guard.ok) return fail(net, SGS_ECUDA, "cudaSetDevice failed");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (flush_bytes > s->flush_bytes) {
+        CU(cudaStreamSynchronize(st));
+        dev_free(net, s->flush, s->flush_bytes);
+        s->flush = nullptr; s->flush_bytes = 0;
+        sgs_status_t rc = dev_alloc(net, &s->flush, flush_bytes);
+        if (rc != SGS_OK) return rc;
+        s->flush_bytes = flush_bytes;
+    }
+    std::vector<cudaEvent_t> ev(2 * (size_t)reps);
+    for (auto &e : ev) CU(cudaEventCreate(&e));
+    sgs_status_t rc = SGS_OK;
+    std::vector<float> ms((size_t)reps);
+    for (int j = 0; j <= s->M && rc == SGS_OK; j++) {
+        cache_pin(net, j < s->M ? j : -1);
+        for (int i = 0; i < s->N && rc == SGS_OK; i++) {
+            // one untimed run builds the plan and brings the SubNet's weights in under the hints of column j
+            rc = run_query(net, &s->subnets[i], d_input, batch, res, d_logits, st, false, 0, nullptr);
+            for (int r = 0; r < reps && rc == SGS_OK; r++) {
+                if (flush_bytes && cudaMemsetAsync(s->flush, r & 1, flush_bytes, st) != cudaSuccess) rc = fail(net, SGS_ECUDA, "flush failed");
+                if (rc == SGS_OK && cudaEventRecord(ev[2 * r], st) != cudaSuccess) rc = fail(net, SGS_ECUDA, "event record failed");
+                if (rc == SGS_OK) rc = run_query(net, &s->subnets[i], d_input, batch, res, d_logits, st, false, 0, nullptr);
+                if (rc == SGS_OK && cudaEventRecord(ev[2 * r + 1], st) != cudaSuccess) rc = fail(net, SGS_ECUDA, "event record failed");
+            }
+            if (rc != SGS_OK) break;
+            if (cudaStreamSynchronize(st) != cudaSuccess) { rc = fail(net, SGS_ECUDA, "stream synchronise failed"); break; }
+            for (int r = 0; r < reps; r++) cudaEventElapsedTime(&ms[r], ev[2 * r], ev[2 * r + 1]);
+            std::vector<float> sorted = ms;
+            std::sort(sorted.begin(), sorted.end());
+            s->table[(size_t)i * (s->M + 1) + j] = reps & 1 ? sorted[reps / 2] : 0.5 * ((double)sorted[reps / 2 - 1] + sorted[reps / 2]);
+        }
+    }
+    cudaStreamSynchronize(st);
+    for (auto &e : ev) cudaEventDestroy(e);
+    cache_pin(net, s->state < s->M ? s->state : -1);
+    if (rc == SGS_OK && tc_conv_status()) return fail(net, SGS_ETIMEOUT, "a bounded wait ran out in a tensor-core kernel");
+    return rc;
+}
+
+sgs_status_t sgs_sched_step(sgs_sched_t *s, int n, const int *policy, const double *a_t, const double *l_t, int *subnet,
+                            int *cache_state) {
+    if (!s) return SGS_EINVAL;
+    if (n < 0 || (n && (!policy || !a_t || !l_t || !subnet))) return fail(s->net, SGS_EINVAL, "bad argument");
+    for (int t = 0; t < n; t++)
+        if (policy[t] != SGS_STRICT_ACCURACY && policy[t] != SGS_STRICT_LATENCY) return fail(s->net, SGS_EINVAL, "unknown query policy");
+    const int before = s->state;
+    for (int t = 0; t < n; t++) {
+        const int i = sched_select(s, policy[t], a_t[t], l_t[t]);
+        subnet[t] = i;
+        if (cache_state) cache_state[t] = s->state;
+        s->window.push_back(s->encs[i]);
+        while ((int)s->window.size() > s->q) s->window.pop_front();
+        if (++s->since >= s->q) {
+            s->since = 0;
+            s->state = nearest_candidate(s->window, s->net->cache.cand);
+        }
+    }
+    if (s->state != before || s->net->cache.policy != 2) cache_pin(s->net, s->state < s->M ? s->state : -1);
+    return SGS_OK;
+}
+
+sgs_status_t sgs_sched_subnet(const sgs_sched_t *s, int i, sgs_subnet_cfg_t *out) {
+    if (!s || !out || i < 0 || i >= s->N) return SGS_EINVAL;
+    *out = s->subnets[i];
     return SGS_OK;
 }
 

@@ -349,6 +349,28 @@ def candidate_cfgs(family: int, n: int, seed: int) -> List[SubnetCfg]:
     return out
 
 
+def proxy_accuracy(flops: Sequence[float], lo: float = 0.70, hi: float = 0.80) -> np.ndarray:
+    """Stand-in for the trained SubNets' accuracies (inputs of the scheduler): monotone in the SubNet's FLOPs,
+    spread linearly in log-FLOPs over [lo, hi]."""
+    f = np.log(np.asarray(flops, dtype=np.float64))
+    span = float(f.max() - f.min())
+    return lo + (hi - lo) * ((f - f.min()) / span if span > 0 else np.zeros_like(f))
+
+
+def sched_queries(n: int, seed: int, accuracy: Sequence[float], latency: Sequence[float], p_accuracy: float = 0.5):
+    """n scheduler queries (policy, A_t, L_t): policy 0 (accuracy is the hard constraint) with probability
+    p_accuracy, else 1 (latency is); targets drawn uniformly from a range slightly wider than the SubNets'
+    own accuracies and latencies, so that some queries have an empty feasible set."""
+    rng = np.random.default_rng(seed)
+    acc = np.asarray(accuracy, dtype=np.float64)
+    lat = np.asarray(latency, dtype=np.float64)
+    da, dl = float(acc.max() - acc.min()), float(lat.max() - lat.min())
+    policy = (rng.random(n) >= p_accuracy).astype(np.int32)
+    a_t = rng.uniform(acc.min() - 0.1 * da, acc.max() + 0.1 * da, n)
+    l_t = rng.uniform(lat.min() - 0.1 * dl, lat.max() + 0.1 * dl, n)
+    return policy, a_t, l_t
+
+
 def copy_cfg(c: SubnetCfg) -> SubnetCfg:
     d = SubnetCfg()
     ctypes.memmove(ctypes.byref(d), ctypes.byref(c), ctypes.sizeof(SubnetCfg))

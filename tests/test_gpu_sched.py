@@ -85,3 +85,99 @@ def test_avgnet_policy_needs_candidates_and_valid_configs():
     finally:
         gnet.cache_set_candidates([])
         gnet.cache_configure(False, 0, 4)
+
+
+def _sched_case(q, budget, measured):
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    res = 64
+    subnets = wl.candidate_cfgs(wl.RESNET, 8, seed=11)
+    cands = wl.candidate_cfgs(wl.RESNET, 6, seed=5)
+    acc = wl.proxy_accuracy([gnet.subnet_cost(c, 1, res)[0] for c in subnets])
+    d_in = gu.to_device(wl.make_inputs(1, 1, res, seed=2, bf16=True).reshape(1, res, res, 3), True)
+    d_out = torch.zeros((1, 1000), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    gnet.cache_set_candidates(cands)
+    sched = None
+    try:
+        gnet.cache_configure(True, budget, q)
+        budget_bytes = gnet.cache_stats().budget_bytes
+        sched = sgs.Scheduler(gnet, subnets, acc, q)
+        assert (sched.n_subnets, sched.n_columns) == (8, 7)
+        assert gnet.cache_stats().policy == 2 and gnet.cache_stats().cached_subgraph_bytes == 0
+        if measured:
+            sched.measure(d_in.data_ptr(), 1, res, d_out.data_ptr(), reps=3, flush_bytes=160 << 20, stream=stream.cuda_stream)
+            table = sched.get_table()
+            assert table.shape == (8, 7) and np.all(table > 0) and np.all(table < 50)   # milliseconds of a batch-1 query
+            assert table[1].mean() > table[0].mean()                                    # the largest SubNet is slower than the smallest
+        else:
+            # a synthetic table: latency grows with the SubNet, shrinks with the weights the column's SubGraph shares with it
+            rng = np.random.default_rng(3)
+            encs_ = [onet.encode(c) for c in subnets]
+            cand_ = [oracle.clip_to_budget(onet.encode(c), budget_bytes // 2) for c in cands] + [np.zeros_like(encs_[0])]
+            table = np.array([[1e-6 * oracle.encoding_weights(e) * (1.0 - 0.5 * oracle.encoding_weights(oracle.intersect(e, g)) / oracle.encoding_weights(e))
+                               for g in cand_] for e in encs_]) + rng.uniform(0, 0.01, (8, 7))
+            sched.set_table(table)
+            np.testing.assert_array_equal(sched.get_table(), table)
+        n = 90
+        policy, a_t, l_t = wl.sched_queries(n, seed=17 + q, accuracy=acc, latency=table.reshape(-1))
+        got_sub, got_state = [], []
+        for lo, hi in ((0, 1), (1, 31), (31, 31), (31, n)):     # state carries over calls of any length
+            s, c = sched.step(policy[lo:hi], a_t[lo:hi], l_t[lo:hi])
+            got_sub += list(s)
+            got_state += list(c)
+        encs = [onet.encode(c) for c in subnets]
+        cand_encs = [oracle.clip_to_budget(onet.encode(c), budget_bytes // 2) for c in cands]
+        served, states = oracle.sushi_sched(list(zip(policy.tolist(), a_t.tolist(), l_t.tolist())), acc.tolist(), table.tolist(), encs, cand_encs, q)
+        assert got_sub == served and got_state == states
+        assert len(set(served)) >= 3 and len(set(states)) >= 2      # the queries and the table really move both decisions
+        # the scheduler's last decision is what the device cache holds, and running queries does not move it
+        final = oracle.nearest_candidate([encs[i] for i in served[-q:]], cand_encs) if n % q == 0 else None
+        cs = gnet.cache_stats()
+        if final is not None:
+            assert cs.last_choice == final
+        assert cs.policy == 2 and cs.cached_subgraph_bytes == 2 * oracle.encoding_weights(cand_encs[cs.last_choice])
+        for i in served[-3:]:
+            cfg = sched.subnet(i)
+            gnet.subnet_run(cfg, d_in.data_ptr(), 1, res, d_out.data_ptr(), stream.cuda_stream)
+            stream.synchronize()
+            ref = onet.forward(cfg, wl.make_inputs(1, 1, res, seed=2, bf16=True).reshape(1, res, res, 3), oracle.BF16_STORE)
+            assert gu.rel_err(d_out.cpu().numpy(), ref) < 2e-2
+        assert gnet.cache_stats().last_choice == cs.last_choice
+    finally:
+        if sched is not None:
+            sched.close()
+        gnet.cache_set_candidates([])
+        gnet.cache_configure(False, 0, 4)
+    assert gnet.cache_stats().policy == 0 and gnet.cache_stats().enabled == 0
+
+
+def test_scheduler_on_a_synthetic_table_matches_checker():
+    _sched_case(q=3, budget=24 << 20, measured=False)
+    _sched_case(q=1, budget=0, measured=False)
+
+
+def test_scheduler_on_its_measured_table_matches_checker():
+    _sched_case(q=5, budget=32 << 20, measured=True)
+
+
+def test_scheduler_argument_errors():
+    _, _, gnet = gu.nets(wl.TINY, True)
+    cfgs = wl.uniform_stream(wl.TINY, 3, seed=1)
+    with pytest.raises(sgs.SgsError, match="EINVAL"):       # no candidate set
+        sgs.Scheduler(gnet, cfgs, [0.1, 0.2, 0.3], 2)
+    gnet.cache_set_candidates(cfgs[:2])
+    try:
+        with pytest.raises(sgs.SgsError, match="EINVAL"):
+            sgs.Scheduler(gnet, cfgs, [0.1, 0.2, 0.3], 0)
+        s = sgs.Scheduler(gnet, cfgs, [0.1, 0.2, 0.3], 2)
+        with pytest.raises(sgs.SgsError, match="EINVAL"):
+            s.step([7], [0.0], [0.0])
+        with pytest.raises(ValueError):
+            s.set_table(np.zeros((2, 2)))
+        sub, state = s.step([], [], [])
+        assert len(sub) == 0
+        s.close()
+    finally:
+        gnet.cache_set_candidates([])
+        gnet.cache_configure(False, 0, 4)
