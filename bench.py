@@ -220,20 +220,22 @@ def run_suite(args):
     elif args.suite == "sched":
         # caching decision of Algorithm 1 (nearest candidate SubGraph to the running average) beside the
         # intersection of the window, over the window length Q, the size of the candidate set and the budget
-        net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
+        fam = wl.MBV3 if args.family == "mbv3" else wl.RESNET
+        net = sgs.SuperNet(fam, wl.make_blob(fam, seed=0, bf16_weights=True), sgs.SGS_BF16)
         n = args.queries
-        cfgs = wl.markov_stream(n, seed=4)
+        cfgs = wl.markov_stream(n, seed=4, family=fam)
         rows = []
         warm = sgs.StreamOpts(cache_enabled=0, window_q=4, record_latency=0, concurrency=args.concurrency, wave=args.wave)
-        _stream_pool(net, sgs, torch, cfgs, 1, 224, warm, stream, n, wl.RESNET)
-        for budget_mb in (0, 24):
+        _stream_pool(net, sgs, torch, cfgs, 1, 224, warm, stream, n, fam)
+        # budgets: the device maximum, and about a quarter of the SuperNet's weights
+        for budget_mb in ((0, 24) if fam == wl.RESNET else (0, 4)):
             for n_cand in (0, 16, 64, 256):
-                net.cache_set_candidates(wl.candidate_cfgs(wl.RESNET, n_cand, seed=6) if n_cand else [])
+                net.cache_set_candidates(wl.candidate_cfgs(fam, n_cand, seed=6) if n_cand else [])
                 for q in (1, 2, 4, 8, 16):
                     opts = sgs.StreamOpts(cache_enabled=1, window_q=q, cache_budget_bytes=budget_mb << 20, record_latency=0,
                                           concurrency=args.concurrency, wave=args.wave,
                                           policy=sgs.SGS_POLICY_AVGNET if n_cand else sgs.SGS_POLICY_INTERSECTION)
-                    t = _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, n, wl.RESNET)
+                    t = _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, n, fam)
                     rows.append({"policy": "avgnet" if n_cand else "intersection", "candidates": n_cand, "window_q": q,
                                  "budget_mb": net.cache_stats().budget_bytes / 2**20, "hit_ratio": t["hit"] / t["q"],
                                  "weight_mb_per_query": t["wbytes"] / t["q"] / 1e6, "hbm_weight_mb_per_query": t["miss"] / t["q"] / 1e6,
@@ -241,7 +243,7 @@ def run_suite(args):
         net.cache_set_candidates([])
         best = max(rows, key=lambda r: r["hit_ratio"])
         out.update({"metric": "cache_hit_ratio", "unit": "mean ||SN ∩ G|| / ||SN|| (analytic)", "value": best["hit_ratio"], "best": best, "rows": rows,
-                    "config": {"workload": f"SGS locality stream on the ResNet-50-shaped SuperNet: {n} queries, Markov chain of configs (p=0.9 one stage's depth or width changes), seed 4, 224x224, batch 1",
+                    "config": {"workload": f"SGS locality stream on the {'MobileNetV3' if fam == wl.MBV3 else 'ResNet-50'}-shaped SuperNet: {n} queries, Markov chain of configs (p=0.9 one elastic choice changes), seed 4, 224x224, batch 1",
                                "candidates": "smallest and largest SubNet plus uniform draws (seed 6), each clipped to the budget",
                                "execution": f"waves of {args.wave}, {args.concurrency} in flight" if args.wave > 0 else f"one stream per query, {args.concurrency} in flight"}})
     elif args.suite == "table":
@@ -342,6 +344,7 @@ def main():
     ap.add_argument("--concurrency", type=int, default=None, help="waves in flight (default 4), or with --wave 0 queries in flight (default 16)")
     ap.add_argument("--batch", type=int, default=1, help="images per query (sgs-probe)")
     ap.add_argument("--evict-first", type=int, default=0, help="with --cache 0: mark weight loads evict-first (sgs-probe)")
+    ap.add_argument("--family", default="resnet", choices=["resnet", "mbv3"], help="SuperNet of the sched suite")
     ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3", "sched", "table"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()

@@ -377,27 +377,38 @@ def copy_cfg(c: SubnetCfg) -> SubnetCfg:
     return d
 
 
-def markov_stream(n: int, seed: int = 4, p_local: float = 0.9) -> List[SubnetCfg]:
-    """Locality stream on the ResNet-50-shaped SuperNet.
+def markov_stream(n: int, seed: int = 4, p_local: float = 0.9, family: int = RESNET) -> List[SubnetCfg]:
+    """Locality stream on the ResNet-50-shaped (default) or MobileNetV3-shaped SuperNet.
 
-    With probability ``p_local`` the next config differs from the previous one in at most one
-    stage's depth or width (one of the two is redrawn, possibly to the same value); otherwise the
-    whole config is redrawn uniformly.  This gives consecutive queries a large shared SubGraph,
-    the temporal locality the paper's SubGraph-Stationary reuse exploits (Section 2.2).
+    With probability ``p_local`` the next config differs from the previous one in one place (ResNet: one
+    stage's depth or width; MobileNetV3: one stage's depth, or one block's expansion ratio or kernel size),
+    redrawn possibly to the same value; otherwise the whole config is redrawn uniformly.  This gives
+    consecutive queries a large shared SubGraph, the temporal locality the paper's SubGraph-Stationary reuse
+    exploits (Section 2.2).
     """
+    if family not in (RESNET, MBV3):
+        raise ValueError("locality streams exist for the ResNet- and MobileNetV3-shaped families")
     rng = np.random.default_rng(seed)
-    cur = sample_cfg(RESNET, rng)
+    cur = sample_cfg(family, rng)
     out = [cur]
     for _ in range(n - 1):
         nxt = copy_cfg(cur)
-        if rng.random() < p_local:
+        if rng.random() >= p_local:
+            nxt = sample_cfg(family, rng)
+        elif family == RESNET:
             s = int(rng.integers(4))
             if int(rng.integers(2)) == 0:
                 nxt.depth[s] = RESNET_BASE_DEPTH[s] + _pick(rng, RESNET_EXTRA_DEPTH_SET)
             else:
                 nxt.width[s + 1] = _pick(rng, RESNET_WIDTH_SET)
         else:
-            nxt = sample_cfg(RESNET, rng)
+            s, what = int(rng.integers(5)), int(rng.integers(3))
+            if what == 0:
+                nxt.depth[s] = _pick(rng, MBV3_DEPTH_SET)
+            elif what == 1:
+                nxt.expand[s][int(rng.integers(4))] = _pick(rng, MBV3_EXPAND_SET)
+            else:
+                nxt.kernel[s][int(rng.integers(4))] = _pick(rng, MBV3_KERNEL_SET)
         out.append(nxt)
         cur = nxt
     return out

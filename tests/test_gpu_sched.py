@@ -24,12 +24,13 @@ def _expected(onet, cfgs, cands, q, budget_bytes):
     return float(np.mean(hits)), 2.0 * float(sum(missed)), choices, updates
 
 
-@pytest.mark.parametrize("q,budget,wave", [(4, 0, 0), (1, 48 << 20, 0), (3, 24 << 20, 8), (8, 2 << 20, 4)])
-def test_avgnet_policy_matches_checker(q, budget, wave):
-    _, onet, gnet = gu.nets(wl.RESNET, True)
+@pytest.mark.parametrize("family,q,budget,wave", [(wl.RESNET, 4, 0, 0), (wl.RESNET, 1, 48 << 20, 0), (wl.RESNET, 3, 24 << 20, 8),
+                                                  (wl.RESNET, 8, 2 << 20, 4), (wl.MBV3, 2, 0, 0), (wl.MBV3, 3, 6 << 20, 8)])
+def test_avgnet_policy_matches_checker(family, q, budget, wave):
+    _, onet, gnet = gu.nets(family, True)
     n, res = 26, 64
-    cfgs = wl.markov_stream(n, seed=21 + q)
-    cands = wl.candidate_cfgs(wl.RESNET, 12, seed=5)
+    cfgs = wl.markov_stream(n, seed=21 + q, family=family)
+    cands = wl.candidate_cfgs(family, 12, seed=5)
     d_in = gu.to_device(wl.make_inputs(n, 1, res, seed=2, bf16=True).reshape(n, res, res, 3), True)
     stream = torch.cuda.Stream()
     torch.cuda.synchronize()
