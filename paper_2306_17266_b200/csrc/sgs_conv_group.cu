@@ -328,8 +328,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                 }
                 const int cend = min((int)e.bn_tile, K - f0);  // filters of this tile, a multiple of 8
                 const size_t obase = (size_t)(m < 0 ? 0 : m) * K + f0;
-                // the residual does not depend on the accumulator: the first 32 columns' part is requested
-                // before waiting, every further part one step ahead of its use
+                // the residual does not depend on the accumulator: the first 64 columns' part is requested
+                // before waiting, every further part two steps ahead of its use (a thread then has 8 loads of
+                // 16 bytes in flight: the epilogue of a tile with a residual is bound by their latency)
                 auto load_res = [&](int c0, uint4 *rv) {
 #pragma unroll
                     for (int g = 0; g < 4; g++) {
@@ -337,8 +338,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                         rv[g] = (res && m >= 0 && c < cend) ? __ldg(reinterpret_cast<const uint4 *>(res + obase + c)) : make_uint4(0u, 0u, 0u, 0u);
                     }
                 };
-                uint4 rv[4];
+                uint4 rv[4], rn[4];
                 load_res(0, rv);
+                load_res(32, rn);
                 { ROLE_T0(); group_bar(grp); ROLE_ADD(tbar_); }  // this tile's scale / shift (written during the group's previous tile) are visible
                 const float *sc = scale_g[sb], *sh = shift_g[sb];
                 { ROLE_T0(); if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&acc_full[grp], jj & 1, abort_flag)); ROLE_ADD(tacc_); }
@@ -349,8 +351,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                     for (int c0 = 0; c0 < cend; c0 += 32) {  // warp-uniform bounds
                         uint32_t v[32];
                         tmem_ld32(tacc + c0, v);
-                        uint4 rn[4];
-                        load_res(c0 + 32, rn);
+                        uint4 rf[4];
+                        load_res(c0 + 64, rf);
                         tmem_ld_wait();
                         if (m >= 0) {
 #pragma unroll
@@ -368,7 +370,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                             }
                         }
 #pragma unroll
-                        for (int g = 0; g < 4; g++) rv[g] = rn[g];
+                        for (int g = 0; g < 4; g++) { rv[g] = rn[g]; rn[g] = rf[g]; }
                     }
                 }
                 ROLE_ADD(twork_);
