@@ -773,10 +773,21 @@ __device__ __forceinline__ void scale_body(const SmallEntry &e, int bx, int nbx)
     }
 }
 
-// Squeeze-excite gate of one image of one member (se_gate_kernel's arithmetic): x = pooled vector,
-// w / bias = first FC (K = squeeze width, ld), w2 / bias2 = second FC (ld2), y = gate; C = mid channels.
+// Dot product of 8 bf16 weights (one 16-byte vector) with 8 fp32 values.
+__device__ __forceinline__ float dot8(uint4 wv, float4 x0, float4 x1, float s) {
+    const float2 a = bf2f(wv.x), b = bf2f(wv.y), c = bf2f(wv.z), d = bf2f(wv.w);
+    s = fmaf(a.x, x0.x, s); s = fmaf(a.y, x0.y, s); s = fmaf(b.x, x0.z, s); s = fmaf(b.y, x0.w, s);
+    s = fmaf(c.x, x1.x, s); s = fmaf(c.y, x1.y, s); s = fmaf(d.x, x1.z, s); s = fmaf(d.y, x1.w, s);
+    return s;
+}
+
+// Squeeze-excite gate of one image of one member (se_gate_kernel's arithmetic, other summation order):
+// x = pooled vector, w / bias = first FC (K = squeeze width, ld), w2 / bias2 = second FC (ld2), y = gate;
+// C = mid channels.  Both FCs are a few hundred short dot products: a warp takes JB outputs at a time and
+// issues the 16-byte weight loads of all of them before the first use, so a block pays the memory
+// latency a handful of times instead of once per output.
 __global__ void __launch_bounds__(1024) se_gate_group_kernel(const SmallEntry *__restrict__ tbl) {
-    extern __shared__ float sm[];
+    extern __shared__ __align__(16) float sm[];
     __shared__ SmallEntry e;
     if (threadIdx.x < 8) reinterpret_cast<uint4 *>(&e)[threadIdx.x] = __ldg(reinterpret_cast<const uint4 *>(tbl + blockIdx.y) + threadIdx.x);
     __syncthreads();
@@ -789,20 +800,69 @@ __global__ void __launch_bounds__(1024) se_gate_group_kernel(const SmallEntry *_
     float *gate = static_cast<float *>(e.y);
     for (int c = threadIdx.x; c < mid; c += blockDim.x) gs[c] = g[(size_t)n * mid + c];
     __syncthreads();
-    for (int j = warp; j < sq; j += nw) {
-        float s = 0.f;
-        for (int c = lane; c < mid; c += 32) s = fmaf(__bfloat162float(w1[(size_t)j * e.ld + c]), gs[c], s);
+    const bool vec = ((mid | sq | e.ld | e.ld2) & 7) == 0 && ((reinterpret_cast<uintptr_t>(w1) | reinterpret_cast<uintptr_t>(w2)) & 15) == 0;
+    if (vec) {
+        constexpr int JB = 4;
+        for (int j0 = warp * JB; j0 < sq; j0 += nw * JB) {
+            float s[JB];
 #pragma unroll
-        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0) zs[j] = fmaxf(s + e.bias[j], 0.f);
+            for (int u = 0; u < JB; u++) s[u] = 0.f;
+            for (int c = lane * 8; c < mid; c += 256) {
+                uint4 wv[JB];
+#pragma unroll
+                for (int u = 0; u < JB; u++)
+                    wv[u] = j0 + u < sq ? __ldg(reinterpret_cast<const uint4 *>(w1 + (size_t)(j0 + u) * e.ld + c)) : make_uint4(0u, 0u, 0u, 0u);
+                const float4 x0 = *reinterpret_cast<const float4 *>(gs + c), x1 = *reinterpret_cast<const float4 *>(gs + c + 4);
+#pragma unroll
+                for (int u = 0; u < JB; u++) s[u] = dot8(wv[u], x0, x1, s[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < JB; u++) {
+#pragma unroll
+                for (int o = 16; o; o >>= 1) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
+                if (lane == 0 && j0 + u < sq) zs[j0 + u] = fmaxf(s[u] + e.bias[j0 + u], 0.f);
+            }
+        }
+    } else {
+        for (int j = warp; j < sq; j += nw) {
+            float s = 0.f;
+            for (int c = lane; c < mid; c += 32) s = fmaf(__bfloat162float(w1[(size_t)j * e.ld + c]), gs[c], s);
+#pragma unroll
+            for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (lane == 0) zs[j] = fmaxf(s + e.bias[j], 0.f);
+        }
     }
     __syncthreads();
-    for (int c = warp; c < mid; c += nw) {
-        float s = 0.f;
-        for (int j = lane; j < sq; j += 32) s = fmaf(__bfloat162float(w2[(size_t)c * e.ld2 + j]), zs[j], s);
+    if (vec) {
+        constexpr int JB = 8;
+        for (int c0 = warp * JB; c0 < mid; c0 += nw * JB) {
+            float s[JB];
 #pragma unroll
-        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0) gate[(size_t)n * mid + c] = fminf(fmaxf(s + e.bias2[c] + 3.f, 0.f), 6.f) / 6.f;
+            for (int u = 0; u < JB; u++) s[u] = 0.f;
+            for (int j = lane * 8; j < sq; j += 256) {
+                uint4 wv[JB];
+#pragma unroll
+                for (int u = 0; u < JB; u++)
+                    wv[u] = c0 + u < mid ? __ldg(reinterpret_cast<const uint4 *>(w2 + (size_t)(c0 + u) * e.ld2 + j)) : make_uint4(0u, 0u, 0u, 0u);
+                const float4 x0 = *reinterpret_cast<const float4 *>(zs + j), x1 = *reinterpret_cast<const float4 *>(zs + j + 4);
+#pragma unroll
+                for (int u = 0; u < JB; u++) s[u] = dot8(wv[u], x0, x1, s[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < JB; u++) {
+#pragma unroll
+                for (int o = 16; o; o >>= 1) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
+                if (lane == 0 && c0 + u < mid) gate[(size_t)n * mid + c0 + u] = fminf(fmaxf(s[u] + e.bias2[c0 + u] + 3.f, 0.f), 6.f) / 6.f;
+            }
+        }
+    } else {
+        for (int c = warp; c < mid; c += nw) {
+            float s = 0.f;
+            for (int j = lane; j < sq; j += 32) s = fmaf(__bfloat162float(w2[(size_t)c * e.ld2 + j]), zs[j], s);
+#pragma unroll
+            for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (lane == 0) gate[(size_t)n * mid + c] = fminf(fmaxf(s + e.bias2[c] + 3.f, 0.f), 6.f) / 6.f;
+        }
     }
 }
 
