@@ -361,6 +361,23 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
 sgs_status_t sgs_profile_read(sgs_supernet_t *net, int kernel_class, long long *launches, double *total_ms,
                               double *alg_bytes, double *flops);
 
+/*
+ * Per-launch timing of waves.  While the profile is on, every launch of a wave (sgs_stream_opts_t.wave > 0)
+ * also leaves one record, in issue order, until the next reset (at most 65536 are kept): its kernel class,
+ * the stored layer it ran (index as in sgs_subnet_encode; the first of two for a launch that merges two
+ * layers; -1 for operations without weights: pools, padding, SE scale), how many wave members it served, its
+ * tiles (tensor-core convolutions, else 0), its device time and its algorithmic bytes and useful FLOPs.
+ * sgs_profile_trace copies up to `cap` records to the host array `out` and returns how many exist (-1 on a
+ * bad argument).  sgs_layer_name copies the name of a stored layer (NUL-terminated, truncated to cap - 1
+ * characters) and returns its full length, -1 for a bad argument.
+ */
+typedef struct {
+    int kernel_class, layer, members, tiles;
+    double ms, alg_bytes, flops;
+} sgs_launch_record_t;
+int sgs_profile_trace(sgs_supernet_t *net, sgs_launch_record_t *out, int cap);
+int sgs_layer_name(const sgs_supernet_t *net, int layer, char *out, int cap);
+
 /* Counters by name ("kernel_launches", "plan_hits", "plan_misses", "device_bytes", "tc_convs";
  * diagnostics: "host_us_stream", "host_us_query", "host_us_table", "host_us_graph", "host_us_direct" =
  * accumulated host microseconds spent issuing streams / queries / cache-table updates / graph

@@ -27,7 +27,7 @@ EXPORTS = [
     "sgs_set_option", "sgs_get_counter", "sgs_last_error", "sgs_supernet_free", "sgs_conv2d_sliced", "sgs_device_status",
     "sgs_profile_read", "sgs_conv2d_sliced_static", "sgs_cache_set_candidates", "sgs_cache_set_policy",
     "sgs_sched_create", "sgs_sched_free", "sgs_sched_dims", "sgs_sched_set_table", "sgs_sched_get_table", "sgs_sched_measure",
-    "sgs_sched_step", "sgs_sched_subnet",
+    "sgs_sched_step", "sgs_sched_subnet", "sgs_profile_trace", "sgs_layer_name",
 ]
 
 
@@ -63,6 +63,11 @@ class CacheStats(ctypes.Structure):
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class LaunchRecord(ctypes.Structure):
+    _fields_ = [("kernel_class", ctypes.c_int), ("layer", ctypes.c_int), ("members", ctypes.c_int), ("tiles", ctypes.c_int),
+                ("ms", ctypes.c_double), ("alg_bytes", ctypes.c_double), ("flops", ctypes.c_double)]
 
 
 class Scheduler:
@@ -163,6 +168,8 @@ def lib():
         L.sgs_sched_measure.argtypes = [vp, vp, ci, ci, vp, ci, cs, vp]
         L.sgs_sched_step.argtypes = [vp, ci, vp, vp, vp, vp, vp]
         L.sgs_sched_subnet.argtypes = [vp, ci, vp]
+        L.sgs_profile_trace.argtypes = [vp, vp, ci]
+        L.sgs_layer_name.argtypes = [vp, ci, ctypes.c_char_p, ci]
         L.sgs_num_layers.argtypes = [vp]
         L.sgs_subnet_encode.argtypes = [vp, vp, vp]
         L.sgs_subnet_cost.argtypes = [vp, vp, ci, ci, vp, vp, vp]
@@ -282,6 +289,20 @@ class SuperNet:
         self._check(lib().sgs_subnet_cost(self._h, ctypes.byref(cfg), batch, res, ctypes.addressof(f), ctypes.addressof(w),
                                           ctypes.addressof(a)))
         return f.value, w.value, a.value
+
+    def profile_trace(self):
+        """Per-launch records of the profiled waves: list of dicts with the stored layer's name."""
+        n = lib().sgs_profile_trace(self._h, None, 0)
+        if n < 0:
+            raise SgsError(SGS_EINVAL, "sgs_profile_trace")
+        arr = (LaunchRecord * max(n, 1))()
+        n = min(n, lib().sgs_profile_trace(self._h, ctypes.addressof(arr), n))
+        out, buf = [], ctypes.create_string_buffer(128)
+        for r in arr[:n]:
+            name = buf.value.decode() if r.layer >= 0 and lib().sgs_layer_name(self._h, r.layer, buf, 128) >= 0 else ""
+            out.append({"kernel_class": r.kernel_class, "layer": r.layer, "name": name, "members": r.members, "tiles": r.tiles,
+                        "ms": r.ms, "alg_bytes": r.alg_bytes, "flops": r.flops})
+        return out
 
     def profile_read(self, kernel_class: int):
         n, ms, b, f = ctypes.c_longlong(), ctypes.c_double(), ctypes.c_double(), ctypes.c_double()

@@ -216,6 +216,7 @@ struct sgs_supernet {
     std::vector<Plan *> prof_used;  // plans run since the last fold, in order
     double prof_ms[4] = {0, 0, 0, 0}, prof_bytes[4] = {0, 0, 0, 0}, prof_flops[4] = {0, 0, 0, 0};
     long long prof_launches[4] = {0, 0, 0, 0};
+    std::vector<sgs_launch_record_t> prof_trace;  // waves: one record per launch of the profiled passes (bounded)
     mutable std::string err;
     size_t elem() const { return dtype == SGS_BF16 ? 2 : 4; }
     int idx(const std::string &n) const {
@@ -1315,7 +1316,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
     const int G = std::min(o.wave, TC_GROUP_MAX_ENTRIES);
     // per-launch timing (option "profile") wants the launches of one wave at a time
     const int W = net->profile ? 1 : std::max(1, std::min(o.concurrency ? o.concurrency : 2, 8));
-    struct ProfRec { cudaEvent_t e0, e1; int cls; double bytes, flops; };
+    struct ProfRec { cudaEvent_t e0, e1; int cls; double bytes, flops; int layer, members, tiles; };
     std::vector<ProfRec> prof;
     sgs_status_t rc = ensure_slots(net, G * W);
     if (rc != SGS_OK) return rc;
@@ -1536,9 +1537,9 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
         // Profiling brackets every launch with events.  A sleeping kernel first holds the stream while the
         // host queues the whole wave, so that the intervals hold device time, not launch latency.
         if (net->profile) CU(launch_delay(1500, ws));
-        auto prof_begin = [&](int cls, double bytes, double fl) -> sgs_status_t {
+        auto prof_begin = [&](int cls, double bytes, double fl, int layer, int members, int tiles) -> sgs_status_t {
             if (!net->profile) return SGS_OK;
-            ProfRec r{nullptr, nullptr, cls, bytes, fl};
+            ProfRec r{nullptr, nullptr, cls, bytes, fl, layer, members, tiles};
             CU(cudaEventCreate(&r.e0));
             CU(cudaEventCreate(&r.e1));
             CU(cudaEventRecord(r.e0, ws));
@@ -1548,6 +1549,10 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
         auto prof_end = [&]() -> sgs_status_t {
             if (net->profile) CU(cudaEventRecord(prof.back().e1, ws));
             return SGS_OK;
+        };
+        auto first_layer = [&](int rank) -> int {  // stored layer of the launch's first member (-1: an op without weights)
+            const auto &b = buckets[(size_t)rank];
+            return b.empty() ? -1 : plans[b.front().first]->ops[(size_t)b.front().second].layer;
         };
         auto bucket_cost = [&](int rank, bool tc, double *bytes, double *fl) {
             *bytes = 0; *fl = 0;
@@ -1565,7 +1570,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                 // 64 members or 248 tensor maps do not occur while profiling waves of <= 64)
                 bucket_cost(L.rank, true, &pb, &pf);
                 if (L.rank2 >= 0) { double b2 = 0, f2 = 0; bucket_cost(L.rank2, true, &b2, &f2); pb += b2; pf += f2; }
-                if ((rc = prof_begin(0, pb, pf)) != SGS_OK) break;
+                if ((rc = prof_begin(0, pb, pf, first_layer(L.rank), L.group->members(), L.group->tiles())) != SGS_OK) break;
                 CU(L.group->launch(net->cache_tbl, net->sms, ws));
                 if ((rc = prof_end()) != SGS_OK) break;
                 net->kernel_launches++;
@@ -1573,7 +1578,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             }
             if (L.small_kind == OP_DW) {
                 bucket_cost(L.rank, false, &pb, &pf);
-                if ((rc = prof_begin(2, pb, pf)) != SGS_OK) break;
+                if ((rc = prof_begin(2, pb, pf, first_layer(L.rank), L.count, 0)) != SGS_OK) break;
                 cudaError_t de = launch_dw_group(cx.h_tbl + L.off, cx.d_tbl + L.off, L.count, ws);
                 if (de == cudaErrorNotSupported) {
                     // (not expected after the checks above) run these members one by one
@@ -1591,7 +1596,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             }
             if (L.small_kind >= 0) {
                 bucket_cost(L.rank, false, &pb, &pf);
-                if ((rc = prof_begin(3, pb, pf)) != SGS_OK) break;
+                if ((rc = prof_begin(3, pb, pf, first_layer(L.rank), L.count, 0)) != SGS_OK) break;
                 CU(launch_small(L.small_kind, reinterpret_cast<const SmallEntry *>(cx.h_tbl + L.off),
                                 reinterpret_cast<const SmallEntry *>(cx.d_tbl + L.off), L.count, ws));
                 if ((rc = prof_end()) != SGS_OK) break;
@@ -1641,6 +1646,12 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
         float ms = 0;
         if (rc == SGS_OK && r.e1 && cudaEventElapsedTime(&ms, r.e0, r.e1) == cudaSuccess) {
             net->prof_ms[r.cls] += ms; net->prof_bytes[r.cls] += r.bytes; net->prof_flops[r.cls] += r.flops; net->prof_launches[r.cls]++;
+            if (net->prof_trace.size() < 65536) {
+                sgs_launch_record_t tr;
+                tr.kernel_class = r.cls; tr.layer = r.layer; tr.members = r.members; tr.tiles = r.tiles;
+                tr.ms = ms; tr.alg_bytes = r.bytes; tr.flops = r.flops;
+                net->prof_trace.push_back(tr);
+            }
         }
         if (r.e0) cudaEventDestroy(r.e0);
         if (r.e1) cudaEventDestroy(r.e1);
@@ -2084,6 +2095,19 @@ sgs_status_t sgs_profile_read(sgs_supernet_t *net, int kernel_class, long long *
     return SGS_OK;
 }
 
+int sgs_profile_trace(sgs_supernet_t *net, sgs_launch_record_t *out, int cap) {
+    if (!net || cap < 0 || (cap && !out)) return -1;
+    const int n = (int)std::min<size_t>(net->prof_trace.size(), (size_t)cap);
+    if (n) std::memcpy(out, net->prof_trace.data(), (size_t)n * sizeof(sgs_launch_record_t));
+    return (int)net->prof_trace.size();
+}
+
+int sgs_layer_name(const sgs_supernet_t *net, int layer, char *out, int cap) {
+    if (!net || layer < 0 || layer >= (int)net->layers.size() || !out || cap < 1) return -1;
+    std::snprintf(out, (size_t)cap, "%s", net->layers[(size_t)layer].name.c_str());
+    return (int)net->layers[(size_t)layer].name.size();
+}
+
 sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long value) {
     if (!net || !name) return SGS_EINVAL;
     std::string n(name);
@@ -2102,6 +2126,7 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
         net->profile = value != 0;
         if (value == 2 || value == 0)
             for (int i = 0; i < 4; i++) { net->prof_ms[i] = net->prof_bytes[i] = net->prof_flops[i] = 0; net->prof_launches[i] = 0; }
+            net->prof_trace.clear();
         return SGS_OK;
     }
     return fail(net, SGS_EINVAL, "unknown option " + n);

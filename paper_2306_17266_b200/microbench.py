@@ -102,14 +102,55 @@ def bench_dw(shape, iters=20, once=0):
     return {"shape": shape, "us": us, "gbs": nbytes / us / 1e3, "mbytes": nbytes / 1e6}
 
 
+def wave_trace(family, wave, queries, res, batch):
+    """Per-layer device time of a stream run as waves (one wave at a time, every launch between two events)."""
+    from . import workload as wl
+    fam = {"resnet": wl.RESNET, "mbv3": wl.MBV3}[family]
+    net = sgs.SuperNet(fam, wl.make_blob(fam, seed=0, bf16_weights=True), sgs.SGS_BF16)
+    cfgs = wl.cfg_array(wl.uniform_stream(fam, queries, seed=2 if fam == wl.RESNET else 3))
+    x = torch.from_numpy(wl.make_inputs(queries, batch, res, seed=1, bf16=True).reshape(queries * batch, res, res, 3)).cuda().to(torch.bfloat16).contiguous()
+    out = torch.zeros((queries * batch, 1000), dtype=torch.float32, device="cuda")
+    st = torch.cuda.Stream()
+    opts = sgs.StreamOpts(cache_enabled=1, window_q=4, record_latency=0, concurrency=1, wave=wave)
+    for _ in range(2):
+        net.stream_run(cfgs, x.data_ptr(), batch, res, out.data_ptr(), opts, st.cuda_stream)
+    net.set_option("profile", 2)
+    net.stream_run(cfgs, x.data_ptr(), batch, res, out.data_ptr(), opts, st.cuda_stream)
+    recs = net.profile_trace()
+    net.set_option("profile", 0)
+    rows, order = {}, []
+    for r in recs:
+        key = (r["kernel_class"], r["name"] or "(no weights)")
+        if key not in rows:
+            rows[key] = {"n": 0, "ms": 0.0, "bytes": 0.0, "flops": 0.0, "members": 0, "tiles": 0}
+            order.append(key)
+        a = rows[key]
+        a["n"] += 1; a["ms"] += r["ms"]; a["bytes"] += r["alg_bytes"]; a["flops"] += r["flops"]; a["members"] += r["members"]; a["tiles"] += r["tiles"]
+    total = sum(a["ms"] for a in rows.values())
+    names = ["conv_tc", "conv_cuda_core", "depthwise", "other"]
+    print(f"{family}: {queries} queries, waves of {wave}, batch {batch}, {res}x{res}: {len(recs)} launches, {total:.2f} ms of kernel time")
+    for key in order:
+        a = rows[key]
+        print(f"{names[key[0]]:10s} {key[1]:28s} launches {a['n']:4d}  members {a['members'] / a['n']:5.1f}  tiles {a['tiles'] / a['n']:7.1f}  "
+              f"{1e3 * a['ms'] / a['n']:7.1f} us  {100 * a['ms'] / total:5.1f} %  {a['bytes'] / a['ms'] / 1e6:8.1f} GB/s  {a['flops'] / a['ms'] / 1e9:7.1f} TFLOP/s")
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["conv", "dw"])
+    ap.add_argument("kind", choices=["conv", "dw", "trace"])
+    ap.add_argument("--family", default="resnet", choices=["resnet", "mbv3"])
+    ap.add_argument("--wave", type=int, default=32)
+    ap.add_argument("--queries", type=int, default=128)
+    ap.add_argument("--res", type=int, default=224)
+    ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--preset", default=None)
     ap.add_argument("--shape", default=None, help="comma-separated shape")
     ap.add_argument("--once", type=int, default=0, help="only run this many launches (profiling)")
     ap.add_argument("--split-off", type=int, default=0)
     args = ap.parse_args()
+    if args.kind == "trace":
+        wave_trace(args.family, args.wave, args.queries, args.res, args.batch)
+        return
     if args.shape:
         shapes = [tuple(int(v) for v in args.shape.split(","))]
     else:
