@@ -119,3 +119,38 @@ def test_bench_wave_configuration_sampled_against_checker():
     print(f"wave configuration: worst rel err {worst:.2e}, top-1 agreement {strict}/{len(sample)}")
     assert worst <= TOL_BF16
     assert strict >= len(sample) - 1
+
+
+def test_profile_trace_lists_every_launch_of_a_wave():
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    n, res, G = 8, 64, 4
+    cfgs = wl.uniform_stream(wl.RESNET, n, seed=12)
+    d_in = gu.to_device(wl.make_inputs(n, 1, res, seed=2, bf16=True).reshape(n, res, res, 3), True)
+    d_out = torch.zeros((n, 1000), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    opts = sgs.StreamOpts(cache_enabled=1, window_q=2, record_latency=0, concurrency=1, wave=G)
+    plain = gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+    ref = d_out.cpu().numpy().copy()
+    gnet.set_option("profile", 2)
+    try:
+        st = gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+        trace = gnet.profile_trace()
+        by_class = [gnet.profile_read(c) for c in range(4)]
+    finally:
+        gnet.set_option("profile", 0)
+    np.testing.assert_array_equal(d_out.cpu().numpy(), ref)            # profiling does not change results
+    assert len(trace) == st.kernel_launches == plain.kernel_launches   # one record per launch, in issue order
+    for c in range(4):
+        rows = [r for r in trace if r["kernel_class"] == c]
+        assert len(rows) == by_class[c]["launches"]
+        assert abs(sum(r["ms"] for r in rows) - by_class[c]["total_ms"]) < 1e-6 * max(1.0, by_class[c]["total_ms"])
+        assert abs(sum(r["flops"] for r in rows) - by_class[c]["flops"]) <= 1e-9 * max(1.0, by_class[c]["flops"])
+    conv = [r for r in trace if r["kernel_class"] == 0]
+    assert conv and all(r["ms"] > 0 and 1 <= r["members"] <= 2 * G and r["tiles"] >= r["members"] and r["name"] for r in conv)
+    assert conv[0]["name"] == "stem" and trace[-1]["name"] == "fc"
+    # useful FLOPs of the trace = those of the stream
+    assert abs(sum(r["flops"] for r in trace) - st.useful_flops) <= 1e-6 * st.useful_flops
+    gnet.set_option("profile", 2)                                      # reset empties the trace
+    gnet.set_option("profile", 0)
+    assert gnet.profile_trace() == []
