@@ -7,6 +7,7 @@
 #include "sgs_internal.h"
 
 #include <algorithm>
+#include <cooperative_groups.h>
 
 namespace sgs {
 
@@ -785,16 +786,24 @@ __device__ __forceinline__ float dot8(uint4 wv, float4 x0, float4 x1, float s) {
 // x = pooled vector, w / bias = first FC (K = squeeze width, ld), w2 / bias2 = second FC (ld2), y = gate;
 // C = mid channels.  Both FCs are a few hundred short dot products: a warp takes JB outputs at a time and
 // issues the 16-byte weight loads of all of them before the first use, so a block pays the memory
-// latency a handful of times instead of once per output.
-__global__ void __launch_bounds__(1024) se_gate_group_kernel(const SmallEntry *__restrict__ tbl) {
+// latency a handful of times instead of once per output.  The gate of one image is the work of a cluster
+// of SE_SPLIT blocks (one block alone streams both weight matrices through a single SM): every block
+// computes a share of the first FC's outputs and writes them into all the blocks' shared memory, and
+// after the cluster barrier a share of the second FC's.
+constexpr int SE_SPLIT = 4, SE_THREADS = 512;
+__global__ void __cluster_dims__(SE_SPLIT, 1, 1) __launch_bounds__(SE_THREADS) se_gate_group_kernel(const SmallEntry *__restrict__ tbl) {
     extern __shared__ __align__(16) float sm[];
     __shared__ SmallEntry e;
+    cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
+    const int rank = (int)cluster.block_rank();
     if (threadIdx.x < 8) reinterpret_cast<uint4 *>(&e)[threadIdx.x] = __ldg(reinterpret_cast<const uint4 *>(tbl + blockIdx.y) + threadIdx.x);
     __syncthreads();
     const int mid = e.C, sq = e.K;
     float *gs = sm, *zs = sm + mid;
-    const int n = blockIdx.x, lane = threadIdx.x % 32, warp = threadIdx.x / 32, nw = blockDim.x / 32;
-    if (n >= e.N) return;
+    const int n = blockIdx.x / SE_SPLIT, lane = threadIdx.x % 32, nwb = blockDim.x / 32;
+    const int warp = rank * nwb + threadIdx.x / 32, nw = nwb * SE_SPLIT;  // warps of the whole cluster share the outputs
+    if (n >= e.N) return;  // (the same for every block of a cluster)
+    float *zs_peer = cluster.map_shared_rank(zs, lane < SE_SPLIT ? lane : 0);  // lanes 0..SE_SPLIT-1 each write one block's copy
     const float *g = static_cast<const float *>(e.x);
     const __nv_bfloat16 *w1 = static_cast<const __nv_bfloat16 *>(e.w), *w2 = static_cast<const __nv_bfloat16 *>(e.w2);
     float *gate = static_cast<float *>(e.y);
@@ -820,7 +829,7 @@ __global__ void __launch_bounds__(1024) se_gate_group_kernel(const SmallEntry *_
             for (int u = 0; u < JB; u++) {
 #pragma unroll
                 for (int o = 16; o; o >>= 1) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
-                if (lane == 0 && j0 + u < sq) zs[j0 + u] = fmaxf(s[u] + e.bias[j0 + u], 0.f);
+                if (lane < SE_SPLIT && j0 + u < sq) zs_peer[j0 + u] = fmaxf(s[u] + e.bias[j0 + u], 0.f);
             }
         }
     } else {
@@ -829,10 +838,10 @@ __global__ void __launch_bounds__(1024) se_gate_group_kernel(const SmallEntry *_
             for (int c = lane; c < mid; c += 32) s = fmaf(__bfloat162float(w1[(size_t)j * e.ld + c]), gs[c], s);
 #pragma unroll
             for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            if (lane == 0) zs[j] = fmaxf(s + e.bias[j], 0.f);
+            if (lane < SE_SPLIT) zs_peer[j] = fmaxf(s + e.bias[j], 0.f);
         }
     }
-    __syncthreads();
+    cluster.sync();  // every block's zs is complete (and no block leaves while others may still write into it)
     if (vec) {
         constexpr int JB = 8;
         for (int c0 = warp * JB; c0 < mid; c0 += nw * JB) {
@@ -1074,7 +1083,7 @@ cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int
         if (!d) return cudaErrorInvalidValue;
         int nimg = 0, fl = 0;
         for (int i = 0; i < n; i++) { nimg = std::max(nimg, h[i].N); fl = std::max(fl, h[i].C + h[i].K); }
-        se_gate_group_kernel<<<dim3((unsigned)nimg, (unsigned)n), 1024, (size_t)fl * sizeof(float), st>>>(d);
+        se_gate_group_kernel<<<dim3((unsigned)nimg * SE_SPLIT, (unsigned)n), SE_THREADS, (size_t)fl * sizeof(float), st>>>(d);
         return cudaGetLastError();
     }
     case OP_LINEAR: {
