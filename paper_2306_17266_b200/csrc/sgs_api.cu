@@ -1995,6 +1995,7 @@ sgs_status_t sgs_sched_measure(sgs_sched_t *s, const void *d_input, int batch, i
     if (!s) return SGS_EINVAL;
     sgs_supernet *net = s->net;
     if (!d_input || !d_logits || batch <= 0 || res < 8 || res > 1024 || reps < 1 || reps > 1000) return fail(net, SGS_EINVAL, "bad argument");
+    if ((int)net->cache.cand.size() != s->M) return fail(net, SGS_EINVAL, "the candidate set changed under the scheduler");
     DeviceGuard guard(net->device);
     if (!guard.ok) return fail(net, SGS_ECUDA, "cudaSetDevice failed");
     cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -2040,6 +2041,7 @@ sgs_status_t sgs_sched_step(sgs_sched_t *s, int n, const int *policy, const doub
                             int *cache_state) {
     if (!s) return SGS_EINVAL;
     if (n < 0 || (n && (!policy || !a_t || !l_t || !subnet))) return fail(s->net, SGS_EINVAL, "bad argument");
+    if ((int)s->net->cache.cand.size() != s->M) return fail(s->net, SGS_EINVAL, "the candidate set changed under the scheduler");
     for (int t = 0; t < n; t++)
         if (policy[t] != SGS_STRICT_ACCURACY && policy[t] != SGS_STRICT_LATENCY) return fail(s->net, SGS_EINVAL, "unknown query policy");
     const int before = s->state;

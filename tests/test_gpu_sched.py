@@ -178,6 +178,12 @@ def test_scheduler_argument_errors():
             s.set_table(np.zeros((2, 2)))
         sub, state = s.step([], [], [])
         assert len(sub) == 0
+        gnet.cache_set_candidates(cfgs)                      # another set under a live scheduler: refused, not followed
+        with pytest.raises(sgs.SgsError, match="EINVAL"):
+            s.step([0], [0.0], [0.0])
+        gnet.cache_set_candidates(cfgs[:2])
+        sub, _ = s.step([0], [0.0], [0.0])
+        assert len(sub) == 1
         s.close()
     finally:
         gnet.cache_set_candidates([])
