@@ -53,7 +53,11 @@ struct __align__(16) GroupEntry {
     short bn_tile;           // MMA columns of a full tile
     short pix_rows;          // rows of the pixel box (bw * bh * bn)
     short pad0_;
-    unsigned char k, stride, p, act, swap, kw, pad1_[2];  // k x kw taps
+    unsigned char k, stride, p, act, swap, kw;  // k x kw taps
+    // Two members with at most 64 output pixels each can share a tile: the first ("pair") owns the tile's
+    // geometry, filters and weight map and takes MMA rows 0..63, the entry after it ("second") takes rows
+    // 64..127 with its own activation map, outputs and filter count (not larger than the first's).
+    unsigned char pair, second;
     int pad2_[3];
 };
 static_assert(sizeof(GroupEntry) == TC_GROUP_ENTRY_BYTES, "entry size");
@@ -71,7 +75,12 @@ __device__ __forceinline__ int find_entry_serial(const GroupEntry *es, int n, in
         const int mid = (lo + hi + 1) >> 1;
         if (es[mid].tile_begin <= t) lo = mid; else hi = mid - 1;
     }
-    return lo;
+    return es[lo].second ? lo - 1 : lo;
+}
+// The entry that owns tile t's geometry (the first member of a pair); the whole warp calls it.
+__device__ __forceinline__ int tile_entry(const GroupEntry *es, int n, int t, int lane) {
+    const int i = find_entry(es, n, t, lane);
+    return es[i].second ? i - 1 : i;
 }
 
 // Named barrier of one epilogue group (4 warps): id 1 or 2.
@@ -150,7 +159,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         long long tw_ = 0; (void)tw_;
         const long long tk0_ = clock64(); (void)tk0_;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
+            const GroupEntry &e = es[tile_entry(es, n_entries, t, lane)];
             const int nt = (t - e.tile_begin) / e.mtiles;
             const int wrows = e.swap ? 128 : e.bn_tile;  // rows of the weight box
             const int f0 = nt * wrows;
@@ -194,12 +203,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         const long long tk0_ = clock64(); (void)tk0_;
         { ROLE_T0(); pdl_wait(); ROLE_ADD(tpdl_); }  // activations (and the buffers this layer overwrites) belong to the previous layers until here
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
+            const GroupEntry &e = es[tile_entry(es, n_entries, t, lane)];
             const int mt = (t - e.tile_begin) % e.mtiles;
             const int n0 = (mt / e.tiles_hw) * e.bn, h0 = ((mt % e.tiles_hw) / e.tiles_w) * e.bh, w0 = (mt % e.tiles_w) * e.bw;
             const uint32_t pix_bytes = (uint32_t)(e.pix_rows * CHUNK_C * 2);
             uint8_t *dst0 = smem + (e.swap ? G_X_BYTES : 0);
             const CUtensorMap *map_a = &P.maps[e.map_a];
+            const uint32_t pix_bytes2 = e.pair ? (uint32_t)((&e)[1].pix_rows * CHUNK_C * 2) : 0u;
+            const CUtensorMap *map_a2 = &P.maps[e.pair ? (&e)[1].map_a : e.map_a];
             const int k = e.k, kw = e.kw, cchunks = e.cchunks, pad = e.p, stride = e.stride;
             for (int r = 0; r < k && ok; r++) {
                 for (int sx = 0; sx < kw && ok; sx++) {
@@ -212,8 +223,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                         { ROLE_T0(); if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag)); ROLE_ADD(tw_); }
                         if (!ok) break;
                         if (elect_one()) {
-                            mbar_expect_tx(&full_bar[s], pix_bytes);
+                            mbar_expect_tx(&full_bar[s], pix_bytes + pix_bytes2);
                             tma_load_4d(dst0 + s * stage_bytes, m, &full_bar[s], c0, cw, ch, n0);
+                            // (a pair is a single tile of a stride-1 layer: same tap offsets, box origin 0)
+                            if (pix_bytes2) tma_load_4d(dst0 + s * stage_bytes + 64 * CHUNK_C * 2, map_a2, &full_bar[s], c0, cw, ch, n0);
                         }
                         __syncwarp();
                         if (++s == n_stages) { s = 0; phase ^= 1; wrapped = true; }
@@ -235,7 +248,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         long long tfull_ = 0, tacc_ = 0; (void)tfull_; (void)tacc_;
         const long long tk0_ = clock64(); (void)tk0_;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, j++) {
-            const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
+            const GroupEntry &e = es[tile_entry(es, n_entries, t, lane)];
             const int nt = (t - e.tile_begin) / e.mtiles;
             // MMA shape: 128 rows; columns = this tile's filters (normal) or the member's pixels (swapped),
             // rounded up to 16; bf16 x bf16 -> fp32, both operands K-major
@@ -277,7 +290,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         // side; a thread handles one accumulator row and all of the tile's columns, 32 at a time.
         const int quad = warp & 3;                // tensor-memory lane quadrant this warp may read
         const int grp = (warp - 2) >> 2;          // epilogue group = accumulator buffer
-        const int row = quad * 32 + lane;         // accumulator row: output pixel (normal) or filter (swapped)
+        const int row_all = quad * 32 + lane;     // accumulator row: output pixel (normal) or filter (swapped)
         const int et = (threadIdx.x - 64) & 127;  // thread within the group
         float(*scale_g)[G_ACC_COLS] = scale_s[grp];
         float(*shift_g)[G_ACC_COLS] = shift_s[grp];
@@ -290,7 +303,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         auto fetch_bn = [&](int tile, float *v) {
             v[0] = v[1] = v[2] = v[3] = 0.f;
             if (tile >= total_tiles) return;
-            const GroupEntry &e = es[find_entry(es, n_entries, tile, lane)];
+            const GroupEntry &e = es[tile_entry(es, n_entries, tile, lane)];
             if (e.swap) return;
             const int f = ((tile - e.tile_begin) / e.mtiles) * e.bn_tile + et;
             if (et < e.bn_tile && f < e.K) { v[0] = __ldg(e.scale + f); v[1] = __ldg(e.shift + f); }
@@ -306,8 +319,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         }
         int jj = 0;  // tiles this group has taken
         for (int t = (int)blockIdx.x + grp * (int)gridDim.x; t < total_tiles; t += stride2, jj++) {
-            const GroupEntry &e = es[find_entry(es, n_entries, t, lane)];
-            const int local = t - e.tile_begin, nt = local / e.mtiles, mt = local % e.mtiles;
+            const GroupEntry &e0 = es[tile_entry(es, n_entries, t, lane)];
+            const int local = t - e0.tile_begin, nt = local / e0.mtiles, mt = local % e0.mtiles;
+            // rows 64..127 of a pair's tile belong to the second member (a warp lies on one side)
+            const bool second_half = e0.pair && quad >= 2;
+            const GroupEntry &e = second_half ? (&e0)[1] : e0;
+            const int row = second_half ? row_all - 64 : row_all;
             const int K = e.K, act = e.act;
             const __nv_bfloat16 *res = e.res;
             __nv_bfloat16 *y = e.y;
@@ -318,7 +335,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             if (!e.swap) {
                 // ---- normal tile: this thread owns output pixel `m`, columns are filters
                 const int n0 = (mt / e.tiles_hw) * e.bn, h0 = ((mt % e.tiles_hw) / e.tiles_w) * e.bh, w0 = (mt % e.tiles_w) * e.bw;
-                const int f0 = nt * e.bn_tile;
+                const int f0 = nt * e0.bn_tile;
                 int m;
                 {
                     const int dn = row / (e.bh * e.bw), dhh = (row / e.bw) % e.bh, dww = row % e.bw;
@@ -326,7 +343,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                     const bool valid = row < e.pix_rows && n < e.N && h < e.Ho && w < e.Wo;
                     m = valid ? (int)(((size_t)n * e.Ho + h) * e.Wo + w) : -1;
                 }
-                const int cend = min((int)e.bn_tile, K - f0);  // filters of this tile, a multiple of 8
+                const int cend = min((int)e0.bn_tile, K - f0);  // filters of this tile, a multiple of 8 (<= 0: none of this member's)
                 const size_t obase = (size_t)(m < 0 ? 0 : m) * K + f0;
                 // the residual does not depend on the accumulator: the first 64 columns' part is requested
                 // before waiting, every further part two steps ahead of its use (a thread then has 8 loads of
@@ -501,8 +518,26 @@ void GroupLaunch::add(void *host_entry, const TcConvPlan &pl, const ConvArgs &a)
     e.bn_tile = (short)(pl.swap ? (e.pix_rows + 15) / 16 * 16 : pl.bn_tile);
     e.k = (unsigned char)p.k; e.kw = (unsigned char)pl.kw; e.stride = (unsigned char)p.stride; e.p = (unsigned char)p.p; e.act = (unsigned char)p.act;
     if ((pl.swap ? e.pix_rows : e.bn_tile) > 128) impl->wide = true;
-    std::memcpy(host_entry, &e, sizeof e);
     impl->prm.n_entries++;
+    // Pairing: this member and the previous one of the launch each fit the lower / upper half of a tile's 128
+    // rows, run the same stored layer with stride 1, and one's slice contains the other's (filters and
+    // channels): they share the larger one's tiles and weight copies.
+    auto half = [](const GroupEntry &g) { return !g.swap && g.mtiles == 1 && g.pix_rows <= 64 && g.stride == 1 && g.kw == g.k; };
+    GroupEntry *prev = impl->prm.n_entries >= 2 ? static_cast<GroupEntry *>(host_entry) - 1 : nullptr;
+    if (prev && !a.win && half(e) && half(*prev) && !prev->pair && !prev->second && prev->layer == e.layer && prev->k == e.k &&
+        prev->act == e.act && ((prev->K >= e.K && prev->C >= e.C) || (e.K >= prev->K && e.C >= prev->C))) {
+        GroupEntry first = *prev, second = e;
+        if (!(prev->K >= e.K && prev->C >= e.C)) { first = e; second = *prev; }
+        first.tile_begin = second.tile_begin = prev->tile_begin;
+        first.pair = 1; first.second = 0;
+        second.pair = 0; second.second = 1;
+        const int ntiles = (first.K + first.bn_tile - 1) / first.bn_tile;
+        impl->prm.total_tiles = first.tile_begin + ntiles;
+        *prev = first;
+        std::memcpy(host_entry, &second, sizeof second);
+        return;
+    }
+    std::memcpy(host_entry, &e, sizeof e);
     impl->prm.total_tiles += e.mtiles * (int)pl.grid.y;
 }
 

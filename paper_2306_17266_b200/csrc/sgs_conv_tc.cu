@@ -402,7 +402,9 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
     if (flat) {
         // 1x1 stride 1: the activation tensor is a plain [M][C] matrix, tiles are 128 consecutive pixels
         const uint64_t M = (uint64_t)a.N * a.H * a.W;
-        p.bw = swap ? (int)M : TILE_M; p.bh = 1; p.bn = 1;
+        // (a member of a grouped launch with fewer than 128 pixels gets a box of exactly its pixels, so that
+        // two such members can share the 128 rows of a tile)
+        p.bw = swap ? (int)M : a.throughput == 2 ? (int)std::min<uint64_t>(M, TILE_M) : TILE_M; p.bh = 1; p.bn = 1;
         p.N = 1; p.Ho = 1; p.Wo = (int)M;
         uint64_t dims[4] = {C, M, 1, 1}, str[3] = {C * eb, M * C * eb, M * C * eb};
         uint32_t box[4] = {CHUNK_C, (uint32_t)p.bw, 1, 1};

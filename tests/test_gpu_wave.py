@@ -147,10 +147,36 @@ def test_profile_trace_lists_every_launch_of_a_wave():
         assert abs(sum(r["ms"] for r in rows) - by_class[c]["total_ms"]) < 1e-6 * max(1.0, by_class[c]["total_ms"])
         assert abs(sum(r["flops"] for r in rows) - by_class[c]["flops"]) <= 1e-9 * max(1.0, by_class[c]["flops"])
     conv = [r for r in trace if r["kernel_class"] == 0]
-    assert conv and all(r["ms"] > 0 and 1 <= r["members"] <= 2 * G and r["tiles"] >= r["members"] and r["name"] for r in conv)
+    assert conv and all(r["ms"] > 0 and 1 <= r["members"] <= 2 * G and 2 * r["tiles"] >= r["members"] and r["name"] for r in conv)   # (two small members may share a tile)
     assert conv[0]["name"] == "stem" and trace[-1]["name"] == "fc"
     # useful FLOPs of the trace = those of the stream
     assert abs(sum(r["flops"] for r in trace) - st.useful_flops) <= 1e-6 * st.useful_flops
     gnet.set_option("profile", 2)                                      # reset empties the trace
     gnet.set_option("profile", 0)
     assert gnet.profile_trace() == []
+
+
+@pytest.mark.parametrize("family", [wl.RESNET, wl.MBV3])
+def test_members_sharing_a_tile_at_7x7_maps(family):
+    # at 224x224 the last stage works on 7x7 maps: two members of a wave then share the 128 rows of a tile
+    # (the one with the larger slice owns the weight copies).  Results must not depend on who shares with whom.
+    _, onet, gnet = gu.nets(family, True)
+    n, res = 7, 224
+    cfgs = wl.uniform_stream(family, n, seed=31)
+    cfgs[2] = wl.extreme_cfg(family, True)      # the largest and the smallest SubNet side by side
+    cfgs[3] = wl.extreme_cfg(family, False)
+    x = wl.make_inputs(n, 1, res, seed=4, bf16=True).reshape(n, res, res, 3)
+    d_in = gu.to_device(x, True)
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs = []
+    for G in (1, 7, 2):
+        d_out = torch.zeros((n, 1000), dtype=torch.float32, device="cuda")
+        opts = sgs.StreamOpts(cache_enabled=1, window_q=2, record_latency=0, concurrency=2, wave=G)
+        gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+        outs.append(d_out.cpu().numpy())
+    np.testing.assert_array_equal(outs[1], outs[0])     # waves of 7 (pairs) against waves of 1 (no pairs)
+    np.testing.assert_array_equal(outs[2], outs[0])
+    for t in (2, 3, 5):
+        ref = onet.forward(cfgs[t], x[t:t + 1], oracle.BF16_STORE)
+        assert gu.rel_err(outs[1][t:t + 1], ref) < 2e-2
