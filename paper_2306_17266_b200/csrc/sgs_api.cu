@@ -1417,7 +1417,35 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             if (b.empty() || merged[(size_t)r]) continue;
             GroupLaunch *g = nullptr;
             const size_t first_launch = launches.size();
-            for (const auto &mo : b) {
+            // Members with at most 64 output pixels can share a tile in pairs if one's slice (filters and channels)
+            // contains the other's, and a pair is two consecutive records: order such a bucket so that every
+            // member is followed by the largest not yet placed member it contains.
+            std::vector<std::pair<int, int>> order(b.begin(), b.end());
+            {
+                const Op &o0 = plans[b[0].first]->ops[(size_t)b[0].second];
+                if (o0.type == OP_CONV && o0.impl == 1 && (long long)o0.conv.N * o0.conv.Ho * o0.conv.Wo <= 64 && b.size() > 2) {
+                    auto opof = [&](const std::pair<int, int> &mo) -> const Op & { return plans[mo.first]->ops[(size_t)mo.second]; };
+                    std::stable_sort(order.begin(), order.end(), [&](const std::pair<int, int> &x, const std::pair<int, int> &y) {
+                        const ConvArgs &cx_ = opof(x).conv, &cy_ = opof(y).conv;
+                        return cx_.K != cy_.K ? cx_.K > cy_.K : cx_.C > cy_.C;
+                    });
+                    std::vector<std::pair<int, int>> placed;
+                    std::vector<char> used_m(order.size(), 0);
+                    for (size_t i = 0; i < order.size(); i++) {
+                        if (used_m[i]) continue;
+                        used_m[i] = 1;
+                        placed.push_back(order[i]);
+                        for (size_t j = i + 1; j < order.size(); j++) {
+                            if (used_m[j] || opof(order[j]).conv.C > opof(order[i]).conv.C) continue;
+                            used_m[j] = 1;
+                            placed.push_back(order[j]);
+                            break;
+                        }
+                    }
+                    order.swap(placed);
+                }
+            }
+            for (const auto &mo : order) {
                 Plan *pl = plans[mo.first];
                 const Op &op = pl->ops[(size_t)mo.second];
                 if (op.type != OP_CONV || op.impl != 1) continue;  // launched per member below
