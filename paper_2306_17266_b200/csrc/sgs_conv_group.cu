@@ -225,8 +225,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                         if (elect_one()) {
                             mbar_expect_tx(&full_bar[s], pix_bytes + pix_bytes2);
                             tma_load_4d(dst0 + s * stage_bytes, m, &full_bar[s], c0, cw, ch, n0);
-                            // (a pair is a single tile of a stride-1 layer: same tap offsets, box origin 0)
-                            if (pix_bytes2) tma_load_4d(dst0 + s * stage_bytes + 64 * CHUNK_C * 2, map_a2, &full_bar[s], c0, cw, ch, n0);
+                            // (a pair is a single tile of one layer: same tap offsets and parity view, box origin 0)
+                            if (pix_bytes2) tma_load_4d(dst0 + s * stage_bytes + 64 * CHUNK_C * 2, map_a2 + (m - map_a), &full_bar[s], c0, cw, ch, n0);
                         }
                         __syncwarp();
                         if (++s == n_stages) { s = 0; phase ^= 1; wrapped = true; }
@@ -520,12 +520,12 @@ void GroupLaunch::add(void *host_entry, const TcConvPlan &pl, const ConvArgs &a)
     if ((pl.swap ? e.pix_rows : e.bn_tile) > 128) impl->wide = true;
     impl->prm.n_entries++;
     // Pairing: this member and the previous one of the launch each fit the lower / upper half of a tile's 128
-    // rows, run the same stored layer with stride 1, and one's slice contains the other's (filters and
-    // channels): they share the larger one's tiles and weight copies.
-    auto half = [](const GroupEntry &g) { return !g.swap && g.mtiles == 1 && g.pix_rows <= 64 && g.stride == 1 && g.kw == g.k; };
+    // rows, run the same stored layer, and one's slice contains the other's (filters and channels): they
+    // share the larger one's tiles and weight copies.
+    auto half = [](const GroupEntry &g) { return !g.swap && g.mtiles == 1 && g.pix_rows <= 64 && g.kw == g.k; };
     GroupEntry *prev = impl->prm.n_entries >= 2 ? static_cast<GroupEntry *>(host_entry) - 1 : nullptr;
     if (prev && !a.win && half(e) && half(*prev) && !prev->pair && !prev->second && prev->layer == e.layer && prev->k == e.k &&
-        prev->act == e.act && ((prev->K >= e.K && prev->C >= e.C) || (e.K >= prev->K && e.C >= prev->C))) {
+        prev->stride == e.stride && prev->act == e.act && ((prev->K >= e.K && prev->C >= e.C) || (e.K >= prev->K && e.C >= prev->C))) {
         GroupEntry first = *prev, second = e;
         if (!(prev->K >= e.K && prev->C >= e.C)) { first = e; second = *prev; }
         first.tile_begin = second.tile_begin = prev->tile_begin;
