@@ -156,12 +156,12 @@ def test_profile_trace_lists_every_launch_of_a_wave():
     assert gnet.profile_trace() == []
 
 
-@pytest.mark.parametrize("family", [wl.RESNET, wl.MBV3])
-def test_members_sharing_a_tile_at_7x7_maps(family):
+@pytest.mark.parametrize("family,res", [(wl.RESNET, 224), (wl.MBV3, 224), (wl.RESNET, 192)])
+def test_members_sharing_a_tile_at_7x7_maps(family, res):
     # at 224x224 the last stage works on 7x7 maps: two members of a wave then share the 128 rows of a tile
     # (the one with the larger slice owns the weight copies).  Results must not depend on who shares with whom.
     _, onet, gnet = gu.nets(family, True)
-    n, res = 7, 224
+    n = 7                                       # (192x192: 6x6 maps, 36 rows per member)
     cfgs = wl.uniform_stream(family, n, seed=31)
     cfgs[2] = wl.extreme_cfg(family, True)      # the largest and the smallest SubNet side by side
     cfgs[3] = wl.extreme_cfg(family, False)
