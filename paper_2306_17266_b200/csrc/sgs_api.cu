@@ -1517,12 +1517,13 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                 off = off0;
             }
             if (kind == OP_DW) {
-                // depthwise: members with the same kernel size share a launch (stride, activation and image
+                // depthwise: all members share a launch, ordered by kernel size (stride, activation and image
                 // size are the layer's); a member the vectorised kernels do not take sends the bucket back
                 // to member-by-member launches
                 const size_t off0 = off;
                 const size_t l0 = launches.size();
                 bool ok = true;
+                int total_dw = 0;
                 for (int kk : {3, 5, 7}) {
                     const size_t offk = off;
                     int cnt = 0;
@@ -1535,8 +1536,11 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                         off += DW_ENTRY_BYTES;
                         cnt++;
                     }
-                    if (cnt) launches.push_back({r, nullptr, OP_DW, offk, cnt});
+                    (void)offk;
+                    total_dw += cnt;
                 }
+                // one launch for the layer: blocks pick the kernel body of their member's kernel size
+                if (total_dw) launches.push_back({r, nullptr, OP_DW, off0, total_dw});
                 size_t total = 0;
                 for (size_t i = l0; i < launches.size(); i++) total += (size_t)launches[i].count;
                 ok = total == b.size() && net->dtype == SGS_BF16;

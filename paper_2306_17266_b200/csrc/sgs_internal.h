@@ -144,8 +144,9 @@ static_assert(sizeof(SmallEntry) == 128, "record size");
 bool small_supported(int kind, const SmallEntry &e);
 cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int n, cudaStream_t st);
 // Depthwise convolution of several members in one launch: h_tbl / d_tbl = host image and device copy of
-// `members` ConvArgs records, DW_ENTRY_BYTES apart.  All members must share kernel size, stride, activation and
-// image dims and take the vectorised bf16 kernels; otherwise cudaErrorNotSupported and nothing is launched.
+// `members` ConvArgs records, DW_ENTRY_BYTES apart.  All members must share stride, activation and image dims
+// and take the vectorised bf16 kernels (kernel sizes 3, 5, 7 may be mixed); otherwise cudaErrorNotSupported and
+// nothing is launched.
 constexpr int DW_ENTRY_BYTES = 256;
 cudaError_t launch_dw_group(const char *h_tbl, const char *d_tbl, int members, cudaStream_t st);
 // Stem weights for the window view: dst[f][r][px * 8 + c] = src[f][r][px][c] (px < k, c < 3), else 0; dst [K][k][64].

@@ -187,9 +187,8 @@ __device__ __forceinline__ float2 bf2_lo(uint32_t u) { return make_float2(__uint
     const int n = GROUP ? (int)(blockIdx.z % n_img) : (int)blockIdx.z;
 static_assert(sizeof(ConvArgs) % 4 == 0 && sizeof(ConvArgs) <= DW_ENTRY_BYTES, "depthwise table record");
 
-template <int K, int ST, bool GROUP>
-__global__ void __launch_bounds__(256) dw_vec_kernel(const ConvArgs a1, const char *__restrict__ tbl, int n_img) {
-    SGS_DW_ARGS()
+template <int K, int ST>
+__device__ __forceinline__ void dw_vec_body(const ConvArgs &a, const int n) {
     constexpr int TW = 4, NCOL = (TW - 1) * ST + K, P = (K - 1) / 2;
     // grid: x covers (channel vector, pixel block) of one output row, y = output row, z = image;
     // all index arithmetic stays in 32 bits
@@ -251,6 +250,11 @@ __global__ void __launch_bounds__(256) dw_vec_kernel(const ConvArgs a1, const ch
         *reinterpret_cast<uint4 *>(yrow + wo * a.K) = ov;
     }
 }
+template <int K, int ST, bool GROUP>
+__global__ void __launch_bounds__(256) dw_vec_kernel(const ConvArgs a1, const char *__restrict__ tbl, int n_img) {
+    SGS_DW_ARGS()
+    dw_vec_body<K, ST>(a, n);
+}
 
 // Tiled variant: a thread owns 8 channels of a TH x TW patch of output pixels.  Every vector of the
 // patch's halo is loaded and unpacked ONCE and used for all the output rows and taps it belongs to, so
@@ -260,13 +264,12 @@ __global__ void __launch_bounds__(256) dw_vec_kernel(const ConvArgs a1, const ch
 // in flight, not by occupancy).  Patches whose halo lies inside the image take a path without bounds
 // tests.  The epilogue is packed: one FMA for the folded batch norm per channel pair, and h-swish as
 // x * clamp(x / 6 + 0.5, 0, 1) (= x * relu6(x + 3) / 6): one saturating FMA and one packed multiply.
-template <int K, int ST, int TH, int TW, bool PRELOAD, int ACT, bool GROUP>
-__global__ void __launch_bounds__(128) dw_tile_kernel(const ConvArgs a1, const char *__restrict__ tbl, int n_img) {
-    SGS_DW_ARGS()
+template <int K, int ST, int TH, int TW, bool PRELOAD, int ACT>
+__device__ __forceinline__ void dw_tile_body(const ConvArgs &a, const int n) {
     constexpr int P = (K - 1) / 2, NCOL = (TW - 1) * ST + K, NROW = (TH - 1) * ST + K;
     const int groups = a.K / 8, wblocks = (a.Wo + TW - 1) / TW;
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= groups * wblocks) return;
+    if (idx >= groups * wblocks || (int)blockIdx.y * TH >= a.Ho) return;
     const int cg = idx % groups, wb = idx / groups;
     const int ho0 = blockIdx.y * TH;
     const int c0 = cg * 8, wo0 = wb * TW, o = (a.R - K) / 2;
@@ -383,6 +386,36 @@ __global__ void __launch_bounds__(128) dw_tile_kernel(const ConvArgs a1, const c
         }
     }
 }
+template <int K, int ST, int TH, int TW, bool PRELOAD, int ACT, bool GROUP>
+__global__ void __launch_bounds__(128) dw_tile_kernel(const ConvArgs a1, const char *__restrict__ tbl, int n_img) {
+    SGS_DW_ARGS()
+    if (GROUP) { const ConvArgs al = a; dw_tile_body<K, ST, TH, TW, PRELOAD, ACT>(al, n); }  // (register copy, see dw_mixed_kernel)
+    else dw_tile_body<K, ST, TH, TW, PRELOAD, ACT>(a, n);
+}
+// Members of one launch with different kernel sizes (a wave's depthwise layer: every member crops its own
+// k x k window out of the stored 7x7): each block runs the body of its member's kernel size.  The grid
+// covers the largest member; blocks beyond a member's own extent leave at once.
+template <int ST, int ACT> __device__ __forceinline__ void dw_mixed_dispatch(const ConvArgs &a, const int n);
+template <int ST, int ACT>
+__global__ void __launch_bounds__(128, 3) dw_mixed_kernel(const char *__restrict__ tbl, int n_img) {
+    constexpr bool GROUP = true;
+    const ConvArgs a1 = ConvArgs();
+    SGS_DW_ARGS()
+    const ConvArgs al = a;  // (a copy in registers: reading the fields from shared memory at every use costs the tiled bodies 100 registers more)
+    dw_mixed_dispatch<ST, ACT>(al, n);
+}
+template <int ST, int ACT>
+__device__ __forceinline__ void dw_mixed_dispatch(const ConvArgs &a, const int n) {
+    if (a.k == 3) {
+        if (ST == 1) dw_tile_body<3, 1, 2, 4, true, ACT>(a, n);
+        else dw_tile_body<3, 2, 1, 4, false, ACT>(a, n);
+    } else if (a.k == 5) {
+        if (ST == 1) dw_tile_body<5, 1, 1, 4, true, ACT>(a, n);
+        else dw_vec_body<5, 2>(a, n);
+    } else {
+        dw_vec_body<7, ST>(a, n);
+    }
+}
 
 // `a` = the (first) member; grouped: kmax = the widest member's channel count, tbl = device table, members > 0
 template <int K, int ST, int TH, int TW, bool PRELOAD, bool GROUP>
@@ -430,15 +463,30 @@ cudaError_t launch_dw_group(const char *h_tbl, const char *d_tbl, int members, c
     if (members <= 0) return cudaSuccess;
     const ConvArgs &a0 = *reinterpret_cast<const ConvArgs *>(h_tbl);
     int kmax = 0;
+    bool mixed = false;
     for (int i = 0; i < members; i++) {
         const ConvArgs &a = *reinterpret_cast<const ConvArgs *>(h_tbl + (size_t)i * DW_ENTRY_BYTES);
-        if (!dw_vec_eligible(a) || a.k != a0.k || a.stride != a0.stride || a.act != a0.act || a.N != a0.N || a.H != a0.H || a.W != a0.W ||
-            a.Ho != a0.Ho || a.Wo != a0.Wo)
+        if (!dw_vec_eligible(a) || (a.k != 3 && a.k != 5 && a.k != 7) || a.stride != a0.stride || a.act != a0.act || a.N != a0.N ||
+            a.H != a0.H || a.W != a0.W)
             return cudaErrorNotSupported;
         kmax = std::max(kmax, a.K);
+        mixed = mixed || a.k != a0.k;
     }
     if ((long long)a0.N * members > 65535) return cudaErrorNotSupported;
-    return launch_dw_bf16<true>(a0, kmax, d_tbl, members, st);
+    if (!mixed) return launch_dw_bf16<true>(a0, kmax, d_tbl, members, st);
+    // (same input size and stride, odd kernels with padding (k - 1) / 2: every member has the same output size)
+    const int per_row = ((a0.Wo + 3) / 4) * (kmax / 8);
+    dim3 grid((per_row + 127) / 128, a0.Ho, a0.N * members);
+    if (a0.stride == 1) {
+        if (a0.act == ACT_RELU) dw_mixed_kernel<1, ACT_RELU><<<grid, 128, 0, st>>>(d_tbl, a0.N);
+        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<1, ACT_HSWISH><<<grid, 128, 0, st>>>(d_tbl, a0.N);
+        else dw_mixed_kernel<1, ACT_NONE><<<grid, 128, 0, st>>>(d_tbl, a0.N);
+    } else {
+        if (a0.act == ACT_RELU) dw_mixed_kernel<2, ACT_RELU><<<grid, 128, 0, st>>>(d_tbl, a0.N);
+        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<2, ACT_HSWISH><<<grid, 128, 0, st>>>(d_tbl, a0.N);
+        else dw_mixed_kernel<2, ACT_NONE><<<grid, 128, 0, st>>>(d_tbl, a0.N);
+    }
+    return cudaGetLastError();
 }
 
 template <typename T> cudaError_t launch_dw(const ConvArgs &a, cudaStream_t st) {
