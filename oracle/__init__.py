@@ -73,6 +73,9 @@ def lib():
         L.orc_layer_epilogue.argtypes = [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int] + [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_int]
         L.orc_layer_maxpool.argtypes = [ctypes.c_void_p] + [ctypes.c_int] * 4 + [ctypes.c_void_p]
         L.orc_layer_gap.argtypes = [ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c_void_p]
+        L.orc_layer_linear.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 4 + [ctypes.c_void_p]
+        L.orc_layer_se_gate.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c_void_p]
+        L.orc_layer_se_scale.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 4
         L.orc_bf16_round.restype = ctypes.c_float
         L.orc_bf16_round.argtypes = [ctypes.c_float]
         L.orc_set_tap.argtypes = [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t]
@@ -214,6 +217,35 @@ def layer_gap(x) -> np.ndarray:
     g = np.empty((N, C), dtype=np.float32)
     lib().orc_layer_gap(_ptr(x), N, H * W, C, _ptr(g))
     return g
+
+
+def layer_linear(w, bias, v, Cp: int, Kp: int, act: int = ACT_NONE) -> np.ndarray:
+    """Sliced fully connected layer on the stored matrix ``w`` [Kmax][Cmax]: first Kp outputs of the first Cp inputs."""
+    w, v = _f32(w), _f32(v)
+    bias = None if bias is None else _f32(bias)
+    y = np.empty((v.shape[0], Kp), dtype=np.float32)
+    lib().orc_layer_linear(_ptr(w), w.shape[1], _ptr(bias), _ptr(v), v.shape[0], Cp, Kp, act, _ptr(y))
+    return y
+
+
+def layer_se_gate(w1, b1, w2, b2, g, sq: int) -> np.ndarray:
+    """Squeeze-excite gate of the pooled vectors ``g`` [N][mid]: hsigmoid(FC2(relu(FC1(g)))), FC1 = first sq rows of
+    ``w1`` [.][>=mid], FC2 = first mid rows of ``w2`` [.][>=sq]."""
+    w1, w2, g = _f32(w1), _f32(w2), _f32(g)
+    b1, b2 = _f32(b1), _f32(b2)
+    gate = np.empty_like(g)
+    if lib().orc_layer_se_gate(_ptr(w1), w1.shape[1], _ptr(b1), _ptr(w2), w2.shape[1], _ptr(b2), _ptr(g), g.shape[0], g.shape[1], sq, _ptr(gate)):
+        raise MemoryError
+    return gate
+
+
+def layer_se_scale(x, gate, mode: int = FP32) -> np.ndarray:
+    """x[n][h][w][c] * gate[n][c] with the storage rounding of ``mode``."""
+    y = _f32(x).copy()
+    gate = _f32(gate)
+    N, H, W, C = y.shape
+    lib().orc_layer_se_scale(_ptr(y), _ptr(gate), N, H * W, C, mode)
+    return y
 
 
 def bf16_round(v: float) -> float:

@@ -512,6 +512,25 @@ static void linear_sliced(const orc_layer *L, const float *v, int N, int Cp, int
         }
 }
 
+/* Squeeze-excite gate from the pooled vector g[n][mid] (config text: SE with squeeze width sq, FCs with bias):
+ * gate[n][c] = hsigmoid(FC2(relu(FC1(g[n]))))[c].  tmp holds N * sq floats. */
+static void se_gate(const orc_layer *fc1, const orc_layer *fc2, const float *g, int N, int mid, int sq, float *tmp, float *gate) {
+    linear_sliced(fc1, g, N, mid, sq, tmp);
+    for (int i = 0; i < N * sq; i++) tmp[i] = act_apply(tmp[i], ACT_RELU);
+    linear_sliced(fc2, tmp, N, sq, mid, gate);
+    for (int i = 0; i < N * mid; i++) gate[i] = hsigmoid(gate[i]);
+}
+/* x[n][i][c] *= gate[n][c], then storage rounding. */
+static void se_scale(float *x, const float *gate, int N, int HW, int C, int mode) {
+    for (int n = 0; n < N; n++)
+        for (int i = 0; i < HW; i++)
+            for (int c = 0; c < C; c++) {
+                size_t idx = ((size_t)n * HW + i) * C + c;
+                x[idx] = x[idx] * gate[(size_t)n * C + c];
+            }
+    store_round(x, (size_t)N * HW * C, mode);
+}
+
 /* ------------------------------------------------------------------------------------------ */
 /* Optional tap: copy the activation a given stored layer produced (debug aid for the tests)    */
 /* ------------------------------------------------------------------------------------------ */
@@ -565,7 +584,8 @@ int orc_forward(const orc_net *net, const orc_cfg *cfg, const float *input, int 
     float *A = (float *)malloc(cap * sizeof(float)), *B = (float *)malloc(cap * sizeof(float));
     float *Cb = (float *)malloc(cap * sizeof(float)), *D = (float *)malloc(cap * sizeof(float));
     float *vec = (float *)malloc((size_t)N * 4096 * sizeof(float)), *vec2 = (float *)malloc((size_t)N * 4096 * sizeof(float));
-    if (!A || !B || !Cb || !D || !vec || !vec2) { free(A); free(B); free(Cb); free(D); free(vec); free(vec2); return -2; }
+    float *vec3 = (float *)malloc((size_t)N * 4096 * sizeof(float));
+    if (!A || !B || !Cb || !D || !vec || !vec2 || !vec3) { free(A); free(B); free(Cb); free(D); free(vec); free(vec2); free(vec3); return -2; }
     int H = res, W = res, Ho, Wo;
     float *x = A, *t1 = B, *t2 = Cb, *sc = D, *tmp;
     int C;
@@ -626,16 +646,8 @@ int orc_forward(const orc_net *net, const orc_cfg *cfg, const float *input, int 
                     /* squeeze-excite: gate[c] = hsigmoid(FC2(relu(FC1(mean_hw t2)))), t2 *= gate */
                     int sq = sl[net->se1[s][b]].K;
                     gap(t2, N, H2 * W2, mid, vec);
-                    linear_sliced(&net->L[net->se1[s][b]], vec, N, mid, sq, vec2);
-                    for (int i = 0; i < N * sq; i++) vec2[i] = act_apply(vec2[i], ACT_RELU);
-                    linear_sliced(&net->L[net->se2[s][b]], vec2, N, sq, mid, vec);
-                    for (int n = 0; n < N; n++)
-                        for (int i = 0; i < H2 * W2; i++)
-                            for (int c = 0; c < mid; c++) {
-                                size_t idx = ((size_t)n * H2 * W2 + i) * mid + c;
-                                t2[idx] = t2[idx] * hsigmoid(vec[(size_t)n * mid + c]);
-                            }
-                    store_round(t2, (size_t)N * H2 * W2 * mid, mode);
+                    se_gate(&net->L[net->se1[s][b]], &net->L[net->se2[s][b]], vec, N, mid, sq, vec2, vec3);
+                    se_scale(t2, vec3, N, H2 * W2, mid, mode);
                     tap(net->se2[s][b], t2, N, H2, W2, mid);
                 }
                 const float *resid = (st == 1 && C == out) ? x : NULL;
@@ -649,7 +661,7 @@ int orc_forward(const orc_net *net, const orc_cfg *cfg, const float *input, int 
         for (int i = 0; i < N * 1280; i++) vec2[i] = act_apply(vec2[i], ACT_HSWISH);
         linear_sliced(&net->L[net->fc], vec2, N, 1280, 1000, logits);
     }
-    free(A); free(B); free(Cb); free(D); free(vec); free(vec2);
+    free(A); free(B); free(Cb); free(D); free(vec); free(vec2); free(vec3);
     return 0;
 }
 
@@ -880,6 +892,31 @@ void orc_layer_epilogue(float *y, size_t npix, int Kp, const float *gamma, const
 
 void orc_layer_maxpool(const float *x, int N, int H, int W, int C, float *y) { maxpool3s2(x, N, H, W, C, y); }
 void orc_layer_gap(const float *x, int N, int HW, int C, float *g) { gap(x, N, HW, C, g); }
+
+static orc_layer raw_linear(const float *w, int ld, const float *bias) {
+    orc_layer L;
+    memset(&L, 0, sizeof(L));
+    L.kind = ORC_LINEAR; L.C = ld; L.w = (float *)w; L.has_bias = bias != NULL; L.bias = (float *)bias;
+    return L;
+}
+/* Sliced fully connected layer on a raw stored matrix w[Kmax][ld]: y[n][j] = act(sum_{c<Cp} w[j][c] v[n][c] + bias[j]), j < Kp. */
+void orc_layer_linear(const float *w, int ld, const float *bias, const float *v, int N, int Cp, int Kp, int act, float *y) {
+    orc_layer L = raw_linear(w, ld, bias);
+    linear_sliced(&L, v, N, Cp, Kp, y);
+    for (int i = 0; i < N * Kp; i++) y[i] = act_apply(y[i], act);
+}
+/* Squeeze-excite gate on raw stored matrices w1[.][ld1] (first FC, sq outputs of mid inputs) and w2[.][ld2]. */
+int orc_layer_se_gate(const float *w1, int ld1, const float *b1, const float *w2, int ld2, const float *b2, const float *g,
+                      int N, int mid, int sq, float *gate) {
+    orc_layer L1 = raw_linear(w1, ld1, b1), L2 = raw_linear(w2, ld2, b2);
+    float *tmp = (float *)malloc((size_t)N * sq * sizeof(float));
+    if (!tmp) return -2;
+    se_gate(&L1, &L2, g, N, mid, sq, tmp, gate);
+    free(tmp);
+    return 0;
+}
+/* In place: x[n][i][c] *= gate[n][c], with the storage rounding of `mode`. */
+void orc_layer_se_scale(float *x, const float *gate, int N, int HW, int C, int mode) { se_scale(x, gate, N, HW, C, mode); }
 float orc_bf16_round(float x) { return bf16_round(x); }
 
 #ifdef _OPENMP

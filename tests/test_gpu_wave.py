@@ -180,3 +180,56 @@ def test_members_sharing_a_tile_at_7x7_maps(family, res):
     for t in (2, 3, 5):
         ref = onet.forward(cfgs[t], x[t:t + 1], oracle.BF16_STORE)
         assert gu.rel_err(outs[1][t:t + 1], ref) < 2e-2
+
+
+@pytest.mark.parametrize("res", [160, 192, 224])
+def test_sweep_launch_shape_16_images_per_member(res):
+    # the throughput sweep's launch shape: waves of 4 SubNet configs x 16 images each (one batch of 64 per grouped
+    # launch), two waves in flight; two members per resolution are recomputed by the checker (both modes), and the
+    # result must be the bits of the same queries run one member per wave
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    groups, batch = 8, 16
+    cfgs = wl.uniform_stream(wl.RESNET, groups, seed=5)
+    cfgs[5] = wl.extreme_cfg(wl.RESNET, True)
+    xs = wl.make_inputs(groups, batch, res, seed=3, bf16=True)
+    d_in = gu.to_device(xs.reshape(groups * batch, res, res, 3), True)
+    got, _ = _run(gnet, cfgs, d_in, batch, res, 1000, wave=4, conc=2)
+    assert np.all(np.isfinite(got))
+    single, _ = _run(gnet, cfgs, d_in, batch, res, 1000, wave=1, conc=1)
+    np.testing.assert_array_equal(single, got)
+    for g in (1, 5):
+        rows = got[g * batch:(g + 1) * batch]
+        assert gu.rel_err(rows, onet.forward(cfgs[g], xs[g], oracle.BF16_STORE)) <= TOL_BF16, g
+        assert gu.rel_err(rows, onet.forward(cfgs[g], xs[g], oracle.FP32)) <= TOL_BF16, g
+
+
+def test_mbv3_bench_wave_configuration_sampled_against_checker():
+    # the MobileNetV3-shaped stream as the benchmark runs it: 224x224, waves of 32, 4 in flight, the first 128 queries
+    # of its stream (depthwise kernels of 3, 5 and 7 mixed inside every wave, so one depthwise launch dispatches all
+    # three bodies); sampled queries against the checker, bit-identical to waves of 5
+    _, onet, gnet = gu.nets(wl.MBV3, True)
+    n, res = 128, 224
+    cfgs = wl.uniform_stream(wl.MBV3, 1000, seed=3)[:n]
+    kernels = {int(c.kernel[s][b]) for c in cfgs[:32] for s in range(5) for b in range(c.depth[s])}
+    assert kernels == {3, 5, 7}
+    xs = wl.make_inputs(n, 1, res, seed=1, bf16=True)
+    d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
+    first, _ = _run(gnet, cfgs, d_in, 1, res, 1000, wave=32, conc=4)
+    other, _ = _run(gnet, cfgs, d_in, 1, res, 1000, wave=5, conc=2)
+    np.testing.assert_array_equal(other, first)
+    assert np.all(np.isfinite(first))
+    for t in range(0, n, 9):
+        assert gu.rel_err(first[t:t + 1], onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)) <= TOL_BF16, t
+        assert gu.rel_err(first[t:t + 1], onet.forward(cfgs[t], xs[t], oracle.FP32)) <= TOL_BF16, t
+
+
+@pytest.mark.parametrize("fam", [wl.RESNET, wl.MBV3])
+def test_fp32_mode_at_full_resolution(fam):
+    # fp32 handles at 224x224 (CUDA-core kernels throughout): max|err| <= 1e-4 * max|ref| against the fp32 checker
+    _, onet, gnet = gu.nets(fam, False)
+    c = wl.uniform_stream(fam, 2, seed=17)[1]
+    x = wl.make_inputs(1, 2, 224, seed=6)[0]
+    got = gu.gpu_forward(gnet, c, x, False)
+    ref = onet.forward(c, x, oracle.FP32)
+    assert gu.rel_err(got, ref) <= 1e-4
+    np.testing.assert_array_equal(got.argmax(-1), ref.argmax(-1))

@@ -205,6 +205,73 @@ def test_network_matches_library_restatement(nets, fam):
         assert np.abs(got - ref).max() <= 2e-4 * max(1.0, np.abs(ref).max())
 
 
+def _bf16_representable(a):
+    return bool(np.all((np.ascontiguousarray(a, dtype=np.float32).view(np.uint32) & 0xFFFF) == 0))
+
+
+def _stored_tensors(net, fam, cfg, x, mode):
+    """Every tensor the checker stores on the way (one tapped run per stored layer the SubNet uses) and its logits."""
+    names = [r.name for r in wl.supernet_records(fam)]
+    out, logits = {}, None
+    for i, name in enumerate(names):
+        logits, t = net.forward_tap(cfg, x, i, mode)
+        if t is not None:
+            out[name] = t
+    return out, logits
+
+
+@pytest.mark.parametrize("fam,res", [(wl.TINY, 32), (wl.RESNET, 64), (wl.MBV3, 64)])
+def test_bf16_store_mode_rounds_exactly_the_stored_tensors(fam, res):
+    """Pins where the bf16-store mode rounds.  Layer by layer, each layer fed with the checker's own stored inputs:
+    a tensor the mode stores (layer outputs, SE-scaled maps) holds only bf16 values and equals the fp64 library
+    restatement rounded once, up to a few one-step flips from the order of additions; what is not stored (pooled and
+    SE vectors, the head's mixing vector, logits) is not rounded, so the logits computed from the last stored tensor
+    agree to fp32 accuracy.  (The max-pooled map is stored too, but the maximum of bf16 values is one of them: rounding
+    it changes nothing and cannot be pinned.)"""
+    blob = wl.make_blob(fam, seed=0, bf16_weights=True)
+    net = oracle.Net(fam, blob)
+    P = torch_ref.parse_blob(fam, blob)
+    x = wl.make_inputs(1, 2, res, seed=3, bf16=True)[0]
+    for c in wl.uniform_stream(fam, 2, seed=11) + [wl.extreme_cfg(fam, True)]:
+        taught, logits = _stored_tensors(net, fam, c, x, oracle.BF16_STORE)
+        assert len(taught) >= 5
+        store = torch_ref.Store(True, teacher=taught)
+        ref_logits = torch_ref.forward(fam, P, c, x, store)
+        assert set(store.report) == set(taught)  # every tapped tensor was met on the way
+        for name, t in taught.items():
+            rep = store.report[name]
+            assert _bf16_representable(t), name
+            assert rep["beyond_one_step"] == 0, (name, rep)
+            assert rep["unequal"] <= max(2, 0.005 * rep["n"]), (name, rep)
+        assert np.abs(logits - ref_logits).max() <= 2e-5 * max(1.0, np.abs(ref_logits).max())
+        # a checker that forgot to round (its fp32 mode) is caught by the same checks
+        plain, _ = _stored_tensors(net, fam, c, x, oracle.FP32)
+        assert not any(_bf16_representable(t) for t in plain.values())
+
+
+@pytest.mark.parametrize("fam,res", [(wl.TINY, 32), (wl.MBV3, 64)])
+def test_bf16_store_network_matches_library_restatement(fam, res):
+    """Whole network, no teacher: on the shallow family, and on MobileNetV3-shaped SubNets of minimum depth, the two
+    implementations stay within a few flips of each other end to end, and leaving out the rounding of the layer
+    outputs (or, with squeeze-excite blocks, of the SE-scaled map) moves the logits visibly further away."""
+    blob = wl.make_blob(fam, seed=0, bf16_weights=True)
+    net = oracle.Net(fam, blob)
+    P = torch_ref.parse_blob(fam, blob)
+    x = wl.make_inputs(1, 2, res, seed=3, bf16=True)[0]
+    c = wl.extreme_cfg(fam, False)
+    got = net.forward(c, x, oracle.BF16_STORE)
+
+    def dist(skip):
+        ref = torch_ref.forward(fam, P, c, x, torch_ref.Store(True, skip))
+        return np.abs(got - ref).max() / np.abs(ref).max()
+
+    base = dist(())
+    assert base <= 2e-5
+    assert dist(("layer",)) > 20 * max(base, 1e-6)
+    if fam == wl.MBV3:
+        assert dist(("se_scale",)) > 20 * max(base, 1e-6)
+
+
 def _record_offsets(fam):
     """word offset of each record's float payload in the blob"""
     pos, out = 8, {}
@@ -366,3 +433,29 @@ def test_hit_ratio_formula(nets):
     big = np.array([[9, 9, 3], [9, 9, 3]], dtype=np.int32)
     assert oracle.hit_ratio(sn, big) == 1.0          # cache contains the SubNet
     assert oracle.hit_ratio(sn, np.zeros_like(sn)) == 0.0
+
+
+def test_linear_and_squeeze_excite_layers_against_plain_formulas():
+    # sliced fully connected layer = a matrix product on the prefix block; SE gate = hsigmoid(FC2(relu(FC1(g)))) with
+    # hsigmoid(x) = min(max(x + 3, 0), 6) / 6; SE scale multiplies every pixel's channels by the gate of its image.
+    # fp64 numpy on Python slices; a transposed operand, a wrong prefix or a missing bias fails.
+    rng = np.random.default_rng(5)
+    w = rng.standard_normal((40, 56)).astype(np.float32)
+    b = rng.standard_normal(40).astype(np.float32)
+    v = rng.standard_normal((3, 48)).astype(np.float32)
+    for Cp, Kp in ((48, 40), (24, 17), (1, 1)):
+        want = v[:, :Cp].astype(np.float64) @ w[:Kp, :Cp].astype(np.float64).T + b[:Kp]
+        np.testing.assert_allclose(oracle.layer_linear(w, b, v[:, :Cp], Cp, Kp), want, rtol=0, atol=2e-5)
+        np.testing.assert_allclose(oracle.layer_linear(w, None, v[:, :Cp], Cp, Kp, oracle.ACT_RELU), np.maximum(want - b[:Kp], 0), rtol=0, atol=2e-5)
+    mid, sq = 24, 8
+    w1 = rng.standard_normal((16, 40)).astype(np.float32)   # stored [sq_max][mid_max]
+    w2 = rng.standard_normal((40, 16)).astype(np.float32)   # stored [mid_max][sq_max]
+    b1, b2 = rng.standard_normal(16).astype(np.float32), rng.standard_normal(40).astype(np.float32)
+    g = rng.standard_normal((2, mid)).astype(np.float32)
+    h = np.maximum(g.astype(np.float64) @ w1[:sq, :mid].astype(np.float64).T + b1[:sq], 0)
+    gate = np.clip(h @ w2[:mid, :sq].astype(np.float64).T + b2[:mid] + 3, 0, 6) / 6
+    got = oracle.layer_se_gate(w1, b1, w2, b2, g, sq)
+    np.testing.assert_allclose(got, gate, rtol=0, atol=2e-6)
+    x = rng.standard_normal((2, 3, 5, mid)).astype(np.float32)
+    np.testing.assert_allclose(oracle.layer_se_scale(x, got), x.astype(np.float64) * got[:, None, None, :], rtol=1e-6, atol=0)
+    np.testing.assert_array_equal(oracle.layer_se_scale(x, got, oracle.BF16_STORE), wl.round_to_bf16(oracle.layer_se_scale(x, got)))
