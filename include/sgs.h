@@ -315,9 +315,9 @@ sgs_status_t sgs_conv2d_sliced(const sgs_conv_desc_t *desc, const void *d_x, con
  * sgs_conv2d_sliced_static - sgs_conv2d_sliced for callers that may not allocate device memory.
  * (The paper has no counterpart to this call; it exists for the way the library is deployed.)
  *
- * Who needs it: code that runs while a stream is being captured into a CUDA graph, services that gave
- * all device memory to their own pool at start-up, and latency-critical loops that cannot afford the
- * device-wide synchronisation cudaMalloc and cudaFree imply.  sgs_conv2d_sliced may call cudaMalloc to
+ * Who needs it: serving processes that gave all device memory to their own pool at start-up (a cudaMalloc
+ * from a library then simply fails), and latency-critical loops that cannot afford the device-wide
+ * synchronisation cudaMalloc and cudaFree imply.  sgs_conv2d_sliced may call cudaMalloc to
  * grow its split-reduction scratch; this variant never does.  Its scratch is a fixed array of
  * SGS_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the library
  * holds that much memory until the process exits.
@@ -342,8 +342,59 @@ sgs_status_t sgs_conv2d_sliced(const sgs_conv_desc_t *desc, const void *d_x, con
 sgs_status_t sgs_conv2d_sliced_static(const sgs_conv_desc_t *desc, const void *d_x, const void *d_w, const float *d_scale,
                                       const float *d_shift, const void *d_res, void *d_y, void *cuda_stream);
 
-/* Nonzero once a kernel of this process has reported that one of its bounded waits ran out. */
+/*
+ * sgs_aux_op - the layers of a SubNet that are not convolutions, one at a time on caller-owned device tensors
+ * (the paper's SuperNets are the OFA ResNet50 / MobileNetV3 families of Section 5.1: max pool after the stem,
+ * global average pool before the classifier and inside squeeze-excite blocks, fully connected layers sliced by
+ * prefix like every other stored layer, Section 2.1).  For layer-level tests and microbenchmarks.
+ *   SGS_AUX_MAXPOOL   y[n][ho][wo][c] = max over the 3x3 window at stride 2, padding 1 (padding never wins);
+ *                     x [N][H][W][C] -> y [N][(H-1)/2+1][(W-1)/2+1][C], dtype elements
+ *   SGS_AUX_AVGPOOL   y[n][c] = mean over H*W pixels (fixed summation order); x [N][H][W][C] dtype -> y [N][C] fp32
+ *   SGS_AUX_LINEAR    y[n][j] = act(sum_{c<C} w[j][c] x[n][c] + bias[j]), j < K; x [N][C] fp32, w [>=K][ld] dtype
+ *                     (ld = stored input width >= C), bias [>=K] fp32, y [N][K] fp32
+ *   SGS_AUX_SE_GATE   y[n][c] = hsigmoid(b2[c] + sum_{j<K} w2[c][j] relu(b1[j] + sum_{i<C} w[j][i] x[n][i])), c < C;
+ *                     x [N][C] fp32 pooled vectors, w [>=K][ld], w2 [>=C][ld2] dtype, y [N][C] fp32
+ *   SGS_AUX_SE_SCALE  y[n][h][w][c] = x[n][h][w][c] * g[n][c]; x, y [N][H][W][C] dtype, g = `w` [N][C] fp32
+ * n_members >= 1 independent problems desc[m] / args[m].  grouped = 0: each runs in the kernel a single query
+ * uses; grouped = 1: all of them (same kind and dtype SGS_BF16) run in ONE launch of the kernel a wave uses, whose
+ * per-member records this call uploads to a temporary device table (it allocates and synchronises the stream).
+ * Shapes the vectorised kernels do not take (channel counts that are not multiples of 8, unaligned pointers) fall back
+ * to scalar kernels when grouped = 0 and are SGS_EUNSUPPORTED when grouped = 1.
+ * Errors: SGS_EINVAL (NULL, non-positive size, K > ld ...), SGS_EUNSUPPORTED, SGS_ENOMEM, SGS_ECUDA.
+ */
+typedef enum { SGS_AUX_MAXPOOL = 0, SGS_AUX_AVGPOOL = 1, SGS_AUX_LINEAR = 2, SGS_AUX_SE_GATE = 3, SGS_AUX_SE_SCALE = 4 } sgs_aux_kind_t;
+typedef struct {
+    int kind;         /* sgs_aux_kind_t */
+    int dtype;        /* sgs_dtype_t of tensors and weights */
+    int N, H, W, C;   /* images, map size (1 x 1 for vectors), channels / input features */
+    int K;            /* linear: outputs; SE gate: squeeze width */
+    int ld, ld2;      /* row pitch (elements) of w and of w2 */
+    int act;          /* linear: 0 none / 1 ReLU / 2 h-swish */
+} sgs_aux_desc_t;
+typedef struct {
+    const void *x;
+    void *y;
+    const void *w;
+    const float *bias;
+    const void *w2;
+    const float *bias2;
+} sgs_aux_args_t;
+sgs_status_t sgs_aux_op(int n_members, const sgs_aux_desc_t *desc, const sgs_aux_args_t *args, int grouped, void *cuda_stream);
+
+/* Nonzero once a kernel of this process has reported that one of its bounded waits ran out (the paper has no
+ * counterpart: every device-side wait of the kernels carries a time limit, after which the kernel records the fact
+ * in a status word of its device, lets its copies land, frees its tensor memory and returns; calls that follow
+ * report SGS_ETIMEOUT).  Reads the status words of the current device (sgs_conv2d_sliced_static keeps its own);
+ * the answer is sticky until sgs_device_status_clear. */
 int sgs_device_status(void);
+
+/* Synchronises the current device, zeroes its status words and forgets earlier time-outs. */
+sgs_status_t sgs_device_status_clear(void);
+
+/* Test aid for the time-out path: enqueues a one-block kernel on `cuda_stream` whose only wait can never be
+ * satisfied, with a limit of limit_us microseconds (1 .. 1000000).  The kernel gives up after the limit, sets the
+ * device status word exactly as the convolution kernels do, and returns normally; nothing faults or hangs. */
+sgs_status_t sgs_debug_expire_wait(unsigned limit_us, void *cuda_stream);
 
 /* Library options by name (debug and measurement aids): "conv_impl" 0 = automatic, 1 = force the
  * CUDA-core kernels; "profile" see sgs_profile_read.  Unknown name -> SGS_EINVAL. */

@@ -27,13 +27,24 @@ EXPORTS = [
     "sgs_set_option", "sgs_get_counter", "sgs_last_error", "sgs_supernet_free", "sgs_conv2d_sliced", "sgs_device_status",
     "sgs_profile_read", "sgs_conv2d_sliced_static", "sgs_cache_set_candidates", "sgs_cache_set_policy",
     "sgs_sched_create", "sgs_sched_free", "sgs_sched_dims", "sgs_sched_set_table", "sgs_sched_get_table", "sgs_sched_measure",
-    "sgs_sched_step", "sgs_sched_subnet", "sgs_profile_trace", "sgs_layer_name",
+    "sgs_sched_step", "sgs_sched_subnet", "sgs_profile_trace", "sgs_layer_name", "sgs_aux_op", "sgs_device_status_clear", "sgs_debug_expire_wait",
 ]
 
 
 class ConvDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("N", "H", "W", "C", "K", "Kmax", "Cmax", "R", "k", "stride", "act", "dtype",
                                              "impl", "depthwise", "cache_k", "cache_c", "weight_policy", "split_k_off")]
+
+
+SGS_AUX_MAXPOOL, SGS_AUX_AVGPOOL, SGS_AUX_LINEAR, SGS_AUX_SE_GATE, SGS_AUX_SE_SCALE = range(5)
+
+
+class AuxDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("kind", "dtype", "N", "H", "W", "C", "K", "ld", "ld2", "act")]
+
+
+class AuxArgs(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("x", "y", "w", "bias", "w2", "bias2")]
 
 
 class StreamOpts(ctypes.Structure):
@@ -183,6 +194,9 @@ def lib():
         L.sgs_conv2d_sliced.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
         L.sgs_conv2d_sliced_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
         L.sgs_device_status.argtypes = []
+        L.sgs_aux_op.argtypes = [ci, vp, vp, ci, vp]
+        L.sgs_device_status_clear.argtypes = []
+        L.sgs_debug_expire_wait.argtypes = [ctypes.c_uint, vp]
         L.sgs_profile_read.argtypes = [vp, ci, vp, vp, vp, vp]
         _lib = L
     return _lib
@@ -211,6 +225,28 @@ def conv2d_sliced_static(desc: ConvDesc, d_x: int, d_w: int, d_scale: int, d_shi
     st = lib().sgs_conv2d_sliced_static(ctypes.byref(desc), d_x, d_w, d_scale, d_shift, d_res or None, d_y, stream)
     if st != SGS_OK:
         raise SgsError(st, "sgs_conv2d_sliced_static")
+
+
+def device_status_clear():
+    st = lib().sgs_device_status_clear()
+    if st != SGS_OK:
+        raise SgsError(st, "sgs_device_status_clear")
+
+
+def debug_expire_wait(limit_us: int, stream: int = 0):
+    st = lib().sgs_debug_expire_wait(limit_us, ctypes.c_void_p(stream))
+    if st != SGS_OK:
+        raise SgsError(st, "sgs_debug_expire_wait")
+
+
+def aux_op(descs: Sequence[AuxDesc], args: Sequence[AuxArgs], grouped: bool = False, stream: int = 0):
+    """sgs_aux_op on len(descs) members (device addresses in ``args``)."""
+    n = len(descs)
+    d = (AuxDesc * n)(*descs)
+    a = (AuxArgs * n)(*args)
+    st = lib().sgs_aux_op(n, d, a, int(grouped), ctypes.c_void_p(stream))
+    if st != SGS_OK:
+        raise SgsError(st, "sgs_aux_op")
 
 
 def device_status() -> int:

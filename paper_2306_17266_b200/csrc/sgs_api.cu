@@ -2239,6 +2239,78 @@ sgs_status_t sgs_conv2d_sliced(const sgs_conv_desc_t *d, const void *d_x, const 
     return e == cudaSuccess ? SGS_OK : SGS_ECUDA;
 }
 
+// Non-convolution layers on caller tensors (see sgs.h).  Mirrors the dispatch of launch_op / wave_impl.
+sgs_status_t sgs_aux_op(int n, const sgs_aux_desc_t *desc, const sgs_aux_args_t *args, int grouped, void *cuda_stream) {
+    if (n <= 0 || n > 65535 || !desc || !args) return SGS_EINVAL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    std::vector<SmallEntry> es((size_t)n);
+    int kind0 = -1;
+    for (int m = 0; m < n; m++) {
+        const sgs_aux_desc_t &d = desc[m];
+        const sgs_aux_args_t &a = args[m];
+        if (d.kind < SGS_AUX_MAXPOOL || d.kind > SGS_AUX_SE_SCALE || (d.dtype != SGS_F32 && d.dtype != SGS_BF16)) return SGS_EINVAL;
+        if (!a.x || !a.y || d.N <= 0 || d.H <= 0 || d.W <= 0 || d.C <= 0 || d.act < 0 || d.act > 2) return SGS_EINVAL;
+        const bool fc = d.kind == SGS_AUX_LINEAR || d.kind == SGS_AUX_SE_GATE;
+        if (fc && (!a.w || !a.bias || d.K <= 0 || d.ld < d.C)) return SGS_EINVAL;
+        if (d.kind == SGS_AUX_SE_GATE && (!a.w2 || !a.bias2 || d.ld2 < d.K)) return SGS_EINVAL;
+        if (d.kind == SGS_AUX_SE_SCALE && !a.w) return SGS_EINVAL;
+        SmallEntry &e = es[(size_t)m];
+        std::memset(&e, 0, sizeof e);
+        e.x = a.x; e.y = a.y; e.w = a.w; e.bias = a.bias; e.w2 = a.w2; e.bias2 = a.bias2;
+        e.N = d.N; e.H = d.H; e.W = d.W; e.C = d.C; e.K = d.K; e.ld = d.ld; e.ld2 = d.ld2; e.act = d.act;
+        e.Ho = (d.H - 1) / 2 + 1; e.Wo = (d.W - 1) / 2 + 1;
+        static const int kinds[5] = {OP_MAXPOOL, OP_GAP, OP_LINEAR, OP_SE_GATE, OP_SCALE};
+        const int kind = kinds[d.kind];
+        if (m == 0) kind0 = kind;
+        if (grouped && (kind != kind0 || d.dtype != SGS_BF16 || d.dtype != desc[0].dtype || !small_supported(kind, e))) return SGS_EUNSUPPORTED;
+    }
+    if (grouped) {
+        SmallEntry *d_tbl = nullptr;
+        if (cudaMalloc((void **)&d_tbl, (size_t)n * sizeof(SmallEntry)) != cudaSuccess) return SGS_ENOMEM;
+        cudaError_t e = cudaMemcpyAsync(d_tbl, es.data(), (size_t)n * sizeof(SmallEntry), cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = launch_small(kind0, es.data(), d_tbl, n, st);
+        const cudaError_t e2 = cudaStreamSynchronize(st);
+        cudaFree(d_tbl);
+        return (e == cudaSuccess && e2 == cudaSuccess) ? SGS_OK : SGS_ECUDA;
+    }
+    for (int m = 0; m < n; m++) {
+        const sgs_aux_desc_t &d = desc[m];
+        const SmallEntry &e = es[(size_t)m];
+        const bool bf = d.dtype == SGS_BF16;
+        cudaError_t ce = cudaSuccess;
+        using B = __nv_bfloat16;
+        switch (d.kind) {
+        case SGS_AUX_MAXPOOL:
+            ce = bf ? launch_maxpool3s2<B>((const B *)e.x, (B *)e.y, d.N, d.H, d.W, d.C, st) : launch_maxpool3s2<float>((const float *)e.x, (float *)e.y, d.N, d.H, d.W, d.C, st);
+            break;
+        case SGS_AUX_AVGPOOL:
+            ce = bf ? launch_gap<B>((const B *)e.x, (float *)e.y, d.N, d.H * d.W, d.C, st) : launch_gap<float>((const float *)e.x, (float *)e.y, d.N, d.H * d.W, d.C, st);
+            break;
+        case SGS_AUX_LINEAR:
+            ce = bf ? launch_linear<B>((const float *)e.x, (const B *)e.w, e.bias, (float *)e.y, d.N, d.C, d.K, d.ld, d.act, st)
+                    : launch_linear<float>((const float *)e.x, (const float *)e.w, e.bias, (float *)e.y, d.N, d.C, d.K, d.ld, d.act, st);
+            break;
+        case SGS_AUX_SE_GATE:
+            ce = bf ? launch_se_gate<B>((const float *)e.x, (const B *)e.w, e.bias, (const B *)e.w2, e.bias2, (float *)e.y, d.N, d.C, d.K, d.ld, d.ld2, st)
+                    : launch_se_gate<float>((const float *)e.x, (const float *)e.w, e.bias, (const float *)e.w2, e.bias2, (float *)e.y, d.N, d.C, d.K, d.ld, d.ld2, st);
+            break;
+        default:
+            ce = bf ? launch_scale<B>((const B *)e.x, (const float *)e.w, (B *)e.y, d.N, d.H * d.W, d.C, st)
+                    : launch_scale<float>((const float *)e.x, (const float *)e.w, (float *)e.y, d.N, d.H * d.W, d.C, st);
+            break;
+        }
+        if (ce != cudaSuccess) return SGS_ECUDA;
+    }
+    return SGS_OK;
+}
+
 int sgs_device_status(void) { return tc_conv_status(); }
+
+sgs_status_t sgs_device_status_clear(void) { return tc_conv_status_clear() == cudaSuccess ? SGS_OK : SGS_ECUDA; }
+
+sgs_status_t sgs_debug_expire_wait(unsigned limit_us, void *cuda_stream) {
+    if (limit_us == 0 || limit_us > 1000000u) return SGS_EINVAL;
+    return tc_expire_wait(limit_us, (cudaStream_t)cuda_stream) == cudaSuccess ? SGS_OK : SGS_ECUDA;
+}
 
 }  // extern "C"

@@ -20,10 +20,6 @@
 
 namespace sgs {
 
-#ifdef SGS_ROLE_TIMING
-__device__ unsigned long long g_role_cycles[16];
-#endif
-
 namespace {
 
 constexpr int G_MAX_STAGES = 6;
@@ -87,16 +83,6 @@ __device__ __forceinline__ int tile_entry(const GroupEntry *es, int n, int t, in
 __device__ __forceinline__ void group_bar(int grp) { asm volatile("bar.sync %0, 128;" ::"r"(grp + 1) : "memory"); }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *m) { asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory"); }
 
-#ifdef SGS_ROLE_TIMING
-// Development aid (not compiled into the library): cycles each warp role spends waiting, summed over CTAs and launches.
-#define ROLE_T0() const long long rt0_ = clock64()
-#define ROLE_ADD(var) var += clock64() - rt0_
-#define ROLE_FLUSH(idx, var) do { if (lane == 0) atomicAdd(&g_role_cycles[idx], (unsigned long long)(var)); } while (0)
-#else
-#define ROLE_T0()
-#define ROLE_ADD(var)
-#define ROLE_FLUSH(idx, var)
-#endif
 
 // Kernel parameters.  The tensor maps travel in the parameter block (the TMA unit reads them from
 // there); the per-member records travel in a device table.
@@ -156,8 +142,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         int s = 0;
         uint32_t phase = 0;
         bool wrapped = false, ok = true;
-        long long tw_ = 0; (void)tw_;
-        const long long tk0_ = clock64(); (void)tk0_;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const GroupEntry &e = es[tile_entry(es, n_entries, t, lane)];
             const int nt = (t - e.tile_begin) / e.mtiles;
@@ -175,7 +159,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             for (int r = 0; r < k && ok; r++, tap_row += R) {
                 for (int sx = 0; sx < kw && ok; sx++) {
                     for (int cc = 0, c0 = 0; cc < cchunks; cc++, c0 += CHUNK_C) {
-                        { ROLE_T0(); if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag)); ROLE_ADD(tw_); }
+                        if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag));
                         if (!ok) break;
                         if (elect_one()) {
                             uint8_t *sb = dst0 + s * stage_bytes;
@@ -193,15 +177,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             if (ok && tn < total_tiles && elect_one()) prefetch_tensormap(&P.maps[es[find_entry_serial(es, n_entries, tn)].map_w]);
             __syncwarp();
         }
-        ROLE_FLUSH(0, tw_); ROLE_FLUSH(1, clock64() - tk0_);
     } else if (warp == G_PIX_WARP) {
         // ------------------------------------------------------------------ activation producer
         int s = 0;
         uint32_t phase = 0;
         bool wrapped = false, ok = true;
-        long long tw_ = 0, tpdl_ = 0; (void)tw_; (void)tpdl_;
-        const long long tk0_ = clock64(); (void)tk0_;
-        { ROLE_T0(); pdl_wait(); ROLE_ADD(tpdl_); }  // activations (and the buffers this layer overwrites) belong to the previous layers until here
+        pdl_wait();  // activations (and the buffers this layer overwrites) belong to the previous layers until here
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const GroupEntry &e = es[tile_entry(es, n_entries, t, lane)];
             const int mt = (t - e.tile_begin) % e.mtiles;
@@ -220,7 +201,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                     const CUtensorMap *m = map_a + ph * 2 + pw;
                     const int cw = stride == 2 ? w0 + ((dw - pw) >> 1) : w0 + dw, ch = stride == 2 ? h0 + ((dh - ph) >> 1) : h0 + dh;
                     for (int cc = 0, c0 = 0; cc < cchunks; cc++, c0 += CHUNK_C) {
-                        { ROLE_T0(); if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag)); ROLE_ADD(tw_); }
+                        if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag));
                         if (!ok) break;
                         if (elect_one()) {
                             mbar_expect_tx(&full_bar[s], pix_bytes + pix_bytes2);
@@ -237,7 +218,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             if (ok && tn < total_tiles && elect_one()) prefetch_tensormap(&P.maps[es[find_entry_serial(es, n_entries, tn)].map_a]);
             __syncwarp();
         }
-        ROLE_FLUSH(2, tw_); ROLE_FLUSH(3, tpdl_); ROLE_FLUSH(4, clock64() - tk0_);
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         int s = 0;
@@ -245,8 +225,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         int j = 0;
         const uint32_t ring = smem_u32(smem);
         bool ok = true;
-        long long tfull_ = 0, tacc_ = 0; (void)tfull_; (void)tacc_;
-        const long long tk0_ = clock64(); (void)tk0_;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, j++) {
             const GroupEntry &e = es[tile_entry(es, n_entries, t, lane)];
             const int nt = (t - e.tile_begin) / e.mtiles;
@@ -257,15 +235,15 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             const int buf = j & 1;
             const int cchunks = e.cchunks, taps = e.k * e.kw;
             const int last_ksteps = (e.C - (cchunks - 1) * CHUNK_C + 15) / 16;  // 16-channel steps of a tap's last chunk
-            { ROLE_T0(); ok = j < 2 || mbar_wait(&acc_empty[buf], ((j >> 1) - 1) & 1, abort_flag);  // epilogue drained this buffer
-            ok = __all_sync(0xffffffffu, ok); ROLE_ADD(tacc_); }
+            ok = j < 2 || mbar_wait(&acc_empty[buf], ((j >> 1) - 1) & 1, abort_flag);  // epilogue drained this buffer
+            ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * G_ACC_COLS);
             uint32_t accumulate = 0;
             for (int tap = 0; tap < taps && ok; tap++) {
                 for (int cc = 0; cc < cchunks; cc++) {
-                    { ROLE_T0(); ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], phase, abort_flag)); ROLE_ADD(tfull_); }
+                    ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], phase, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                     const int ksteps = cc == cchunks - 1 ? last_ksteps : CHUNK_C / 16;
@@ -282,7 +260,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                 }
             }
         }
-        ROLE_FLUSH(5, tfull_); ROLE_FLUSH(6, tacc_); ROLE_FLUSH(7, clock64() - tk0_);
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9)
         // Two groups of four warps (one per tensor-memory lane quadrant).  Group g owns accumulator buffer g
@@ -295,9 +272,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         float(*scale_g)[G_ACC_COLS] = scale_s[grp];
         float(*shift_g)[G_ACC_COLS] = shift_s[grp];
         const int stride2 = 2 * (int)gridDim.x;
-        long long tpdl_ = 0, tbar_ = 0, tacc_ = 0, twork_ = 0; (void)tpdl_; (void)tbar_; (void)tacc_; (void)twork_;
-        const long long tk0_ = clock64(); (void)tk0_;
-        { ROLE_T0(); pdl_wait(); ROLE_ADD(tpdl_); }  // residual reads and output writes must not pass the previous layers
+        pdl_wait();  // residual reads and output writes must not pass the previous layers
         bool alive = true;  // after a failed wait the warp only keeps the named barrier in step
         // folded batch norm of a normal tile: thread et fetches the scale and shift of filters et and et + 128
         auto fetch_bn = [&](int tile, float *v) {
@@ -358,10 +333,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                 uint4 rv[4], rn[4];
                 load_res(0, rv);
                 load_res(32, rn);
-                { ROLE_T0(); group_bar(grp); ROLE_ADD(tbar_); }  // this tile's scale / shift (written during the group's previous tile) are visible
+                group_bar(grp);  // this tile's scale / shift (written during the group's previous tile) are visible
                 const float *sc = scale_g[sb], *sh = shift_g[sb];
-                { ROLE_T0(); if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&acc_full[grp], jj & 1, abort_flag)); ROLE_ADD(tacc_); }
-                ROLE_T0();
+                if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&acc_full[grp], jj & 1, abort_flag));
                 if (alive) {
                     tc_fence_after();
 #pragma unroll 1
@@ -390,7 +364,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                         for (int g = 0; g < 4; g++) { rv[g] = rn[g]; rn[g] = rf[g]; }
                     }
                 }
-                ROLE_ADD(twork_);
             } else {
                 // ---- swapped tile: this thread owns filter `f`, columns are the member's output pixels
                 const int f = nt * 128 + row;
@@ -448,7 +421,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             // threads have left (barrier above)
             store_bn(sb ^ 1, nbn);
         }
-        if (warp == 2) { ROLE_FLUSH(8, tpdl_); ROLE_FLUSH(9, tbar_); ROLE_FLUSH(10, tacc_); ROLE_FLUSH(11, twork_); ROLE_FLUSH(12, clock64() - tk0_); }
     }
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
@@ -578,14 +550,3 @@ cudaError_t GroupLaunch::launch(const int *cache_tbl, int sms, cudaStream_t st) 
 }
 
 }  // namespace sgs
-
-#ifdef SGS_ROLE_TIMING
-extern "C" int sgs_debug_role_cycles(unsigned long long *out16, int reset) {
-    cudaError_t e = cudaMemcpyFromSymbol(out16, sgs::g_role_cycles, sizeof(unsigned long long) * 16);
-    if (e == cudaSuccess && reset) {
-        unsigned long long z[16] = {};
-        e = cudaMemcpyToSymbol(sgs::g_role_cycles, z, sizeof z);
-    }
-    return e == cudaSuccess ? 0 : 1;
-}
-#endif

@@ -335,17 +335,62 @@ int *tc_status_word(int device) {
     return g_dev[device].status;
 }
 
+int *static_status_word(int device);  // status word inside the fixed scratch array (below); nullptr before its set-up
+
+// Both status words of the current device (the allocated one and the one inside the fixed scratch array of the
+// allocation-free entry point); a word of another device is readable only while that device is current.
 int tc_conv_status() {
     std::lock_guard<std::mutex> lk(g_mu);
-    for (int d = 0; d < 64; d++) {
-        if (!g_dev[d].status) continue;
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess || cur < 0 || cur >= 64) return g_status_seen;
+    int *words[2] = {g_dev[cur].status, static_status_word(cur)};
+    for (int *w : words) {
         int v = 0;
-        int cur = -1;
-        cudaGetDevice(&cur);
-        if (cur != d) continue;  // only the current device's word is readable without switching
-        if (cudaMemcpy(&v, g_dev[d].status, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess && v) g_status_seen = 1;
+        if (w && cudaMemcpy(&v, w, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess && v) g_status_seen = 1;
     }
     return g_status_seen;
+}
+
+cudaError_t tc_conv_status_clear() {
+    std::lock_guard<std::mutex> lk(g_mu);
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return e;
+    if (cur < 0 || cur >= 64) return cudaErrorInvalidDevice;
+    if ((e = cudaDeviceSynchronize()) != cudaSuccess) return e;
+    int *words[2] = {g_dev[cur].status, static_status_word(cur)};
+    for (int *w : words)
+        if (w && (e = cudaMemset(w, 0, sizeof(int))) != cudaSuccess) return e;
+    g_status_seen = 0;
+    return cudaSuccess;
+}
+
+namespace {
+// One block whose single wait can never be satisfied (nothing arrives at the barrier): it gives up after
+// limit_ns, records that in the status word like the convolution kernels do, and returns.
+__global__ void expire_wait_kernel(unsigned long long limit_ns, int *status) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_s;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    volatile int *abort_flag = &abort_s;
+    const bool ok = mbar_wait(&bar, 0, abort_flag, limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0 && (!ok || abort_s)) atomicExch(status, 1);
+}
+}  // namespace
+
+cudaError_t tc_expire_wait(unsigned limit_us, cudaStream_t st) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if ((e = tc_conv_init(dev)) != cudaSuccess) return e;
+    expire_wait_kernel<<<1, 64, 0, st>>>((unsigned long long)limit_us * 1000ull, g_dev[dev].status);
+    return cudaGetLastError();
 }
 
 // Picks the output-pixel box (bw, bh, bn), bw*bh*bn <= 128, that wastes the fewest tile rows.
@@ -578,10 +623,9 @@ cudaError_t tc_conv_launch(const TcConvPlan &pl, const ConvArgs &a, cudaStream_t
 // =============================================================================================
 // Sliced convolution for callers that must not allocate device memory.
 //
-// Some users of this library run where cudaMalloc is off limits: inside a region that is being
-// captured into a CUDA graph, inside a serving process whose whole device memory was handed to a
-// pool at start-up, or in a latency-critical loop where an implicit device synchronisation (which
-// cudaMalloc / cudaFree cause) is not acceptable.  For them the split-reduction scratch of the
+// Some users of this library run where cudaMalloc is off limits: inside a serving process whose
+// whole device memory was handed to a pool at start-up, or in a latency-critical loop where an
+// implicit device synchronisation (which cudaMalloc / cudaFree cause) is not acceptable.  For them the split-reduction scratch of the
 // tensor-core kernel lives in a fixed array that is part of the loaded library image.
 // =============================================================================================
 namespace sgs {
@@ -618,6 +662,11 @@ cudaError_t static_scratch_setup(int dev, StaticScratch **out) {
 }
 
 }  // namespace
+
+int *static_status_word(int device) {
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    return (device >= 0 && device < 64 && g_static_ptr[device]) ? &g_static_ptr[device]->status : nullptr;
+}
 }  // namespace sgs
 
 extern "C" sgs_status_t sgs_conv2d_sliced_static(const sgs_conv_desc_t *d, const void *d_x, const void *d_w,
@@ -628,6 +677,7 @@ extern "C" sgs_status_t sgs_conv2d_sliced_static(const sgs_conv_desc_t *d, const
     if (d->N <= 0 || d->H <= 0 || d->W <= 0 || d->C <= 0 || d->K <= 0 || d->k <= 0 || (d->k & 1) == 0 || d->k > d->R ||
         ((d->R - d->k) & 1) || d->K > d->Kmax || d->C > d->Cmax || (d->stride != 1 && d->stride != 2) || d->act < 0 || d->act > 2)
         return SGS_EINVAL;
+    if (d->impl < 0 || d->impl > 2) return SGS_EINVAL;
     if (d->dtype != SGS_BF16 || d->depthwise || d->impl == 1 || !tc_available()) return SGS_EUNSUPPORTED;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SGS_ECUDA;

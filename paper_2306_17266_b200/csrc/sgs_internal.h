@@ -163,6 +163,8 @@ cudaError_t tc_conv_init(int device);  // one-time device set-up; call outside s
 bool tc_available();
 int tc_conv_status();  // nonzero once any tensor-core kernel reported a bounded wait running out
 int *tc_status_word(int device);  // device address of that status word (after tc_conv_init), else nullptr
+cudaError_t tc_conv_status_clear();  // synchronises the current device, then zeroes its status words and the sticky flag
+cudaError_t tc_expire_wait(unsigned limit_us, cudaStream_t st);  // a kernel whose only wait runs out after limit_us (test of the time-out path)
 
 // ---- grouped tensor-core convolution (sgs_conv_group.cu) -------------------------------------
 // One launch runs the same stored layer for up to TC_GROUP_MAX_ENTRIES members (queries in flight).

@@ -64,15 +64,16 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: false if the phase did not complete within WAIT_LIMIT_NS or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+// Bounded wait: false if the phase did not complete within limit_ns or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (;;) {
         for (int i = 0; i < 64; i++)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+        if (global_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
 }
 __device__ __forceinline__ uint64_t make_policy(int kind) {  // 0 normal, 1 evict-last, 2 evict-first

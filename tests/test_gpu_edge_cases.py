@@ -78,3 +78,33 @@ def test_repeated_configs_reuse_plans_and_agree():
     assert st.plan_misses <= 3                      # one plan per slot at most
     assert st.hit_ratio > 0.5                       # same SubNet over and over: after the first window the
     assert st.hbm_weight_bytes < 0.6 * st.weight_bytes  # cached SubGraph is the SubNet itself (paper App. A.4)
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    # Every device-side wait of the kernels carries a time limit.  A one-block test kernel of the library waits on a
+    # barrier nothing arrives at (limit 1 ms): it must return by itself, the status word must say so, the next stream
+    # call must report SGS_ETIMEOUT, and after clearing the status the same stream must pass parity again.
+    _, onet, gnet = gu.nets(wl.RESNET, True)
+    n, res = 4, 64
+    cfgs = wl.uniform_stream(wl.RESNET, n, seed=61)
+    xs = wl.make_inputs(n, 1, res, seed=9, bf16=True)
+    d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
+    d_out = torch.zeros((n, 1000), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    opts = sgs.StreamOpts(cache_enabled=1, window_q=2, record_latency=0, concurrency=1, wave=4)
+    torch.cuda.synchronize()
+    assert sgs.device_status() == 0
+    try:
+        sgs.debug_expire_wait(1000, stream.cuda_stream)
+        torch.cuda.synchronize()               # returns: the kernel ended on its own
+        assert sgs.device_status() != 0
+        with pytest.raises(sgs.SgsError) as e:
+            gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+        assert e.value.status == sgs.binding.SGS_ETIMEOUT
+    finally:
+        sgs.device_status_clear()
+    assert sgs.device_status() == 0
+    gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, d_out.data_ptr(), opts, stream.cuda_stream)
+    got = d_out.cpu().numpy()
+    for t in range(n):
+        assert gu.rel_err(got[t:t + 1], onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)) <= 2e-2

@@ -1,11 +1,12 @@
 """The allocation-free sliced convolution (sgs_conv2d_sliced_static) against sgs_conv2d_sliced.
 
-Some callers of the library cannot allocate device memory when they call it: they are inside a
-stream capture, they own all device memory through a pool of their own, or they cannot afford the
-device-wide synchronisation an allocation implies.  For them the library offers a variant whose
+Some callers of the library cannot allocate device memory when they call it: they own all device
+memory through a pool of their own, or they cannot afford the device-wide synchronisation an
+allocation implies.  For them the library offers a variant whose
 split-reduction scratch is a fixed array inside the library image.  This file checks, through the C
 interface, that the variant returns what the ordinary entry point returns (within the layer tests'
-tolerance, 1e-2 * max|ref|), on two calls in a row, and that it refuses work beyond its fixed scratch.
+tolerance, 1e-2 * max|ref|), on two calls in a row, that free device memory does not change across
+its calls, and that it refuses work beyond its fixed scratch.
 
 Collected last on purpose (file name), so a run that stops at the first failure has already run every
 other test.  It needs nothing from the other tests and passes in a fresh process as well.
@@ -43,12 +44,17 @@ def test_static_variant_matches_the_allocating_entry_point_twice(case):
     want = want.float().cpu().numpy()
     tol = 1e-2 * np.abs(ref).max()
     assert np.abs(want - ref).max() <= tol
-    for _ in range(2):  # the second call meets the array as the first one left it
-        got = torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
-        sgs.conv2d_sliced_static(desc, *args, got.data_ptr(), stream)
+    outs = [torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    sgs.conv2d_sliced_static(desc, *args, outs[0].data_ptr(), stream)  # the first call on a device does the one-time set-up
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for i in (1, 2):  # the second call meets the array as the first one left it
+        sgs.conv2d_sliced_static(desc, *args, outs[i].data_ptr(), stream)
         torch.cuda.synchronize()
-        got = got.float().cpu().numpy()
-        assert sgs.device_status() == 0
+        # no device memory was taken (the outputs were allocated before the measurement started)
+        assert torch.cuda.mem_get_info()[0] == free_before
+        got = outs[i].float().cpu().numpy()
+        assert sgs.device_status() == 0  # also reads the status word that lives inside the fixed array
         assert np.all(np.isfinite(got))
         assert np.abs(got - want).max() <= tol
         assert np.abs(got - ref).max() <= tol
@@ -75,3 +81,8 @@ def test_static_variant_rejects_what_it_cannot_hold():
     with pytest.raises(sgs.SgsError) as e:
         sgs.conv2d_sliced_static(d, x.data_ptr(), w.data_ptr(), sc.data_ptr(), sh.data_ptr(), 0, y.data_ptr())
     assert e.value.status == sgs.binding.SGS_EUNSUPPORTED
+    d = _desc(SPLIT_CASE)
+    d.impl = 7
+    with pytest.raises(sgs.SgsError) as e:
+        sgs.conv2d_sliced_static(d, x.data_ptr(), w.data_ptr(), sc.data_ptr(), sh.data_ptr(), 0, y.data_ptr())
+    assert e.value.status == sgs.binding.SGS_EINVAL
