@@ -201,8 +201,14 @@ sgs_status_t sgs_stream_run_host(sgs_supernet_t *net, int n_queries, const sgs_s
                                  const void *h_inputs, int batch_per_query, int res, void *h_logits,
                                  const sgs_stream_opts_t *opts, sgs_stream_stats_t *stats, void *cuda_stream);
 
-/* Configure the SubGraph cache used by sgs_subnet_run (sgs_stream_run takes its own options).
- * budget_bytes 0 = device maximum.  window_q >= 1. */
+/* sgs_cache_configure - the SubGraph cache used by sgs_subnet_run (sgs_stream_run takes its own options).
+ * budget_bytes plays the part of the Persistent Buffer's capacity (Section 4.2: the buffer that holds the cached
+ * SubGraph across queries); 0 = the most the device lets a process keep resident in L2.  window_q >= 1 is the
+ * number of queries a caching decision is amortised over (Section 3.3 "Amortizing Caching Choices", Appendix A.1:
+ * the cached SubGraph is re-chosen every Q queries from the last Q SubNets).  Errors: SGS_EINVAL.
+ * sgs_cache_stats - state of that cache: what the device offers, the budget in force, the bytes of the SubGraph
+ * currently marked resident (Section 4.3.1: the part of a query's weights that is not fetched again), and the
+ * policy's counters.  `out` is a host struct.  Errors: SGS_EINVAL. */
 sgs_status_t sgs_cache_configure(sgs_supernet_t *net, int enabled, size_t budget_bytes, int window_q);
 sgs_status_t sgs_cache_stats(const sgs_supernet_t *net, sgs_cache_stats_t *out);
 
@@ -276,7 +282,11 @@ sgs_status_t sgs_sched_subnet(const sgs_sched_t *sched, int i, sgs_subnet_cfg_t 
 int sgs_num_layers(const sgs_supernet_t *net);
 sgs_status_t sgs_subnet_encode(const sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, int *out);
 
-/* Useful FLOPs (2*M*K'*C'*k*k over sliced layers) and touched weight bytes of one query. */
+/* sgs_subnet_cost - what one query of SubNet `cfg` costs, from its slices alone (Section 2.1: the elastic choices
+ * fix which weights take part; Section 2.2 / Figure on arithmetic intensity: FLOPs against bytes moved decides
+ * whether a SubNet is memory bound): useful FLOPs (2*M*K'*C'*k*k over the sliced layers), the stored-weight bytes
+ * the SubNet touches, and the activation bytes its layers read and write.  Host pointers, any may be NULL.
+ * Errors: SGS_EINVAL, SGS_ECONFIG. */
 sgs_status_t sgs_subnet_cost(const sgs_supernet_t *net, const sgs_subnet_cfg_t *cfg, int batch, int res,
                              double *flops, double *weight_bytes, double *activation_bytes);
 
@@ -397,7 +407,8 @@ sgs_status_t sgs_device_status_clear(void);
 sgs_status_t sgs_debug_expire_wait(unsigned limit_us, void *cuda_stream);
 
 /* Library options by name (debug and measurement aids): "conv_impl" 0 = automatic, 1 = force the
- * CUDA-core kernels; "profile" see sgs_profile_read.  Unknown name -> SGS_EINVAL. */
+ * CUDA-core kernels; "profile" see sgs_profile_read; "stage_group" 0 = default, 1..4 = pipeline stages that
+ * share one barrier pair in the grouped convolution kernel (process-wide, a tuning aid).  Unknown name -> SGS_EINVAL. */
 sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long value);
 
 /*
@@ -435,7 +446,11 @@ int sgs_layer_name(const sgs_supernet_t *net, int layer, char *out, int cap);
  * launches / direct launches). */
 long long sgs_get_counter(const sgs_supernet_t *net, const char *name);
 
+/* Text of the last failure reported by a call on `net` (owned by the handle, valid until its next call); "null
+ * handle" for NULL.  Library housekeeping: the paper has no counterpart. */
 const char *sgs_last_error(const sgs_supernet_t *net);
+/* Releases the SuperNet (Section 2.1: the one stored set of weights) with every device and host resource the handle
+ * owns: weights, workspaces, plans, graphs, streams.  Synchronises the device first.  NULL is ignored. */
 void sgs_supernet_free(sgs_supernet_t *net);
 
 #ifdef __cplusplus

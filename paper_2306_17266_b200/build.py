@@ -48,14 +48,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
                     sys.stderr.write(r.stdout + r.stderr)
                 if r.returncode:
                     raise RuntimeError("nvcc failed: " + " ".join(r.args))
-    # the stand-alone copy-rate microbenchmark (python -m paper_2306_17266_b200.microbench copy-rate)
-    tool_src, tool = os.path.join(CSRC, "copy_rate.cu"), os.path.join(obj_dir, "copy_rate")
-    if force or _stale(tool, [tool_src]):
-        r = subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "-o", tool, tool_src, "-lcuda"],
-                           capture_output=True, text=True)
-        if r.returncode:
-            sys.stderr.write(r.stdout + r.stderr)
-            raise RuntimeError("nvcc failed: copy_rate.cu")
     objs = [os.path.join(obj_dir, s.replace(".cu", ".o")) for s in SOURCES]
     if force or jobs or _stale(LIB, objs):
         cmd = [_nvcc(), "-shared", "-o", LIB + ".tmp", *objs, "-lcudart"]

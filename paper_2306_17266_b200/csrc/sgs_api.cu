@@ -2158,9 +2158,15 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
         DeviceGuard guard(net->device);
         fold_profile(net);
         net->profile = value != 0;
-        if (value == 2 || value == 0)
+        if (value == 2 || value == 0) {
             for (int i = 0; i < 4; i++) { net->prof_ms[i] = net->prof_bytes[i] = net->prof_flops[i] = 0; net->prof_launches[i] = 0; }
             net->prof_trace.clear();
+        }
+        return SGS_OK;
+    }
+    if (n == "stage_group") {  // tuning aid: stages per barrier pair of the grouped convolution kernel (0 = default)
+        if (value < 0 || value > 4) return fail(net, SGS_EINVAL, "stage_group");
+        tc_group_set_stage_group((int)value);
         return SGS_OK;
     }
     return fail(net, SGS_EINVAL, "unknown option " + n);

@@ -22,9 +22,9 @@ namespace sgs {
 
 namespace {
 
-constexpr int G_MAX_STAGES = 6;
+constexpr int G_MAX_STAGES = 8;
 constexpr int G_X_BYTES = 128 * CHUNK_C * 2;  // operand on the MMA's row side: 128 rows
-constexpr int G_RING_BYTES = 192 * 1024;      // operand ring: 6 stages of 16 + 16 KB, or 4 stages of 16 + 32 KB (256-column tiles)
+constexpr int G_RING_BYTES = 192 * 1024;      // operand ring: 8 stages of 16 + 8 KB (tiles of at most 64 columns), 6 of 16 + 16 KB, or 4 of 16 + 32 KB (256-column tiles)
 constexpr int G_SMEM_BYTES = G_RING_BYTES + 1024;
 constexpr int G_ACC_COLS = 256;                   // tensor-memory columns of one accumulator buffer
 constexpr int G_EPI_WARPS = 8;                    // two groups of four (one warp per tensor-memory lane quadrant)
@@ -92,7 +92,8 @@ template <int NMAPS> struct GroupParams {
     int *status;
     int n_entries, total_tiles;
     int n_stages, stage_bytes;  // operand ring of this launch
-    int pad_[6];
+    int group;                  // consecutive stages that share one pair of barriers (n_stages is a multiple of it)
+    int pad_[5];
     CUtensorMap maps[NMAPS];
 };
 static_assert(sizeof(GroupParams<TC_GROUP_MAPS_LARGE>) <= 32764, "kernel parameter block");
@@ -119,8 +120,11 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
     for (int i = threadIdx.x; i < n_entries * (int)(sizeof(GroupEntry) / 16); i += blockDim.x)
         reinterpret_cast<uint4 *>(es)[i] = __ldg(reinterpret_cast<const uint4 *>(entries) + i);
     if (threadIdx.x == 0) {
-        // a stage is full once both producers' copies have landed; it is empty once its MMAs have read it
-        for (int s = 0; s < G_MAX_STAGES; s++) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
+        // Barriers are per GROUP of consecutive stages: a group is full once both producers' copies of all its
+        // stages have landed (each producer arrives once per stage), and empty once the MMAs of its last stage
+        // have read it.  One wait and one commit then serve `group` stages: the issuing threads pay their fixed
+        // cost per wait (a few hundred cycles) once per group instead of once per 64 channels.
+        for (int s = 0; s < G_MAX_STAGES; s++) { mbar_init(&full_bar[s], 2 * (uint32_t)P.group); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], G_EPI_WARPS / 2); }
         abort_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -130,7 +134,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
-    const int n_stages = P.n_stages, stage_bytes = P.stage_bytes;
+    const int n_stages = P.n_stages, stage_bytes = P.stage_bytes, gsz = P.group;
     pdl_launch_dependents();
 
     if (warp == 0) {
@@ -139,7 +143,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         // as far as the ring allows.  The warp runs its loop converged; one elected lane issues.
         const uint64_t pol_keep = make_policy(1), pol_stream = make_policy(2);
         const int weight_policy = cache_tbl ? __ldg(cache_tbl) : 0;
-        int s = 0;
+        int s = 0, g = 0, gi = 0;  // stage, its group, its position in the group
         uint32_t phase = 0;
         bool wrapped = false, ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
@@ -159,17 +163,18 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             for (int r = 0; r < k && ok; r++, tap_row += R) {
                 for (int sx = 0; sx < kw && ok; sx++) {
                     for (int cc = 0, c0 = 0; cc < cchunks; cc++, c0 += CHUNK_C) {
-                        if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag));
+                        if (wrapped && gi == 0) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[g], phase ^ 1, abort_flag));
                         if (!ok) break;
                         if (elect_one()) {
                             uint8_t *sb = dst0 + s * stage_bytes;
-                            mbar_expect_tx(&full_bar[s], w_bytes);
-                            if (kind == 2) tma_load_3d_hint(sb, map_w, &full_bar[s], c0, tap_row + sx, f0, pol_stream);
-                            else if (kind == 1 && c0 < cacheC) tma_load_3d_hint(sb, map_w, &full_bar[s], c0, tap_row + sx, f0, pol_keep);
-                            else tma_load_3d(sb, map_w, &full_bar[s], c0, tap_row + sx, f0);
+                            mbar_expect_tx(&full_bar[g], w_bytes);
+                            if (kind == 2) tma_load_3d_hint(sb, map_w, &full_bar[g], c0, tap_row + sx, f0, pol_stream);
+                            else if (kind == 1 && c0 < cacheC) tma_load_3d_hint(sb, map_w, &full_bar[g], c0, tap_row + sx, f0, pol_keep);
+                            else tma_load_3d(sb, map_w, &full_bar[g], c0, tap_row + sx, f0);
                         }
                         __syncwarp();
-                        if (++s == n_stages) { s = 0; phase ^= 1; wrapped = true; }
+                        if (++gi == gsz) { gi = 0; ++g; }
+                        if (++s == n_stages) { s = 0; g = 0; phase ^= 1; wrapped = true; }
                     }
                 }
             }
@@ -177,9 +182,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             if (ok && tn < total_tiles && elect_one()) prefetch_tensormap(&P.maps[es[find_entry_serial(es, n_entries, tn)].map_w]);
             __syncwarp();
         }
+        // the CTA's last group may be partial: arrive for the stages it does not have
+        if (gi != 0 && elect_one())
+            for (; gi < gsz; gi++) mbar_arrive(&full_bar[g]);
     } else if (warp == G_PIX_WARP) {
         // ------------------------------------------------------------------ activation producer
-        int s = 0;
+        int s = 0, g = 0, gi = 0;
         uint32_t phase = 0;
         bool wrapped = false, ok = true;
         pdl_wait();  // activations (and the buffers this layer overwrites) belong to the previous layers until here
@@ -201,16 +209,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                     const CUtensorMap *m = map_a + ph * 2 + pw;
                     const int cw = stride == 2 ? w0 + ((dw - pw) >> 1) : w0 + dw, ch = stride == 2 ? h0 + ((dh - ph) >> 1) : h0 + dh;
                     for (int cc = 0, c0 = 0; cc < cchunks; cc++, c0 += CHUNK_C) {
-                        if (wrapped) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[s], phase ^ 1, abort_flag));
+                        if (wrapped && gi == 0) ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[g], phase ^ 1, abort_flag));
                         if (!ok) break;
                         if (elect_one()) {
-                            mbar_expect_tx(&full_bar[s], pix_bytes + pix_bytes2);
-                            tma_load_4d(dst0 + s * stage_bytes, m, &full_bar[s], c0, cw, ch, n0);
+                            mbar_expect_tx(&full_bar[g], pix_bytes + pix_bytes2);
+                            tma_load_4d(dst0 + s * stage_bytes, m, &full_bar[g], c0, cw, ch, n0);
                             // (a pair is a single tile of one layer: same tap offsets and parity view, box origin 0)
-                            if (pix_bytes2) tma_load_4d(dst0 + s * stage_bytes + 64 * CHUNK_C * 2, map_a2 + (m - map_a), &full_bar[s], c0, cw, ch, n0);
+                            if (pix_bytes2) tma_load_4d(dst0 + s * stage_bytes + 64 * CHUNK_C * 2, map_a2 + (m - map_a), &full_bar[g], c0, cw, ch, n0);
                         }
                         __syncwarp();
-                        if (++s == n_stages) { s = 0; phase ^= 1; wrapped = true; }
+                        if (++gi == gsz) { gi = 0; ++g; }
+                        if (++s == n_stages) { s = 0; g = 0; phase ^= 1; wrapped = true; }
                     }
                 }
             }
@@ -218,9 +227,11 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             if (ok && tn < total_tiles && elect_one()) prefetch_tensormap(&P.maps[es[find_entry_serial(es, n_entries, tn)].map_a]);
             __syncwarp();
         }
+        if (gi != 0 && elect_one())
+            for (; gi < gsz; gi++) mbar_arrive(&full_bar[g]);
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        int s = 0;
+        int s = 0, g = 0, gi = 0;
         uint32_t phase = 0;
         int j = 0;
         const uint32_t ring = smem_u32(smem);
@@ -243,20 +254,23 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             uint32_t accumulate = 0;
             for (int tap = 0; tap < taps && ok; tap++) {
                 for (int cc = 0; cc < cchunks; cc++) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], phase, abort_flag));
-                    if (!ok) break;
-                    tc_fence_after();
+                    if (gi == 0) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[g], phase, abort_flag));
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
                     const int ksteps = cc == cchunks - 1 ? last_ksteps : CHUNK_C / 16;
                     const uint32_t sx_ = ring + (uint32_t)(s * stage_bytes);
                     const uint64_t da = smem_desc_sw128(sx_), db = smem_desc_sw128(sx_ + G_X_BYTES);
                     if (elect_one()) {
                         for (int q = 0; q < ksteps; q++) { umma_bf16(d_tmem, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), idesc, accumulate); accumulate = 1; }
-                        umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+                        if (gi == gsz - 1) umma_commit(&empty_bar[g]);  // frees the group once the MMAs of all its stages have read it
                         if (tap == taps - 1 && cc == cchunks - 1) umma_commit(&acc_full[buf]);  // accumulator complete
                     }
                     __syncwarp();
                     accumulate = 1;
-                    if (++s == n_stages) { s = 0; phase ^= 1; }
+                    if (++gi == gsz) { gi = 0; ++g; }
+                    if (++s == n_stages) { s = 0; g = 0; phase ^= 1; }
                 }
             }
         }
@@ -443,7 +457,7 @@ static int views_of(const TcParams &p) { return (p.stride == 2 && p.k > 1) ? 4 :
 struct GroupLaunch::Impl {
     GroupParams<TC_GROUP_MAPS_LARGE> prm;  // host image of the parameter block (the small variant is a prefix)
     int n_maps = 0;
-    bool wide = false;  // some member's column-side operand has more than 128 rows
+    int col_rows = 0;   // most rows any member's column-side operand has (64, 128 or 256: sizes the stages)
 };
 
 GroupLaunch::GroupLaunch() : impl(new Impl) { reset(nullptr); }
@@ -451,7 +465,7 @@ GroupLaunch::~GroupLaunch() { delete impl; }
 
 void GroupLaunch::reset(const void *d_entries) {
     impl->n_maps = 0;
-    impl->wide = false;
+    impl->col_rows = 0;
     impl->prm.entries = static_cast<const GroupEntry *>(d_entries);
     impl->prm.n_entries = 0;
     impl->prm.total_tiles = 0;
@@ -489,7 +503,7 @@ void GroupLaunch::add(void *host_entry, const TcConvPlan &pl, const ConvArgs &a)
     e.swap = (unsigned char)pl.swap;
     e.bn_tile = (short)(pl.swap ? (e.pix_rows + 15) / 16 * 16 : pl.bn_tile);
     e.k = (unsigned char)p.k; e.kw = (unsigned char)pl.kw; e.stride = (unsigned char)p.stride; e.p = (unsigned char)p.p; e.act = (unsigned char)p.act;
-    if ((pl.swap ? e.pix_rows : e.bn_tile) > 128) impl->wide = true;
+    impl->col_rows = std::max(impl->col_rows, (int)(pl.swap ? e.pix_rows : e.bn_tile));
     impl->prm.n_entries++;
     // Pairing: this member and the previous one of the launch each fit the lower / upper half of a tile's 128
     // rows, run the same stored layer, and one's slice contains the other's (filters and channels): they
@@ -513,6 +527,9 @@ void GroupLaunch::add(void *host_entry, const TcConvPlan &pl, const ConvArgs &a)
     impl->prm.total_tiles += e.mtiles * (int)pl.grid.y;
 }
 
+static int g_group_stages = 0;  // 0 = default
+void tc_group_set_stage_group(int stages) { g_group_stages = stages; }
+
 cudaError_t tc_group_init(int) {
     cudaError_t e = cudaFuncSetAttribute(conv_group_kernel<TC_GROUP_MAPS_SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
     if (e != cudaSuccess) return e;
@@ -527,9 +544,12 @@ cudaError_t GroupLaunch::launch(const int *cache_tbl, int sms, cudaStream_t st) 
     impl->prm.status = tc_status_word(dev);
     if (!impl->prm.status) return cudaErrorInitializationError;
     impl->prm.cache_tbl = cache_tbl;
-    // 256-column tiles need 16 + 32 KB per stage (4 stages); everything narrower gets 6 stages of 16 + 16 KB
-    impl->prm.stage_bytes = G_X_BYTES + (impl->wide ? 256 : 128) * CHUNK_C * 2;
-    impl->prm.n_stages = G_RING_BYTES / impl->prm.stage_bytes;
+    // stage = 16 KB for the row-side operand + room for the widest column-side operand of the launch
+    const int col_rows = impl->col_rows <= 64 ? 64 : impl->col_rows <= 128 ? 128 : 256;
+    impl->prm.stage_bytes = G_X_BYTES + col_rows * CHUNK_C * 2;
+    impl->prm.n_stages = G_RING_BYTES / impl->prm.stage_bytes;  // 8, 6 or 4
+    const int want = g_group_stages > 0 ? g_group_stages : 1;  // (measured on batch-16 members: 2 or 4 stages per barrier pair change nothing for narrow tiles and cost 10-25 % on 256-column tiles)
+    impl->prm.group = (want <= impl->prm.n_stages / 2 && impl->prm.n_stages % want == 0) ? want : 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)std::min(impl->prm.total_tiles, std::max(1, sms)));
     cfg.blockDim = dim3(G_THREADS);

@@ -193,5 +193,6 @@ private:
     Impl *impl;
 };
 cudaError_t tc_group_init(int device);
+void tc_group_set_stage_group(int stages);  // tuning: stages per barrier pair of the grouped kernel (0 = default)
 
 }  // namespace sgs

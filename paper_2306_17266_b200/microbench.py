@@ -135,19 +135,9 @@ def wave_trace(family, wave, queries, res, batch):
               f"{1e3 * a['ms'] / a['n']:7.1f} us  {100 * a['ms'] / total:5.1f} %  {a['bytes'] / a['ms'] / 1e6:8.1f} GB/s  {a['flops'] / a['ms'] / 1e9:7.1f} TFLOP/s")
 
 
-def copy_rate():
-    """Runs the stand-alone microbenchmark csrc/copy_rate.cu (copy rate into shared memory per SM, tiled boxes
-    against bulk copies); the package's build step compiles it."""
-    import os
-    import subprocess
-    from . import build
-    build.build()
-    subprocess.run([os.path.join(os.path.dirname(os.path.abspath(__file__)), "_build", "copy_rate")], check=True)
-
-
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["conv", "dw", "trace", "copy-rate"])
+    ap.add_argument("kind", choices=["conv", "dw", "trace"])
     ap.add_argument("--family", default="resnet", choices=["resnet", "mbv3"])
     ap.add_argument("--wave", type=int, default=32)
     ap.add_argument("--queries", type=int, default=128)
@@ -158,9 +148,6 @@ def main():
     ap.add_argument("--once", type=int, default=0, help="only run this many launches (profiling)")
     ap.add_argument("--split-off", type=int, default=0)
     args = ap.parse_args()
-    if args.kind == "copy-rate":
-        copy_rate()
-        return
     if args.kind == "trace":
         wave_trace(args.family, args.wave, args.queries, args.res, args.batch)
         return
