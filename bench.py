@@ -153,6 +153,81 @@ def _stream_pool(net, sgs, torch, cfgs, batch, res, opts, stream, pool_groups, f
     return tot
 
 
+SWEEP_WORKLOAD = ("ResNet-50-shaped SuperNet throughput sweep: batches of 64 = 4 SubNet configs x 16 images in one grouped launch per layer, "
+                  "configs uniform (seed 5)")
+
+
+def measure_sweep(net, sgs, torch, stream, peaks, n_groups=1250, resolutions=(160, 192, 224), cache=1, window=4, concurrency=4):
+    """Throughput sweep (waves of 4 members x 16 images): images/s, useful TFLOP/s and fractions of the bf16 peaks."""
+    cfgs = wl.uniform_stream(wl.RESNET, n_groups, seed=5)
+    rows = []
+    for res in resolutions:
+        opts = sgs.StreamOpts(cache_enabled=cache, window_q=window, cache_budget_bytes=0, use_graphs=1, record_latency=0,
+                              concurrency=concurrency, wave=4)
+        _stream_pool(net, sgs, torch, cfgs[:64], 16, res, opts, stream, 64, wl.RESNET)  # warm-up: workspaces
+        t = _stream_pool(net, sgs, torch, cfgs, 16, res, opts, stream, 64, wl.RESNET)
+        tf = t["flops"] / (t["ms"] * 1e-3) / 1e12
+        rows.append({"res": res, "images": t["q"] * 16, "images_per_s": t["q"] * 16 / (t["ms"] * 1e-3), "useful_tflops": tf,
+                     "frac_of_bf16_sustained_peak": tf / peaks["bf16_tflops_sustained"], "frac_of_bf16_burst_peak": tf / peaks["bf16_tflops"],
+                     "gflop_per_image": t["flops"] / (t["q"] * 16) / 1e9, "ms": t["ms"]})
+    return rows
+
+
+def measure_mbv3(sgs, torch, stream, queries=1000, wave=32, concurrency=4, cache=1, window=4, profile=False):
+    """The MobileNetV3-shaped stream (1000 queries, batch 1, 224x224, configs uniform seed 3)."""
+    net = sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16)
+    cfgs = wl.uniform_stream(wl.MBV3, queries, seed=3)
+    opts = sgs.StreamOpts(cache_enabled=cache, window_q=window, cache_budget_bytes=0, use_graphs=1, record_latency=1,
+                          concurrency=concurrency, wave=wave)
+    for _ in range(2):
+        _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
+    t = _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
+    out = {"queries_per_s": t["q"] / (t["ms"] * 1e-3), "p50_ms": float(np.median(t["p50"])), "gflop_per_query": t["flops"] / t["q"] / 1e9,
+           "kernel_launches_per_query": t["launches"] / t["q"],
+           "execution": f"waves of {wave}, {concurrency} in flight" if wave > 0 else f"one stream per query, {concurrency} in flight"}
+    if profile:
+        net.set_option("profile", 2)
+        popts = sgs.StreamOpts(cache_enabled=cache, window_q=window, cache_budget_bytes=0, use_graphs=0, record_latency=0, wave=wave)
+        _stream_pool(net, sgs, torch, cfgs, 1, 224, popts, stream, len(cfgs), wl.MBV3)
+        prof = [net.profile_read(c) for c in range(4)]
+        net.set_option("profile", 0)
+        out["kernel_time_ms_by_class"] = {"conv_tc": prof[0]["total_ms"], "conv_cuda_core": prof[1]["total_ms"],
+                                          "depthwise": prof[2]["total_ms"], "other": prof[3]["total_ms"]}
+        out["depthwise_gbs_at_batch1"] = prof[2]["alg_bytes"] / (prof[2]["total_ms"] * 1e-3) / 1e9 if prof[2]["total_ms"] else None
+    net.close()
+    return out
+
+
+def measure_depthwise(sgs, peaks, fma_tflops):
+    """Depthwise kernels on working sets larger than L2 (64 x 56 x 56 x 480 bf16 in, same or a quarter out): GB/s of
+    algorithmic bytes (input + output), fraction of the HBM peak, and for the 5x5 / 7x7 windows the fraction of the
+    measured fp32 FMA rate (2 * k * k FLOP per output element)."""
+    from paper_2306_17266_b200 import microbench
+    rows = []
+    for shape in microbench.DW_PRESETS["large"][:6]:
+        r = microbench.bench_dw(shape)
+        N, H, W, K, k, stride = shape
+        outs = N * (H // stride) * (W // stride) * K
+        tf = 2.0 * k * k * outs / r["us"] / 1e6
+        rows.append({"k": k, "stride": stride, "shape": f"{N}x{H}x{W}x{K}", "us": r["us"], "gbs": r["gbs"], "frac_of_hbm_peak": r["gbs"] / peaks["hbm_gbs"],
+                     "fma_tflops": tf, "frac_of_fma_peak": tf / fma_tflops if fma_tflops else None})
+    return rows
+
+
+def measure_plan_miss(net, sgs, torch, stream, x_dev, logits, opts, n=1000):
+    """What a never-seen config costs: the plan cache is emptied, a stream of `n` fresh configs (uniform, seed 99) runs
+    once cold and once warm; the difference per planned query is host planning + tensor-map encoding."""
+    cfgs = wl.cfg_array(wl.uniform_stream(wl.RESNET, n, seed=99))
+    net.set_option("drop_plans", 1)
+    cold = net.stream_run(cfgs, x_dev.data_ptr(), BATCH, RES, logits.data_ptr(), opts, stream.cuda_stream)
+    warm = net.stream_run(cfgs, x_dev.data_ptr(), BATCH, RES, logits.data_ptr(), opts, stream.cuda_stream)
+    misses = max(1, cold.plan_misses)
+    return {"fresh_configs": n, "plan_misses_cold": cold.plan_misses, "plan_misses_warm": warm.plan_misses,
+            "cold_queries_per_s": cold.queries_per_s, "warm_queries_per_s": warm.queries_per_s,
+            "us_per_never_seen_config": (cold.total_ms - warm.total_ms) * 1e3 / misses,
+            "note": "device-timed stream with the plan cache emptied first (cold) against the same stream again (warm)"}
+
+
 def run_suite(args):
     import torch
     import paper_2306_17266_b200 as sgs
@@ -163,59 +238,56 @@ def run_suite(args):
         # throughput sweep: 20k images as groups of 16 images sharing a config (4 groups = one batch of 64)
         net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
         n_groups = args.queries // 16 if args.queries != 1000 else 1250
-        cfgs = wl.uniform_stream(wl.RESNET, n_groups, seed=5)
-        rows = []
-        for res in (160, 192, 224):
-            # one launch per layer covers the 4 configs of a batch of 64 (wave of 4 members x 16 images)
-            opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=0,
-                                  concurrency=args.concurrency, wave=min(args.wave, 4))
-            _stream_pool(net, sgs, torch, cfgs[:64], 16, res, opts, stream, 64, wl.RESNET)  # warm-up: plans
-            t = _stream_pool(net, sgs, torch, cfgs, 16, res, opts, stream, 64, wl.RESNET)
-            tf = t["flops"] / (t["ms"] * 1e-3) / 1e12
-            rows.append({"res": res, "images_per_s": t["q"] * 16 / (t["ms"] * 1e-3), "useful_tflops": tf,
-                         "frac_of_bf16_sustained_peak": tf / peaks["bf16_tflops_sustained"], "frac_of_bf16_burst_peak": tf / peaks["bf16_tflops"],
-                         "gflop_per_image": t["flops"] / (t["q"] * 16) / 1e9, "ms": t["ms"]})
+        rows = measure_sweep(net, sgs, torch, stream, peaks, n_groups, cache=args.cache, window=args.window, concurrency=args.concurrency)
         out.update({"metric": "subnet_images_per_s", "unit": "images/s", "value": rows[-1]["images_per_s"], "rows": rows,
-                    "config": {"workload": "ResNet-50-shaped SuperNet throughput sweep, 16 images per SubNet config, 20k images per resolution, configs uniform (seed 5)",
-                               "peaks": peaks}})
+                    "config": {"workload": SWEEP_WORKLOAD + ", 20k images per resolution", "peaks": peaks}})
     elif args.suite == "sgs":
-        # locality stream: Markov chain of configs; cache on / off, window Q in {1, 4, 8}, batch 1 and 16
+        # locality stream: Markov chain of configs; cache on / off, window Q in {1, 4, 8}, batch 1 (waves of 32) and
+        # batch 16 (waves of 4 configs x 16 images), the execution modes of the stream and sweep benchmarks
         net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
         n = args.queries if args.queries != 1000 else 5000
         cfgs = wl.markov_stream(n, seed=4)
         rows = []
-        for batch, nq in ((1, n), (16, max(64, n // 8))):
-            pool = 500 if batch == 1 else 32
+        for batch, nq, wave in ((1, n, 32), (16, max(64, n // 8), 4)):
+            pool = 512 if batch == 1 else 32
             warm = sgs.StreamOpts(cache_enabled=0, window_q=4, cache_budget_bytes=0, use_graphs=1, record_latency=0, weights_evict_first=0,
-                                  concurrency=args.concurrency)
-            _stream_pool(net, sgs, torch, cfgs[:nq], batch, 224, warm, stream, pool, wl.RESNET)  # builds every plan and graph
-            for cache, q, ef in ((0, 4, 0), (0, 4, 1), (1, 1, 0), (1, 4, 0), (1, 8, 0)):
-                opts = sgs.StreamOpts(cache_enabled=cache, window_q=q, cache_budget_bytes=0, use_graphs=1, record_latency=1, weights_evict_first=ef, concurrency=args.concurrency)
+                                  concurrency=args.concurrency, wave=wave)
+            _stream_pool(net, sgs, torch, cfgs[:nq], batch, 224, warm, stream, pool, wl.RESNET)  # builds every plan
+            for cache, q, ef, mech in ((0, 4, 0, 0), (0, 4, 1, 0), (1, 1, 0, 0), (1, 4, 0, 0), (1, 8, 0, 0), (1, 4, 0, 1), (1, 4, 0, 2)):
+                net.set_option("cache_mechanism", mech)
+                opts = sgs.StreamOpts(cache_enabled=cache, window_q=q, cache_budget_bytes=0, use_graphs=1, record_latency=1, weights_evict_first=ef,
+                                      concurrency=args.concurrency, wave=wave)
                 _stream_pool(net, sgs, torch, cfgs[:pool], batch, 224, opts, stream, pool, wl.RESNET)
                 t = _stream_pool(net, sgs, torch, cfgs[:nq], batch, 224, opts, stream, pool, wl.RESNET)
-                rows.append({"batch": batch, "cache": cache, "window_q": q, "weights_evict_first": ef, "queries": t["q"],
+                rows.append({"batch": batch, "wave": wave, "cache": cache, "window_q": q, "weights_evict_first": ef,
+                             "mechanism": ["tile hints", "launch window", "both"][mech] if cache else None, "queries": t["q"],
                              "queries_per_s": t["q"] / (t["ms"] * 1e-3), "p50_ms": float(np.median(t["p50"])),
                              "weight_mb_per_query": t["wbytes"] / t["q"] / 1e6, "hbm_weight_mb_per_query": t["miss"] / t["q"] / 1e6,
                              "hit_ratio": t["hit"] / t["q"]})
+            net.set_option("cache_mechanism", 0)
         out.update({"metric": "hbm_weight_bytes_per_query", "unit": "MB/query (analytic)", "value": rows[3]["hbm_weight_mb_per_query"], "rows": rows,
                     "config": {"workload": "SGS locality stream on the ResNet-50-shaped SuperNet: Markov chain of configs (p=0.9 one stage's depth or width changes), seed 4, 224x224",
-                               "note": "the cached SubGraph restarts at every pool boundary (500 queries at batch 1, 32 at batch 16)"}})
+                               "note": "the cached SubGraph restarts at every pool boundary (512 queries at batch 1, 32 at batch 16)"}})
     elif args.suite == "sgs-probe":
-        # one short locality stream, one variant, one query at a time, no graphs: meant to be run under a
-        # profiler that sums DRAM bytes over the kernels of the measured part (its launch range is printed)
+        # one short locality stream, one variant, one wave (or query) at a time: meant to be run under a profiler that
+        # sums DRAM bytes over the convolution kernels of the measured part (its launch range is printed)
         net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
         n = args.queries if args.queries != 1000 else 48
-        cfgs = wl.markov_stream(16 + n, seed=4)
-        opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=0, record_latency=0,
-                              weights_evict_first=args.evict_first, concurrency=1)
+        warm_n = 16
+        cfgs = wl.markov_stream(warm_n + n, seed=4)
+        net.set_option("cache_mechanism", args.mechanism)
+        opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=args.budget_mb << 20, use_graphs=0, record_latency=0,
+                              weights_evict_first=args.evict_first, concurrency=1, wave=args.wave)
         before = net.get_counter("kernel_launches")
-        _stream_pool(net, sgs, torch, cfgs[:16], args.batch, 224, opts, stream, 16, wl.RESNET)
+        _stream_pool(net, sgs, torch, cfgs[:warm_n], args.batch, 224, opts, stream, warm_n, wl.RESNET)
         skip = net.get_counter("kernel_launches") - before
-        t = _stream_pool(net, sgs, torch, cfgs[16:], args.batch, 224, opts, stream, n, wl.RESNET)
+        tcs = net.get_counter("tc_convs")
+        t = _stream_pool(net, sgs, torch, cfgs[warm_n:], args.batch, 224, opts, stream, n, wl.RESNET)
         out.update({"metric": "hbm_weight_bytes_per_query", "unit": "MB/query (analytic)", "value": t["miss"] / t["q"] / 1e6,
                     "weight_mb_per_query": t["wbytes"] / t["q"] / 1e6, "hit_ratio": t["hit"] / t["q"], "queries": t["q"],
                     "launches_before_measured_part": skip, "launches_in_measured_part": t["launches"],
-                    "config": {"batch": args.batch, "cache": args.cache, "window_q": args.window, "weights_evict_first": args.evict_first,
+                    "config": {"batch": args.batch, "wave": args.wave, "cache": args.cache, "window_q": args.window, "weights_evict_first": args.evict_first,
+                               "mechanism": args.mechanism, "budget_mb": args.budget_mb,
                                "note": "load-time kernels precede the warm-up launches; count them with the profiler's launch list"}})
     elif args.suite == "sched":
         # caching decision of Algorithm 1 (nearest candidate SubGraph to the running average) beside the
@@ -285,48 +357,37 @@ def run_suite(args):
                     "config": {"workload": f"ResNet-50-shaped SuperNet, {n_sub} SubNets x ({n_cand} candidate SubGraphs + empty cache), batch {batch}, 224x224; one query at a time, 256 MB overwritten before every timed run, median of 9",
                                "scheduler": f"Algorithm 1 with Q = {args.window} on 100000 synthetic (policy, A_t, L_t) queries (seed 8); step_ns includes the caching decision every Q queries"}})
     elif args.suite == "mbv3":
-        net = sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16)
-        cfgs = wl.uniform_stream(wl.MBV3, args.queries, seed=3)
-        opts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=1, record_latency=1,
-                              concurrency=args.concurrency, wave=args.wave)
-        _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
-        t = _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
-        net.set_option("profile", 2)
-        popts = sgs.StreamOpts(cache_enabled=args.cache, window_q=args.window, cache_budget_bytes=0, use_graphs=0, record_latency=0, wave=args.wave)
-        _stream_pool(net, sgs, torch, cfgs, 1, 224, popts, stream, len(cfgs), wl.MBV3)
-        prof = [net.profile_read(c) for c in range(4)]
-        net.set_option("profile", 0)
-        out.update({"metric": METRIC, "unit": UNIT, "value": t["q"] / (t["ms"] * 1e-3), "p50_ms": float(np.median(t["p50"])),
-                    "gflop_per_query": t["flops"] / t["q"] / 1e9, "kernel_launches_per_query": t["launches"] / t["q"],
-                    "kernel_time_ms_by_class": {"conv_tc": prof[0]["total_ms"], "conv_cuda_core": prof[1]["total_ms"],
-                                                "depthwise": prof[2]["total_ms"], "other": prof[3]["total_ms"]},
-                    "depthwise_gbs_at_batch1": prof[2]["alg_bytes"] / (prof[2]["total_ms"] * 1e-3) / 1e9 if prof[2]["total_ms"] else None,
+        r = measure_mbv3(sgs, torch, stream, args.queries, args.wave, args.concurrency, args.cache, args.window, profile=True)
+        out.update({"metric": METRIC, "unit": UNIT, "value": r["queries_per_s"], **r,
                     "config": {"workload": "MobileNetV3-shaped SuperNet, 1000-query stream at batch 1, 224x224, configs uniform (seed 3)",
-                               "execution": f"waves of {args.wave}, {args.concurrency} in flight" if args.wave > 0 else f"one stream per query, {args.concurrency} in flight"}})
+                               "execution": r["execution"]}})
+    elif args.suite == "dw":
+        fma = sgs.measure_fma_peak(stream.cuda_stream)
+        rows = measure_depthwise(sgs, peaks, fma)
+        out.update({"metric": "depthwise_gbs", "unit": "GB/s (input + output bytes)", "value": rows[0]["gbs"], "rows": rows, "fp32_fma_tflops_measured": fma,
+                    "config": {"workload": "depthwise k x k (centre window of the stored 7x7), 64 x 56 x 56 x 480 bf16, h-swish, working set beyond L2", "peaks": peaks}})
     print(json.dumps(out))
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per conv_group_kernel launch, from the one-pass ncu capture
-# summarised in profiles/conv_group_wave32_resnet_b1.md.  Valid only for the kernel source it was taken
-# on: once that file changes the figure is reported as null.
-NCU_TRAFFIC = {
-    "kernel_source_sha256_16": "1ac81309430c617d",
-    "bytes_per_launch": 15250000,
-    "note": "ncu flushes the caches before every launch: cold-cache reads; writes that still sit in L2 when the kernel ends are not counted",
-}
-
-
-def ncu_traffic_per_launch(grouped=True):
+def ncu_record(name):
+    """Counters taken under the profiler cannot be measured inside a timed run; they are read from the `key: value`
+    lines of a small record kept beside the profile summaries.  A record carries the hash of the kernel source it was
+    taken on: once that source changes the figures are reported as null."""
     import hashlib
-    if not grouped:
-        return None
-    src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2306_17266_b200", "csrc", "sgs_conv_group.cu")
+    path = os.path.join(ROOT, "profiles", name)
+    rec = {}
     try:
-        with open(src, "rb") as f:
-            h = hashlib.sha256(f.read()).hexdigest()[:16]
-    except OSError:
+        with open(path) as f:
+            for line in f:
+                if ":" in line and not line.startswith("#"):
+                    k, v = line.split(":", 1)
+                    rec[k.strip()] = v.strip()
+        with open(os.path.join(ROOT, "paper_2306_17266_b200", "csrc", rec["kernel_source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest()[:16] != rec["kernel_source_sha256_16"]:
+                return None
+    except (OSError, KeyError):
         return None
-    return NCU_TRAFFIC["bytes_per_launch"] if h == NCU_TRAFFIC["kernel_source_sha256_16"] else None
+    return rec
 
 
 def main():
@@ -342,14 +403,16 @@ def main():
     ap.add_argument("--window", type=int, default=4)
     ap.add_argument("--wave", type=int, default=32, help="queries per wave (grouped launches over the wave's members); 0 = one stream per query")
     ap.add_argument("--concurrency", type=int, default=None, help="waves in flight (default 4), or with --wave 0 queries in flight (default 16)")
+    ap.add_argument("--quick", action="store_true", help="default line without the sweep / depthwise / MobileNetV3 / plan-miss measurements")
+    ap.add_argument("--sweep-groups", type=int, default=1250, help="16-image groups per resolution of the sweep measured inside the default line")
     ap.add_argument("--batch", type=int, default=1, help="images per query (sgs-probe)")
     ap.add_argument("--evict-first", type=int, default=0, help="with --cache 0: mark weight loads evict-first (sgs-probe)")
+    ap.add_argument("--mechanism", type=int, default=0, help="sgs-probe: 0 per-tile L2 hints, 1 access-policy window per launch, 2 both")
+    ap.add_argument("--budget-mb", type=int, default=0, help="sgs-probe: cache budget in MiB (0 = device maximum)")
     ap.add_argument("--family", default="resnet", choices=["resnet", "mbv3"], help="SuperNet of the sched suite")
-    ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3", "sched", "table"],
+    ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3", "sched", "table", "dw"],
                     help="stream = the default benchmark line; the others measure one more configuration each")
     args = ap.parse_args()
-    if args.suite in ("sgs", "sgs-probe"):
-        args.wave = 0  # these suites run one stream per query (cache on / off comparisons and the DRAM probe)
     if args.concurrency is None:
         args.concurrency = 4 if args.wave > 0 else 16
     if args.impl == "reference":
@@ -380,7 +443,15 @@ def main():
     blob = wl.make_blob(wl.RESNET, seed=0, bf16_weights=True)
     net = sgs.SuperNet(wl.RESNET, blob, sgs.SGS_BF16, device=local)
     from paper_2306_17266_b200 import replicas
-    cfgs = replicas.rotated_stream(wl.uniform_stream(wl.RESNET, 1000, seed=2), rank, nq)
+    # N replicas serve a stream of N * nq queries (weak scaling); queries whose SubNets are close in the vector
+    # encoding go to the same replica, so that each replica's SubGraph cache sees a larger common SubGraph.  Every
+    # rank computes the same partition by itself.  With one replica the shard is the stream as it is.
+    base = wl.uniform_stream(wl.RESNET, nq * world, seed=2)
+    if world > 1:
+        enc = np.stack([np.asarray(net.subnet_encode(c)).reshape(-1, 3)[:, :2].reshape(-1) for c in base])
+        cfgs = [base[q] for q in replicas.affinity_shards(enc, world)[rank]]
+    else:
+        cfgs = base
     arr = wl.cfg_array(cfgs)
     x_host = torch.from_numpy(wl.make_inputs(nq, BATCH, RES, seed=1 + rank, bf16=True).reshape(nq * BATCH, RES, RES, 3))
     x_host = x_host.to(torch.bfloat16).contiguous().pin_memory()
@@ -446,7 +517,7 @@ def main():
         # region, so its launches are timed in one more pass of the same stream with one wave at a time: an
         # event pair on the launching stream around every launch, the stream held by a sleeping kernel while
         # the host queues the wave (the intervals then hold device time, not launch latency).
-        seq = step(o=mk_opts(conc=1, wave=0))
+        step(o=mk_opts(conc=1, wave=0))  # (first pass: plans and graphs of this execution mode)
         seq_lat = step(o=mk_opts(conc=1, latency=1, wave=0))
         net.set_option("profile", 2)
         step(o=mk_opts(graphs=0))
@@ -456,24 +527,61 @@ def main():
         total_ms = sum(p["total_ms"] for p in prof)
         share = tc["total_ms"] / total_ms if total_ms > 0 else 0.0
         sec = tc["total_ms"] * 1e-3
+        n_launch = max(1, tc["launches"])
+        us_launch = sec * 1e6 / n_launch
         achieved_gbs = tc["alg_bytes"] / sec / 1e9 if sec > 0 else 0.0
         achieved_tf = tc["flops"] / sec / 1e12 if sec > 0 else 0.0
         grouped = args.wave > 0
+        rec = ncu_record("conv_group_wave32_resnet_b1.counters.txt") if grouped else None
+        traffic = float(rec["dram_bytes_per_launch"]) if rec else None
+        ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+        flop_per_launch = tc["flops"] / n_launch
+        # what bounds a launch: FLOP per byte that actually crosses the DRAM interface (members of a wave share the
+        # weights they have in common) against the ridge of the measured peaks; per ALGORITHMIC byte when there is no
+        # counter for the kernel as it stands
+        intensity = flop_per_launch / traffic if traffic else tc["flops"] / max(1.0, tc["alg_bytes"])
+        bound = "tensor" if intensity >= ridge else "hbm"
+        in_flight_gbs = sum(p["alg_bytes"] for p in prof) / (ms / args.steps * 1e-3) / 1e9
+        in_flight_tf = st_lat.useful_flops / (ms / args.steps * 1e-3) / 1e12
+        hbm_view = {"achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved_gbs / peaks["hbm_gbs"],
+                    "what": "algorithmic bytes (sliced weights + input + output + residual of every member) / launch time, launches timed one wave at a time"}
+        tensor_view = {"achieved": achieved_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"],
+                       "what": "useful FLOPs (2*M*K'*C'*k*k on the sliced extents) / launch time, launches timed one wave at a time; burst bf16 peak"}
+        head = tensor_view if bound == "tensor" else hbm_view
         roofline = {
             "kernel": ("conv_group_kernel (one launch = one stored layer for all members of a wave; sliced implicit GEMM, tcgen05 + TMA)" if grouped
                        else "conv_tc_kernel (sliced implicit-GEMM convolution, tcgen05 + TMA)"),
-            "bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic_per_launch(grouped), "traffic_note": NCU_TRAFFIC["note"],
+            "bound": bound, "achieved": head["achieved"], "peak": head["peak"], "unit": head["unit"], "frac": head["frac"],
+            "traffic": traffic,
+            "traffic_note": (rec or {}).get("note", "no counter record for the kernel source as it stands"),
             "peak_source": peaks["source"],
-            "launches": tc["launches"], "avg_launch_us": sec * 1e6 / max(1, tc["launches"]),
-            "method": "CUDA events around every launch, one wave at a time, host launch latency hidden behind a sleeping kernel; "
-                      "achieved = algorithmic bytes (sliced weights + input + output + residual of every member) / summed launch time",
-            "alg_bytes_per_launch": tc["alg_bytes"] / max(1, tc["launches"]),
+            "intensity_flop_per_dram_byte": intensity, "ridge_flop_per_byte": ridge,
+            "launches": tc["launches"], "avg_launch_us": us_launch,
+            "method": "CUDA events around every launch on the launching stream, one wave at a time, host launch latency hidden behind a sleeping kernel",
+            "alg_bytes_per_launch": tc["alg_bytes"] / n_launch, "flop_per_launch": flop_per_launch,
             "share_of_kernel_time": share,
-            "tensor_tflops": achieved_tf, "tensor_frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"],
+            "isolated_launch": {"tensor": tensor_view, "hbm_algorithmic": hbm_view,
+                                "dram_measured": ({"achieved": traffic / (us_launch * 1e-6) / 1e9, "unit": "GB/s", "frac": traffic / (us_launch * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                                                   "what": "DRAM read + write bytes per launch from the profiler's counters / launch time"} if traffic else None)},
+            "in_flight": {"what": "the timed region itself (waves overlap; all kernels together): algorithmic bytes and useful FLOPs of a step / ms_per_step",
+                          "alg_gbs": in_flight_gbs, "frac_of_hbm_peak": in_flight_gbs / peaks["hbm_gbs"],
+                          "useful_tflops": in_flight_tf, "frac_of_bf16_burst_peak": in_flight_tf / peaks["bf16_tflops"],
+                          "frac_of_bf16_sustained_peak": in_flight_tf / peaks["bf16_tflops_sustained"]},
             "kernel_time_ms_by_class": {"conv_tc": prof[0]["total_ms"], "conv_cuda_core": prof[1]["total_ms"],
                                         "depthwise": prof[2]["total_ms"], "other": prof[3]["total_ms"]},
         }
+        extras = {}
+        if world == 1 and not args.quick:
+            extras["plan_miss"] = measure_plan_miss(net, sgs, torch, stream, x_dev, logits, mk_opts())
+            sweep_rows = measure_sweep(net, sgs, torch, stream, peaks, n_groups=args.sweep_groups, concurrency=args.concurrency)
+            extras["sweep"] = {"workload": SWEEP_WORKLOAD + f", {args.sweep_groups * 16} images per resolution", "rows": sweep_rows}
+            fma = sgs.measure_fma_peak(stream.cuda_stream)
+            extras["depthwise"] = {"workload": "depthwise k x k (centre window of the stored 7x7), 64 x 56 x 56 x 480 bf16, h-swish: working set beyond L2",
+                                   "fp32_fma_tflops_measured": fma, "rows": measure_depthwise(sgs, peaks, fma)}
+            extras["mbv3"] = {"workload": "MobileNetV3-shaped SuperNet, 1000-query stream at batch 1, 224x224, configs uniform (seed 3)",
+                              **measure_mbv3(sgs, torch, stream, 1000, args.wave, args.concurrency, args.cache, args.window)}
+            sgs_rec = ncu_record("sgs_cache_wave_dram_bytes.counters.txt")
+            extras["sgs_measured"] = sgs_rec
         cpu = None
         if args.cpu_queries > 0 and world == 1:
             qps, dt, cores = cpu_oracle_qps(args.cpu_queries)
@@ -489,12 +597,13 @@ def main():
                        "cache": bool(args.cache), "window_q": args.window,
                        "execution": (f"waves of {args.wave} queries, one grouped launch per layer, {args.concurrency} waves in flight" if args.wave > 0
                                      else f"one stream per query, {args.concurrency} queries in flight"),
-                       "parallelism": f"replicas x{world}"},
+                       "parallelism": f"replicas x{world}" + (", stream sharded by config affinity" if world > 1 else "")},
             "p50_ms": st_lat.p50_ms, "p99_ms": st_lat.p99_ms, "mean_ms": st_lat.mean_ms,
             "one_query_at_a_time": {"queries_per_s": seq_lat.queries_per_s, "p50_ms": seq_lat.p50_ms, "p99_ms": seq_lat.p99_ms},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_bytes},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu,
             "useful_tflops": st_lat.useful_flops / (st_lat.total_ms * 1e-3) / 1e12,
+            **extras,
             "sgs": {"weight_bytes_per_query": st_lat.weight_bytes / nq, "hbm_weight_bytes_per_query": st_lat.hbm_weight_bytes / nq,
                     "hit_ratio": st_lat.hit_ratio, "byte_hit_ratio": st_lat.byte_hit_ratio, "cache_updates": st_lat.cache_updates,
                     "budget_bytes": cs.budget_bytes, "l2_bytes": cs.l2_bytes},

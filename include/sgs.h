@@ -102,8 +102,9 @@ typedef struct {
                            GPU although a single batch-1 SubNet cannot.  `concurrency` then counts waves
                            in flight (0 = 2, at most 8) and use_graphs is ignored.  Every query of a wave
                            starts and ends with its wave (that is its recorded latency).  The cached
-                           SubGraph is still re-chosen in stream order; the L2 hints of a wave use the
-                           choice in force when the wave was issued. */
+                           SubGraph is still re-chosen in stream order, and every member's weight loads carry
+                           the choice in force when ITS query is served (a wave of 32 with window_q = 4 sees
+                           eight choices). */
     int policy;         /* how the cached SubGraph is chosen every window_q queries:
                            SGS_POLICY_INTERSECTION (0): the SubGraph common to the last window_q SubNets;
                            SGS_POLICY_AVGNET (1): Algorithm 1 - the candidate SubGraph (sgs_cache_set_candidates)
@@ -401,13 +402,25 @@ int sgs_device_status(void);
 /* Synchronises the current device, zeroes its status words and forgets earlier time-outs. */
 sgs_status_t sgs_device_status_clear(void);
 
+/* Measurement aid: the fp32 fused-multiply-add rate of the device's CUDA cores in TFLOP/s (2 FLOP per FMA), from a
+ * kernel of independent register-only FMA chains, best of four timed launches on `cuda_stream`.  It is the ceiling
+ * for the depthwise kernels with 5x5 and 7x7 windows, whose arithmetic intensity exceeds what the CUDA cores
+ * sustain per byte of HBM traffic (paper Section 4.4: depthwise layers have the least reuse).  Allocates a small
+ * scratch buffer and synchronises. */
+sgs_status_t sgs_measure_fma_peak(double *tflops, void *cuda_stream);
+
 /* Test aid for the time-out path: enqueues a one-block kernel on `cuda_stream` whose only wait can never be
  * satisfied, with a limit of limit_us microseconds (1 .. 1000000).  The kernel gives up after the limit, sets the
  * device status word exactly as the convolution kernels do, and returns normally; nothing faults or hangs. */
 sgs_status_t sgs_debug_expire_wait(unsigned limit_us, void *cuda_stream);
 
 /* Library options by name (debug and measurement aids): "conv_impl" 0 = automatic, 1 = force the
- * CUDA-core kernels; "profile" see sgs_profile_read; "stage_group" 0 = default, 1..4 = pipeline stages that
+ * CUDA-core kernels; "pad_channels" 1 (default) = waves of the ResNet-shaped family keep their activation tensors
+ * at 16-channel pixels (zeros beyond the slice), 0 = dense pixels; "cache_mechanism" how grouped launches keep the cached SubGraph in L2: 0 (default) = an evict-last
+ * hint on every weight tile inside the SubGraph's box, 1 = an access-policy window on the launch (the cached filter
+ * prefix of the launch's stored layer, persisting; the persisting-L2 carve-out of the process is sized to the cache
+ * budget), 2 = both; "drop_plans" forgets every cached plan (measuring what a never-seen config costs); "profile" see
+ * sgs_profile_read; "stage_group" 0 = default, 1..4 = pipeline stages that
  * share one barrier pair in the grouped convolution kernel (process-wide, a tuning aid).  Unknown name -> SGS_EINVAL. */
 sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long value);
 

@@ -27,7 +27,7 @@ EXPORTS = [
     "sgs_set_option", "sgs_get_counter", "sgs_last_error", "sgs_supernet_free", "sgs_conv2d_sliced", "sgs_device_status",
     "sgs_profile_read", "sgs_conv2d_sliced_static", "sgs_cache_set_candidates", "sgs_cache_set_policy",
     "sgs_sched_create", "sgs_sched_free", "sgs_sched_dims", "sgs_sched_set_table", "sgs_sched_get_table", "sgs_sched_measure",
-    "sgs_sched_step", "sgs_sched_subnet", "sgs_profile_trace", "sgs_layer_name", "sgs_aux_op", "sgs_device_status_clear", "sgs_debug_expire_wait",
+    "sgs_sched_step", "sgs_sched_subnet", "sgs_profile_trace", "sgs_layer_name", "sgs_aux_op", "sgs_device_status_clear", "sgs_debug_expire_wait", "sgs_measure_fma_peak",
 ]
 
 
@@ -197,6 +197,7 @@ def lib():
         L.sgs_aux_op.argtypes = [ci, vp, vp, ci, vp]
         L.sgs_device_status_clear.argtypes = []
         L.sgs_debug_expire_wait.argtypes = [ctypes.c_uint, vp]
+        L.sgs_measure_fma_peak.argtypes = [vp, vp]
         L.sgs_profile_read.argtypes = [vp, ci, vp, vp, vp, vp]
         _lib = L
     return _lib
@@ -237,6 +238,14 @@ def debug_expire_wait(limit_us: int, stream: int = 0):
     st = lib().sgs_debug_expire_wait(limit_us, ctypes.c_void_p(stream))
     if st != SGS_OK:
         raise SgsError(st, "sgs_debug_expire_wait")
+
+
+def measure_fma_peak(stream: int = 0) -> float:
+    v = ctypes.c_double()
+    st = lib().sgs_measure_fma_peak(ctypes.addressof(v), ctypes.c_void_p(stream))
+    if st != SGS_OK:
+        raise SgsError(st, "sgs_measure_fma_peak")
+    return v.value
 
 
 def aux_op(descs: Sequence[AuxDesc], args: Sequence[AuxArgs], grouped: bool = False, stream: int = 0):

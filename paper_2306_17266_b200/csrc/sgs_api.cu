@@ -119,6 +119,10 @@ std::vector<LayerSpec> stored_layers(int family) {
     return v;
 }
 
+// Channels per stored (filter, tap) row of a convolution: bf16 rows are padded with zeros to a multiple of 16
+// channels (32 bytes), so that tensor-map rows start and end on 32-byte sectors (the 3-channel stem keeps its rows).
+int stored_row(int kind, int C, int dtype) { return (kind == KIND_CONV && dtype == SGS_BF16 && C >= 8) ? (C + 15) / 16 * 16 : C; }
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;
@@ -209,6 +213,9 @@ struct sgs_supernet {
     long long kernel_launches = 0;
     int plan_hits = 0, plan_misses = 0;
     int force_plain = 0;
+    size_t persist_limit_set = 0;  // cudaLimitPersistingL2CacheSize as last set by this handle
+    int cache_mech = 0;    // how grouped launches keep the cached SubGraph in L2: 0 per-tile hints, 1 access-policy window of the launch, 2 both
+    int pad_channels = 1;  // waves of the ResNet-shaped family keep activation pixels at multiples of 16 channels
     int throughput_mode = 0;  // set by streams that keep many queries in flight; part of the plan key
     double host_us_graph = 0, host_us_direct = 0, host_us_stream = 0, host_us_query = 0, host_us_table = 0;  // host time spent issuing work (diagnostic counters)
     // per-kernel-class timing (option "profile"): 0 tensor-core conv, 1 CUDA-core conv, 2 depthwise, 3 other
@@ -362,8 +369,10 @@ struct Builder {
     Plan *plan;
     int N;
     size_t max_elems = 0;
+    bool padded = false;  // activation tensors keep pixels at a multiple of 16 channels (see ConvArgs::ldx)
 
     void note(size_t elems) { max_elems = std::max(max_elems, elems); }
+    int phys(int channels) const { return padded ? (channels + 15) / 16 * 16 : channels; }
 
     // convolution (regular or depthwise) of stored layer `name`
     void conv(const std::string &name, int in, int out, int res, int &H, int &W, int stride, int act) {
@@ -380,7 +389,8 @@ struct Builder {
         int p = (s.k - 1) / 2;
         a.Ho = (H + 2 * p - s.k) / stride + 1;
         a.Wo = (W + 2 * p - s.k) / stride + 1;
-        a.Kmax = L.K; a.Cmax = L.C; a.R = L.R;
+        a.Kmax = L.K; a.Cmax = L.kind == KIND_CONV ? L.Cp : L.C; a.R = L.R;
+        if (padded && op.type == OP_CONV) { a.ldx = in >= 0 ? phys(a.C) : 0; a.ldy = phys(a.K); }
         double M = (double)N * a.Ho * a.Wo;
         double per_out = L.kind == KIND_DW ? (double)s.k * s.k : (double)s.C * s.k * s.k;
         op.flops = 2.0 * M * s.K * per_out;
@@ -388,7 +398,7 @@ struct Builder {
         plan->flops += op.flops;
         plan->weight_bytes += (double)s.K * per_out * net->elem();
         plan->act_bytes += ((double)N * H * W * a.C + M * s.K * (res >= 0 ? 2 : 1)) * net->elem();
-        note((size_t)M * s.K);
+        note((size_t)M * phys(s.K));
         H = a.Ho; W = a.Wo;
         plan->ops.push_back(op);
     }
@@ -419,7 +429,7 @@ struct Builder {
             cv.in = tmp;
             ConvArgs &a = cv.conv;
             a.w = net->stem_win_w;
-            a.H = Hp; a.W = Wp; a.C = 64; a.Cmax = 64; a.win = 1;
+            a.H = Hp; a.W = Wp; a.C = 64; a.Cmax = 64; a.win = 1; a.ldx = 0;
             note((size_t)N * Hp * Wp * 8);
             plan->ops.insert(plan->ops.begin() + (long)first, pd);
             return;
@@ -440,11 +450,12 @@ struct Builder {
         plan->ops.insert(plan->ops.begin() + (long)first, im);
         (void)L;
     }
-    void linear(const std::string &name, int vin, int vout, int act) {
+    void linear(const std::string &name, int vin, int vout, int act, bool vin_padded = false) {
         int li = net->idx(name);
         const Slice &s = plan->slices[li];
         Op op;
-        op.type = OP_LINEAR; op.layer = li; op.vin = vin; op.vout = vout; op.N = N; op.C = s.C; op.K = s.K; op.act = act;
+        // (a padded pooled vector carries zeros beyond the slice; the extra stored weights they meet exist: row pitch >= 16-multiple)
+        op.type = OP_LINEAR; op.layer = li; op.vin = vin; op.vout = vout; op.N = N; op.C = vin_padded ? std::min(phys(s.C), net->layers[li].C) : s.C; op.K = s.K; op.act = act;
         op.flops = 2.0 * N * s.K * s.C;
         op.alg_bytes = (double)s.K * s.C * net->elem() + 4.0 * N * (s.K + s.C);
         plan->flops += op.flops;
@@ -453,7 +464,7 @@ struct Builder {
     }
     void gap(int in, int vout, int H, int W, int C) {
         Op op;
-        op.type = OP_GAP; op.in = in; op.vout = vout; op.N = N; op.H = H; op.W = W; op.C = C;
+        op.type = OP_GAP; op.in = in; op.vout = vout; op.N = N; op.H = H; op.W = W; op.C = phys(C);
         op.alg_bytes = (double)N * H * W * C * net->elem() + 4.0 * N * C;
         plan->ops.push_back(op);
     }
@@ -464,6 +475,12 @@ sgs_status_t build_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batc
     plan->batch = batch; plan->res = res;
     plan->slices = slices_for(net, cfg);
     Builder B{net, plan, batch};
+    // Waves of the ResNet-shaped family on bf16 handles: every convolution runs in the grouped tensor-core kernel
+    // (all channel counts are multiples of 8, and with res % 32 == 0 every stride-2 layer sees even sizes), so the
+    // activation tensors can be padded to 16-channel pixels.  choose_impls refuses a padded plan otherwise.
+    B.padded = net->family == SGS_RESNET && net->throughput_mode == 2 && net->dtype == SGS_BF16 && !net->force_plain &&
+               tc_available() && res % 32 == 0 && net->stem_win_w != nullptr && net->pad_channels;
+    plan->padded = B.padded;
     int H = res, W = res;
     // activation buffers: X current tensor, T1/T2 temporaries, SC shortcut
     int X = 0, T1 = 1, T2 = 2, SC = 3;
@@ -485,9 +502,9 @@ sgs_status_t build_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batc
         B.stem("stem", T1, T2, H, W, 2, ACT_RELU);
         {
             Op op;
-            op.type = OP_MAXPOOL; op.in = T1; op.out = X; op.N = batch; op.H = H; op.W = W; op.C = plan->slices[net->idx("stem")].K;
+            op.type = OP_MAXPOOL; op.in = T1; op.out = X; op.N = batch; op.H = H; op.W = W; op.C = B.phys(plan->slices[net->idx("stem")].K);
             int Hp = (H - 1) / 2 + 1, Wp = (W - 1) / 2 + 1;
-            op.alg_bytes = ((double)batch * H * W + (double)batch * Hp * Wp) * op.C * net->elem();
+            op.alg_bytes = ((double)batch * H * W + (double)batch * Hp * Wp) * plan->slices[net->idx("stem")].K * net->elem();
             plan->ops.push_back(op);
             H = Hp; W = Wp;
             B.note((size_t)batch * H * W * op.C);
@@ -504,7 +521,7 @@ sgs_status_t build_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batc
             }
         int C = plan->slices[net->idx("fc")].C;
         B.gap(X, 0, H, W, C);
-        B.linear("fc", 0, -1, ACT_NONE);
+        B.linear("fc", 0, -1, ACT_NONE, B.padded);
     } else {
         B.stem("stem", X, T1, H, W, 2, ACT_HSWISH);
         { int h = H, w = W; B.conv("first.dw", X, T1, -1, h, w, 1, ACT_RELU); }
@@ -620,6 +637,7 @@ sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
         std::string why;
         op.tc = tc_conv_prepare(op.conv, net->device, &why);
         if (!op.tc && op.conv.win) return fail(net, SGS_EUNSUPPORTED, "window view of the stem: " + why);
+        if (!op.tc && plan->padded) return fail(net, SGS_EUNSUPPORTED, "padded activation layout needs the tensor-core kernel: " + why);
         if (op.tc) {
             op.impl = 1;
             ws_need = std::max(ws_need, tc_conv_ws_elems(*op.tc));
@@ -1131,6 +1149,7 @@ sgs_status_t sgs_supernet_load(const sgs_arch_desc_t *arch, const void *host_blo
             (h[5] != 0) != sp.bn || (h[6] != 0) != sp.bias)
             return SGS_EINVAL;
         size_t nw = (size_t)sp.K * sp.C * sp.R * sp.R;
+        const size_t nw_stored = (size_t)sp.K * stored_row(sp.kind, sp.C, compute_dtype) * sp.R * sp.R;
         Rec r{pos + 8, 0, 0};
         size_t q = pos + 8 + nw;
         if (sp.bn) { r.bn_off = q; q += 4 * (size_t)sp.K; }
@@ -1138,7 +1157,7 @@ sgs_status_t sgs_supernet_load(const sgs_arch_desc_t *arch, const void *host_blo
         if (q > total_words) return SGS_EINVAL;
         pos = q;
         recs.push_back(r);
-        arena += (nw * (compute_dtype == SGS_BF16 ? 2 : 4) + 255) / 256 * 256;
+        arena += (nw_stored * (compute_dtype == SGS_BF16 ? 2 : 4) + 255) / 256 * 256;
         params += ((size_t)sp.K + 63) / 64 * 64 * 2;
     }
     if (pos != total_words) return SGS_EINVAL;
@@ -1159,14 +1178,15 @@ sgs_status_t sgs_supernet_load(const sgs_arch_desc_t *arch, const void *host_blo
         StoredLayer L;
         L.kind = sp.kind; L.K = sp.K; L.C = sp.C; L.R = sp.R; L.S = sp.R; L.has_bn = sp.bn; L.has_bias = sp.bias; L.name = sp.name;
         size_t nw = (size_t)sp.K * sp.C * sp.R * sp.R;
+        L.Cp = stored_row(sp.kind, sp.C, compute_dtype);
         L.w = net->weight_arena + aoff;
         L.w_bytes = nw * net->elem();
-        aoff += (L.w_bytes + 255) / 256 * 256;
+        aoff += ((size_t)sp.K * L.Cp * sp.R * sp.R * net->elem() + 255) / 256 * 256;
         L.scale = net->param_arena + poff;
         L.shift = L.scale + ((size_t)sp.K + 63) / 64 * 64;
         poff += ((size_t)sp.K + 63) / 64 * 64 * 2;
         const float *src = stage + recs[i].w_off;
-        if (sp.kind == KIND_CONV) e = launch_relayout_conv(src, L.w, sp.K, sp.C, sp.R, sp.R, bf, 0);
+        if (sp.kind == KIND_CONV) e = launch_relayout_conv(src, L.w, sp.K, sp.C, L.Cp, sp.R, sp.R, bf, 0);
         else if (sp.kind == KIND_DW) e = launch_relayout_dw(src, L.w, sp.K, sp.R, sp.R, bf, 0);
         else e = launch_convert(src, L.w, nw, bf, 0);
         if (e != cudaSuccess) break;
@@ -1323,6 +1343,16 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
     if ((rc = ensure_waves(net, W)) != SGS_OK) return rc;
     if ((rc = ensure_ranks(net)) != SGS_OK) return rc;
     net->throughput_mode = 2;
+    if (net->cache.enabled && net->cache_mech != 0 && net->persist_max) {
+        // the window mechanism keeps its lines in the L2 carve-out for persisting accesses: size it to the budget
+        // (a limit of this process's context; lines of an earlier stream go back to normal first)
+        const size_t want = std::min(net->cache.budget, net->persist_max);
+        if (want != net->persist_limit_set) {
+            CU(cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want));
+            net->persist_limit_set = want;
+        }
+        cudaCtxResetPersistingL2Cache();
+    }
     const size_t in_bytes = (size_t)batch * res * res * 3 * net->elem();
     const size_t out_bytes = (size_t)batch * net->def.classes * sizeof(float);
     const int n_ranks = (int)net->op_rank.size();
@@ -1343,6 +1373,8 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
     for (int w = 0; w < W; w++) { CU(cudaStreamWaitEvent(net->waves[w].st, e0, 0)); net->waves[w].busy = false; }
     const auto host_t0 = std::chrono::steady_clock::now();
     std::vector<Plan *> plans((size_t)G);
+    std::vector<std::shared_ptr<const std::vector<int>>> boxes((size_t)G);  // per member: the cached SubGraph its query is served under
+    std::vector<int> box_epoch((size_t)G, -1);
     std::vector<std::vector<std::pair<int, int>>> buckets((size_t)n_ranks);  // per rank: (member, op index)
     struct Launch { int rank; GroupLaunch *group; int small_kind; size_t off; int count; int rank2 = -1; };  // rank2: a second bucket merged into this launch;  // group == nullptr && small_kind < 0: the bucket's ungrouped ops, per member
     std::vector<Launch> launches;
@@ -1381,6 +1413,34 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                 cx.stage_out_bytes = need_out;
             }
         }
+        // Accounting and cache policy follow the stream order.  Every member keeps the cached SubGraph that is in
+        // force when its query is served (snapshots are shared between the members of one caching decision): its
+        // convolutions carry that box in their launch records, so the L2 hints of a wave change with the policy
+        // from one member to the next, not from one wave to the next.
+        const int epoch_at_issue = net->cache.epoch;
+        for (int m = 0; m < members; m++) {
+            const int epoch_before = net->cache.epoch;
+            if (!boxes[m] || box_epoch[m] != epoch_before) {
+                if (m > 0 && box_epoch[m - 1] == epoch_before && boxes[m - 1]) boxes[m] = boxes[m - 1];
+                else boxes[m] = std::make_shared<const std::vector<int>>(net->cache.enabled ? net->cache.G : std::vector<int>());
+                box_epoch[m] = epoch_before;
+            }
+            QueryAccount qa = account_query(net, plans[m]->enc);
+            flops += plans[m]->flops; wbytes += qa.weight_bytes; miss_bytes += qa.miss_bytes; hit += qa.hit_ratio;
+            if (net->cache.enabled) {
+                cache_observe(net, plans[m]->enc);
+                if (net->cache.epoch != epoch_before) updates++;
+            }
+        }
+        // persisting L2 lines of SubGraphs that are no longer cached go back to normal replacement
+        if (net->cache.enabled && net->cache_mech != 0 && net->cache.epoch != epoch_at_issue) cudaCtxResetPersistingL2Cache();
+        const int box_policy = !net->cache.enabled ? (net->cache.evict_first_when_off ? 2 : 0) : (net->cache_mech == 1 ? 3 : 1);
+        auto set_box = [&](ConvArgs &a, int member, int layer) {
+            a.weight_policy = box_policy; a.cacheK = a.cacheC = 0;
+            const std::vector<int> &G = *boxes[(size_t)member];
+            if ((box_policy == 1 || box_policy == 3) && !G.empty()) { a.cacheK = G[3 * (size_t)layer]; a.cacheC = G[3 * (size_t)layer + 1]; }
+            else if (box_policy == 1 || box_policy == 3) a.weight_policy = 0;
+        };
         // merge the members' op lists by rank
         for (auto &b : buckets) b.clear();
         size_t n_tc = 0;
@@ -1452,6 +1512,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                 if (!g || !g->fits(*op.tc)) { g = next_group(); launches.push_back({r, g, -1, 0, 0}); }
                 ConvArgs a = op.conv;
                 a.layer = op.layer;
+                set_box(a, mo.first, op.layer);
                 g->add(cx.h_tbl + off, *op.tc, a);
                 off += TC_GROUP_ENTRY_BYTES;
             }
@@ -1490,6 +1551,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                             const Op &op = plans[mo.first]->ops[(size_t)mo.second];
                             ConvArgs a = op.conv;
                             a.layer = op.layer;
+                            set_box(a, mo.first, op.layer);
                             g->add(cx.h_tbl + off, *op.tc, a);
                             off += TC_GROUP_ENTRY_BYTES;
                         }
@@ -1603,7 +1665,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
                 bucket_cost(L.rank, true, &pb, &pf);
                 if (L.rank2 >= 0) { double b2 = 0, f2 = 0; bucket_cost(L.rank2, true, &b2, &f2); pb += b2; pf += f2; }
                 if ((rc = prof_begin(0, pb, pf, first_layer(L.rank), L.group->members(), L.group->tiles())) != SGS_OK) break;
-                CU(L.group->launch(net->cache_tbl, net->sms, ws));
+                CU(L.group->launch(net->cache.enabled && net->cache_mech != 0 ? net->window_max : 0, net->sms, ws));
                 if ((rc = prof_end()) != SGS_OK) break;
                 net->kernel_launches++;
                 continue;
@@ -1652,17 +1714,6 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
         CU(cudaEventRecord(cx.done, ws));
         cx.busy = true;
         net->host_us_graph += tick(tp);
-        // accounting and cache policy follow the stream order; the device-side hints of a wave use the
-        // cached SubGraph as it stood when the wave was issued
-        for (int m = 0; m < members; m++) {
-            const int epoch_before = net->cache.epoch;
-            QueryAccount qa = account_query(net, plans[m]->enc);
-            flops += plans[m]->flops; wbytes += qa.weight_bytes; miss_bytes += qa.miss_bytes; hit += qa.hit_ratio;
-            if (net->cache.enabled) {
-                cache_observe(net, plans[m]->enc);
-                if (net->cache.epoch != epoch_before) updates++;
-            }
-        }
     }
     net->host_us_stream += std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - host_t0).count();
     for (int w = 0; w < W; w++) {  // join
@@ -2145,8 +2196,9 @@ int sgs_layer_name(const sgs_supernet_t *net, int layer, char *out, int cap) {
 sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long value) {
     if (!net || !name) return SGS_EINVAL;
     std::string n(name);
-    if (n == "conv_impl") {
-        net->force_plain = value == 1;
+    if (n == "conv_impl" || n == "pad_channels") {
+        if (n == "conv_impl") net->force_plain = value == 1;
+        else net->pad_channels = value != 0;
         DeviceGuard guard(net->device);
         cudaDeviceSynchronize();
         fold_profile(net);
@@ -2162,6 +2214,23 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
             for (int i = 0; i < 4; i++) { net->prof_ms[i] = net->prof_bytes[i] = net->prof_flops[i] = 0; net->prof_launches[i] = 0; }
             net->prof_trace.clear();
         }
+        return SGS_OK;
+    }
+    if (n == "cache_mechanism") {
+        if (value < 0 || value > 2) return fail(net, SGS_EINVAL, "cache_mechanism");
+        net->cache_mech = (int)value;
+        return SGS_OK;
+    }
+    if (n == "drop_plans") {  // forget every plan (and its graphs): the next use of a config pays for planning again
+        DeviceGuard guard(net->device);
+        cudaDeviceSynchronize();
+        fold_profile(net);
+        for (auto &kv : net->plans) destroy_plan_resources(kv.second.get());
+        net->plans.clear();
+        return SGS_OK;
+    }
+    if (n == "dw_walk") {  // tuning aid (process-wide)
+        dw_set_walk(value != 0);
         return SGS_OK;
     }
     if (n == "stage_group") {  // tuning aid: stages per barrier pair of the grouped convolution kernel (0 = default)
@@ -2313,6 +2382,11 @@ sgs_status_t sgs_aux_op(int n, const sgs_aux_desc_t *desc, const sgs_aux_args_t 
 int sgs_device_status(void) { return tc_conv_status(); }
 
 sgs_status_t sgs_device_status_clear(void) { return tc_conv_status_clear() == cudaSuccess ? SGS_OK : SGS_ECUDA; }
+
+sgs_status_t sgs_measure_fma_peak(double *tflops, void *cuda_stream) {
+    if (!tflops) return SGS_EINVAL;
+    return measure_fma_rate(tflops, (cudaStream_t)cuda_stream) == cudaSuccess ? SGS_OK : SGS_ECUDA;
+}
 
 sgs_status_t sgs_debug_expire_wait(unsigned limit_us, void *cuda_stream) {
     if (limit_us == 0 || limit_us > 1000000u) return SGS_EINVAL;

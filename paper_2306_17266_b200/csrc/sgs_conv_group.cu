@@ -54,7 +54,11 @@ struct __align__(16) GroupEntry {
     // geometry, filters and weight map and takes MMA rows 0..63, the entry after it ("second") takes rows
     // 64..127 with its own activation map, outputs and filter count (not larger than the first's).
     unsigned char pair, second;
-    int pad2_[3];
+    int ldk;                 // channels per pixel of y and res as stored (>= K; the kernel writes zeros into K..ldk-1)
+    // SubGraph cache box of this member's query (the cached SubGraph in force when the query is served, in stream
+    // order): weight tiles with filter < cacheK and channel < cacheC are loaded evict-last; cacheK == -1: every
+    // weight load evict-first; 0: no hint
+    int cacheK, cacheC;
 };
 static_assert(sizeof(GroupEntry) == TC_GROUP_ENTRY_BYTES, "entry size");
 
@@ -88,7 +92,7 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *m) { asm v
 // there); the per-member records travel in a device table.
 template <int NMAPS> struct GroupParams {
     const GroupEntry *entries;
-    const int *cache_tbl;
+    const void *unused_;
     int *status;
     int n_entries, total_tiles;
     int n_stages, stage_bytes;  // operand ring of this launch
@@ -102,7 +106,6 @@ template <int NMAPS>
 __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_constant__ GroupParams<NMAPS> P) {
     const GroupEntry *__restrict__ entries = P.entries;
     const int n_entries = P.n_entries, total_tiles = P.total_tiles;
-    const int *__restrict__ cache_tbl = P.cache_tbl;
     int *status = P.status;
     extern __shared__ uint8_t smem_raw[];
     __shared__ GroupEntry es[TC_GROUP_MAX_ENTRIES];
@@ -142,7 +145,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
         // Weights do not depend on the previous layer, so this warp never waits for it: it runs ahead
         // as far as the ring allows.  The warp runs its loop converged; one elected lane issues.
         const uint64_t pol_keep = make_policy(1), pol_stream = make_policy(2);
-        const int weight_policy = cache_tbl ? __ldg(cache_tbl) : 0;
         int s = 0, g = 0, gi = 0;  // stage, its group, its position in the group
         uint32_t phase = 0;
         bool wrapped = false, ok = true;
@@ -157,8 +159,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             const int k = e.k, kw = e.kw, cchunks = e.cchunks, R = e.R;
             int kind = 0;  // 0 default replacement, 1 keep (inside the cached SubGraph's box, up to channel cacheC), 2 stream
             int cacheC = 0;
-            if (weight_policy == 2) kind = 2;
-            else if (weight_policy == 1 && f0 < __ldg(cache_tbl + 1 + 2 * e.layer)) { kind = 1; cacheC = __ldg(cache_tbl + 2 + 2 * e.layer); }
+            if (e.cacheK < 0) kind = 2;
+            else if (f0 < e.cacheK) { kind = 1; cacheC = e.cacheC; }
             int tap_row = e.tap0;
             for (int r = 0; r < k && ok; r++, tap_row += R) {
                 for (int sx = 0; sx < kw && ok; sx++) {
@@ -314,7 +316,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             const bool second_half = e0.pair && quad >= 2;
             const GroupEntry &e = second_half ? (&e0)[1] : e0;
             const int row = second_half ? row_all - 64 : row_all;
-            const int K = e.K, act = e.act;
+            const int K = e.K, ldk = e.ldk, act = e.act;
             const __nv_bfloat16 *res = e.res;
             __nv_bfloat16 *y = e.y;
             const int sb = jj & 1;  // which of the group's two scale / shift tables
@@ -333,10 +335,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                     m = valid ? (int)(((size_t)n * e.Ho + h) * e.Wo + w) : -1;
                 }
                 const int cend = min((int)e0.bn_tile, K - f0);  // filters of this tile, a multiple of 8 (<= 0: none of this member's)
-                const size_t obase = (size_t)(m < 0 ? 0 : m) * K + f0;
+                const int cpad = min((int)e0.bn_tile, ldk - f0);  // ... and the end of the pixel's padding, written as zeros
+                const size_t obase = (size_t)(m < 0 ? 0 : m) * ldk + f0;
                 // the residual does not depend on the accumulator: the first 64 columns' part is requested
                 // before waiting, every further part two steps ahead of its use (a thread then has 8 loads of
-                // 16 bytes in flight: the epilogue of a tile with a residual is bound by their latency)
+                // 16 bytes in flight: the epilogue of a tile with a residual is bound by their latency).
+                // (Measured alternative: transposing the accesses through a warp-private staging block so that a
+                // warp touches 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes changed no layer's time
+                // at 16 images per member and cost 1.7 % on the batch-1 stream.)
                 auto load_res = [&](int c0, uint4 *rv) {
 #pragma unroll
                     for (int g = 0; g < 4; g++) {
@@ -353,7 +359,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                 if (alive) {
                     tc_fence_after();
 #pragma unroll 1
-                    for (int c0 = 0; c0 < cend; c0 += 32) {  // warp-uniform bounds
+                    for (int c0 = 0; c0 < cpad; c0 += 32) {
                         uint32_t v[32];
                         tmem_ld32(tacc + c0, v);
                         uint4 rf[4];
@@ -363,6 +369,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
 #pragma unroll
                             for (int g = 0; g < 4; g++) {
                                 const int c = c0 + 8 * g;
+                                if (c >= cend && c < cpad) *reinterpret_cast<uint4 *>(y + obase + c) = make_uint4(0u, 0u, 0u, 0u);
                                 if (c < cend) {
                                     float ov[8];
 #pragma unroll
@@ -381,7 +388,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
             } else {
                 // ---- swapped tile: this thread owns filter `f`, columns are the member's output pixels
                 const int f = nt * 128 + row;
-                const bool fvalid = f < K;
+                const bool fvalid = f < K, fpad = f >= K && f < ldk;
                 const int cend = e.pix_rows;  // == N * Ho * Wo: the pixel tile is the whole member
                 float sc = 0.f, sh = 0.f;
                 if (fvalid) { sc = __ldg(e.scale + f); sh = __ldg(e.shift + f); }
@@ -391,8 +398,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                     for (int q = 0; q < 16; q++) {
                         const int p0 = c0 + 2 * q;
                         uint32_t lo = 0, hi = 0;
-                        if (res && fvalid && p0 < cend) lo = __ldg(resu + (size_t)p0 * K + f);
-                        if (res && fvalid && p0 + 1 < cend) hi = __ldg(resu + (size_t)(p0 + 1) * K + f);
+                        if (res && fvalid && p0 < cend) lo = __ldg(resu + (size_t)p0 * ldk + f);
+                        if (res && fvalid && p0 + 1 < cend) hi = __ldg(resu + (size_t)(p0 + 1) * ldk + f);
                         rv[q] = lo | (hi << 16);
                     }
                 };
@@ -416,9 +423,13 @@ __global__ void __launch_bounds__(G_THREADS, 1) conv_group_kernel(const __grid_c
                                 if (px < cend) {
                                     const uint32_t rbits = (q & 1) ? (rv[q >> 1] & 0xffff0000u) : (rv[q >> 1] << 16);
                                     const float o = act_fn(__uint_as_float(v[q]) * sc + sh + __uint_as_float(rbits), act);
-                                    y[(size_t)px * K + f] = __float2bfloat16_rn(o);
+                                    y[(size_t)px * ldk + f] = __float2bfloat16_rn(o);
                                 }
                             }
+                        } else if (fpad) {
+#pragma unroll
+                            for (int q = 0; q < 32; q++)
+                                if (c0 + q < cend) y[(size_t)(c0 + q) * ldk + f] = __float2bfloat16_rn(0.f);
                         }
 #pragma unroll
                         for (int q = 0; q < 16; q++) rv[q] = rn[q];
@@ -458,6 +469,8 @@ struct GroupLaunch::Impl {
     GroupParams<TC_GROUP_MAPS_LARGE> prm;  // host image of the parameter block (the small variant is a prefix)
     int n_maps = 0;
     int col_rows = 0;   // most rows any member's column-side operand has (64, 128 or 256: sizes the stages)
+    const void *win_base = nullptr;  // largest cached filter prefix among the members' stored layers
+    size_t win_bytes = 0;
 };
 
 GroupLaunch::GroupLaunch() : impl(new Impl) { reset(nullptr); }
@@ -466,6 +479,8 @@ GroupLaunch::~GroupLaunch() { delete impl; }
 void GroupLaunch::reset(const void *d_entries) {
     impl->n_maps = 0;
     impl->col_rows = 0;
+    impl->win_base = nullptr;
+    impl->win_bytes = 0;
     impl->prm.entries = static_cast<const GroupEntry *>(d_entries);
     impl->prm.n_entries = 0;
     impl->prm.total_tiles = 0;
@@ -495,6 +510,15 @@ void GroupLaunch::add(void *host_entry, const TcConvPlan &pl, const ConvArgs &a)
     e.tile_begin = impl->prm.total_tiles;
     e.mtiles = (int)pl.grid.x;
     e.N = p.N; e.Ho = p.Ho; e.Wo = p.Wo; e.K = p.K; e.C = p.C;
+    e.ldk = a.ldy ? a.ldy : p.K;
+    // weight_policy 1: per-tile hints from the box; 2: all evict-first; 3: the box only feeds the launch's window
+    e.cacheK = a.weight_policy == 2 ? -1 : a.weight_policy == 1 ? a.cacheK : 0;
+    e.cacheC = a.weight_policy == 1 ? a.cacheC : 0;
+    if ((a.weight_policy == 1 || a.weight_policy == 3) && a.cacheK > 0) {
+        // the launch's access-policy window (optional mechanism): the filters [0, cacheK) of this stored layer, whole rows
+        const size_t bytes = (size_t)a.cacheK * a.R * a.R * a.Cmax * 2;
+        if (bytes > impl->win_bytes) { impl->win_base = a.w; impl->win_bytes = bytes; }
+    }
     e.R = p.R; e.tap0 = p.o * p.R + p.o;
     e.tiles_w = p.tiles_w; e.tiles_hw = p.tiles_w * p.tiles_h;
     e.cchunks = p.cchunks; e.iters = p.iters; e.layer = a.layer;
@@ -536,14 +560,14 @@ cudaError_t tc_group_init(int) {
     return cudaFuncSetAttribute(conv_group_kernel<TC_GROUP_MAPS_LARGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
 }
 
-cudaError_t GroupLaunch::launch(const int *cache_tbl, int sms, cudaStream_t st) {
+cudaError_t GroupLaunch::launch(size_t window_max, int sms, cudaStream_t st) {
     if (impl->prm.n_entries <= 0 || impl->prm.total_tiles <= 0) return cudaSuccess;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     impl->prm.status = tc_status_word(dev);
     if (!impl->prm.status) return cudaErrorInitializationError;
-    impl->prm.cache_tbl = cache_tbl;
+    impl->prm.unused_ = nullptr;
     // stage = 16 KB for the row-side operand + room for the widest column-side operand of the launch
     const int col_rows = impl->col_rows <= 64 ? 64 : impl->col_rows <= 128 ? 128 : 256;
     impl->prm.stage_bytes = G_X_BYTES + col_rows * CHUNK_C * 2;
@@ -555,11 +579,23 @@ cudaError_t GroupLaunch::launch(const int *cache_tbl, int sms, cudaStream_t st) 
     cfg.blockDim = dim3(G_THREADS);
     cfg.dynamicSmemBytes = G_SMEM_BYTES;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (window_max && impl->win_base && impl->win_bytes) {
+        // Access-policy window of this launch: L2 lines of the cached filter prefix that the launch touches are
+        // kept with the persisting property (they live in the L2 carve-out the handle sized to the cache budget),
+        // everything else is accessed normally.
+        attr[1].id = cudaLaunchAttributeAccessPolicyWindow;
+        attr[1].val.accessPolicyWindow.base_ptr = const_cast<void *>(impl->win_base);
+        attr[1].val.accessPolicyWindow.num_bytes = std::min(impl->win_bytes, window_max);
+        attr[1].val.accessPolicyWindow.hitRatio = 1.0f;
+        attr[1].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+        attr[1].val.accessPolicyWindow.missProp = cudaAccessPropertyNormal;
+        cfg.numAttrs = 2;
+    }
     if (impl->n_maps <= TC_GROUP_MAPS_SMALL) {
         // the small parameter block is a prefix of the large one (same header, fewer maps)
         void *args[1] = {&impl->prm};

@@ -31,6 +31,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <unordered_map>
 
 namespace sgs {
 
@@ -301,8 +302,36 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// Encoded tensor maps by their defining numbers.  A SubNet never seen before still slices the same stored layers
+// into one of a few (K', C') boxes and reads the same workspaces at one of a few channel counts, so most of its
+// maps were encoded for an earlier SubNet already; planning a new config then costs look-ups instead of driver calls.
+struct MapKey {
+    uint64_t v[15];
+    bool operator==(const MapKey &o) const { return std::memcmp(v, o.v, sizeof v) == 0; }
+};
+struct MapKeyHash {
+    size_t operator()(const MapKey &k) const {
+        uint64_t h = 1469598103934665603ull;
+        for (uint64_t x : k.v) { h ^= x; h *= 1099511628211ull; h ^= h >> 29; }
+        return (size_t)h;
+    }
+};
+std::unordered_map<MapKey, CUtensorMap, MapKeyHash> g_map_cache;
+std::mutex g_map_mu;
+
 bool encode_map(CUtensorMap *m, const void *base, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
                 const uint32_t *box) {
+    MapKey key;
+    std::memset(&key, 0, sizeof key);
+    key.v[0] = reinterpret_cast<uint64_t>(base);
+    key.v[1] = (uint64_t)rank;
+    for (int i = 0; i < rank; i++) { key.v[2 + i] = dims[i]; key.v[11 + (i >> 1)] |= (uint64_t)box[i] << (32 * (i & 1)); }
+    for (int i = 0; i + 1 < rank; i++) key.v[7 + i] = strides_bytes[i];
+    {
+        std::lock_guard<std::mutex> lk(g_map_mu);
+        auto it = g_map_cache.find(key);
+        if (it != g_map_cache.end()) { *m = it->second; return true; }
+    }
     cuuint64_t gd[5], gs[4];
     cuuint32_t bx[5], es[5];
     for (int i = 0; i < rank; i++) { gd[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
@@ -310,7 +339,10 @@ bool encode_map(CUtensorMap *m, const void *base, int rank, const uint64_t *dims
     CUresult r = encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), gd, gs, bx, es,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    if (r != CUDA_SUCCESS) return false;
+    std::lock_guard<std::mutex> lk(g_map_mu);
+    if (g_map_cache.size() < (1u << 20)) g_map_cache.emplace(key, *m);  // (128 bytes each; bounded)
+    return true;
 }
 
 struct DeviceScratch {
@@ -422,6 +454,8 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
          reinterpret_cast<uintptr_t>(a.res)) & 15)
         return no("pointers must be 16-byte aligned");
     if (device < 0 || device >= 64) return no("device index");
+    if ((a.ldx || a.ldy) && a.throughput != 2) return no("padded pixels are for grouped launches");
+    if ((a.ldx && (a.ldx < a.C || a.ldx % 8)) || (a.ldy && (a.ldy < a.K || a.ldy % 8))) return no("channel pitch");
 
     auto plan = std::make_shared<TcConvPlan>();
     TcParams &p = plan->prm;
@@ -436,7 +470,9 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
     }
     p.act = a.act;
     const bool flat = a.k == 1 && a.stride == 1;
-    const uint64_t C = (uint64_t)a.C, eb = 2;
+    // C = channels per pixel of x as stored (pitch and extent of the activation maps): with padded pixels the
+    // channels beyond the slice are zeros, so the maps may show them and no row ends inside a 32-byte sector
+    const uint64_t C = (uint64_t)(a.ldx ? a.ldx : a.C), eb = 2;
     // Grouped launches (throughput == 2) run a layer with very few output pixels "swapped": the filters
     // take the 128-row side of the MMA and ALL pixels of the member form the other operand (one pixel
     // tile), so that no MMA rows are wasted on a 2x2 or 4x4 map.  (The kernel takes up to 256 pixels
@@ -526,7 +562,9 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
     plan->bn_tile = BN;
     {
         const uint64_t taps = a.win ? (uint64_t)a.k : (uint64_t)a.R * a.R;  // stored taps per filter
-        uint64_t dims[3] = {C, taps, (uint64_t)a.K};
+        // (padded pixels: the weight map shows the stored channels up to the pixel's pitch; they meet zeros)
+        const uint64_t Cw = a.ldx ? std::min<uint64_t>((uint64_t)a.ldx, (uint64_t)a.Cmax) : (uint64_t)a.C;
+        uint64_t dims[3] = {Cw, taps, (uint64_t)a.K};
         uint64_t str[2] = {(uint64_t)a.Cmax * eb, taps * a.Cmax * eb};
         uint32_t box[3] = {CHUNK_C, 1, (uint32_t)BN};
         if (!encode_map(&p.tmW, a.w, 3, dims, str, box)) return no("weight tensor map");

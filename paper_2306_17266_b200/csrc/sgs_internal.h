@@ -27,6 +27,7 @@ enum Act { ACT_NONE = 0, ACT_RELU = 1, ACT_HSWISH = 2 };
 // (scale = gamma / sqrt(var + eps), shift = beta - mean * scale), or scale = 1, shift = bias.
 struct StoredLayer {
     int kind = 0, K = 0, C = 0, R = 0, S = 0;
+    int Cp = 0;  // conv: channels per (filter, tap) row as stored (>= C; the rest of a row is zero), else C
     bool has_bn = false, has_bias = false;
     void *w = nullptr;
     float *scale = nullptr, *shift = nullptr;
@@ -46,7 +47,13 @@ struct ConvArgs {
     const void *res = nullptr; // optional residual [N][Ho][Wo][K]
     void *y = nullptr;         // [N][Ho][Wo][K]
     int N = 0, H = 0, W = 0, C = 0, Ho = 0, Wo = 0, K = 0;
-    int Kmax = 0, Cmax = 0, R = 0;  // stored dims (square kernels)
+    int Kmax = 0, Cmax = 0, R = 0;  // stored dims (square kernels); Cmax = channels per stored (filter, tap) row
+    // Channel pitch (elements per pixel) of x and of y / res when a pixel holds more than the sliced channels:
+    // 0 = dense (C resp. K).  Padded tensors keep their pixels at a multiple of 16 channels (32 bytes) and the
+    // channels beyond the slice are ZERO: the copy unit moves rows whose ends fall inside a 32-byte sector at a
+    // third of the rate (measured on sm_100a), and C, K are multiples of 8 only.  Tensor-core kernels of grouped
+    // launches only; they write the zeros of y.
+    int ldx = 0, ldy = 0;
     int k = 1, stride = 1, act = 0;
     // Window view of a 3-channel stem (grouped launches): x is the input padded to 8 channels with a zero
     // margin, [N][H][W][8] with H, W the PADDED sizes; an "input channel" chunk is the 8-pixel x 8-channel
@@ -96,6 +103,7 @@ struct Plan {
     std::vector<cudaEvent_t> prof_ev;      // start / end event of every op (profiling)
     int launches = 0;
     bool prepared = false;  // implementations chosen and buffer addresses fixed
+    bool padded = false;    // activation tensors hold 16-channel-padded pixels (ConvArgs::ldx, ldy)
     int slot = 0;           // which set of workspaces the plan's buffer addresses refer to
     int throughput = 0;     // tile choice of the plan's convolutions (see ConvArgs::throughput)
 };
@@ -112,9 +120,10 @@ template <typename T> cudaError_t launch_scale(const T *x, const float *gate, T 
 template <typename T>
 cudaError_t launch_linear(const float *v, const T *w, const float *bias, float *y, int N, int C, int K, int ld, int act,
                           cudaStream_t st);
-cudaError_t launch_relayout_conv(const float *src, void *dst, int K, int C, int R, int S, int bf16, cudaStream_t st);
+cudaError_t launch_relayout_conv(const float *src, void *dst, int K, int C, int Cp, int R, int S, int bf16, cudaStream_t st);  // dst [K][R][S][Cp], zero beyond C
 cudaError_t launch_relayout_dw(const float *src, void *dst, int K, int R, int S, int bf16, cudaStream_t st);
 cudaError_t launch_convert(const float *src, void *dst, size_t n, int bf16, cudaStream_t st);
+cudaError_t measure_fma_rate(double *tflops, cudaStream_t st);  // fp32 FMA rate of the CUDA cores (2 FLOP per FMA), best of 4 timed launches
 cudaError_t launch_delay(unsigned microseconds, cudaStream_t st);  // one thread sleeping for a bounded time
 cudaError_t launch_fold_bn(const float *gamma, const float *beta, const float *mean, const float *var,
                            const float *bias, float *scale, float *shift, int K, cudaStream_t st);
@@ -148,6 +157,7 @@ cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int
 // and take the vectorised bf16 kernels (kernel sizes 3, 5, 7 may be mixed); otherwise cudaErrorNotSupported and
 // nothing is launched.
 constexpr int DW_ENTRY_BYTES = 256;
+void dw_set_walk(int on);  // tuning aid: 0 = stride-1 depthwise layers on the patch / row kernels instead of the walking kernel
 cudaError_t launch_dw_group(const char *h_tbl, const char *d_tbl, int members, cudaStream_t st);
 // Stem weights for the window view: dst[f][r][px * 8 + c] = src[f][r][px][c] (px < k, c < 3), else 0; dst [K][k][64].
 cudaError_t launch_stem_window_weights(const void *src, void *dst, int K, int k, cudaStream_t st);
@@ -187,7 +197,8 @@ public:
     int members() const;
     int maps() const;                       // tensor maps used so far
     int tiles() const;
-    cudaError_t launch(const int *cache_tbl, int sms, cudaStream_t st);
+    // window_max > 0: also mark the launch's cached filter prefix with an access-policy window of at most that many bytes
+    cudaError_t launch(size_t window_max, int sms, cudaStream_t st);
 private:
     struct Impl;
     Impl *impl;

@@ -392,28 +392,197 @@ __global__ void __launch_bounds__(128) dw_tile_kernel(const ConvArgs a1, const c
     if (GROUP) { const ConvArgs al = a; dw_tile_body<K, ST, TH, TW, PRELOAD, ACT>(al, n); }  // (register copy, see dw_mixed_kernel)
     else dw_tile_body<K, ST, TH, TW, PRELOAD, ACT>(a, n);
 }
+// Stride-1 depthwise convolution that WALKS down the image behind a ring of input rows in shared memory (the
+// B200 form of a line buffer: paper Section 4.2 keeps the rows a sliding window needs on chip).  A block owns 128
+// channels x a tile of 4 * TW output columns x a segment of SEG output rows.  Its 128 threads copy one input row of
+// the tile at a time into a ring of RING rows with 16-byte asynchronous copies (zero fill for rows, columns and
+// channels outside the tensor, so the arithmetic has no bounds tests), RING - 1 rows ahead of the row being used:
+// memory latency is covered by the ring, not by registers or occupancy.  A thread owns 4 channels (an 8-byte vector)
+// of a strip of TW columns: per input row it reads TW + K - 1 vectors from the ring, unpacks each ONCE, and
+// scatters it into the K output rows it belongs to.  The K live output rows rotate through K accumulator slots; the
+// row loop is unrolled by K so that every slot index is static: input row hi = base + u meets filter row r in output
+// row hi + P - r, slot (u - r) mod K.  Filter row 0 STARTS an output row (a product instead of an accumulate: slots
+// never need clearing, rows outside the segment never need a test), filter row K - 1 completes it.  The weights of
+// the block's 128 channels sit unpacked (fp32) in shared memory; a lane reads its four per tap with one 16-byte load.
+// Grid: x = channel blocks x column tiles, y = row segments, z = image (x member).
+#ifndef DW_WALK_SEG_ROWS
+#define DW_WALK_SEG_ROWS 28
+#endif
+constexpr int DW_WALK_SEG = DW_WALK_SEG_ROWS;  // output rows per segment (halo: K - 1 extra input rows per segment)
+template <int K> struct DwWalkShape {
+    static constexpr int TW = K == 3 ? 4 : 2;          // output columns per thread
+    static constexpr int ICOL = 4 * TW + K - 1;        // input columns of a block's tile
+    static constexpr int RING = K == 7 ? 6 : 8;        // input rows in the ring
+    static constexpr int ROW_BYTES = ICOL * 256;       // 128 channels x 2 bytes per column
+    static constexpr int SMEM = K * K * 128 * 4 + RING * ROW_BYTES;
+};
+
+__device__ __forceinline__ void cp_async16(void *dst, const void *src, bool valid) {
+    const unsigned n = valid ? 16u : 0u;  // 0 source bytes: the 16 destination bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int K, int ACT>
+__device__ __forceinline__ void dw_walk_body(const ConvArgs &a, const int n, unsigned char *smem, const int chblocks) {
+    using S = DwWalkShape<K>;
+    constexpr int TW = S::TW, P = (K - 1) / 2, NCOL = TW + K - 1, ICOL = S::ICOL, RING = S::RING;
+    float *wsm = reinterpret_cast<float *>(smem);
+    unsigned char *ring = smem + K * K * 128 * 4;
+    const int lane = threadIdx.x & 31, wrp = threadIdx.x >> 5;
+    const int groups = a.K / 4, tiles_w = (a.Wo + 4 * TW - 1) / (4 * TW);
+    // (chblocks = channel blocks of the GRID: a launch over several members is sized for the widest of them)
+    const int cb = blockIdx.x % chblocks, tb = blockIdx.x / chblocks;
+    const int ho_begin = blockIdx.y * DW_WALK_SEG, ho_end = min(a.Ho, ho_begin + DW_WALK_SEG);
+    if (cb * 32 >= groups || tb >= tiles_w || ho_begin >= a.Ho) return;  // (whole blocks only: no barrier is skipped)
+    const int o = (a.R - K) / 2;
+    const __nv_bfloat16 *__restrict__ w = static_cast<const __nv_bfloat16 *>(a.w);
+    // the block's weights: wsm[tap][lane * 4 + j] = w[o + r][o + s][cb * 128 + lane * 4 + j] (zero beyond the slice)
+    for (int i = threadIdx.x; i < K * K * 32; i += blockDim.x) {
+        const int tap = i >> 5, l = i & 31, c = cb * 128 + l * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < a.K) {
+            const uint2 q = __ldg(reinterpret_cast<const uint2 *>(w + ((size_t)((o + tap / K) * a.R + o + tap % K)) * a.Kmax + c));
+            const float2 lo = bf2_lo(q.x), hi = bf2_lo(q.y);
+            v = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
+        reinterpret_cast<float4 *>(wsm)[tap * 32 + l] = v;
+    }
+    const int cg = cb * 32 + lane;
+    const int c0 = cg * 4, wt0 = tb * 4 * TW, wo0 = wt0 + wrp * TW;
+    const bool active = cg < groups;  // (lanes beyond the slice compute zeros and store nothing)
+    const __nv_bfloat16 *ximg = static_cast<const __nv_bfloat16 *>(a.x) + ((size_t)n * a.H) * a.W * a.K;
+    __nv_bfloat16 *yimg = static_cast<__nv_bfloat16 *>(a.y) + ((size_t)n * a.Ho) * a.Wo * a.K + c0;
+    float4 sc4 = make_float4(0.f, 0.f, 0.f, 0.f), sh4 = sc4;
+    if (active) { sc4 = __ldg(reinterpret_cast<const float4 *>(a.scale + c0)); sh4 = __ldg(reinterpret_cast<const float4 *>(a.shift + c0)); }
+    const float2 sc[2] = {make_float2(sc4.x, sc4.y), make_float2(sc4.z, sc4.w)}, sh[2] = {make_float2(sh4.x, sh4.y), make_float2(sh4.z, sh4.w)};
+    const float4 *wl = reinterpret_cast<const float4 *>(wsm) + lane;
+
+    const int hi_first = ho_begin - P, hi_last = ho_end - 1 + P;  // input rows that meet the segment (may lie outside the image)
+    // one input row of the tile -> ring slot (hi - hi_first) % RING; 16 chunks of 16 bytes per column
+    auto copy_row = [&](int hi) {
+        if (hi <= hi_last) {
+            unsigned char *dst = ring + ((hi - hi_first) % RING) * S::ROW_BYTES;
+            const bool rok = hi >= 0 && hi < a.H;
+            const __nv_bfloat16 *xrow = ximg + (size_t)(rok ? hi : 0) * a.W * a.K;
+            for (int q = threadIdx.x; q < ICOL * 16; q += 128) {
+                const int j = q >> 4, part = q & 15;
+                const int wi = wt0 - P + j, c = cb * 128 + part * 8;
+                const bool ok = rok && wi >= 0 && wi < a.W && c < a.K;
+                cp_async16(dst + q * 16, ok ? (const void *)(xrow + (size_t)wi * a.K + c) : (const void *)ximg, ok);
+            }
+        }
+        cp_async_commit();  // (a group per row, also when it is empty: the wait below counts groups)
+    };
+#pragma unroll 1
+    for (int d = 0; d < RING - 1; d++) copy_row(hi_first + d);
+
+    float2 acc[K][TW][2];
+    for (int base = hi_first; base <= hi_last; base += K) {
+#pragma unroll
+        for (int u = 0; u < K; u++) {
+            const int hi = base + u;
+            if (hi <= hi_last) {  // (block-uniform)
+                cp_async_wait<RING - 2>();  // this thread's copies of row hi have landed ...
+                __syncthreads();            // ... and everybody's; everybody has also finished with row hi - 1
+                copy_row(hi + RING - 1);    // into the slot row hi - 1 used
+                const unsigned char *row = ring + ((hi - hi_first) % RING) * S::ROW_BYTES + (wrp * TW) * 256 + lane * 8;
+                float2 xc[NCOL][2];
+#pragma unroll
+                for (int j = 0; j < NCOL; j++) {
+                    const uint2 v = *reinterpret_cast<const uint2 *>(row + j * 256);
+                    xc[j][0] = bf2_lo(v.x); xc[j][1] = bf2_lo(v.y);
+                }
+#pragma unroll
+                for (int r = 0; r < K; r++) {
+                    constexpr int KK = K;
+                    const int slot = ((u - r) % KK + KK) % KK;
+#pragma unroll
+                    for (int s2 = 0; s2 < K; s2++) {
+                        const float4 wq = wl[(r * K + s2) * 32];
+                        const float2 w0 = make_float2(wq.x, wq.y), w1 = make_float2(wq.z, wq.w);
+#pragma unroll
+                        for (int t = 0; t < TW; t++) {
+                            if (r == 0 && s2 == 0) {
+                                acc[slot][t][0] = __fmul2_rn(xc[t + s2][0], w0);
+                                acc[slot][t][1] = __fmul2_rn(xc[t + s2][1], w1);
+                            } else {
+                                acc[slot][t][0] = __ffma2_rn(xc[t + s2][0], w0, acc[slot][t][0]);
+                                acc[slot][t][1] = __ffma2_rn(xc[t + s2][1], w1, acc[slot][t][1]);
+                            }
+                        }
+                    }
+                }
+                // the output row this input row completes (filter row K - 1): hi - P
+                const int oh = hi - P;
+                if (active && oh >= ho_begin && oh < ho_end) {
+                    constexpr int KK = K;
+                    const int slot = ((u - (K - 1)) % KK + KK) % KK;
+                    __nv_bfloat16 *yrow = yimg + (size_t)oh * a.Wo * a.K;
+#pragma unroll
+                    for (int t = 0; t < TW; t++) {
+                        if (wo0 + t < a.Wo) {
+                            uint2 ov;
+                            __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+                            for (int j = 0; j < 2; j++) {
+                                float2 v = __ffma2_rn(acc[slot][t][j], sc[j], sh[j]);
+                                if (ACT == ACT_RELU) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); }
+                                if (ACT == ACT_HSWISH) {
+                                    const float2 g = make_float2(__saturatef(fmaf(v.x, 1.f / 6.f, 0.5f)), __saturatef(fmaf(v.y, 1.f / 6.f, 0.5f)));
+                                    v = __fmul2_rn(v, g);
+                                }
+                                ob[j] = __float22bfloat162_rn(v);
+                            }
+                            *reinterpret_cast<uint2 *>(yrow + (size_t)(wo0 + t) * a.K) = ov;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    cp_async_wait<0>();
+}
+template <int K, int ACT, bool GROUP>
+__global__ void __launch_bounds__(128) dw_walk_kernel(const ConvArgs a1, const char *__restrict__ tbl, int n_img, int chblocks) {
+    __shared__ __align__(16) unsigned char smem[DwWalkShape<K>::SMEM];
+    SGS_DW_ARGS()
+    if (GROUP) { const ConvArgs al = a; dw_walk_body<K, ACT>(al, n, smem, chblocks); }
+    else dw_walk_body<K, ACT>(a, n, smem, chblocks);
+}
+// grid of the walking kernel for a member with `kmax` channels at most
+static dim3 dw_walk_grid(const ConvArgs &a, int kmax, int TW, int images) {
+    const int chblocks = (kmax / 4 + 31) / 32, tiles_w = (a.Wo + 4 * TW - 1) / (4 * TW);
+    return dim3((unsigned)(chblocks * tiles_w), (unsigned)((a.Ho + DW_WALK_SEG - 1) / DW_WALK_SEG), (unsigned)images);
+}
+
 // Members of one launch with different kernel sizes (a wave's depthwise layer: every member crops its own
 // k x k window out of the stored 7x7): each block runs the body of its member's kernel size.  The grid
 // covers the largest member; blocks beyond a member's own extent leave at once.
-template <int ST, int ACT> __device__ __forceinline__ void dw_mixed_dispatch(const ConvArgs &a, const int n);
+// Stride 1: the walking bodies on the walking kernel's grid (sized for strips of 2 columns and the widest member);
+// stride 2: the patch / row bodies on their grid.
+template <int ST, int ACT> __device__ __forceinline__ void dw_mixed_dispatch(const ConvArgs &a, const int n, unsigned char *wsm, int chblocks);
 template <int ST, int ACT>
-__global__ void __launch_bounds__(128, 3) dw_mixed_kernel(const char *__restrict__ tbl, int n_img) {
+__global__ void __launch_bounds__(128, 3) dw_mixed_kernel(const char *__restrict__ tbl, int n_img, int chblocks) {
     constexpr bool GROUP = true;
+    __shared__ __align__(16) unsigned char wsm[ST == 1 ? DwWalkShape<7>::SMEM : 16];  // (7x7 needs the most; 5x5: 37376, 3x3: 41472 bytes)
+    static_assert(DwWalkShape<7>::SMEM >= DwWalkShape<5>::SMEM && DwWalkShape<7>::SMEM >= DwWalkShape<3>::SMEM && DwWalkShape<7>::SMEM <= 48 * 1024, "ring sizes");
     const ConvArgs a1 = ConvArgs();
     SGS_DW_ARGS()
     const ConvArgs al = a;  // (a copy in registers: reading the fields from shared memory at every use costs the tiled bodies 100 registers more)
-    dw_mixed_dispatch<ST, ACT>(al, n);
+    dw_mixed_dispatch<ST, ACT>(al, n, wsm, chblocks);
 }
 template <int ST, int ACT>
-__device__ __forceinline__ void dw_mixed_dispatch(const ConvArgs &a, const int n) {
-    if (a.k == 3) {
-        if (ST == 1) dw_tile_body<3, 1, 2, 4, true, ACT>(a, n);
-        else dw_tile_body<3, 2, 1, 4, false, ACT>(a, n);
-    } else if (a.k == 5) {
-        if (ST == 1) dw_tile_body<5, 1, 1, 4, true, ACT>(a, n);
-        else dw_vec_body<5, 2>(a, n);
+__device__ __forceinline__ void dw_mixed_dispatch(const ConvArgs &a, const int n, unsigned char *wsm, int chblocks) {
+    if (ST == 1) {
+        if (a.k == 3) dw_walk_body<3, ACT>(a, n, wsm, chblocks);
+        else if (a.k == 5) dw_walk_body<5, ACT>(a, n, wsm, chblocks);
+        else dw_walk_body<7, ACT>(a, n, wsm, chblocks);
     } else {
-        dw_vec_body<7, ST>(a, n);
+        if (a.k == 3) dw_tile_body<3, 2, 1, 4, false, ACT>(a, n);
+        else if (a.k == 5) dw_vec_body<5, 2>(a, n);
+        else dw_vec_body<7, 2>(a, n);
     }
 }
 
@@ -425,6 +594,16 @@ static cudaError_t launch_dw_tile(const ConvArgs &a, int kmax, const char *tbl, 
     if (a.act == ACT_RELU) dw_tile_kernel<K, ST, TH, TW, PRELOAD, ACT_RELU, GROUP><<<grid, 128, 0, st>>>(a, tbl, a.N);
     else if (a.act == ACT_HSWISH) dw_tile_kernel<K, ST, TH, TW, PRELOAD, ACT_HSWISH, GROUP><<<grid, 128, 0, st>>>(a, tbl, a.N);
     else dw_tile_kernel<K, ST, TH, TW, PRELOAD, ACT_NONE, GROUP><<<grid, 128, 0, st>>>(a, tbl, a.N);
+    return cudaGetLastError();
+}
+
+template <int K, bool GROUP>
+static cudaError_t launch_dw_walk(const ConvArgs &a, int kmax, const char *tbl, int members, cudaStream_t st) {
+    const dim3 grid = dw_walk_grid(a, kmax, DwWalkShape<K>::TW, a.N * (GROUP ? members : 1));
+    const int chblocks = (kmax / 4 + 31) / 32;
+    if (a.act == ACT_RELU) dw_walk_kernel<K, ACT_RELU, GROUP><<<grid, 128, 0, st>>>(a, tbl, a.N, chblocks);
+    else if (a.act == ACT_HSWISH) dw_walk_kernel<K, ACT_HSWISH, GROUP><<<grid, 128, 0, st>>>(a, tbl, a.N, chblocks);
+    else dw_walk_kernel<K, ACT_NONE, GROUP><<<grid, 128, 0, st>>>(a, tbl, a.N, chblocks);
     return cudaGetLastError();
 }
 
@@ -444,16 +623,19 @@ static bool dw_vec_eligible(const ConvArgs &a) {
            ((reinterpret_cast<uintptr_t>(a.scale) | reinterpret_cast<uintptr_t>(a.shift)) & 15) == 0;
 }
 
+static int g_dw_walk = 1;  // tuning aid: 0 = the patch / row kernels also for stride 1
+void dw_set_walk(int on) { g_dw_walk = on; }
+
 // The vectorised bf16 kernel of a (kernel size, stride) pair; measured on working sets beyond L2
 // (N64 56x56 C480) the tiled kernel wins for k3 and for k5 stride 1.
 template <bool GROUP>
 static cudaError_t launch_dw_bf16(const ConvArgs &a, int kmax, const char *tbl, int members, cudaStream_t st) {
     switch (a.k * 10 + a.stride) {
-    case 31: return launch_dw_tile<3, 1, 2, 4, true, GROUP>(a, kmax, tbl, members, st);
+    case 31: return g_dw_walk ? launch_dw_walk<3, GROUP>(a, kmax, tbl, members, st) : launch_dw_tile<3, 1, 2, 4, true, GROUP>(a, kmax, tbl, members, st);
     case 32: return launch_dw_tile<3, 2, 1, 4, false, GROUP>(a, kmax, tbl, members, st);
-    case 51: return launch_dw_tile<5, 1, 1, 4, true, GROUP>(a, kmax, tbl, members, st);
+    case 51: return g_dw_walk ? launch_dw_walk<5, GROUP>(a, kmax, tbl, members, st) : launch_dw_tile<5, 1, 1, 4, true, GROUP>(a, kmax, tbl, members, st);
     case 52: return launch_dw_vec<5, 2, GROUP>(a, kmax, tbl, members, st);
-    case 71: return launch_dw_vec<7, 1, GROUP>(a, kmax, tbl, members, st);
+    case 71: return g_dw_walk ? launch_dw_walk<7, GROUP>(a, kmax, tbl, members, st) : launch_dw_vec<7, 1, GROUP>(a, kmax, tbl, members, st);
     case 72: return launch_dw_vec<7, 2, GROUP>(a, kmax, tbl, members, st);
     default: return cudaErrorNotSupported;
     }
@@ -476,15 +658,17 @@ cudaError_t launch_dw_group(const char *h_tbl, const char *d_tbl, int members, c
     if (!mixed) return launch_dw_bf16<true>(a0, kmax, d_tbl, members, st);
     // (same input size and stride, odd kernels with padding (k - 1) / 2: every member has the same output size)
     const int per_row = ((a0.Wo + 3) / 4) * (kmax / 8);
-    dim3 grid((per_row + 127) / 128, a0.Ho, a0.N * members);
+    const int chblocks = (kmax / 4 + 31) / 32;
     if (a0.stride == 1) {
-        if (a0.act == ACT_RELU) dw_mixed_kernel<1, ACT_RELU><<<grid, 128, 0, st>>>(d_tbl, a0.N);
-        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<1, ACT_HSWISH><<<grid, 128, 0, st>>>(d_tbl, a0.N);
-        else dw_mixed_kernel<1, ACT_NONE><<<grid, 128, 0, st>>>(d_tbl, a0.N);
+        const dim3 grid = dw_walk_grid(a0, kmax, 2, a0.N * members);
+        if (a0.act == ACT_RELU) dw_mixed_kernel<1, ACT_RELU><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<1, ACT_HSWISH><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else dw_mixed_kernel<1, ACT_NONE><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
     } else {
-        if (a0.act == ACT_RELU) dw_mixed_kernel<2, ACT_RELU><<<grid, 128, 0, st>>>(d_tbl, a0.N);
-        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<2, ACT_HSWISH><<<grid, 128, 0, st>>>(d_tbl, a0.N);
-        else dw_mixed_kernel<2, ACT_NONE><<<grid, 128, 0, st>>>(d_tbl, a0.N);
+        dim3 grid((per_row + 127) / 128, a0.Ho, a0.N * members);
+        if (a0.act == ACT_RELU) dw_mixed_kernel<2, ACT_RELU><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<2, ACT_HSWISH><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else dw_mixed_kernel<2, ACT_NONE><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
     }
     return cudaGetLastError();
 }
@@ -1185,21 +1369,21 @@ cudaError_t launch_stem_gemm_weights(const void *src, void *dst, int K, int KK, 
 // Load-time kernels
 // ---------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void relayout_conv_kernel(const float *__restrict__ src, T *__restrict__ dst, int K, int C, int R, int S) {
-    size_t total = (size_t)K * C * R * S;
+__global__ void relayout_conv_kernel(const float *__restrict__ src, T *__restrict__ dst, int K, int C, int Cp, int R, int S) {
+    size_t total = (size_t)K * Cp * R * S;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        // i indexes dst [K][R][S][C]
-        int c = (int)(i % C);
-        size_t q = i / C;
+        // i indexes dst [K][R][S][Cp]; channels C..Cp-1 of a row are zero
+        int c = (int)(i % Cp);
+        size_t q = i / Cp;
         int s = (int)(q % S), r = (int)((q / S) % R), f = (int)(q / ((size_t)S * R));
-        dst[i] = from_f<T>(src[(((size_t)f * C + c) * R + r) * S + s]);
+        dst[i] = from_f<T>(c < C ? src[(((size_t)f * C + c) * R + r) * S + s] : 0.f);
     }
 }
-cudaError_t launch_relayout_conv(const float *src, void *dst, int K, int C, int R, int S, int bf16, cudaStream_t st) {
-    size_t total = (size_t)K * C * R * S;
+cudaError_t launch_relayout_conv(const float *src, void *dst, int K, int C, int Cp, int R, int S, int bf16, cudaStream_t st) {
+    size_t total = (size_t)K * Cp * R * S;
     int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 32);
-    if (bf16) relayout_conv_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(src, static_cast<__nv_bfloat16 *>(dst), K, C, R, S);
-    else relayout_conv_kernel<float><<<blocks, 256, 0, st>>>(src, static_cast<float *>(dst), K, C, R, S);
+    if (bf16) relayout_conv_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(src, static_cast<__nv_bfloat16 *>(dst), K, C, Cp, R, S);
+    else relayout_conv_kernel<float><<<blocks, 256, 0, st>>>(src, static_cast<float *>(dst), K, C, Cp, R, S);
     return cudaGetLastError();
 }
 
@@ -1245,6 +1429,48 @@ __global__ void delay_kernel(unsigned us) {
 cudaError_t launch_delay(unsigned microseconds, cudaStream_t st) {
     delay_kernel<<<1, 1, 0, st>>>(microseconds > 50000u ? 50000u : microseconds);
     return cudaGetLastError();
+}
+
+// Measurement aid: fp32 FMA rate of the CUDA cores.  Every thread runs `iters` rounds of 16 independent
+// fused multiply-adds on registers (no memory traffic, no dependence between the 16 chains inside a round);
+// the sum is stored so that the loop cannot be removed.
+__global__ void __launch_bounds__(256) fma_rate_kernel(float *out, int iters, float a, float b) {
+    float x[16];
+#pragma unroll
+    for (int j = 0; j < 16; j++) x[j] = (float)(threadIdx.x + j) * 1e-3f;
+    for (int i = 0; i < iters; i++) {
+#pragma unroll
+        for (int j = 0; j < 16; j++) x[j] = fmaf(x[j], a, b);
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < 16; j++) s += x[j];
+    out[blockIdx.x * blockDim.x + threadIdx.x] = s;
+}
+cudaError_t measure_fma_rate(double *tflops, cudaStream_t st) {
+    const int blocks = 148 * 8, threads = 256, iters = 4096;
+    float *out = nullptr;
+    cudaError_t e = cudaMalloc((void **)&out, (size_t)blocks * threads * sizeof(float));
+    if (e != cudaSuccess) return e;
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0);
+    cudaEventCreate(&e1);
+    float best = 0.f;
+    for (int rep = 0; rep < 5 && e == cudaSuccess; rep++) {
+        cudaEventRecord(e0, st);
+        fma_rate_kernel<<<blocks, threads, 0, st>>>(out, iters, 0.999f, 1e-3f);
+        cudaEventRecord(e1, st);
+        e = cudaEventSynchronize(e1);
+        float ms = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+        if (e == cudaSuccess && rep > 0 && (best == 0.f || ms < best)) best = ms;  // (first round: warm-up)
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    cudaFree(out);
+    if (e != cudaSuccess) return e;
+    *tflops = best > 0.f ? 2.0 * blocks * threads * 16.0 * iters / (best * 1e-3) / 1e12 : 0.0;
+    return cudaSuccess;
 }
 
 // Batch-norm folding: scale = gamma / sqrt(var + 1e-5), shift = beta - mean * scale (+ bias).
