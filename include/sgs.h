@@ -354,6 +354,38 @@ sgs_status_t sgs_conv2d_sliced_static(const sgs_conv_desc_t *desc, const void *d
                                       const float *d_shift, const void *d_res, void *d_y, void *cuda_stream);
 
 /*
+ * sgs_conv2d_sliced_i8 - one sliced convolution layer in the paper's own numeric format (Section 5.1, workload
+ * footnote: weights, activations and zero points are 8-bit integers, the scale a 32-bit integer; Section 4.2
+ * "Zero Point/Scale Buffer": the per-filter parameters the accelerator applies to its accumulators), on the 8-bit
+ * tensor cores with int32 accumulation.  Slicing is the same as in sgs_conv2d_sliced (first K filters, first C
+ * channels, centre k x k window).  All arithmetic is exact integer arithmetic:
+ *   acc[n][ho][wo][f] = sum_{r,s<k} sum_{c<C} (x[n][ho*stride+r-p][wo*stride+s-p][c] - zx) * w[f][o+r][o+s][c]
+ *                       (positions outside the image count as the real value 0, i.e. as zx)
+ *   t = rsr(acc * mult[f], 31 + shift[f]) + bias[f]  [+ rsr((res[n][ho][wo][f] - zr) * res_mult, 31 + res_shift)]  + zy
+ *   y = saturate(relu ? max(t, zy) : t)      with rsr(v, s) = floor((v + 2^(s-1)) / 2^s) in 64-bit arithmetic
+ * so that a real-valued layer y_r = act(scale_f * conv(x_r, w_r) + shift_f + res_r) with x_r = sx (x - zx),
+ * w_r = sw_f w, y_r = sy (y - zy) is represented by mult[f] * 2^-(31 + shift[f]) ~ sx * sw_f * scale_f / sy and
+ * bias[f] ~ shift_f / sy.
+ *   d_x    [N][H][W][C] bytes (unsigned, or signed if x_signed)     d_y, d_res  [N][Ho][Wo][K] bytes
+ *   d_w    stored weights [Kmax][R][R][Cmax] signed bytes            d_mult, d_shift, d_bias  [>= K] int32
+ * Limits of this entry point: C and Cmax multiples of 16, K a multiple of 8, 16-byte aligned pointers, stride-2
+ * inputs of even size, 0 <= shift[f] <= 31, and zx == 0 (an input zero point other than 0 would need the sum of the
+ * sliced weights under every window position, which changes with the slice and at image borders; post-ReLU tensors
+ * and symmetric signed tensors have zx = 0).  Other values: SGS_EUNSUPPORTED.  Asynchronous on `cuda_stream`.
+ */
+typedef struct {
+    int N, H, W, C, K;       /* input dims, sliced channels C, sliced filters K */
+    int Kmax, Cmax, R;       /* stored tensor dims */
+    int k, stride;           /* kernel size, stride (1 or 2) */
+    int relu;                /* 1: y = max(t, zy) */
+    int x_signed, y_signed, res_signed; /* 0: bytes are 0..255, 1: -128..127 */
+    int zx, zy, zr;          /* zero points of x, y, res */
+    int res_mult, res_shift; /* residual rescaling (ignored without d_res) */
+} sgs_conv_i8_desc_t;
+sgs_status_t sgs_conv2d_sliced_i8(const sgs_conv_i8_desc_t *desc, const void *d_x, const void *d_w, const int32_t *d_mult,
+                                  const int32_t *d_shift, const int32_t *d_bias, const void *d_res, void *d_y, void *cuda_stream);
+
+/*
  * sgs_aux_op - the layers of a SubNet that are not convolutions, one at a time on caller-owned device tensors
  * (the paper's SuperNets are the OFA ResNet50 / MobileNetV3 families of Section 5.1: max pool after the stem,
  * global average pool before the classifier and inside squeeze-excite blocks, fully connected layers sliced by

@@ -76,6 +76,8 @@ def lib():
         L.orc_layer_linear.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 4 + [ctypes.c_void_p]
         L.orc_layer_se_gate.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c_void_p]
         L.orc_layer_se_scale.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 4
+        L.orc_layer_conv_i8.argtypes = ([ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c_void_p] + [ctypes.c_int] * 9 + [ctypes.c_void_p] * 4
+                                        + [ctypes.c_int] * 7 + [ctypes.c_void_p])
         L.orc_bf16_round.restype = ctypes.c_float
         L.orc_bf16_round.argtypes = [ctypes.c_float]
         L.orc_set_tap.argtypes = [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t]
@@ -245,6 +247,30 @@ def layer_se_scale(x, gate, mode: int = FP32) -> np.ndarray:
     gate = _f32(gate)
     N, H, W, C = y.shape
     lib().orc_layer_se_scale(_ptr(y), _ptr(gate), N, H * W, C, mode)
+    return y
+
+
+def layer_conv_i8(w, x, Cp: int, Kp: int, k: int, stride: int, mult, shift, bias, zx: int = 0, zy: int = 0, relu: bool = False,
+                  res=None, zr: int = 0, res_mult: int = 0, res_shift: int = 0, y_signed: bool = False) -> np.ndarray:
+    """8-bit sliced convolution layer in exact integer arithmetic (see the C function).  ``w`` int8 [Kmax][Cmax][R][R];
+    ``x`` (and ``res``) uint8 or int8 NHWC, their dtype says how the bytes are read; returns uint8, or int8 if y_signed."""
+    w = np.ascontiguousarray(w, dtype=np.int8)
+    x = np.ascontiguousarray(x)
+    assert x.dtype in (np.uint8, np.int8)
+    Kmax, Cmax, R, _ = w.shape
+    N, H, W, _ = x.shape
+    p = (k - 1) // 2
+    Ho, Wo = (H + 2 * p - k) // stride + 1, (W + 2 * p - k) // stride + 1
+    mult, shift, bias = (np.ascontiguousarray(a, dtype=np.int32) for a in (mult, shift, bias))
+    if res is not None:
+        res = np.ascontiguousarray(res)
+        assert res.dtype in (np.uint8, np.int8) and res.shape == (N, Ho, Wo, Kp)
+    y = np.empty((N, Ho, Wo, Kp), dtype=np.int8 if y_signed else np.uint8)
+    rc = lib().orc_layer_conv_i8(_ptr(w), Kmax, Cmax, R, _ptr(x), int(x.dtype == np.int8), zx, N, H, W, Cp, Kp, k, stride,
+                                 _ptr(mult), _ptr(shift), _ptr(bias), _ptr(res), int(res is not None and res.dtype == np.int8), zr,
+                                 res_mult, res_shift, zy, int(relu), int(y_signed), _ptr(y))
+    if rc:
+        raise OverflowError("accumulator beyond 32 bits" if rc == -3 else f"orc_layer_conv_i8 failed ({rc})")
     return y
 
 

@@ -917,6 +917,64 @@ int orc_layer_se_gate(const float *w1, int ld1, const float *b1, const float *w2
 }
 /* In place: x[n][i][c] *= gate[n][c], with the storage rounding of `mode`. */
 void orc_layer_se_scale(float *x, const float *gate, int N, int HW, int C, int mode) { se_scale(x, gate, N, HW, C, mode); }
+/* ------------------------------------------------------------------------------------------ */
+/* 8-bit sliced convolution layer (the paper's numeric format: Section 5.1, workload footnote:   */
+/* int8 weights, activations and zero points, int32 scale; Section 4.2 Zero Point/Scale Buffer). */
+/* Exact integer arithmetic, direct loops.  w[Kmax][Cmax][R][R] signed bytes; x, res, y one byte */
+/* per element, read as 0..255 or (signed flag) -128..127.                                       */
+/*   acc = sum over in-image taps and c < Cp of (x - zx) * w      (outside the image: real 0)    */
+/*   t   = rsr(acc * mult[f], 31 + shift[f]) + bias[f] + rsr((res - zr) * res_mult, 31 + res_shift) + zy */
+/*   y   = saturate(relu ? max(t, zy) : t),   rsr(v, s) = floor((v + 2^(s-1)) / 2^s)             */
+/* ------------------------------------------------------------------------------------------ */
+static long long rsr64(long long v, int s) {
+    long long q = v + ((long long)1 << (s - 1));
+    /* floor division by 2^s written without relying on the shift of a negative number */
+    long long d = (long long)1 << s, r = q / d;
+    if (q % d != 0 && q < 0) r -= 1;
+    return r;
+}
+static int byte_value(const unsigned char *p, size_t i, int is_signed) { return is_signed ? (int)(signed char)p[i] : (int)p[i]; }
+
+int orc_layer_conv_i8(const signed char *w, int Kmax, int Cmax, int R, const unsigned char *x, int x_signed, int zx, int N,
+                      int H, int W, int Cp, int Kp, int k, int st, const int *mult, const int *shift, const int *bias,
+                      const unsigned char *res, int res_signed, int zr, int res_mult, int res_shift, int zy, int relu,
+                      int y_signed, unsigned char *y) {
+    const int p = (k - 1) / 2, o = (R - k) / 2;
+    const int Ho = (H + 2 * p - k) / st + 1, Wo = (W + 2 * p - k) / st + 1;
+    (void)Kmax;
+    for (int n = 0; n < N; n++)
+        for (int ho = 0; ho < Ho; ho++)
+            for (int wo = 0; wo < Wo; wo++)
+                for (int f = 0; f < Kp; f++) {
+                    long long acc = 0;
+                    for (int r = 0; r < k; r++) {
+                        int hi = ho * st + r - p;
+                        if (hi < 0 || hi >= H) continue;
+                        for (int s = 0; s < k; s++) {
+                            int wi = wo * st + s - p;
+                            if (wi < 0 || wi >= W) continue;
+                            for (int c = 0; c < Cp; c++) {
+                                int xv = byte_value(x, (((size_t)n * H + hi) * W + wi) * Cp + c, x_signed) - zx;
+                                int wv = (int)w[(((size_t)f * Cmax + c) * R + (o + r)) * R + (o + s)];
+                                acc += (long long)xv * wv;
+                            }
+                        }
+                    }
+                    if (acc > 2147483647ll || acc < -2147483648ll) return -3; /* the format's accumulator is 32 bits */
+                    int sh = shift[f] < 0 ? 0 : (shift[f] > 31 ? 31 : shift[f]);
+                    size_t oi = (((size_t)n * Ho + ho) * Wo + wo) * Kp + f;
+                    long long t = rsr64(acc * (long long)mult[f], 31 + sh) + bias[f];
+                    if (res) t += rsr64((long long)(byte_value(res, oi, res_signed) - zr) * (long long)res_mult, 31 + res_shift);
+                    t += zy;
+                    if (relu && t < zy) t = zy;
+                    long long lo = y_signed ? -128 : 0, hi2 = y_signed ? 127 : 255;
+                    if (t < lo) t = lo;
+                    if (t > hi2) t = hi2;
+                    y[oi] = (unsigned char)(t & 0xff);
+                }
+    return 0;
+}
+
 float orc_bf16_round(float x) { return bf16_round(x); }
 
 #ifdef _OPENMP

@@ -27,13 +27,18 @@ EXPORTS = [
     "sgs_set_option", "sgs_get_counter", "sgs_last_error", "sgs_supernet_free", "sgs_conv2d_sliced", "sgs_device_status",
     "sgs_profile_read", "sgs_conv2d_sliced_static", "sgs_cache_set_candidates", "sgs_cache_set_policy",
     "sgs_sched_create", "sgs_sched_free", "sgs_sched_dims", "sgs_sched_set_table", "sgs_sched_get_table", "sgs_sched_measure",
-    "sgs_sched_step", "sgs_sched_subnet", "sgs_profile_trace", "sgs_layer_name", "sgs_aux_op", "sgs_device_status_clear", "sgs_debug_expire_wait", "sgs_measure_fma_peak",
+    "sgs_sched_step", "sgs_sched_subnet", "sgs_profile_trace", "sgs_layer_name", "sgs_aux_op", "sgs_device_status_clear", "sgs_debug_expire_wait", "sgs_measure_fma_peak", "sgs_conv2d_sliced_i8",
 ]
 
 
 class ConvDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("N", "H", "W", "C", "K", "Kmax", "Cmax", "R", "k", "stride", "act", "dtype",
                                              "impl", "depthwise", "cache_k", "cache_c", "weight_policy", "split_k_off")]
+
+
+class ConvI8Desc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("N", "H", "W", "C", "K", "Kmax", "Cmax", "R", "k", "stride", "relu", "x_signed", "y_signed",
+                                             "res_signed", "zx", "zy", "zr", "res_mult", "res_shift")]
 
 
 SGS_AUX_MAXPOOL, SGS_AUX_AVGPOOL, SGS_AUX_LINEAR, SGS_AUX_SE_GATE, SGS_AUX_SE_SCALE = range(5)
@@ -198,6 +203,7 @@ def lib():
         L.sgs_device_status_clear.argtypes = []
         L.sgs_debug_expire_wait.argtypes = [ctypes.c_uint, vp]
         L.sgs_measure_fma_peak.argtypes = [vp, vp]
+        L.sgs_conv2d_sliced_i8.argtypes = [vp] * 9
         L.sgs_profile_read.argtypes = [vp, ci, vp, vp, vp, vp]
         _lib = L
     return _lib
@@ -226,6 +232,12 @@ def conv2d_sliced_static(desc: ConvDesc, d_x: int, d_w: int, d_scale: int, d_shi
     st = lib().sgs_conv2d_sliced_static(ctypes.byref(desc), d_x, d_w, d_scale, d_shift, d_res or None, d_y, stream)
     if st != SGS_OK:
         raise SgsError(st, "sgs_conv2d_sliced_static")
+
+
+def conv2d_sliced_i8(desc: ConvI8Desc, d_x: int, d_w: int, d_mult: int, d_shift: int, d_bias: int, d_res: int, d_y: int, stream: int = 0):
+    st = lib().sgs_conv2d_sliced_i8(ctypes.byref(desc), d_x, d_w, d_mult, d_shift, d_bias, d_res or None, d_y, stream)
+    if st != SGS_OK:
+        raise SgsError(st, "sgs_conv2d_sliced_i8")
 
 
 def device_status_clear():

@@ -2314,6 +2314,34 @@ sgs_status_t sgs_conv2d_sliced(const sgs_conv_desc_t *d, const void *d_x, const 
     return e == cudaSuccess ? SGS_OK : SGS_ECUDA;
 }
 
+// One sliced convolution layer with 8-bit operands on the tensor cores (see sgs.h).
+sgs_status_t sgs_conv2d_sliced_i8(const sgs_conv_i8_desc_t *d, const void *d_x, const void *d_w, const int32_t *d_mult,
+                                  const int32_t *d_shift, const int32_t *d_bias, const void *d_res, void *d_y, void *cuda_stream) {
+    if (!d || !d_x || !d_w || !d_mult || !d_shift || !d_bias || !d_y) return SGS_EINVAL;
+    if (d->N <= 0 || d->H <= 0 || d->W <= 0 || d->C <= 0 || d->K <= 0 || d->k <= 0 || (d->k & 1) == 0 || d->k > d->R ||
+        ((d->R - d->k) & 1) || d->K > d->Kmax || d->C > d->Cmax || (d->stride != 1 && d->stride != 2) || d->res_shift < 0 || d->res_shift > 31)
+        return SGS_EINVAL;
+    if (d->zx != 0 || !tc_available()) return SGS_EUNSUPPORTED;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SGS_ECUDA;
+    ConvArgs a;
+    a.x = d_x; a.w = d_w; a.res = d_res; a.y = d_y;
+    a.N = d->N; a.H = d->H; a.W = d->W; a.C = d->C; a.K = d->K;
+    a.Kmax = d->Kmax; a.Cmax = d->Cmax; a.R = d->R; a.k = d->k; a.stride = d->stride;
+    const int p = (d->k - 1) / 2;
+    a.Ho = (d->H + 2 * p - d->k) / d->stride + 1;
+    a.Wo = (d->W + 2 * p - d->k) / d->stride + 1;
+    a.i8 = 1;
+    a.q_mult = d_mult; a.q_shift = d_shift; a.q_bias = d_bias;
+    a.q_zy = d->zy; a.q_zr = d->zr; a.q_res_mult = d->res_mult; a.q_res_shift = d->res_shift;
+    a.q_flags = (d->x_signed ? 1 : 0) | (d->y_signed ? 2 : 0) | (d->res_signed ? 4 : 0) | (d->relu ? 8 : 0);
+    std::string why;
+    std::shared_ptr<TcConvPlan> plan = tc_conv_prepare(a, dev, &why);
+    if (!plan) return SGS_EUNSUPPORTED;
+    int n = 0;
+    return tc_conv_launch(*plan, a, (cudaStream_t)cuda_stream, &n) == cudaSuccess ? SGS_OK : SGS_ECUDA;
+}
+
 // Non-convolution layers on caller tensors (see sgs.h).  Mirrors the dispatch of launch_op / wave_impl.
 sgs_status_t sgs_aux_op(int n, const sgs_aux_desc_t *desc, const sgs_aux_args_t *args, int grouped, void *cuda_stream) {
     if (n <= 0 || n > 65535 || !desc || !args) return SGS_EINVAL;

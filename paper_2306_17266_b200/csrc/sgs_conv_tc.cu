@@ -41,8 +41,10 @@ namespace {
 // The kernel.  grid = (m tiles, n tiles, K splits), block = 192.
 // Dynamic shared memory (1024-byte aligned): STAGES x [A tile 16 KB | B tile BN*128 B].
 // ---------------------------------------------------------------------------------------------
-template <int BN, int STAGES>
+template <int BN, int STAGES, bool I8>
 __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__ TcParams p) {
+    // (a stage row is 128 bytes either way: 64 bf16 or 128 8-bit channels; an MMA takes 32 bytes of it)
+    constexpr int CH = I8 ? 2 * CHUNK_C : CHUNK_C, KS = I8 ? 32 : 16;
     constexpr int B_STAGE_BYTES = BN * CHUNK_C * 2;
     constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
@@ -50,7 +52,8 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
     __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
-    __shared__ float scale_s[BN], shift_s[BN];
+    __shared__ float scale_s[BN], shift_s[BN];  // folded batch norm (8-bit layers: multiplier and shift as integers, plus the bias)
+    __shared__ int bias_s[I8 ? BN : 1];
 
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -63,7 +66,10 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
     const int f0 = blockIdx.y * BN;
     // MMA shape: M = 128, N = this tile's filters rounded up to 16, bf16 x bf16 -> fp32, both K-major
     const int n_mma = min(BN, (p.K - f0 + 15) & ~15);
-    const uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+    // instruction descriptor: accumulator format (1 fp32, 2 int32) at bit 4, A / B formats at bits 7 / 10 (bf16 = 1;
+    // 8-bit: 0 unsigned, 1 signed), N >> 3 at bit 17, M >> 4 at bit 24; both operands K-major
+    const uint32_t IDESC = I8 ? ((2u << 4) | ((uint32_t)(p.q_flags & 1) << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24))
+                              : ((1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24));
     // K range of this split
     const int per = (p.iters + p.splits - 1) / p.splits;
     const int it_begin = blockIdx.z * per, it_end = min(p.iters, it_begin + per);
@@ -79,8 +85,14 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
     if (warp >= 2) {
         for (int j = threadIdx.x - 64; j < BN; j += 128) {
             int f = f0 + j;
-            scale_s[j] = f < p.K ? p.scale[f] : 0.f;
-            shift_s[j] = f < p.K ? p.shift[f] : 0.f;
+            if (I8) {
+                reinterpret_cast<int *>(scale_s)[j] = f < p.K ? p.q_mult[f] : 0;
+                reinterpret_cast<int *>(shift_s)[j] = f < p.K ? min(max(p.q_shift[f], 0), 31) : 0;  // (0..31 by contract)
+                bias_s[I8 ? j : 0] = f < p.K ? p.q_bias[f] : 0;
+            } else {
+                scale_s[j] = f < p.K ? p.scale[f] : 0.f;
+                shift_s[j] = f < p.K ? p.shift[f] : 0.f;
+            }
         }
     }
     tc_fence_before();
@@ -121,7 +133,7 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
             int cc2 = cc, r2 = r, sx2 = sx;
             const int pre = min(n_it, STAGES);
             for (int i = 0; i < pre; i++) {
-                if (elect_one()) load_weights(i, cc2 * CHUNK_C, (p.o + r2) * p.R + (p.o + sx2));
+                if (elect_one()) load_weights(i, cc2 * CH, (p.o + r2) * p.R + (p.o + sx2));
                 __syncwarp();
                 if (++cc2 == p.cchunks) { cc2 = 0; if (++sx2 == p.k) { sx2 = 0; ++r2; } }
             }
@@ -131,7 +143,7 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
             const int s = i % STAGES, round = i / STAGES;
             bool ok = round == 0 || mbar_wait(&empty_bar[s], (round - 1) & 1, abort_flag);
             if (!__all_sync(0xffffffffu, ok)) break;
-            const int c0 = cc * CHUNK_C;
+            const int c0 = cc * CH;
             uint8_t *sa = smem + s * STAGE_BYTES;
             const int dh = r - p.p, dw = sx - p.p;
             if (elect_one()) {
@@ -156,12 +168,14 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
             ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], round & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            const int ksteps = (min(CHUNK_C, p.C - cc * CHUNK_C) + 15) / 16;
+            const int ksteps = (min(CH, p.C - cc * CH) + KS - 1) / KS;
             const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_STAGE_BYTES;
             const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
             if (elect_one()) {
-                for (int q = 0; q < ksteps; q++)
-                    umma_bf16(tmem_base, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), IDESC, (i > 0 || q > 0) ? 1u : 0u);
+                for (int q = 0; q < ksteps; q++) {
+                    if (I8) umma_i8(tmem_base, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), IDESC, (i > 0 || q > 0) ? 1u : 0u);
+                    else umma_bf16(tmem_base, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), IDESC, (i > 0 || q > 0) ? 1u : 0u);
+                }
                 umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
                 if (i == n_it - 1) umma_commit(&accum_bar);  // accumulator complete
             }
@@ -186,7 +200,51 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
         const int ncols = min(BN, p.K - f0);  // filters of this tile, a multiple of 8
-        if (p.splits == 1) {
+        if (I8) {
+            // integer epilogue: requantise the int32 accumulator per filter, add bias, residual and the output
+            // zero point, ReLU as a maximum with the zero point, saturate, store 8 filters (8 bytes) at a time
+            if (ok) {
+                const int m = row_m[row];
+                const int *mult = reinterpret_cast<const int *>(scale_s), *shf = reinterpret_cast<const int *>(shift_s);
+                const uint8_t *res8 = reinterpret_cast<const uint8_t *>(p.res);
+                uint8_t *y8 = reinterpret_cast<uint8_t *>(p.y);
+                const bool ysig = p.q_flags & 2, rsig = p.q_flags & 4, relu = p.q_flags & 8;
+                const int lo = ysig ? -128 : 0, hi = ysig ? 127 : 255;
+#pragma unroll 1
+                for (int j0 = 0; j0 < ncols; j0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + j0, v);
+                    tmem_ld_wait();
+                    if (m >= 0) {
+#pragma unroll
+                        for (int g = 0; g < 4; g++) {
+                            const int c = j0 + 8 * g;
+                            if (c < ncols) {
+                                const size_t oi = (size_t)m * p.K + f0 + c;
+                                uint2 rraw = make_uint2(0u, 0u);
+                                if (res8) rraw = *reinterpret_cast<const uint2 *>(res8 + oi);
+                                uint2 outw = make_uint2(0u, 0u);
+#pragma unroll
+                                for (int j = 0; j < 8; j++) {
+                                    long long t = rshift_round((long long)(int)v[8 * g + j] * (long long)mult[c + j], 31 + shf[c + j]) + (long long)bias_s[I8 ? c + j : 0];
+                                    if (res8) {
+                                        const uint32_t rb = ((j < 4 ? rraw.x : rraw.y) >> (8 * (j & 3))) & 0xffu;
+                                        const int rq = rsig ? (int)(signed char)rb : (int)rb;
+                                        t += rshift_round((long long)(rq - p.q_zr) * (long long)p.q_res_mult, 31 + p.q_res_shift);
+                                    }
+                                    t += p.q_zy;
+                                    if (relu && t < p.q_zy) t = p.q_zy;
+                                    const int q8 = (int)(t < lo ? lo : (t > hi ? hi : t));
+                                    const uint32_t byte = (uint32_t)q8 & 0xffu;
+                                    if (j < 4) outw.x |= byte << (8 * j); else outw.y |= byte << (8 * (j - 4));
+                                }
+                                *reinterpret_cast<uint2 *>(y8 + oi) = outw;
+                            }
+                        }
+                    }
+                }
+            }
+        } else if (p.splits == 1) {
             // straight from tensor memory to global memory: each thread finishes its own pixel row,
             // 8 filters (16 bytes) per store
             if (ok) {
@@ -320,11 +378,11 @@ std::unordered_map<MapKey, CUtensorMap, MapKeyHash> g_map_cache;
 std::mutex g_map_mu;
 
 bool encode_map(CUtensorMap *m, const void *base, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
-                const uint32_t *box) {
+                const uint32_t *box, bool bytes = false) {
     MapKey key;
     std::memset(&key, 0, sizeof key);
     key.v[0] = reinterpret_cast<uint64_t>(base);
-    key.v[1] = (uint64_t)rank;
+    key.v[1] = (uint64_t)rank | (bytes ? 256u : 0u);
     for (int i = 0; i < rank; i++) { key.v[2 + i] = dims[i]; key.v[11 + (i >> 1)] |= (uint64_t)box[i] << (32 * (i & 1)); }
     for (int i = 0; i + 1 < rank; i++) key.v[7 + i] = strides_bytes[i];
     {
@@ -336,7 +394,7 @@ bool encode_map(CUtensorMap *m, const void *base, int rank, const uint64_t *dims
     cuuint32_t bx[5], es[5];
     for (int i = 0; i < rank; i++) { gd[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
     for (int i = 0; i + 1 < rank; i++) gs[i] = strides_bytes[i];
-    CUresult r = encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), gd, gs, bx, es,
+    CUresult r = encode_fn()(m, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), gd, gs, bx, es,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return false;
@@ -427,6 +485,15 @@ cudaError_t tc_expire_wait(unsigned limit_us, cudaStream_t st) {
 
 // Picks the output-pixel box (bw, bh, bn), bw*bh*bn <= 128, that wastes the fewest tile rows.
 static void choose_box(int N, int Ho, int Wo, int *bw_, int *bh_, int *bn_) {
+    // (the search visits a few hundred candidates; a stream of never-seen SubNets asks for the same few shapes)
+    static std::unordered_map<uint64_t, uint32_t> memo;
+    static std::mutex memo_mu;
+    const uint64_t key = ((uint64_t)(uint32_t)N << 40) | ((uint64_t)(uint32_t)Ho << 20) | (uint32_t)Wo;
+    {
+        std::lock_guard<std::mutex> lk(memo_mu);
+        auto it = memo.find(key);
+        if (it != memo.end()) { *bw_ = it->second & 0xff; *bh_ = (it->second >> 8) & 0xff; *bn_ = (it->second >> 16) & 0xff; return; }
+    }
     double best = -1;
     int bbw = 1, bbh = 1, bbn = 1;
     for (int bw = 1; bw <= std::min(Wo, TILE_M); bw++) {
@@ -440,12 +507,17 @@ static void choose_box(int N, int Ho, int Wo, int *bw_, int *bh_, int *bn_) {
         }
     }
     *bw_ = bbw; *bh_ = bbh; *bn_ = bbn;
+    if (N < (1 << 20) && Ho < (1 << 20) && Wo < (1 << 20)) {
+        std::lock_guard<std::mutex> lk(memo_mu);
+        if (memo.size() < 65536) memo.emplace(key, (uint32_t)bbw | ((uint32_t)bbh << 8) | ((uint32_t)bbn << 16));
+    }
 }
 
 std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::string *why) {
     auto no = [&](const char *msg) { if (why) *why = msg; return std::shared_ptr<TcConvPlan>(); };
     if (!encode_fn()) return no("cuTensorMapEncodeTiled unavailable");
     if (a.C % 8 || a.K % 8 || a.Cmax % 8) return no("channel counts must be multiples of 8");
+    if (a.i8 && (a.C % 16 || a.Cmax % 16 || a.throughput || a.ldx || a.ldy || a.win)) return no("8-bit layers: channels in multiples of 16, single launches");
     if (a.C < 8 || a.K < 8) return no("too few channels");
     if (a.k % 2 == 0 || a.k > a.R) return no("kernel size");
     if (a.stride != 1 && a.stride != 2) return no("stride");
@@ -472,7 +544,10 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
     const bool flat = a.k == 1 && a.stride == 1;
     // C = channels per pixel of x as stored (pitch and extent of the activation maps): with padded pixels the
     // channels beyond the slice are zeros, so the maps may show them and no row ends inside a 32-byte sector
-    const uint64_t C = (uint64_t)(a.ldx ? a.ldx : a.C), eb = 2;
+    const uint64_t C = (uint64_t)(a.ldx ? a.ldx : a.C), eb = a.i8 ? 1 : 2;
+    const uint32_t CH = a.i8 ? 2 * CHUNK_C : CHUNK_C;  // channels per stage (128 bytes)
+    const bool b8 = a.i8 != 0;
+    plan->i8 = a.i8;
     // Grouped launches (throughput == 2) run a layer with very few output pixels "swapped": the filters
     // take the 128-row side of the MMA and ALL pixels of the member form the other operand (one pixel
     // tile), so that no MMA rows are wasted on a 2x2 or 4x4 map.  (The kernel takes up to 256 pixels
@@ -488,8 +563,8 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
         p.bw = swap ? (int)M : a.throughput == 2 ? (int)std::min<uint64_t>(M, TILE_M) : TILE_M; p.bh = 1; p.bn = 1;
         p.N = 1; p.Ho = 1; p.Wo = (int)M;
         uint64_t dims[4] = {C, M, 1, 1}, str[3] = {C * eb, M * C * eb, M * C * eb};
-        uint32_t box[4] = {CHUNK_C, (uint32_t)p.bw, 1, 1};
-        if (!encode_map(&p.tmA[0], a.x, 4, dims, str, box)) return no("activation tensor map");
+        uint32_t box[4] = {CH, (uint32_t)p.bw, 1, 1};
+        if (!encode_map(&p.tmA[0], a.x, 4, dims, str, box, b8)) return no("activation tensor map");
     } else {
         if (swap) { p.bw = a.Wo; p.bh = a.Ho; p.bn = a.N; }
         else choose_box(a.N, a.Ho, a.Wo, &p.bw, &p.bh, &p.bn);
@@ -505,20 +580,20 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
                 if (!encode_map(&p.tmA[ph * 2], base, 4, dims, str, wbox)) return no("window tensor map");
             }
         }
-        uint32_t box[4] = {CHUNK_C, (uint32_t)p.bw, (uint32_t)p.bh, (uint32_t)p.bn};
+        uint32_t box[4] = {CH, (uint32_t)p.bw, (uint32_t)p.bh, (uint32_t)p.bn};
         if (a.win) {
             // (encoded above)
         } else if (a.stride == 1) {
             uint64_t dims[4] = {C, (uint64_t)a.W, (uint64_t)a.H, (uint64_t)a.N};
             uint64_t str[3] = {C * eb, (uint64_t)a.W * C * eb, (uint64_t)a.H * a.W * C * eb};
-            if (!encode_map(&p.tmA[0], a.x, 4, dims, str, box)) return no("activation tensor map");
+            if (!encode_map(&p.tmA[0], a.x, 4, dims, str, box, b8)) return no("activation tensor map");
         } else {
             for (int ph = 0; ph < 2; ph++)
                 for (int pw = 0; pw < 2; pw++) {
                     const char *base = static_cast<const char *>(a.x) + ((size_t)ph * a.W + pw) * C * eb;
                     uint64_t dims[4] = {C, (uint64_t)a.W / 2, (uint64_t)a.H / 2, (uint64_t)a.N};
                     uint64_t str[3] = {2 * C * eb, 2 * (uint64_t)a.W * C * eb, (uint64_t)a.H * a.W * C * eb};
-                    if (!encode_map(&p.tmA[ph * 2 + pw], base, 4, dims, str, box)) return no("activation tensor map");
+                    if (!encode_map(&p.tmA[ph * 2 + pw], base, 4, dims, str, box, b8)) return no("activation tensor map");
                 }
         }
     }
@@ -535,7 +610,7 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
         if (!ds.sms) cudaDeviceGetAttribute(&ds.sms, cudaDevAttrMultiProcessorCount, device);
         if (ds.sms > 0) sms = ds.sms;
     }
-    p.cchunks = (a.C + CHUNK_C - 1) / CHUNK_C;
+    p.cchunks = (a.C + (int)CH - 1) / (int)CH;
     p.iters = a.k * plan->kw * p.cchunks;
     // Filter tile.  Issuing one MMA costs the issuing thread about the same whatever its width, so wide
     // tiles are preferred as long as tiles x K splits can still occupy every SM.
@@ -559,6 +634,7 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
         max_splits = 1;
         BN = swap ? 128 : a.K <= 64 ? 64 : a.K <= 128 ? 128 : 256;
     }
+    if (a.i8) max_splits = 1;  // (the integer epilogue has no second step)
     plan->bn_tile = BN;
     {
         const uint64_t taps = a.win ? (uint64_t)a.k : (uint64_t)a.R * a.R;  // stored taps per filter
@@ -566,8 +642,8 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
         const uint64_t Cw = a.ldx ? std::min<uint64_t>((uint64_t)a.ldx, (uint64_t)a.Cmax) : (uint64_t)a.C;
         uint64_t dims[3] = {Cw, taps, (uint64_t)a.K};
         uint64_t str[2] = {(uint64_t)a.Cmax * eb, taps * a.Cmax * eb};
-        uint32_t box[3] = {CHUNK_C, 1, (uint32_t)BN};
-        if (!encode_map(&p.tmW, a.w, 3, dims, str, box)) return no("weight tensor map");
+        uint32_t box[3] = {CH, 1, (uint32_t)BN};
+        if (!encode_map(&p.tmW, a.w, 3, dims, str, box, b8)) return no("weight tensor map");
     }
     const int ntiles = (a.K + BN - 1) / BN;
     // split the K loop when the tiles alone cannot fill the machine
@@ -596,7 +672,7 @@ static cudaError_t launch_finish(const TcParams &prm, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-template <int BN, int STAGES> static cudaError_t launch_variant(const TcConvPlan &pl, const TcParams &prm, cudaStream_t st) {
+template <int BN, int STAGES, bool I8 = false> static cudaError_t launch_variant(const TcConvPlan &pl, const TcParams &prm, cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = pl.grid;
     cfg.blockDim = dim3(192);
@@ -607,7 +683,7 @@ template <int BN, int STAGES> static cudaError_t launch_variant(const TcConvPlan
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, conv_tc_kernel<BN, STAGES>, prm);
+    return cudaLaunchKernelEx(&cfg, conv_tc_kernel<BN, STAGES, I8>, prm);
 }
 
 // One-time set-up of the current device: status word and the kernels' shared-memory limits.  Must
@@ -622,9 +698,11 @@ cudaError_t tc_conv_init(int dev) {
         if ((e = cudaMalloc(&ds.status, sizeof(int))) != cudaSuccess) return e;
         if ((e = cudaMemset(ds.status, 0, sizeof(int))) != cudaSuccess) return e;
     }
-    if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 3>())) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(conv_tc_kernel<256, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<256, 4>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 3>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(conv_tc_kernel<256, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<256, 4>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 3>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
     if ((e = tc_group_init(dev)) != cudaSuccess) return e;
     ds.attrs_set = true;
     return cudaSuccess;
@@ -646,6 +724,14 @@ cudaError_t tc_conv_launch(const TcConvPlan &pl, const ConvArgs &a, cudaStream_t
     if (prm.splits > 1 && (!a.ws || a.ws_elems < pl.ws_elems)) prm.splits = 1;  // no workspace: run unsplit
     TcConvPlan run = pl;
     run.grid.z = (unsigned)prm.splits;
+    if (pl.i8) {
+        if (!a.q_mult || !a.q_shift || !a.q_bias || pl.bn_tile > 128 || prm.splits != 1) return cudaErrorInvalidValue;
+        prm.q_mult = a.q_mult; prm.q_shift = a.q_shift; prm.q_bias = a.q_bias;
+        prm.q_zy = a.q_zy; prm.q_zr = a.q_zr; prm.q_res_mult = a.q_res_mult; prm.q_res_shift = a.q_res_shift; prm.q_flags = a.q_flags;
+        e = pl.bn_tile == 64 ? launch_variant<64, 3, true>(run, prm, st) : launch_variant<128, 3, true>(run, prm, st);
+        if (launches) *launches = 1;
+        return e;
+    }
     if (pl.bn_tile == 64) e = launch_variant<64, 3>(run, prm, st);
     else if (pl.bn_tile == 128) e = launch_variant<128, 3>(run, prm, st);
     else e = launch_variant<256, 4>(run, prm, st);
@@ -689,9 +775,9 @@ cudaError_t static_scratch_setup(int dev, StaticScratch **out) {
         StaticScratch *ptr = nullptr;
         cudaError_t e = cudaGetSymbolAddress((void **)&ptr, g_static_scratch);
         if (e != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 3>())) != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(conv_tc_kernel<256, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<256, 4>())) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 3>())) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(conv_tc_kernel<256, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<256, 4>())) != cudaSuccess) return e;
         if ((e = cudaMemset(&ptr->status, 0, sizeof(int))) != cudaSuccess) return e;
         g_static_ptr[dev] = ptr;
     }

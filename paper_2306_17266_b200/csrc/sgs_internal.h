@@ -54,6 +54,9 @@ struct ConvArgs {
     // third of the rate (measured on sm_100a), and C, K are multiples of 8 only.  Tensor-core kernels of grouped
     // launches only; they write the zeros of y.
     int ldx = 0, ldy = 0;
+    int i8 = 0;  // 8-bit operands (x, w, res, y one byte per element; sgs_conv2d_sliced_i8): tensor-core kernel only
+    const int *q_mult = nullptr, *q_shift = nullptr, *q_bias = nullptr;  // ... with the integer epilogue of TcParams
+    int q_zy = 0, q_zr = 0, q_res_mult = 0, q_res_shift = 0, q_flags = 0;
     int k = 1, stride = 1, act = 0;
     // Window view of a 3-channel stem (grouped launches): x is the input padded to 8 channels with a zero
     // margin, [N][H][W][8] with H, W the PADDED sizes; an "input channel" chunk is the 8-pixel x 8-channel

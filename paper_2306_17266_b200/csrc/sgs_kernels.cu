@@ -406,7 +406,7 @@ __global__ void __launch_bounds__(128) dw_tile_kernel(const ConvArgs a1, const c
 // the block's 128 channels sit unpacked (fp32) in shared memory; a lane reads its four per tap with one 16-byte load.
 // Grid: x = channel blocks x column tiles, y = row segments, z = image (x member).
 #ifndef DW_WALK_SEG_ROWS
-#define DW_WALK_SEG_ROWS 28
+#define DW_WALK_SEG_ROWS 56
 #endif
 constexpr int DW_WALK_SEG = DW_WALK_SEG_ROWS;  // output rows per segment (halo: K - 1 extra input rows per segment)
 template <int K> struct DwWalkShape {
@@ -460,17 +460,30 @@ __device__ __forceinline__ void dw_walk_body(const ConvArgs &a, const int n, uns
     const float4 *wl = reinterpret_cast<const float4 *>(wsm) + lane;
 
     const int hi_first = ho_begin - P, hi_last = ho_end - 1 + P;  // input rows that meet the segment (may lie outside the image)
-    // one input row of the tile -> ring slot (hi - hi_first) % RING; 16 chunks of 16 bytes per column
+    // One input row of the tile -> ring slot (hi - hi_first) % RING, 16 chunks of 16 bytes per column.  A thread
+    // copies the same (column, channel) chunks of every row: their offsets and whether they lie inside the tensor
+    // are fixed before the row loop.
+    constexpr int NCH = (ICOL * 16 + 127) / 128;  // chunks per thread and row
+    int src_off[NCH], dst_off[NCH];               // element offset inside an input row (-1: outside), byte offset in the slot
+#pragma unroll
+    for (int i = 0; i < NCH; i++) {
+        const int q = threadIdx.x + i * 128;
+        const int j = q >> 4, part = q & 15;
+        const int wi = wt0 - P + j, c = cb * 128 + part * 8;
+        dst_off[i] = q < ICOL * 16 ? q * 16 : -1;
+        src_off[i] = (q < ICOL * 16 && wi >= 0 && wi < a.W && c < a.K) ? wi * a.K + c : -1;
+    }
     auto copy_row = [&](int hi) {
         if (hi <= hi_last) {
             unsigned char *dst = ring + ((hi - hi_first) % RING) * S::ROW_BYTES;
             const bool rok = hi >= 0 && hi < a.H;
             const __nv_bfloat16 *xrow = ximg + (size_t)(rok ? hi : 0) * a.W * a.K;
-            for (int q = threadIdx.x; q < ICOL * 16; q += 128) {
-                const int j = q >> 4, part = q & 15;
-                const int wi = wt0 - P + j, c = cb * 128 + part * 8;
-                const bool ok = rok && wi >= 0 && wi < a.W && c < a.K;
-                cp_async16(dst + q * 16, ok ? (const void *)(xrow + (size_t)wi * a.K + c) : (const void *)ximg, ok);
+#pragma unroll
+            for (int i = 0; i < NCH; i++) {
+                if (dst_off[i] >= 0) {
+                    const bool ok = rok && src_off[i] >= 0;
+                    cp_async16(dst + dst_off[i], ok ? (const void *)(xrow + src_off[i]) : (const void *)ximg, ok);
+                }
             }
         }
         cp_async_commit();  // (a group per row, also when it is empty: the wait below counts groups)
@@ -545,7 +558,7 @@ __device__ __forceinline__ void dw_walk_body(const ConvArgs &a, const int n, uns
     cp_async_wait<0>();
 }
 template <int K, int ACT, bool GROUP>
-__global__ void __launch_bounds__(128) dw_walk_kernel(const ConvArgs a1, const char *__restrict__ tbl, int n_img, int chblocks) {
+__global__ void __launch_bounds__(128, K == 7 ? 3 : 4) dw_walk_kernel(const ConvArgs a1, const char *__restrict__ tbl, int n_img, int chblocks) {
     __shared__ __align__(16) unsigned char smem[DwWalkShape<K>::SMEM];
     SGS_DW_ARGS()
     if (GROUP) { const ConvArgs al = a; dw_walk_body<K, ACT>(al, n, smem, chblocks); }

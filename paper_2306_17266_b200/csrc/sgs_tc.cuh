@@ -30,6 +30,11 @@ struct TcParams {
     int cacheK, cacheC, weight_policy;
     const int *cache_tbl;    // optional device table overriding the three values above (see ConvArgs)
     int layer;
+    // int8 layers (8-bit operands, int32 accumulator): per-filter requantisation parameters and the integer epilogue
+    //   v = rshift_round(acc * q_mult[f], 31 + q_shift[f]) + q_bias[f] + rshift_round((res - q_zr) * q_res_mult, 31 + q_res_shift) + q_zy
+    const int *q_mult, *q_shift, *q_bias;
+    int q_zy, q_zr, q_res_mult, q_res_shift;
+    int q_flags;             // bit 0: x signed, bit 1: y signed, bit 2: res signed, bit 3: ReLU (max with q_zy)
 };
 
 namespace {
@@ -139,6 +144,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint
         ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// 8-bit operands (signedness in the instruction descriptor), int32 accumulator; K = 32 per instruction
+__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint64_t *bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -196,8 +210,12 @@ __device__ __forceinline__ void finish_store(float *o, const __nv_bfloat16 *res,
 
 }  // namespace
 
+// Rounding right shift of the integer epilogue: floor((v + 2^(s-1)) / 2^s), 1 <= s <= 62 (ties go up).
+__host__ __device__ __forceinline__ long long rshift_round(long long v, int s) { return (v + (1ll << (s - 1))) >> s; }
+
 struct TcConvPlan {
     TcParams prm;
+    int i8 = 0;          // 8-bit operands: 128 channels per stage, 32 per MMA
     dim3 grid;
     int bn_tile = 128;   // filters per tile
     int swap = 0;        // grouped launches only: filters on the MMA's row side, all pixels on the column side

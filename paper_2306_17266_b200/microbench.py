@@ -2,6 +2,7 @@
 
     python -m paper_2306_17266_b200.microbench conv --preset resnet_b1
     python -m paper_2306_17266_b200.microbench conv --shape 1,7,7,720,720,720,720,3,3,1 --once 3
+    python -m paper_2306_17266_b200.microbench conv-i8 --preset resnet_b16
     python -m paper_2306_17266_b200.microbench dw --preset large
 
 conv shapes: N,H,W,Cmax,C,Kmax,K,R,k,stride; dw shapes: N,H,W,K,k,stride (stored kernel 7x7).
@@ -75,6 +76,46 @@ def bench_conv(shape, iters=200, once=0, split_off=0, impl=2):
     return {"shape": shape, "us": us, "tflops": flops / us / 1e6, "gbs": nbytes / us / 1e3}
 
 
+def bench_conv_i8(shape, iters=200):
+    """The same layer shapes with 8-bit operands (sgs_conv2d_sliced_i8); channel counts are rounded up to 16."""
+    N, H, W, Cmax, C, Kmax, K, R, k, stride = shape
+    r16 = lambda v: (v + 15) // 16 * 16
+    Cmax, C = r16(Cmax), r16(C)
+    p = (k - 1) // 2
+    Ho, Wo = (H + 2 * p - k) // stride + 1, (W + 2 * p - k) // stride + 1
+    x = torch.randint(0, 256, (N, H, W, C), device="cuda", dtype=torch.uint8)
+    w = torch.randint(-127, 128, (Kmax, R, R, Cmax), device="cuda", dtype=torch.int8)
+    mult = torch.full((Kmax,), 1 << 30, device="cuda", dtype=torch.int32)
+    shift = torch.full((Kmax,), 12, device="cuda", dtype=torch.int32)
+    bias = torch.zeros(Kmax, device="cuda", dtype=torch.int32)
+    y = torch.empty(N, Ho, Wo, K, device="cuda", dtype=torch.uint8)
+    d = sgs.ConvI8Desc(N=N, H=H, W=W, C=C, K=K, Kmax=Kmax, Cmax=Cmax, R=R, k=k, stride=stride, relu=1)
+    st = torch.cuda.Stream()
+
+    def launch(stream):
+        sgs.conv2d_sliced_i8(d, x.data_ptr(), w.data_ptr(), mult.data_ptr(), shift.data_ptr(), bias.data_ptr(), 0, y.data_ptr(), stream)
+
+    with torch.cuda.stream(st):
+        for _ in range(3):
+            launch(st.cuda_stream)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        for _ in range(iters):
+            launch(st.cuda_stream)
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1000 / iters
+    ops = 2.0 * N * Ho * Wo * K * C * k * k
+    nbytes = 1.0 * (N * H * W * C + N * Ho * Wo * K + K * C * k * k)
+    return {"shape": (N, H, W, Cmax, C, Kmax, K, R, k, stride), "us": us, "tops": ops / us / 1e6, "gbs": nbytes / us / 1e3}
+
+
 def bench_dw(shape, iters=20, once=0):
     N, H, W, K, k, stride = shape
     p = (k - 1) // 2
@@ -137,7 +178,7 @@ def wave_trace(family, wave, queries, res, batch):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["conv", "dw", "trace"])
+    ap.add_argument("kind", choices=["conv", "conv-i8", "dw", "trace"])
     ap.add_argument("--family", default="resnet", choices=["resnet", "mbv3"])
     ap.add_argument("--wave", type=int, default=32)
     ap.add_argument("--queries", type=int, default=128)
@@ -154,10 +195,14 @@ def main():
     if args.shape:
         shapes = [tuple(int(v) for v in args.shape.split(","))]
     else:
-        table = CONV_PRESETS if args.kind == "conv" else DW_PRESETS
-        shapes = table[args.preset or ("resnet_b1" if args.kind == "conv" else "large")]
+        table = DW_PRESETS if args.kind == "dw" else CONV_PRESETS
+        shapes = table[args.preset or ("large" if args.kind == "dw" else "resnet_b1")]
     for sh in shapes:
-        if args.kind == "conv":
+        if args.kind == "conv-i8":
+            r = bench_conv_i8(sh)
+            sh = r["shape"]
+            print(f"conv-i8 N{sh[0]} {sh[1]}x{sh[2]} C{sh[4]} K{sh[6]} k{sh[8]} s{sh[9]}: {r['us']:8.2f} us  {r['tops']:8.2f} TOP/s  {r['gbs']:8.1f} GB/s", flush=True)
+        elif args.kind == "conv":
             r = bench_conv(sh, once=args.once, split_off=args.split_off)
             if r:
                 print(f"conv N{sh[0]} {sh[1]}x{sh[2]} C{sh[4]} K{sh[6]} k{sh[8]} s{sh[9]}: {r['us']:8.2f} us  {r['tflops']:8.2f} TFLOP/s  {r['gbs']:8.1f} GB/s", flush=True)

@@ -459,3 +459,71 @@ def test_linear_and_squeeze_excite_layers_against_plain_formulas():
     x = rng.standard_normal((2, 3, 5, mid)).astype(np.float32)
     np.testing.assert_allclose(oracle.layer_se_scale(x, got), x.astype(np.float64) * got[:, None, None, :], rtol=1e-6, atol=0)
     np.testing.assert_array_equal(oracle.layer_se_scale(x, got, oracle.BF16_STORE), wl.round_to_bf16(oracle.layer_se_scale(x, got)))
+
+
+def _i8_case(rng, N, H, W, Cmax, C, Kmax, K, R, x_signed):
+    w = rng.integers(-127, 128, (Kmax, Cmax, R, R), dtype=np.int64).astype(np.int8)
+    x = (rng.integers(-128, 128, (N, H, W, C)) if x_signed else rng.integers(0, 256, (N, H, W, C)))
+    x = x.astype(np.int8 if x_signed else np.uint8)
+    mult = rng.integers(1 << 29, (1 << 31) - 1, Kmax, dtype=np.int64).astype(np.int32)
+    shift = rng.integers(6, 12, Kmax).astype(np.int32)
+    bias = rng.integers(-40, 40, Kmax).astype(np.int32)
+    return w, x, mult, shift, bias
+
+
+def test_int8_layer_against_big_integer_arithmetic():
+    # the 8-bit layer of the paper's numeric format, restated with numpy int64 sums on Python slices and Python's
+    # unbounded integers for the requantisation (floor division, so the rounding rule is explicit): zero padding
+    # counts as the real value 0 (= the zero point), slices are prefixes / centre windows, ties of the rounding
+    # shift go up, ReLU is a maximum with the output zero point, results saturate
+    rng = np.random.default_rng(8)
+    for (N, H, W, Cmax, C, Kmax, K, R, k, st, xs, zx, zy, relu, ys, use_res) in [
+            (1, 5, 6, 16, 16, 8, 8, 3, 3, 1, False, 0, 0, True, False, False),
+            (2, 7, 5, 32, 16, 16, 8, 7, 5, 2, False, 3, 10, False, False, True),
+            (1, 6, 6, 16, 16, 16, 16, 3, 1, 1, True, -5, -7, True, True, True),
+            (1, 4, 4, 48, 32, 24, 16, 3, 3, 2, True, 0, 4, False, True, False)]:
+        w, x, mult, shift, bias = _i8_case(rng, N, H, W, Cmax, C, Kmax, K, R, xs)
+        p, o = (k - 1) // 2, (R - k) // 2
+        Ho, Wo = (H + 2 * p - k) // st + 1, (W + 2 * p - k) // st + 1
+        res = None
+        zr, rm, rs = 2, 1518500250, 1   # about 0.354
+        if use_res:
+            res = rng.integers(0, 256, (N, Ho, Wo, K)).astype(np.uint8)
+        got = oracle.layer_conv_i8(w, x, C, K, k, st, mult, shift, bias, zx=zx, zy=zy, relu=relu, res=res, zr=zr, res_mult=rm, res_shift=rs, y_signed=ys)
+        xp = np.zeros((N, H + 2 * p, W + 2 * p, C), dtype=np.int64)
+        xp[:, p:p + H, p:p + W, :] = x.astype(np.int64) - zx
+        wk = w[:K, :C, o:o + k, o:o + k].astype(np.int64)
+        for n in range(N):
+            for ho in range(Ho):
+                for wo in range(Wo):
+                    win = xp[n, ho * st:ho * st + k, wo * st:wo * st + k, :]          # [k][k][C]
+                    acc = np.einsum("rsc,fcrs->f", win, wk)
+                    for f in range(K):
+                        s = 31 + int(shift[f])
+                        t = (int(acc[f]) * int(mult[f]) + (1 << (s - 1))) // (1 << s) + int(bias[f])
+                        if use_res:
+                            t += ((int(res[n, ho, wo, f]) - zr) * rm + (1 << (31 + rs - 1))) // (1 << (31 + rs))
+                        t += zy
+                        if relu:
+                            t = max(t, zy)
+                        t = min(max(t, -128 if ys else 0), 127 if ys else 255)
+                        assert int(got[n, ho, wo, f]) == t, (n, ho, wo, f)
+
+
+def test_int8_layer_invariants():
+    rng = np.random.default_rng(9)
+    w, x, mult, shift, bias = _i8_case(rng, 1, 6, 6, 32, 32, 16, 16, 3, False)
+    x = (x // 2).astype(np.uint8)          # 0..127, so that a shifted copy still fits a byte
+    base = oracle.layer_conv_i8(w, x, 32, 16, 3, 1, mult, shift, bias, zx=0, zy=5)
+    # a tensor and its zero point moved together describe the same real values, also next to the zero padding
+    moved = oracle.layer_conv_i8(w, (x + 100).astype(np.uint8), 32, 16, 3, 1, mult, shift, bias, zx=100, zy=5)
+    np.testing.assert_array_equal(moved, base)
+    # the same numbers read as signed bytes give the same result
+    np.testing.assert_array_equal(oracle.layer_conv_i8(w, x.astype(np.int8), 32, 16, 3, 1, mult, shift, bias, zx=0, zy=5), base)
+    # multiplier 2^30 with shift s is a division by 2^(s+1), ties up: checked on a 1x1 layer with unit weights
+    w1 = np.zeros((8, 16, 1, 1), dtype=np.int8)
+    w1[np.arange(8), np.arange(8)] = 1
+    xv = np.zeros((1, 1, 8, 16), dtype=np.int8)
+    xv[0, 0, :, :8] = np.array([[-5, -3, -2, -1, 1, 2, 3, 5]] * 8, dtype=np.int8)
+    y = oracle.layer_conv_i8(w1, xv, 16, 8, 1, 1, np.full(8, 1 << 30), np.zeros(8), np.zeros(8), y_signed=True)
+    np.testing.assert_array_equal(y[0, 0, 0], np.array([-2, -1, -1, 0, 1, 1, 2, 3], dtype=np.int8))  # floor(v / 2 + 1 / 2)
