@@ -173,9 +173,18 @@ def measure_sweep(net, sgs, torch, stream, peaks, n_groups=1250, resolutions=(16
     return rows
 
 
+EXTRA_OPTIONS = []  # (name, value) pairs of --option: library tuning aids, applied to every SuperNet the run creates
+
+
+def apply_options(net):
+    for name, value in EXTRA_OPTIONS:
+        net.set_option(name, value)
+    return net
+
+
 def measure_mbv3(sgs, torch, stream, queries=1000, wave=32, concurrency=4, cache=1, window=4, profile=False):
     """The MobileNetV3-shaped stream (1000 queries, batch 1, 224x224, configs uniform seed 3)."""
-    net = sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16)
+    net = apply_options(sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16))
     cfgs = wl.uniform_stream(wl.MBV3, queries, seed=3)
     opts = sgs.StreamOpts(cache_enabled=cache, window_q=window, cache_budget_bytes=0, use_graphs=1, record_latency=1,
                           concurrency=concurrency, wave=wave)
@@ -238,7 +247,8 @@ def run_suite(args):
         # throughput sweep: 20k images as groups of 16 images sharing a config (4 groups = one batch of 64)
         net = sgs.SuperNet(wl.RESNET, wl.make_blob(wl.RESNET, seed=0, bf16_weights=True), sgs.SGS_BF16)
         n_groups = args.queries // 16 if args.queries != 1000 else 1250
-        rows = measure_sweep(net, sgs, torch, stream, peaks, n_groups, cache=args.cache, window=args.window, concurrency=args.concurrency)
+        rows = measure_sweep(net, sgs, torch, stream, peaks, n_groups, resolutions=(args.res,) if args.res else (160, 192, 224), cache=args.cache,
+                             window=args.window, concurrency=args.concurrency)
         out.update({"metric": "subnet_images_per_s", "unit": "images/s", "value": rows[-1]["images_per_s"], "rows": rows,
                     "config": {"workload": SWEEP_WORKLOAD + ", 20k images per resolution", "peaks": peaks}})
     elif args.suite == "sgs":
@@ -407,6 +417,8 @@ def main():
     ap.add_argument("--sweep-groups", type=int, default=1250, help="16-image groups per resolution of the sweep measured inside the default line")
     ap.add_argument("--batch", type=int, default=1, help="images per query (sgs-probe)")
     ap.add_argument("--evict-first", type=int, default=0, help="with --cache 0: mark weight loads evict-first (sgs-probe)")
+    ap.add_argument("--option", action="append", default=[], help="library tuning aid as name=value (sgs_set_option), may repeat")
+    ap.add_argument("--res", type=int, default=0, help="sweep suite: only this resolution (profiling a single launch shape)")
     ap.add_argument("--mechanism", type=int, default=0, help="sgs-probe: 0 per-tile L2 hints, 1 access-policy window per launch, 2 both")
     ap.add_argument("--budget-mb", type=int, default=0, help="sgs-probe: cache budget in MiB (0 = device maximum)")
     ap.add_argument("--family", default="resnet", choices=["resnet", "mbv3"], help="SuperNet of the sched suite")
@@ -415,6 +427,7 @@ def main():
     args = ap.parse_args()
     if args.concurrency is None:
         args.concurrency = 4 if args.wave > 0 else 16
+    EXTRA_OPTIONS.extend((o.split("=")[0], int(o.split("=")[1])) for o in args.option)
     if args.impl == "reference":
         run_reference(args)
         return
@@ -441,7 +454,7 @@ def main():
     warmup = max(3, args.warmup)
     # replicas: every rank holds the SuperNet and serves its own query stream (no data-path collective)
     blob = wl.make_blob(wl.RESNET, seed=0, bf16_weights=True)
-    net = sgs.SuperNet(wl.RESNET, blob, sgs.SGS_BF16, device=local)
+    net = apply_options(sgs.SuperNet(wl.RESNET, blob, sgs.SGS_BF16, device=local))
     from paper_2306_17266_b200 import replicas
     # N replicas serve a stream of N * nq queries (weak scaling); queries whose SubNets are close in the vector
     # encoding go to the same replica, so that each replica's SubGraph cache sees a larger common SubGraph.  Every
@@ -539,8 +552,10 @@ def main():
         # what bounds a launch: FLOP per byte that actually crosses the DRAM interface (members of a wave share the
         # weights they have in common) against the ridge of the measured peaks; per ALGORITHMIC byte when there is no
         # counter for the kernel as it stands
+        # (the counters are cold-cache, an upper bound of the traffic in the timed region, so a launch within a
+        # quarter of the ridge counts as tensor bound: the tensor fraction is then also the lower, stricter figure)
         intensity = flop_per_launch / traffic if traffic else tc["flops"] / max(1.0, tc["alg_bytes"])
-        bound = "tensor" if intensity >= ridge else "hbm"
+        bound = "tensor" if intensity >= 0.75 * ridge else "hbm"
         in_flight_gbs = sum(p["alg_bytes"] for p in prof) / (ms / args.steps * 1e-3) / 1e9
         in_flight_tf = st_lat.useful_flops / (ms / args.steps * 1e-3) / 1e12
         hbm_view = {"achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved_gbs / peaks["hbm_gbs"],

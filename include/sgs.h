@@ -451,7 +451,8 @@ sgs_status_t sgs_debug_expire_wait(unsigned limit_us, void *cuda_stream);
  * at 16-channel pixels (zeros beyond the slice), 0 = dense pixels; "cache_mechanism" how grouped launches keep the cached SubGraph in L2: 0 (default) = an evict-last
  * hint on every weight tile inside the SubGraph's box, 1 = an access-policy window on the launch (the cached filter
  * prefix of the launch's stored layer, persisting; the persisting-L2 carve-out of the process is sized to the cache
- * budget), 2 = both; "drop_plans" forgets every cached plan (measuring what a never-seen config costs); "profile" see
+ * budget), 2 = both; "dw_walk" N = stride-1 depthwise launches of at least N million output
+ * elements take the walking kernel (default 48; 0 never, negative always; process-wide); "drop_plans" forgets every cached plan (measuring what a never-seen config costs); "profile" see
  * sgs_profile_read; "stage_group" 0 = default, 1..4 = pipeline stages that
  * share one barrier pair in the grouped convolution kernel (process-wide, a tuning aid).  Unknown name -> SGS_EINVAL. */
 sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long value);

@@ -2230,7 +2230,7 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
         return SGS_OK;
     }
     if (n == "dw_walk") {  // tuning aid (process-wide)
-        dw_set_walk(value != 0);
+        dw_set_walk((int)value);
         return SGS_OK;
     }
     if (n == "stage_group") {  // tuning aid: stages per barrier pair of the grouped convolution kernel (0 = default)

@@ -160,7 +160,7 @@ cudaError_t launch_small(int kind, const SmallEntry *h, const SmallEntry *d, int
 // and take the vectorised bf16 kernels (kernel sizes 3, 5, 7 may be mixed); otherwise cudaErrorNotSupported and
 // nothing is launched.
 constexpr int DW_ENTRY_BYTES = 256;
-void dw_set_walk(int on);  // tuning aid: 0 = stride-1 depthwise layers on the patch / row kernels instead of the walking kernel
+void dw_set_walk(int min_million_elements);  // tuning aid: stride-1 depthwise launches of at least this many million outputs take the walking kernel (0 = never)
 cudaError_t launch_dw_group(const char *h_tbl, const char *d_tbl, int members, cudaStream_t st);
 // Stem weights for the window view: dst[f][r][px * 8 + c] = src[f][r][px][c] (px < k, c < 3), else 0; dst [K][k][64].
 cudaError_t launch_stem_window_weights(const void *src, void *dst, int K, int k, cudaStream_t st);

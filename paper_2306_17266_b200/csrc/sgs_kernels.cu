@@ -575,23 +575,27 @@ static dim3 dw_walk_grid(const ConvArgs &a, int kmax, int TW, int images) {
 // covers the largest member; blocks beyond a member's own extent leave at once.
 // Stride 1: the walking bodies on the walking kernel's grid (sized for strips of 2 columns and the widest member);
 // stride 2: the patch / row bodies on their grid.
-template <int ST, int ACT> __device__ __forceinline__ void dw_mixed_dispatch(const ConvArgs &a, const int n, unsigned char *wsm, int chblocks);
-template <int ST, int ACT>
+template <int ST, int ACT, bool WALK> __device__ __forceinline__ void dw_mixed_dispatch(const ConvArgs &a, const int n, unsigned char *wsm, int chblocks);
+template <int ST, int ACT, bool WALK>
 __global__ void __launch_bounds__(128, 3) dw_mixed_kernel(const char *__restrict__ tbl, int n_img, int chblocks) {
     constexpr bool GROUP = true;
-    __shared__ __align__(16) unsigned char wsm[ST == 1 ? DwWalkShape<7>::SMEM : 16];  // (7x7 needs the most; 5x5: 37376, 3x3: 41472 bytes)
+    __shared__ __align__(16) unsigned char wsm[WALK ? DwWalkShape<7>::SMEM : 16];  // (7x7 needs the most; 5x5: 37376, 3x3: 41472 bytes)
     static_assert(DwWalkShape<7>::SMEM >= DwWalkShape<5>::SMEM && DwWalkShape<7>::SMEM >= DwWalkShape<3>::SMEM && DwWalkShape<7>::SMEM <= 48 * 1024, "ring sizes");
     const ConvArgs a1 = ConvArgs();
     SGS_DW_ARGS()
     const ConvArgs al = a;  // (a copy in registers: reading the fields from shared memory at every use costs the tiled bodies 100 registers more)
-    dw_mixed_dispatch<ST, ACT>(al, n, wsm, chblocks);
+    dw_mixed_dispatch<ST, ACT, WALK>(al, n, wsm, chblocks);
 }
-template <int ST, int ACT>
+template <int ST, int ACT, bool WALK>
 __device__ __forceinline__ void dw_mixed_dispatch(const ConvArgs &a, const int n, unsigned char *wsm, int chblocks) {
-    if (ST == 1) {
+    if (WALK) {
         if (a.k == 3) dw_walk_body<3, ACT>(a, n, wsm, chblocks);
         else if (a.k == 5) dw_walk_body<5, ACT>(a, n, wsm, chblocks);
         else dw_walk_body<7, ACT>(a, n, wsm, chblocks);
+    } else if (ST == 1) {
+        if (a.k == 3) dw_tile_body<3, 1, 2, 4, true, ACT>(a, n);
+        else if (a.k == 5) dw_tile_body<5, 1, 1, 4, true, ACT>(a, n);
+        else dw_vec_body<7, 1>(a, n);
     } else {
         if (a.k == 3) dw_tile_body<3, 2, 1, 4, false, ACT>(a, n);
         else if (a.k == 5) dw_vec_body<5, 2>(a, n);
@@ -636,19 +640,29 @@ static bool dw_vec_eligible(const ConvArgs &a) {
            ((reinterpret_cast<uintptr_t>(a.scale) | reinterpret_cast<uintptr_t>(a.shift)) & 15) == 0;
 }
 
-static int g_dw_walk = 1;  // tuning aid: 0 = the patch / row kernels also for stride 1
-void dw_set_walk(int on) { g_dw_walk = on; }
+// Stride-1 layers take the walking kernel when the launch is large: at least this many million output elements over
+// all images and members, on maps at least 28 wide.  A block walks up to 56 rows one after the other, which pays on
+// working sets that stream from HBM (64 x 56 x 56 x 480: +6 % for 3x3, +13 % for 7x7 over the patch / row kernels) and
+// loses on the small launches of batch-1 waves (MobileNetV3-shaped stream: 34.7k queries/s without it, 32.3k with it
+// everywhere), where the patch kernels' many short threads win.  0 = never, negative = always; tuning aid.
+static int g_dw_walk_min_melems = 48;
+void dw_set_walk(int min_million_elements) { g_dw_walk_min_melems = min_million_elements; }
+static bool dw_walks(const ConvArgs &a, int kmax, int members) {
+    if (g_dw_walk_min_melems < 0) return true;  // (tests: every stride-1 shape through the walking kernel)
+    return g_dw_walk_min_melems > 0 && a.Wo >= 28 &&
+           (long long)a.N * members * a.Ho * a.Wo * kmax >= (long long)g_dw_walk_min_melems * 1000000ll;
+}
 
 // The vectorised bf16 kernel of a (kernel size, stride) pair; measured on working sets beyond L2
 // (N64 56x56 C480) the tiled kernel wins for k3 and for k5 stride 1.
 template <bool GROUP>
 static cudaError_t launch_dw_bf16(const ConvArgs &a, int kmax, const char *tbl, int members, cudaStream_t st) {
     switch (a.k * 10 + a.stride) {
-    case 31: return g_dw_walk ? launch_dw_walk<3, GROUP>(a, kmax, tbl, members, st) : launch_dw_tile<3, 1, 2, 4, true, GROUP>(a, kmax, tbl, members, st);
+    case 31: return dw_walks(a, kmax, GROUP ? members : 1) ? launch_dw_walk<3, GROUP>(a, kmax, tbl, members, st) : launch_dw_tile<3, 1, 2, 4, true, GROUP>(a, kmax, tbl, members, st);
     case 32: return launch_dw_tile<3, 2, 1, 4, false, GROUP>(a, kmax, tbl, members, st);
-    case 51: return g_dw_walk ? launch_dw_walk<5, GROUP>(a, kmax, tbl, members, st) : launch_dw_tile<5, 1, 1, 4, true, GROUP>(a, kmax, tbl, members, st);
+    case 51: return dw_walks(a, kmax, GROUP ? members : 1) ? launch_dw_walk<5, GROUP>(a, kmax, tbl, members, st) : launch_dw_tile<5, 1, 1, 4, true, GROUP>(a, kmax, tbl, members, st);
     case 52: return launch_dw_vec<5, 2, GROUP>(a, kmax, tbl, members, st);
-    case 71: return g_dw_walk ? launch_dw_walk<7, GROUP>(a, kmax, tbl, members, st) : launch_dw_vec<7, 1, GROUP>(a, kmax, tbl, members, st);
+    case 71: return dw_walks(a, kmax, GROUP ? members : 1) ? launch_dw_walk<7, GROUP>(a, kmax, tbl, members, st) : launch_dw_vec<7, 1, GROUP>(a, kmax, tbl, members, st);
     case 72: return launch_dw_vec<7, 2, GROUP>(a, kmax, tbl, members, st);
     default: return cudaErrorNotSupported;
     }
@@ -672,16 +686,23 @@ cudaError_t launch_dw_group(const char *h_tbl, const char *d_tbl, int members, c
     // (same input size and stride, odd kernels with padding (k - 1) / 2: every member has the same output size)
     const int per_row = ((a0.Wo + 3) / 4) * (kmax / 8);
     const int chblocks = (kmax / 4 + 31) / 32;
-    if (a0.stride == 1) {
+    if (a0.stride == 1 && dw_walks(a0, kmax, members)) {
         const dim3 grid = dw_walk_grid(a0, kmax, 2, a0.N * members);
-        if (a0.act == ACT_RELU) dw_mixed_kernel<1, ACT_RELU><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
-        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<1, ACT_HSWISH><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
-        else dw_mixed_kernel<1, ACT_NONE><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        if (a0.act == ACT_RELU) dw_mixed_kernel<1, ACT_RELU, true><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<1, ACT_HSWISH, true><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else dw_mixed_kernel<1, ACT_NONE, true><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+    } else if (a0.stride == 1) {
+        // (the patch bodies of 3x3 and 5x5 own 2 resp. 1 output rows per block row: the grid covers single rows,
+        // blocks beyond a member's own extent leave at once)
+        dim3 grid((per_row + 127) / 128, a0.Ho, a0.N * members);
+        if (a0.act == ACT_RELU) dw_mixed_kernel<1, ACT_RELU, false><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<1, ACT_HSWISH, false><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else dw_mixed_kernel<1, ACT_NONE, false><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
     } else {
         dim3 grid((per_row + 127) / 128, a0.Ho, a0.N * members);
-        if (a0.act == ACT_RELU) dw_mixed_kernel<2, ACT_RELU><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
-        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<2, ACT_HSWISH><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
-        else dw_mixed_kernel<2, ACT_NONE><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        if (a0.act == ACT_RELU) dw_mixed_kernel<2, ACT_RELU, false><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else if (a0.act == ACT_HSWISH) dw_mixed_kernel<2, ACT_HSWISH, false><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
+        else dw_mixed_kernel<2, ACT_NONE, false><<<grid, 128, 0, st>>>(d_tbl, a0.N, chblocks);
     }
     return cudaGetLastError();
 }

@@ -111,3 +111,21 @@ def test_shapes_the_tensor_core_kernel_refuses():
 def test_depthwise(k, stride):
     run_case(2, 28, 28, 1, 1, 144, 120, 7, k, stride, 2, False, impl=0, seed=5, depthwise=True)
     run_case(1, 15, 13, 1, 1, 96, 72, 7, k, stride, 1, False, impl=0, seed=6, depthwise=True)
+
+
+@pytest.mark.parametrize("k", [3, 5, 7])
+def test_depthwise_walking_kernel(k):
+    # stride-1 launches of 48 M outputs and more walk down the image behind a shared-memory ring of input rows; the
+    # library option makes every stride-1 shape take that kernel: ragged column tiles, maps shorter than the ring, more
+    # rows than a 56-row segment (two segments with their halo rows), channel counts off the 128-channel block
+    from tests import gpu_util as gu
+    from paper_2306_17266_b200 import workload as wl
+    _, _, net = gu.nets(wl.TINY, True)
+    net.set_option("dw_walk", -1)
+    try:
+        run_case(2, 28, 28, 1, 1, 144, 120, 7, k, 1, 2, False, impl=0, seed=5, depthwise=True)
+        run_case(1, 15, 13, 1, 1, 96, 72, 7, k, 1, 1, False, impl=0, seed=6, depthwise=True)
+        run_case(1, 61, 37, 1, 1, 264, 264, 7, k, 1, 0, False, impl=0, seed=7, depthwise=True)
+        run_case(1, 4, 5, 1, 1, 16, 8, 7, k, 1, 2, False, impl=0, seed=8, depthwise=True)
+    finally:
+        net.set_option("dw_walk", 48)
