@@ -452,7 +452,9 @@ sgs_status_t sgs_debug_expire_wait(unsigned limit_us, void *cuda_stream);
  * hint on every weight tile inside the SubGraph's box, 1 = an access-policy window on the launch (the cached filter
  * prefix of the launch's stored layer, persisting; the persisting-L2 carve-out of the process is sized to the cache
  * budget), 2 = both; "dw_walk" N = stride-1 depthwise launches of at least N million output
- * elements take the walking kernel (default 48; 0 never, negative always; process-wide); "drop_plans" forgets every cached plan (measuring what a never-seen config costs); "profile" see
+ * elements take the walking kernel (default 48; 0 never, negative always; process-wide); "nvtx" 1 = an NVTX range named after the stored layer around
+ * every launch (for timeline tools); "fail_alloc_after" n = the handle's device allocations fail from
+ * the (n+1)-th on with SGS_ENOMEM (fault injection on the host, -1 = off); "drop_plans" forgets every cached plan (measuring what a never-seen config costs); "profile" see
  * sgs_profile_read; "stage_group" 0 = default, 1..4 = pipeline stages that
  * share one barrier pair in the grouped convolution kernel (process-wide, a tuning aid).  Unknown name -> SGS_EINVAL. */
 sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long value);

@@ -10,6 +10,11 @@
 #include <deque>
 #include <map>
 #include <chrono>
+#include <nvtx3/nvToolsExt.h>
+#include <condition_variable>
+#include <functional>
+#include <mutex>
+#include <thread>
 
 using namespace sgs;
 
@@ -214,6 +219,8 @@ struct sgs_supernet {
     int plan_hits = 0, plan_misses = 0;
     int force_plain = 0;
     size_t persist_limit_set = 0;  // cudaLimitPersistingL2CacheSize as last set by this handle
+    int nvtx = 0;  // 1: NVTX ranges named after the stored layer around every launch
+    long long fail_alloc_after = -1;  // < 0: off; else device allocations left before they start failing (test aid)
     int cache_mech = 0;    // how grouped launches keep the cached SubGraph in L2: 0 per-tile hints, 1 access-policy window of the launch, 2 both
     int pad_channels = 1;  // waves of the ResNet-shaped family keep activation pixels at multiples of 16 channels
     int throughput_mode = 0;  // set by streams that keep many queries in flight; part of the plan key
@@ -247,7 +254,17 @@ sgs_status_t fail(const sgs_supernet *n, sgs_status_t st, const std::string &msg
     } while (0)
 
 sgs_status_t dev_alloc(sgs_supernet *net, void **p, size_t bytes) {
-    CU(cudaMalloc(p, bytes));
+    // (fault injection on the host, option "fail_alloc_after": the n-th allocation from now on and every later one fail)
+    if (net->fail_alloc_after >= 0 && net->fail_alloc_after-- == 0) {
+        net->fail_alloc_after = 0;
+        *p = nullptr;
+        return fail(net, SGS_ENOMEM, "device allocation failed (injected)");
+    }
+    if (cudaMalloc(p, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        *p = nullptr;
+        return fail(net, SGS_ENOMEM, "device allocation of " + std::to_string(bytes) + " bytes failed");
+    }
     net->device_bytes += bytes;
     return SGS_OK;
 }
@@ -564,6 +581,13 @@ sgs_status_t build_plan(sgs_supernet *net, const sgs_subnet_cfg_t *cfg, int batc
 }
 
 // Makes sure `n_slots` slots exist, each with buffers for the sizes in use.
+// Frees the activation / vector / split-reduction buffers of a slot (the sizes are the handle's current ones).
+void release_slot_buffers(sgs_supernet *net, sgs_supernet::Slot &sl, bool act, bool vec, bool ws) {
+    for (int i = 0; i < 4 && act; i++) { dev_free(net, sl.act[i], net->act_elems * net->elem() + 256); sl.act[i] = nullptr; }
+    for (int i = 0; i < 3 && vec; i++) { dev_free(net, sl.vec[i], net->vec_elems * 4); sl.vec[i] = nullptr; }
+    if (ws) { dev_free(net, sl.ws, net->splitk_ws_elems * 4); sl.ws = nullptr; }
+}
+
 sgs_status_t ensure_slots(sgs_supernet *net, int n_slots) {
     while ((int)net->slots.size() < n_slots) {
         sgs_supernet::Slot sl;
@@ -571,57 +595,62 @@ sgs_status_t ensure_slots(sgs_supernet *net, int n_slots) {
             CU(cudaStreamCreateWithFlags(&sl.st, cudaStreamNonBlocking));
             CU(cudaEventCreateWithFlags(&sl.ev, cudaEventDisableTiming));
         }
-        for (int i = 0; i < 4 && net->act_elems; i++) {
-            sgs_status_t st = dev_alloc(net, &sl.act[i], net->act_elems * net->elem() + 256);
-            if (st != SGS_OK) return st;
-        }
-        for (int i = 0; i < 3 && net->vec_elems; i++) {
-            sgs_status_t st = dev_alloc(net, (void **)&sl.vec[i], net->vec_elems * 4);
-            if (st != SGS_OK) return st;
-        }
-        if (net->splitk_ws_elems) {
-            sgs_status_t st = dev_alloc(net, (void **)&sl.ws, net->splitk_ws_elems * 4);
-            if (st != SGS_OK) return st;
+        sgs_status_t st = SGS_OK;
+        for (int i = 0; i < 4 && net->act_elems && st == SGS_OK; i++) st = dev_alloc(net, &sl.act[i], net->act_elems * net->elem() + 256);
+        for (int i = 0; i < 3 && net->vec_elems && st == SGS_OK; i++) st = dev_alloc(net, (void **)&sl.vec[i], net->vec_elems * 4);
+        if (net->splitk_ws_elems && st == SGS_OK) st = dev_alloc(net, (void **)&sl.ws, net->splitk_ws_elems * 4);
+        if (st != SGS_OK) {  // nothing of a half-built slot stays behind
+            release_slot_buffers(net, sl, true, true, true);
+            if (sl.st) cudaStreamDestroy(sl.st);
+            if (sl.ev) cudaEventDestroy(sl.ev);
+            return st;
         }
         net->slots.push_back(sl);
     }
     return SGS_OK;
 }
 
+// Grows the workspaces of every slot.  If an allocation fails, ALL slots give up the kind of buffer that was being
+// grown and the handle's size for it returns to zero, so that the next call starts from a consistent state (no slot
+// is ever left with a missing or a smaller buffer than the handle believes).
 sgs_status_t ensure_workspace(sgs_supernet *net, size_t act_elems, int batch) {
     if (net->slots.empty()) { sgs_status_t st = ensure_slots(net, 1); if (st != SGS_OK) return st; }
     if (act_elems > net->act_elems) {
         drop_graphs(net);
         for (auto &kv : net->plans) kv.second->prepared = false;
-        for (auto &sl : net->slots) {
-            for (int i = 0; i < 4; i++) {
-                dev_free(net, sl.act[i], net->act_elems * net->elem() + 256);
-                sl.act[i] = nullptr;
-                sgs_status_t st = dev_alloc(net, &sl.act[i], act_elems * net->elem() + 256);
-                if (st != SGS_OK) return st;
-            }
-        }
+        for (auto &sl : net->slots) release_slot_buffers(net, sl, true, false, false);
         net->act_elems = act_elems;
+        sgs_status_t st = SGS_OK;
+        for (auto &sl : net->slots)
+            for (int i = 0; i < 4 && st == SGS_OK; i++) st = dev_alloc(net, &sl.act[i], act_elems * net->elem() + 256);
+        if (st != SGS_OK) {
+            for (auto &sl : net->slots) release_slot_buffers(net, sl, true, false, false);
+            net->act_elems = 0;
+            return st;
+        }
     }
     size_t vneed = (size_t)batch * 2048;
     if (vneed > net->vec_elems) {
         drop_graphs(net);
-        for (auto &sl : net->slots) {
-            for (int i = 0; i < 3; i++) {
-                dev_free(net, sl.vec[i], net->vec_elems * 4);
-                sl.vec[i] = nullptr;
-                sgs_status_t st = dev_alloc(net, (void **)&sl.vec[i], vneed * 4);
-                if (st != SGS_OK) return st;
-            }
-        }
+        for (auto &sl : net->slots) release_slot_buffers(net, sl, false, true, false);
         net->vec_elems = vneed;
+        sgs_status_t st = SGS_OK;
+        for (auto &sl : net->slots)
+            for (int i = 0; i < 3 && st == SGS_OK; i++) st = dev_alloc(net, (void **)&sl.vec[i], vneed * 4);
+        if (st != SGS_OK) {
+            for (auto &sl : net->slots) release_slot_buffers(net, sl, false, true, false);
+            net->vec_elems = 0;
+            return st;
+        }
     }
     return SGS_OK;
 }
 
 // Chooses the implementation of every convolution of a plan and fixes its buffer addresses (the
 // tensor maps of the tensor-core kernel hold absolute addresses of the activation workspaces).
-sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
+// prepare_impls touches nothing but the plan (several plans may be prepared at the same time by different threads);
+// choose_impls = prepare + the part that may grow the handle's split-reduction scratch.
+sgs_status_t prepare_impls(const sgs_supernet *net, Plan *plan, size_t *ws_need_out, std::string *err) {
     size_t ws_need = 0;
     for (Op &op : plan->ops) {
         if (op.type != OP_CONV && op.type != OP_DW) continue;
@@ -636,25 +665,122 @@ sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
         if (net->dtype != SGS_BF16 || net->force_plain || !tc_available()) continue;
         std::string why;
         op.tc = tc_conv_prepare(op.conv, net->device, &why);
-        if (!op.tc && op.conv.win) return fail(net, SGS_EUNSUPPORTED, "window view of the stem: " + why);
-        if (!op.tc && plan->padded) return fail(net, SGS_EUNSUPPORTED, "padded activation layout needs the tensor-core kernel: " + why);
+        if (!op.tc && op.conv.win) { *err = "window view of the stem: " + why; return SGS_EUNSUPPORTED; }
+        if (!op.tc && plan->padded) { *err = "padded activation layout needs the tensor-core kernel: " + why; return SGS_EUNSUPPORTED; }
         if (op.tc) {
             op.impl = 1;
             ws_need = std::max(ws_need, tc_conv_ws_elems(*op.tc));
         }
     }
+    *ws_need_out = ws_need;
+    return SGS_OK;
+}
+
+sgs_status_t grow_splitk_scratch(sgs_supernet *net, size_t ws_need) {
     if (ws_need > net->splitk_ws_elems) {
         drop_graphs(net);
-        for (auto &sl : net->slots) {
-            dev_free(net, sl.ws, net->splitk_ws_elems * 4);  // cudaFree waits for work in flight
-            sl.ws = nullptr;
-            sgs_status_t st = dev_alloc(net, (void **)&sl.ws, ws_need * 4);
-            if (st != SGS_OK) return st;
-        }
+        for (auto &sl : net->slots) release_slot_buffers(net, sl, false, false, true);  // (cudaFree waits for work in flight)
         net->splitk_ws_elems = ws_need;
+        sgs_status_t st = SGS_OK;
+        for (auto &sl : net->slots)
+            if (st == SGS_OK) st = dev_alloc(net, (void **)&sl.ws, ws_need * 4);
+        if (st != SGS_OK) {
+            for (auto &sl : net->slots) release_slot_buffers(net, sl, false, false, true);
+            net->splitk_ws_elems = 0;
+            for (auto &kv : net->plans) kv.second->prepared = false;  // (plans that counted on the scratch choose again)
+            return st;
+        }
     }
+    return SGS_OK;
+}
+
+sgs_status_t choose_impls(sgs_supernet *net, Plan *plan) {
+    size_t ws_need = 0;
+    std::string err;
+    sgs_status_t st = prepare_impls(net, plan, &ws_need, &err);
+    if (st != SGS_OK) return fail(net, st, err);
+    if ((st = grow_splitk_scratch(net, ws_need)) != SGS_OK) return st;
     plan->prepared = true;
     return SGS_OK;
+}
+
+// NVTX range around the launches of one layer (option "nvtx"; a no-op unless a tool that listens is attached).
+struct LayerRange {
+    bool on;
+    LayerRange(const sgs_supernet *net, int layer, const char *what) : on(net->nvtx != 0) {
+        if (!on) return;
+        const std::string name = layer >= 0 && layer < (int)net->layers.size() ? net->layers[(size_t)layer].name : std::string(what);
+        nvtxRangePushA(name.c_str());
+    }
+    ~LayerRange() { if (on) nvtxRangePop(); }
+    LayerRange(const LayerRange &) = delete;
+    LayerRange &operator=(const LayerRange &) = delete;
+};
+
+// A few host threads for work that is independent per wave member (planning a never-seen SubNet is ~55 convolutions
+// x 2 - 5 tensor maps encoded by the driver, 60 - 70 us on one thread).  parallel_for runs fn(0 .. n-1) on the calling
+// thread and the workers and returns when all are done.
+class HostPool {
+public:
+    explicit HostPool(int workers) {
+        for (int i = 0; i < workers; i++) threads_.emplace_back([this] { work(); });
+    }
+    ~HostPool() {
+        { std::lock_guard<std::mutex> lk(mu_); stop_ = true; }
+        cv_.notify_all();
+        for (auto &t : threads_) t.join();
+    }
+    void parallel_for(int n, const std::function<void(int)> &fn) {
+        if (n <= 0) return;
+        {
+            std::lock_guard<std::mutex> lk(mu_);
+            fn_ = &fn; n_ = n; next_ = 0; pending_ = n; ++epoch_;
+        }
+        cv_.notify_all();
+        run();
+        std::unique_lock<std::mutex> lk(mu_);
+        done_.wait(lk, [this] { return pending_ == 0; });
+        fn_ = nullptr;
+    }
+private:
+    void run() {
+        for (;;) {
+            int i;
+            const std::function<void(int)> *fn;
+            {
+                std::lock_guard<std::mutex> lk(mu_);
+                if (!fn_ || next_ >= n_) return;
+                i = next_++;
+                fn = fn_;
+            }
+            (*fn)(i);
+            std::lock_guard<std::mutex> lk(mu_);
+            if (--pending_ == 0) done_.notify_all();
+        }
+    }
+    void work() {
+        unsigned long long seen = 0;
+        for (;;) {
+            {
+                std::unique_lock<std::mutex> lk(mu_);
+                cv_.wait(lk, [&] { return stop_ || epoch_ != seen; });
+                if (stop_) return;
+                seen = epoch_;
+            }
+            run();
+        }
+    }
+    std::vector<std::thread> threads_;
+    std::mutex mu_;
+    std::condition_variable cv_, done_;
+    const std::function<void(int)> *fn_ = nullptr;
+    int n_ = 0, next_ = 0, pending_ = 0;
+    unsigned long long epoch_ = 0;
+    bool stop_ = false;
+};
+HostPool &host_pool() {
+    static HostPool pool((int)std::min(7u, std::max(1u, std::thread::hardware_concurrency()) - 1u));
+    return pool;
 }
 
 // Key of an op that is the same for every SubNet: its type and the stored layer it uses; ops without
@@ -769,6 +895,7 @@ template <typename T>
 sgs_status_t launch_op(sgs_supernet *net, Plan *plan, Op &op, const void *d_input, void *d_logits, cudaStream_t st) {
     const sgs_supernet::Slot &sl = net->slots[plan->slot];
     auto abuf = [&](int id) -> void * { return id < 0 ? const_cast<void *>(d_input) : sl.act[id]; };
+    LayerRange range(net, op.layer, "layer without weights");
     switch (op.type) {
     case OP_CONV:
     case OP_DW: {
@@ -1393,8 +1520,25 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             rc = get_plan(net, &cfgs[q0 + m], batch, res, ci * G + m, &plans[m]);
             if (rc == SGS_OK) rc = ensure_workspace(net, plans[m]->act_elems, batch);
         }
-        for (int m = 0; m < members && rc == SGS_OK; m++)
-            if (!plans[m]->prepared) rc = choose_impls(net, plans[m]);
+        {
+            // members whose plan is new: tensor maps and tile choices, prepared on a few host threads at once
+            std::vector<int> fresh;
+            for (int m = 0; m < members; m++)
+                if (!plans[m]->prepared) fresh.push_back(m);
+            if (fresh.size() == 1) {
+                rc = choose_impls(net, plans[fresh[0]]);
+            } else if (!fresh.empty()) {
+                std::vector<sgs_status_t> sts(fresh.size(), SGS_OK);
+                std::vector<size_t> need(fresh.size(), 0);
+                std::vector<std::string> errs(fresh.size());
+                // (the driver's tensor-map encoder wants the device's context current on the calling thread)
+                host_pool().parallel_for((int)fresh.size(), [&](int i) { if (cudaSetDevice(net->device) != cudaSuccess) { sts[(size_t)i] = SGS_ECUDA; errs[(size_t)i] = "cudaSetDevice on a planning thread"; return; } sts[(size_t)i] = prepare_impls(net, plans[fresh[(size_t)i]], &need[(size_t)i], &errs[(size_t)i]); });
+                for (size_t i = 0; i < fresh.size() && rc == SGS_OK; i++) {
+                    if (sts[i] != SGS_OK) rc = fail(net, sts[i], errs[i]);
+                    else if ((rc = grow_splitk_scratch(net, need[i])) == SGS_OK) plans[fresh[i]]->prepared = true;
+                }
+            }
+        }
         if (rc != SGS_OK) break;
         net->host_us_query += tick(tp);
         sgs_supernet::WaveCtx &cx = net->waves[ci];  // (taken after ensure_*: the vector does not move later)
@@ -1659,6 +1803,7 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
         void *dlog = host_buffers ? (void *)cx.stage_out : dout;
         for (const Launch &L : launches) {
             double pb = 0, pf = 0;
+            LayerRange range(net, first_layer(L.rank), "layer without weights");
             if (L.group) {
                 // (a bucket split over several launches books its whole cost on each: buckets of more than
                 // 64 members or 248 tensor maps do not occur while profiling waves of <= 64)
@@ -2214,6 +2359,14 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
             for (int i = 0; i < 4; i++) { net->prof_ms[i] = net->prof_bytes[i] = net->prof_flops[i] = 0; net->prof_launches[i] = 0; }
             net->prof_trace.clear();
         }
+        return SGS_OK;
+    }
+    if (n == "nvtx") {
+        net->nvtx = value != 0;
+        return SGS_OK;
+    }
+    if (n == "fail_alloc_after") {
+        net->fail_alloc_after = value < 0 ? -1 : value;
         return SGS_OK;
     }
     if (n == "cache_mechanism") {

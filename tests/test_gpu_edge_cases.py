@@ -108,3 +108,38 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
     got = d_out.cpu().numpy()
     for t in range(n):
         assert gu.rel_err(got[t:t + 1], onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)) <= 2e-2
+
+
+def test_device_allocation_failure_is_reported_and_survivable():
+    # fault injection on the host: the handle's device allocations are made to fail while its workspaces have to grow
+    # (a larger resolution, more wave slots).  The call must come back with SGS_ENOMEM, nothing may be left half
+    # grown, and with allocations working again the same handle must serve the same stream correctly.
+    blob = wl.make_blob(wl.RESNET, seed=0, bf16_weights=True)
+    onet = oracle.Net(wl.RESNET, blob)
+    gnet = sgs.SuperNet(wl.RESNET, blob, sgs.SGS_BF16)
+    n = 6
+    cfgs = wl.uniform_stream(wl.RESNET, n, seed=71)
+    stream = torch.cuda.Stream()
+    out = torch.zeros((n, 1000), dtype=torch.float32, device="cuda")
+
+    def run(res, wave, conc):
+        xs = wl.make_inputs(n, 1, res, seed=10, bf16=True)
+        d_in = gu.to_device(xs.reshape(n, res, res, 3), True)
+        opts = sgs.StreamOpts(cache_enabled=1, window_q=2, record_latency=0, concurrency=conc, wave=wave)
+        gnet.stream_run(cfgs, d_in.data_ptr(), 1, res, out.data_ptr(), opts, stream.cuda_stream)
+        return xs, out.cpu().numpy().copy()
+
+    run(32, 2, 1)                                   # small workspaces exist
+    for after in (0, 3, 9):                         # fail at once, and in the middle of growing several slots
+        gnet.set_option("fail_alloc_after", after)
+        with pytest.raises(sgs.SgsError) as e:
+            run(96, 3, 2)                           # larger maps and more slots: everything has to grow
+        assert e.value.status == sgs.binding.SGS_ENOMEM
+        gnet.set_option("fail_alloc_after", -1)
+        xs, got = run(64, 2, 1)                     # the handle still works ...
+        assert gu.rel_err(got[:1], onet.forward(cfgs[0], xs[0], oracle.BF16_STORE)) <= 2e-2
+    xs, got = run(96, 3, 2)                         # ... and can grow once memory is there
+    for t in (0, 5):
+        assert gu.rel_err(got[t:t + 1], onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)) <= 2e-2
+    assert sgs.device_status() == 0
+    gnet.close()
