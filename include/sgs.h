@@ -109,6 +109,12 @@ typedef struct {
                            SGS_POLICY_INTERSECTION (0): the SubGraph common to the last window_q SubNets;
                            SGS_POLICY_AVGNET (1): Algorithm 1 - the candidate SubGraph (sgs_cache_set_candidates)
                            nearest to the running average of the last window_q SubNets' encodings */
+    int persistent;     /* 1 (bf16 handles of the MobileNetV3-shaped family, one image per query): the whole stream
+                           is ONE launch of a persistent kernel; every SM takes the next unserved query and runs all
+                           layers of its SubNet by itself out of a private scratch area, pointwise convolutions on the
+                           tensor cores (Section 3.1: one query per pass of the accelerator; Section 4.2: what is needed
+                           again stays on chip).  wave, concurrency and use_graphs are ignored; every query starts and
+                           ends with the launch (its recorded latency).  Other handles: SGS_EUNSUPPORTED. */
 } sgs_stream_opts_t;
 
 /* Results of sgs_stream_run (all host-side; filled after the stream has been synchronised). */

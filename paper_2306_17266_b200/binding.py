@@ -55,7 +55,7 @@ class AuxArgs(ctypes.Structure):
 class StreamOpts(ctypes.Structure):
     _fields_ = [("cache_enabled", ctypes.c_int), ("window_q", ctypes.c_int), ("cache_budget_bytes", ctypes.c_size_t),
                 ("use_graphs", ctypes.c_int), ("record_latency", ctypes.c_int), ("weights_evict_first", ctypes.c_int),
-                ("concurrency", ctypes.c_int), ("wave", ctypes.c_int), ("policy", ctypes.c_int)]
+                ("concurrency", ctypes.c_int), ("wave", ctypes.c_int), ("policy", ctypes.c_int), ("persistent", ctypes.c_int)]
 
 
 class StreamStats(ctypes.Structure):

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libsgs.so")
-SOURCES = ["sgs_api.cu", "sgs_kernels.cu", "sgs_conv_tc.cu", "sgs_conv_group.cu"]
+SOURCES = ["sgs_api.cu", "sgs_kernels.cu", "sgs_conv_tc.cu", "sgs_conv_group.cu", "sgs_subnet_kernel.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
 
 

@@ -218,6 +218,15 @@ struct sgs_supernet {
     long long kernel_launches = 0;
     int plan_hits = 0, plan_misses = 0;
     int force_plain = 0;
+    // persistent SubNet kernel: scratch of its blocks, op / query tables (pinned host image and device copy), query counter
+    unsigned char *pq_scratch = nullptr;
+    size_t pq_scratch_bytes = 0;
+    char *pq_h_tbl = nullptr, *pq_d_tbl = nullptr;
+    size_t pq_tbl_bytes = 0;
+    int *pq_counter = nullptr;
+    void *pq_stage_in = nullptr;
+    float *pq_stage_out = nullptr;
+    size_t pq_stage_in_bytes = 0, pq_stage_out_bytes = 0;
     size_t persist_limit_set = 0;  // cudaLimitPersistingL2CacheSize as last set by this handle
     int nvtx = 0;  // 1: NVTX ranges named after the stored layer around every launch
     long long fail_alloc_after = -1;  // < 0: off; else device allocations left before they start failing (test aid)
@@ -1392,6 +1401,12 @@ void sgs_supernet_free(sgs_supernet_t *net) {
         if (w.done) cudaEventDestroy(w.done);
         if (w.st) cudaStreamDestroy(w.st);
     }
+    cudaFree(net->pq_scratch);
+    cudaFree(net->pq_d_tbl);
+    cudaFreeHost(net->pq_h_tbl);
+    cudaFree(net->pq_counter);
+    cudaFree(net->pq_stage_in);
+    cudaFree(net->pq_stage_out);
     cudaFree(net->cache_tbl);
     cudaFreeHost(net->tbl_ring);
     for (int i = 0; i < 16; i++)
@@ -1925,6 +1940,221 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
     return rc;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Persistent execution (sgs_stream_opts_t::persistent): the whole stream is one launch of the SubNet kernel.
+// ---------------------------------------------------------------------------------------------
+// The plan of a config as the op list the kernel interprets (one record per layer; the patch-matrix / padding ops
+// that the layer-by-layer paths put in front of the stem are dropped, the kernel convolves the image directly).
+static sgs_status_t build_pq_ops(sgs_supernet *net, Plan *plan) {
+    plan->pq.clear();
+    const int stem_li = net->idx("stem");
+    auto mult8 = [](int v) { return v > 0 && v % 8 == 0; };
+    for (const Op &op : plan->ops) {
+        PqOp q;
+        std::memset(&q, 0, sizeof q);
+        q.in = q.out = q.res = q.vin = q.vout = -1;
+        q.cache_off = -1;
+        switch (op.type) {
+        case OP_IM2COL:
+        case OP_PAD8: continue;
+        case OP_CONV: {
+            const StoredLayer &L = net->layers[op.layer];
+            const Slice &s = plan->slices[op.layer];
+            const ConvArgs &a = op.conv;
+            q.w = L.w; q.scale = L.scale; q.shift = L.shift; q.act = a.act; q.out = op.out;
+            q.Ho = a.Ho; q.Wo = a.Wo; q.K = s.K; q.R = L.R; q.Kmax = L.K; q.ld = L.Cp;
+            if (op.layer == stem_li) {
+                if (s.k > 3 || !mult8(s.K) || s.K > 64 || L.C != 3) return fail(net, SGS_EUNSUPPORTED, "persistent kernel: stem shape");
+                q.type = PQ_STEM; q.H = plan->res; q.W = plan->res; q.C = 3; q.k = s.k; q.stride = 2;  // (the stem of this family)
+            } else {
+                if (s.k != 1 || a.stride != 1 || !mult8(s.C) || !mult8(s.K) || s.K > 1024) return fail(net, SGS_EUNSUPPORTED, "persistent kernel: convolution shape");
+                q.type = PQ_PW; q.in = op.in; q.res = op.res; q.H = a.H; q.W = a.W; q.C = s.C; q.k = 1; q.stride = 1;
+            }
+            break;
+        }
+        case OP_DW: {
+            const StoredLayer &L = net->layers[op.layer];
+            const ConvArgs &a = op.conv;
+            if (!mult8(a.K) || (a.k != 3 && a.k != 5 && a.k != 7) || (a.stride != 1 && a.stride != 2)) return fail(net, SGS_EUNSUPPORTED, "persistent kernel: depthwise shape");
+            q.type = PQ_DW; q.in = op.in; q.out = op.out; q.H = a.H; q.W = a.W; q.Ho = a.Ho; q.Wo = a.Wo; q.C = a.K; q.K = a.K;
+            q.k = a.k; q.stride = a.stride; q.act = a.act; q.R = L.R; q.Kmax = L.K; q.ld = L.K;
+            q.w = L.w; q.scale = L.scale; q.shift = L.shift;
+            break;
+        }
+        case OP_GAP:
+            if (!mult8(op.C) || op.C > 1280) return fail(net, SGS_EUNSUPPORTED, "persistent kernel: pooled width");
+            q.type = PQ_GAP; q.in = op.in; q.vout = op.vout; q.H = op.H; q.W = op.W; q.C = op.C;
+            break;
+        case OP_SE_GATE: {
+            const StoredLayer &L1 = net->layers[op.layer], &L2 = net->layers[op.layer2];
+            if (!mult8(op.C) || !mult8(op.K) || !mult8(L1.C) || !mult8(L2.C) || op.C > 1280 || op.K > 1280) return fail(net, SGS_EUNSUPPORTED, "persistent kernel: squeeze-excite shape");
+            q.type = PQ_SE_GATE; q.vin = op.vin; q.vout = op.vout; q.C = op.C; q.K = op.K;
+            q.w = L1.w; q.ld = L1.C; q.shift = L1.shift; q.w2 = L2.w; q.ld2 = L2.C; q.bias2 = L2.shift;
+            break;
+        }
+        case OP_SCALE:
+            q.type = PQ_SCALE; q.in = op.in; q.out = op.out; q.vin = op.vin; q.H = op.H; q.W = op.W; q.C = op.C;
+            break;
+        case OP_LINEAR: {
+            const StoredLayer &L = net->layers[op.layer];
+            if (!mult8(op.C) || !mult8(L.C) || op.C > 1280 || (op.vout >= 0 && op.K > 1280)) return fail(net, SGS_EUNSUPPORTED, "persistent kernel: linear shape");
+            q.type = PQ_LINEAR; q.vin = op.vin; q.vout = op.vout; q.C = op.C; q.K = op.K; q.act = op.act;
+            q.w = L.w; q.ld = L.C; q.shift = L.shift;
+            break;
+        }
+        default: return fail(net, SGS_EUNSUPPORTED, "persistent kernel: layer type");
+        }
+        if (q.vin > 1 || q.vout > 1 || q.in > 3 || q.out > 3 || q.res > 3) return fail(net, SGS_EUNSUPPORTED, "persistent kernel: buffer id");
+        plan->pq.push_back(q);
+    }
+    return SGS_OK;
+}
+
+static sgs_status_t persistent_impl(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs, const void *inputs, int res,
+                                    void *logits, const sgs_stream_opts_t &o, sgs_stream_stats_t *stats, cudaStream_t st,
+                                    bool host_buffers) {
+    if (net->family != SGS_MBV3 || net->dtype != SGS_BF16 || !tc_available())
+        return fail(net, SGS_EUNSUPPORTED, "persistent execution serves bf16 handles of the MobileNetV3-shaped family on a tensor-core device");
+    net->throughput_mode = 0;
+    const int hits0 = net->plan_hits, miss0 = net->plan_misses;
+    const long long launches0 = net->kernel_launches;
+    const size_t in_bytes = (size_t)res * res * 3 * net->elem(), out_bytes = (size_t)net->def.classes * sizeof(float);
+    // plans and op lists (one list per distinct config of the call)
+    std::vector<Plan *> plans((size_t)n_queries);
+    std::unordered_map<Plan *, int> begin;
+    std::vector<PqOp> ops;
+    std::vector<PqQuery> qs((size_t)n_queries);
+    size_t act_elems = 0;
+    double flops = 0, wbytes = 0, miss_bytes = 0, hit = 0;
+    int updates = 0;
+    for (int t = 0; t < n_queries; t++) {
+        Plan *pl = nullptr;
+        sgs_status_t rc = get_plan(net, &cfgs[t], 1, res, 0, &pl);
+        if (rc != SGS_OK) return rc;
+        if (pl->pq.empty() && (rc = build_pq_ops(net, pl)) != SGS_OK) return rc;
+        plans[(size_t)t] = pl;
+        act_elems = std::max(act_elems, pl->act_elems);
+        auto it = begin.find(pl);
+        if (it == begin.end()) {
+            it = begin.emplace(pl, (int)ops.size()).first;
+            ops.insert(ops.end(), pl->pq.begin(), pl->pq.end());
+        }
+        PqQuery &q = qs[(size_t)t];
+        std::memset(&q, 0, sizeof q);
+        q.op_begin = it->second; q.op_count = (int)pl->pq.size();
+        const int epoch_before = net->cache.epoch;
+        QueryAccount qa = account_query(net, pl->enc);
+        flops += pl->flops; wbytes += qa.weight_bytes; miss_bytes += qa.miss_bytes; hit += qa.hit_ratio;
+        if (net->cache.enabled) {
+            cache_observe(net, pl->enc);
+            if (net->cache.epoch != epoch_before) updates++;
+        }
+    }
+    // device resources: scratch of the blocks, tables, counter, staging for host buffers
+    const int blocks_max = std::max(1, net->sms);
+    const size_t act_bytes = (act_elems * net->elem() + 255) / 256 * 256, slot_bytes = 4 * act_bytes;
+    if (net->pq_scratch_bytes < slot_bytes * blocks_max) {
+        CU(cudaStreamSynchronize(st));
+        dev_free(net, net->pq_scratch, net->pq_scratch_bytes); net->pq_scratch = nullptr; net->pq_scratch_bytes = 0;
+        sgs_status_t rc = dev_alloc(net, (void **)&net->pq_scratch, slot_bytes * blocks_max);
+        if (rc != SGS_OK) return rc;
+        net->pq_scratch_bytes = slot_bytes * blocks_max;
+    }
+    const size_t ops_bytes = ops.size() * sizeof(PqOp), q_bytes = qs.size() * sizeof(PqQuery), tbl_need = ops_bytes + q_bytes;
+    if (net->pq_tbl_bytes < tbl_need) {
+        CU(cudaStreamSynchronize(st));
+        dev_free(net, net->pq_d_tbl, net->pq_tbl_bytes); net->pq_d_tbl = nullptr;
+        cudaFreeHost(net->pq_h_tbl); net->pq_h_tbl = nullptr;
+        net->pq_tbl_bytes = 0;
+        const size_t cap = tbl_need + tbl_need / 2;
+        if (cudaMallocHost((void **)&net->pq_h_tbl, cap) != cudaSuccess) return fail(net, SGS_ENOMEM, "pinned table of the persistent kernel");
+        sgs_status_t rc = dev_alloc(net, (void **)&net->pq_d_tbl, cap);
+        if (rc != SGS_OK) { cudaFreeHost(net->pq_h_tbl); net->pq_h_tbl = nullptr; return rc; }
+        net->pq_tbl_bytes = cap;
+    }
+    if (!net->pq_counter) {
+        sgs_status_t rc = dev_alloc(net, (void **)&net->pq_counter, 256);
+        if (rc != SGS_OK) return rc;
+    }
+    if (host_buffers) {
+        const size_t need_in = in_bytes * (size_t)n_queries, need_out = out_bytes * (size_t)n_queries;
+        if (net->pq_stage_in_bytes < need_in) {
+            CU(cudaStreamSynchronize(st));
+            dev_free(net, net->pq_stage_in, net->pq_stage_in_bytes); net->pq_stage_in = nullptr; net->pq_stage_in_bytes = 0;
+            sgs_status_t rc = dev_alloc(net, &net->pq_stage_in, need_in);
+            if (rc != SGS_OK) return rc;
+            net->pq_stage_in_bytes = need_in;
+        }
+        if (net->pq_stage_out_bytes < need_out) {
+            CU(cudaStreamSynchronize(st));
+            dev_free(net, net->pq_stage_out, net->pq_stage_out_bytes); net->pq_stage_out = nullptr; net->pq_stage_out_bytes = 0;
+            sgs_status_t rc = dev_alloc(net, (void **)&net->pq_stage_out, need_out);
+            if (rc != SGS_OK) return rc;
+            net->pq_stage_out_bytes = need_out;
+        }
+    }
+    const char *din = host_buffers ? static_cast<const char *>(net->pq_stage_in) : static_cast<const char *>(inputs);
+    char *dout = host_buffers ? reinterpret_cast<char *>(net->pq_stage_out) : static_cast<char *>(logits);
+    for (int t = 0; t < n_queries; t++) {
+        qs[(size_t)t].x = din + (size_t)t * in_bytes;
+        qs[(size_t)t].logits = reinterpret_cast<float *>(dout + (size_t)t * out_bytes);
+    }
+    CU(cudaStreamSynchronize(st));  // the pinned table image may still be the source of an earlier call's copy
+    if (tbl_need) {
+        std::memcpy(net->pq_h_tbl, ops.data(), ops_bytes);
+        std::memcpy(net->pq_h_tbl + ops_bytes, qs.data(), q_bytes);
+    }
+
+    cudaEvent_t e0, e1;
+    CU(cudaEventCreate(&e0));
+    CU(cudaEventCreate(&e1));
+    sgs_status_t rc = SGS_OK;
+    cudaError_t ce = cudaEventRecord(e0, st);
+    if (ce == cudaSuccess && host_buffers && n_queries) ce = cudaMemcpyAsync(net->pq_stage_in, inputs, in_bytes * (size_t)n_queries, cudaMemcpyHostToDevice, st);
+    if (ce == cudaSuccess && tbl_need) ce = cudaMemcpyAsync(net->pq_d_tbl, net->pq_h_tbl, tbl_need, cudaMemcpyHostToDevice, st);
+    if (ce == cudaSuccess) ce = cudaMemsetAsync(net->pq_counter, 0, sizeof(int), st);
+    if (ce == cudaSuccess && n_queries) {
+        PqParams p;
+        p.ops = reinterpret_cast<const PqOp *>(net->pq_d_tbl);
+        p.queries = reinterpret_cast<const PqQuery *>(net->pq_d_tbl + ops_bytes);
+        p.n_queries = n_queries;
+        p.counter = net->pq_counter;
+        p.scratch = net->pq_scratch;
+        p.slot_bytes = slot_bytes; p.act_bytes = act_bytes;
+        p.status = tc_status_word(net->device);
+        LayerRange range(net, -1, "persistent SubNet kernel");
+        ce = subnet_kernel_launch(p, std::min(blocks_max, n_queries), st);
+        net->kernel_launches++;
+    }
+    if (ce == cudaSuccess && host_buffers && n_queries) ce = cudaMemcpyAsync(logits, net->pq_stage_out, out_bytes * (size_t)n_queries, cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaEventRecord(e1, st);
+    cudaError_t se = cudaStreamSynchronize(st);
+    if (ce != cudaSuccess || se != cudaSuccess) rc = fail(net, SGS_ECUDA, std::string("persistent stream: ") + cudaGetErrorString(se != cudaSuccess ? se : ce));
+    if (rc == SGS_OK && tc_conv_status()) rc = fail(net, SGS_ETIMEOUT, "a bounded device-side wait ran out in the persistent SubNet kernel");
+    if (rc == SGS_OK && stats) {
+        std::memset(stats, 0, sizeof(*stats));
+        float ms = 0;
+        cudaEventElapsedTime(&ms, e0, e1);
+        stats->n_queries = n_queries;
+        stats->total_ms = ms;
+        stats->queries_per_s = ms > 0 ? n_queries / (ms * 1e-3) : 0;
+        stats->images_per_s = stats->queries_per_s;
+        if (o.record_latency && n_queries) stats->p50_ms = stats->p99_ms = stats->mean_ms = ms;  // every query starts and ends with the launch
+        stats->useful_flops = flops;
+        stats->weight_bytes = wbytes;
+        stats->hbm_weight_bytes = miss_bytes;
+        stats->hit_ratio = n_queries ? hit / n_queries : 0;
+        stats->byte_hit_ratio = wbytes > 0 ? 1.0 - miss_bytes / wbytes : 0;
+        stats->kernel_launches = net->kernel_launches - launches0;
+        stats->plan_hits = net->plan_hits - hits0;
+        stats->plan_misses = net->plan_misses - miss0;
+        stats->cache_updates = updates;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    return rc;
+}
+
 static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_subnet_cfg_t *cfgs, const void *inputs,
                                 int batch, int res, void *logits, const sgs_stream_opts_t *opts,
                                 sgs_stream_stats_t *stats, cudaStream_t st, bool host_buffers) {
@@ -1935,7 +2165,7 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
     if (!guard.ok) return fail(net, SGS_ECUDA, "cudaSetDevice failed");
     sgs_stream_opts_t o;
     if (opts) o = *opts;
-    else { o.cache_enabled = 1; o.window_q = 4; o.cache_budget_bytes = 0; o.use_graphs = 1; o.record_latency = 1; o.weights_evict_first = 0; o.concurrency = 1; o.wave = 0; o.policy = 0; }
+    else { o.cache_enabled = 1; o.window_q = 4; o.cache_budget_bytes = 0; o.use_graphs = 1; o.record_latency = 1; o.weights_evict_first = 0; o.concurrency = 1; o.wave = 0; o.policy = 0; o.persistent = 0; }
     if (o.window_q < 1) return fail(net, SGS_EINVAL, "window_q must be >= 1");
     if (o.concurrency < 0 || o.concurrency > 16) return fail(net, SGS_EINVAL, "concurrency must be in [0, 16]");
     for (int t = 0; t < n_queries; t++)
@@ -1947,6 +2177,10 @@ static sgs_status_t stream_impl(sgs_supernet_t *net, int n_queries, const sgs_su
     net->cache.policy = o.policy;
     cache_reset(net, o.cache_enabled != 0, o.cache_budget_bytes, o.window_q);
     net->cache.evict_first_when_off = (!o.cache_enabled && o.weights_evict_first) ? 1 : 0;
+    if (o.persistent) {
+        if (batch != 1) return fail(net, SGS_EINVAL, "persistent execution takes one image per query");
+        return persistent_impl(net, n_queries, cfgs, inputs, res, logits, o, stats, st, host_buffers);
+    }
     if (o.wave > 0 && n_queries > 0 && net->dtype == SGS_BF16 && tc_available() && !net->force_plain)
         return wave_impl(net, n_queries, cfgs, inputs, batch, res, logits, o, stats, st, host_buffers);
     // queries in flight at once: each runs in its own slot; per-kernel profiling wants them one by one

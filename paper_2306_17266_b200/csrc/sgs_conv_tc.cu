@@ -704,6 +704,7 @@ cudaError_t tc_conv_init(int dev) {
     if ((e = cudaFuncSetAttribute(conv_tc_kernel<64, 3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64, 3>())) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(conv_tc_kernel<128, 3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128, 3>())) != cudaSuccess) return e;
     if ((e = tc_group_init(dev)) != cudaSuccess) return e;
+    if ((e = subnet_kernel_init(dev)) != cudaSuccess) return e;
     ds.attrs_set = true;
     return cudaSuccess;
 }

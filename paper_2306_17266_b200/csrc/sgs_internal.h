@@ -78,6 +78,43 @@ struct ConvArgs {
     size_t ws_elems = 0;
 };
 
+// ---- persistent SubNet kernel (sgs_subnet_kernel.cu) ------------------------------------------
+// One launch serves a whole stream of one-image queries of the MobileNetV3-shaped family: every block (one per
+// SM) takes the next unserved query and runs ALL layers of that query's SubNet by itself, from the image to the
+// logits, out of a private scratch area; the layers are the records of an op list the host wrote for the config.
+enum PqType { PQ_STEM = 0, PQ_PW = 1, PQ_DW = 2, PQ_GAP = 3, PQ_SE_GATE = 4, PQ_SCALE = 5, PQ_LINEAR = 6 };
+struct alignas(16) PqOp {
+    int type;
+    int in, out, res;     // activation buffers of the block's scratch area (-1: the query's image / none)
+    int vin, vout;        // fp32 vectors held in shared memory (vout -1: the query's logits)
+    int H, W, C, K;       // input map, sliced input channels, sliced filters (depthwise: C == K channels)
+    int Ho, Wo, k, stride;
+    int act, R, Kmax, ld; // stored kernel size, stored filter count (depthwise pitch), row pitch of w in elements
+    int ld2, cache_rows;  // SE gate: pitch of the second FC; pointwise: filters of this layer held in the block's weight buffer
+    const void *w;        // stored weights of the layer (sliced by prefix / centre crop inside the kernel)
+    const float *scale, *shift;  // folded batch norm, or shift = bias
+    const void *w2;       // SE gate: second FC
+    const float *bias2;
+    long long cache_off;  // pointwise: byte offset of this layer's rows in the block's weight buffer (-1: not held)
+};
+static_assert(sizeof(PqOp) == 128, "record size");
+struct alignas(16) PqQuery {
+    const void *x;   // [res][res][3] bf16
+    float *logits;   // [classes]
+    int op_begin, op_count;
+    int pad_[2];
+};
+static_assert(sizeof(PqQuery) == 32, "record size");
+struct PqParams {
+    const PqQuery *queries;
+    const PqOp *ops;
+    int n_queries;
+    int *counter;            // next unserved query (zeroed before the launch)
+    unsigned char *scratch;  // blocks x slot_bytes: four activation buffers of act_bytes per block
+    size_t slot_bytes, act_bytes;
+    int *status;             // device status word: nonzero after a bounded wait ran out
+};
+
 enum OpType { OP_CONV, OP_DW, OP_MAXPOOL, OP_GAP, OP_SE_GATE, OP_SCALE, OP_LINEAR, OP_IM2COL, OP_PAD8 };
 
 struct TcConvPlan;  // tensor-core launch description (sgs_conv_tc.cu)
@@ -109,6 +146,7 @@ struct Plan {
     bool padded = false;    // activation tensors hold 16-channel-padded pixels (ConvArgs::ldx, ldy)
     int slot = 0;           // which set of workspaces the plan's buffer addresses refer to
     int throughput = 0;     // tile choice of the plan's convolutions (see ConvArgs::throughput)
+    std::vector<PqOp> pq;  // the plan as an op list of the persistent SubNet kernel (built on first use)
 };
 
 // ---- launchers implemented in sgs_kernels.cu (T = float or __nv_bfloat16) -------------------
@@ -207,6 +245,10 @@ private:
     Impl *impl;
 };
 cudaError_t tc_group_init(int device);
+
+cudaError_t subnet_kernel_init(int device);
+size_t subnet_kernel_smem();  // dynamic shared memory of a block
+cudaError_t subnet_kernel_launch(const PqParams &p, int blocks, cudaStream_t st);
 void tc_group_set_stage_group(int stages);  // tuning: stages per barrier pair of the grouped kernel (0 = default)
 
 }  // namespace sgs

@@ -29,7 +29,7 @@ def test_struct_sizes_match_the_header():
     # sizes implied by the header's field lists (LP64)
     assert ctypes.sizeof(wl.SubnetCfg) == 4 * (8 + 9 + 64 + 64)
     assert ctypes.sizeof(wl.ArchDesc) == 4 * (2 + 8 + 8 + 3)
-    assert ctypes.sizeof(sgs.StreamOpts) == 40  # 2 ints, size_t, 6 ints
+    assert ctypes.sizeof(sgs.StreamOpts) == 48  # 2 ints, size_t, 7 ints (padded to 8 bytes)
     assert ctypes.sizeof(sgs.StreamStats) == 8 + 11 * 8 + 8 + 16
     assert ctypes.sizeof(sgs.ConvDesc) == 18 * 4
     assert ctypes.sizeof(sgs.CacheStats) == 8 + 7 * 8 + 4 * 4
