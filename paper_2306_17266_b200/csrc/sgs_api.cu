@@ -2051,7 +2051,7 @@ static sgs_status_t persistent_impl(sgs_supernet_t *net, int n_queries, const sg
         }
     }
     // device resources: scratch of the blocks, tables, counter, staging for host buffers
-    const int blocks_max = std::max(1, net->sms);
+    const int blocks_max = std::max(1, net->sms) * subnet_kernel_blocks_per_sm();
     const size_t act_bytes = (act_elems * net->elem() + 255) / 256 * 256, slot_bytes = 4 * act_bytes;
     if (net->pq_scratch_bytes < slot_bytes * blocks_max) {
         CU(cudaStreamSynchronize(st));

@@ -248,6 +248,7 @@ cudaError_t tc_group_init(int device);
 
 cudaError_t subnet_kernel_init(int device);
 size_t subnet_kernel_smem();  // dynamic shared memory of a block
+int subnet_kernel_blocks_per_sm();
 cudaError_t subnet_kernel_launch(const PqParams &p, int blocks, cudaStream_t st);
 void tc_group_set_stage_group(int stages);  // tuning: stages per barrier pair of the grouped kernel (0 = default)
 

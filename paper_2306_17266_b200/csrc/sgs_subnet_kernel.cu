@@ -3,12 +3,12 @@
 // The paper's accelerator serves one query per pass and keeps the weights it will need again on chip
 // (Section 3.1, Section 4.2 "Persistent Buffer").  On this GPU a one-image MobileNetV3-sized SubNet is far too
 // small to fill the machine layer by layer: a wave of 32 such queries needs about a hundred dependent launches of
-// 10 - 20 us each.  Here the whole stream is ONE launch instead.  Every block (one per SM, 256 threads) takes the
+// 10 - 20 us each.  Here the whole stream is ONE launch instead.  Every block (one per SM, 512 threads) takes the
 // next unserved query from a counter and runs all layers of that query's SubNet by itself, image to logits:
 //   * pointwise (1x1) convolutions on the tensor cores: tcgen05.mma with the fp32 accumulator in tensor memory
 //     (two 256-column buffers, so the epilogue of one tile overlaps the MMAs of the next); the operands are
 //     brought into 128-byte-swizzled shared-memory tiles by the block's own threads with 16-byte asynchronous
-//     copies (a ring of 3 - 4 stages, copies two stages ahead of the MMAs) - the tiles of one query are too
+//     copies (a ring of three stages, copies two stages ahead of the MMAs) - the tiles of one query are too
 //     small and too many to be worth a tensor map each;
 //   * depthwise convolutions, the 3-channel stem, pooling, the squeeze-excite gate and the linear layers on the
 //     CUDA cores, with 16-byte accesses;
@@ -27,11 +27,16 @@ namespace {
 
 using bf16 = __nv_bfloat16;
 
-constexpr int PQ_THREADS = 256;
-constexpr int PQ_RING_BYTES = 144 * 1024;  // operand ring: 3 stages of 48 KB (256-filter tiles) or 4 smaller ones
-constexpr int PQ_LAG = 2;                  // copies run this many stages ahead of the MMAs
-constexpr int PQ_VEC = 1280;               // longest fp32 vector held in shared memory (the head's width)
-constexpr int PQ_ACC_COLS = 256;           // tensor-memory columns of one accumulator buffer
+constexpr int PQ_THREADS = 512;
+constexpr int PQ_BLOCKS_PER_SM = 1;          // (measured: two blocks of 256 threads per SM with 96-filter tiles serve 28k queries/s, one of 512 serves 42k)
+constexpr int PQ_WARPS = PQ_THREADS / 32;
+constexpr int PQ_ROWS = PQ_THREADS / 8;      // rows of 128 bytes one round of 16-byte copies covers
+constexpr int PQ_MAX_K = 1024;               // widest pointwise layer (folded batch norm staged in shared memory)
+constexpr int PQ_MAX_BN = 256;               // filters per tile
+constexpr int PQ_RING_BYTES = 144 * 1024;    // operand ring: 3 stages of pixel tile (16 KB) + filter tile (up to 32 KB), or 4 smaller ones
+constexpr int PQ_LAG = 2;                    // copies run this many stages ahead of the MMAs
+constexpr int PQ_VEC = 1280;                 // longest fp32 vector held in shared memory (the head's width)
+constexpr int PQ_ACC_COLS = 256;             // tensor-memory columns of one accumulator buffer
 constexpr unsigned long long PQ_WAIT_NS = 2000000000ull;
 
 // Completed phases of the block's barriers since the kernel started (the same in every thread; only ever
@@ -68,7 +73,12 @@ __device__ __forceinline__ float dot8w(uint4 wv, float4 x0, float4 x1, float s) 
 
 // ---------------------------------------------------------------------------------------------
 // Pointwise convolution  y[m][f] = act(scale[f] * sum_c x[m][c] * w[f][c] + shift[f]) (+ res[m][f])
-// M = H * W pixels of the one image, tiles of 128 pixels x BN filters, channels in chunks of 64.
+// M = H * W pixels of the one image, tiles of 128 pixels x BN filters (BN <= PQ_MAX_BN), channels in chunks of 64;
+// a ring of three stages, each the pixel tile's and the filter tile's 64-channel chunk.
+// (Measured alternatives, both slower: the layer's whole weight matrix copied once and read in place by every pixel
+// tile - the larger shared-memory footprint costs the depthwise layers their L1; and the epilogue's results
+// gathered in a shared-memory tile and written out with fully coalesced stores - the epilogue is bound by its
+// arithmetic, not by its 16-byte stores.)
 // ---------------------------------------------------------------------------------------------
 struct PwShape {
     int M, C, K, n_tiles, BN, cchunks, m_tiles, stage_bytes, S;
@@ -76,8 +86,8 @@ struct PwShape {
 __device__ __forceinline__ PwShape pw_shape(const PqOp &op) {
     PwShape s;
     s.M = op.Ho * op.Wo; s.C = op.C; s.K = op.K;
-    s.n_tiles = (s.K + 255) / 256;
-    s.BN = (((s.K + s.n_tiles - 1) / s.n_tiles) + 15) & ~15;  // MMA width: a multiple of 16, at most 256
+    s.n_tiles = (s.K + PQ_MAX_BN - 1) / PQ_MAX_BN;
+    s.BN = (((s.K + s.n_tiles - 1) / s.n_tiles) + 15) & ~15;  // MMA width: a multiple of 16, at most PQ_MAX_BN
     s.cchunks = (s.C + 63) >> 6;
     s.m_tiles = (s.M + 127) >> 7;
     s.stage_bytes = A_STAGE_BYTES + s.BN * 128;
@@ -85,60 +95,89 @@ __device__ __forceinline__ PwShape pw_shape(const PqOp &op) {
     return s;
 }
 
-// Epilogue of tile (mt, nt) out of accumulator buffer `buf`: warp w reads lane quadrant w % 4 (its 32 pixels)
-// and every second group of 16 filters, starting with group w / 4.
-__device__ __forceinline__ bool pw_epilogue(const PqOp &op, const PwShape &s, const bf16 *res, bf16 *y, int mt, int nt,
+// Epilogue arithmetic of 16 consecutive filters of one pixel, two values at a time (packed fp32 instructions).
+// Hard swish is x * sat(x / 6 + 1 / 2): one saturating multiply-add and one multiply.
+__device__ __forceinline__ void pw_store16(const PwShape &s, const float *bn, const uint32_t *v, const bf16 *res, bf16 *y, int m, int f0,
+                                           int c, int cols, int act) {
+#pragma unroll
+    for (int h = 0; h < 2; h++) {
+        const int cc = c + h * 8;
+        if (cc < cols) {
+            const int f = f0 + cc;
+            const size_t oi = (size_t)m * s.K + f;
+            const float4 s0 = *reinterpret_cast<const float4 *>(bn + f), s1 = *reinterpret_cast<const float4 *>(bn + f + 4);
+            const float4 h0 = *reinterpret_cast<const float4 *>(bn + PQ_MAX_K + f), h1 = *reinterpret_cast<const float4 *>(bn + PQ_MAX_K + f + 4);
+            float2 o[4];
+            o[0] = __ffma2_rn(make_float2(__uint_as_float(v[h * 8 + 0]), __uint_as_float(v[h * 8 + 1])), make_float2(s0.x, s0.y), make_float2(h0.x, h0.y));
+            o[1] = __ffma2_rn(make_float2(__uint_as_float(v[h * 8 + 2]), __uint_as_float(v[h * 8 + 3])), make_float2(s0.z, s0.w), make_float2(h0.z, h0.w));
+            o[2] = __ffma2_rn(make_float2(__uint_as_float(v[h * 8 + 4]), __uint_as_float(v[h * 8 + 5])), make_float2(s1.x, s1.y), make_float2(h1.x, h1.y));
+            o[3] = __ffma2_rn(make_float2(__uint_as_float(v[h * 8 + 6]), __uint_as_float(v[h * 8 + 7])), make_float2(s1.z, s1.w), make_float2(h1.z, h1.w));
+            if (res) {
+                const uint4 rv = *reinterpret_cast<const uint4 *>(res + oi);
+                o[0] = __fadd2_rn(o[0], unpack2(rv.x)); o[1] = __fadd2_rn(o[1], unpack2(rv.y));
+                o[2] = __fadd2_rn(o[2], unpack2(rv.z)); o[3] = __fadd2_rn(o[3], unpack2(rv.w));
+            }
+            uint4 ov;
+            __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                if (act == ACT_RELU) {
+                    o[j].x = fmaxf(o[j].x, 0.f); o[j].y = fmaxf(o[j].y, 0.f);
+                } else if (act == ACT_HSWISH) {
+                    const float2 t = make_float2(__saturatef(fmaf(o[j].x, 1.f / 6.f, 0.5f)), __saturatef(fmaf(o[j].y, 1.f / 6.f, 0.5f)));
+                    o[j] = __fmul2_rn(o[j], t);
+                }
+                ob[j] = __floats2bfloat162_rn(o[j].x, o[j].y);
+            }
+            *reinterpret_cast<uint4 *>(y + oi) = ov;
+        }
+    }
+}
+
+// Epilogue of tile (mt, nt) out of an accumulator buffer: warp w reads lane quadrant w % 4 (its 32 pixels) and the
+// groups of 16 filters g with g % (warps / 4) == w / 4, two groups per tensor-memory wait.  bn: the layer's folded
+// batch norm in shared memory, scale at [f], shift at [PQ_MAX_K + f].
+__device__ __forceinline__ bool pw_epilogue(const PqOp &op, const PwShape &s, const float *bn, const bf16 *res, bf16 *y, int mt, int nt,
                                             uint32_t tmem_acc, uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, quad = warp & 3, half = warp >> 2;
+    constexpr int CG = PQ_WARPS / 4;  // column groups the warps of one quadrant share
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, quad = warp & 3, cgrp = warp >> 2;
     if (!__all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, PQ_WAIT_NS))) return false;
     tc_fence_after();
-    const int m = mt * 128 + quad * 32 + lane;
+    const int m = mt * 128 + quad * 32 + lane, act = op.act;
     const int f0 = nt * s.BN, cols = min(s.BN, s.K - f0);  // a multiple of 8
     const uint32_t t = tmem_acc + ((uint32_t)(quad * 32) << 16);
-    for (int g = half; g * 16 < cols; g += 2) {
-        uint32_t v[16];
-        tmem_ld16(t + (uint32_t)(g * 16), v);
+    for (int g = cgrp; g * 16 < cols; g += 2 * CG) {
+        uint32_t v0[16], v1[16];
+        const bool two = (g + CG) * 16 < cols;  // (the same in every lane)
+        tmem_ld16(t + (uint32_t)(g * 16), v0);
+        if (two) tmem_ld16(t + (uint32_t)((g + CG) * 16), v1);
         tmem_ld_wait();
         if (m < s.M) {
-#pragma unroll
-            for (int h = 0; h < 2; h++) {
-                const int c = g * 16 + h * 8;
-                if (c < cols) {
-                    const int f = f0 + c;
-                    const float4 s0 = __ldg(reinterpret_cast<const float4 *>(op.scale + f)), s1 = __ldg(reinterpret_cast<const float4 *>(op.scale + f + 4));
-                    const float4 h0 = __ldg(reinterpret_cast<const float4 *>(op.shift + f)), h1 = __ldg(reinterpret_cast<const float4 *>(op.shift + f + 4));
-                    float o[8];
-                    o[0] = __uint_as_float(v[h * 8 + 0]) * s0.x + h0.x; o[1] = __uint_as_float(v[h * 8 + 1]) * s0.y + h0.y;
-                    o[2] = __uint_as_float(v[h * 8 + 2]) * s0.z + h0.z; o[3] = __uint_as_float(v[h * 8 + 3]) * s0.w + h0.w;
-                    o[4] = __uint_as_float(v[h * 8 + 4]) * s1.x + h1.x; o[5] = __uint_as_float(v[h * 8 + 5]) * s1.y + h1.y;
-                    o[6] = __uint_as_float(v[h * 8 + 6]) * s1.z + h1.z; o[7] = __uint_as_float(v[h * 8 + 7]) * s1.w + h1.w;
-                    finish_store(o, res, y, (size_t)m * s.K + f, op.act);
-                }
-            }
+            pw_store16(s, bn, v0, res, y, m, f0, g * 16, cols, act);
+            if (two) pw_store16(s, bn, v1, res, y, m, f0, (g + CG) * 16, cols, act);
         }
     }
     tc_fence_before();  // the buffer's next MMAs are issued after a block barrier
     return true;
 }
-
 // Returns false when a wait ran out (the caller leaves at its next block barrier).
-__device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, const bf16 *res, bf16 *y, uint8_t *ring,
-                                             const uint8_t *held, uint64_t *free_bar, uint64_t *acc_bar, uint32_t tmem_base,
-                                             PipeState &ps, volatile int *abort_flag) {
+__device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, const bf16 *res, bf16 *y, uint8_t *ring, float *bn,
+                                             uint64_t *free_bar, uint64_t *acc_bar, uint32_t tmem_base, PipeState &ps,
+                                             volatile int *abort_flag) {
     const int tid = threadIdx.x;
     const PwShape s = pw_shape(op);
+    const int S = s.S;
     const int total = s.n_tiles * s.m_tiles * s.cchunks;
     // instruction descriptor: fp32 accumulator, bf16 x bf16, both K-major, N = BN, M = 128
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(s.BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
     const uint32_t ring_u32 = smem_u32(ring);
     const bf16 *w = static_cast<const bf16 *>(op.w);
-    // this thread's 16-byte piece of every 128-byte row it copies: rows tid / 8 + 32 j, piece tid % 8 (the
+    // the layer's folded batch norm, read by every epilogue (visible after the first block barrier of the loop)
+    for (int f = tid; f < s.K; f += PQ_THREADS) { bn[f] = __ldg(op.scale + f); bn[PQ_MAX_K + f] = __ldg(op.shift + f); }
+    // this thread's 16-byte piece of every 128-byte row it copies: rows tid / 8 + PQ_ROWS j, piece tid % 8 (the
     // swizzle term row % 8 is then the same for all of them)
     const int c16 = tid & 7, r0 = tid >> 3;
     const uint32_t piece = (uint32_t)((c16 ^ (r0 & 7)) << 4);
-    // rows of this layer that the block holds in its weight buffer need no copy: the MMA reads them in place
-    const bool b_held = held != nullptr && op.cache_off >= 0 && s.K <= op.cache_rows;
-    const uint32_t held_u32 = b_held ? smem_u32(held + op.cache_off) : 0u;
 
     bool ok = true;
     int p_chunk = 0, p_mt = 0, p_nt = 0, p_stage = 0;  // next iteration to copy
@@ -154,8 +193,7 @@ __device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, cons
             const uint32_t buf = ps.tiles & 1u;
             if (tid == 0) {
                 tc_fence_after();
-                const uint32_t sa = ring_u32 + (uint32_t)(c_stage * s.stage_bytes);
-                const uint32_t sb = b_held ? held_u32 + (uint32_t)(c_chunk * op.cache_rows * 128) : sa + A_STAGE_BYTES;
+                const uint32_t sa = ring_u32 + (uint32_t)(c_stage * s.stage_bytes), sb = sa + A_STAGE_BYTES;
                 const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
                 const int ksteps = (min(64, s.C - c_chunk * 64) + 15) >> 4;
                 for (int q = 0; q < ksteps; q++)
@@ -167,7 +205,7 @@ __device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, cons
             // the previous tile's epilogue runs while this tile's MMAs do
             if (c_chunk == 0 && e_mt >= 0) {
                 const uint32_t n_acc = e_buf ? ps.acc[1] : ps.acc[0];
-                ok = pw_epilogue(op, s, res, y, e_mt, e_nt, tmem_base + e_buf * PQ_ACC_COLS, &acc_bar[e_buf], (n_acc - 1) & 1u, abort_flag) && ok;
+                ok = pw_epilogue(op, s, bn, res, y, e_mt, e_nt, tmem_base + e_buf * PQ_ACC_COLS, &acc_bar[e_buf], (n_acc - 1) & 1u, abort_flag) && ok;
                 e_mt = -1;
             }
             if (c_chunk == s.cchunks - 1) {
@@ -175,50 +213,49 @@ __device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, cons
                 ps.tiles++;
                 e_mt = c_mt; e_nt = c_nt; e_buf = buf;
             }
-            if (++c_stage == s.S) c_stage = 0;
+            if (++c_stage == S) c_stage = 0;
             if (++c_chunk == s.cchunks) { c_chunk = 0; if (++c_mt == s.m_tiles) { c_mt = 0; ++c_nt; } }
         }
         if (i < total) {
-            // the stage was last read by the MMAs of iteration i - S, issued at least one step ago
+            // the stage was last read by the MMAs of iteration i - S, issued in the previous step
             const uint32_t u = get4(ps.use, p_stage);
-            if (i >= s.S && u > 0) ok = mbar_wait(&free_bar[p_stage], (u - 1) & 1u, abort_flag, PQ_WAIT_NS) && ok;
+            if (i >= S && u > 0) ok = mbar_wait(&free_bar[p_stage], (u - 1) & 1u, abort_flag, PQ_WAIT_NS) && ok;
             const uint32_t sa = ring_u32 + (uint32_t)(p_stage * s.stage_bytes), sb = sa + A_STAGE_BYTES;
             const int c0 = p_chunk * 64 + c16 * 8;
             const bool cvalid = c0 < s.C;
 #pragma unroll
-            for (int j = 0; j < 4; j++) {
-                const int row = r0 + 32 * j, m = p_mt * 128 + row;
+            for (int j = 0; j < 128 / PQ_ROWS; j++) {
+                const int row = r0 + PQ_ROWS * j, m = p_mt * 128 + row;
                 const bool v = cvalid && m < s.M;
                 cp16_cg(sa + (uint32_t)(row * 128) + piece, v ? x + (size_t)m * s.C + c0 : x, v);
             }
-            if (!b_held) {
-                for (int row = r0; row < s.BN; row += 32) {
-                    const int f = p_nt * s.BN + row;
-                    const bool v = cvalid && f < s.K;
-                    cp16_ca(sb + (uint32_t)(row * 128) + piece, v ? w + (size_t)f * op.ld + c0 : w, v);
-                }
+            for (int row = r0; row < s.BN; row += PQ_ROWS) {
+                const int f = p_nt * s.BN + row;
+                const bool v = cvalid && f < s.K;
+                cp16_ca(sb + (uint32_t)(row * 128) + piece, v ? w + (size_t)f * op.ld + c0 : w, v);
             }
-            if (++p_stage == s.S) p_stage = 0;
+            if (++p_stage == S) p_stage = 0;
             if (++p_chunk == s.cchunks) { p_chunk = 0; if (++p_mt == s.m_tiles) { p_mt = 0; ++p_nt; } }
         }
         cp_commit();  // (an empty group in the drain steps keeps the group count in step with i)
     }
     if (e_mt >= 0) {
         const uint32_t n_acc = e_buf ? ps.acc[1] : ps.acc[0];
-        ok = pw_epilogue(op, s, res, y, e_mt, e_nt, tmem_base + e_buf * PQ_ACC_COLS, &acc_bar[e_buf], (n_acc - 1) & 1u, abort_flag) && ok;
+        ok = pw_epilogue(op, s, bn, res, y, e_mt, e_nt, tmem_base + e_buf * PQ_ACC_COLS, &acc_bar[e_buf], (n_acc - 1) & 1u, abort_flag) && ok;
     }
     cp_wait<0>();
     return ok;
 }
 
 // ---------------------------------------------------------------------------------------------
-// Depthwise convolution: a thread owns 8 channels of 4 neighbouring output pixels of one output row and walks
+// Depthwise convolution: a thread owns 8 channels of 4 (2) neighbouring output pixels of one output row and walks
 // the filter rows; per filter row it loads the input columns once and uses each for every tap it belongs to.
 // (Plain loads: the input was written by this block a moment ago.)
 // ---------------------------------------------------------------------------------------------
 template <int K, int ST>
-__device__ __forceinline__ void pq_depthwise(const PqOp &op, const bf16 *x, bf16 *y) {
-    constexpr int TW = 4, NCOL = (TW - 1) * ST + K, P = (K - 1) / 2;
+__device__ __noinline__ void pq_depthwise(const PqOp &op, const bf16 *x, bf16 *y) {
+    constexpr int TW = (ST == 2 && K > 3) ? 2 : 4;  // (the wide stride-2 windows would not fit the register budget of 512 threads)
+    constexpr int NCOL = (TW - 1) * ST + K, P = (K - 1) / 2;
     const int Cn = op.K, groups = Cn >> 3, wblocks = (op.Wo + TW - 1) / TW;
     const int per_row = groups * wblocks, total = per_row * op.Ho;
     const int o = (op.R - K) / 2;
@@ -279,7 +316,7 @@ __device__ __forceinline__ void pq_depthwise(const PqOp &op, const bf16 *x, bf16
 
 // Stem: 3-channel image, k x k taps (k <= 3 here), stride `stride`, direct on the CUDA cores; a thread owns one
 // output pixel and produces the filters eight at a time.  wsm: k * k * 3 * K floats of shared memory.
-__device__ __forceinline__ void pq_stem(const PqOp &op, const bf16 *img, bf16 *y, float *wsm) {
+__device__ __noinline__ void pq_stem(const PqOp &op, const bf16 *img, bf16 *y, float *wsm) {
     const int k = op.k, K = op.K, taps = k * k * 3, o = (op.R - k) / 2, P = (k - 1) / 2;
     const bf16 *w = static_cast<const bf16 *>(op.w);
     for (int i = threadIdx.x; i < taps * K; i += PQ_THREADS) {
@@ -314,9 +351,10 @@ __device__ __forceinline__ void pq_stem(const PqOp &op, const bf16 *img, bf16 *y
 #pragma unroll
                         for (int c = 0; c < 3; c++) {
                             const float xv = in[(r * 3 + sx) * 3 + c];
-                            const float *wp = wsm + ((r * k + sx) * 3 + c) * K + f0;
-#pragma unroll
-                            for (int q = 0; q < 8; q++) acc[q] = fmaf(xv, wp[q], acc[q]);
+                            const float4 *wp = reinterpret_cast<const float4 *>(wsm + ((r * k + sx) * 3 + c) * K + f0);  // (every lane the same address)
+                            const float4 wa = wp[0], wb = wp[1];
+                            acc[0] = fmaf(xv, wa.x, acc[0]); acc[1] = fmaf(xv, wa.y, acc[1]); acc[2] = fmaf(xv, wa.z, acc[2]); acc[3] = fmaf(xv, wa.w, acc[3]);
+                            acc[4] = fmaf(xv, wb.x, acc[4]); acc[5] = fmaf(xv, wb.y, acc[5]); acc[6] = fmaf(xv, wb.z, acc[6]); acc[7] = fmaf(xv, wb.w, acc[7]);
                         }
                     }
             float ov[8];
@@ -331,7 +369,7 @@ __device__ __forceinline__ void pq_stem(const PqOp &op, const bf16 *img, bf16 *y
 __device__ __forceinline__ void pq_gap(const PqOp &op, const bf16 *x, float *out) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, cvecs = op.C >> 3, HW = op.H * op.W;
     const float inv = 1.f / (float)HW;
-    for (int cv = warp; cv < cvecs; cv += PQ_THREADS / 32) {
+    for (int cv = warp; cv < cvecs; cv += PQ_WARPS) {
         const bf16 *base = x + cv * 8;
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int i = lane; i < HW; i += 32) {
@@ -354,9 +392,9 @@ __device__ __forceinline__ void pq_gap(const PqOp &op, const bf16 *x, float *out
 // y[j] = f(bias[j] + sum_c w[j][c] * v[c]) for j < K: a warp takes JB outputs at a time and has the 16-byte weight
 // loads of all of them in flight together.  HS: hard sigmoid (the squeeze-excite gate) instead of `act`.
 template <int JB, bool HS>
-__device__ __forceinline__ void pq_matvec(const bf16 *w, int ld, const float *bias, const float *v, float *y, int C, int K, int act) {
+__device__ __noinline__ void pq_matvec(const bf16 *w, int ld, const float *bias, const float *v, float *y, int C, int K, int act) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int j0 = warp * JB; j0 < K; j0 += (PQ_THREADS / 32) * JB) {
+    for (int j0 = warp * JB; j0 < K; j0 += PQ_WARPS * JB) {
         float s[JB];
 #pragma unroll
         for (int u = 0; u < JB; u++) s[u] = 0.f;
@@ -399,10 +437,11 @@ __device__ __forceinline__ void pq_scale(const PqOp &op, bf16 *x, const float *g
     }
 }
 
-__global__ void __launch_bounds__(PQ_THREADS, 1) subnet_kernel(const PqParams p) {
+__global__ void __launch_bounds__(PQ_THREADS, PQ_BLOCKS_PER_SM) subnet_kernel(const PqParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     __shared__ __align__(16) float vec_s[3][PQ_VEC];
+    __shared__ __align__(16) float bn_s[2 * PQ_MAX_K];
     __shared__ __align__(16) PqOp op_s;
     __shared__ __align__(16) PqQuery q_s;
     __shared__ __align__(8) uint64_t free_bar[4], acc_bar[2];
@@ -447,7 +486,7 @@ __global__ void __launch_bounds__(PQ_THREADS, 1) subnet_kernel(const PqParams p)
             const bf16 *res = op.res < 0 ? nullptr : reinterpret_cast<const bf16 *>(slot + (size_t)op.res * p.act_bytes);
             switch (op.type) {
             case PQ_STEM: pq_stem(op, x, y, reinterpret_cast<float *>(ring)); break;
-            case PQ_PW: ok = pq_pointwise(op, x, res, y, ring, nullptr, free_bar, acc_bar, tmem_base, ps, abort_flag) && ok; break;
+            case PQ_PW: ok = pq_pointwise(op, x, res, y, ring, bn_s, free_bar, acc_bar, tmem_base, ps, abort_flag) && ok; break;
             case PQ_DW:
                 if (op.stride == 1) {
                     if (op.k == 3) pq_depthwise<3, 1>(op, x, y);
@@ -486,6 +525,7 @@ __global__ void __launch_bounds__(PQ_THREADS, 1) subnet_kernel(const PqParams p)
 }  // namespace
 
 size_t subnet_kernel_smem() { return (size_t)PQ_RING_BYTES + 1024; }
+int subnet_kernel_blocks_per_sm() { return PQ_BLOCKS_PER_SM; }
 
 cudaError_t subnet_kernel_init(int device) {
     (void)device;
