@@ -114,7 +114,10 @@ typedef struct {
                            layers of its SubNet by itself out of a private scratch area, pointwise convolutions on the
                            tensor cores (Section 3.1: one query per pass of the accelerator; Section 4.2: what is needed
                            again stays on chip).  wave, concurrency and use_graphs are ignored; every query starts and
-                           ends with the launch (its recorded latency).  Other handles: SGS_EUNSUPPORTED. */
+                           ends with the launch (its recorded latency).  With the cache enabled one SubGraph is chosen for the launch,
+                           from the call's first window_q queries, and every SM keeps its first pointwise layers in shared
+                           memory for all the queries it serves; hit_ratio and hbm_weight_bytes are then against what is
+                           held on chip.  Other handles: SGS_EUNSUPPORTED. */
 } sgs_stream_opts_t;
 
 /* Results of sgs_stream_run (all host-side; filled after the stream has been synchronised). */
@@ -458,7 +461,8 @@ sgs_status_t sgs_debug_expire_wait(unsigned limit_us, void *cuda_stream);
  * hint on every weight tile inside the SubGraph's box, 1 = an access-policy window on the launch (the cached filter
  * prefix of the launch's stored layer, persisting; the persisting-L2 carve-out of the process is sized to the cache
  * budget), 2 = both; "dw_walk" N = stride-1 depthwise launches of at least N million output
- * elements take the walking kernel (default 48; 0 never, negative always; process-wide); "nvtx" 1 = an NVTX range named after the stored layer around
+ * elements take the walking kernel (default 48; 0 never, negative always; process-wide); "persistent_held_kb" n = shared memory per SM that persistent
+ * execution spends on the cached SubGraph's first pointwise layers (default 16, 0 = none); "nvtx" 1 = an NVTX range named after the stored layer around
  * every launch (for timeline tools); "fail_alloc_after" n = the handle's device allocations fail from
  * the (n+1)-th on with SGS_ENOMEM (fault injection on the host, -1 = off); "drop_plans" forgets every cached plan (measuring what a never-seen config costs); "profile" see
  * sgs_profile_read; "stage_group" 0 = default, 1..4 = pipeline stages that

@@ -229,6 +229,7 @@ struct sgs_supernet {
     size_t pq_stage_in_bytes = 0, pq_stage_out_bytes = 0;
     size_t persist_limit_set = 0;  // cudaLimitPersistingL2CacheSize as last set by this handle
     int nvtx = 0;  // 1: NVTX ranges named after the stored layer around every launch
+    int persistent_held_kb = 16;  // persistent execution: shared memory per SM for the cached SubGraph's first layers (0: none)
     long long fail_alloc_after = -1;  // < 0: off; else device allocations left before they start failing (test aid)
     int cache_mech = 0;    // how grouped launches keep the cached SubGraph in L2: 0 per-tile hints, 1 access-policy window of the launch, 2 both
     int pad_channels = 1;  // waves of the ResNet-shaped family keep activation pixels at multiples of 16 channels
@@ -2034,21 +2035,59 @@ static sgs_status_t persistent_impl(sgs_supernet_t *net, int n_queries, const sg
         if (pl->pq.empty() && (rc = build_pq_ops(net, pl)) != SGS_OK) return rc;
         plans[(size_t)t] = pl;
         act_elems = std::max(act_elems, pl->act_elems);
+    }
+    // The weight buffer of this launch: the SubGraph the cache policy chooses from the call's first window_q queries
+    // (their intersection, or the candidate nearest to their average), of which every block keeps the pointwise layers'
+    // boxes in shared memory, front layers first, as far as the buffer reaches.  One launch has one choice; the
+    // accounting below is against what is actually held.
+    std::vector<PqHeld> held;
+    std::unordered_map<const void *, size_t> held_of;  // stored weights -> entry
+    unsigned held_bytes = 0;
+    if (net->cache.enabled && net->persistent_held_kb > 0 && n_queries > 0) {
+        const int first = std::min(n_queries, net->cache.window_q);
+        for (int t = 0; t < first; t++) net->cache.window.push_back(plans[(size_t)t]->enc);
+        recompute_cached_subgraph(net);
+        std::vector<int> g = net->cache.G, kept(g.size(), 0);
+        const size_t budget = (size_t)net->persistent_held_kb * 1024;
+        for (size_t li = 0; li < net->layers.size() && !g.empty(); li++) {
+            const StoredLayer &L = net->layers[li];
+            if (L.kind != KIND_CONV || L.R != 1 || L.C < 8) continue;
+            const int rows = g[3 * li] & ~15, C = g[3 * li + 1];
+            if (rows < 16 || rows > 256 || C < 8) continue;
+            const int chunks = (C + 63) / 64;
+            const size_t bytes = (size_t)chunks * rows * 128;
+            if (held_bytes + bytes > budget) break;  // from the front, as the byte budget of the L2 policy is spent
+            PqHeld h;
+            std::memset(&h, 0, sizeof h);
+            h.w = L.w; h.ld = L.Cp; h.rows = rows; h.chunks = chunks; h.C = C; h.off = held_bytes;
+            held_of.emplace(L.w, held.size());
+            held.push_back(h);
+            held_bytes += (unsigned)bytes;
+            kept[3 * li] = rows; kept[3 * li + 1] = C; kept[3 * li + 2] = 1;
+        }
+        held_bytes = (held_bytes + 1023u) & ~1023u;
+        net->cache.G = kept;
+        net->cache.epoch++;
+        updates = 1;
+    }
+    for (int t = 0; t < n_queries; t++) {
+        Plan *pl = plans[(size_t)t];
         auto it = begin.find(pl);
         if (it == begin.end()) {
             it = begin.emplace(pl, (int)ops.size()).first;
-            ops.insert(ops.end(), pl->pq.begin(), pl->pq.end());
+            for (PqOp q : pl->pq) {
+                if (q.type == PQ_PW) {
+                    auto h = held_of.find(q.w);
+                    if (h != held_of.end()) { const PqHeld &e = held[h->second]; q.cache_off = e.off; q.cache_rows = e.rows; q.ld2 = e.C; }
+                }
+                ops.push_back(q);
+            }
         }
         PqQuery &q = qs[(size_t)t];
         std::memset(&q, 0, sizeof q);
         q.op_begin = it->second; q.op_count = (int)pl->pq.size();
-        const int epoch_before = net->cache.epoch;
         QueryAccount qa = account_query(net, pl->enc);
         flops += pl->flops; wbytes += qa.weight_bytes; miss_bytes += qa.miss_bytes; hit += qa.hit_ratio;
-        if (net->cache.enabled) {
-            cache_observe(net, pl->enc);
-            if (net->cache.epoch != epoch_before) updates++;
-        }
     }
     // device resources: scratch of the blocks, tables, counter, staging for host buffers
     const int blocks_max = std::max(1, net->sms) * subnet_kernel_blocks_per_sm();
@@ -2060,7 +2099,8 @@ static sgs_status_t persistent_impl(sgs_supernet_t *net, int n_queries, const sg
         if (rc != SGS_OK) return rc;
         net->pq_scratch_bytes = slot_bytes * blocks_max;
     }
-    const size_t ops_bytes = ops.size() * sizeof(PqOp), q_bytes = qs.size() * sizeof(PqQuery), tbl_need = ops_bytes + q_bytes;
+    const size_t ops_bytes = ops.size() * sizeof(PqOp), q_bytes = qs.size() * sizeof(PqQuery), h_bytes = held.size() * sizeof(PqHeld);
+    const size_t tbl_need = ops_bytes + q_bytes + h_bytes;
     if (net->pq_tbl_bytes < tbl_need) {
         CU(cudaStreamSynchronize(st));
         dev_free(net, net->pq_d_tbl, net->pq_tbl_bytes); net->pq_d_tbl = nullptr;
@@ -2103,6 +2143,7 @@ static sgs_status_t persistent_impl(sgs_supernet_t *net, int n_queries, const sg
     if (tbl_need) {
         std::memcpy(net->pq_h_tbl, ops.data(), ops_bytes);
         std::memcpy(net->pq_h_tbl + ops_bytes, qs.data(), q_bytes);
+        if (h_bytes) std::memcpy(net->pq_h_tbl + ops_bytes + q_bytes, held.data(), h_bytes);
     }
 
     cudaEvent_t e0, e1;
@@ -2117,6 +2158,9 @@ static sgs_status_t persistent_impl(sgs_supernet_t *net, int n_queries, const sg
         PqParams p;
         p.ops = reinterpret_cast<const PqOp *>(net->pq_d_tbl);
         p.queries = reinterpret_cast<const PqQuery *>(net->pq_d_tbl + ops_bytes);
+        p.held = reinterpret_cast<const PqHeld *>(net->pq_d_tbl + ops_bytes + q_bytes);
+        p.n_held = (int)held.size();
+        p.held_bytes = held_bytes;
         p.n_queries = n_queries;
         p.counter = net->pq_counter;
         p.scratch = net->pq_scratch;
@@ -2593,6 +2637,11 @@ sgs_status_t sgs_set_option(sgs_supernet_t *net, const char *name, long long val
             for (int i = 0; i < 4; i++) { net->prof_ms[i] = net->prof_bytes[i] = net->prof_flops[i] = 0; net->prof_launches[i] = 0; }
             net->prof_trace.clear();
         }
+        return SGS_OK;
+    }
+    if (n == "persistent_held_kb") {
+        if (value < 0 || (size_t)value * 1024 > subnet_kernel_held_max()) return fail(net, SGS_EINVAL, "persistent_held_kb out of range");
+        net->persistent_held_kb = (int)value;
         return SGS_OK;
     }
     if (n == "nvtx") {

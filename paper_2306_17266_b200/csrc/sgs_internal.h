@@ -90,7 +90,7 @@ struct alignas(16) PqOp {
     int H, W, C, K;       // input map, sliced input channels, sliced filters (depthwise: C == K channels)
     int Ho, Wo, k, stride;
     int act, R, Kmax, ld; // stored kernel size, stored filter count (depthwise pitch), row pitch of w in elements
-    int ld2, cache_rows;  // SE gate: pitch of the second FC; pointwise: filters of this layer held in the block's weight buffer
+    int ld2, cache_rows;  // SE gate: pitch of the second FC; pointwise: channels (ld2) and filters (cache_rows) of this layer held in the block's weight buffer
     const void *w;        // stored weights of the layer (sliced by prefix / centre crop inside the kernel)
     const float *scale, *shift;  // folded batch norm, or shift = bias
     const void *w2;       // SE gate: second FC
@@ -105,7 +105,20 @@ struct alignas(16) PqQuery {
     int pad_[2];
 };
 static_assert(sizeof(PqQuery) == 32, "record size");
+// One layer's box in the weight buffer every block keeps in shared memory for the whole launch (Section 4.2,
+// Persistent Buffer): the first `rows` filters (a multiple of 16) x the first C channels of a pointwise layer, stored as
+// `chunks` tiles of rows x 128 bytes (64 channels each, zero beyond C) in the layout the tensor core reads.
+struct alignas(16) PqHeld {
+    const void *w;
+    int ld, rows, chunks, C;
+    unsigned off;
+    int pad_;
+};
+static_assert(sizeof(PqHeld) == 32, "record size");
 struct PqParams {
+    const PqHeld *held;      // n_held boxes, held_bytes in total (0: no weight buffer)
+    int n_held;
+    unsigned held_bytes;
     const PqQuery *queries;
     const PqOp *ops;
     int n_queries;
@@ -250,6 +263,7 @@ cudaError_t subnet_kernel_init(int device);
 size_t subnet_kernel_smem();  // dynamic shared memory of a block
 int subnet_kernel_blocks_per_sm();
 cudaError_t subnet_kernel_launch(const PqParams &p, int blocks, cudaStream_t st);
+size_t subnet_kernel_held_max();  // largest weight buffer a block can keep
 void tc_group_set_stage_group(int stages);  // tuning: stages per barrier pair of the grouped kernel (0 = default)
 
 }  // namespace sgs

@@ -14,6 +14,11 @@
 //     CUDA cores, with 16-byte accesses;
 //   * activations in a private scratch area of the block in global memory (written and read back by the same
 //     SM, so they stay in L1 / L2); pooled vectors and gates in shared memory.
+//   * optionally a weight buffer in shared memory, filled once per block at the start of the launch with the
+//     cached SubGraph's boxes of the first pointwise layers (the first filters x first channels of their stored
+//     rows) and read in place by the MMAs of every query the block serves; filters and channels of a query's
+//     slice beyond the box are streamed through the ring as usual (the SubGraph-stationary dataflow of
+//     Section 4.3: what the queries share is fetched once, the rest per query).
 // Nothing waits on another block, so the kernel needs no co-scheduling guarantee; its only waits are on its own
 // copies and MMAs, and they are bounded like those of the other tensor-core kernels.
 // Slicing is the same as everywhere else in the library: the first K' filters and C' channels of the stored rows,
@@ -37,6 +42,7 @@ constexpr int PQ_RING_BYTES = 144 * 1024;    // operand ring: 3 stages of pixel 
 constexpr int PQ_LAG = 2;                    // copies run this many stages ahead of the MMAs
 constexpr int PQ_VEC = 1280;                 // longest fp32 vector held in shared memory (the head's width)
 constexpr int PQ_ACC_COLS = 256;             // tensor-memory columns of one accumulator buffer
+constexpr int PQ_HELD_MAX = 56 * 1024;       // largest weight buffer (dynamic shared memory beyond the ring)
 constexpr unsigned long long PQ_WAIT_NS = 2000000000ull;
 
 // Completed phases of the block's barriers since the kernel started (the same in every thread; only ever
@@ -162,7 +168,7 @@ __device__ __forceinline__ bool pw_epilogue(const PqOp &op, const PwShape &s, co
 }
 // Returns false when a wait ran out (the caller leaves at its next block barrier).
 __device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, const bf16 *res, bf16 *y, uint8_t *ring, float *bn,
-                                             uint64_t *free_bar, uint64_t *acc_bar, uint32_t tmem_base, PipeState &ps,
+                                             uint32_t held_u32, uint64_t *free_bar, uint64_t *acc_bar, uint32_t tmem_base, PipeState &ps,
                                              volatile int *abort_flag) {
     const int tid = threadIdx.x;
     const PwShape s = pw_shape(op);
@@ -178,6 +184,14 @@ __device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, cons
     // swizzle term row % 8 is then the same for all of them)
     const int c16 = tid & 7, r0 = tid >> 3;
     const uint32_t piece = (uint32_t)((c16 ^ (r0 & 7)) << 4);
+    // Weight buffer: of this layer's box the query can use the first hK filters (a multiple of 16) in every channel
+    // chunk whose channels - as far as the query takes them - lie inside the box; those need no copy and are
+    // multiplied in place, the tile's other filters come through the ring and get an MMA of their own.
+    const int hK = (held_u32 != 0u && op.cache_off >= 0 && s.n_tiles == 1) ? (min(op.cache_rows, s.K) & ~15) : 0;
+    const uint32_t box_u32 = held_u32 + (uint32_t)(op.cache_off < 0 ? 0 : op.cache_off);
+    const uint32_t idesc_h = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(hK >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+    const uint32_t idesc_r = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((s.BN - hK) >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+    auto chunk_held = [&](int ch) { return hK > 0 && min(s.C, (ch + 1) * 64) <= op.ld2; };
 
     bool ok = true;
     int p_chunk = 0, p_mt = 0, p_nt = 0, p_stage = 0;  // next iteration to copy
@@ -196,8 +210,18 @@ __device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, cons
                 const uint32_t sa = ring_u32 + (uint32_t)(c_stage * s.stage_bytes), sb = sa + A_STAGE_BYTES;
                 const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
                 const int ksteps = (min(64, s.C - c_chunk * 64) + 15) >> 4;
-                for (int q = 0; q < ksteps; q++)
-                    umma_bf16(tmem_base + buf * PQ_ACC_COLS, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), idesc, (c_chunk > 0 || q > 0) ? 1u : 0u);
+                if (chunk_held(c_chunk)) {
+                    const uint64_t dh = smem_desc_sw128(box_u32 + (uint32_t)(c_chunk * op.cache_rows * 128));
+                    const uint64_t dr = smem_desc_sw128(sb + (uint32_t)(hK * 128));
+                    for (int q = 0; q < ksteps; q++) {
+                        umma_bf16(tmem_base + buf * PQ_ACC_COLS, da + (uint64_t)(2 * q), dh + (uint64_t)(2 * q), idesc_h, (c_chunk > 0 || q > 0) ? 1u : 0u);
+                        if (s.BN > hK)
+                            umma_bf16(tmem_base + buf * PQ_ACC_COLS + (uint32_t)hK, da + (uint64_t)(2 * q), dr + (uint64_t)(2 * q), idesc_r, (c_chunk > 0 || q > 0) ? 1u : 0u);
+                    }
+                } else {
+                    for (int q = 0; q < ksteps; q++)
+                        umma_bf16(tmem_base + buf * PQ_ACC_COLS, da + (uint64_t)(2 * q), db + (uint64_t)(2 * q), idesc, (c_chunk > 0 || q > 0) ? 1u : 0u);
+                }
                 umma_commit(&free_bar[c_stage]);
                 if (c_chunk == s.cchunks - 1) umma_commit(&acc_bar[buf]);
             }
@@ -229,7 +253,7 @@ __device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, cons
                 const bool v = cvalid && m < s.M;
                 cp16_cg(sa + (uint32_t)(row * 128) + piece, v ? x + (size_t)m * s.C + c0 : x, v);
             }
-            for (int row = r0; row < s.BN; row += PQ_ROWS) {
+            for (int row = r0 + (chunk_held(p_chunk) ? hK : 0); row < s.BN; row += PQ_ROWS) {
                 const int f = p_nt * s.BN + row;
                 const bool v = cvalid && f < s.K;
                 cp16_ca(sb + (uint32_t)(row * 128) + piece, v ? w + (size_t)f * op.ld + c0 : w, v);
@@ -256,6 +280,7 @@ template <int K, int ST>
 __device__ __noinline__ void pq_depthwise(const PqOp &op, const bf16 *x, bf16 *y) {
     constexpr int TW = (ST == 2 && K > 3) ? 2 : 4;  // (the wide stride-2 windows would not fit the register budget of 512 threads)
     constexpr int NCOL = (TW - 1) * ST + K, P = (K - 1) / 2;
+    constexpr int RU = K;  // filter rows unrolled together
     const int Cn = op.K, groups = Cn >> 3, wblocks = (op.Wo + TW - 1) / TW;
     const int per_row = groups * wblocks, total = per_row * op.Ho;
     const int o = (op.R - K) / 2;
@@ -269,7 +294,7 @@ __device__ __noinline__ void pq_depthwise(const PqOp &op, const bf16 *x, bf16 *y
         for (int t = 0; t < TW; t++)
 #pragma unroll
             for (int j = 0; j < 4; j++) acc[t][j] = make_float2(0.f, 0.f);
-#pragma unroll
+#pragma unroll RU
         for (int r = 0; r < K; r++) {
             const int hi = ho * ST + r - P;
             if (hi < 0 || hi >= op.H) continue;
@@ -466,6 +491,25 @@ __global__ void __launch_bounds__(PQ_THREADS, PQ_BLOCKS_PER_SM) subnet_kernel(co
     ps.use[0] = ps.use[1] = ps.use[2] = ps.use[3] = 0u; ps.acc[0] = ps.acc[1] = 0u; ps.tiles = 0u;
     uint8_t *slot = p.scratch + (size_t)blockIdx.x * p.slot_bytes;
     bool ok = true;
+    // the weight buffer: behind the ring, filled once
+    const uint32_t held_u32 = p.n_held > 0 ? smem_u32(ring + PQ_RING_BYTES) : 0u;
+    if (p.n_held > 0) {
+        const int c16 = tid & 7, r0 = tid >> 3;
+        const uint32_t piece = (uint32_t)((c16 ^ (r0 & 7)) << 4);
+        for (int e = 0; e < p.n_held; e++) {
+            const PqHeld h = p.held[e];
+            const bf16 *hw = static_cast<const bf16 *>(h.w);
+            for (int ch = 0; ch < h.chunks; ch++) {
+                const int c0 = ch * 64 + c16 * 8;
+                const uint32_t dst = held_u32 + h.off + (uint32_t)(ch * h.rows * 128);
+                for (int row = r0; row < h.rows; row += PQ_ROWS) cp16_cg(dst + (uint32_t)(row * 128) + piece, c0 < h.C ? hw + (size_t)row * h.ld + c0 : hw, c0 < h.C);
+            }
+        }
+        cp_commit();
+        cp_wait<0>();
+        fence_async_smem();
+        __syncthreads();
+    }
 
     for (;;) {
         if (tid == 0) next_s = atomicAdd(p.counter, 1);
@@ -486,7 +530,7 @@ __global__ void __launch_bounds__(PQ_THREADS, PQ_BLOCKS_PER_SM) subnet_kernel(co
             const bf16 *res = op.res < 0 ? nullptr : reinterpret_cast<const bf16 *>(slot + (size_t)op.res * p.act_bytes);
             switch (op.type) {
             case PQ_STEM: pq_stem(op, x, y, reinterpret_cast<float *>(ring)); break;
-            case PQ_PW: ok = pq_pointwise(op, x, res, y, ring, bn_s, free_bar, acc_bar, tmem_base, ps, abort_flag) && ok; break;
+            case PQ_PW: ok = pq_pointwise(op, x, res, y, ring, bn_s, held_u32, free_bar, acc_bar, tmem_base, ps, abort_flag) && ok; break;
             case PQ_DW:
                 if (op.stride == 1) {
                     if (op.k == 3) pq_depthwise<3, 1>(op, x, y);
@@ -525,16 +569,18 @@ __global__ void __launch_bounds__(PQ_THREADS, PQ_BLOCKS_PER_SM) subnet_kernel(co
 }  // namespace
 
 size_t subnet_kernel_smem() { return (size_t)PQ_RING_BYTES + 1024; }
+size_t subnet_kernel_held_max() { return (size_t)PQ_HELD_MAX; }
 int subnet_kernel_blocks_per_sm() { return PQ_BLOCKS_PER_SM; }
 
 cudaError_t subnet_kernel_init(int device) {
     (void)device;
-    return cudaFuncSetAttribute(subnet_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)subnet_kernel_smem());
+    return cudaFuncSetAttribute(subnet_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(subnet_kernel_smem() + PQ_HELD_MAX));
 }
 
 cudaError_t subnet_kernel_launch(const PqParams &p, int blocks, cudaStream_t st) {
     if (blocks <= 0) return cudaSuccess;
-    subnet_kernel<<<blocks, PQ_THREADS, subnet_kernel_smem(), st>>>(p);
+    if (p.held_bytes > (unsigned)PQ_HELD_MAX || (p.held_bytes & 1023u)) return cudaErrorInvalidValue;
+    subnet_kernel<<<blocks, PQ_THREADS, subnet_kernel_smem() + (p.n_held > 0 ? p.held_bytes : 0u), st>>>(p);
     return cudaGetLastError();
 }
 

@@ -17,11 +17,11 @@ pytestmark = pytest.mark.gpu
 TOL_BF16 = 2e-2
 
 
-def _run(gnet, cfgs, d_in, res, host=False, **kw):
+def _run(gnet, cfgs, d_in, res, host=False, cache=1, window_q=4):
     n = len(cfgs)
     stream = torch.cuda.Stream()
-    opts = sgs.StreamOpts(cache_enabled=1, window_q=4, cache_budget_bytes=0, use_graphs=0, record_latency=0,
-                          concurrency=1, wave=0, policy=0, persistent=1, **kw)
+    opts = sgs.StreamOpts(cache_enabled=cache, window_q=window_q, cache_budget_bytes=0, use_graphs=0, record_latency=0,
+                          concurrency=1, wave=0, policy=0, persistent=1)
     if host:
         h_out = np.zeros((n, 1000), dtype=np.float32)
         h_in = d_in.cpu().view(torch.int16).numpy()
@@ -77,9 +77,36 @@ def test_persistent_stream_many_queries_per_block_equals_the_wave_path():
     for t in (0, 147, 148, 313, 399):
         ref = onet.forward(cfgs[t], xs[t], oracle.BF16_STORE)
         assert gu.rel_err(got[t:t + 1], ref) <= TOL_BF16, t
-    # the accounting follows the stream order whatever the execution mode
     assert st.useful_flops == wst.useful_flops and st.weight_bytes == wst.weight_bytes
-    assert st.hit_ratio == wst.hit_ratio and st.hbm_weight_bytes == wst.hbm_weight_bytes
+
+
+def test_weight_buffer_in_shared_memory_changes_no_bit():
+    # With the cache on, every block keeps the chosen SubGraph's first pointwise layers in shared memory and multiplies
+    # them in place; filters and channels of a query beyond the box still come through the ring.  The arithmetic of an
+    # output column does not depend on where its filter came from, so logits are bit-identical with the buffer off,
+    # small (a box that ends inside a layer's neighbours) and at its largest; the accounting is against what is held.
+    _, _, gnet = gu.nets(wl.MBV3, True)
+    n, res = 200, 96
+    cfgs = wl.markov_stream(n, seed=12, family=wl.MBV3)
+    d_in = gu.to_device(wl.make_inputs(n, 1, res, seed=13, bf16=True).reshape(n, res, res, 3), True)
+    off, st_off = _run(gnet, cfgs, d_in, res, cache=0)
+    assert st_off.hit_ratio == 0 and st_off.hbm_weight_bytes == st_off.weight_bytes
+    try:
+        for kb in (8, 40, 56):
+            gnet.set_option("persistent_held_kb", kb)
+            for q in (1, 4):
+                on, st_on = _run(gnet, cfgs, d_in, res, cache=1, window_q=q)
+                np.testing.assert_array_equal(on, off)
+                assert 0 < st_on.hit_ratio < 1 and st_on.hbm_weight_bytes < st_on.weight_bytes
+                assert st_on.cache_updates == 1
+        gnet.set_option("persistent_held_kb", 0)
+        none, st_none = _run(gnet, cfgs, d_in, res, cache=1)
+        np.testing.assert_array_equal(none, off)
+        assert st_none.hbm_weight_bytes == st_none.weight_bytes
+        with pytest.raises(sgs.SgsError):
+            gnet.set_option("persistent_held_kb", 4096)
+    finally:
+        gnet.set_option("persistent_held_kb", 16)
 
 
 def test_persistent_stream_full_resolution_sampled():
