@@ -182,10 +182,21 @@ def apply_options(net):
     return net
 
 
-def measure_mbv3(sgs, torch, stream, queries=1000, wave=32, concurrency=4, cache=1, window=4, profile=False):
-    """The MobileNetV3-shaped stream (1000 queries, batch 1, 224x224, configs uniform seed 3)."""
+def measure_mbv3(sgs, torch, stream, queries=1000, wave=32, concurrency=4, cache=1, window=4, profile=False, persistent_only=False):
+    """The MobileNetV3-shaped stream (1000 queries, batch 1, 224x224, configs uniform seed 3): layer by layer in waves,
+    and as ONE launch of the persistent SubNet kernel (every SM serves whole queries)."""
     net = apply_options(sgs.SuperNet(wl.MBV3, wl.make_blob(wl.MBV3, seed=0, bf16_weights=True), sgs.SGS_BF16))
     cfgs = wl.uniform_stream(wl.MBV3, queries, seed=3)
+    popt = sgs.StreamOpts(cache_enabled=cache, window_q=window, cache_budget_bytes=0, record_latency=0, persistent=1)
+    for _ in range(2):
+        _stream_pool(net, sgs, torch, cfgs, 1, 224, popt, stream, len(cfgs), wl.MBV3)
+    tp = _stream_pool(net, sgs, torch, cfgs, 1, 224, popt, stream, len(cfgs), wl.MBV3)
+    persistent = {"queries_per_s": tp["q"] / (tp["ms"] * 1e-3), "ms_per_launch": tp["ms"], "kernel_launches": tp["launches"],
+                  "useful_tflops": tp["flops"] / (tp["ms"] * 1e-3) / 1e12, "weight_hit_ratio_on_chip": tp["hit"] / tp["q"],
+                  "execution": "one launch of the persistent SubNet kernel; every SM takes the next query and runs all of its layers"}
+    if persistent_only:
+        net.close()
+        return {"persistent": persistent}
     opts = sgs.StreamOpts(cache_enabled=cache, window_q=window, cache_budget_bytes=0, use_graphs=1, record_latency=1,
                           concurrency=concurrency, wave=wave)
     for _ in range(2):
@@ -193,7 +204,8 @@ def measure_mbv3(sgs, torch, stream, queries=1000, wave=32, concurrency=4, cache
     t = _stream_pool(net, sgs, torch, cfgs, 1, 224, opts, stream, len(cfgs), wl.MBV3)
     out = {"queries_per_s": t["q"] / (t["ms"] * 1e-3), "p50_ms": float(np.median(t["p50"])), "gflop_per_query": t["flops"] / t["q"] / 1e9,
            "kernel_launches_per_query": t["launches"] / t["q"],
-           "execution": f"waves of {wave}, {concurrency} in flight" if wave > 0 else f"one stream per query, {concurrency} in flight"}
+           "execution": f"waves of {wave}, {concurrency} in flight" if wave > 0 else f"one stream per query, {concurrency} in flight",
+           "persistent": persistent}
     if profile:
         net.set_option("profile", 2)
         popts = sgs.StreamOpts(cache_enabled=cache, window_q=window, cache_budget_bytes=0, use_graphs=0, record_latency=0, wave=wave)
@@ -367,7 +379,8 @@ def run_suite(args):
                     "config": {"workload": f"ResNet-50-shaped SuperNet, {n_sub} SubNets x ({n_cand} candidate SubGraphs + empty cache), batch {batch}, 224x224; one query at a time, 256 MB overwritten before every timed run, median of 9",
                                "scheduler": f"Algorithm 1 with Q = {args.window} on 100000 synthetic (policy, A_t, L_t) queries (seed 8); step_ns includes the caching decision every Q queries"}})
     elif args.suite == "mbv3":
-        r = measure_mbv3(sgs, torch, stream, args.queries, args.wave, args.concurrency, args.cache, args.window, profile=True)
+        r = measure_mbv3(sgs, torch, stream, args.queries, args.wave, args.concurrency, args.cache, args.window, profile=not args.persistent,
+                         persistent_only=args.persistent)
         out.update({"metric": METRIC, "unit": UNIT, "value": r["queries_per_s"], **r,
                     "config": {"workload": "MobileNetV3-shaped SuperNet, 1000-query stream at batch 1, 224x224, configs uniform (seed 3)",
                                "execution": r["execution"]}})
@@ -421,6 +434,7 @@ def main():
     ap.add_argument("--res", type=int, default=0, help="sweep suite: only this resolution (profiling a single launch shape)")
     ap.add_argument("--mechanism", type=int, default=0, help="sgs-probe: 0 per-tile L2 hints, 1 access-policy window per launch, 2 both")
     ap.add_argument("--budget-mb", type=int, default=0, help="sgs-probe: cache budget in MiB (0 = device maximum)")
+    ap.add_argument("--persistent", action="store_true", help="mbv3 suite: only the persistent SubNet kernel (one launch per pass over the queries)")
     ap.add_argument("--family", default="resnet", choices=["resnet", "mbv3"], help="SuperNet of the sched suite")
     ap.add_argument("--suite", default="stream", choices=["stream", "sweep", "sgs", "sgs-probe", "mbv3", "sched", "table", "dw"],
                     help="stream = the default benchmark line; the others measure one more configuration each")

@@ -280,7 +280,7 @@ template <int K, int ST>
 __device__ __noinline__ void pq_depthwise(const PqOp &op, const bf16 *x, bf16 *y) {
     constexpr int TW = (ST == 2 && K > 3) ? 2 : 4;  // (the wide stride-2 windows would not fit the register budget of 512 threads)
     constexpr int NCOL = (TW - 1) * ST + K, P = (K - 1) / 2;
-    constexpr int RU = K;  // filter rows unrolled together
+    constexpr int RU = K == 7 ? 1 : K;  // filter rows unrolled together (all 7 rows of the widest filter at once would spill)
     const int Cn = op.K, groups = Cn >> 3, wblocks = (op.Wo + TW - 1) / TW;
     const int per_row = groups * wblocks, total = per_row * op.Ho;
     const int o = (op.R - K) / 2;
