@@ -11,10 +11,7 @@
 #include <map>
 #include <chrono>
 #include <nvtx3/nvToolsExt.h>
-#include <condition_variable>
-#include <functional>
 #include <mutex>
-#include <thread>
 
 using namespace sgs;
 
@@ -726,72 +723,6 @@ struct LayerRange {
     LayerRange(const LayerRange &) = delete;
     LayerRange &operator=(const LayerRange &) = delete;
 };
-
-// A few host threads for work that is independent per wave member (planning a never-seen SubNet is ~55 convolutions
-// x 2 - 5 tensor maps encoded by the driver, 60 - 70 us on one thread).  parallel_for runs fn(0 .. n-1) on the calling
-// thread and the workers and returns when all are done.
-class HostPool {
-public:
-    explicit HostPool(int workers) {
-        for (int i = 0; i < workers; i++) threads_.emplace_back([this] { work(); });
-    }
-    ~HostPool() {
-        { std::lock_guard<std::mutex> lk(mu_); stop_ = true; }
-        cv_.notify_all();
-        for (auto &t : threads_) t.join();
-    }
-    void parallel_for(int n, const std::function<void(int)> &fn) {
-        if (n <= 0) return;
-        {
-            std::lock_guard<std::mutex> lk(mu_);
-            fn_ = &fn; n_ = n; next_ = 0; pending_ = n; ++epoch_;
-        }
-        cv_.notify_all();
-        run();
-        std::unique_lock<std::mutex> lk(mu_);
-        done_.wait(lk, [this] { return pending_ == 0; });
-        fn_ = nullptr;
-    }
-private:
-    void run() {
-        for (;;) {
-            int i;
-            const std::function<void(int)> *fn;
-            {
-                std::lock_guard<std::mutex> lk(mu_);
-                if (!fn_ || next_ >= n_) return;
-                i = next_++;
-                fn = fn_;
-            }
-            (*fn)(i);
-            std::lock_guard<std::mutex> lk(mu_);
-            if (--pending_ == 0) done_.notify_all();
-        }
-    }
-    void work() {
-        unsigned long long seen = 0;
-        for (;;) {
-            {
-                std::unique_lock<std::mutex> lk(mu_);
-                cv_.wait(lk, [&] { return stop_ || epoch_ != seen; });
-                if (stop_) return;
-                seen = epoch_;
-            }
-            run();
-        }
-    }
-    std::vector<std::thread> threads_;
-    std::mutex mu_;
-    std::condition_variable cv_, done_;
-    const std::function<void(int)> *fn_ = nullptr;
-    int n_ = 0, next_ = 0, pending_ = 0;
-    unsigned long long epoch_ = 0;
-    bool stop_ = false;
-};
-HostPool &host_pool() {
-    static HostPool pool((int)std::min(7u, std::max(1u, std::thread::hardware_concurrency()) - 1u));
-    return pool;
-}
 
 // Key of an op that is the same for every SubNet: its type and the stored layer it uses; ops without
 // a layer (pools, the SE scale) are anchored to the next op that has one.
@@ -1536,25 +1467,10 @@ static sgs_status_t wave_impl(sgs_supernet_t *net, int n_queries, const sgs_subn
             rc = get_plan(net, &cfgs[q0 + m], batch, res, ci * G + m, &plans[m]);
             if (rc == SGS_OK) rc = ensure_workspace(net, plans[m]->act_elems, batch);
         }
-        {
-            // members whose plan is new: tensor maps and tile choices, prepared on a few host threads at once
-            std::vector<int> fresh;
-            for (int m = 0; m < members; m++)
-                if (!plans[m]->prepared) fresh.push_back(m);
-            if (fresh.size() == 1) {
-                rc = choose_impls(net, plans[fresh[0]]);
-            } else if (!fresh.empty()) {
-                std::vector<sgs_status_t> sts(fresh.size(), SGS_OK);
-                std::vector<size_t> need(fresh.size(), 0);
-                std::vector<std::string> errs(fresh.size());
-                // (the driver's tensor-map encoder wants the device's context current on the calling thread)
-                host_pool().parallel_for((int)fresh.size(), [&](int i) { if (cudaSetDevice(net->device) != cudaSuccess) { sts[(size_t)i] = SGS_ECUDA; errs[(size_t)i] = "cudaSetDevice on a planning thread"; return; } sts[(size_t)i] = prepare_impls(net, plans[fresh[(size_t)i]], &need[(size_t)i], &errs[(size_t)i]); });
-                for (size_t i = 0; i < fresh.size() && rc == SGS_OK; i++) {
-                    if (sts[i] != SGS_OK) rc = fail(net, sts[i], errs[i]);
-                    else if ((rc = grow_splitk_scratch(net, need[i])) == SGS_OK) plans[fresh[i]]->prepared = true;
-                }
-            }
-        }
+        // members whose plan is new: tensor maps and tile choices.  (Preparing them on several host threads at once was
+        // measured slower, 102 us against 67 us per never-seen config: the driver's tensor-map encoder serialises.)
+        for (int m = 0; m < members && rc == SGS_OK; m++)
+            if (!plans[m]->prepared) rc = choose_impls(net, plans[m]);
         if (rc != SGS_OK) break;
         net->host_us_query += tick(tp);
         sgs_supernet::WaveCtx &cx = net->waves[ci];  // (taken after ensure_*: the vector does not move later)

@@ -274,7 +274,10 @@ __device__ __forceinline__ bool pq_pointwise(const PqOp &op, const bf16 *x, cons
 // ---------------------------------------------------------------------------------------------
 // Depthwise convolution: a thread owns 8 channels of 4 (2) neighbouring output pixels of one output row and walks
 // the filter rows; per filter row it loads the input columns once and uses each for every tap it belongs to.
-// (Plain loads: the input was written by this block a moment ago.)
+// (Plain loads: the input was written by this block a moment ago.  Measured alternatives: the layer's filters
+// converted to fp32 once and read from shared memory, two 16-byte reads per tap instead of one global load and its
+// unpacking: 41k queries/s against 44k; channel blocks of 64 outermost so that the rows a block needs again stay in
+// L1: slower as well.)
 // ---------------------------------------------------------------------------------------------
 template <int K, int ST>
 __device__ __noinline__ void pq_depthwise(const PqOp &op, const bf16 *x, bf16 *y) {
