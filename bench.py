@@ -381,9 +381,10 @@ def run_suite(args):
     elif args.suite == "mbv3":
         r = measure_mbv3(sgs, torch, stream, args.queries, args.wave, args.concurrency, args.cache, args.window, profile=not args.persistent,
                          persistent_only=args.persistent)
-        out.update({"metric": METRIC, "unit": UNIT, "value": r["queries_per_s"], **r,
-                    "config": {"workload": "MobileNetV3-shaped SuperNet, 1000-query stream at batch 1, 224x224, configs uniform (seed 3)",
-                               "execution": r["execution"]}})
+        head = r["persistent"] if args.persistent else r
+        out.update({"metric": METRIC, "unit": UNIT, "value": head["queries_per_s"], **r,
+                    "config": {"workload": f"MobileNetV3-shaped SuperNet, {args.queries}-query stream at batch 1, 224x224, configs uniform (seed 3)",
+                               "execution": head["execution"]}})
     elif args.suite == "dw":
         fma = sgs.measure_fma_peak(stream.cuda_stream)
         rows = measure_depthwise(sgs, peaks, fma)
