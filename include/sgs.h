@@ -377,7 +377,8 @@ sgs_status_t sgs_conv2d_sliced_static(const sgs_conv_desc_t *desc, const void *d
  * bias[f] ~ shift_f / sy.
  *   d_x    [N][H][W][C] bytes (unsigned, or signed if x_signed)     d_y, d_res  [N][Ho][Wo][K] bytes
  *   d_w    stored weights [Kmax][R][R][Cmax] signed bytes            d_mult, d_shift, d_bias  [>= K] int32
- * Limits of this entry point: C and Cmax multiples of 16, K a multiple of 8, 16-byte aligned pointers, stride-2
+ * Limits of this entry point: pixels of x in multiples of 16 bytes (C a multiple of 16, or of 8 with ldx), Cmax a
+ * multiple of 16, K a multiple of 8, 16-byte aligned pointers, stride-2
  * inputs of even size, 0 <= shift[f] <= 31, and zx == 0 (an input zero point other than 0 would need the sum of the
  * sliced weights under every window position, which changes with the slice and at image borders; post-ReLU tensors
  * and symmetric signed tensors have zx = 0).  Other values: SGS_EUNSUPPORTED.  Asynchronous on `cuda_stream`.
@@ -390,6 +391,8 @@ typedef struct {
     int x_signed, y_signed, res_signed; /* 0: bytes are 0..255, 1: -128..127 */
     int zx, zy, zr;          /* zero points of x, y, res */
     int res_mult, res_shift; /* residual rescaling (ignored without d_res) */
+    int ldx, ldy;            /* bytes per pixel of x, and of y and res; 0 = dense (C resp. K).  Padded pixels: multiples of 16 with
+                                ZEROS beyond the slice in x; the layer writes the zeros of y (ldy - K < 16) */
 } sgs_conv_i8_desc_t;
 sgs_status_t sgs_conv2d_sliced_i8(const sgs_conv_i8_desc_t *desc, const void *d_x, const void *d_w, const int32_t *d_mult,
                                   const int32_t *d_shift, const int32_t *d_bias, const void *d_res, void *d_y, void *cuda_stream);

@@ -38,7 +38,7 @@ class ConvDesc(ctypes.Structure):
 
 class ConvI8Desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("N", "H", "W", "C", "K", "Kmax", "Cmax", "R", "k", "stride", "relu", "x_signed", "y_signed",
-                                             "res_signed", "zx", "zy", "zr", "res_mult", "res_shift")]
+                                             "res_signed", "zx", "zy", "zr", "res_mult", "res_shift", "ldx", "ldy")]
 
 
 SGS_AUX_MAXPOOL, SGS_AUX_AVGPOOL, SGS_AUX_LINEAR, SGS_AUX_SE_GATE, SGS_AUX_SE_SCALE = range(5)

@@ -2684,6 +2684,8 @@ sgs_status_t sgs_conv2d_sliced_i8(const sgs_conv_i8_desc_t *d, const void *d_x, 
     a.Ho = (d->H + 2 * p - d->k) / d->stride + 1;
     a.Wo = (d->W + 2 * p - d->k) / d->stride + 1;
     a.i8 = 1;
+    if (d->ldx < 0 || d->ldy < 0 || (d->ldx && d->ldx < d->C) || (d->ldy && d->ldy < d->K)) return SGS_EINVAL;
+    a.ldx = d->ldx; a.ldy = d->ldy;
     a.q_mult = d_mult; a.q_shift = d_shift; a.q_bias = d_bias;
     a.q_zy = d->zy; a.q_zr = d->zr; a.q_res_mult = d->res_mult; a.q_res_shift = d->res_shift;
     a.q_flags = (d->x_signed ? 1 : 0) | (d->y_signed ? 2 : 0) | (d->res_signed ? 4 : 0) | (d->relu ? 8 : 0);

@@ -220,7 +220,7 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
                         for (int g = 0; g < 4; g++) {
                             const int c = j0 + 8 * g;
                             if (c < ncols) {
-                                const size_t oi = (size_t)m * p.K + f0 + c;
+                                const size_t oi = (size_t)m * p.q_ldy + f0 + c;
                                 uint2 rraw = make_uint2(0u, 0u);
                                 if (res8) rraw = *reinterpret_cast<const uint2 *>(res8 + oi);
                                 uint2 outw = make_uint2(0u, 0u);
@@ -243,6 +243,8 @@ __global__ void __launch_bounds__(192, 1) conv_tc_kernel(const __grid_constant__
                         }
                     }
                 }
+                // a padded pixel (16-byte multiples for the next layer's copies): the 8 bytes beyond the last filter are zeros
+                if (m >= 0 && f0 + ncols == p.K && p.q_ldy > p.K) *reinterpret_cast<uint2 *>(y8 + (size_t)m * p.q_ldy + p.K) = make_uint2(0u, 0u);
             }
         } else if (p.splits == 1) {
             // straight from tensor memory to global memory: each thread finishes its own pixel row,
@@ -517,7 +519,8 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
     auto no = [&](const char *msg) { if (why) *why = msg; return std::shared_ptr<TcConvPlan>(); };
     if (!encode_fn()) return no("cuTensorMapEncodeTiled unavailable");
     if (a.C % 8 || a.K % 8 || a.Cmax % 8) return no("channel counts must be multiples of 8");
-    if (a.i8 && (a.C % 16 || a.Cmax % 16 || a.throughput || a.ldx || a.ldy || a.win)) return no("8-bit layers: channels in multiples of 16, single launches");
+    if (a.i8 && ((a.ldx ? a.ldx : a.C) % 16 || a.C % 8 || a.Cmax % 16 || a.throughput || a.win || (a.ldy && (a.ldy % 16 || a.ldy < a.K || a.ldy - a.K >= 16)) || (!a.ldy && a.K % 8)))
+        return no("8-bit layers: pixels in multiples of 16 bytes, single launches");
     if (a.C < 8 || a.K < 8) return no("too few channels");
     if (a.k % 2 == 0 || a.k > a.R) return no("kernel size");
     if (a.stride != 1 && a.stride != 2) return no("stride");
@@ -526,7 +529,7 @@ std::shared_ptr<TcConvPlan> tc_conv_prepare(const ConvArgs &a, int device, std::
          reinterpret_cast<uintptr_t>(a.res)) & 15)
         return no("pointers must be 16-byte aligned");
     if (device < 0 || device >= 64) return no("device index");
-    if ((a.ldx || a.ldy) && a.throughput != 2) return no("padded pixels are for grouped launches");
+    if ((a.ldx || a.ldy) && a.throughput != 2 && !a.i8) return no("padded pixels are for grouped launches and 8-bit layers");
     if ((a.ldx && (a.ldx < a.C || a.ldx % 8)) || (a.ldy && (a.ldy < a.K || a.ldy % 8))) return no("channel pitch");
 
     auto plan = std::make_shared<TcConvPlan>();
@@ -729,6 +732,7 @@ cudaError_t tc_conv_launch(const TcConvPlan &pl, const ConvArgs &a, cudaStream_t
         if (!a.q_mult || !a.q_shift || !a.q_bias || pl.bn_tile > 128 || prm.splits != 1) return cudaErrorInvalidValue;
         prm.q_mult = a.q_mult; prm.q_shift = a.q_shift; prm.q_bias = a.q_bias;
         prm.q_zy = a.q_zy; prm.q_zr = a.q_zr; prm.q_res_mult = a.q_res_mult; prm.q_res_shift = a.q_res_shift; prm.q_flags = a.q_flags;
+        prm.q_ldy = a.ldy ? a.ldy : a.K;
         e = pl.bn_tile == 64 ? launch_variant<64, 3, true>(run, prm, st) : launch_variant<128, 3, true>(run, prm, st);
         if (launches) *launches = 1;
         return e;

@@ -35,6 +35,7 @@ struct TcParams {
     const int *q_mult, *q_shift, *q_bias;
     int q_zy, q_zr, q_res_mult, q_res_shift;
     int q_flags;             // bit 0: x signed, bit 1: y signed, bit 2: res signed, bit 3: ReLU (max with q_zy)
+    int q_ldy;               // bytes per pixel of y and res (>= K; the bytes beyond K are written as zeros)
 };
 
 namespace {

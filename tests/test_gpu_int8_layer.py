@@ -63,6 +63,42 @@ def test_int8_layer_is_bit_exact(case):
         np.testing.assert_array_equal(dy.cpu().numpy(), ref)
 
 
+# N, H, W, Cmax, C, Kmax, K, R, k, stride, x_signed, relu, y_signed, residual: channel counts that are multiples of 8 only
+PADDED_CASES = [
+    (2, 28, 28, 96, 72, 128, 88, 1, 1, 1, False, True, False, True),      # 72 -> 80 bytes per input pixel, 88 -> 96 per output pixel
+    (1, 14, 14, 368, 328, 368, 328, 3, 3, 1, False, True, False, False),  # 3x3 over padded pixels, last chunk ragged
+    (3, 56, 56, 64, 56, 256, 168, 1, 1, 2, False, False, True, True),     # strided 1x1 (projection shortcut), signed output
+    (1, 30, 30, 32, 24, 64, 40, 3, 3, 2, False, True, False, False),      # stride-2 3x3, 24 -> 32 bytes, K = 40 -> 48
+]
+
+
+@pytest.mark.parametrize("case", PADDED_CASES)
+def test_int8_layer_on_padded_pixels_is_bit_exact(case):
+    # Pixels of 16-byte multiples with zeros beyond the slice (what a network of such layers keeps between them): the
+    # layer reads x at pitch ldx, writes y at pitch ldy with zeros in the padding, reads the residual at pitch ldy.
+    N, H, W, Cmax, C, Kmax, K, R, k, stride, x_signed, relu, y_signed, use_res = case
+    w, x, mult, shift, bias, res, zy, ref = make(case, seed=5)
+    ldx, ldy = (C + 15) // 16 * 16, (K + 15) // 16 * 16
+    xp = np.zeros(x.shape[:3] + (ldx,), dtype=x.dtype); xp[..., :C] = x
+    rp = None
+    if use_res:
+        rp = np.zeros(res.shape[:3] + (ldy,), dtype=res.dtype); rp[..., :K] = res
+    dw = torch.from_numpy(np.ascontiguousarray(w.transpose(0, 2, 3, 1))).cuda()
+    dx = torch.from_numpy(xp).cuda()
+    dm, ds, db = (torch.from_numpy(a).cuda() for a in (mult, shift, bias))
+    dr = torch.from_numpy(rp).cuda() if use_res else None
+    dy = torch.full(ref.shape[:3] + (ldy,), 77, dtype=torch.int8 if y_signed else torch.uint8, device="cuda")
+    desc = sgs.ConvI8Desc(N=N, H=H, W=W, C=C, K=K, Kmax=Kmax, Cmax=Cmax, R=R, k=k, stride=stride, relu=int(relu), x_signed=int(x_signed),
+                          y_signed=int(y_signed), res_signed=0, zx=0, zy=zy, zr=11, res_mult=1932735283, res_shift=1, ldx=ldx, ldy=ldy)
+    sgs.conv2d_sliced_i8(desc, dx.data_ptr(), dw.data_ptr(), dm.data_ptr(), ds.data_ptr(), db.data_ptr(), dr.data_ptr() if use_res else 0,
+                         dy.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert sgs.device_status() == 0
+    got = dy.cpu().numpy()
+    np.testing.assert_array_equal(got[..., :K], ref)
+    assert not got[..., K:].any()
+
+
 def test_int8_layer_refuses_what_it_does_not_take():
     x = torch.zeros((1, 8, 8, 16), dtype=torch.uint8, device="cuda")
     w = torch.zeros((16, 3, 3, 16), dtype=torch.int8, device="cuda")
